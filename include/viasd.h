@@ -1,0 +1,187 @@
+/*
+ * viasd.h -- C ABI of the VIA-SD multi-tier verification step for NVIDIA B200 (sm_100a).
+ *
+ * One decoding cycle of hierarchical speculative verification (Algorithm 1, the body of the
+ * while loop; Algorithm 2, lines "run q' in parallel on prefixes" to "append"; Sec. 3.5 steps 3-4):
+ *   1. every drafted token is routed to one of three tiers by its confidence relative to the mode of
+ *      the gating distribution (App. B, Eq. B.1-B.3): 0 = accept, 1 = slim verifier q', 2 = full
+ *      verifier q;
+ *   2. q' = Pi_z(q), the routed sub-network of q (Sec. 3.4: layers with z_l = 0 are bypassed; embeddings
+ *      and output head are shared), runs on the block against its own KV cache;
+ *   3. q runs on the block against its KV cache;
+ *   4. the longest accepted prefix and the replacement token are resolved on the device (Sec. 3.5 step 4;
+ *      App. A, Eq. A.2-A.3 for the sampling test and the residual distribution);
+ *   5. the emitted tokens are committed to both caches; the rest of the block is discarded.
+ *
+ * Conventions
+ *   - Every tensor argument is a DEVICE pointer owned by the caller unless marked "host".  The library
+ *     allocates no device memory: scratch comes from the caller's workspace.  It keeps the pointers passed
+ *     to viasd_init_model (weights, workspace); they must outlive the handle.
+ *   - All work is enqueued on the caller's stream (a cudaStream_t passed as void*); no call synchronises
+ *     except viasd_init_model and viasd_get_stats.
+ *   - Every function returns 0 (VIASD_OK) or a negative error code; nothing throws, exits or traps.
+ *     Conditions only the device can see (a sequence too long for the cache, a token id outside the
+ *     vocabulary) are clamped to a safe value and recorded in a device status word that
+ *     viasd_get_stats reports.
+ *   - A block has N draft nodes and M = N + 1 rows per sequence: row 0 is the pending token (the last
+ *     emitted token, whose K/V is not cached yet), row n + 1 is draft node n.  The logits of a row are
+ *     the next-token distribution for that row's children.  M <= 64.
+ *   - Matrices are row-major [out, in].  dtype 0 = fp32, 1 = bf16 applies to weights and KV caches;
+ *     norm gains, logits and the residual stream are fp32.
+ */
+#ifndef VIASD_H
+#define VIASD_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    VIASD_OK = 0,
+    VIASD_EINVAL = -1,        /* null or misaligned pointer, shape out of range */
+    VIASD_ECAPACITY = -2,     /* workspace too small, or (device status) len + M > max_ctx */
+    VIASD_ECUDA = -3,         /* a CUDA runtime call failed; see viasd_last_cuda_error() */
+    VIASD_EDEVICE = -4,       /* device status word set: bad token id, bad tree, bounded wait expired */
+    VIASD_EUNSUPPORTED = -5   /* no CUDA device of compute capability 10.x */
+};
+
+typedef struct viasd_model viasd_model; /* opaque */
+
+typedef struct {
+    int n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ff, vocab;
+    int dtype;                 /* 0 fp32, 1 bf16 */
+    float rms_eps;             /* RMSNorm epsilon */
+    float rope_theta;          /* rotary base; pairs (p, p + head_dim/2), angle pos * theta^(-2p/head_dim) */
+    int max_batch, max_ctx;    /* cache geometry */
+    int max_query;             /* largest M the handle will see, <= 64 */
+} viasd_config;
+
+typedef struct {
+    const void *embed;                 /* [vocab, d_model] */
+    const void *lm_head;               /* [vocab, d_model] */
+    const float *final_norm;           /* [d_model] */
+    /* host arrays of n_layers device pointers */
+    const void *const *wq, *const *wk, *const *wv, *const *wo;   /* [H*hd,d] [Hkv*hd,d] [Hkv*hd,d] [d,H*hd] */
+    const void *const *wg, *const *wu, *const *wd;               /* [ff,d] [ff,d] [d,ff] */
+    const float *const *norm1, *const *norm2;                    /* [d] */
+} viasd_weights;
+
+typedef struct {
+    void *k_full, *v_full;     /* [n_layers, max_batch, n_kv_heads, max_ctx, head_dim]; K is stored rotated */
+    void *k_slim, *v_slim;     /* [n_routed, ...] indexed by the routed layer's ordinal */
+    int *len;                  /* [batch] committed length, shared by both caches */
+    int *pending;              /* [batch] last emitted token */
+    int *tokens;               /* [batch, max_ctx] committed token ids, or NULL */
+} viasd_cache;
+
+typedef struct {
+    int batch, n_nodes;                /* B, N */
+    const int *draft_tok;              /* [B, N] */
+    const int *parent;                 /* [N] parent node, -1 = child of the pending token; parents first */
+    const int *prow;                   /* [N] drafter-logit row the node was drafted from */
+    int n_prows;                       /* R */
+    const float *drafter_logits;       /* [B, R, vocab] */
+} viasd_draft;
+
+typedef struct {
+    float log_tau_hi, log_tau_lo;      /* log of the relative-confidence thresholds, log_tau_lo <= log_tau_hi */
+    int conf_source;                   /* 0: drafter confidence; 1: q' confidence at the parent row (Alg. 2) */
+    int mode;                          /* 0 greedy, 1 sampling */
+    float temperature;                 /* sampling only; divides verifier and drafter logits */
+    float alpha, beta;                 /* Eq. A.2 / A.3; 0 and 1 give the lossless rule */
+    float log_acc_rel[3];              /* greedy gate per tier: accept if l[v] - max l >= this; 0 = argmax */
+    int strict_break;                  /* 1: an accepted tier-1 token still ends the block (Alg. 2 as printed) */
+    int emit_bonus;                    /* 1: when the whole path is accepted, add a token from q at the leaf */
+    int policy;                        /* 0: both passes always run (the only policy implemented) */
+    unsigned long long seed, step;     /* counter-based random numbers for sampling mode */
+} viasd_params;
+
+typedef struct {
+    unsigned char *tier;               /* [B, N] */
+    float *conf;                       /* [B, N] log relative confidence d = l[v] - max l */
+    int *n_acc;                        /* [B] kappa: accepted draft nodes */
+    int *path;                         /* [B, N] accepted node ids, first n_acc valid */
+    int *out_tok;                      /* [B, N+1] emitted tokens, first n_emit valid */
+    int *n_emit;                       /* [B] */
+    unsigned char *judge;              /* [B, N] 0 untouched, 1 accepted, 2 rejected, | judging tier << 4 */
+    int *corr_src;                     /* [B] who emitted the last token: 0 nobody, 1 q', 2 q */
+} viasd_result;
+
+typedef struct {
+    unsigned long long steps;          /* verify steps / tier passes since init */
+    unsigned long long tier_count[3];  /* histogram of tiers: empirical region masses of Eq. B.4-B.6 */
+    unsigned long long emitted;        /* tokens emitted by accept passes */
+    unsigned long long accepted;       /* draft nodes accepted */
+    int device_status;                 /* 0 or a VIASD_E* code recorded by a kernel */
+    int need_slim, need_full;          /* last tier pass: any node in tier 1 / tier 2 */
+} viasd_stats;
+
+/* Bytes of workspace viasd_init_model needs for this geometry. */
+size_t viasd_workspace_bytes(const viasd_config *cfg, int n_routed);
+
+/* Build a handle.  route_mask: host, [n_layers], the routing mask z (1 = layer kept by q').
+ * workspace: device, 256-byte aligned, at least viasd_workspace_bytes().  Synchronises the device once
+ * (it fills the rotary table).  Errors: EINVAL, ECAPACITY, ECUDA, EUNSUPPORTED. */
+int viasd_init_model(const viasd_config *cfg, const viasd_weights *w, const unsigned char *route_mask,
+                     void *workspace, size_t workspace_bytes, viasd_model **out);
+
+/* Forward pass of q (all layers) / q' (routed layers) over the block: logits [B, M, vocab] fp32.
+ * K/V of the M rows are written at slots len[b] .. len[b]+M-1 of the model's cache; len is not changed,
+ * so the rows stay invisible until viasd_kv_commit.  (Algorithm 2, parallel block verification.) */
+int viasd_full_forward(viasd_model *m, const viasd_cache *cache, const viasd_draft *draft, float *logits,
+                       void *stream);
+int viasd_slim_forward(viasd_model *m, const viasd_cache *cache, const viasd_draft *draft, float *logits,
+                       void *stream);
+
+/* phase 1: tier routing only (Eq. B.1-B.3) -> result.tier, result.conf.
+ * phase 2: accept / resolve only (reads result.tier) -> n_acc, path, out_tok, n_emit, judge, corr_src.
+ * phase 3: both.  slim_logits / full_logits [B, M, vocab]; phase 1 needs slim_logits only when
+ * conf_source = 1. */
+int viasd_tier_accept(viasd_model *m, const viasd_draft *draft, const viasd_params *params,
+                      const float *slim_logits, const float *full_logits, int phase, viasd_result *result,
+                      void *stream);
+
+/* Commit: move the accepted path's K/V rows to slots len+1.., len += n_emit, pending = last emitted
+ * token, committed ids appended to cache.tokens.  Rejected rows are left beyond len (rollback). */
+int viasd_kv_commit(viasd_model *m, viasd_cache *cache, const viasd_draft *draft, const viasd_result *result,
+                    void *stream);
+
+/* tier -> slim forward -> full forward -> accept -> commit, identical to calling the pieces.
+ * slim_logits / full_logits: caller's buffers [B, M, vocab], filled as a side effect. */
+int viasd_verify_step(viasd_model *m, viasd_cache *cache, const viasd_draft *draft, const viasd_params *params,
+                      float *slim_logits, float *full_logits, viasd_result *result, void *stream);
+
+/* Copies the device counters out; synchronises `stream`. */
+int viasd_get_stats(viasd_model *m, viasd_stats *host_out, void *stream);
+
+void viasd_free_model(viasd_model *m);
+const char *viasd_strerror(int code);
+int viasd_last_cuda_error(void);
+
+/* One projection of the decoder block on its own: y[rows, n] = x[rows, k] * W[n, k]^T (the contraction
+ * every layer of q and q' is made of, Sec. 3.4).  dtype as in viasd_config (x and W share it: fp32, or
+ * bf16 with fp32 accumulation); y is fp32.  scratch: device, scratch_bytes >= viasd_gemm_scratch_bytes(),
+ * used for split-K partial sums.  rows <= 256. */
+size_t viasd_gemm_scratch_bytes(int rows, int n, int k);
+int viasd_gemm(const void *x, const void *w, float *y, int rows, int n, int k, int dtype, void *scratch,
+               size_t scratch_bytes, void *stream);
+
+/* Measurement hooks (the paper has no counterpart; they exist so that a benchmark can attribute time).
+ * viasd_launch_count: kernels launched by this library in this process so far.
+ * viasd_set_timing(on): when on, every launch of the forward / tier / accept / commit path is bracketed by
+ * CUDA events on the caller's stream (a few thousand launches are kept; later ones are dropped).
+ * viasd_get_timing: synchronises `stream`, sums the recorded intervals per kernel class into `out`
+ * (VIASD_T_COUNT entries each) and clears the record. */
+enum { VIASD_T_GEMM = 0, VIASD_T_ATTENTION, VIASD_T_NORM, VIASD_T_ROPE, VIASD_T_EMBED, VIASD_T_TIER_ACCEPT,
+       VIASD_T_COMMIT, VIASD_T_COUNT };
+typedef struct { double ms[VIASD_T_COUNT]; long long launches[VIASD_T_COUNT]; long long dropped; } viasd_timing;
+unsigned long long viasd_launch_count(void);
+int viasd_set_timing(viasd_model *m, int on);
+int viasd_get_timing(viasd_model *m, viasd_timing *out, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VIASD_H */

@@ -58,8 +58,8 @@ def stream_key(seed: int, step: int, b: int, stream: int) -> int:
 
 
 def unit(key: int, idx: int) -> float:
-    """Uniform on (0, 1) with 24 random bits: ((word >> 40) + 0.5) / 2^24."""
-    return ((_mix(key + idx * _GAMMA + 3) >> 40) + 0.5) * 2.0 ** -24
+    """Uniform on (0, 1) with 23 random bits, ((word >> 41) + 0.5) / 2^23: exact in fp32, never 0 or 1."""
+    return ((_mix(key + idx * _GAMMA + 3) >> 41) + 0.5) * 2.0 ** -23
 
 
 def unit_vec(key: int, idx0: int, n: int) -> np.ndarray:
@@ -69,7 +69,7 @@ def unit_vec(key: int, idx0: int, n: int) -> np.ndarray:
         z = (z ^ (z >> np.uint64(30))) * np.uint64(0xBF58476D1CE4E5B9)
         z = (z ^ (z >> np.uint64(27))) * np.uint64(0x94D049BB133111EB)
         z = z ^ (z >> np.uint64(31))
-    return ((z >> np.uint64(40)).astype(np.float64) + 0.5) * 2.0 ** -24
+    return ((z >> np.uint64(41)).astype(np.float64) + 0.5) * 2.0 ** -23
 
 
 STREAM_ACCEPT, STREAM_GUMBEL = 0, 1

@@ -1,0 +1,363 @@
+// C ABI: argument checks, workspace carving, and the sequence of launches that makes up each call.
+#include "common.cuh"
+#include <new>
+#include <string.h>
+
+int g_last_cuda_error = 0;
+unsigned long long g_launch_count = 0;
+
+namespace {
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+size_t elem_size(int dtype) { return dtype == 0 ? 4 : 2; }
+
+struct Carver {
+    char *base; size_t off;
+    template <typename T> T *take(size_t bytes) {
+        off = align_up(off, 256);
+        T *p = base ? reinterpret_cast<T *>(base + off) : nullptr;
+        off += bytes;
+        return p;
+    }
+};
+
+size_t part_bytes_for(const viasd_config &c) {
+    const size_t R = (size_t)c.max_batch * c.max_query;
+    // attention split-KV partials: up to 16 key ranges of (head_dim + 2) floats per (row, head)
+    size_t att = R * c.n_heads * 16 * (size_t)(c.head_dim + 2) * sizeof(float);
+    const size_t cap = (size_t)256 << 20;
+    return att < cap ? att : cap;
+}
+
+// One layout routine serves both the size query (base = null) and the real carve.
+size_t carve(const viasd_config &c, char *base, Workspace *ws) {
+    Carver cv{base, 0};
+    const size_t R = (size_t)c.max_batch * c.max_query, es = elem_size(c.dtype);
+    const size_t qd = (size_t)c.n_heads * c.head_dim, kvd = (size_t)c.n_kv_heads * c.head_dim;
+    Workspace w;
+    w.rope_cos = cv.take<float>((size_t)c.max_ctx * (c.head_dim / 2) * 4);
+    w.rope_sin = cv.take<float>((size_t)c.max_ctx * (c.head_dim / 2) * 4);
+    w.h = cv.take<float>(R * c.d_model * 4);
+    w.a = cv.take<void>(R * c.d_model * es);
+    w.qkv = cv.take<float>(R * (qd + 2 * kvd) * 4);
+    w.q = cv.take<void>(R * qd * es);
+    w.attn = cv.take<void>(R * qd * es);
+    w.act = cv.take<void>(R * c.d_ff * es);
+    w.part_bytes = part_bytes_for(c);
+    w.part = cv.take<float>(w.part_bytes);
+    w.len_eff = cv.take<int>((size_t)c.max_batch * 4);
+    w.row_tok = cv.take<int>(R * 4);
+    w.tree = cv.take<TreeInfo>(sizeof(TreeInfo));
+    w.stats = cv.take<DeviceStats>(sizeof(DeviceStats));
+    w.accept_scratch = cv.take<float>((size_t)c.max_batch * 3 * c.vocab * 4);
+    if (ws) *ws = w;
+    return align_up(cv.off, 256);
+}
+
+// Runs one launcher, bracketed by events when timing is on.
+template <typename F>
+int timed(viasd_model *m, int cls, cudaStream_t st, F &&f) {
+    KernelTimer &t = m->timer;
+    if (!t.on) return f();
+    if (t.n >= KernelTimer::CAP) { ++t.dropped; return f(); }
+    const int i = t.n++;
+    t.cls[i] = cls;
+    CUDA_TRY(cudaEventRecord(t.beg[i], st));
+    int rc = f();
+    CUDA_TRY(cudaEventRecord(t.end[i], st));
+    return rc;
+}
+
+int check_config(const viasd_config *c) {
+    if (!c) return VIASD_EINVAL;
+    if (c->n_layers < 1 || c->n_layers > 512 || c->d_model < 8 || c->n_heads < 1 || c->n_kv_heads < 1) return VIASD_EINVAL;
+    if (c->n_heads % c->n_kv_heads) return VIASD_EINVAL;
+    if (c->head_dim != 64 && c->head_dim != 128) return VIASD_EINVAL;
+    if (c->d_model % 8 || c->d_ff % 8 || c->d_ff < 8 || c->vocab < 2) return VIASD_EINVAL;
+    if (c->dtype != 0 && c->dtype != 1) return VIASD_EINVAL;
+    if (c->max_batch < 1 || c->max_query < 1 || c->max_query > VIASD_MAX_ROWS_PER_SEQ) return VIASD_EINVAL;
+    if (c->max_ctx < c->max_query) return VIASD_EINVAL;
+    if (!(c->rms_eps >= 0.f) || !(c->rope_theta > 0.f)) return VIASD_EINVAL;
+    return VIASD_OK;
+}
+
+int check_draft(const viasd_model *m, const viasd_draft *d) {
+    if (!m || !d) return VIASD_EINVAL;
+    if (d->batch < 1 || d->batch > m->cfg.max_batch) return VIASD_EINVAL;
+    if (d->n_nodes < 0 || d->n_nodes + 1 > m->cfg.max_query) return VIASD_EINVAL;
+    if (!d->draft_tok && d->n_nodes) return VIASD_EINVAL;
+    if (!d->parent && d->n_nodes) return VIASD_EINVAL;
+    return VIASD_OK;
+}
+
+int check_cache(const viasd_cache *c) {
+    if (!c || !c->k_full || !c->v_full || !c->k_slim || !c->v_slim || !c->len || !c->pending) return VIASD_EINVAL;
+    return VIASD_OK;
+}
+
+// One pass of the sub-network made of `layers` (all of them for q, the routed ones for q').
+int forward(viasd_model *m, const viasd_cache *cache, const viasd_draft *d, bool slim, float *logits,
+            cudaStream_t st) {
+    int rc;
+    if ((rc = check_draft(m, d)) || (rc = check_cache(cache))) return rc;
+    if (!logits) return VIASD_EINVAL;
+    const viasd_config &c = m->cfg;
+    const int B = d->batch, M = d->n_nodes + 1, rows = B * M;
+    const int qd = c.n_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
+    void *kc = slim ? cache->k_slim : cache->k_full, *vc = slim ? cache->v_slim : cache->v_full;
+    const int n_run = slim ? m->n_routed : c.n_layers;
+
+    if ((rc = timed(m, VIASD_T_EMBED, st, [&] { return launch_prep(m, cache, d, st); }))) return rc;
+    if ((rc = timed(m, VIASD_T_EMBED, st, [&] { return launch_embed(m, rows, st); }))) return rc;
+    for (int ord = 0; ord < n_run; ++ord) {
+        const int l = slim ? m->routed[ord] : ord;
+        if ((rc = timed(m, VIASD_T_NORM, st, [&] { return launch_rmsnorm(m, m->norm1[l], rows, st); }))) return rc;
+        GemmSegs qkv{{m->wq[l], m->wk[l], m->wv[l]}, {qd, kvd, kvd}, 3};
+        if ((rc = timed(m, VIASD_T_GEMM, st, [&] { return launch_gemm_rowwarp(m->ws.a, qkv, rows, c.d_model, c.dtype,
+                EPI_STORE, m->ws.qkv, nullptr, qd + 2 * kvd, st); }))) return rc;
+        if ((rc = timed(m, VIASD_T_ROPE, st, [&] { return launch_rope_append(m, kc, vc, ord, B, M, st); }))) return rc;
+        if ((rc = timed(m, VIASD_T_ATTENTION, st, [&] { return launch_attention(m, kc, vc, ord, B, M, st); }))) return rc;
+        GemmSegs wo{{m->wo[l], nullptr, nullptr}, {c.d_model, 0, 0}, 1};
+        if ((rc = timed(m, VIASD_T_GEMM, st, [&] { return launch_gemm_rowwarp(m->ws.attn, wo, rows, qd, c.dtype, EPI_ADD,
+                m->ws.h, nullptr, c.d_model, st); }))) return rc;
+        if ((rc = timed(m, VIASD_T_NORM, st, [&] { return launch_rmsnorm(m, m->norm2[l], rows, st); }))) return rc;
+        GemmSegs gu{{m->wg[l], m->wu[l], nullptr}, {c.d_ff, c.d_ff, 0}, 2};
+        if ((rc = timed(m, VIASD_T_GEMM, st, [&] { return launch_gemm_rowwarp(m->ws.a, gu, rows, c.d_model, c.dtype,
+                EPI_SWIGLU, nullptr, m->ws.act, c.d_ff, st); }))) return rc;
+        GemmSegs wd{{m->wd[l], nullptr, nullptr}, {c.d_model, 0, 0}, 1};
+        if ((rc = timed(m, VIASD_T_GEMM, st, [&] { return launch_gemm_rowwarp(m->ws.act, wd, rows, c.d_ff, c.dtype, EPI_ADD,
+                m->ws.h, nullptr, c.d_model, st); }))) return rc;
+    }
+    if ((rc = timed(m, VIASD_T_NORM, st, [&] { return launch_rmsnorm(m, m->final_norm, rows, st); }))) return rc;
+    GemmSegs head{{m->lm_head, nullptr, nullptr}, {c.vocab, 0, 0}, 1};
+    return timed(m, VIASD_T_GEMM, st, [&] { return launch_gemm_rowwarp(m->ws.a, head, rows, c.d_model, c.dtype, EPI_STORE,
+                                                                   logits, nullptr, c.vocab, st); });
+}
+
+int check_params(const viasd_params *p) {
+    if (!p) return VIASD_EINVAL;
+    if (!(p->log_tau_lo <= p->log_tau_hi)) return VIASD_EINVAL;
+    if (p->conf_source != 0 && p->conf_source != 1) return VIASD_EINVAL;
+    if (p->mode != 0 && p->mode != 1) return VIASD_EINVAL;
+    if (p->mode == 1 && !(p->temperature > 0.f)) return VIASD_EINVAL;
+    if (!(p->alpha >= 0.f && p->alpha < 1.f) || !(p->beta > 0.f)) return VIASD_EINVAL;
+    if (p->policy != 0) return VIASD_EINVAL;
+    return VIASD_OK;
+}
+
+int check_result(const viasd_result *r, int phase) {
+    if (!r || !r->tier) return VIASD_EINVAL;
+    if ((phase & 1) && !r->conf) return VIASD_EINVAL;
+    if ((phase & 2) && (!r->n_acc || !r->path || !r->out_tok || !r->n_emit || !r->judge || !r->corr_src))
+        return VIASD_EINVAL;
+    return VIASD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t viasd_workspace_bytes(const viasd_config *cfg, int n_routed) {
+    (void)n_routed;
+    if (check_config(cfg)) return 0;
+    return carve(*cfg, nullptr, nullptr);
+}
+
+int viasd_init_model(const viasd_config *cfg, const viasd_weights *w, const unsigned char *route_mask,
+                     void *workspace, size_t workspace_bytes, viasd_model **out) {
+    int rc = check_config(cfg);
+    if (rc) return rc;
+    if (!w || !route_mask || !workspace || !out) return VIASD_EINVAL;
+    if (((uintptr_t)workspace & 255) != 0) return VIASD_EINVAL;
+    if (!w->embed || !w->lm_head || !w->final_norm || !w->wq || !w->wk || !w->wv || !w->wo || !w->wg || !w->wu ||
+        !w->wd || !w->norm1 || !w->norm2) return VIASD_EINVAL;
+    if (workspace_bytes < carve(*cfg, nullptr, nullptr)) return VIASD_ECAPACITY;
+    int dev = 0;
+    cudaDeviceProp prop;
+    CUDA_TRY(cudaGetDevice(&dev));
+    CUDA_TRY(cudaGetDeviceProperties(&prop, dev));
+    if (prop.major != 10) return VIASD_EUNSUPPORTED;
+
+    viasd_model *m = new (std::nothrow) viasd_model();
+    if (!m) return VIASD_EINVAL;
+    memset(&m->timer, 0, sizeof(m->timer));
+    m->cfg = *cfg;
+    m->sm_count = prop.multiProcessorCount;
+    m->n_routed = 0;
+    for (int l = 0; l < cfg->n_layers; ++l) if (route_mask[l]) m->routed[m->n_routed++] = l;
+    if (m->n_routed == 0) { delete m; return VIASD_EINVAL; }
+    const int L = cfg->n_layers;
+    const void ***arrs[] = {&m->wq, &m->wk, &m->wv, &m->wo, &m->wg, &m->wu, &m->wd};
+    const void *const *srcs[] = {w->wq, w->wk, w->wv, w->wo, w->wg, w->wu, w->wd};
+    for (int i = 0; i < 7; ++i) {
+        *arrs[i] = new const void *[L];
+        for (int l = 0; l < L; ++l) {
+            if (!srcs[i][l] || ((uintptr_t)srcs[i][l] & 15)) { viasd_free_model(m); return VIASD_EINVAL; }
+            (*arrs[i])[l] = srcs[i][l];
+        }
+    }
+    m->norm1 = new const float *[L];
+    m->norm2 = new const float *[L];
+    for (int l = 0; l < L; ++l) {
+        if (!w->norm1[l] || !w->norm2[l]) { viasd_free_model(m); return VIASD_EINVAL; }
+        m->norm1[l] = w->norm1[l];
+        m->norm2[l] = w->norm2[l];
+    }
+    m->embed = w->embed; m->lm_head = w->lm_head; m->final_norm = w->final_norm;
+    carve(*cfg, (char *)workspace, &m->ws);
+    cudaError_t e = cudaMemset(m->ws.stats, 0, sizeof(DeviceStats));
+    if (e == cudaSuccess) { rc = launch_rope_table(m, 0); if (rc == VIASD_OK) e = cudaDeviceSynchronize(); }
+    if (e != cudaSuccess) { g_last_cuda_error = (int)e; rc = VIASD_ECUDA; }
+    if (rc) { viasd_free_model(m); return rc; }
+    *out = m;
+    return VIASD_OK;
+}
+
+void viasd_free_model(viasd_model *m) {
+    if (!m) return;
+    const void ***arrs[] = {&m->wq, &m->wk, &m->wv, &m->wo, &m->wg, &m->wu, &m->wd};
+    for (int i = 0; i < 7; ++i) delete[] *arrs[i];
+    delete[] m->norm1;
+    delete[] m->norm2;
+    for (int i = 0; i < m->timer.created; ++i) { cudaEventDestroy(m->timer.beg[i]); cudaEventDestroy(m->timer.end[i]); }
+    delete[] m->timer.beg;
+    delete[] m->timer.end;
+    delete[] m->timer.cls;
+    delete m;
+}
+
+int viasd_full_forward(viasd_model *m, const viasd_cache *cache, const viasd_draft *draft, float *logits, void *stream) {
+    return forward(m, cache, draft, false, logits, (cudaStream_t)stream);
+}
+
+int viasd_slim_forward(viasd_model *m, const viasd_cache *cache, const viasd_draft *draft, float *logits, void *stream) {
+    return forward(m, cache, draft, true, logits, (cudaStream_t)stream);
+}
+
+int viasd_tier_accept(viasd_model *m, const viasd_draft *draft, const viasd_params *params, const float *slim_logits,
+                      const float *full_logits, int phase, viasd_result *result, void *stream) {
+    int rc;
+    if ((rc = check_draft(m, draft)) || (rc = check_params(params))) return rc;
+    if (phase < 1 || phase > 3) return VIASD_EINVAL;
+    if ((rc = check_result(result, phase))) return rc;
+    if (draft->n_nodes < 1 || !draft->prow || !draft->drafter_logits || draft->n_prows < 1) return VIASD_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (phase & 1) {
+        if ((rc = timed(m, VIASD_T_TIER_ACCEPT, st, [&] { return launch_tier(m, draft, params, slim_logits, result, st); })))
+            return rc;
+    }
+    if (phase & 2) {
+        if (!slim_logits || !full_logits) return VIASD_EINVAL;
+        if ((rc = timed(m, VIASD_T_TIER_ACCEPT, st, [&] { return launch_accept(m, draft, params, slim_logits, full_logits,
+                                                                          result, st); }))) return rc;
+    }
+    return VIASD_OK;
+}
+
+int viasd_kv_commit(viasd_model *m, viasd_cache *cache, const viasd_draft *draft, const viasd_result *result,
+                    void *stream) {
+    int rc;
+    if ((rc = check_draft(m, draft)) || (rc = check_cache(cache))) return rc;
+    if (!result || !result->n_acc || !result->path || !result->out_tok || !result->n_emit) return VIASD_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    return timed(m, VIASD_T_COMMIT, st, [&] { return launch_commit(m, cache, draft, result, st); });
+}
+
+int viasd_verify_step(viasd_model *m, viasd_cache *cache, const viasd_draft *draft, const viasd_params *params,
+                      float *slim_logits, float *full_logits, viasd_result *result, void *stream) {
+    int rc;
+    if (!slim_logits || !full_logits) return VIASD_EINVAL;
+    if ((rc = check_params(params))) return rc;
+    if (params->conf_source == 0) {
+        if ((rc = viasd_tier_accept(m, draft, params, nullptr, nullptr, 1, result, stream))) return rc;
+        if ((rc = viasd_slim_forward(m, cache, draft, slim_logits, stream))) return rc;
+    } else {
+        if ((rc = viasd_slim_forward(m, cache, draft, slim_logits, stream))) return rc;
+        if ((rc = viasd_tier_accept(m, draft, params, slim_logits, nullptr, 1, result, stream))) return rc;
+    }
+    if ((rc = viasd_full_forward(m, cache, draft, full_logits, stream))) return rc;
+    if ((rc = viasd_tier_accept(m, draft, params, slim_logits, full_logits, 2, result, stream))) return rc;
+    return viasd_kv_commit(m, cache, draft, result, stream);
+}
+
+int viasd_get_stats(viasd_model *m, viasd_stats *host_out, void *stream) {
+    if (!m || !host_out) return VIASD_EINVAL;
+    DeviceStats s;
+    CUDA_TRY(cudaMemcpyAsync(&s, m->ws.stats, sizeof(s), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    host_out->steps = s.steps;
+    for (int i = 0; i < 3; ++i) host_out->tier_count[i] = s.tier_count[i];
+    host_out->emitted = s.emitted;
+    host_out->accepted = s.accepted;
+    host_out->device_status = s.device_status;
+    host_out->need_slim = s.need_slim;
+    host_out->need_full = s.need_full;
+    return VIASD_OK;
+}
+
+const char *viasd_strerror(int code) {
+    switch (code) {
+    case VIASD_OK: return "ok";
+    case VIASD_EINVAL: return "invalid argument";
+    case VIASD_ECAPACITY: return "capacity exceeded";
+    case VIASD_ECUDA: return "CUDA runtime error";
+    case VIASD_EDEVICE: return "device-side check failed";
+    case VIASD_EUNSUPPORTED: return "unsupported device";
+    default: return "unknown error";
+    }
+}
+
+int viasd_last_cuda_error(void) { return g_last_cuda_error; }
+
+unsigned long long viasd_launch_count(void) { return g_launch_count; }
+
+int viasd_set_timing(viasd_model *m, int on) {
+    if (!m) return VIASD_EINVAL;
+    KernelTimer &t = m->timer;
+    if (on && !t.beg) {
+        t.beg = new cudaEvent_t[KernelTimer::CAP];
+        t.end = new cudaEvent_t[KernelTimer::CAP];
+        t.cls = new int[KernelTimer::CAP];
+        for (t.created = 0; t.created < KernelTimer::CAP; ++t.created) {
+            CUDA_TRY(cudaEventCreate(&t.beg[t.created]));
+            CUDA_TRY(cudaEventCreate(&t.end[t.created]));
+        }
+    }
+    t.on = on != 0;
+    t.n = 0;
+    t.dropped = 0;
+    return VIASD_OK;
+}
+
+int viasd_get_timing(viasd_model *m, viasd_timing *out, void *stream) {
+    if (!m || !out) return VIASD_EINVAL;
+    KernelTimer &t = m->timer;
+    CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    memset(out, 0, sizeof(*out));
+    for (int i = 0; i < t.n; ++i) {
+        float ms = 0.f;
+        CUDA_TRY(cudaEventElapsedTime(&ms, t.beg[i], t.end[i]));
+        out->ms[t.cls[i]] += ms;
+        out->launches[t.cls[i]] += 1;
+    }
+    out->dropped = t.dropped;
+    t.n = 0;
+    t.dropped = 0;
+    return VIASD_OK;
+}
+
+size_t viasd_gemm_scratch_bytes(int rows, int n, int k) {
+    (void)rows; (void)n; (void)k;
+    return 256;
+}
+
+int viasd_gemm(const void *x, const void *w, float *y, int rows, int n, int k, int dtype, void *scratch,
+               size_t scratch_bytes, void *stream) {
+    if (!x || !w || !y || rows < 1 || rows > 256 || n < 1 || k < 8 || (dtype != 0 && dtype != 1)) return VIASD_EINVAL;
+    if (((uintptr_t)x & 15) || ((uintptr_t)w & 15)) return VIASD_EINVAL;
+    if (scratch_bytes < viasd_gemm_scratch_bytes(rows, n, k) || !scratch) return VIASD_ECAPACITY;
+    GemmSegs s{{w, nullptr, nullptr}, {n, 0, 0}, 1};
+    return launch_gemm_rowwarp(x, s, rows, k, dtype, EPI_STORE, y, nullptr, n, (cudaStream_t)stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,175 @@
+// KV-append attention over a drafted block: each of the M query rows of a sequence attends to the
+// committed cache rows 0..n-1 and to the block rows on its own root path (causal mask for a chain,
+// ancestor mask for a tree).  Split-KV: a CTA handles one (sequence, kv head, key range, group of
+// query rows), keeps an online softmax per query row and writes unnormalised partials; a second
+// kernel merges the key ranges.
+#include "common.cuh"
+
+namespace {
+
+constexpr int TK = 32;          // keys per shared-memory tile
+constexpr int QG = 16;          // query rows per CTA (2 per warp, 8 warps)
+constexpr int ATT_WARPS = 8;
+
+template <typename T, int HD>
+__global__ void __launch_bounds__(ATT_WARPS * 32)
+attention_split_kernel(float *__restrict__ part, const T *__restrict__ q, const T *__restrict__ kc,
+                       const T *__restrict__ vc, const int *__restrict__ len_eff, const TreeInfo *__restrict__ tree,
+                       int M, int H, int Hkv, int max_batch, int max_ctx, int layer_ord, int nsplit, float scale) {
+    __shared__ float Qs[QG][HD];
+    __shared__ float Ks[TK][HD + 1];
+    __shared__ float Vs[TK][HD];
+    constexpr int DPL = HD / 32;                     // output dims per lane
+    const int b = blockIdx.x / Hkv, g = blockIdx.x % Hkv, split = blockIdx.y, qg = blockIdx.z;
+    const int grp = H / Hkv, QR = grp * M;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n = len_eff[b], Tk = n + M;
+    int chunk = (Tk + nsplit - 1) / nsplit;
+    chunk = (chunk + TK - 1) / TK * TK;
+    const int k_begin = split * chunk, k_end = min(Tk, k_begin + chunk);
+
+    // stage this CTA's query rows, pre-scaled
+    for (int idx = threadIdx.x; idx < QG * HD; idx += blockDim.x) {
+        int qq = idx / HD, dd = idx % HD;
+        int qidx = qg * QG + qq;
+        float v = 0.f;
+        if (qidx < QR) {
+            int h = g * grp + qidx / M, i = qidx % M;
+            v = to_f32<T>(q[((size_t)(b * M + i) * H + h) * HD + dd]) * scale;
+        }
+        Qs[qq][dd] = v;
+    }
+    float mrun[2] = {-INFINITY, -INFINITY}, lrun[2] = {0.f, 0.f}, o[2][DPL];
+#pragma unroll
+    for (int r = 0; r < 2; ++r)
+#pragma unroll
+        for (int c = 0; c < DPL; ++c) o[r][c] = 0.f;
+    unsigned long long anc[2];
+    int qrow[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        int qidx = qg * QG + warp * 2 + r;
+        qrow[r] = qidx < QR ? qidx : -1;
+        anc[r] = qidx < QR ? tree->anc[qidx % M] : 0ull;
+    }
+    const size_t cbase = (((size_t)layer_ord * max_batch + b) * Hkv + g) * (size_t)max_ctx * HD;
+
+    for (int k0 = k_begin; k0 < k_end; k0 += TK) {
+        __syncthreads();
+        for (int idx = threadIdx.x; idx < TK * HD; idx += blockDim.x) {
+            int j = idx / HD, dd = idx % HD;
+            float kv = 0.f, vv = 0.f;
+            if (k0 + j < k_end) {
+                kv = to_f32<T>(kc[cbase + (size_t)(k0 + j) * HD + dd]);
+                vv = to_f32<T>(vc[cbase + (size_t)(k0 + j) * HD + dd]);
+            }
+            Ks[j][dd] = kv;
+            Vs[j][dd] = vv;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            if (qrow[r] < 0) continue;
+            const int j = k0 + lane;
+            const bool valid = j < k_end && (j < n || ((anc[r] >> (j - n)) & 1ull));
+            float s = 0.f;
+            const float *qs = Qs[warp * 2 + r];
+#pragma unroll 8
+            for (int dd = 0; dd < HD; ++dd) s = fmaf(qs[dd], Ks[lane][dd], s);
+            s = valid ? s : -INFINITY;
+            float mnew = fmaxf(mrun[r], warp_max(s));
+            if (mnew == -INFINITY) continue;                     // nothing visible yet
+            float p = valid ? expf(s - mnew) : 0.f;
+            float corr = expf(mrun[r] - mnew);                   // exp(-inf) = 0 on the first tile
+            lrun[r] = lrun[r] * corr + warp_sum(p);
+#pragma unroll
+            for (int c = 0; c < DPL; ++c) o[r][c] *= corr;
+#pragma unroll 8
+            for (int jj = 0; jj < TK; ++jj) {
+                float pj = __shfl_sync(0xffffffffu, p, jj);
+#pragma unroll
+                for (int c = 0; c < DPL; ++c) o[r][c] = fmaf(pj, Vs[jj][lane + 32 * c], o[r][c]);
+            }
+            mrun[r] = mnew;
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        if (qrow[r] < 0) continue;
+        int h = g * grp + qrow[r] / M, i = qrow[r] % M;
+        float *dst = part + ((((size_t)b * H + h) * M + i) * nsplit + split) * (HD + 2);
+#pragma unroll
+        for (int c = 0; c < DPL; ++c) dst[lane + 32 * c] = o[r][c];
+        if (lane == 0) { dst[HD] = mrun[r]; dst[HD + 1] = lrun[r]; }
+    }
+}
+
+template <typename T, int HD>
+__global__ void attention_combine_kernel(T *__restrict__ out, const float *__restrict__ part, int M, int H, int nsplit) {
+    const int r = blockIdx.x, h = blockIdx.y;        // r = b * M + i
+    const int b = r / M, i = r % M;
+    const float *src = part + (((size_t)b * H + h) * M + i) * (size_t)nsplit * (HD + 2);
+    float mmax = -INFINITY;
+    for (int s = 0; s < nsplit; ++s) mmax = fmaxf(mmax, src[(size_t)s * (HD + 2) + HD]);
+    for (int dd = threadIdx.x; dd < HD; dd += blockDim.x) {
+        float num = 0.f, den = 0.f;
+        for (int s = 0; s < nsplit; ++s) {
+            const float *p = src + (size_t)s * (HD + 2);
+            float ms = p[HD];
+            if (ms == -INFINITY) continue;
+            float w = expf(ms - mmax);
+            num = fmaf(p[dd], w, num);
+            den = fmaf(p[HD + 1], w, den);
+        }
+        out[((size_t)r * H + h) * HD + dd] = from_f32<T>(num / den);
+    }
+}
+
+template <typename T, int HD>
+int run(const viasd_model *m, const void *kc, const void *vc, int layer_ord, int batch, int M, int nsplit,
+        cudaStream_t st) {
+    const viasd_config &c = m->cfg;
+    const int grp = c.n_heads / c.n_kv_heads;
+    const int qgroups = (grp * M + QG - 1) / QG;
+    dim3 grid(batch * c.n_kv_heads, nsplit, qgroups);
+    attention_split_kernel<T, HD><<<grid, ATT_WARPS * 32, 0, st>>>(m->ws.part, (const T *)m->ws.q, (const T *)kc,
+        (const T *)vc, m->ws.len_eff, m->ws.tree, M, c.n_heads, c.n_kv_heads, c.max_batch, c.max_ctx, layer_ord, nsplit,
+        1.0f / sqrtf((float)HD));
+    LAUNCH_CHECK();
+    attention_combine_kernel<T, HD><<<dim3(batch * M, c.n_heads), HD < 128 ? HD : 128, 0, st>>>((T *)m->ws.attn,
+        m->ws.part, M, c.n_heads, nsplit);
+    LAUNCH_CHECK();
+    return VIASD_OK;
+}
+
+}  // namespace
+
+int attention_nsplit(const viasd_model *m, int batch, int M) {
+    const viasd_config &c = m->cfg;
+    const int grp = c.n_heads / c.n_kv_heads;
+    const int qgroups = (grp * M + QG - 1) / QG;
+    int ctas = batch * c.n_kv_heads * qgroups;
+    int nsplit = (2 * m->sm_count + ctas - 1) / ctas;
+    int by_len = (c.max_ctx + 127) / 128;            // at least 128 keys per split
+    if (nsplit > by_len) nsplit = by_len;
+    if (nsplit > 16) nsplit = 16;
+    if (nsplit < 1) nsplit = 1;
+    // never beyond what the partial buffer holds
+    size_t per_split = (size_t)batch * c.n_heads * M * (c.head_dim + 2) * sizeof(float);
+    while (nsplit > 1 && per_split * nsplit > m->ws.part_bytes) --nsplit;
+    return nsplit;
+}
+
+int launch_attention(const viasd_model *m, const void *kc, const void *vc, int layer_ord, int batch, int M,
+                     cudaStream_t st) {
+    const viasd_config &c = m->cfg;
+    int nsplit = attention_nsplit(m, batch, M);
+    if (c.dtype == 0) {
+        if (c.head_dim == 64) return run<float, 64>(m, kc, vc, layer_ord, batch, M, nsplit, st);
+        if (c.head_dim == 128) return run<float, 128>(m, kc, vc, layer_ord, batch, M, nsplit, st);
+    } else {
+        if (c.head_dim == 64) return run<__nv_bfloat16, 64>(m, kc, vc, layer_ord, batch, M, nsplit, st);
+        if (c.head_dim == 128) return run<__nv_bfloat16, 128>(m, kc, vc, layer_ord, batch, M, nsplit, st);
+    }
+    return VIASD_EINVAL;
+}

@@ -1,0 +1,128 @@
+// Shared declarations of the CUDA side: model handle, workspace layout, launch prototypes.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+#include "../../include/viasd.h"
+
+#define VIASD_MAX_ROWS_PER_SEQ 64
+
+// ---------------------------------------------------------------------------------------------
+// device-side records kept in the workspace
+// ---------------------------------------------------------------------------------------------
+struct TreeInfo {                       // rebuilt from `parent` at the start of every pass
+    unsigned long long anc[VIASD_MAX_ROWS_PER_SEQ];   // bit r set: row r is on the root path of row i
+    int depth[VIASD_MAX_ROWS_PER_SEQ];
+    int first_child[VIASD_MAX_ROWS_PER_SEQ];          // per row: first child node or -1
+    int next_sibling[VIASD_MAX_ROWS_PER_SEQ];         // per node: next child of the same parent or -1
+    int is_chain;
+};
+
+struct DeviceStats {
+    unsigned long long steps;
+    unsigned long long tier_count[3];
+    unsigned long long emitted;
+    unsigned long long accepted;
+    int device_status;
+    int need_slim, need_full;
+};
+
+struct Workspace {                      // pointers into the caller's workspace block
+    float *rope_cos, *rope_sin;         // [max_ctx, hd/2]
+    float *h;                           // [R, d] residual stream
+    void *a;                            // [R, d] normed activations (model dtype)
+    float *qkv;                         // [R, (H + 2 Hkv) hd]
+    void *q;                            // [R, H hd] rotated queries (model dtype)
+    void *attn;                         // [R, H hd] attention output (model dtype)
+    void *act;                          // [R, ff] SwiGLU output (model dtype)
+    float *part;                        // split partial sums (GEMM split-K / attention split-KV)
+    size_t part_bytes;
+    int *len_eff;                       // [B] committed length clamped to the cache capacity
+    int *row_tok;                       // [R] token id per row
+    TreeInfo *tree;
+    DeviceStats *stats;
+    float *accept_scratch;              // [B, 3, V] sampling-mode distributions
+};
+
+struct KernelTimer {                    // optional per-launch CUDA-event record (measurement only)
+    static constexpr int CAP = 8192;
+    cudaEvent_t *beg, *end;
+    int *cls;
+    int n, created;
+    long long dropped;
+    bool on;
+};
+
+struct viasd_model {
+    KernelTimer timer;
+    viasd_config cfg;
+    int n_routed;
+    int routed[512];                    // routed layer ids, increasing
+    const void *embed, *lm_head;
+    const float *final_norm;
+    const void **wq, **wk, **wv, **wo, **wg, **wu, **wd;   // host arrays [L] of device pointers
+    const float **norm1, **norm2;
+    Workspace ws;
+    int sm_count;
+};
+
+// error helpers -------------------------------------------------------------------------------
+extern int g_last_cuda_error;
+extern unsigned long long g_launch_count;
+#define CUDA_TRY(expr)                                                     \
+    do {                                                                   \
+        cudaError_t e__ = (expr);                                          \
+        if (e__ != cudaSuccess) { g_last_cuda_error = (int)e__; return VIASD_ECUDA; } \
+    } while (0)
+#define LAUNCH_CHECK() do { ++g_launch_count; CUDA_TRY(cudaGetLastError()); } while (0)
+
+// ---------------------------------------------------------------------------------------------
+// kernel launchers (one .cu file each); all enqueue on `st` and return a VIASD_* code
+// ---------------------------------------------------------------------------------------------
+// misc.cu
+int launch_rope_table(const viasd_model *m, cudaStream_t st);
+int launch_prep(const viasd_model *m, const viasd_cache *c, const viasd_draft *d, cudaStream_t st);
+int launch_embed(const viasd_model *m, int rows, cudaStream_t st);
+int launch_rmsnorm(const viasd_model *m, const float *gain, int rows, cudaStream_t st);
+int launch_rope_append(const viasd_model *m, void *kc, void *vc, int layer_ord, int batch, int M,
+                       cudaStream_t st);
+int launch_commit(const viasd_model *m, viasd_cache *c, const viasd_draft *d, const viasd_result *r,
+                  cudaStream_t st);
+
+// gemm_rowwarp.cu -- generic CUDA-core GEMM (fp32 models; shapes the tensor-core kernels do not take)
+enum GemmEpilogue { EPI_STORE = 0, EPI_ADD = 1, EPI_SWIGLU = 2 };
+struct GemmSegs { const void *w[3]; int n[3]; int count; };
+int launch_gemm_rowwarp(const void *x, const GemmSegs &segs, int rows, int k, int dtype, int epilogue,
+                        float *out_f32, void *out_act, int ld_out, cudaStream_t st);
+
+// attention.cu
+int launch_attention(const viasd_model *m, const void *kc, const void *vc, int layer_ord, int batch, int M,
+                     cudaStream_t st);
+
+// tier_accept.cu
+int launch_tier(const viasd_model *m, const viasd_draft *d, const viasd_params *p, const float *slim_logits,
+                viasd_result *r, cudaStream_t st);
+int launch_accept(const viasd_model *m, const viasd_draft *d, const viasd_params *p, const float *slim_logits,
+                  const float *full_logits, viasd_result *r, cudaStream_t st);
+
+// ---------------------------------------------------------------------------------------------
+// small device helpers
+// ---------------------------------------------------------------------------------------------
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}

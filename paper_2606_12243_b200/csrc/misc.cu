@@ -1,0 +1,242 @@
+// Small memory-bound kernels of the decoder block and the cache bookkeeping:
+// rotary table, per-pass preparation (tree layout, row tokens, clamped lengths), embedding gather,
+// RMSNorm, rotary embedding + KV append, KV commit.
+#include "common.cuh"
+
+// ---------------------------------------------------------------------------------------------
+// rotary table: cos/sin(pos * theta^(-2p/hd)), computed in double once per handle
+// ---------------------------------------------------------------------------------------------
+__global__ void rope_table_kernel(float *cosv, float *sinv, int max_ctx, int half, double theta) {
+    int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= max_ctx * half) return;
+    int pos = idx / half, p = idx % half;
+    double inv = pow(theta, -2.0 * (double)p / (double)(2 * half));
+    double ang = (double)pos * inv;
+    cosv[idx] = (float)cos(ang);
+    sinv[idx] = (float)sin(ang);
+}
+
+int launch_rope_table(const viasd_model *m, cudaStream_t st) {
+    int half = m->cfg.head_dim / 2;
+    int n = m->cfg.max_ctx * half;
+    rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(m->ws.rope_cos, m->ws.rope_sin, m->cfg.max_ctx, half,
+                                                       (double)m->cfg.rope_theta);
+    LAUNCH_CHECK();
+    return VIASD_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// per-pass preparation
+// ---------------------------------------------------------------------------------------------
+__global__ void prep_kernel(TreeInfo *tree, int *len_eff, int *row_tok, DeviceStats *stats, const int *len,
+                            const int *pending, const int *draft_tok, const int *parent, int B, int N,
+                            int max_ctx, int vocab) {
+    const int M = N + 1;
+    if (threadIdx.x == 0) {
+        int last_child[VIASD_MAX_ROWS_PER_SEQ];
+        for (int i = 0; i < M; ++i) { tree->first_child[i] = -1; tree->next_sibling[i] = -1; last_child[i] = -1; }
+        tree->anc[0] = 1ull;
+        tree->depth[0] = 0;
+        int chain = 1;
+        for (int n = 0; n < N; ++n) {
+            int p = parent[n];
+            if (p < -1 || p >= n) { stats->device_status = VIASD_EDEVICE; p = -1; }
+            if (p != n - 1) chain = 0;
+            int pr = p + 1, i = n + 1;
+            tree->anc[i] = tree->anc[pr] | (1ull << i);
+            tree->depth[i] = tree->depth[pr] + 1;
+            if (last_child[pr] < 0) tree->first_child[pr] = n; else tree->next_sibling[last_child[pr]] = n;
+            last_child[pr] = n;
+        }
+        tree->is_chain = chain;
+    }
+    for (int b = threadIdx.x; b < B; b += blockDim.x) {
+        int l = len[b];
+        int c = min(max(l, 0), max_ctx - M);
+        if (c != l) stats->device_status = VIASD_ECAPACITY;
+        len_eff[b] = c;
+    }
+    for (int r = threadIdx.x; r < B * M; r += blockDim.x) {
+        int b = r / M, i = r % M;
+        int t = (i == 0) ? pending[b] : draft_tok[b * N + i - 1];
+        if (t < 0 || t >= vocab) { stats->device_status = VIASD_EDEVICE; t = 0; }
+        row_tok[r] = t;
+    }
+}
+
+int launch_prep(const viasd_model *m, const viasd_cache *c, const viasd_draft *d, cudaStream_t st) {
+    prep_kernel<<<1, 128, 0, st>>>(m->ws.tree, m->ws.len_eff, m->ws.row_tok, m->ws.stats, c->len, c->pending,
+                                   d->draft_tok, d->parent, d->batch, d->n_nodes, m->cfg.max_ctx, m->cfg.vocab);
+    LAUNCH_CHECK();
+    return VIASD_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// embedding gather: h[r] = E[row_tok[r]]
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void embed_kernel(float *h, const T *E, const int *row_tok, int d) {
+    int r = blockIdx.x;
+    const T *src = E + (size_t)row_tok[r] * d;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) h[(size_t)r * d + i] = to_f32<T>(src[i]);
+}
+
+int launch_embed(const viasd_model *m, int rows, cudaStream_t st) {
+    if (m->cfg.dtype == 0)
+        embed_kernel<float><<<rows, 256, 0, st>>>(m->ws.h, (const float *)m->embed, m->ws.row_tok, m->cfg.d_model);
+    else
+        embed_kernel<__nv_bfloat16><<<rows, 256, 0, st>>>(m->ws.h, (const __nv_bfloat16 *)m->embed,
+                                                          m->ws.row_tok, m->cfg.d_model);
+    LAUNCH_CHECK();
+    return VIASD_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// RMSNorm: a[r] = h[r] / sqrt(mean(h[r]^2) + eps) * gain, written in the model dtype
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void rmsnorm_kernel(T *a, const float *h, const float *gain, int d, float eps) {
+    __shared__ float red[32];
+    int r = blockIdx.x;
+    const float *x = h + (size_t)r * d;
+    float s = 0.f;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) { float v = x[i]; s += v * v; }
+    s = warp_sum(s);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        float v = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0.f;
+        v = warp_sum(v);
+        if (threadIdx.x == 0) red[0] = rsqrtf(v / (float)d + eps);
+    }
+    __syncthreads();
+    float inv = red[0];
+    for (int i = threadIdx.x; i < d; i += blockDim.x) a[(size_t)r * d + i] = from_f32<T>(x[i] * inv * gain[i]);
+}
+
+int launch_rmsnorm(const viasd_model *m, const float *gain, int rows, cudaStream_t st) {
+    if (m->cfg.dtype == 0)
+        rmsnorm_kernel<float><<<rows, 256, 0, st>>>((float *)m->ws.a, m->ws.h, gain, m->cfg.d_model, m->cfg.rms_eps);
+    else
+        rmsnorm_kernel<__nv_bfloat16><<<rows, 256, 0, st>>>((__nv_bfloat16 *)m->ws.a, m->ws.h, gain,
+                                                            m->cfg.d_model, m->cfg.rms_eps);
+    LAUNCH_CHECK();
+    return VIASD_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// rotary embedding of q and k, KV append at slot len + row
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void rope_append_kernel(T *q_out, T *kc, T *vc, const float *qkv, const float *cosv, const float *sinv,
+                                   const int *len_eff, const TreeInfo *tree, int M, int H, int Hkv, int hd,
+                                   int max_batch, int max_ctx, int layer_ord) {
+    int r = blockIdx.x, head = blockIdx.y;
+    int b = r / M, i = r % M;
+    int half = hd >> 1;
+    int n = len_eff[b];
+    int pos = n + tree->depth[i], slot = n + i;
+    const float *src = qkv + (size_t)r * (H + 2 * Hkv) * hd + (size_t)head * hd;
+    for (int p = threadIdx.x; p < half; p += blockDim.x) {
+        float x1 = src[p], x2 = src[p + half];
+        if (head < H + Hkv) {
+            float c = cosv[(size_t)pos * half + p], s = sinv[(size_t)pos * half + p];
+            float y1 = x1 * c - x2 * s, y2 = x2 * c + x1 * s;
+            if (head < H) {
+                T *dst = q_out + (size_t)r * H * hd + (size_t)head * hd;
+                dst[p] = from_f32<T>(y1);
+                dst[p + half] = from_f32<T>(y2);
+            } else {
+                int g = head - H;
+                T *dst = kc + ((((size_t)layer_ord * max_batch + b) * Hkv + g) * max_ctx + slot) * hd;
+                dst[p] = from_f32<T>(y1);
+                dst[p + half] = from_f32<T>(y2);
+            }
+        } else {
+            int g = head - H - Hkv;
+            T *dst = vc + ((((size_t)layer_ord * max_batch + b) * Hkv + g) * max_ctx + slot) * hd;
+            dst[p] = from_f32<T>(x1);
+            dst[p + half] = from_f32<T>(x2);
+        }
+    }
+}
+
+int launch_rope_append(const viasd_model *m, void *kc, void *vc, int layer_ord, int batch, int M, cudaStream_t st) {
+    const viasd_config &c = m->cfg;
+    dim3 grid(batch * M, c.n_heads + 2 * c.n_kv_heads);
+    int threads = c.head_dim / 2 < 32 ? 32 : c.head_dim / 2;
+    if (c.dtype == 0)
+        rope_append_kernel<float><<<grid, threads, 0, st>>>((float *)m->ws.q, (float *)kc, (float *)vc, m->ws.qkv,
+            m->ws.rope_cos, m->ws.rope_sin, m->ws.len_eff, m->ws.tree, M, c.n_heads, c.n_kv_heads, c.head_dim,
+            c.max_batch, c.max_ctx, layer_ord);
+    else
+        rope_append_kernel<__nv_bfloat16><<<grid, threads, 0, st>>>((__nv_bfloat16 *)m->ws.q, (__nv_bfloat16 *)kc,
+            (__nv_bfloat16 *)vc, m->ws.qkv, m->ws.rope_cos, m->ws.rope_sin, m->ws.len_eff, m->ws.tree, M, c.n_heads,
+            c.n_kv_heads, c.head_dim, c.max_batch, c.max_ctx, layer_ord);
+    LAUNCH_CHECK();
+    return VIASD_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// KV commit: compact the accepted path, then advance len / pending / tokens
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void commit_move_kernel(T *kf, T *vf, T *ks, T *vs, const int *len_eff, const int *n_acc,
+                                   const int *path, int N, int L, int Ls, int Hkv, int hd, int max_batch,
+                                   int max_ctx) {
+    int layer = blockIdx.x, b = blockIdx.y, g = blockIdx.z;
+    T *kc = layer < L ? kf : ks;
+    T *vc = layer < L ? vf : vs;
+    int lo = layer < L ? layer : layer - L;
+    size_t base = (((size_t)lo * max_batch + b) * Hkv + g) * (size_t)max_ctx * hd;
+    int n = len_eff[b];
+    int na = min(n_acc[b], N);
+    // each thread owns fixed columns, so walking j in order is enough to keep sources intact
+    for (int j = 0; j < na; ++j) {
+        int node = path[b * N + j];
+        if (node < j || node >= N) break;           // not a valid path entry: stop (never moves rows up)
+        int src = n + node + 1, dst = n + 1 + j;
+        if (src == dst) continue;
+        for (int c = threadIdx.x; c < hd; c += blockDim.x) {
+            kc[base + (size_t)dst * hd + c] = kc[base + (size_t)src * hd + c];
+            vc[base + (size_t)dst * hd + c] = vc[base + (size_t)src * hd + c];
+        }
+    }
+}
+
+__global__ void commit_advance_kernel(int *len, int *pending, int *tokens, const int *len_eff, const int *n_emit,
+                                      const int *out_tok, int B, int N, int max_ctx) {
+    int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    int n = len_eff[b];
+    int ne = min(max(n_emit[b], 0), N + 1);
+    if (ne == 0) return;
+    if (tokens) {
+        tokens[(size_t)b * max_ctx + n] = pending[b];
+        for (int j = 0; j + 1 < ne; ++j) tokens[(size_t)b * max_ctx + n + 1 + j] = out_tok[b * (N + 1) + j];
+    }
+    len[b] = n + ne;
+    pending[b] = out_tok[b * (N + 1) + ne - 1];
+}
+
+int launch_commit(const viasd_model *m, viasd_cache *c, const viasd_draft *d, const viasd_result *r,
+                  cudaStream_t st) {
+    const viasd_config &cf = m->cfg;
+    int rc = launch_prep(m, c, d, st);
+    if (rc) return rc;
+    dim3 grid(cf.n_layers + m->n_routed, d->batch, cf.n_kv_heads);
+    int threads = cf.head_dim < 32 ? 32 : (cf.head_dim > 256 ? 256 : cf.head_dim);
+    if (cf.dtype == 0)
+        commit_move_kernel<float><<<grid, threads, 0, st>>>((float *)c->k_full, (float *)c->v_full, (float *)c->k_slim,
+            (float *)c->v_slim, m->ws.len_eff, r->n_acc, r->path, d->n_nodes, cf.n_layers, m->n_routed, cf.n_kv_heads,
+            cf.head_dim, cf.max_batch, cf.max_ctx);
+    else
+        commit_move_kernel<__nv_bfloat16><<<grid, threads, 0, st>>>((__nv_bfloat16 *)c->k_full,
+            (__nv_bfloat16 *)c->v_full, (__nv_bfloat16 *)c->k_slim, (__nv_bfloat16 *)c->v_slim, m->ws.len_eff, r->n_acc,
+            r->path, d->n_nodes, cf.n_layers, m->n_routed, cf.n_kv_heads, cf.head_dim, cf.max_batch, cf.max_ctx);
+    LAUNCH_CHECK();
+    commit_advance_kernel<<<(d->batch + 63) / 64, 64, 0, st>>>(c->len, c->pending, c->tokens, m->ws.len_eff,
+                                                               r->n_emit, r->out_tok, d->batch, d->n_nodes, cf.max_ctx);
+    LAUNCH_CHECK();
+    return VIASD_OK;
+}

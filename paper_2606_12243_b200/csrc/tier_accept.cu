@@ -1,0 +1,357 @@
+// Fused confidence-tier kernel and accept / resolve kernel.
+//
+// Tier kernel (App. B, Eq. B.1-B.3): per drafted token v, d = l[v] - max_u l[u] on the gating logits;
+// tier 0 if d >= log_tau_hi, 1 if d >= log_tau_lo, else 2.  One CTA per gating row scans the
+// vocabulary once and serves every node gated by that row.
+//
+// Accept kernel (Algorithm 2, per-position loop; Algorithm 1, what is appended; App. A, Eq. A.2-A.3):
+// one CTA per sequence walks the draft from the pending token: children of the current row are tried in
+// index order; tier-0 children are taken at once, tier-1 children are judged by q', tier-2 children by
+// q.  The first row where no child passes ends the walk and the strongest judge that rejected there
+// emits the replacement token.  The walk is sequential over depth; every test is a reduction over the
+// vocabulary done by the whole CTA.
+#include "common.cuh"
+
+namespace {
+
+constexpr int ACC_THREADS = 512;
+
+// ---- counter-based uniforms -------------------------------------------------------------------
+__device__ __forceinline__ unsigned long long mix64(unsigned long long z) {
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+constexpr unsigned long long GAMMA = 0x9E3779B97F4A7C15ull;
+__device__ __forceinline__ unsigned long long stream_key(unsigned long long seed, unsigned long long step, int b,
+                                                         int stream) {
+    unsigned long long k = mix64(seed + GAMMA);
+    k = mix64(k + step * GAMMA + 1ull);
+    return mix64(k + (unsigned long long)(b * 256 + stream) * GAMMA + 2ull);
+}
+// 23 random bits -> (k + 0.5) / 2^23: exact in fp32, strictly inside (0, 1)
+__device__ __forceinline__ float unit_f32(unsigned long long key, unsigned long long idx) {
+    unsigned long long w = mix64(key + idx * GAMMA + 3ull);
+    return ((float)(w >> 41) + 0.5f) * 1.1920928955078125e-7f;
+}
+
+// ---- block reductions ---------------------------------------------------------------------------
+struct MaxIdx { float v; int i; };
+__device__ __forceinline__ MaxIdx better(MaxIdx a, MaxIdx b) {   // larger value, lowest index on ties
+    if (b.v > a.v || (b.v == a.v && b.i < a.i)) return b;
+    return a;
+}
+__device__ MaxIdx block_argmax(MaxIdx x, MaxIdx *sh) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        MaxIdx y;
+        y.v = __shfl_xor_sync(0xffffffffu, x.v, o);
+        y.i = __shfl_xor_sync(0xffffffffu, x.i, o);
+        x = better(x, y);
+    }
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = x;
+    __syncthreads();
+    MaxIdx r = sh[0];
+    for (int w = 1; w < (int)(blockDim.x >> 5); ++w) r = better(r, sh[w]);
+    return r;
+}
+__device__ float block_sum(float x, float *sh) {
+    x = warp_sum(x);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = x;
+    __syncthreads();
+    float r = 0.f;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) r += sh[w];
+    return r;
+}
+__device__ float block_max(float x, float *sh) {
+    x = warp_max(x);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = x;
+    __syncthreads();
+    float r = sh[0];
+    for (int w = 1; w < (int)(blockDim.x >> 5); ++w) r = fmaxf(r, sh[w]);
+    return r;
+}
+
+// ---- tier kernel ------------------------------------------------------------------------------
+// grid (gate rows per sequence, B).  conf_source 0: gate row of node n = prow[n], rows = drafter logits
+// [B, R, V]; conf_source 1: gate row = parent[n] + 1, rows = slim logits [B, M, V].
+__global__ void __launch_bounds__(256)
+tier_kernel(unsigned char *__restrict__ tier, float *__restrict__ conf, DeviceStats *stats,
+            const float *__restrict__ gate_logits, const int *__restrict__ draft_tok, const int *__restrict__ prow,
+            const int *__restrict__ parent, int conf_source, int rows_per_seq, int N, int V, float log_tau_lo,
+            float log_tau_hi) {
+    __shared__ float sh[32];
+    const int gr = blockIdx.x, b = blockIdx.y;
+    const float *row = gate_logits + ((size_t)b * rows_per_seq + gr) * V;
+    float mx = -INFINITY;
+    if ((V & 3) == 0 && ((uintptr_t)row & 15) == 0) {
+        const float4 *r4 = reinterpret_cast<const float4 *>(row);
+        for (int i = threadIdx.x; i < V / 4; i += blockDim.x) {
+            float4 v = r4[i];
+            mx = fmaxf(mx, fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)));
+        }
+    } else {
+        for (int i = threadIdx.x; i < V; i += blockDim.x) mx = fmaxf(mx, row[i]);
+    }
+    mx = block_max(mx, sh);
+    for (int n = threadIdx.x; n < N; n += blockDim.x) {
+        int g = conf_source == 0 ? prow[n] : parent[n] + 1;
+        if (g != gr) continue;
+        int t = draft_tok[b * N + n];
+        t = min(max(t, 0), V - 1);
+        float d = row[t] - mx;
+        int tr = d >= log_tau_hi ? 0 : (d >= log_tau_lo ? 1 : 2);
+        tier[b * N + n] = (unsigned char)tr;
+        conf[b * N + n] = d;
+        atomicAdd(&stats->tier_count[tr], 1ull);
+        if (tr == 1) stats->need_slim = 1;
+        if (tr == 2) stats->need_full = 1;
+    }
+    if (gr == 0 && b == 0 && threadIdx.x == 0) atomicAdd(&stats->steps, 1ull);
+}
+
+// ---- accept kernel ----------------------------------------------------------------------------
+struct AcceptArgs {
+    const float *slim, *full, *drafter;      // [B, M, V], [B, M, V], [B, R, V]
+    const int *draft_tok, *prow;             // [B, N], [N]
+    const unsigned char *tier;               // [B, N]
+    const TreeInfo *tree;
+    float *scratch;                          // [B, 3, V]
+    int *n_acc, *path, *out_tok, *n_emit, *corr_src;
+    unsigned char *judge;
+    DeviceStats *stats;
+    int N, R, V;
+    int mode, strict_break, emit_bonus;
+    float inv_temp, log1m_alpha, inv_beta;
+    float log_acc_rel[3];
+    unsigned long long seed, step;
+};
+
+// numerators of softmax(l / T) into dst, returns their sum
+__device__ float softmax_numerators(float *dst, const float *row, int V, float inv_temp, float *sh) {
+    float mx = -INFINITY;
+    for (int i = threadIdx.x; i < V; i += blockDim.x) mx = fmaxf(mx, row[i]);
+    mx = block_max(mx, sh);
+    float s = 0.f;
+    for (int i = threadIdx.x; i < V; i += blockDim.x) {
+        float e = expf((row[i] - mx) * inv_temp);
+        dst[i] = e;
+        s += e;
+    }
+    return block_sum(s, sh);
+}
+
+// argmax_v (log w[v] - log(-log u_v)): a draw from w / sum(w)
+__device__ int gumbel_argmax(const float *w, int V, unsigned long long key, int row, MaxIdx *shm) {
+    MaxIdx best; best.v = -INFINITY; best.i = 0x7fffffff;
+    for (int i = threadIdx.x; i < V; i += blockDim.x) {
+        float wi = w[i];
+        if (wi > 0.f) {
+            float u = unit_f32(key, ((unsigned long long)row << 32) + (unsigned long long)i);
+            MaxIdx c; c.v = logf(wi) - logf(-logf(u)); c.i = i;
+            best = better(best, c);
+        }
+    }
+    best = block_argmax(best, shm);
+    return best.i == 0x7fffffff ? 0 : best.i;
+}
+
+__device__ int row_argmax(const float *row, int V, MaxIdx *shm) {
+    MaxIdx best; best.v = -INFINITY; best.i = 0x7fffffff;
+    for (int i = threadIdx.x; i < V; i += blockDim.x) { MaxIdx c; c.v = row[i]; c.i = i; best = better(best, c); }
+    best = block_argmax(best, shm);
+    return best.i == 0x7fffffff ? 0 : best.i;
+}
+
+__global__ void __launch_bounds__(ACC_THREADS)
+accept_kernel(AcceptArgs a) {
+    __shared__ float sh[32];
+    __shared__ MaxIdx shm[32];
+    const int b = blockIdx.x, N = a.N, M = N + 1, V = a.V;
+    const TreeInfo *tree = a.tree;
+    const bool sampling = a.mode == 1;
+    float *P[3] = {a.scratch + ((size_t)b * 3 + 0) * V, a.scratch + ((size_t)b * 3 + 1) * V,
+                   a.scratch + ((size_t)b * 3 + 2) * V};
+    const unsigned long long k_acc = stream_key(a.seed, a.step, b, 0), k_gum = stream_key(a.seed, a.step, b, 1);
+    for (int n = threadIdx.x; n < N; n += blockDim.x) a.judge[b * N + n] = 0;
+    __syncthreads();
+
+    int cur = 0, n_acc = 0, corr = -1, corr_src = 0;
+    while (true) {
+        int c = tree->first_child[cur];
+        const float *Lrow[3] = {nullptr, a.slim + ((size_t)b * M + cur) * V, a.full + ((size_t)b * M + cur) * V};
+        if (c < 0) {                                             // leaf: whole path accepted
+            if (a.emit_bonus) {
+                if (sampling) {
+                    softmax_numerators(P[2], Lrow[2], V, a.inv_temp, sh);
+                    __syncthreads();
+                    corr = gumbel_argmax(P[2], V, k_gum, cur, shm);
+                } else {
+                    corr = row_argmax(Lrow[2], V, shm);
+                }
+                corr_src = 2;
+            }
+            break;
+        }
+        float Z[3] = {0.f, 0.f, 0.f};
+        bool have[3] = {false, false, false};
+        float rowmax[3] = {0.f, 0.f, 0.f};
+        int failed = 0, taken = -1, taken_tier = 0;
+        for (; c >= 0; c = tree->next_sibling[c]) {
+            const int t = a.tier[b * N + c];
+            int v = a.draft_tok[b * N + c];
+            v = min(max(v, 0), V - 1);
+            if (t == 0) {
+                taken = c; taken_tier = 0;
+                if (threadIdx.x == 0) a.judge[b * N + c] = 1;
+                break;
+            }
+            bool pass;
+            if (!sampling) {
+                if (!have[t]) {
+                    float mx = -INFINITY;
+                    for (int i = threadIdx.x; i < V; i += blockDim.x) mx = fmaxf(mx, Lrow[t][i]);
+                    rowmax[t] = block_max(mx, sh);
+                    have[t] = true;
+                }
+                pass = (Lrow[t][v] - rowmax[t]) >= a.log_acc_rel[t];
+            } else {
+                if (!have[0]) {
+                    const float *prow_logits = a.drafter + ((size_t)b * a.R + a.prow[c]) * V;
+                    Z[0] = softmax_numerators(P[0], prow_logits, V, a.inv_temp, sh);
+                    have[0] = true;
+                }
+                if (!have[t]) {
+                    Z[t] = softmax_numerators(P[t], Lrow[t], V, a.inv_temp, sh);
+                    have[t] = true;
+                }
+                __syncthreads();
+                const float u = unit_f32(k_acc, (unsigned long long)c);
+                const float lp = logf(P[0][v] / Z[0]);
+                const float lj = logf(P[t][v] / Z[t]);
+                pass = (logf(u) + a.log1m_alpha + lp) < lj;       // u < j(v) / ((1 - alpha) p(v)), Eq. A.2
+            }
+            if (pass) {
+                taken = c; taken_tier = t;
+                if (threadIdx.x == 0) a.judge[b * N + c] = (unsigned char)(1 | (t << 4));
+                break;
+            }
+            if (threadIdx.x == 0) a.judge[b * N + c] = (unsigned char)(2 | (t << 4));
+            failed = max(failed, t);
+            if (sampling) {
+                // Eq. A.3 round by round: the rejecting judge becomes its residual against the proposal
+                // (kept as is if the residual vanishes); the rejected token leaves the proposal.
+                const float sj = a.inv_beta / Z[t], sp = 1.f / Z[0];
+                float s = 0.f;
+                for (int i = threadIdx.x; i < V; i += blockDim.x) s += fmaxf(0.f, P[t][i] * sj - P[0][i] * sp);
+                s = block_sum(s, sh);
+                if (s > 0.f) {
+                    for (int i = threadIdx.x; i < V; i += blockDim.x) P[t][i] = fmaxf(0.f, P[t][i] * sj - P[0][i] * sp);
+                    Z[t] = s;
+                }
+                __syncthreads();
+                if (threadIdx.x == 0) P[0][v] = 0.f;
+                __syncthreads();
+                float z = 0.f;
+                for (int i = threadIdx.x; i < V; i += blockDim.x) z += P[0][i];
+                z = block_sum(z, sh);
+                if (z > 0.f) Z[0] = z;
+            }
+        }
+        if (taken >= 0) {
+            if (a.strict_break && taken_tier == 1) {
+                corr = min(max(a.draft_tok[b * N + taken], 0), V - 1);
+                corr_src = 1;
+                break;
+            }
+            if (threadIdx.x == 0) a.path[b * N + n_acc] = taken;
+            ++n_acc;
+            cur = taken + 1;
+            continue;
+        }
+        corr_src = failed;
+        if (sampling) {
+            __syncthreads();
+            corr = gumbel_argmax(P[failed], V, k_gum, cur, shm);
+        } else {
+            corr = row_argmax(Lrow[failed], V, shm);
+        }
+        break;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int ne = 0;
+        for (int j = 0; j < n_acc; ++j) {
+            int node = a.path[b * N + j];
+            a.out_tok[b * (N + 1) + ne++] = min(max(a.draft_tok[b * N + node], 0), V - 1);
+        }
+        if (corr >= 0) a.out_tok[b * (N + 1) + ne++] = corr;
+        a.n_acc[b] = n_acc;
+        a.n_emit[b] = ne;
+        a.corr_src[b] = corr_src;
+        atomicAdd(&a.stats->emitted, (unsigned long long)ne);
+        atomicAdd(&a.stats->accepted, (unsigned long long)n_acc);
+    }
+}
+
+// the accept kernel needs the tree layout but no cache: build it here when called on its own
+__global__ void tree_only_kernel(TreeInfo *tree, DeviceStats *stats, const int *parent, int N) {
+    if (threadIdx.x != 0) return;
+    const int M = N + 1;
+    int last_child[VIASD_MAX_ROWS_PER_SEQ];
+    for (int i = 0; i < M; ++i) { tree->first_child[i] = -1; tree->next_sibling[i] = -1; last_child[i] = -1; }
+    tree->anc[0] = 1ull;
+    tree->depth[0] = 0;
+    int chain = 1;
+    for (int n = 0; n < N; ++n) {
+        int p = parent[n];
+        if (p < -1 || p >= n) { stats->device_status = VIASD_EDEVICE; p = -1; }
+        if (p != n - 1) chain = 0;
+        int pr = p + 1, i = n + 1;
+        tree->anc[i] = tree->anc[pr] | (1ull << i);
+        tree->depth[i] = tree->depth[pr] + 1;
+        if (last_child[pr] < 0) tree->first_child[pr] = n; else tree->next_sibling[last_child[pr]] = n;
+        last_child[pr] = n;
+    }
+    tree->is_chain = chain;
+}
+
+}  // namespace
+
+int launch_tier(const viasd_model *m, const viasd_draft *d, const viasd_params *p, const float *slim_logits,
+                viasd_result *r, cudaStream_t st) {
+    const int M = d->n_nodes + 1;
+    CUDA_TRY(cudaMemsetAsync(&m->ws.stats->need_slim, 0, 2 * sizeof(int), st));
+    const float *gate = p->conf_source == 0 ? d->drafter_logits : slim_logits;
+    const int rows = p->conf_source == 0 ? d->n_prows : M;
+    if (!gate) return VIASD_EINVAL;
+    tier_kernel<<<dim3(rows, d->batch), 256, 0, st>>>(r->tier, r->conf, m->ws.stats, gate, d->draft_tok, d->prow,
+        d->parent, p->conf_source, rows, d->n_nodes, m->cfg.vocab, p->log_tau_lo, p->log_tau_hi);
+    LAUNCH_CHECK();
+    return VIASD_OK;
+}
+
+int launch_accept(const viasd_model *m, const viasd_draft *d, const viasd_params *p, const float *slim_logits,
+                  const float *full_logits, viasd_result *r, cudaStream_t st) {
+    tree_only_kernel<<<1, 32, 0, st>>>(m->ws.tree, m->ws.stats, d->parent, d->n_nodes);
+    LAUNCH_CHECK();
+    AcceptArgs a;
+    a.slim = slim_logits; a.full = full_logits; a.drafter = d->drafter_logits;
+    a.draft_tok = d->draft_tok; a.prow = d->prow; a.tier = r->tier; a.tree = m->ws.tree;
+    a.scratch = m->ws.accept_scratch;
+    a.n_acc = r->n_acc; a.path = r->path; a.out_tok = r->out_tok; a.n_emit = r->n_emit; a.corr_src = r->corr_src;
+    a.judge = r->judge; a.stats = m->ws.stats;
+    a.N = d->n_nodes; a.R = d->n_prows; a.V = m->cfg.vocab;
+    a.mode = p->mode; a.strict_break = p->strict_break; a.emit_bonus = p->emit_bonus;
+    a.inv_temp = 1.0f / p->temperature;
+    a.log1m_alpha = log1pf(-p->alpha);
+    a.inv_beta = 1.0f / p->beta;
+    for (int i = 0; i < 3; ++i) a.log_acc_rel[i] = p->log_acc_rel[i];
+    a.seed = p->seed; a.step = p->step;
+    accept_kernel<<<d->batch, ACC_THREADS, 0, st>>>(a);
+    LAUNCH_CHECK();
+    return VIASD_OK;
+}

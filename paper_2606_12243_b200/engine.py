@@ -1,0 +1,115 @@
+"""Device-side set-up of a synthetic workload: weights, caches and step inputs in HBM.
+
+Memory management only (torch allocations and host->device copies of generated tensors);
+every step of the verification path runs in the CUDA library through `binding`.
+"""
+from __future__ import annotations
+
+from typing import Dict, List, Optional
+
+import numpy as np
+import torch
+
+from synth import workloads as W
+from . import binding as vb
+
+
+def to_device(a: np.ndarray, device="cuda") -> torch.Tensor:
+    """Generated tensor (fp32, int32, or bf16 as raw uint16 words) -> CUDA tensor of the right dtype."""
+    if a.dtype == np.uint16:
+        return torch.from_numpy(a.view(np.int16)).to(device).view(torch.bfloat16)
+    return torch.from_numpy(np.ascontiguousarray(a)).to(device)
+
+
+class Engine:
+    def __init__(self, wl: W.Workload, device="cuda", max_query: Optional[int] = None,
+                 extra_ctx: int = 0, fill_context: bool = True):
+        self.wl, self.device = wl, device
+        s = wl.shape
+        self.tdtype = torch.float32 if s.dtype == "f32" else torch.bfloat16
+        self.max_query = max_query or wl.rows
+        self.max_ctx = wl.ctx + max(self.max_query, wl.rows) + extra_ctx
+        self.cfg = vb.make_config(s.n_layers, s.d_model, s.n_heads, s.n_kv_heads, s.head_dim, s.d_ff, s.vocab,
+                                  s.dtype, wl.batch, self.max_ctx, self.max_query, s.rms_eps, s.rope_theta)
+        gen = W.Model(wl)
+        self.embed = to_device(gen.tensor(-1, "embed"), device)
+        self.lm_head = to_device(gen.tensor(-1, "lm_head"), device)
+        self.final_norm = to_device(gen.tensor(-1, "final_norm"), device)
+        self.layers: List[Dict[str, torch.Tensor]] = []
+        for l in range(s.n_layers):
+            self.layers.append({k: to_device(v, device) for k, v in gen.layer(l).items()})
+        self.routed = wl.routed
+        mask = [1 if l in set(self.routed) else 0 for l in range(s.n_layers)]
+        nbytes = vb.workspace_bytes(self.cfg, len(self.routed))
+        assert nbytes > 0, "configuration rejected by viasd_workspace_bytes"
+        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=device)
+        self.model = vb.init_model(self.cfg, self.embed, self.lm_head, self.final_norm, self.layers, mask,
+                                   self.workspace)
+        kv = lambda nl: torch.zeros((nl, wl.batch, s.n_kv_heads, self.max_ctx, s.head_dim), dtype=self.tdtype,
+                                    device=device)
+        self.k_full, self.v_full = kv(s.n_layers), kv(s.n_layers)
+        self.k_slim, self.v_slim = kv(len(self.routed)), kv(len(self.routed))
+        self.len = torch.zeros(wl.batch, dtype=torch.int32, device=device)
+        self.pending = torch.zeros(wl.batch, dtype=torch.int32, device=device)
+        self.tokens = torch.zeros((wl.batch, self.max_ctx), dtype=torch.int32, device=device)
+        self.cache = vb.make_cache(self.k_full, self.v_full, self.k_slim, self.v_slim, self.len, self.pending,
+                                   self.tokens)
+        if fill_context and not wl.real_prefill and wl.ctx > 0:
+            self.fill_synthetic_context()
+        self.draft = None
+        self.inputs = None
+
+    # -- committed context ---------------------------------------------------------------
+    def fill_synthetic_context(self) -> None:
+        wl = self.wl
+        for cache_id, (kc, vc, nl) in enumerate(((self.k_full, self.v_full, wl.shape.n_layers),
+                                                 (self.k_slim, self.v_slim, len(self.routed)))):
+            for o in range(nl):
+                kc[o, :, :, :wl.ctx] = to_device(W.context_kv(wl, cache_id, o, 0), self.device)
+                vc[o, :, :, :wl.ctx] = to_device(W.context_kv(wl, cache_id, o, 1), self.device)
+        self.len.fill_(wl.ctx)
+
+    def prefill(self, prompt: np.ndarray) -> None:
+        """Push a prompt [B, T] through both models with the library's own forward + commit calls."""
+        B, T = prompt.shape
+        V = self.wl.shape.vocab
+        self.pending.copy_(torch.from_numpy(prompt[:, 0].astype(np.int32)))
+        pos = 1
+        while pos < T:
+            n = min(self.max_query - 1, T - pos)
+            tok = torch.from_numpy(prompt[:, pos:pos + n].astype(np.int32)).to(self.device).contiguous()
+            parent = torch.arange(-1, n - 1, dtype=torch.int32, device=self.device)
+            d = vb.make_draft(tok, parent, parent, 0, None)
+            logits = torch.empty((B, n + 1, V), dtype=torch.float32, device=self.device)
+            vb.full_forward(self.model, self.cache, d, logits)
+            vb.slim_forward(self.model, self.cache, d, logits)
+            res = vb.alloc_result(B, n, self.device)
+            res.n_acc.fill_(n)
+            res.n_emit.fill_(n)
+            res.path.copy_(torch.arange(n, dtype=torch.int32, device=self.device).expand(B, n))
+            res.out_tok[:, :n] = tok
+            vb.kv_commit(self.model, self.cache, d, res)
+            pos += n
+
+    # -- step inputs -------------------------------------------------------------------------
+    def set_inputs(self, si: W.StepInputs, set_pending: bool = True) -> None:
+        dev = self.device
+        self.inputs = si
+        self.draft_tok = torch.from_numpy(si.draft_tok.astype(np.int32)).to(dev).contiguous()
+        self.parent = torch.from_numpy(si.parent.astype(np.int32)).to(dev)
+        self.prow = torch.from_numpy(si.prow.astype(np.int32)).to(dev)
+        self.drafter_logits = torch.from_numpy(si.drafter_logits).to(dev)
+        if set_pending:
+            self.pending.copy_(torch.from_numpy(si.pending.astype(np.int32)))
+        self.draft = vb.make_draft(self.draft_tok, self.parent, self.prow, si.n_prows, self.drafter_logits)
+
+    def logits_buffer(self) -> torch.Tensor:
+        return torch.empty((self.wl.batch, self.wl.rows, self.wl.shape.vocab), dtype=torch.float32,
+                           device=self.device)
+
+    def params(self, step: int = 0, **kw) -> vb.Params:
+        lo, hi = W.thresholds(self.wl)
+        kw.setdefault("mode", 1 if self.wl.mode == "sampling" else 0)
+        kw.setdefault("temperature", self.wl.temperature)
+        kw.setdefault("seed", self.wl.seed)
+        return vb.make_params(kw.pop("log_tau_lo", lo), kw.pop("log_tau_hi", hi), step=step, **kw)

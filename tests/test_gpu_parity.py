@@ -1,0 +1,439 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded inputs."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+
+import synth
+from synth import workloads as W
+from oracle import decoder, step, tiers
+from tests import parity_util as PU
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+def _engine(wl, **kw):
+    from paper_2606_12243_b200.engine import Engine
+    return Engine(wl, **kw)
+
+
+def _vb():
+    from paper_2606_12243_b200 import binding
+    return binding
+
+
+def _prepare(wl, dt=np.float64, extra=0, step_no=0):
+    """Engine + oracle state in the same starting condition, with the step inputs loaded."""
+    eng = _engine(wl, extra_ctx=extra)
+    st = PU.oracle_state(wl, dt, extra)
+    si = W.step_inputs(wl, step_no)
+    model = W.Model(wl, keep=wl.shape.n_layers <= 8)
+    if wl.real_prefill:
+        step.prefill(model, wl.shape, wl.routed, st, np.concatenate([si.prompt, si.pending[:, None]], axis=1), dt)
+        eng.prefill(np.concatenate([si.prompt, si.pending[:, None]], axis=1))
+    else:
+        st.pending[:] = si.pending
+    eng.set_inputs(si, set_pending=not wl.real_prefill)
+    return eng, st, si, model
+
+
+# ---------------------------------------------------------------------------------------------
+# GEMM on its own
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("rows,n,k", [(1, 64, 64), (5, 1024, 256), (9, 4096, 512), (9, 1000, 1408), (27, 776, 4096),
+                                      (56, 520, 640), (64, 256, 11008), (96, 384, 1024), (108, 2048, 512)])
+def test_gemm_matches_matmul(dtype, rows, n, k):
+    vb = _vb()
+    from paper_2606_12243_b200.engine import to_device
+    if dtype == "bf16":
+        xw, ww = synth.normal_bf16(1, 1, (rows, k), 1.0), synth.normal_bf16(1, 2, (n, k), 0.05)
+        x64, w64 = synth.bf16_to_f32(xw).astype(np.float64), synth.bf16_to_f32(ww).astype(np.float64)
+    else:
+        xw, ww = synth.normal_f32(1, 1, (rows, k), 1.0), synth.normal_f32(1, 2, (n, k), 0.05)
+        x64, w64 = xw.astype(np.float64), ww.astype(np.float64)
+    x, w = to_device(xw), to_device(ww)
+    y = torch.full((rows, n), float("nan"), dtype=torch.float32, device="cuda")
+    scratch = torch.empty(max(256, vb.gemm_scratch_bytes(rows, n, k)), dtype=torch.uint8, device="cuda")
+    vb.gemm(x, w, y, scratch)
+    want = x64 @ w64.T
+    got = y.cpu().numpy()
+    # exact products, fp32 accumulation of k terms
+    tol = 2e-6 * np.sqrt(k) * np.abs(want).max() + 1e-6
+    assert np.abs(got - want).max() <= tol, (np.abs(got - want).max(), tol)
+
+
+# ---------------------------------------------------------------------------------------------
+# forward passes
+# ---------------------------------------------------------------------------------------------
+FORWARD_CASES = ["c1_tiny", "tiny_tree_f32", "mini_7b", "mini_8b_tree", "mini_13b", "mini_32b", "mini_32b_b3"]
+
+
+@pytest.mark.parametrize("name", FORWARD_CASES)
+def test_forward_logits_and_appended_kv(name):
+    wl = W.get(name)
+    vb = _vb()
+    eng, st, si, model = _prepare(wl)
+    rows = step.block_rows(st.pending, si.draft_tok)
+    for slim in (False, True):
+        layers = wl.routed if slim else range(wl.shape.n_layers)
+        ocache = st.slim if slim else st.full
+        want = decoder.forward(model, wl.shape, layers, ocache, st.lens, rows, wl.parent)
+        got = eng.logits_buffer()
+        (vb.slim_forward if slim else vb.full_forward)(eng.model, eng.cache, eng.draft, got)
+        torch.cuda.synchronize()
+        PU.assert_logits_close(got.cpu().numpy(), want, wl.shape.dtype, f"{name} slim={slim}")
+        # K/V rows appended at slots len .. len+M-1 (len itself untouched)
+        assert eng.len.cpu().tolist() == [int(x) for x in st.lens]
+        kc, vc = (eng.k_slim, eng.v_slim) if slim else (eng.k_full, eng.v_full)
+        tol = 2e-2 if wl.shape.dtype == "bf16" else 1e-4
+        for o in (0, len(layers) - 1):
+            for b in (0, wl.batch - 1):
+                n = int(st.lens[b])
+                gk = kc[o, b, :, n:n + wl.rows].float().cpu().numpy()
+                gv = vc[o, b, :, n:n + wl.rows].float().cpu().numpy()
+                ok = ocache.k[o][b, :, n - ocache.base_len:n - ocache.base_len + wl.rows]
+                ov = ocache.v[o][b, :, n - ocache.base_len:n - ocache.base_len + wl.rows]
+                assert np.abs(gk - ok).max() <= tol * max(1.0, np.abs(ok).max())
+                assert np.abs(gv - ov).max() <= tol * max(1.0, np.abs(ov).max())
+    assert vb.get_stats(eng.model).device_status == 0
+
+
+def test_forward_is_deterministic_and_slim_all_layers_equals_full():
+    wl = replace(W.get("mini_8b_tree"), n_routed=W.get("mini_8b_tree").shape.n_layers, name="mini_8b_tree")
+    vb = _vb()
+    eng, st, si, model = _prepare(wl)
+    a, b, c = eng.logits_buffer(), eng.logits_buffer(), eng.logits_buffer()
+    vb.full_forward(eng.model, eng.cache, eng.draft, a)
+    vb.full_forward(eng.model, eng.cache, eng.draft, b)
+    # the slim cache holds different synthetic context, so give q' the full cache to compare like with like
+    cache2 = vb.make_cache(eng.k_full, eng.v_full, eng.k_full, eng.v_full, eng.len, eng.pending, eng.tokens)
+    vb.slim_forward(eng.model, cache2, eng.draft, c)
+    torch.cuda.synchronize()
+    assert torch.equal(a, b)
+    assert torch.equal(a, c)
+
+
+# ---------------------------------------------------------------------------------------------
+# tier kernel: bit-exact
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("name", ["c1_tiny", "mini_7b", "mini_8b_tree", "mini_13b", "mini_32b", "c2_7b", "c3_8b_tree"])
+def test_tier_kernel_bit_exact(name):
+    wl = W.get(name)
+    vb = _vb()
+    si = W.step_inputs(wl)
+    lo, hi = W.thresholds(wl)
+    want_tier, want_d = tiers.tier_rule(si.drafter_logits, si.draft_tok, si.prow, lo, hi)
+    eng = _tier_only_engine(wl)
+    eng.set_inputs(si)
+    res = vb.alloc_result(wl.batch, wl.n_nodes)
+    vb.tier_accept(eng.model, eng.draft, eng.params(), None, None, 1, res)
+    torch.cuda.synchronize()
+    assert np.array_equal(res.tier.cpu().numpy(), want_tier)
+    assert np.array_equal(res.conf.cpu().numpy(), want_d)           # same fp32 subtraction on both sides
+    s = vb.get_stats(eng.model)
+    assert list(s.tier_count) == [int((want_tier == t).sum()) for t in range(3)]
+    assert s.need_slim == int((want_tier == 1).any()) and s.need_full == int((want_tier == 2).any())
+    # degenerate thresholds: everything accepted / everything escalated
+    vb.tier_accept(eng.model, eng.draft, eng.params(log_tau_lo=-1e30, log_tau_hi=-1e30), None, None, 1, res)
+    assert int(res.tier.max()) == 0
+    vb.tier_accept(eng.model, eng.draft, eng.params(log_tau_lo=1.0, log_tau_hi=1.0), None, None, 1, res)
+    assert int(res.tier.min()) == 2
+
+
+def _tier_only_engine(wl):
+    """The tier / accept kernels need no model weights: a 1-layer stand-in of the same vocabulary."""
+    small = replace(wl.shape, n_layers=1, d_model=64, n_heads=1, n_kv_heads=1, head_dim=64, d_ff=64)
+    return _engine(replace(wl, shape=small, n_routed=1, ctx=0, real_prefill=False), fill_context=False)
+
+
+# ---------------------------------------------------------------------------------------------
+# accept kernel on oracle-supplied logits
+# ---------------------------------------------------------------------------------------------
+def _accept_case(wl, mode, seed, n_steps=6, **pk):
+    vb = _vb()
+    eng = _tier_only_engine(wl)
+    B, N, M, V = wl.batch, wl.n_nodes, wl.rows, wl.shape.vocab
+    lo, hi = W.thresholds(wl)
+    pinned = total = full = 0
+    for it in range(n_steps):
+        si = W.step_inputs(wl, it)
+        # verifier logits: noise plus a bump on some drafted tokens, so that acceptances of every length occur
+        slim = synth.normal_f32(seed, 10 + it, (B, M, V), 1.5)
+        full_l = synth.normal_f32(seed, 50 + it, (B, M, V), 1.5)
+        depth, _ = decoder.tree_layout(wl.parent)
+        for b in range(B):
+            for n in range(N):
+                if (n + b + it) % 4 != 3:
+                    bump = 6.0 if mode == "greedy" else 3.0
+                    slim[b, wl.parent[n] + 1, si.draft_tok[b, n]] += bump
+                    full_l[b, wl.parent[n] + 1, si.draft_tok[b, n]] += bump
+        tier, _ = tiers.tier_rule(si.drafter_logits, si.draft_tok, si.prow, lo, hi)
+        P = tiers.Params(mode=mode, seed=wl.seed, step=it, **pk)
+        want = tiers.resolve(si.draft_tok, wl.parent, si.prow, tier, si.drafter_logits, slim, full_l, P)
+        eng.set_inputs(si)
+        res = vb.alloc_result(B, N)
+        gp = eng.params(step=it, mode=1 if mode == "sampling" else 0,
+                        **{k: (tuple(v) if k == "log_acc_rel" else (int(v) if isinstance(v, bool) else v))
+                           for k, v in pk.items()})
+        vb.tier_accept(eng.model, eng.draft, gp, torch.from_numpy(slim).cuda(), torch.from_numpy(full_l).cuda(),
+                       3, res)
+        torch.cuda.synchronize()
+        assert np.array_equal(res.tier.cpu().numpy(), tier)
+        # fp32 logs and sums over the vocabulary against fp64: decisions with margin > 1e-4 must agree
+        p, t, f = PU.compare_resolution(want, res.n_acc.cpu().numpy(), res.path.cpu().numpy(),
+                                        res.out_tok.cpu().numpy(), res.n_emit.cpu().numpy(),
+                                        res.corr_src.cpu().numpy(), eps_row=2.5e-5)
+        for b, s in enumerate(want):
+            if all(d.margin > 1e-4 for d in s.decisions):
+                assert np.array_equal(res.judge[b].cpu().numpy(), s.judge), (b, res.judge[b], s.judge)
+        pinned += p; total += t; full += f
+    assert vb.get_stats(eng.model).device_status == 0
+    return pinned, total, full, n_steps * B
+
+
+@pytest.mark.parametrize("name", ["c1_tiny", "mini_7b", "mini_8b_tree_greedy", "mini_13b"])
+def test_accept_greedy_on_oracle_logits(name):
+    wl = W.get(name)
+    pinned, total, full, nseq = _accept_case(replace(wl, mode="greedy"), "greedy", 900)
+    assert full >= 0.95 * nseq, (full, nseq)
+
+
+@pytest.mark.parametrize("name", ["mini_8b_tree", "mini_7b", "mini_32b"])
+def test_accept_sampling_on_oracle_logits(name):
+    wl = replace(W.get(name), mode="sampling")
+    pinned, total, full, nseq = _accept_case(wl, "sampling", 901)
+    assert full >= 0.9 * nseq, (full, nseq)
+
+
+def test_accept_options_on_oracle_logits():
+    wl = replace(W.get("mini_8b_tree"), mode="greedy")
+    for pk in (dict(emit_bonus=True), dict(strict_break=True), dict(log_acc_rel=(0.0, -0.7, -0.3))):
+        _, _, full, nseq = _accept_case(wl, "greedy", 902, n_steps=3, **pk)
+        assert full >= 0.9 * nseq
+    wl = replace(W.get("mini_8b_tree"), mode="sampling")
+    for pk in (dict(emit_bonus=True), dict(alpha=0.2, beta=0.8), dict(temperature=0.7)):
+        _, _, full, nseq = _accept_case(wl, "sampling", 903, n_steps=3, **pk)
+        assert full >= 0.9 * nseq
+
+
+def test_sampling_draws_follow_the_judge_distribution():
+    """Property at any size: with one tier-2 child, the emitted token is distributed as softmax(full)."""
+    vb = _vb()
+    V, B = 1024, 64
+    wl = replace(W.get("c1_tiny"), batch=B, parent=W.chain(1), mode="sampling")
+    eng = _tier_only_engine(wl)
+    si = W.step_inputs(wl)
+    rng = np.random.default_rng(0)
+    full_row = (rng.standard_normal(V) * 2.0).astype(np.float32)
+    q = tiers.softmax64(full_row, 1.0)
+    p = tiers.softmax64(si.drafter_logits[0, 0], 1.0)
+    si.drafter_logits[:] = si.drafter_logits[0, 0]
+    full_l = np.broadcast_to(full_row, (B, 2, V)).copy()
+    counts = np.zeros(V)
+    n_rej = 0
+    trials = 0
+    for it in range(40):
+        si.draft_tok[:, 0] = rng.choice(V, size=B, p=p)
+        eng.set_inputs(si)
+        res = vb.alloc_result(B, 1)
+        res.tier.fill_(2)
+        vb.tier_accept(eng.model, eng.draft, eng.params(step=it, mode=1), torch.from_numpy(full_l).cuda(),
+                       torch.from_numpy(full_l).cuda(), 2, res)
+        out = res.out_tok[:, 0].cpu().numpy()
+        assert np.all(res.n_emit.cpu().numpy() == 1)
+        np.add.at(counts, out, 1)
+        n_rej += int((res.n_acc.cpu().numpy() == 0).sum())
+        trials += B
+    # compare on the 8 most likely tokens and on the rejection rate (= TV distance, Eq. 2-3)
+    top = np.argsort(q)[-8:]
+    assert np.abs(counts[top] / trials - q[top]).max() < 4.0 * np.sqrt(q[top].max() / trials) + 0.004
+    assert abs(n_rej / trials - 0.5 * np.abs(p - q).sum()) < 0.04
+
+
+# ---------------------------------------------------------------------------------------------
+# whole step and multi-step loop
+# ---------------------------------------------------------------------------------------------
+def _check_state(eng, st, wl, check_cache=True):
+    assert eng.len.cpu().tolist() == [int(x) for x in st.lens]
+    assert eng.pending.cpu().tolist() == [int(x) for x in st.pending]
+    tok = eng.tokens.cpu().numpy()
+    for b in range(wl.batch):
+        own = st.tokens[b]
+        n = int(st.lens[b])
+        if wl.real_prefill:
+            assert tok[b, :n].tolist() == own[:n]
+        else:
+            assert tok[b, wl.ctx:n].tolist() == own[:n - wl.ctx]
+    if check_cache:
+        tol = 2e-2 if wl.shape.dtype == "bf16" else 1e-4
+        for cache, kc in ((st.full, eng.k_full), (st.slim, eng.k_slim)):
+            o = cache.n_layers - 1
+            for b in range(wl.batch):
+                n = int(st.lens[b])
+                lo = cache.base_len
+                if n > lo:
+                    g = kc[o, b, :, lo:n].float().cpu().numpy()
+                    w = cache.k[o][b, :, :n - lo]
+                    assert np.abs(g - w).max() <= tol * max(1.0, np.abs(w).max()), (b, o)
+
+
+STEP_CASES = ["c1_tiny", "tiny_tree_f32", "mini_7b", "mini_8b_tree", "mini_8b_tree_greedy", "mini_13b", "mini_32b"]
+
+
+@pytest.mark.parametrize("name", STEP_CASES)
+def test_verify_step_matches_oracle(name):
+    wl = W.get(name)
+    vb = _vb()
+    eng, st, si, model = _prepare(wl)
+    lo, hi = W.thresholds(wl)
+    want = step.verify_step(model, wl.shape, wl.routed, st, si.draft_tok, wl.parent, si.prow, si.drafter_logits,
+                            lo, hi, PU.oracle_params(wl))
+    sl, fl = eng.logits_buffer(), eng.logits_buffer()
+    res = vb.alloc_result(wl.batch, wl.n_nodes)
+    vb.verify_step(eng.model, eng.cache, eng.draft, eng.params(), sl, fl, res)
+    torch.cuda.synchronize()
+    assert vb.get_stats(eng.model).device_status == 0
+    assert np.array_equal(res.tier.cpu().numpy(), want.tier)
+    e1, _ = PU.assert_logits_close(sl.cpu().numpy(), want.slim_logits, wl.shape.dtype, "slim")
+    e2, _ = PU.assert_logits_close(fl.cpu().numpy(), want.full_logits, wl.shape.dtype, "full")
+    pinned, total, full = PU.compare_resolution(want.seqs, res.n_acc.cpu().numpy(), res.path.cpu().numpy(),
+                                                res.out_tok.cpu().numpy(), res.n_emit.cpu().numpy(),
+                                                res.corr_src.cpu().numpy(), eps_row=max(e1, e2))
+    assert total == 0 or pinned / total > 0.6, (pinned, total)
+    if full == wl.batch:
+        _check_state(eng, st, wl)
+
+
+def test_step_pieces_equal_fused_call():
+    wl = W.get("mini_8b_tree")
+    vb = _vb()
+    outs = []
+    for fused in (True, False):
+        eng, st, si, model = _prepare(wl)
+        sl, fl = eng.logits_buffer(), eng.logits_buffer()
+        res = vb.alloc_result(wl.batch, wl.n_nodes)
+        p = eng.params()
+        if fused:
+            vb.verify_step(eng.model, eng.cache, eng.draft, p, sl, fl, res)
+        else:
+            vb.tier_accept(eng.model, eng.draft, p, None, None, 1, res)
+            vb.slim_forward(eng.model, eng.cache, eng.draft, sl)
+            vb.full_forward(eng.model, eng.cache, eng.draft, fl)
+            vb.tier_accept(eng.model, eng.draft, p, sl, fl, 2, res)
+            vb.kv_commit(eng.model, eng.cache, eng.draft, res)
+        torch.cuda.synchronize()
+        outs.append([x.clone() for x in (sl, fl, res.tier, res.n_acc, res.path, res.out_tok, res.n_emit, res.judge,
+                                         res.corr_src, eng.len, eng.pending, eng.k_full, eng.v_slim)])
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("name", ["c1_tiny", "tiny_tree_f32"])
+def test_greedy_full_tier_loop_reproduces_autoregressive_decoding(name):
+    """All tokens to the full tier, greedy: the GPU loop (verify_step with commits) emits the oracle's greedy
+    autoregressive continuation of q wherever the oracle's top-2 logit gap exceeds the fp32 tolerance."""
+    wl = W.get(name)
+    vb = _vb()
+    n_steps = 6
+    eng, st, si, model = _prepare(wl, extra=n_steps * wl.rows)
+    ref_state = PU.oracle_state(wl, extra=n_steps * wl.rows)
+    prompt = np.concatenate([si.prompt, si.pending[:, None]], axis=1)
+    step.prefill(model, wl.shape, wl.routed, ref_state, prompt)
+    n_ref = n_steps * (max(decoder.tree_layout(wl.parent)[0]) + 1)
+    gaps = []
+    ref = [[] for _ in range(wl.batch)]
+    for _ in range(n_ref):
+        rows = np.asarray(ref_state.pending, dtype=np.int64)[:, None]
+        lg = decoder.forward(model, wl.shape, range(wl.shape.n_layers), ref_state.full, ref_state.lens, rows, ())
+        nxt = lg[:, 0].argmax(-1)
+        srt = np.sort(lg[:, 0], axis=-1)
+        gaps.append(srt[:, -1] - srt[:, -2])
+        for b in range(wl.batch):
+            ref[b].append(int(nxt[b]))
+        ref_state.lens += 1
+        ref_state.pending[:] = nxt
+    gaps = np.array(gaps)                     # [n_ref, B]
+    emitted = [[] for _ in range(wl.batch)]
+    depth = decoder.tree_layout(wl.parent)[0][1:]
+    sl, fl = eng.logits_buffer(), eng.logits_buffer()
+    for it in range(n_steps):
+        s2 = W.step_inputs(wl, it + 1)
+        for b in range(wl.batch):                       # plant the true continuation on part of the draft
+            k = len(emitted[b])
+            for n in range(wl.n_nodes):
+                if (it + n + b) % 3 != 0 and wl.parent[n] <= 0 and k + depth[n] - 1 < n_ref:
+                    s2.draft_tok[b, n] = ref[b][k + depth[n] - 1]
+        eng.set_inputs(s2, set_pending=False)
+        res = vb.alloc_result(wl.batch, wl.n_nodes)
+        vb.verify_step(eng.model, eng.cache, eng.draft, eng.params(log_tau_lo=1.0, log_tau_hi=2.0), sl, fl, res)
+        ne = res.n_emit.cpu().numpy()
+        ot = res.out_tok.cpu().numpy()
+        assert int(res.tier.min()) == 2
+        for b in range(wl.batch):
+            assert ne[b] >= 1
+            emitted[b].extend(int(t) for t in ot[b, :ne[b]])
+    assert vb.get_stats(eng.model).device_status == 0
+    assert max(len(e) for e in emitted) > n_steps                # some drafts were accepted
+    for b in range(wl.batch):
+        for i, t in enumerate(emitted[b][:n_ref]):
+            if gaps[i, b] <= 4e-4:
+                break                                            # unpinned decision: stop comparing
+            assert t == ref[b][i], (b, i)
+    assert eng.len.cpu().tolist() == [wl.ctx + len(e) for e in emitted]
+
+
+# ---------------------------------------------------------------------------------------------
+# commit on its own; edge cases
+# ---------------------------------------------------------------------------------------------
+def test_kv_commit_moves_tree_rows_bit_exact():
+    wl = W.get("mini_8b_tree")
+    vb = _vb()
+    eng, st, si, model = _prepare(wl)
+    fl = eng.logits_buffer()
+    vb.full_forward(eng.model, eng.cache, eng.draft, fl)
+    vb.slim_forward(eng.model, eng.cache, eng.draft, fl)
+    before_k, before_v = eng.k_full.clone(), eng.v_slim.clone()
+    res = vb.alloc_result(wl.batch, wl.n_nodes)
+    paths = [[1, 7, 18], [3], [], [0, 4, 16, 24, 25]]
+    out = [[11, 12, 13, 14], [21, 22], [31], [41, 42, 43, 44, 45]]
+    for b in range(4):
+        res.n_acc[b] = len(paths[b]); res.n_emit[b] = len(out[b])
+        res.path[b, :len(paths[b])] = torch.tensor(paths[b], dtype=torch.int32)
+        res.out_tok[b, :len(out[b])] = torch.tensor(out[b], dtype=torch.int32)
+    pend0 = eng.pending.clone()
+    vb.kv_commit(eng.model, eng.cache, eng.draft, res)
+    torch.cuda.synchronize()
+    n = wl.ctx
+    for b in range(4):
+        assert int(eng.len[b]) == n + len(out[b]) and int(eng.pending[b]) == out[b][-1]
+        assert eng.tokens[b, n:n + len(out[b])].tolist() == [int(pend0[b])] + out[b][:-1]
+        for j, node in enumerate(paths[b]):
+            assert torch.equal(eng.k_full[:, b, :, n + 1 + j], before_k[:, b, :, n + 1 + node])
+            assert torch.equal(eng.v_slim[:, b, :, n + 1 + j], before_v[:, b, :, n + 1 + node])
+        assert torch.equal(eng.k_full[:, b, :, :n + 1], before_k[:, b, :, :n + 1])   # context and row 0 untouched
+
+
+def test_argument_and_capacity_errors():
+    vb = _vb()
+    wl = W.get("mini_7b")
+    eng, st, si, model = _prepare(wl)
+    fl = eng.logits_buffer()
+    bad = vb.make_draft(eng.draft_tok, eng.parent, eng.prow, si.n_prows, eng.drafter_logits)
+    bad.n_nodes = 64                                     # M = 65 > 64
+    with pytest.raises(vb.ViasdError) as e:
+        vb.full_forward(eng.model, eng.cache, bad, fl)
+    assert e.value.code == vb.VIASD_EINVAL
+    with pytest.raises(vb.ViasdError):
+        vb.tier_accept(eng.model, eng.draft, eng.params(log_tau_lo=0.0, log_tau_hi=-1.0), None, None, 1,
+                       vb.alloc_result(wl.batch, wl.n_nodes))
+    cfg = vb.make_config(2, 256, 4, 4, 48, 512, 1000, "bf16", 1, 64, 8)   # head_dim 48 unsupported
+    assert vb.workspace_bytes(cfg, 1) == 0
+    # a sequence already at capacity: the pass clamps, stays in bounds and records the condition
+    eng.len.fill_(eng.max_ctx - 2)
+    vb.full_forward(eng.model, eng.cache, eng.draft, fl)
+    torch.cuda.synchronize()
+    assert vb.get_stats(eng.model).device_status == vb.VIASD_ECAPACITY
+    assert vb.lib().viasd_strerror(vb.VIASD_ECAPACITY).decode() == "capacity exceeded"
