@@ -2,6 +2,7 @@
 #include "common.cuh"
 #include <new>
 #include <string.h>
+#include <stdlib.h>
 
 int g_last_cuda_error = 0;
 unsigned long long g_launch_count = 0;
@@ -21,6 +22,8 @@ struct Carver {
     }
 };
 
+constexpr int MAX_SMS = 160;            // workspace is sized without asking the device
+
 size_t part_bytes_for(const viasd_config &c) {
     const size_t R = (size_t)c.max_batch * c.max_query;
     // attention split-KV partials: up to 16 key ranges of (head_dim + 2) floats per (row, head)
@@ -38,11 +41,13 @@ size_t carve(const viasd_config &c, char *base, Workspace *ws) {
     w.rope_cos = cv.take<float>((size_t)c.max_ctx * (c.head_dim / 2) * 4);
     w.rope_sin = cv.take<float>((size_t)c.max_ctx * (c.head_dim / 2) * 4);
     w.h = cv.take<float>(R * c.d_model * 4);
-    w.a = cv.take<void>(R * c.d_model * es);
+    (void)es;
+    w.rows_alloc = R;
+    w.a = cv.take<void>(R * c.d_model * 4);            // fp32 plane, or bf16 hi + lo planes
     w.qkv = cv.take<float>(R * (qd + 2 * kvd) * 4);
-    w.q = cv.take<void>(R * qd * es);
-    w.attn = cv.take<void>(R * qd * es);
-    w.act = cv.take<void>(R * c.d_ff * es);
+    w.q = cv.take<float>(R * qd * 4);
+    w.attn = cv.take<void>(R * qd * 4);
+    w.act = cv.take<void>(R * c.d_ff * 4);
     w.part_bytes = part_bytes_for(c);
     w.part = cv.take<float>(w.part_bytes);
     w.len_eff = cv.take<int>((size_t)c.max_batch * 4);
@@ -50,6 +55,15 @@ size_t carve(const viasd_config &c, char *base, Workspace *ws) {
     w.tree = cv.take<TreeInfo>(sizeof(TreeInfo));
     w.stats = cv.take<DeviceStats>(sizeof(DeviceStats));
     w.accept_scratch = cv.take<float>((size_t)c.max_batch * 3 * c.vocab * 4);
+    {
+        const int nt = tc_pick_nt(R < 128 ? (int)R : 128);
+        w.gemm_scratch = cv.take<float>(tc_scratch_floats(MAX_SMS, nt, true) * 4);
+        size_t widest = (size_t)c.vocab;
+        if (qd + 2 * kvd > widest) widest = qd + 2 * kvd;
+        if ((size_t)c.d_ff > widest) widest = c.d_ff;
+        w.n_counters = widest / 128 + 8;
+        w.gemm_counters = cv.take<int>(w.n_counters * 4);
+    }
     if (ws) *ws = w;
     return align_up(cv.off, 256);
 }
@@ -95,6 +109,44 @@ int check_cache(const viasd_cache *c) {
     return VIASD_OK;
 }
 
+// One projection.  bf16 models go to the tcgen05 kernel (activation hi/lo planes through TMA); fp32 models
+// and anything that kernel does not take go to the CUDA-core kernel.
+struct GemmCall {
+    const void *x; size_t x_plane; const ActMaps *xmaps;      // input activation buffer
+    const void *w[3]; const WMap *wmap[3]; int n[3]; int count;
+    int k, epi;
+    float *out_f32; void *out_act; size_t act_plane; int ld_out;
+};
+
+int run_gemm(viasd_model *m, const GemmCall &g, int rows, cudaStream_t st) {
+    const viasd_config &c = m->cfg;
+    if (!m->use_tc) {
+        GemmSegs s{{g.w[0], g.w[1], g.w[2]}, {g.n[0], g.n[1], g.n[2]}, g.count};
+        return launch_gemm_rowwarp(g.x, g.x_plane, s, rows, g.k, c.dtype, g.epi, g.out_f32, g.out_act, g.act_plane,
+                                   g.ld_out, st);
+    }
+    for (int row0 = 0; row0 < rows; row0 += 128) {
+        const int nr = rows - row0 < 128 ? rows - row0 : 128;
+        const int nt = tc_pick_nt(nr);
+        const int ni = nt == 16 ? 0 : nt == 32 ? 1 : nt == 64 ? 2 : 3;
+        TcLaunch L;
+        memset(&L, 0, sizeof(L));
+        for (int i = 0; i < g.count; ++i) { L.map_w[i] = &g.wmap[i]->map; L.seg_n[i] = g.n[i]; L.w_box_rows[i] = g.wmap[i]->box_rows; }
+        L.n_seg = g.count;
+        L.map_x = &g.xmaps->map[ni];
+        L.x_box_rows = g.xmaps->box_rows[ni];
+        L.has_lo = 1;
+        L.lo_row_offset = (int)m->ws.rows_alloc;
+        L.rows = nr; L.row0 = row0; L.k = g.k; L.nt = nt; L.epi = g.epi;
+        L.out_f32 = g.out_f32; L.out_act = g.out_act; L.act_plane = g.act_plane; L.ld_out = g.ld_out;
+        L.scratch = m->ws.gemm_scratch; L.counters = m->ws.gemm_counters; L.status = &m->ws.stats->device_status;
+        L.sm_count = m->sm_count;
+        int rc = launch_gemm_tc(L, st);
+        if (rc) return rc;
+    }
+    return VIASD_OK;
+}
+
 // One pass of the sub-network made of `layers` (all of them for q, the routed ones for q').
 int forward(viasd_model *m, const viasd_cache *cache, const viasd_draft *d, bool slim, float *logits,
             cudaStream_t st) {
@@ -106,32 +158,36 @@ int forward(viasd_model *m, const viasd_cache *cache, const viasd_draft *d, bool
     const int qd = c.n_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
     void *kc = slim ? cache->k_slim : cache->k_full, *vc = slim ? cache->v_slim : cache->v_full;
     const int n_run = slim ? m->n_routed : c.n_layers;
+    const size_t R = m->ws.rows_alloc;
+    const size_t pa = c.dtype ? R * c.d_model : 0, pq = c.dtype ? R * qd : 0, pf = c.dtype ? R * c.d_ff : 0;
 
     if ((rc = timed(m, VIASD_T_EMBED, st, [&] { return launch_prep(m, cache, d, st); }))) return rc;
     if ((rc = timed(m, VIASD_T_EMBED, st, [&] { return launch_embed(m, rows, st); }))) return rc;
     for (int ord = 0; ord < n_run; ++ord) {
         const int l = slim ? m->routed[ord] : ord;
+        const LayerMaps *lm = m->use_tc ? &m->lmaps[l] : nullptr;
         if ((rc = timed(m, VIASD_T_NORM, st, [&] { return launch_rmsnorm(m, m->norm1[l], rows, st); }))) return rc;
-        GemmSegs qkv{{m->wq[l], m->wk[l], m->wv[l]}, {qd, kvd, kvd}, 3};
-        if ((rc = timed(m, VIASD_T_GEMM, st, [&] { return launch_gemm_rowwarp(m->ws.a, qkv, rows, c.d_model, c.dtype,
-                EPI_STORE, m->ws.qkv, nullptr, qd + 2 * kvd, st); }))) return rc;
+        GemmCall qkv{m->ws.a, pa, &m->maps_a, {m->wq[l], m->wk[l], m->wv[l]},
+                     {lm ? &lm->wq : nullptr, lm ? &lm->wk : nullptr, lm ? &lm->wv : nullptr}, {qd, kvd, kvd}, 3,
+                     c.d_model, EPI_STORE, m->ws.qkv, nullptr, 0, qd + 2 * kvd};
+        if ((rc = timed(m, VIASD_T_GEMM, st, [&] { return run_gemm(m, qkv, rows, st); }))) return rc;
         if ((rc = timed(m, VIASD_T_ROPE, st, [&] { return launch_rope_append(m, kc, vc, ord, B, M, st); }))) return rc;
         if ((rc = timed(m, VIASD_T_ATTENTION, st, [&] { return launch_attention(m, kc, vc, ord, B, M, st); }))) return rc;
-        GemmSegs wo{{m->wo[l], nullptr, nullptr}, {c.d_model, 0, 0}, 1};
-        if ((rc = timed(m, VIASD_T_GEMM, st, [&] { return launch_gemm_rowwarp(m->ws.attn, wo, rows, qd, c.dtype, EPI_ADD,
-                m->ws.h, nullptr, c.d_model, st); }))) return rc;
+        GemmCall wo{m->ws.attn, pq, &m->maps_attn, {m->wo[l], nullptr, nullptr}, {lm ? &lm->wo : nullptr, nullptr, nullptr},
+                    {c.d_model, 0, 0}, 1, qd, EPI_ADD, m->ws.h, nullptr, 0, c.d_model};
+        if ((rc = timed(m, VIASD_T_GEMM, st, [&] { return run_gemm(m, wo, rows, st); }))) return rc;
         if ((rc = timed(m, VIASD_T_NORM, st, [&] { return launch_rmsnorm(m, m->norm2[l], rows, st); }))) return rc;
-        GemmSegs gu{{m->wg[l], m->wu[l], nullptr}, {c.d_ff, c.d_ff, 0}, 2};
-        if ((rc = timed(m, VIASD_T_GEMM, st, [&] { return launch_gemm_rowwarp(m->ws.a, gu, rows, c.d_model, c.dtype,
-                EPI_SWIGLU, nullptr, m->ws.act, c.d_ff, st); }))) return rc;
-        GemmSegs wd{{m->wd[l], nullptr, nullptr}, {c.d_model, 0, 0}, 1};
-        if ((rc = timed(m, VIASD_T_GEMM, st, [&] { return launch_gemm_rowwarp(m->ws.act, wd, rows, c.d_ff, c.dtype, EPI_ADD,
-                m->ws.h, nullptr, c.d_model, st); }))) return rc;
+        GemmCall gu{m->ws.a, pa, &m->maps_a, {m->wg[l], m->wu[l], nullptr}, {lm ? &lm->wg : nullptr, lm ? &lm->wu : nullptr, nullptr},
+                    {c.d_ff, c.d_ff, 0}, 2, c.d_model, EPI_SWIGLU, nullptr, m->ws.act, pf, c.d_ff};
+        if ((rc = timed(m, VIASD_T_GEMM, st, [&] { return run_gemm(m, gu, rows, st); }))) return rc;
+        GemmCall wd{m->ws.act, pf, &m->maps_act, {m->wd[l], nullptr, nullptr}, {lm ? &lm->wd : nullptr, nullptr, nullptr},
+                    {c.d_model, 0, 0}, 1, c.d_ff, EPI_ADD, m->ws.h, nullptr, 0, c.d_model};
+        if ((rc = timed(m, VIASD_T_GEMM, st, [&] { return run_gemm(m, wd, rows, st); }))) return rc;
     }
     if ((rc = timed(m, VIASD_T_NORM, st, [&] { return launch_rmsnorm(m, m->final_norm, rows, st); }))) return rc;
-    GemmSegs head{{m->lm_head, nullptr, nullptr}, {c.vocab, 0, 0}, 1};
-    return timed(m, VIASD_T_GEMM, st, [&] { return launch_gemm_rowwarp(m->ws.a, head, rows, c.d_model, c.dtype, EPI_STORE,
-                                                                   logits, nullptr, c.vocab, st); });
+    GemmCall head{m->ws.a, pa, &m->maps_a, {m->lm_head, nullptr, nullptr}, {m->use_tc ? &m->head_map : nullptr, nullptr, nullptr},
+                  {c.vocab, 0, 0}, 1, c.d_model, EPI_STORE, logits, nullptr, 0, c.vocab};
+    return timed(m, VIASD_T_GEMM, st, [&] { return run_gemm(m, head, rows, st); });
 }
 
 int check_params(const viasd_params *p) {
@@ -205,7 +261,42 @@ int viasd_init_model(const viasd_config *cfg, const viasd_weights *w, const unsi
     }
     m->embed = w->embed; m->lm_head = w->lm_head; m->final_norm = w->final_norm;
     carve(*cfg, (char *)workspace, &m->ws);
+    {
+        const char *force = getenv("VIASD_GEMM");
+        m->use_tc = cfg->dtype == 1 && m->sm_count <= MAX_SMS && !(force && strcmp(force, "rowwarp") == 0);
+    }
+    if (m->use_tc) {
+        const uint64_t d = cfg->d_model, qd = (uint64_t)cfg->n_heads * cfg->head_dim,
+                       kvd = (uint64_t)cfg->n_kv_heads * cfg->head_dim, ff = cfg->d_ff, R = m->ws.rows_alloc;
+        m->lmaps = new (std::nothrow) LayerMaps[L];
+        auto wm = [&](WMap &o, const void *base, uint64_t n, uint64_t k) {
+            o.box_rows = tc_box_rows(n, 128);
+            return tc_make_map(&o.map, base, n, k, o.box_rows);
+        };
+        rc = m->lmaps ? VIASD_OK : VIASD_EINVAL;
+        for (int l = 0; l < L && !rc; ++l) {
+            LayerMaps &lm = m->lmaps[l];
+            if ((rc = wm(lm.wq, m->wq[l], qd, d)) || (rc = wm(lm.wk, m->wk[l], kvd, d)) || (rc = wm(lm.wv, m->wv[l], kvd, d)) ||
+                (rc = wm(lm.wo, m->wo[l], d, qd)) || (rc = wm(lm.wg, m->wg[l], ff, d)) || (rc = wm(lm.wu, m->wu[l], ff, d)) ||
+                (rc = wm(lm.wd, m->wd[l], d, ff))) break;
+        }
+        if (!rc) rc = wm(m->head_map, m->lm_head, cfg->vocab, d);
+        auto am = [&](ActMaps &o, const void *base, uint64_t k) {
+            const int nts[4] = {16, 32, 64, 128};
+            for (int i = 0; i < 4; ++i) {
+                o.box_rows[i] = tc_box_rows(2 * R, nts[i]);
+                int r2 = tc_make_map(&o.map[i], base, 2 * R, k, o.box_rows[i]);
+                if (r2) return r2;
+            }
+            return (int)VIASD_OK;
+        };
+        if (!rc) rc = am(m->maps_a, m->ws.a, d);
+        if (!rc) rc = am(m->maps_attn, m->ws.attn, qd);
+        if (!rc) rc = am(m->maps_act, m->ws.act, ff);
+        if (rc) { viasd_free_model(m); return rc; }
+    }
     cudaError_t e = cudaMemset(m->ws.stats, 0, sizeof(DeviceStats));
+    if (e == cudaSuccess) e = cudaMemset(m->ws.gemm_counters, 0, m->ws.n_counters * 4);
     if (e == cudaSuccess) { rc = launch_rope_table(m, 0); if (rc == VIASD_OK) e = cudaDeviceSynchronize(); }
     if (e != cudaSuccess) { g_last_cuda_error = (int)e; rc = VIASD_ECUDA; }
     if (rc) { viasd_free_model(m); return rc; }
@@ -219,6 +310,7 @@ void viasd_free_model(viasd_model *m) {
     for (int i = 0; i < 7; ++i) delete[] *arrs[i];
     delete[] m->norm1;
     delete[] m->norm2;
+    delete[] m->lmaps;
     for (int i = 0; i < m->timer.created; ++i) { cudaEventDestroy(m->timer.beg[i]); cudaEventDestroy(m->timer.end[i]); }
     delete[] m->timer.beg;
     delete[] m->timer.end;
@@ -347,17 +439,53 @@ int viasd_get_timing(viasd_model *m, viasd_timing *out, void *stream) {
 }
 
 size_t viasd_gemm_scratch_bytes(int rows, int n, int k) {
-    (void)rows; (void)n; (void)k;
-    return 256;
+    (void)k;
+    if (rows < 1 || n < 1) return 256;
+    const int nt = tc_pick_nt(rows < 128 ? rows : 128);
+    // [tile counters | one status word] then the partial-tile slots
+    return align_up((size_t)(tc_tiles(n) + 1) * 4, 256) + tc_scratch_floats(MAX_SMS, nt, false) * 4;
 }
 
 int viasd_gemm(const void *x, const void *w, float *y, int rows, int n, int k, int dtype, void *scratch,
                size_t scratch_bytes, void *stream) {
-    if (!x || !w || !y || rows < 1 || rows > 256 || n < 1 || k < 8 || (dtype != 0 && dtype != 1)) return VIASD_EINVAL;
+    if (!x || !w || !y || rows < 1 || rows > 256 || n < 1 || k < 8 || (k % 8) || (dtype != 0 && dtype != 1)) return VIASD_EINVAL;
     if (((uintptr_t)x & 15) || ((uintptr_t)w & 15)) return VIASD_EINVAL;
-    if (scratch_bytes < viasd_gemm_scratch_bytes(rows, n, k) || !scratch) return VIASD_ECAPACITY;
-    GemmSegs s{{w, nullptr, nullptr}, {n, 0, 0}, 1};
-    return launch_gemm_rowwarp(x, s, rows, k, dtype, EPI_STORE, y, nullptr, n, (cudaStream_t)stream);
+    if (!scratch || ((uintptr_t)scratch & 255)) return VIASD_EINVAL;
+    if (scratch_bytes < viasd_gemm_scratch_bytes(rows, n, k)) return VIASD_ECAPACITY;
+    cudaStream_t st = (cudaStream_t)stream;
+    const char *force = getenv("VIASD_GEMM");
+    if (dtype == 0 || (force && strcmp(force, "rowwarp") == 0)) {
+        GemmSegs s{{w, nullptr, nullptr}, {n, 0, 0}, 1};
+        return launch_gemm_rowwarp(x, 0, s, rows, k, dtype, EPI_STORE, y, nullptr, 0, n, st);
+    }
+    int dev = 0, sms = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    if (sms > MAX_SMS) sms = MAX_SMS;
+    const size_t counter_bytes = align_up((size_t)(tc_tiles(n) + 1) * 4, 256);
+    CUDA_TRY(cudaMemsetAsync(scratch, 0, counter_bytes, st));       // tile counters and the status word
+    CUtensorMap mw, mx;
+    int rc;
+    const uint32_t wbox = tc_box_rows(n, 128);
+    if ((rc = tc_make_map(&mw, w, n, k, wbox))) return rc;
+    for (int row0 = 0; row0 < rows; row0 += 128) {
+        const int nr = rows - row0 < 128 ? rows - row0 : 128;
+        const int nt = tc_pick_nt(nr);
+        const uint32_t xbox = tc_box_rows(rows, nt);
+        if ((rc = tc_make_map(&mx, x, rows, k, xbox))) return rc;
+        TcLaunch L;
+        memset(&L, 0, sizeof(L));
+        L.map_w[0] = &mw; L.seg_n[0] = n; L.w_box_rows[0] = wbox; L.n_seg = 1;
+        L.map_x = &mx; L.x_box_rows = xbox; L.has_lo = 0; L.lo_row_offset = 0;
+        L.rows = nr; L.row0 = row0; L.k = k; L.nt = nt; L.epi = EPI_STORE;
+        L.out_f32 = y; L.ld_out = n;
+        L.counters = (int *)scratch;
+        L.scratch = (float *)((char *)scratch + counter_bytes);
+        L.status = (int *)scratch + tc_tiles(n);                    // no handle here: an expired wait is recorded there
+        L.sm_count = sms;
+        if ((rc = launch_gemm_tc(L, st))) return rc;
+    }
+    return VIASD_OK;
 }
 
 }  // extern "C"

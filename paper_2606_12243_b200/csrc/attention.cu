@@ -13,7 +13,7 @@ constexpr int ATT_WARPS = 8;
 
 template <typename T, int HD>
 __global__ void __launch_bounds__(ATT_WARPS * 32)
-attention_split_kernel(float *__restrict__ part, const T *__restrict__ q, const T *__restrict__ kc,
+attention_split_kernel(float *__restrict__ part, const float *__restrict__ q, const T *__restrict__ kc,
                        const T *__restrict__ vc, const int *__restrict__ len_eff, const TreeInfo *__restrict__ tree,
                        int M, int H, int Hkv, int max_batch, int max_ctx, int layer_ord, int nsplit, float scale) {
     __shared__ float Qs[QG][HD];
@@ -35,7 +35,7 @@ attention_split_kernel(float *__restrict__ part, const T *__restrict__ q, const 
         float v = 0.f;
         if (qidx < QR) {
             int h = g * grp + qidx / M, i = qidx % M;
-            v = to_f32<T>(q[((size_t)(b * M + i) * H + h) * HD + dd]) * scale;
+            v = q[((size_t)(b * M + i) * H + h) * HD + dd] * scale;
         }
         Qs[qq][dd] = v;
     }
@@ -105,7 +105,8 @@ attention_split_kernel(float *__restrict__ part, const T *__restrict__ q, const 
 }
 
 template <typename T, int HD>
-__global__ void attention_combine_kernel(T *__restrict__ out, const float *__restrict__ part, int M, int H, int nsplit) {
+__global__ void attention_combine_kernel(T *__restrict__ out, size_t plane, const float *__restrict__ part, int M, int H,
+                                         int nsplit) {
     const int r = blockIdx.x, h = blockIdx.y;        // r = b * M + i
     const int b = r / M, i = r % M;
     const float *src = part + (((size_t)b * H + h) * M + i) * (size_t)nsplit * (HD + 2);
@@ -121,7 +122,7 @@ __global__ void attention_combine_kernel(T *__restrict__ out, const float *__res
             num = fmaf(p[dd], w, num);
             den = fmaf(p[HD + 1], w, den);
         }
-        out[((size_t)r * H + h) * HD + dd] = from_f32<T>(num / den);
+        store_act<T>(out, plane, ((size_t)r * H + h) * HD + dd, num / den);
     }
 }
 
@@ -132,12 +133,12 @@ int run(const viasd_model *m, const void *kc, const void *vc, int layer_ord, int
     const int grp = c.n_heads / c.n_kv_heads;
     const int qgroups = (grp * M + QG - 1) / QG;
     dim3 grid(batch * c.n_kv_heads, nsplit, qgroups);
-    attention_split_kernel<T, HD><<<grid, ATT_WARPS * 32, 0, st>>>(m->ws.part, (const T *)m->ws.q, (const T *)kc,
+    attention_split_kernel<T, HD><<<grid, ATT_WARPS * 32, 0, st>>>(m->ws.part, m->ws.q, (const T *)kc,
         (const T *)vc, m->ws.len_eff, m->ws.tree, M, c.n_heads, c.n_kv_heads, c.max_batch, c.max_ctx, layer_ord, nsplit,
         1.0f / sqrtf((float)HD));
     LAUNCH_CHECK();
     attention_combine_kernel<T, HD><<<dim3(batch * M, c.n_heads), HD < 128 ? HD : 128, 0, st>>>((T *)m->ws.attn,
-        m->ws.part, M, c.n_heads, nsplit);
+        sizeof(T) == 2 ? m->ws.rows_alloc * (size_t)c.n_heads * HD : 0, m->ws.part, M, c.n_heads, nsplit);
     LAUNCH_CHECK();
     return VIASD_OK;
 }

@@ -5,6 +5,7 @@
 #include <stdint.h>
 #include <stddef.h>
 #include "../../include/viasd.h"
+#include "gemm_tc.cuh"
 
 #define VIASD_MAX_ROWS_PER_SEQ 64
 
@@ -31,11 +32,15 @@ struct DeviceStats {
 struct Workspace {                      // pointers into the caller's workspace block
     float *rope_cos, *rope_sin;         // [max_ctx, hd/2]
     float *h;                           // [R, d] residual stream
-    void *a;                            // [R, d] normed activations (model dtype)
+    // GEMM input activations.  fp32 models: one fp32 plane [R, K].  bf16 models: two bf16 planes
+    // [2][R, K], hi = bf16(x) and lo = bf16(x - hi), so that the tensor-core product with the (exact)
+    // bf16 weights keeps ~16 mantissa bits of the activation; the planes are R * K elements apart.
+    void *a;                            // normed activations, K = d
     float *qkv;                         // [R, (H + 2 Hkv) hd]
-    void *q;                            // [R, H hd] rotated queries (model dtype)
-    void *attn;                         // [R, H hd] attention output (model dtype)
-    void *act;                          // [R, ff] SwiGLU output (model dtype)
+    float *q;                           // [R, H hd] rotated queries
+    void *attn;                         // attention output, K = H hd
+    void *act;                          // SwiGLU output, K = ff
+    size_t rows_alloc;                  // R = max_batch * max_query
     float *part;                        // split partial sums (GEMM split-K / attention split-KV)
     size_t part_bytes;
     int *len_eff;                       // [B] committed length clamped to the cache capacity
@@ -43,7 +48,14 @@ struct Workspace {                      // pointers into the caller's workspace 
     TreeInfo *tree;
     DeviceStats *stats;
     float *accept_scratch;              // [B, 3, V] sampling-mode distributions
+    float *gemm_scratch;                // partial tiles of split GEMM work (tcgen05 kernel)
+    int *gemm_counters;                 // per-tile arrival counters, zero between launches
+    size_t n_counters;
 };
+
+struct WMap { CUtensorMap map; uint32_t box_rows; };        // TMA view of one weight matrix
+struct ActMaps { CUtensorMap map[4]; uint32_t box_rows[4]; }; // TMA views of an activation buffer, NT = 16,32,64,128
+struct LayerMaps { WMap wq, wk, wv, wo, wg, wu, wd; };
 
 struct KernelTimer {                    // optional per-launch CUDA-event record (measurement only)
     static constexpr int CAP = 8192;
@@ -65,6 +77,11 @@ struct viasd_model {
     const float **norm1, **norm2;
     Workspace ws;
     int sm_count;
+    // tcgen05 GEMM path (bf16 models)
+    bool use_tc;
+    LayerMaps *lmaps;                   // [L]
+    WMap head_map;
+    ActMaps maps_a, maps_attn, maps_act;
 };
 
 // error helpers -------------------------------------------------------------------------------
@@ -93,8 +110,9 @@ int launch_commit(const viasd_model *m, viasd_cache *c, const viasd_draft *d, co
 // gemm_rowwarp.cu -- generic CUDA-core GEMM (fp32 models; shapes the tensor-core kernels do not take)
 enum GemmEpilogue { EPI_STORE = 0, EPI_ADD = 1, EPI_SWIGLU = 2 };
 struct GemmSegs { const void *w[3]; int n[3]; int count; };
-int launch_gemm_rowwarp(const void *x, const GemmSegs &segs, int rows, int k, int dtype, int epilogue,
-                        float *out_f32, void *out_act, int ld_out, cudaStream_t st);
+// x_plane / act_plane: element distance between the hi and lo planes (0: single plane)
+int launch_gemm_rowwarp(const void *x, size_t x_plane, const GemmSegs &segs, int rows, int k, int dtype,
+                        int epilogue, float *out_f32, void *out_act, size_t act_plane, int ld_out, cudaStream_t st);
 
 // attention.cu
 int launch_attention(const viasd_model *m, const void *kc, const void *vc, int layer_ord, int batch, int M,
@@ -115,6 +133,15 @@ template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16
 template <typename T> __device__ __forceinline__ T from_f32(float v);
 template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// activation store: fp32 plane, or bf16 hi/lo planes
+template <typename T> __device__ __forceinline__ void store_act(T *buf, size_t plane, size_t idx, float v);
+template <> __device__ __forceinline__ void store_act<float>(float *buf, size_t, size_t idx, float v) { buf[idx] = v; }
+template <> __device__ __forceinline__ void store_act<__nv_bfloat16>(__nv_bfloat16 *buf, size_t plane, size_t idx, float v) {
+    __nv_bfloat16 hi = __float2bfloat16_rn(v);
+    buf[idx] = hi;
+    if (plane) buf[plane + idx] = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

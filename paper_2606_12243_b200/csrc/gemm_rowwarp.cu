@@ -47,8 +47,8 @@ __device__ __forceinline__ const T *weight_row(const SegTable &s, int n, int k) 
 // RC rows are kept in registers at a time; more rows loop (weights then come from L2).
 template <typename T, int RC, int EPI>
 __global__ void __launch_bounds__(WARPS * 32)
-gemm_rowwarp_kernel(const T *__restrict__ x, SegTable segs, int rows, int k, int n_total,
-                    float *__restrict__ out_f32, T *__restrict__ out_act, int ld_out) {
+gemm_rowwarp_kernel(const T *__restrict__ x, size_t x_plane, SegTable segs, int rows, int k, int n_total,
+                    float *__restrict__ out_f32, T *__restrict__ out_act, size_t act_plane, int ld_out) {
     constexpr int VN = Vec<T>::N;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int group = blockIdx.x * WARPS + warp;
@@ -97,6 +97,12 @@ gemm_rowwarp_kernel(const T *__restrict__ x, SegTable segs, int rows, int k, int
                 if (r0 + r < rows) {
                     float xv[VN];
                     load16<T>(x + (size_t)(r0 + r) * k + k0, xv);
+                    if (x_plane) {                      // bf16 activations come as hi + lo planes
+                        float lo[VN];
+                        load16<T>(x + x_plane + (size_t)(r0 + r) * k + k0, lo);
+#pragma unroll
+                        for (int e = 0; e < VN; ++e) xv[e] += lo[e];
+                    }
 #pragma unroll
                     for (int j = 0; j < FEAT; ++j)
 #pragma unroll
@@ -118,7 +124,7 @@ gemm_rowwarp_kernel(const T *__restrict__ x, SegTable segs, int rows, int k, int
                         if (!wrow[j]) continue;
                         float g = acc[r][j], u = acc[r][2 + j];
                         float s = g / (1.f + expf(-g));
-                        out_act[(size_t)(r0 + r) * ld_out + feat[j]] = from_f32<T>(s * u);
+                        store_act<T>(out_act, act_plane, (size_t)(r0 + r) * ld_out + feat[j], s * u);
                     }
                 } else {
 #pragma unroll
@@ -134,19 +140,19 @@ gemm_rowwarp_kernel(const T *__restrict__ x, SegTable segs, int rows, int k, int
 }
 
 template <typename T, int RC>
-int dispatch_epi(const T *x, const SegTable &s, int rows, int k, int n_total, int epi, float *out_f32, T *out_act,
-                 int ld_out, cudaStream_t st) {
+int dispatch_epi(const T *x, size_t x_plane, const SegTable &s, int rows, int k, int n_total, int epi, float *out_f32,
+                 T *out_act, size_t act_plane, int ld_out, cudaStream_t st) {
     int groups = epi == EPI_SWIGLU ? (s.end[0] + 1) / 2 : (n_total + FEAT - 1) / FEAT;
     int blocks = (groups + WARPS - 1) / WARPS;
     switch (epi) {
     case EPI_STORE:
-        gemm_rowwarp_kernel<T, RC, EPI_STORE><<<blocks, WARPS * 32, 0, st>>>(x, s, rows, k, n_total, out_f32, out_act, ld_out);
+        gemm_rowwarp_kernel<T, RC, EPI_STORE><<<blocks, WARPS * 32, 0, st>>>(x, x_plane, s, rows, k, n_total, out_f32, out_act, act_plane, ld_out);
         break;
     case EPI_ADD:
-        gemm_rowwarp_kernel<T, RC, EPI_ADD><<<blocks, WARPS * 32, 0, st>>>(x, s, rows, k, n_total, out_f32, out_act, ld_out);
+        gemm_rowwarp_kernel<T, RC, EPI_ADD><<<blocks, WARPS * 32, 0, st>>>(x, x_plane, s, rows, k, n_total, out_f32, out_act, act_plane, ld_out);
         break;
     case EPI_SWIGLU:
-        gemm_rowwarp_kernel<T, RC, EPI_SWIGLU><<<blocks, WARPS * 32, 0, st>>>(x, s, rows, k, n_total, out_f32, out_act, ld_out);
+        gemm_rowwarp_kernel<T, RC, EPI_SWIGLU><<<blocks, WARPS * 32, 0, st>>>(x, x_plane, s, rows, k, n_total, out_f32, out_act, act_plane, ld_out);
         break;
     default:
         return VIASD_EINVAL;
@@ -156,17 +162,17 @@ int dispatch_epi(const T *x, const SegTable &s, int rows, int k, int n_total, in
 }
 
 template <typename T>
-int dispatch_rows(const T *x, const SegTable &s, int rows, int k, int n_total, int epi, float *out_f32, T *out_act,
-                  int ld_out, cudaStream_t st) {
-    if (rows <= 4) return dispatch_epi<T, 4>(x, s, rows, k, n_total, epi, out_f32, out_act, ld_out, st);
-    if (rows <= 8) return dispatch_epi<T, 8>(x, s, rows, k, n_total, epi, out_f32, out_act, ld_out, st);
-    return dispatch_epi<T, 12>(x, s, rows, k, n_total, epi, out_f32, out_act, ld_out, st);
+int dispatch_rows(const T *x, size_t x_plane, const SegTable &s, int rows, int k, int n_total, int epi, float *out_f32,
+                  T *out_act, size_t act_plane, int ld_out, cudaStream_t st) {
+    if (rows <= 4) return dispatch_epi<T, 4>(x, x_plane, s, rows, k, n_total, epi, out_f32, out_act, act_plane, ld_out, st);
+    if (rows <= 8) return dispatch_epi<T, 8>(x, x_plane, s, rows, k, n_total, epi, out_f32, out_act, act_plane, ld_out, st);
+    return dispatch_epi<T, 12>(x, x_plane, s, rows, k, n_total, epi, out_f32, out_act, act_plane, ld_out, st);
 }
 
 }  // namespace
 
-int launch_gemm_rowwarp(const void *x, const GemmSegs &segs, int rows, int k, int dtype, int epilogue,
-                        float *out_f32, void *out_act, int ld_out, cudaStream_t st) {
+int launch_gemm_rowwarp(const void *x, size_t x_plane, const GemmSegs &segs, int rows, int k, int dtype,
+                        int epilogue, float *out_f32, void *out_act, size_t act_plane, int ld_out, cudaStream_t st) {
     if (rows <= 0) return VIASD_OK;
     if (k % 8 != 0) return VIASD_EINVAL;
     SegTable s;
@@ -179,7 +185,7 @@ int launch_gemm_rowwarp(const void *x, const GemmSegs &segs, int rows, int k, in
     }
     if (epilogue == EPI_SWIGLU && (segs.count != 2 || segs.n[0] != segs.n[1])) return VIASD_EINVAL;
     if (dtype == 0)
-        return dispatch_rows<float>((const float *)x, s, rows, k, total, epilogue, out_f32, (float *)out_act, ld_out, st);
-    return dispatch_rows<__nv_bfloat16>((const __nv_bfloat16 *)x, s, rows, k, total, epilogue, out_f32,
-                                        (__nv_bfloat16 *)out_act, ld_out, st);
+        return dispatch_rows<float>((const float *)x, 0, s, rows, k, total, epilogue, out_f32, (float *)out_act, 0, ld_out, st);
+    return dispatch_rows<__nv_bfloat16>((const __nv_bfloat16 *)x, x_plane, s, rows, k, total, epilogue, out_f32,
+                                        (__nv_bfloat16 *)out_act, act_plane, ld_out, st);
 }

@@ -1,0 +1,413 @@
+// Weight-streaming bf16 GEMM on the 5th-generation tensor cores (tcgen05 + TMEM), fed by TMA.
+//
+//   y[rows, n] = x[rows, k] * W[n, k]^T        rows <= 128 per launch, W streamed once from HBM
+//
+// The operands are swapped: a tile of 128 output features is the MMA's M dimension (A operand, the
+// weights), the token rows are its N dimension (B operand, 16..128 wide).  Both are K-major in shared
+// memory with the 128-byte swizzle, exactly as a 2-D TMA box of 64 bf16 x rows lands there.  The
+// activation comes as two bf16 planes hi + lo (x = hi + lo to ~16 mantissa bits); each weight tile is
+// multiplied with both, which costs tensor time the kernel has in abundance and no extra weight traffic.
+//
+// Persistent stream-K schedule: the (tile, k-block) units of the whole GEMM are cut into one contiguous
+// range per CTA, so every SM streams the same number of bytes whatever the shape.  A CTA that holds all
+// k-blocks of a tile finishes it from TMEM; otherwise it writes an fp32 partial and the last CTA to
+// arrive at the tile (an atomic counter, no waiting) sums the partials in CTA order - bit-reproducible.
+//
+// Warp roles (192 threads): warp 0 issues TMA loads into a ring of stages, warp 1 allocates TMEM and
+// issues tcgen05.mma, warps 2-5 read the accumulators (tcgen05.ld) and run the epilogue.  Accumulators
+// are double-buffered in TMEM so the epilogue of one tile overlaps the main loop of the next.
+// Every wait is bounded: on expiry the CTA records VIASD_EDEVICE, lets its copies land and leaves.
+#include "common.cuh"
+#include "gemm_tc.cuh"
+
+namespace {
+
+constexpr int TILE_F = 128;          // output features per tile (MMA M)
+constexpr int TILE_K = 64;           // bf16 per k-block: 128 bytes, one swizzle row
+constexpr int MAX_STAGES = 12;
+constexpr int THREADS = 192;
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about two seconds
+
+// ---- PTX wrappers ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the limit expired or another role of this CTA already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    int spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 255) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+                *abort_flag = 1;
+                atomicExch(status, VIASD_EDEVICE);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// K-major operand tile, 128-byte swizzle, rows 128 bytes apart, 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+    return (uint64_t)((addr >> 4) & 0x3FFF) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+
+struct Seg { int tile, ka, kb; };      // one contiguous piece of this CTA's unit range inside a tile
+
+__device__ __forceinline__ bool next_seg(int &u, int u1, int k_tiles, Seg &s) {
+    if (u >= u1) return false;
+    s.tile = u / k_tiles;
+    s.ka = u - s.tile * k_tiles;
+    s.kb = min(k_tiles, s.ka + (u1 - u));
+    u += s.kb - s.ka;
+    return true;
+}
+
+// epilogue for one (feature lane, token row)
+template <bool DUAL>
+__device__ __forceinline__ void finish(const TcParams &p, int tile, int f, int r, float g, float u) {
+    if (r >= p.rows) return;
+    if (DUAL) {
+        const int n = tile * TILE_F + f;
+        if (n >= p.seg_n[0]) return;
+        const float s = g / (1.f + expf(-g));
+        store_act<__nv_bfloat16>(p.out_act, p.act_plane, (size_t)(p.row0 + r) * p.ld_out + n, s * u);
+    } else {
+        int s = 0, t0 = 0, nbase = 0;
+        while (s < 2 && tile >= p.seg_tile_end[s]) { t0 = p.seg_tile_end[s]; nbase += p.seg_n[s]; ++s; }
+        const int nin = (tile - t0) * TILE_F + f;
+        if (nin >= p.seg_n[s]) return;
+        float *dst = p.out_f32 + (size_t)(p.row0 + r) * p.ld_out + nbase + nin;
+        if (p.epi == EPI_ADD) *dst += g; else *dst = g;
+    }
+}
+
+template <bool DUAL>
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
+               const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_x, const TcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) unsigned long long bars[2 * MAX_STAGES + 4];
+    __shared__ uint32_t tmem_base_sh;
+    __shared__ int abort_sh, last_sh;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int NT = p.nt, S = p.stages;
+    constexpr int NACC = DUAL ? 2 : 1;
+    const uint32_t a_bytes = TILE_F * TILE_K * 2, b_bytes = (uint32_t)NT * TILE_K * 2;
+    const uint32_t stage_bytes = NACC * a_bytes + 2 * b_bytes;
+    auto full_bar = [&](int s) { return smem_u32(&bars[s]); };
+    auto empty_bar = [&](int s) { return smem_u32(&bars[MAX_STAGES + s]); };
+    auto tfull_bar = [&](int b) { return smem_u32(&bars[2 * MAX_STAGES + b]); };
+    auto tempty_bar = [&](int b) { return smem_u32(&bars[2 * MAX_STAGES + 2 + b]); };
+    const uint32_t acc_cols = NACC * NT;                    // TMEM columns per accumulator buffer
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+        abort_sh = 0;
+        last_sh = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_sh)),
+                     "r"(p.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_sh;
+
+    const int total_units = p.n_tiles * p.k_tiles;
+    const int u_begin = blockIdx.x * p.units_per_cta;
+    const int u_end = min(total_units, u_begin + p.units_per_cta);
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            int it = 0, u = u_begin;
+            Seg sg;
+            bool ok = true;
+            while (ok && next_seg(u, u_end, p.k_tiles, sg)) {
+                // which weight matrix and which of its rows this tile covers
+                int s = 0, t0 = 0;
+                if (!DUAL) while (s < 2 && sg.tile >= p.seg_tile_end[s]) { t0 = p.seg_tile_end[s]; ++s; }
+                const CUtensorMap *mw = s == 0 ? &map_w0 : (s == 1 ? &map_w1 : &map_w2);
+                const int wrow = (sg.tile - t0) * TILE_F;
+                const uint32_t tx = DUAL ? 2 * p.a_tx[0] + 2 * p.b_tx : p.a_tx[s] + 2 * p.b_tx;
+                for (int kt = sg.ka; kt < sg.kb; ++kt, ++it) {
+                    const int st = it % S;
+                    if (!(ok = mbar_wait(empty_bar(st), ((it / S) & 1) ^ 1, &abort_sh, p.status))) break;
+                    const uint32_t base = smem_base + st * stage_bytes;
+                    mbar_expect_tx(full_bar(st), tx);
+                    tma_load_2d(base, mw, full_bar(st), kt * TILE_K, wrow);
+                    if (DUAL) tma_load_2d(base + a_bytes, &map_w1, full_bar(st), kt * TILE_K, wrow);
+                    tma_load_2d(base + NACC * a_bytes, &map_x, full_bar(st), kt * TILE_K, p.row0);
+                    tma_load_2d(base + NACC * a_bytes + b_bytes, &map_x, full_bar(st), kt * TILE_K,
+                                p.row0 + p.lo_row_offset);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NT >> 3) << 17) | ((TILE_F >> 4) << 24);
+            int it = 0, acc_it = 0, u = u_begin;
+            Seg sg;
+            bool ok = true;
+            while (ok && next_seg(u, u_end, p.k_tiles, sg)) {
+                const int buf = acc_it & 1;
+                if (!(ok = mbar_wait(tempty_bar(buf), ((acc_it >> 1) & 1) ^ 1, &abort_sh, p.status))) break;
+                tc_fence_after();
+                const uint32_t d0 = tmem_base + buf * acc_cols;
+                for (int kt = sg.ka; kt < sg.kb; ++kt, ++it) {
+                    const int st = it % S;
+                    if (!(ok = mbar_wait(full_bar(st), (it / S) & 1, &abort_sh, p.status))) break;
+                    tc_fence_after();
+                    const uint32_t base = smem_base + st * stage_bytes;
+                    const uint32_t bh = base + NACC * a_bytes, bl = bh + b_bytes;
+#pragma unroll
+                    for (int k = 0; k < TILE_K / 16; ++k) {
+                        const uint32_t first = (kt > sg.ka || k > 0) ? 1u : 0u;
+                        tc_mma(d0, smem_desc(base + k * 32), smem_desc(bh + k * 32), idesc, first);
+                        if (p.has_lo) tc_mma(d0, smem_desc(base + k * 32), smem_desc(bl + k * 32), idesc, 1u);
+                        if (DUAL) {
+                            tc_mma(d0 + NT, smem_desc(base + a_bytes + k * 32), smem_desc(bh + k * 32), idesc, first);
+                            if (p.has_lo)
+                                tc_mma(d0 + NT, smem_desc(base + a_bytes + k * 32), smem_desc(bl + k * 32), idesc, 1u);
+                        }
+                    }
+                    tc_commit(empty_bar(st));              // the stage is free once these MMAs have read it
+                }
+                if (ok) tc_commit(tfull_bar(buf));          // accumulator complete
+                ++acc_it;
+            }
+        }
+    } else {
+        // ---------------- epilogue (warps 2..5 <-> TMEM lane quarters 2,3,0,1) ----------------
+        const int quarter = warp & 3;
+        const int f = quarter * 32 + lane;                  // feature lane inside the tile
+        const int et = threadIdx.x - 64;                    // 0..127 among epilogue threads
+        const size_t slot_floats = (size_t)NACC * NT * TILE_F;
+        int acc_it = 0, u = u_begin, seg_i = 0;
+        Seg sg;
+        bool ok = true;
+        while (ok && next_seg(u, u_end, p.k_tiles, sg)) {
+            const int buf = acc_it & 1;
+            if (!(ok = mbar_wait(tfull_bar(buf), (acc_it >> 1) & 1, &abort_sh, p.status))) break;
+            tc_fence_after();
+            const bool whole = sg.ka == 0 && sg.kb == p.k_tiles;
+            const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * acc_cols;
+            // partial of a split tile: slot 0 if the tile is the first one this CTA touches, else slot 1
+            float *slot = p.scratch + ((size_t)blockIdx.x * 2 + (seg_i == 0 ? 0 : 1)) * slot_floats;
+            for (int c = 0; c < NT; c += 16) {
+                float g[16], uu[16];
+                tc_ld16(t0 + c, g);
+                if (DUAL) tc_ld16(t0 + NT + c, uu);
+                if (c >= p.rows) continue;                   // padding rows: nothing to keep
+                if (whole) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) finish<DUAL>(p, sg.tile, f, c + j, g[j], DUAL ? uu[j] : 0.f);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        slot[(size_t)(c + j) * TILE_F + f] = g[j];
+                        if (DUAL) slot[(size_t)(NT + c + j) * TILE_F + f] = uu[j];
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(buf));   // accumulator buffer may be overwritten
+            if (!whole) {
+                // publish the partial; the last contributor of the tile sums all of them in CTA order
+                __threadfence();
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (et == 0) {
+                    const int first_cta = (sg.tile * p.k_tiles) / p.units_per_cta;
+                    const int last_cta = ((sg.tile + 1) * p.k_tiles - 1) / p.units_per_cta;
+                    const int old = atomicAdd(&p.counters[sg.tile], 1);
+                    last_sh = (old == last_cta - first_cta) ? 1 : 0;
+                    if (last_sh) p.counters[sg.tile] = 0;   // ready for the next launch
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (last_sh) {
+                    __threadfence();
+                    const int first_cta = (sg.tile * p.k_tiles) / p.units_per_cta;
+                    const int last_cta = ((sg.tile + 1) * p.k_tiles - 1) / p.units_per_cta;
+                    for (int r = 0; r < p.rows; ++r) {
+                        float g = 0.f, uu = 0.f;
+                        for (int c = first_cta; c <= last_cta; ++c) {
+                            const int c_first_tile = (c * p.units_per_cta) / p.k_tiles;
+                            const float *src = p.scratch + ((size_t)c * 2 + (c_first_tile == sg.tile ? 0 : 1)) * slot_floats;
+                            g += __ldcg(src + (size_t)r * TILE_F + et);
+                            if (DUAL) uu += __ldcg(src + (size_t)(NT + r) * TILE_F + et);
+                        }
+                        finish<DUAL>(p, sg.tile, et, r, g, uu);
+                    }
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");   // last_sh is reused by the next split tile
+            }
+            ++acc_it;
+            ++seg_i;
+        }
+    }
+
+    // ---------------- teardown ----------------
+    __syncwarp();
+    if (abort_sh && threadIdx.x == 0) {
+        // give copies and MMAs that are still in flight time to land before shared memory and TMEM go away
+        const long long t0 = clock64();
+        while (clock64() - t0 < 400000) { }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                             const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                             CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeFn g_encode = nullptr;
+
+}  // namespace
+
+int tc_make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t k, uint32_t box_rows) {
+    if (!g_encode) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
+        if (!fn || q != cudaDriverEntryPointSuccess) return VIASD_EUNSUPPORTED;
+        g_encode = (EncodeFn)fn;
+    }
+    if (((uintptr_t)base & 15) || (k % 8) || rows == 0) return VIASD_EINVAL;
+    cuuint64_t dims[2] = {k, rows};
+    cuuint64_t strides[1] = {k * 2};
+    cuuint32_t box[2] = {TILE_K, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return VIASD_ECUDA; }
+    return VIASD_OK;
+}
+
+int tc_pick_nt(int rows) { return rows <= 16 ? 16 : rows <= 32 ? 32 : rows <= 64 ? 64 : 128; }
+
+uint32_t tc_box_rows(uint64_t tensor_rows, uint32_t want) { return tensor_rows < want ? (uint32_t)tensor_rows : want; }
+
+size_t tc_scratch_floats(int sm_count, int nt, bool dual) { return (size_t)sm_count * 2 * (dual ? 2 : 1) * nt * TILE_F; }
+
+int tc_tiles(int n) { return (n + TILE_F - 1) / TILE_F; }
+
+int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {
+    TcParams p;
+    memset(&p, 0, sizeof(p));
+    const bool dual = L.epi == EPI_SWIGLU;
+    p.nt = L.nt;
+    p.rows = L.rows;
+    p.row0 = L.row0;
+    p.k_tiles = (L.k + TILE_K - 1) / TILE_K;
+    int tiles = 0;
+    for (int s = 0; s < 3; ++s) {
+        p.seg_n[s] = s < L.n_seg ? L.seg_n[s] : 0;
+        if (!dual && s < L.n_seg) tiles += tc_tiles(L.seg_n[s]);
+        p.seg_tile_end[s] = tiles;
+        p.a_tx[s] = (s < L.n_seg ? L.w_box_rows[s] : 0) * TILE_K * 2;
+    }
+    if (dual) tiles = tc_tiles(L.seg_n[0]);
+    p.n_tiles = tiles;
+    p.b_tx = L.x_box_rows * TILE_K * 2;
+    p.has_lo = L.has_lo;
+    p.lo_row_offset = L.lo_row_offset;
+    p.epi = L.epi;
+    p.out_f32 = L.out_f32;
+    p.out_act = (__nv_bfloat16 *)L.out_act;
+    p.act_plane = L.act_plane;
+    p.ld_out = L.ld_out;
+    p.scratch = L.scratch;
+    p.counters = L.counters;
+    p.status = L.status;
+    const int units = p.n_tiles * p.k_tiles;
+    if (units <= 0) return VIASD_OK;
+    int grid = L.sm_count < units ? L.sm_count : units;
+    p.units_per_cta = (units + grid - 1) / grid;
+    grid = (units + p.units_per_cta - 1) / p.units_per_cta;
+    const int nacc = dual ? 2 : 1;
+    const size_t stage = (size_t)nacc * TILE_F * TILE_K * 2 + 2 * (size_t)L.nt * TILE_K * 2;
+    int stages = (int)((size_t)200 * 1024 / stage);
+    if (stages > MAX_STAGES) stages = MAX_STAGES;
+    if (stages < 2) return VIASD_EINVAL;
+    p.stages = stages;
+    int cols = 2 * nacc * L.nt;
+    p.tmem_cols = cols <= 32 ? 32 : cols <= 64 ? 64 : cols <= 128 ? 128 : cols <= 256 ? 256 : 512;
+    const size_t smem = stage * stages + 1024;
+    static bool attr_done[2] = {false, false};
+    if (!attr_done[dual]) {
+        if (dual) CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        else CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        attr_done[dual] = true;
+    }
+    const CUtensorMap &w0 = *L.map_w[0], &w1 = *L.map_w[L.n_seg > 1 ? 1 : 0], &w2 = *L.map_w[L.n_seg > 2 ? 2 : 0];
+    if (dual) gemm_tc_kernel<true><<<grid, THREADS, smem, st>>>(w0, w1, w2, *L.map_x, p);
+    else gemm_tc_kernel<false><<<grid, THREADS, smem, st>>>(w0, w1, w2, *L.map_x, p);
+    LAUNCH_CHECK();
+    return VIASD_OK;
+}

@@ -1,0 +1,50 @@
+// Interface of the tcgen05 weight-streaming GEMM (gemm_tc.cu).
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <string.h>
+
+struct TcParams {                       // kernel argument block
+    int nt, stages, tmem_cols;          // token-tile width (MMA N), smem ring depth, TMEM columns to allocate
+    int rows, row0;                     // token rows of this launch and the first one
+    int k_tiles, n_tiles, units_per_cta;
+    int seg_n[3], seg_tile_end[3];      // output features per weight matrix; running tile count
+    uint32_t a_tx[3], b_tx;             // bytes one TMA box of each operand delivers
+    int has_lo, lo_row_offset;          // activation lo plane: present, and its row offset in the 2-D map
+    int epi;                            // EPI_STORE / EPI_ADD / EPI_SWIGLU
+    float *out_f32;
+    __nv_bfloat16 *out_act;
+    size_t act_plane;
+    int ld_out;
+    float *scratch;                     // [grid][2] partial-tile slots
+    int *counters;                      // [n_tiles], zero between launches
+    int *status;                        // device status word
+};
+
+struct TcLaunch {                       // host-side description of one GEMM
+    const CUtensorMap *map_w[3];
+    int seg_n[3], n_seg;
+    uint32_t w_box_rows[3];
+    const CUtensorMap *map_x;
+    uint32_t x_box_rows;
+    int has_lo, lo_row_offset;
+    int rows, row0, k, nt;
+    int epi;
+    float *out_f32;
+    void *out_act;
+    size_t act_plane;
+    int ld_out;
+    float *scratch;
+    int *counters;
+    int *status;
+    int sm_count;
+};
+
+// 2-D bf16 tensor [rows, k] row-major -> TMA map with a (64 x box_rows) box and the 128-byte swizzle
+int tc_make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t k, uint32_t box_rows);
+int tc_pick_nt(int rows);
+uint32_t tc_box_rows(uint64_t tensor_rows, uint32_t want);
+size_t tc_scratch_floats(int sm_count, int nt, bool dual);
+int tc_tiles(int n);
+int launch_gemm_tc(const TcLaunch &L, cudaStream_t st);

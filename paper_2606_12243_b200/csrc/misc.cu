@@ -95,7 +95,7 @@ int launch_embed(const viasd_model *m, int rows, cudaStream_t st) {
 // RMSNorm: a[r] = h[r] / sqrt(mean(h[r]^2) + eps) * gain, written in the model dtype
 // ---------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void rmsnorm_kernel(T *a, const float *h, const float *gain, int d, float eps) {
+__global__ void rmsnorm_kernel(T *a, size_t plane, const float *h, const float *gain, int d, float eps) {
     __shared__ float red[32];
     int r = blockIdx.x;
     const float *x = h + (size_t)r * d;
@@ -111,15 +111,15 @@ __global__ void rmsnorm_kernel(T *a, const float *h, const float *gain, int d, f
     }
     __syncthreads();
     float inv = red[0];
-    for (int i = threadIdx.x; i < d; i += blockDim.x) a[(size_t)r * d + i] = from_f32<T>(x[i] * inv * gain[i]);
+    for (int i = threadIdx.x; i < d; i += blockDim.x) store_act<T>(a, plane, (size_t)r * d + i, x[i] * inv * gain[i]);
 }
 
 int launch_rmsnorm(const viasd_model *m, const float *gain, int rows, cudaStream_t st) {
     if (m->cfg.dtype == 0)
-        rmsnorm_kernel<float><<<rows, 256, 0, st>>>((float *)m->ws.a, m->ws.h, gain, m->cfg.d_model, m->cfg.rms_eps);
+        rmsnorm_kernel<float><<<rows, 256, 0, st>>>((float *)m->ws.a, 0, m->ws.h, gain, m->cfg.d_model, m->cfg.rms_eps);
     else
-        rmsnorm_kernel<__nv_bfloat16><<<rows, 256, 0, st>>>((__nv_bfloat16 *)m->ws.a, m->ws.h, gain,
-                                                            m->cfg.d_model, m->cfg.rms_eps);
+        rmsnorm_kernel<__nv_bfloat16><<<rows, 256, 0, st>>>((__nv_bfloat16 *)m->ws.a, m->ws.rows_alloc * m->cfg.d_model,
+                                                            m->ws.h, gain, m->cfg.d_model, m->cfg.rms_eps);
     LAUNCH_CHECK();
     return VIASD_OK;
 }
@@ -128,7 +128,7 @@ int launch_rmsnorm(const viasd_model *m, const float *gain, int rows, cudaStream
 // rotary embedding of q and k, KV append at slot len + row
 // ---------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void rope_append_kernel(T *q_out, T *kc, T *vc, const float *qkv, const float *cosv, const float *sinv,
+__global__ void rope_append_kernel(float *q_out, T *kc, T *vc, const float *qkv, const float *cosv, const float *sinv,
                                    const int *len_eff, const TreeInfo *tree, int M, int H, int Hkv, int hd,
                                    int max_batch, int max_ctx, int layer_ord) {
     int r = blockIdx.x, head = blockIdx.y;
@@ -143,9 +143,9 @@ __global__ void rope_append_kernel(T *q_out, T *kc, T *vc, const float *qkv, con
             float c = cosv[(size_t)pos * half + p], s = sinv[(size_t)pos * half + p];
             float y1 = x1 * c - x2 * s, y2 = x2 * c + x1 * s;
             if (head < H) {
-                T *dst = q_out + (size_t)r * H * hd + (size_t)head * hd;
-                dst[p] = from_f32<T>(y1);
-                dst[p + half] = from_f32<T>(y2);
+                float *dst = q_out + (size_t)r * H * hd + (size_t)head * hd;
+                dst[p] = y1;
+                dst[p + half] = y2;
             } else {
                 int g = head - H;
                 T *dst = kc + ((((size_t)layer_ord * max_batch + b) * Hkv + g) * max_ctx + slot) * hd;
@@ -166,11 +166,11 @@ int launch_rope_append(const viasd_model *m, void *kc, void *vc, int layer_ord, 
     dim3 grid(batch * M, c.n_heads + 2 * c.n_kv_heads);
     int threads = c.head_dim / 2 < 32 ? 32 : c.head_dim / 2;
     if (c.dtype == 0)
-        rope_append_kernel<float><<<grid, threads, 0, st>>>((float *)m->ws.q, (float *)kc, (float *)vc, m->ws.qkv,
+        rope_append_kernel<float><<<grid, threads, 0, st>>>(m->ws.q, (float *)kc, (float *)vc, m->ws.qkv,
             m->ws.rope_cos, m->ws.rope_sin, m->ws.len_eff, m->ws.tree, M, c.n_heads, c.n_kv_heads, c.head_dim,
             c.max_batch, c.max_ctx, layer_ord);
     else
-        rope_append_kernel<__nv_bfloat16><<<grid, threads, 0, st>>>((__nv_bfloat16 *)m->ws.q, (__nv_bfloat16 *)kc,
+        rope_append_kernel<__nv_bfloat16><<<grid, threads, 0, st>>>(m->ws.q, (__nv_bfloat16 *)kc,
             (__nv_bfloat16 *)vc, m->ws.qkv, m->ws.rope_cos, m->ws.rope_sin, m->ws.len_eff, m->ws.tree, M, c.n_heads,
             c.n_kv_heads, c.head_dim, c.max_batch, c.max_ctx, layer_ord);
     LAUNCH_CHECK();
