@@ -23,6 +23,7 @@ struct Carver {
 };
 
 constexpr int MAX_SMS = 160;            // workspace is sized without asking the device
+constexpr int MAX_GEMM_CTAS = 2 * MAX_SMS;
 
 size_t part_bytes_for(const viasd_config &c) {
     const size_t R = (size_t)c.max_batch * c.max_query;
@@ -57,7 +58,7 @@ size_t carve(const viasd_config &c, char *base, Workspace *ws) {
     w.accept_scratch = cv.take<float>((size_t)c.max_batch * 3 * c.vocab * 4);
     {
         const int nt = tc_pick_nt(R < 128 ? (int)R : 128);
-        w.gemm_scratch = cv.take<float>(tc_scratch_floats(MAX_SMS, nt, true) * 4);
+        w.gemm_scratch = cv.take<float>(tc_scratch_floats(MAX_GEMM_CTAS, nt, true) * 4);
         size_t widest = (size_t)c.vocab;
         if (qd + 2 * kvd > widest) widest = qd + 2 * kvd;
         if ((size_t)c.d_ff > widest) widest = c.d_ff;
@@ -443,7 +444,7 @@ size_t viasd_gemm_scratch_bytes(int rows, int n, int k) {
     if (rows < 1 || n < 1) return 256;
     const int nt = tc_pick_nt(rows < 128 ? rows : 128);
     // [tile counters | one status word] then the partial-tile slots
-    return align_up((size_t)(tc_tiles(n) + 1) * 4, 256) + tc_scratch_floats(MAX_SMS, nt, false) * 4;
+    return align_up((size_t)(tc_tiles(n) + 1) * 4, 256) + tc_scratch_floats(MAX_GEMM_CTAS, nt, false) * 4;
 }
 
 int viasd_gemm(const void *x, const void *w, float *y, int rows, int n, int k, int dtype, void *scratch,

@@ -19,6 +19,7 @@
 // Every wait is bounded: on expiry the CTA records VIASD_EDEVICE, lets its copies land and leaves.
 #include "common.cuh"
 #include "gemm_tc.cuh"
+#include <stdlib.h>
 
 namespace {
 
@@ -103,6 +104,15 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
     return (uint64_t)((addr >> 4) & 0x3FFF) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
 }
 
+#ifdef VIASD_TC_TRACE
+__device__ long long g_tc_trace[160 * 8];
+#define TRACE(slot) do { g_tc_trace[blockIdx.x * 8 + (slot)] = clock64(); } while (0)
+#define DBG(p, bit) ((p).dbg & (bit))
+#else
+#define DBG(p, bit) 0
+#define TRACE(slot) do { } while (0)
+#endif
+
 struct Seg { int tile, ka, kb; };      // one contiguous piece of this CTA's unit range inside a tile
 
 __device__ __forceinline__ bool next_seg(int &u, int u1, int k_tiles, Seg &s) {
@@ -143,6 +153,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
     __shared__ int abort_sh, last_sh;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) TRACE(0);
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int NT = p.nt, S = p.stages;
     constexpr int NACC = DUAL ? 2 : 1;
@@ -152,7 +163,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
     auto empty_bar = [&](int s) { return smem_u32(&bars[MAX_STAGES + s]); };
     auto tfull_bar = [&](int b) { return smem_u32(&bars[2 * MAX_STAGES + b]); };
     auto tempty_bar = [&](int b) { return smem_u32(&bars[2 * MAX_STAGES + 2 + b]); };
-    const uint32_t acc_cols = NACC * NT;                    // TMEM columns per accumulator buffer
+    const int NB = p.has_lo ? 2 * NT : NT;                  // MMA N: hi and lo token columns side by side
+    const uint32_t acc_cols = NACC * NB;                    // TMEM columns per accumulator buffer
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -171,6 +183,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_sh;
+    if (threadIdx.x == 0) TRACE(1);
 
     const int total_units = p.n_tiles * p.k_tiles;
     const int u_begin = blockIdx.x * p.units_per_cta;
@@ -188,7 +201,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                 if (!DUAL) while (s < 2 && sg.tile >= p.seg_tile_end[s]) { t0 = p.seg_tile_end[s]; ++s; }
                 const CUtensorMap *mw = s == 0 ? &map_w0 : (s == 1 ? &map_w1 : &map_w2);
                 const int wrow = (sg.tile - t0) * TILE_F;
-                const uint32_t tx = DUAL ? 2 * p.a_tx[0] + 2 * p.b_tx : p.a_tx[s] + 2 * p.b_tx;
+                uint32_t tx = DUAL ? 2 * p.a_tx[0] + 2 * p.b_tx : p.a_tx[s] + 2 * p.b_tx;
+                if (DBG(p, 1)) tx -= 2 * p.b_tx;
                 for (int kt = sg.ka; kt < sg.kb; ++kt, ++it) {
                     const int st = it % S;
                     if (!(ok = mbar_wait(empty_bar(st), ((it / S) & 1) ^ 1, &abort_sh, p.status))) break;
@@ -196,46 +210,46 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                     mbar_expect_tx(full_bar(st), tx);
                     tma_load_2d(base, mw, full_bar(st), kt * TILE_K, wrow);
                     if (DUAL) tma_load_2d(base + a_bytes, &map_w1, full_bar(st), kt * TILE_K, wrow);
+                    if (!DBG(p, 1)) {
                     tma_load_2d(base + NACC * a_bytes, &map_x, full_bar(st), kt * TILE_K, p.row0);
                     tma_load_2d(base + NACC * a_bytes + b_bytes, &map_x, full_bar(st), kt * TILE_K,
                                 p.row0 + p.lo_row_offset);
+                    }
                 }
             }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NT >> 3) << 17) | ((TILE_F >> 4) << 24);
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NB >> 3) << 17) | ((TILE_F >> 4) << 24);
             int it = 0, acc_it = 0, u = u_begin;
             Seg sg;
             bool ok = true;
             while (ok && next_seg(u, u_end, p.k_tiles, sg)) {
-                const int buf = acc_it & 1;
-                if (!(ok = mbar_wait(tempty_bar(buf), ((acc_it >> 1) & 1) ^ 1, &abort_sh, p.status))) break;
+                const int buf = acc_it % p.acc_bufs;
+                if (!(ok = mbar_wait(tempty_bar(buf), ((acc_it / p.acc_bufs) & 1) ^ 1, &abort_sh, p.status))) break;
                 tc_fence_after();
                 const uint32_t d0 = tmem_base + buf * acc_cols;
                 for (int kt = sg.ka; kt < sg.kb; ++kt, ++it) {
                     const int st = it % S;
                     if (!(ok = mbar_wait(full_bar(st), (it / S) & 1, &abort_sh, p.status))) break;
+                    if (it == 0) TRACE(2);
                     tc_fence_after();
                     const uint32_t base = smem_base + st * stage_bytes;
-                    const uint32_t bh = base + NACC * a_bytes, bl = bh + b_bytes;
+                    // the hi tile is followed by the lo tile: together one K-major operand of NB rows
+                    const uint32_t bh = base + NACC * a_bytes;
 #pragma unroll
                     for (int k = 0; k < TILE_K / 16; ++k) {
-                        const uint32_t first = (kt > sg.ka || k > 0) ? 1u : 0u;
-                        tc_mma(d0, smem_desc(base + k * 32), smem_desc(bh + k * 32), idesc, first);
-                        if (p.has_lo) tc_mma(d0, smem_desc(base + k * 32), smem_desc(bl + k * 32), idesc, 1u);
-                        if (DUAL) {
-                            tc_mma(d0 + NT, smem_desc(base + a_bytes + k * 32), smem_desc(bh + k * 32), idesc, first);
-                            if (p.has_lo)
-                                tc_mma(d0 + NT, smem_desc(base + a_bytes + k * 32), smem_desc(bl + k * 32), idesc, 1u);
-                        }
+                        const uint32_t acc = (kt > sg.ka || k > 0) ? 1u : 0u;
+                        tc_mma(d0, smem_desc(base + k * 32), smem_desc(bh + k * 32), idesc, acc);
+                        if (DUAL) tc_mma(d0 + NB, smem_desc(base + a_bytes + k * 32), smem_desc(bh + k * 32), idesc, acc);
                     }
                     tc_commit(empty_bar(st));              // the stage is free once these MMAs have read it
                 }
                 if (ok) tc_commit(tfull_bar(buf));          // accumulator complete
                 ++acc_it;
             }
+            TRACE(3);
         }
     } else {
         // ---------------- epilogue (warps 2..5 <-> TMEM lane quarters 2,3,0,1) ----------------
@@ -247,8 +261,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
         Seg sg;
         bool ok = true;
         while (ok && next_seg(u, u_end, p.k_tiles, sg)) {
-            const int buf = acc_it & 1;
-            if (!(ok = mbar_wait(tfull_bar(buf), (acc_it >> 1) & 1, &abort_sh, p.status))) break;
+            const int buf = acc_it % p.acc_bufs;
+            if (!(ok = mbar_wait(tfull_bar(buf), (acc_it / p.acc_bufs) & 1, &abort_sh, p.status))) break;
             tc_fence_after();
             const bool whole = sg.ka == 0 && sg.kb == p.k_tiles;
             const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * acc_cols;
@@ -256,9 +270,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
             float *slot = p.scratch + ((size_t)blockIdx.x * 2 + (seg_i == 0 ? 0 : 1)) * slot_floats;
             for (int c = 0; c < NT; c += 16) {
                 float g[16], uu[16];
+                if (c >= p.rows) break;                      // padding rows: nothing to keep
                 tc_ld16(t0 + c, g);
-                if (DUAL) tc_ld16(t0 + NT + c, uu);
-                if (c >= p.rows) continue;                   // padding rows: nothing to keep
+                if (DUAL) tc_ld16(t0 + NB + c, uu);
+                if (p.has_lo) {                              // add the product with the lo plane
+                    float lo[16];
+                    tc_ld16(t0 + NT + c, lo);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) g[j] += lo[j];
+                    if (DUAL) {
+                        tc_ld16(t0 + NB + NT + c, lo);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) uu[j] += lo[j];
+                    }
+                }
                 if (whole) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j) finish<DUAL>(p, sg.tile, f, c + j, g[j], DUAL ? uu[j] : 0.f);
@@ -289,21 +314,30 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                     __threadfence();
                     const int first_cta = (sg.tile * p.k_tiles) / p.units_per_cta;
                     const int last_cta = ((sg.tile + 1) * p.k_tiles - 1) / p.units_per_cta;
-                    for (int r = 0; r < p.rows; ++r) {
-                        float g = 0.f, uu = 0.f;
+                    for (int r0 = 0; r0 < p.rows; r0 += 16) {
+                        float g[16], uu[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) { g[j] = 0.f; uu[j] = 0.f; }
                         for (int c = first_cta; c <= last_cta; ++c) {
                             const int c_first_tile = (c * p.units_per_cta) / p.k_tiles;
                             const float *src = p.scratch + ((size_t)c * 2 + (c_first_tile == sg.tile ? 0 : 1)) * slot_floats;
-                            g += __ldcg(src + (size_t)r * TILE_F + et);
-                            if (DUAL) uu += __ldcg(src + (size_t)(NT + r) * TILE_F + et);
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                if (r0 + j < p.rows) {
+                                    g[j] += __ldcg(src + (size_t)(r0 + j) * TILE_F + et);
+                                    if (DUAL) uu[j] += __ldcg(src + (size_t)(NT + r0 + j) * TILE_F + et);
+                                }
+                            }
                         }
-                        finish<DUAL>(p, sg.tile, et, r, g, uu);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) finish<DUAL>(p, sg.tile, et, r0 + j, g[j], uu[j]);
                     }
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");   // last_sh is reused by the next split tile
             }
             ++acc_it;
             ++seg_i;
+            if (et == 0) TRACE(4 + (seg_i > 2 ? 2 : seg_i - 1));
         }
     }
 
@@ -316,6 +350,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
     }
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) TRACE(7);
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
@@ -348,6 +383,12 @@ int tc_make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t k, u
     if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return VIASD_ECUDA; }
     return VIASD_OK;
 }
+
+#ifdef VIASD_TC_TRACE
+extern "C" int viasd_debug_trace(long long *host_out) {
+    return (int)cudaMemcpyFromSymbol(host_out, g_tc_trace, sizeof(long long) * 160 * 8);
+}
+#endif
 
 int tc_pick_nt(int rows) { return rows <= 16 ? 16 : rows <= 32 ? 32 : rows <= 64 ? 64 : 128; }
 
@@ -387,16 +428,27 @@ int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {
     p.status = L.status;
     const int units = p.n_tiles * p.k_tiles;
     if (units <= 0) return VIASD_OK;
-    int grid = L.sm_count < units ? L.sm_count : units;
+    int ctas_per_sm = 1;
+#ifdef VIASD_TC_TRACE
+    if (getenv("VIASD_TC_PER_SM")) ctas_per_sm = atoi(getenv("VIASD_TC_PER_SM"));
+#endif
+    int grid = L.sm_count * ctas_per_sm < units ? L.sm_count * ctas_per_sm : units;
     p.units_per_cta = (units + grid - 1) / grid;
     grid = (units + p.units_per_cta - 1) / p.units_per_cta;
     const int nacc = dual ? 2 : 1;
     const size_t stage = (size_t)nacc * TILE_F * TILE_K * 2 + 2 * (size_t)L.nt * TILE_K * 2;
     int stages = (int)((size_t)200 * 1024 / stage);
     if (stages > MAX_STAGES) stages = MAX_STAGES;
+#ifdef VIASD_TC_TRACE
+    if (getenv("VIASD_TC_DBG")) p.dbg = atoi(getenv("VIASD_TC_DBG"));
+    if (getenv("VIASD_TC_STAGES")) { int v = atoi(getenv("VIASD_TC_STAGES")); if (v >= 2 && v < stages) stages = v; }
+#endif
     if (stages < 2) return VIASD_EINVAL;
     p.stages = stages;
-    int cols = 2 * nacc * L.nt;
+    // accumulators are double-buffered when two of them fit in the 512 TMEM columns
+    const int acc_cols = nacc * L.nt * (L.has_lo ? 2 : 1);
+    p.acc_bufs = 2 * acc_cols <= 512 ? 2 : 1;
+    int cols = p.acc_bufs * acc_cols;
     p.tmem_cols = cols <= 32 ? 32 : cols <= 64 ? 64 : cols <= 128 ? 128 : cols <= 256 ? 256 : 512;
     const size_t smem = stage * stages + 1024;
     static bool attr_done[2] = {false, false};

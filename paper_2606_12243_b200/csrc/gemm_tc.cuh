@@ -7,6 +7,7 @@
 
 struct TcParams {                       // kernel argument block
     int nt, stages, tmem_cols;          // token-tile width (MMA N), smem ring depth, TMEM columns to allocate
+    int acc_bufs;                       // accumulator buffers in TMEM (2 when they fit, else 1)
     int rows, row0;                     // token rows of this launch and the first one
     int k_tiles, n_tiles, units_per_cta;
     int seg_n[3], seg_tile_end[3];      // output features per weight matrix; running tile count
@@ -20,6 +21,7 @@ struct TcParams {                       // kernel argument block
     float *scratch;                     // [grid][2] partial-tile slots
     int *counters;                      // [n_tiles], zero between launches
     int *status;                        // device status word
+    int dbg;                            // measurement knobs, honoured by trace builds only
 };
 
 struct TcLaunch {                       // host-side description of one GEMM
