@@ -173,7 +173,7 @@ int forward(viasd_model *m, const viasd_cache *cache, const viasd_draft *d, bool
                      c.d_model, EPI_STORE, m->ws.qkv, nullptr, 0, qd + 2 * kvd};
         if ((rc = timed(m, VIASD_T_GEMM, st, [&] { return run_gemm(m, qkv, rows, st); }))) return rc;
         if ((rc = timed(m, VIASD_T_ROPE, st, [&] { return launch_rope_append(m, kc, vc, ord, B, M, st); }))) return rc;
-        if ((rc = timed(m, VIASD_T_ATTENTION, st, [&] { return launch_attention(m, kc, vc, ord, B, M, st); }))) return rc;
+        if ((rc = timed(m, VIASD_T_ATTENTION, st, [&] { return launch_attention(m, kc, vc, slim, ord, B, M, st); }))) return rc;
         GemmCall wo{m->ws.attn, pq, &m->maps_attn, {m->wo[l], nullptr, nullptr}, {lm ? &lm->wo : nullptr, nullptr, nullptr},
                     {c.d_model, 0, 0}, 1, qd, EPI_ADD, m->ws.h, nullptr, 0, c.d_model};
         if ((rc = timed(m, VIASD_T_GEMM, st, [&] { return run_gemm(m, wo, rows, st); }))) return rc;

@@ -161,9 +161,25 @@ int attention_nsplit(const viasd_model *m, int batch, int M) {
     return nsplit;
 }
 
-int launch_attention(const viasd_model *m, const void *kc, const void *vc, int layer_ord, int batch, int M,
+int launch_attention(viasd_model *m, const void *kc, const void *vc, bool slim, int layer_ord, int batch, int M,
                      cudaStream_t st) {
     const viasd_config &c = m->cfg;
+    if (attention_mma_supported(m, M)) {
+        // tensor-core kernel: one CTA per (sequence, kv head, key range of whole 128-key tiles)
+        const int ctas = batch * c.n_kv_heads;
+        int nsplit = (m->sm_count + ctas - 1) / ctas;
+        const int max_tiles = (c.max_ctx + 127) / 128;
+        if (nsplit > max_tiles) nsplit = max_tiles;
+        if (nsplit > 16) nsplit = 16;
+        size_t per_split = (size_t)batch * c.n_heads * M * (c.head_dim + 2) * sizeof(float);
+        while (nsplit > 1 && per_split * nsplit > m->ws.part_bytes) --nsplit;
+        int rc = launch_attention_mma(m, kc, vc, slim, layer_ord, batch, M, nsplit, st);
+        if (rc || nsplit == 1) return rc;
+        attention_combine_kernel<__nv_bfloat16, 128><<<dim3(batch * M, c.n_heads), 128, 0, st>>>(
+            (__nv_bfloat16 *)m->ws.attn, m->ws.rows_alloc * (size_t)c.n_heads * 128, m->ws.part, M, c.n_heads, nsplit);
+        LAUNCH_CHECK();
+        return VIASD_OK;
+    }
     int nsplit = attention_nsplit(m, batch, M);
     if (c.dtype == 0) {
         if (c.head_dim == 64) return run<float, 64>(m, kc, vc, layer_ord, batch, M, nsplit, st);

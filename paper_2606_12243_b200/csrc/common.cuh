@@ -56,6 +56,7 @@ struct Workspace {                      // pointers into the caller's workspace 
 struct WMap { CUtensorMap map; uint32_t box_rows; };        // TMA view of one weight matrix
 struct ActMaps { CUtensorMap map[4]; uint32_t box_rows[4]; }; // TMA views of an activation buffer, NT = 16,32,64,128
 struct LayerMaps { WMap wq, wk, wv, wo, wg, wu, wd; };
+struct CacheMaps { CUtensorMap k, v; const void *k_ptr, *v_ptr; };   // TMA views of one model's KV cache
 
 struct KernelTimer {                    // optional per-launch CUDA-event record (measurement only)
     static constexpr int CAP = 8192;
@@ -82,6 +83,7 @@ struct viasd_model {
     LayerMaps *lmaps;                   // [L]
     WMap head_map;
     ActMaps maps_a, maps_attn, maps_act;
+    CacheMaps cmaps_full, cmaps_slim;
 };
 
 // error helpers -------------------------------------------------------------------------------
@@ -115,8 +117,12 @@ int launch_gemm_rowwarp(const void *x, size_t x_plane, const GemmSegs &segs, int
                         int epilogue, float *out_f32, void *out_act, size_t act_plane, int ld_out, cudaStream_t st);
 
 // attention.cu
-int launch_attention(const viasd_model *m, const void *kc, const void *vc, int layer_ord, int batch, int M,
+int launch_attention(viasd_model *m, const void *kc, const void *vc, bool slim, int layer_ord, int batch, int M,
                      cudaStream_t st);
+// attention_mma.cu
+int attention_mma_supported(const viasd_model *m, int M);
+int launch_attention_mma(viasd_model *m, const void *kc, const void *vc, bool slim, int layer_ord, int batch, int M,
+                         int nsplit, cudaStream_t st);
 
 // tier_accept.cu
 int launch_tier(const viasd_model *m, const viasd_draft *d, const viasd_params *p, const float *slim_logits,
