@@ -6,6 +6,7 @@
 
 int g_last_cuda_error = 0;
 unsigned long long g_launch_count = 0;
+int g_use_pdl = -1;
 
 namespace {
 
@@ -62,6 +63,7 @@ size_t carve(const viasd_config &c, char *base, Workspace *ws) {
         size_t widest = (size_t)c.vocab;
         if (qd + 2 * kvd > widest) widest = qd + 2 * kvd;
         if ((size_t)c.d_ff > widest) widest = c.d_ff;
+        w.ssq = cv.take<float>((size_t)(c.d_model / 128 + 1) * 4 * R * 4);
         w.n_counters = widest / 128 + 8;
         w.gemm_counters = cv.take<int>(w.n_counters * 4);
     }
@@ -148,12 +150,91 @@ int run_gemm(viasd_model *m, const GemmCall &g, int rows, cudaStream_t st) {
     return VIASD_OK;
 }
 
+// Tensor-core path with fused epilogues: per layer QKV (+RMS scale, rotary, KV append) -> attention ->
+// O (+residual, next-norm preparation) -> gate/up (+RMS scale, SwiGLU) -> down (+residual, next-norm preparation).
+int forward_fused(viasd_model *m, const viasd_cache *cache, const viasd_draft *d, bool slim, float *logits, cudaStream_t st) {
+    const viasd_config &c = m->cfg;
+    const int B = d->batch, M = d->n_nodes + 1, rows = B * M;
+    const int qd = c.n_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
+    void *kc = slim ? cache->k_slim : cache->k_full, *vc = slim ? cache->v_slim : cache->v_full;
+    const int n_run = slim ? m->n_routed : c.n_layers;
+    const size_t R = m->ws.rows_alloc;
+    int rc;
+    auto layer_id = [&](int ord) { return slim ? m->routed[ord] : ord; };
+    // common part of a launch description; rows beyond 128 go in chunks
+    auto gemm = [&](int cls, TcLaunch L, const ActMaps &xm) -> int {
+        return timed(m, cls, st, [&]() -> int {
+            for (int row0 = 0; row0 < rows; row0 += 128) {
+                const int nr = rows - row0 < 128 ? rows - row0 : 128, nt = tc_pick_nt(nr);
+                const int ni = nt == 16 ? 0 : nt == 32 ? 1 : nt == 64 ? 2 : 3;
+                L.map_x = &xm.map[ni]; L.x_box_rows = xm.box_rows[ni];
+                L.has_lo = 1; L.lo_row_offset = (int)R;
+                L.rows = nr; L.row0 = row0; L.nt = nt;
+                L.scratch = m->ws.gemm_scratch; L.counters = m->ws.gemm_counters; L.status = &m->ws.stats->device_status;
+                L.sm_count = m->sm_count;
+                L.ssq_stride = (int)R; L.inv_d = 1.0f / (float)c.d_model; L.eps = c.rms_eps;
+                int r2 = launch_gemm_tc(L, st);
+                if (r2) return r2;
+            }
+            return (int)VIASD_OK;
+        });
+    };
+    auto wseg = [&](TcLaunch &L, int i, const WMap &w, int n) { L.map_w[i] = &w.map; L.seg_n[i] = n; L.w_box_rows[i] = w.box_rows; };
+    const int ssq_n = (c.d_model / 128) * 4;
+
+    if ((rc = timed(m, VIASD_T_EMBED, st, [&] { return launch_prep(m, cache, d, st); }))) return rc;
+    if ((rc = timed(m, VIASD_T_EMBED, st, [&] { return launch_embed_norm(m, m->norm1[layer_id(0)], rows, st); }))) return rc;
+    for (int ord = 0; ord < n_run; ++ord) {
+        const int l = layer_id(ord);
+        const LayerMaps &lm = m->lmaps[l];
+        {   // QKV: scale by 1/rms, rotate q and k, append k and v to the cache
+            TcLaunch L; memset(&L, 0, sizeof(L));
+            wseg(L, 0, lm.wq, qd); wseg(L, 1, lm.wk, kvd); wseg(L, 2, lm.wv, kvd); L.n_seg = 3;
+            L.k = c.d_model; L.epi = EPI_QKV_ROPE; L.ld_out = qd + 2 * kvd;
+            L.ssq_in = m->ws.ssq; L.ssq_in_n = ssq_n;
+            L.q_out = m->ws.q; L.kc = kc; L.vc = vc; L.cosv = m->ws.rope_cos; L.sinv = m->ws.rope_sin;
+            L.len_eff = m->ws.len_eff; L.depth = m->ws.tree->depth; L.rope_M = M; L.rope_H = c.n_heads; L.rope_Hkv = c.n_kv_heads;
+            L.max_batch = c.max_batch; L.max_ctx = c.max_ctx; L.layer_ord = ord;
+            if ((rc = gemm(VIASD_T_GEMM, L, m->maps_a))) return rc;
+        }
+        if ((rc = timed(m, VIASD_T_ATTENTION, st, [&] { return launch_attention(m, kc, vc, slim, ord, B, M, st); }))) return rc;
+        {   // O projection into the residual; prepare the input of the post-attention norm
+            TcLaunch L; memset(&L, 0, sizeof(L));
+            wseg(L, 0, lm.wo, c.d_model); L.n_seg = 1;
+            L.k = qd; L.epi = EPI_ADD_NORM; L.out_f32 = m->ws.h; L.ld_out = c.d_model;
+            L.next_gain = m->norm2[l]; L.next_act = m->ws.a; L.next_plane = R * c.d_model; L.ssq_out = m->ws.ssq;
+            if ((rc = gemm(VIASD_T_GEMM, L, m->maps_attn))) return rc;
+        }
+        {   // gate / up with SwiGLU
+            TcLaunch L; memset(&L, 0, sizeof(L));
+            wseg(L, 0, lm.wg, c.d_ff); wseg(L, 1, lm.wu, c.d_ff); L.n_seg = 2;
+            L.k = c.d_model; L.epi = EPI_SWIGLU; L.out_act = m->ws.act; L.act_plane = R * c.d_ff; L.ld_out = c.d_ff;
+            L.ssq_in = m->ws.ssq; L.ssq_in_n = ssq_n;
+            if ((rc = gemm(VIASD_T_GEMM, L, m->maps_a))) return rc;
+        }
+        {   // down projection into the residual; prepare the input of the next norm (next layer's or the final one)
+            TcLaunch L; memset(&L, 0, sizeof(L));
+            wseg(L, 0, lm.wd, c.d_model); L.n_seg = 1;
+            L.k = c.d_ff; L.epi = EPI_ADD_NORM; L.out_f32 = m->ws.h; L.ld_out = c.d_model;
+            L.next_gain = ord + 1 < n_run ? m->norm1[layer_id(ord + 1)] : m->final_norm;
+            L.next_act = m->ws.a; L.next_plane = R * c.d_model; L.ssq_out = m->ws.ssq;
+            if ((rc = gemm(VIASD_T_GEMM, L, m->maps_act))) return rc;
+        }
+    }
+    TcLaunch L; memset(&L, 0, sizeof(L));
+    wseg(L, 0, m->head_map, c.vocab); L.n_seg = 1;
+    L.k = c.d_model; L.epi = EPI_STORE; L.out_f32 = logits; L.ld_out = c.vocab;
+    L.ssq_in = m->ws.ssq; L.ssq_in_n = ssq_n;
+    return gemm(VIASD_T_GEMM, L, m->maps_a);
+}
+
 // One pass of the sub-network made of `layers` (all of them for q, the routed ones for q').
 int forward(viasd_model *m, const viasd_cache *cache, const viasd_draft *d, bool slim, float *logits,
             cudaStream_t st) {
     int rc;
     if ((rc = check_draft(m, d)) || (rc = check_cache(cache))) return rc;
     if (!logits) return VIASD_EINVAL;
+    if (m->fused) return forward_fused(m, cache, d, slim, logits, st);
     const viasd_config &c = m->cfg;
     const int B = d->batch, M = d->n_nodes + 1, rows = B * M;
     const int qd = c.n_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
@@ -235,6 +316,7 @@ int viasd_init_model(const viasd_config *cfg, const viasd_weights *w, const unsi
     CUDA_TRY(cudaGetDeviceProperties(&prop, dev));
     if (prop.major != 10) return VIASD_EUNSUPPORTED;
 
+    if (g_use_pdl < 0) { const char *e = getenv("VIASD_PDL"); g_use_pdl = (e && e[0] == '0') ? 0 : 1; }
     viasd_model *m = new (std::nothrow) viasd_model();
     if (!m) return VIASD_EINVAL;
     memset(&m->timer, 0, sizeof(m->timer));
@@ -265,6 +347,10 @@ int viasd_init_model(const viasd_config *cfg, const viasd_weights *w, const unsi
     {
         const char *force = getenv("VIASD_GEMM");
         m->use_tc = cfg->dtype == 1 && m->sm_count <= MAX_SMS && !(force && strcmp(force, "rowwarp") == 0);
+    }
+    {
+        const char *nf = getenv("VIASD_FUSED");
+        m->fused = m->use_tc && cfg->head_dim == 128 && cfg->d_model % 128 == 0 && !(nf && nf[0] == '0');
     }
     if (m->use_tc) {
         const uint64_t d = cfg->d_model, qd = (uint64_t)cfg->n_heads * cfg->head_dim,
@@ -454,6 +540,7 @@ int viasd_gemm(const void *x, const void *w, float *y, int rows, int n, int k, i
     if (!scratch || ((uintptr_t)scratch & 255)) return VIASD_EINVAL;
     if (scratch_bytes < viasd_gemm_scratch_bytes(rows, n, k)) return VIASD_ECAPACITY;
     cudaStream_t st = (cudaStream_t)stream;
+    if (g_use_pdl < 0) { const char *e = getenv("VIASD_PDL"); g_use_pdl = (e && e[0] == '0') ? 0 : 1; }
     const char *force = getenv("VIASD_GEMM");
     if (dtype == 0 || (force && strcmp(force, "rowwarp") == 0)) {
         GemmSegs s{{w, nullptr, nullptr}, {n, 0, 0}, 1};

@@ -20,6 +20,7 @@ attention_split_kernel(float *__restrict__ part, const float *__restrict__ q, co
     __shared__ float Ks[TK][HD + 1];
     __shared__ float Vs[TK][HD];
     constexpr int DPL = HD / 32;                     // output dims per lane
+    PDL_TRIGGER();
     const int b = blockIdx.x / Hkv, g = blockIdx.x % Hkv, split = blockIdx.y, qg = blockIdx.z;
     const int grp = H / Hkv, QR = grp * M;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -108,6 +109,7 @@ template <typename T, int HD>
 __global__ void attention_combine_kernel(T *__restrict__ out, size_t plane, const float *__restrict__ part, int M, int H,
                                          int nsplit) {
     const int r = blockIdx.x, h = blockIdx.y;        // r = b * M + i
+    PDL_TRIGGER();
     const int b = r / M, i = r % M;
     const float *src = part + (((size_t)b * H + h) * M + i) * (size_t)nsplit * (HD + 2);
     float mmax = -INFINITY;

@@ -192,6 +192,7 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) unsigned long long bars[NSTAGE];
     constexpr int MTW = 2;                                   // query tiles per warp at most
+    PDL_TRIGGER();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int b = blockIdx.x / a.Hkv, g = blockIdx.x % a.Hkv, split = blockIdx.y;
     const int grp = a.H / a.Hkv, QR = grp * a.M, QRP = a.mt * 16;

@@ -51,6 +51,7 @@ struct Workspace {                      // pointers into the caller's workspace 
     float *gemm_scratch;                // partial tiles of split GEMM work (tcgen05 kernel)
     int *gemm_counters;                 // per-tile arrival counters, zero between launches
     size_t n_counters;
+    float *ssq;                         // [(d / 128) * 4][R] partial sums of h^2 for the fused RMSNorm
 };
 
 struct WMap { CUtensorMap map; uint32_t box_rows; };        // TMA view of one weight matrix
@@ -80,6 +81,7 @@ struct viasd_model {
     int sm_count;
     // tcgen05 GEMM path (bf16 models)
     bool use_tc;
+    bool fused;                         // RMSNorm and rotary/append folded into the GEMM epilogues
     LayerMaps *lmaps;                   // [L]
     WMap head_map;
     ActMaps maps_a, maps_attn, maps_act;
@@ -96,6 +98,22 @@ extern unsigned long long g_launch_count;
     } while (0)
 #define LAUNCH_CHECK() do { ++g_launch_count; CUDA_TRY(cudaGetLastError()); } while (0)
 
+// Programmatic dependent launch: a kernel launched with this configuration may begin (prologue, weight
+// prefetch) while the kernel before it in the stream is still finishing; it must execute griddepcontrol.wait
+// before it touches anything that kernel reads or writes.  VIASD_PDL=0 turns the overlap off.
+extern int g_use_pdl;
+inline void pdl_config(cudaLaunchConfig_t &cfg, cudaLaunchAttribute *attr, dim3 grid, dim3 block, size_t smem,
+                       cudaStream_t st) {
+    cfg = cudaLaunchConfig_t{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_use_pdl ? 1 : 0;
+}
+#define PDL_WAIT() asm volatile("griddepcontrol.wait;" ::: "memory")
+#define PDL_TRIGGER() asm volatile("griddepcontrol.launch_dependents;" ::: "memory")
+
 // ---------------------------------------------------------------------------------------------
 // kernel launchers (one .cu file each); all enqueue on `st` and return a VIASD_* code
 // ---------------------------------------------------------------------------------------------
@@ -103,6 +121,7 @@ extern unsigned long long g_launch_count;
 int launch_rope_table(const viasd_model *m, cudaStream_t st);
 int launch_prep(const viasd_model *m, const viasd_cache *c, const viasd_draft *d, cudaStream_t st);
 int launch_embed(const viasd_model *m, int rows, cudaStream_t st);
+int launch_embed_norm(const viasd_model *m, const float *gain, int rows, cudaStream_t st);
 int launch_rmsnorm(const viasd_model *m, const float *gain, int rows, cudaStream_t st);
 int launch_rope_append(const viasd_model *m, void *kc, void *vc, int layer_ord, int batch, int M,
                        cudaStream_t st);
@@ -110,7 +129,7 @@ int launch_commit(const viasd_model *m, viasd_cache *c, const viasd_draft *d, co
                   cudaStream_t st);
 
 // gemm_rowwarp.cu -- generic CUDA-core GEMM (fp32 models; shapes the tensor-core kernels do not take)
-enum GemmEpilogue { EPI_STORE = 0, EPI_ADD = 1, EPI_SWIGLU = 2 };
+enum GemmEpilogue { EPI_STORE = 0, EPI_ADD = 1, EPI_SWIGLU = 2, EPI_ADD_NORM = 3, EPI_QKV_ROPE = 4 };
 struct GemmSegs { const void *w[3]; int n[3]; int count; };
 // x_plane / act_plane: element distance between the hi and lo planes (0: single plane)
 int launch_gemm_rowwarp(const void *x, size_t x_plane, const GemmSegs &segs, int rows, int k, int dtype,

@@ -124,22 +124,86 @@ __device__ __forceinline__ bool next_seg(int &u, int u1, int k_tiles, Seg &s) {
     return true;
 }
 
-// epilogue for one (feature lane, token row)
+// Epilogue for 16 token rows r0..r0+15 of one tile; thread f holds the full-K sums g (and u for the
+// gate/up pair) of output feature f.  Called by all 128 epilogue threads together.
 template <bool DUAL>
-__device__ __forceinline__ void finish(const TcParams &p, int tile, int f, int r, float g, float u) {
-    if (r >= p.rows) return;
+__device__ __forceinline__ void finish_chunk(const TcParams &p, int tile, int f, int r0, float (&g)[16], float (&uu)[16],
+                                             float *xch, const float *inv_sh, int lane) {
+    if (p.ssq_in) {                       // the input was h * gain without its RMS factor: apply it per row here
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const float sc = r0 + j < p.rows ? inv_sh[r0 + j] : 0.f;
+            g[j] *= sc;
+            if (DUAL) uu[j] *= sc;
+        }
+    }
     if (DUAL) {
         const int n = tile * TILE_F + f;
         if (n >= p.seg_n[0]) return;
-        const float s = g / (1.f + expf(-g));
-        store_act<__nv_bfloat16>(p.out_act, p.act_plane, (size_t)(p.row0 + r) * p.ld_out + n, s * u);
-    } else {
-        int s = 0, t0 = 0, nbase = 0;
-        while (s < 2 && tile >= p.seg_tile_end[s]) { t0 = p.seg_tile_end[s]; nbase += p.seg_n[s]; ++s; }
-        const int nin = (tile - t0) * TILE_F + f;
-        if (nin >= p.seg_n[s]) return;
-        float *dst = p.out_f32 + (size_t)(p.row0 + r) * p.ld_out + nbase + nin;
-        if (p.epi == EPI_ADD) *dst += g; else *dst = g;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            if (r0 + j >= p.rows) break;
+            const float sg = g[j] / (1.f + expf(-g[j]));
+            store_act<__nv_bfloat16>(p.out_act, p.act_plane, (size_t)(p.row0 + r0 + j) * p.ld_out + n, sg * uu[j]);
+        }
+        return;
+    }
+    int s = 0, t0 = 0, nbase = 0;
+    while (s < 2 && tile >= p.seg_tile_end[s]) { t0 = p.seg_tile_end[s]; nbase += p.seg_n[s]; ++s; }
+    const int nin = (tile - t0) * TILE_F + f;
+    const bool valid = nin < p.seg_n[s];
+    const int n = nbase + nin;
+    if (p.epi == EPI_STORE || p.epi == EPI_ADD) {
+        if (!valid) return;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            if (r0 + j >= p.rows) break;
+            float *dst = p.out_f32 + (size_t)(p.row0 + r0 + j) * p.ld_out + n;
+            if (p.epi == EPI_ADD) *dst += g[j]; else *dst = g[j];
+        }
+    } else if (p.epi == EPI_ADD_NORM) {
+        // residual update, plus what the next RMSNorm needs: h * gain as hi/lo planes and partial sums of h^2
+        const float gain = valid ? p.next_gain[n] : 0.f;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const int r = r0 + j;
+            if (r >= p.rows) break;
+            float v = 0.f;
+            if (valid) {
+                float *dst = p.out_f32 + (size_t)(p.row0 + r) * p.ld_out + n;
+                v = *dst + g[j];
+                *dst = v;
+                store_act<__nv_bfloat16>(p.next_act, p.next_plane, (size_t)(p.row0 + r) * p.ld_out + n, v * gain);
+            }
+            const float sq = warp_sum(v * v);
+            if (lane == 0) p.ssq_out[((size_t)tile * 4 + (f >> 5)) * p.ssq_stride + p.row0 + r] = sq;
+        }
+    } else {   // EPI_QKV_ROPE: one tile is one head of 128 dims; rotate pairs (p, p + 64), write q / K cache / V cache
+#pragma unroll
+        for (int j = 0; j < 16; ++j) xch[j * TILE_F + f] = g[j];
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        const int head = tile - t0, pidx = f & 63;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const int r = r0 + j;
+            if (r >= p.rows) break;
+            const int row = p.row0 + r, b = row / p.rope_M, i = row - b * p.rope_M;
+            const int n_ctx = p.len_eff[b], pos = n_ctx + p.depth[i], slot = n_ctx + i;
+            float y = g[j];
+            if (s < 2) {
+                const float c = p.cosv[(size_t)pos * 64 + pidx], sn = p.sinv[(size_t)pos * 64 + pidx];
+                const float other = xch[j * TILE_F + (f ^ 64)];
+                y = f < 64 ? g[j] * c - other * sn : g[j] * c + other * sn;
+            }
+            if (s == 0) {
+                p.q_out[((size_t)row * p.rope_H + head) * TILE_F + f] = y;
+            } else {
+                __nv_bfloat16 *cache = s == 1 ? p.kc : p.vc;
+                cache[((((size_t)p.layer_ord * p.max_batch + b) * p.rope_Hkv + head) * p.max_ctx + slot) * TILE_F + f] =
+                    __float2bfloat16_rn(y);
+            }
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
     }
 }
 
@@ -151,8 +215,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
     __shared__ __align__(8) unsigned long long bars[2 * MAX_STAGES + 4];
     __shared__ uint32_t tmem_base_sh;
     __shared__ int abort_sh, last_sh;
+    __shared__ float inv_sh[128];                       // per-row 1/rms of the input (fused RMSNorm)
+    __shared__ float xch[16 * TILE_F];                  // rotary partner exchange
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may start its prologue
     if (threadIdx.x == 0) TRACE(0);
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int NT = p.nt, S = p.stages;
@@ -192,30 +259,50 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            int it = 0, u = u_begin;
-            Seg sg;
-            bool ok = true;
-            while (ok && next_seg(u, u_end, p.k_tiles, sg)) {
-                // which weight matrix and which of its rows this tile covers
+            const int n_it = u_end - u_begin;
+            // unit -> weight matrix, its first row, k-block
+            auto unit = [&](int it, const CUtensorMap *&mw, int &wrow, int &kt, int &sidx) {
+                const int u = u_begin + it, tile = u / p.k_tiles;
+                kt = u - tile * p.k_tiles;
                 int s = 0, t0 = 0;
-                if (!DUAL) while (s < 2 && sg.tile >= p.seg_tile_end[s]) { t0 = p.seg_tile_end[s]; ++s; }
-                const CUtensorMap *mw = s == 0 ? &map_w0 : (s == 1 ? &map_w1 : &map_w2);
-                const int wrow = (sg.tile - t0) * TILE_F;
-                uint32_t tx = DUAL ? 2 * p.a_tx[0] + 2 * p.b_tx : p.a_tx[s] + 2 * p.b_tx;
-                if (DBG(p, 1)) tx -= 2 * p.b_tx;
-                for (int kt = sg.ka; kt < sg.kb; ++kt, ++it) {
-                    const int st = it % S;
-                    if (!(ok = mbar_wait(empty_bar(st), ((it / S) & 1) ^ 1, &abort_sh, p.status))) break;
-                    const uint32_t base = smem_base + st * stage_bytes;
-                    mbar_expect_tx(full_bar(st), tx);
-                    tma_load_2d(base, mw, full_bar(st), kt * TILE_K, wrow);
-                    if (DUAL) tma_load_2d(base + a_bytes, &map_w1, full_bar(st), kt * TILE_K, wrow);
-                    if (!DBG(p, 1)) {
-                    tma_load_2d(base + NACC * a_bytes, &map_x, full_bar(st), kt * TILE_K, p.row0);
-                    tma_load_2d(base + NACC * a_bytes + b_bytes, &map_x, full_bar(st), kt * TILE_K,
-                                p.row0 + p.lo_row_offset);
-                    }
-                }
+                if (!DUAL) while (s < 2 && tile >= p.seg_tile_end[s]) { t0 = p.seg_tile_end[s]; ++s; }
+                mw = s == 0 ? &map_w0 : (s == 1 ? &map_w1 : &map_w2);
+                wrow = (tile - t0) * TILE_F;
+                sidx = s;
+            };
+            auto load_w = [&](int st, const CUtensorMap *mw, int wrow, int kt) {
+                const uint32_t base = smem_base + st * stage_bytes;
+                tma_load_2d(base, mw, full_bar(st), kt * TILE_K, wrow);
+                if (DUAL) tma_load_2d(base + a_bytes, &map_w1, full_bar(st), kt * TILE_K, wrow);
+            };
+            auto load_x = [&](int st, int kt) {
+                const uint32_t base = smem_base + st * stage_bytes + NACC * a_bytes;
+                tma_load_2d(base, &map_x, full_bar(st), kt * TILE_K, p.row0);
+                tma_load_2d(base + b_bytes, &map_x, full_bar(st), kt * TILE_K, p.row0 + p.lo_row_offset);
+            };
+            const CUtensorMap *mw; int wrow, kt, sidx;
+            // Weights do not depend on the kernel before this one: fill the ring with them first, and only then
+            // wait for that kernel (programmatic dependent launch) before touching the activations.
+            const int pre = n_it < S ? n_it : S;
+            for (int it = 0; it < pre; ++it) {
+                unit(it, mw, wrow, kt, sidx);
+                asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(full_bar(it)),
+                             "r"(DUAL ? 2 * p.a_tx[0] : p.a_tx[sidx]) : "memory");
+                load_w(it, mw, wrow, kt);
+            }
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            for (int it = 0; it < pre; ++it) {
+                unit(it, mw, wrow, kt, sidx);
+                mbar_expect_tx(full_bar(it), 2 * p.b_tx);
+                load_x(it, kt);
+            }
+            for (int it = pre; it < n_it; ++it) {
+                const int st = it % S;
+                if (!mbar_wait(empty_bar(st), ((it / S) & 1) ^ 1, &abort_sh, p.status)) break;
+                unit(it, mw, wrow, kt, sidx);
+                mbar_expect_tx(full_bar(st), (DUAL ? 2 * p.a_tx[0] : p.a_tx[sidx]) + 2 * p.b_tx);
+                load_w(st, mw, wrow, kt);
+                load_x(st, kt);
             }
         }
     } else if (warp == 1) {
@@ -253,10 +340,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
         }
     } else {
         // ---------------- epilogue (warps 2..5 <-> TMEM lane quarters 2,3,0,1) ----------------
+        asm volatile("griddepcontrol.wait;" ::: "memory");     // outputs, scratch and counters belong to the chain
         const int quarter = warp & 3;
         const int f = quarter * 32 + lane;                  // feature lane inside the tile
         const int et = threadIdx.x - 64;                    // 0..127 among epilogue threads
         const size_t slot_floats = (size_t)NACC * NT * TILE_F;
+        if (p.ssq_in) {
+            for (int r = et; r < p.rows; r += 128) {
+                float ss = 0.f;
+                for (int j = 0; j < p.ssq_in_n; ++j) ss += __ldcg(p.ssq_in + (size_t)j * p.ssq_stride + p.row0 + r);
+                inv_sh[r] = rsqrtf(ss * p.inv_d + p.eps);
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+        }
         int acc_it = 0, u = u_begin, seg_i = 0;
         Seg sg;
         bool ok = true;
@@ -285,8 +381,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                     }
                 }
                 if (whole) {
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) finish<DUAL>(p, sg.tile, f, c + j, g[j], DUAL ? uu[j] : 0.f);
+                    finish_chunk<DUAL>(p, sg.tile, f, c, g, uu, xch, inv_sh, lane);
                 } else {
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
@@ -329,8 +424,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                                 }
                             }
                         }
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) finish<DUAL>(p, sg.tile, et, r0 + j, g[j], uu[j]);
+                        finish_chunk<DUAL>(p, sg.tile, et, r0, g, uu, xch, inv_sh, lane);
                     }
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");   // last_sh is reused by the next split tile
@@ -426,6 +520,11 @@ int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {
     p.scratch = L.scratch;
     p.counters = L.counters;
     p.status = L.status;
+    p.ssq_in = L.ssq_in; p.ssq_in_n = L.ssq_in_n; p.ssq_stride = L.ssq_stride; p.inv_d = L.inv_d; p.eps = L.eps;
+    p.next_gain = L.next_gain; p.next_act = (__nv_bfloat16 *)L.next_act; p.next_plane = L.next_plane; p.ssq_out = L.ssq_out;
+    p.q_out = L.q_out; p.kc = (__nv_bfloat16 *)L.kc; p.vc = (__nv_bfloat16 *)L.vc; p.cosv = L.cosv; p.sinv = L.sinv;
+    p.len_eff = L.len_eff; p.depth = L.depth; p.rope_M = L.rope_M; p.rope_H = L.rope_H; p.rope_Hkv = L.rope_Hkv;
+    p.max_batch = L.max_batch; p.max_ctx = L.max_ctx; p.layer_ord = L.layer_ord;
     const int units = p.n_tiles * p.k_tiles;
     if (units <= 0) return VIASD_OK;
     int ctas_per_sm = 1;
@@ -437,7 +536,10 @@ int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {
     grid = (units + p.units_per_cta - 1) / p.units_per_cta;
     const int nacc = dual ? 2 : 1;
     const size_t stage = (size_t)nacc * TILE_F * TILE_K * 2 + 2 * (size_t)L.nt * TILE_K * 2;
-    int stages = (int)((size_t)200 * 1024 / stage);
+    // a ring of about 100 KB keeps HBM busy (deeper rings measured no faster) and lets the CTA of the next
+    // kernel in the stream become resident beside this one, so that its weight prefetch overlaps this tail
+    int stages = (int)((size_t)104 * 1024 / stage);
+    if (stages < 2) stages = 2;
     if (stages > MAX_STAGES) stages = MAX_STAGES;
 #ifdef VIASD_TC_TRACE
     if (getenv("VIASD_TC_DBG")) p.dbg = atoi(getenv("VIASD_TC_DBG"));
@@ -458,8 +560,11 @@ int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {
         attr_done[dual] = true;
     }
     const CUtensorMap &w0 = *L.map_w[0], &w1 = *L.map_w[L.n_seg > 1 ? 1 : 0], &w2 = *L.map_w[L.n_seg > 2 ? 2 : 0];
-    if (dual) gemm_tc_kernel<true><<<grid, THREADS, smem, st>>>(w0, w1, w2, *L.map_x, p);
-    else gemm_tc_kernel<false><<<grid, THREADS, smem, st>>>(w0, w1, w2, *L.map_x, p);
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    pdl_config(cfg, attr, dim3(grid), dim3(THREADS), smem, st);
+    if (dual) CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<true>, w0, w1, w2, *L.map_x, p));
+    else CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<false>, w0, w1, w2, *L.map_x, p));
     LAUNCH_CHECK();
     return VIASD_OK;
 }

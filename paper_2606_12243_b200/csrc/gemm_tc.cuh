@@ -22,6 +22,13 @@ struct TcParams {                       // kernel argument block
     int *counters;                      // [n_tiles], zero between launches
     int *status;                        // device status word
     int dbg;                            // measurement knobs, honoured by trace builds only
+    // fused RMSNorm on the input side: per-row partial sums of squares written by the producer
+    const float *ssq_in; int ssq_in_n, ssq_stride; float inv_d, eps;
+    // EPI_ADD_NORM: what the next RMSNorm needs
+    const float *next_gain; __nv_bfloat16 * next_act; size_t next_plane; float *ssq_out;
+    // EPI_QKV_ROPE
+    float *q_out; __nv_bfloat16 *kc, *vc; const float *cosv, *sinv; const int *len_eff, *depth;
+    int rope_M, rope_H, rope_Hkv, max_batch, max_ctx, layer_ord;
 };
 
 struct TcLaunch {                       // host-side description of one GEMM
@@ -41,6 +48,13 @@ struct TcLaunch {                       // host-side description of one GEMM
     int *counters;
     int *status;
     int sm_count;
+    // fused RMSNorm on the input side: per-row partial sums of squares written by the producer
+    const float *ssq_in; int ssq_in_n, ssq_stride; float inv_d, eps;
+    // EPI_ADD_NORM: what the next RMSNorm needs
+    const float *next_gain; void * next_act; size_t next_plane; float *ssq_out;
+    // EPI_QKV_ROPE
+    float *q_out; void *kc, *vc; const float *cosv, *sinv; const int *len_eff, *depth;
+    int rope_M, rope_H, rope_Hkv, max_batch, max_ctx, layer_ord;
 };
 
 // 2-D bf16 tensor [rows, k] row-major -> TMA map with a (64 x box_rows) box and the 128-byte swizzle

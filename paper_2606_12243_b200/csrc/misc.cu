@@ -32,6 +32,7 @@ __global__ void prep_kernel(TreeInfo *tree, int *len_eff, int *row_tok, DeviceSt
                             const int *pending, const int *draft_tok, const int *parent, int B, int N,
                             int max_ctx, int vocab) {
     const int M = N + 1;
+    PDL_TRIGGER();
     if (threadIdx.x == 0) {
         int last_child[VIASD_MAX_ROWS_PER_SEQ];
         for (int i = 0; i < M; ++i) { tree->first_child[i] = -1; tree->next_sibling[i] = -1; last_child[i] = -1; }
@@ -77,8 +78,38 @@ int launch_prep(const viasd_model *m, const viasd_cache *c, const viasd_draft *d
 template <typename T>
 __global__ void embed_kernel(float *h, const T *E, const int *row_tok, int d) {
     int r = blockIdx.x;
+    PDL_TRIGGER();
     const T *src = E + (size_t)row_tok[r] * d;
     for (int i = threadIdx.x; i < d; i += blockDim.x) h[(size_t)r * d + i] = to_f32<T>(src[i]);
+}
+
+// Embedding gather fused with the preparation of the first RMSNorm of the pass (tensor-core path):
+// h = E[tok]; a = hi/lo(h * gain); partial sums of h^2 per 32 features in the layout the GEMM epilogue reads.
+__global__ void __launch_bounds__(256)
+embed_norm_kernel(float *h, __nv_bfloat16 *a, size_t plane, float *ssq, int ssq_stride, const __nv_bfloat16 *E,
+                  const float *gain, const int *row_tok, int d) {
+    const int r = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    PDL_TRIGGER();
+    const __nv_bfloat16 *src = E + (size_t)row_tok[r] * d;
+    for (int base = 0; base < d; base += 256) {
+        const int i = base + warp * 32 + lane;            // d is a multiple of 128: whole warps stay in range
+        float v = 0.f;
+        if (base + warp * 32 < d) {
+            v = __bfloat162float(src[i]);
+            h[(size_t)r * d + i] = v;
+            store_act<__nv_bfloat16>(a, plane, (size_t)r * d + i, v * gain[i]);
+            const float sq = warp_sum(v * v);
+            if (lane == 0) ssq[(size_t)(i >> 5) * ssq_stride + r] = sq;   // (tile * 4 + quarter) == feature / 32
+        }
+    }
+}
+
+int launch_embed_norm(const viasd_model *m, const float *gain, int rows, cudaStream_t st) {
+    embed_norm_kernel<<<rows, 256, 0, st>>>(m->ws.h, (__nv_bfloat16 *)m->ws.a, m->ws.rows_alloc * m->cfg.d_model, m->ws.ssq,
+                                            (int)m->ws.rows_alloc, (const __nv_bfloat16 *)m->embed, gain, m->ws.row_tok,
+                                            m->cfg.d_model);
+    LAUNCH_CHECK();
+    return VIASD_OK;
 }
 
 int launch_embed(const viasd_model *m, int rows, cudaStream_t st) {
@@ -95,23 +126,44 @@ int launch_embed(const viasd_model *m, int rows, cudaStream_t st) {
 // RMSNorm: a[r] = h[r] / sqrt(mean(h[r]^2) + eps) * gain, written in the model dtype
 // ---------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void rmsnorm_kernel(T *a, size_t plane, const float *h, const float *gain, int d, float eps) {
-    __shared__ float red[32];
-    int r = blockIdx.x;
-    const float *x = h + (size_t)r * d;
+__global__ void __launch_bounds__(256)
+rmsnorm_kernel(T *a, size_t plane, const float *h, const float *gain, int d, float eps) {
+    __shared__ float red[8];
+    PDL_TRIGGER();
+    const int r = blockIdx.x;
+    const float4 *x4 = reinterpret_cast<const float4 *>(h + (size_t)r * d);
+    const float4 *g4 = reinterpret_cast<const float4 *>(gain);
+    constexpr int MAXV = 8;                           // up to 8 float4 per thread: d <= 8192 stays in registers
+    const int nv = d >> 2;
+    float4 v[MAXV];
     float s = 0.f;
-    for (int i = threadIdx.x; i < d; i += blockDim.x) { float v = x[i]; s += v * v; }
+#pragma unroll
+    for (int j = 0; j < MAXV; ++j) {
+        const int i = threadIdx.x + j * 256;
+        if (i < nv) { v[j] = x4[i]; s += v[j].x * v[j].x + v[j].y * v[j].y + v[j].z * v[j].z + v[j].w * v[j].w; }
+    }
+    for (int i = threadIdx.x + MAXV * 256; i < nv; i += 256) { float4 t = x4[i]; s += t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w; }
     s = warp_sum(s);
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = s;
     __syncthreads();
-    if (threadIdx.x < 32) {
-        float v = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0.f;
-        v = warp_sum(v);
-        if (threadIdx.x == 0) red[0] = rsqrtf(v / (float)d + eps);
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += red[w];
+    const float inv = rsqrtf(tot / (float)d + eps);
+    auto emit = [&](int i, float4 t) {
+        const float4 g = g4[i];
+        const size_t o = (size_t)r * d + (size_t)i * 4;
+        store_act<T>(a, plane, o, t.x * inv * g.x);
+        store_act<T>(a, plane, o + 1, t.y * inv * g.y);
+        store_act<T>(a, plane, o + 2, t.z * inv * g.z);
+        store_act<T>(a, plane, o + 3, t.w * inv * g.w);
+    };
+#pragma unroll
+    for (int j = 0; j < MAXV; ++j) {
+        const int i = threadIdx.x + j * 256;
+        if (i < nv) emit(i, v[j]);
     }
-    __syncthreads();
-    float inv = red[0];
-    for (int i = threadIdx.x; i < d; i += blockDim.x) store_act<T>(a, plane, (size_t)r * d + i, x[i] * inv * gain[i]);
+    for (int i = threadIdx.x + MAXV * 256; i < nv; i += 256) emit(i, x4[i]);
 }
 
 int launch_rmsnorm(const viasd_model *m, const float *gain, int rows, cudaStream_t st) {
@@ -132,6 +184,7 @@ __global__ void rope_append_kernel(float *q_out, T *kc, T *vc, const float *qkv,
                                    const int *len_eff, const TreeInfo *tree, int M, int H, int Hkv, int hd,
                                    int max_batch, int max_ctx, int layer_ord) {
     int r = blockIdx.x, head = blockIdx.y;
+    PDL_TRIGGER();
     int b = r / M, i = r % M;
     int half = hd >> 1;
     int n = len_eff[b];
