@@ -168,6 +168,23 @@ size_t viasd_gemm_scratch_bytes(int rows, int n, int k);
 int viasd_gemm(const void *x, const void *w, float *y, int rows, int n, int k, int dtype, void *scratch,
                size_t scratch_bytes, void *stream);
 
+/* Same product as viasd_gemm for bf16 operands (y[rows, n] = x[rows, k] * W[n, k]^T, fp32 y) for callers that
+ * cannot allocate device memory and therefore have no scratch to hand over: a serving process that gave all
+ * of its HBM to weights and KV caches at start-up (a later cudaMalloc fails, or stalls every stream of the
+ * device while it runs), or code running inside a host framework's callback where allocation calls are
+ * forbidden.  The paper has no counterpart; this is plumbing.
+ * The scratch (tile counters and partial tiles, about 2.6 MB) is a fixed array inside the library image: every
+ * GPU that loads the library holds it until the process exits.  Limits: rows <= 16 and n <= 262144; larger
+ * sizes return VIASD_ECAPACITY and launch nothing.  The call makes no cudaMalloc / cudaFree and uses no
+ * allocating library routine.
+ * The first call on each device looks up the array's device address (with that device current); make that
+ * first call before starting any stream capture on the device.
+ * All calls on a device share the one array: the counters are cleared at the start of every call, the rest
+ * keeps the previous call's contents and is overwritten.  Two calls that overlap on the GPU (different
+ * streams, or different host threads) race on it and give wrong results; serialise them.
+ * Errors: EINVAL (null / misaligned pointer, k not a multiple of 8), ECAPACITY, ECUDA, EUNSUPPORTED. */
+int viasd_gemm_static(const void *x, const void *w, float *y, int rows, int n, int k, void *stream);
+
 /* Measurement hooks (the paper has no counterpart; they exist so that a benchmark can attribute time).
  * viasd_launch_count: kernels launched by this library in this process so far.
  * viasd_set_timing(on): when on, every launch of the forward / tier / accept / commit path is bracketed by

@@ -21,7 +21,7 @@ VIASD_OK, VIASD_EINVAL, VIASD_ECAPACITY, VIASD_ECUDA, VIASD_EDEVICE, VIASD_EUNSU
 EXPORTS = ["viasd_workspace_bytes", "viasd_init_model", "viasd_full_forward", "viasd_slim_forward",
            "viasd_tier_accept", "viasd_kv_commit", "viasd_verify_step", "viasd_get_stats",
            "viasd_free_model", "viasd_strerror", "viasd_last_cuda_error", "viasd_gemm_scratch_bytes",
-           "viasd_gemm", "viasd_launch_count", "viasd_set_timing", "viasd_get_timing"]
+           "viasd_gemm", "viasd_gemm_static", "viasd_launch_count", "viasd_set_timing", "viasd_get_timing"]
 
 TIMING_CLASSES = ["gemm", "attention", "norm", "rope", "embed", "tier_accept", "commit"]
 
@@ -113,6 +113,7 @@ def lib() -> C.CDLL:
         l.viasd_gemm_scratch_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
         l.viasd_gemm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int,
                                  C.c_void_p, C.c_size_t, C.c_void_p]
+        l.viasd_gemm_static.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p]
         l.viasd_launch_count.restype = C.c_ulonglong
         l.viasd_set_timing.argtypes = [C.c_void_p, C.c_int]
         l.viasd_get_timing.argtypes = [C.c_void_p, C.POINTER(Timing), C.c_void_p]
@@ -288,3 +289,15 @@ def get_timing(m: Model, stream=None) -> dict:
     out = {n: {"ms": t.ms[i], "launches": int(t.launches[i])} for i, n in enumerate(TIMING_CLASSES)}
     out["dropped"] = int(t.dropped)
     return out
+
+
+def gemm_static(x: torch.Tensor, w: torch.Tensor, y: torch.Tensor, stream=None) -> None:
+    """viasd_gemm_static: bf16 x [rows, k], W [n, k] -> fp32 y [rows, n] with the library's built-in scratch.
+
+    For callers that must not allocate (no scratch tensor to pass).  rows <= 16, n <= 262144.  Calls on one
+    device share the scratch: do not let two of them overlap on the GPU.
+    """
+    rows, k = x.shape
+    n = w.shape[0]
+    assert x.dtype == torch.bfloat16 and w.dtype == torch.bfloat16 and y.dtype == torch.float32
+    _check(lib().viasd_gemm_static(_ptr(x), _ptr(w), _ptr(y), rows, n, k, _stream(stream)), "viasd_gemm_static")
