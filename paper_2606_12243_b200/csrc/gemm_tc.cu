@@ -87,16 +87,15 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
-__device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
-    uint32_t r[16];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr));
+constexpr int CH = 8;                // token rows per epilogue chunk
+__device__ __forceinline__ void tc_ld8(uint32_t taddr, float (&v)[CH]) {
+    uint32_t r[8];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr));
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
 }
 
 // K-major operand tile, 128-byte swizzle, rows 128 bytes apart, 8-row groups 1024 bytes apart
@@ -106,9 +105,15 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
 
 #ifdef VIASD_TC_TRACE
 __device__ long long g_tc_trace[160 * 8];
-#define TRACE(slot) do { g_tc_trace[blockIdx.x * 8 + (slot)] = clock64(); } while (0)
+#define TRACE(slot) do { if (p.trace_on) g_tc_trace[blockIdx.x * 8 + (slot)] = clock64(); } while (0)
 #define DBG(p, bit) ((p).dbg & (bit))
+__device__ unsigned long long g_tc_span[8192 * 2];       // per launch: earliest CTA start, latest CTA end (globaltimer ns)
+__device__ __forceinline__ unsigned long long gtimer() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define SPAN_BEGIN(p) do { if (threadIdx.x == 0) atomicMin(&g_tc_span[((p).launch_idx & 8191) * 2], gtimer()); } while (0)
+#define SPAN_END(p) do { if (threadIdx.x == 0) atomicMax(&g_tc_span[((p).launch_idx & 8191) * 2 + 1], gtimer()); } while (0)
 #else
+#define SPAN_BEGIN(p) do { } while (0)
+#define SPAN_END(p) do { } while (0)
 #define DBG(p, bit) 0
 #define TRACE(slot) do { } while (0)
 #endif
@@ -124,27 +129,35 @@ __device__ __forceinline__ bool next_seg(int &u, int u1, int k_tiles, Seg &s) {
     return true;
 }
 
-// Epilogue for 16 token rows r0..r0+15 of one tile; thread f holds the full-K sums g (and u for the
-// gate/up pair) of output feature f.  Called by all 128 epilogue threads together.
-template <bool DUAL>
-__device__ __forceinline__ void finish_chunk(const TcParams &p, int tile, int f, int r0, float (&g)[16], float (&uu)[16],
-                                             float *xch, const float *inv_sh, int lane) {
-    if (p.ssq_in) {                       // the input was h * gain without its RMS factor: apply it per row here
+// Epilogue for CH token rows r0..r0+CH-1 of one tile; thread f holds the full-K sums g (and u for the gate/up
+// pair) of output feature f.  Called by all 128 epilogue threads together.  The epilogue kind is a template
+// parameter so that each kernel carries one short epilogue: this code runs once per tile, straight from the
+// instruction cache's cold side, and its size is what its latency is made of.
+template <int EPI>
+__device__ __forceinline__ void finish_chunk(const TcParams &p, int tile, int f, int r0, float (&g)[CH], float (&uu)[CH],
+                                             float *xch, const float *inv_sh, const int4 *rowmeta, int lane) {
+    constexpr bool DUAL = EPI == EPI_SWIGLU;
+    if (EPI == EPI_STORE || EPI == EPI_SWIGLU || EPI == EPI_QKV_ROPE) {
+        if (p.ssq_in) {                   // the input was h * gain without its RMS factor: apply it per row here
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            const float sc = r0 + j < p.rows ? inv_sh[r0 + j] : 0.f;
-            g[j] *= sc;
-            if (DUAL) uu[j] *= sc;
+            for (int j = 0; j < CH; ++j) {
+                const float sc = inv_sh[min(r0 + j, 127)];
+                g[j] *= sc;
+                if (DUAL) uu[j] *= sc;
+            }
         }
     }
+    const int nrow = min(CH, p.rows - r0);
     if (DUAL) {
         const int n = tile * TILE_F + f;
         if (n >= p.seg_n[0]) return;
+        __nv_bfloat16 *dst = p.out_act + (size_t)(p.row0 + r0) * p.ld_out + n;
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            if (r0 + j >= p.rows) break;
-            const float sg = g[j] / (1.f + expf(-g[j]));
-            store_act<__nv_bfloat16>(p.out_act, p.act_plane, (size_t)(p.row0 + r0 + j) * p.ld_out + n, sg * uu[j]);
+        for (int j = 0; j < CH; ++j) {
+            if (j < nrow) {
+                const float sg = g[j] / (1.f + __expf(-g[j]));
+                store_act<__nv_bfloat16>(dst, p.act_plane, (size_t)j * p.ld_out, sg * uu[j]);
+            }
         }
         return;
     }
@@ -153,61 +166,82 @@ __device__ __forceinline__ void finish_chunk(const TcParams &p, int tile, int f,
     const int nin = (tile - t0) * TILE_F + f;
     const bool valid = nin < p.seg_n[s];
     const int n = nbase + nin;
-    if (p.epi == EPI_STORE || p.epi == EPI_ADD) {
+    if (EPI == EPI_STORE) {
         if (!valid) return;
+        float *dst = p.out_f32 + (size_t)(p.row0 + r0) * p.ld_out + n;
+        if (p.epi == EPI_ADD) {
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            if (r0 + j >= p.rows) break;
-            float *dst = p.out_f32 + (size_t)(p.row0 + r0 + j) * p.ld_out + n;
-            if (p.epi == EPI_ADD) *dst += g[j]; else *dst = g[j];
+            for (int j = 0; j < CH; ++j) if (j < nrow) dst[(size_t)j * p.ld_out] += g[j];
+        } else {
+#pragma unroll
+            for (int j = 0; j < CH; ++j) if (j < nrow) dst[(size_t)j * p.ld_out] = g[j];
         }
-    } else if (p.epi == EPI_ADD_NORM) {
-        // residual update, plus what the next RMSNorm needs: h * gain as hi/lo planes and partial sums of h^2
+    } else if (EPI == EPI_ADD_NORM) {
+        // residual update, plus what the next RMSNorm needs: h * gain as hi/lo planes and partial sums of h^2.
+        // Loads first, then arithmetic, then stores: the CH rows cost one memory round trip.
         const float gain = valid ? p.next_gain[n] : 0.f;
+        float *hp = p.out_f32 + (size_t)(p.row0 + r0) * p.ld_out + n;
+        __nv_bfloat16 *ap = p.next_act + (size_t)(p.row0 + r0) * p.ld_out + n;
+        float v[CH];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            const int r = r0 + j;
-            if (r >= p.rows) break;
-            float v = 0.f;
-            if (valid) {
-                float *dst = p.out_f32 + (size_t)(p.row0 + r) * p.ld_out + n;
-                v = *dst + g[j];
-                *dst = v;
-                store_act<__nv_bfloat16>(p.next_act, p.next_plane, (size_t)(p.row0 + r) * p.ld_out + n, v * gain);
+        for (int j = 0; j < CH; ++j) v[j] = (valid && j < nrow) ? __ldcg(hp + (size_t)j * p.ld_out) + g[j] : 0.f;
+#pragma unroll
+        for (int j = 0; j < CH; ++j) {
+            if (valid && j < nrow) {
+                hp[(size_t)j * p.ld_out] = v[j];
+                store_act<__nv_bfloat16>(ap, p.next_plane, (size_t)j * p.ld_out, v[j] * gain);
             }
-            const float sq = warp_sum(v * v);
-            if (lane == 0) p.ssq_out[((size_t)tile * 4 + (f >> 5)) * p.ssq_stride + p.row0 + r] = sq;
+            v[j] *= v[j];
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+            for (int j = 0; j < CH; ++j) v[j] += __shfl_xor_sync(0xffffffffu, v[j], o);
+        if (lane < nrow) {
+            float mine = v[0];
+#pragma unroll
+            for (int j = 1; j < CH; ++j) mine = lane == j ? v[j] : mine;
+            p.ssq_out[((size_t)tile * 4 + (f >> 5)) * p.ssq_stride + p.row0 + r0 + lane] = mine;
         }
     } else {   // EPI_QKV_ROPE: one tile is one head of 128 dims; rotate pairs (p, p + 64), write q / K cache / V cache
 #pragma unroll
-        for (int j = 0; j < 16; ++j) xch[j * TILE_F + f] = g[j];
+        for (int j = 0; j < CH; ++j) xch[j * TILE_F + f] = g[j];
         asm volatile("bar.sync 1, 128;" ::: "memory");
         const int head = tile - t0, pidx = f & 63;
+        if (s < 2) {
+            float c[CH], sn[CH];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            const int r = r0 + j;
-            if (r >= p.rows) break;
-            const int row = p.row0 + r, b = row / p.rope_M, i = row - b * p.rope_M;
-            const int n_ctx = p.len_eff[b], pos = n_ctx + p.depth[i], slot = n_ctx + i;
-            float y = g[j];
-            if (s < 2) {
-                const float c = p.cosv[(size_t)pos * 64 + pidx], sn = p.sinv[(size_t)pos * 64 + pidx];
-                const float other = xch[j * TILE_F + (f ^ 64)];
-                y = f < 64 ? g[j] * c - other * sn : g[j] * c + other * sn;
+            for (int j = 0; j < CH; ++j) {
+                const int pos = rowmeta[min(r0 + j, 127)].x;
+                c[j] = p.cosv[(size_t)pos * 64 + pidx];
+                sn[j] = p.sinv[(size_t)pos * 64 + pidx];
             }
-            if (s == 0) {
-                p.q_out[((size_t)row * p.rope_H + head) * TILE_F + f] = y;
-            } else {
-                __nv_bfloat16 *cache = s == 1 ? p.kc : p.vc;
-                cache[((((size_t)p.layer_ord * p.max_batch + b) * p.rope_Hkv + head) * p.max_ctx + slot) * TILE_F + f] =
-                    __float2bfloat16_rn(y);
+#pragma unroll
+            for (int j = 0; j < CH; ++j) {
+                const float other = xch[j * TILE_F + (f ^ 64)];
+                g[j] = f < 64 ? g[j] * c[j] - other * sn[j] : g[j] * c[j] + other * sn[j];
+            }
+        }
+        if (s == 0) {
+            float *dst = p.q_out + ((size_t)(p.row0 + r0) * p.rope_H + head) * TILE_F + f;
+#pragma unroll
+            for (int j = 0; j < CH; ++j) if (j < nrow) dst[(size_t)j * p.rope_H * TILE_F] = g[j];
+        } else {
+            __nv_bfloat16 *cache = s == 1 ? p.kc : p.vc;
+#pragma unroll
+            for (int j = 0; j < CH; ++j) {
+                if (j < nrow) {
+                    const int4 rm = rowmeta[r0 + j];
+                    cache[((((size_t)p.layer_ord * p.max_batch + rm.z) * p.rope_Hkv + head) * p.max_ctx + rm.y) * TILE_F + f] =
+                        __float2bfloat16_rn(g[j]);
+                }
             }
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
     }
 }
 
-template <bool DUAL>
+template <int EPI>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
                const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_x, const TcParams p) {
@@ -216,11 +250,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
     __shared__ uint32_t tmem_base_sh;
     __shared__ int abort_sh, last_sh;
     __shared__ float inv_sh[128];                       // per-row 1/rms of the input (fused RMSNorm)
-    __shared__ float xch[16 * TILE_F];                  // rotary partner exchange
+    __shared__ float xch[CH * TILE_F];                  // rotary partner exchange
+    __shared__ int4 rowmeta[128];                       // per token row: rotary position, cache slot, sequence
 
+    constexpr bool DUAL = EPI == EPI_SWIGLU;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may start its prologue
     if (threadIdx.x == 0) TRACE(0);
+    SPAN_BEGIN(p);
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int NT = p.nt, S = p.stages;
     constexpr int NACC = DUAL ? 2 : 1;
@@ -320,7 +357,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                 for (int kt = sg.ka; kt < sg.kb; ++kt, ++it) {
                     const int st = it % S;
                     if (!(ok = mbar_wait(full_bar(st), (it / S) & 1, &abort_sh, p.status))) break;
-                    if (it == 0) TRACE(2);
                     tc_fence_after();
                     const uint32_t base = smem_base + st * stage_bytes;
                     // the hi tile is followed by the lo tile: together one K-major operand of NB rows
@@ -345,14 +381,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
         const int f = quarter * 32 + lane;                  // feature lane inside the tile
         const int et = threadIdx.x - 64;                    // 0..127 among epilogue threads
         const size_t slot_floats = (size_t)NACC * NT * TILE_F;
+        // per-row tables (all 128 entries defined: chunks read a few rows past p.rows and discard them)
+        inv_sh[et] = 0.f;
+        rowmeta[et] = make_int4(0, 0, 0, 0);
+        asm volatile("bar.sync 1, 128;" ::: "memory");
         if (p.ssq_in) {
-            for (int r = et; r < p.rows; r += 128) {
+            // 1/rms per input row: a warp sums the row's partial sums of squares (fixed order: reproducible)
+            for (int r = (et >> 5); r < p.rows; r += 4) {
                 float ss = 0.f;
-                for (int j = 0; j < p.ssq_in_n; ++j) ss += __ldcg(p.ssq_in + (size_t)j * p.ssq_stride + p.row0 + r);
-                inv_sh[r] = rsqrtf(ss * p.inv_d + p.eps);
+                for (int j = lane; j < p.ssq_in_n; j += 32) ss += __ldcg(p.ssq_in + (size_t)j * p.ssq_stride + p.row0 + r);
+                ss = warp_sum(ss);
+                if (lane == 0) inv_sh[r] = rsqrtf(ss * p.inv_d + p.eps);
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
         }
+        if (EPI == EPI_QKV_ROPE) {
+            if (et < p.rows) {
+                const int row = p.row0 + et, b = row / p.rope_M, i = row - b * p.rope_M;
+                const int n_ctx = p.len_eff[b];
+                rowmeta[et] = make_int4(n_ctx + p.depth[i], n_ctx + i, b, 0);
+            }
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
         int acc_it = 0, u = u_begin, seg_i = 0;
         Seg sg;
         bool ok = true;
@@ -364,32 +413,32 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
             const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * acc_cols;
             // partial of a split tile: slot 0 if the tile is the first one this CTA touches, else slot 1
             float *slot = p.scratch + ((size_t)blockIdx.x * 2 + (seg_i == 0 ? 0 : 1)) * slot_floats;
-            for (int c = 0; c < NT; c += 16) {
-                float g[16], uu[16];
-                if (c >= p.rows) break;                      // padding rows: nothing to keep
-                tc_ld16(t0 + c, g);
-                if (DUAL) tc_ld16(t0 + NB + c, uu);
+            for (int c = 0; c < p.rows; c += CH) {           // padding rows beyond p.rows are never read
+                float g[CH], uu[CH];
+                tc_ld8(t0 + c, g);
+                if (DUAL) tc_ld8(t0 + NB + c, uu);
                 if (p.has_lo) {                              // add the product with the lo plane
-                    float lo[16];
-                    tc_ld16(t0 + NT + c, lo);
+                    float lo[CH];
+                    tc_ld8(t0 + NT + c, lo);
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) g[j] += lo[j];
+                    for (int j = 0; j < CH; ++j) g[j] += lo[j];
                     if (DUAL) {
-                        tc_ld16(t0 + NB + NT + c, lo);
+                        tc_ld8(t0 + NB + NT + c, lo);
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) uu[j] += lo[j];
+                        for (int j = 0; j < CH; ++j) uu[j] += lo[j];
                     }
                 }
                 if (whole) {
-                    finish_chunk<DUAL>(p, sg.tile, f, c, g, uu, xch, inv_sh, lane);
+                    finish_chunk<EPI>(p, sg.tile, f, c, g, uu, xch, inv_sh, rowmeta, lane);
                 } else {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
+                    for (int j = 0; j < CH; ++j) {
                         slot[(size_t)(c + j) * TILE_F + f] = g[j];
                         if (DUAL) slot[(size_t)(NT + c + j) * TILE_F + f] = uu[j];
                     }
                 }
             }
+            if (et == 0) TRACE(2);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(buf));   // accumulator buffer may be overwritten
@@ -405,33 +454,47 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                     if (last_sh) p.counters[sg.tile] = 0;   // ready for the next launch
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (et == 0) TRACE(5);
                 if (last_sh) {
                     __threadfence();
                     const int first_cta = (sg.tile * p.k_tiles) / p.units_per_cta;
                     const int last_cta = ((sg.tile + 1) * p.k_tiles - 1) / p.units_per_cta;
-                    for (int r0 = 0; r0 < p.rows; r0 += 16) {
-                        float g[16], uu[16];
+                    for (int r0 = 0; r0 < p.rows; r0 += CH) {
+                        float g[CH], uu[CH];
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) { g[j] = 0.f; uu[j] = 0.f; }
-                        for (int c = first_cta; c <= last_cta; ++c) {
-                            const int c_first_tile = (c * p.units_per_cta) / p.k_tiles;
-                            const float *src = p.scratch + ((size_t)c * 2 + (c_first_tile == sg.tile ? 0 : 1)) * slot_floats;
+                        for (int j = 0; j < CH; ++j) { g[j] = 0.f; uu[j] = 0.f; }
+                        // contributors four at a time: all their loads are in flight before the first add, and the
+                        // sums still run in CTA order
+                        for (int c0 = first_cta; c0 <= last_cta; c0 += 4) {
+                            float pg[4][CH], pu[4][CH];
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) {
-                                if (r0 + j < p.rows) {
-                                    g[j] += __ldcg(src + (size_t)(r0 + j) * TILE_F + et);
-                                    if (DUAL) uu[j] += __ldcg(src + (size_t)(NT + r0 + j) * TILE_F + et);
+                            for (int q = 0; q < 4; ++q) {
+                                const int c = c0 + q;
+                                const bool on = c <= last_cta;
+                                const int c_first_tile = (c * p.units_per_cta) / p.k_tiles;
+                                const float *src = p.scratch + ((size_t)(on ? c : first_cta) * 2 + (c_first_tile == sg.tile ? 0 : 1)) *
+                                                   slot_floats + (size_t)r0 * TILE_F + et;
+#pragma unroll
+                                for (int j = 0; j < CH; ++j) {     // slots are NT >= rows + CH - 1 rows deep: in bounds
+                                    pg[q][j] = on ? __ldcg(src + (size_t)j * TILE_F) : 0.f;
+                                    if (DUAL) pu[q][j] = on ? __ldcg(src + (size_t)(NT + j) * TILE_F) : 0.f;
                                 }
                             }
+#pragma unroll
+                            for (int q = 0; q < 4; ++q)
+#pragma unroll
+                                for (int j = 0; j < CH; ++j) { g[j] += pg[q][j]; if (DUAL) uu[j] += pu[q][j]; }
                         }
-                        finish_chunk<DUAL>(p, sg.tile, et, r0, g, uu, xch, inv_sh, lane);
+                        if (et == 0) TRACE(6);
+                        finish_chunk<EPI>(p, sg.tile, et, r0, g, uu, xch, inv_sh, rowmeta, lane);
+                        if (et == 0) TRACE(1);
                     }
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");   // last_sh is reused by the next split tile
             }
             ++acc_it;
             ++seg_i;
-            if (et == 0) TRACE(4 + (seg_i > 2 ? 2 : seg_i - 1));
+            if (et == 0) TRACE(4);
         }
     }
 
@@ -445,6 +508,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
     tc_fence_before();
     __syncthreads();
     if (threadIdx.x == 0) TRACE(7);
+    SPAN_END(p);
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
@@ -481,6 +545,18 @@ int tc_make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t k, u
 #ifdef VIASD_TC_TRACE
 extern "C" int viasd_debug_trace(long long *host_out) {
     return (int)cudaMemcpyFromSymbol(host_out, g_tc_trace, sizeof(long long) * 160 * 8);
+}
+static int g_span_launches = 0;
+extern "C" int viasd_debug_span_reset(void) {
+    static unsigned long long init[8192 * 2];
+    for (int i = 0; i < 8192; ++i) { init[2 * i] = ~0ull; init[2 * i + 1] = 0ull; }
+    g_span_launches = 0;
+    return (int)cudaMemcpyToSymbol(g_tc_span, init, sizeof(init));
+}
+extern "C" int viasd_debug_span_read(unsigned long long *host_out, int *n_launches, int *meta) {
+    *n_launches = g_span_launches;
+    (void)meta;
+    return (int)cudaMemcpyFromSymbol(host_out, g_tc_span, sizeof(unsigned long long) * 8192 * 2);
 }
 #endif
 
@@ -543,6 +619,8 @@ int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {
     if (stages > MAX_STAGES) stages = MAX_STAGES;
 #ifdef VIASD_TC_TRACE
     if (getenv("VIASD_TC_DBG")) p.dbg = atoi(getenv("VIASD_TC_DBG"));
+    p.launch_idx = g_span_launches++;
+    p.trace_on = getenv("VIASD_TC_TRACE_IDX") ? (atoi(getenv("VIASD_TC_TRACE_IDX")) == p.launch_idx) : 1;
     if (getenv("VIASD_TC_STAGES")) { int v = atoi(getenv("VIASD_TC_STAGES")); if (v >= 2 && v < stages) stages = v; }
 #endif
     if (stages < 2) return VIASD_EINVAL;
@@ -553,18 +631,26 @@ int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {
     int cols = p.acc_bufs * acc_cols;
     p.tmem_cols = cols <= 32 ? 32 : cols <= 64 ? 64 : cols <= 128 ? 128 : cols <= 256 ? 256 : 512;
     const size_t smem = stage * stages + 1024;
-    static bool attr_done[2] = {false, false};
-    if (!attr_done[dual]) {
-        if (dual) CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 208 * 1024));
-        else CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 208 * 1024));
-        attr_done[dual] = true;
-    }
     const CUtensorMap &w0 = *L.map_w[0], &w1 = *L.map_w[L.n_seg > 1 ? 1 : 0], &w2 = *L.map_w[L.n_seg > 2 ? 2 : 0];
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
     pdl_config(cfg, attr, dim3(grid), dim3(THREADS), smem, st);
-    if (dual) CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<true>, w0, w1, w2, *L.map_x, p));
-    else CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<false>, w0, w1, w2, *L.map_x, p));
+    static bool attr_done[4] = {false, false, false, false};
+#define TC_LAUNCH(IDX, KIND)                                                                                          \
+    do {                                                                                                              \
+        if (!attr_done[IDX]) {                                                                                        \
+            CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, 208 * 1024)); \
+            attr_done[IDX] = true;                                                                                    \
+        }                                                                                                             \
+        CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<KIND>, w0, w1, w2, *L.map_x, p));                            \
+    } while (0)
+    switch (L.epi) {
+    case EPI_SWIGLU: TC_LAUNCH(0, EPI_SWIGLU); break;
+    case EPI_ADD_NORM: TC_LAUNCH(1, EPI_ADD_NORM); break;
+    case EPI_QKV_ROPE: TC_LAUNCH(2, EPI_QKV_ROPE); break;
+    default: TC_LAUNCH(3, EPI_STORE); break;          // EPI_STORE and EPI_ADD share one kernel
+    }
+#undef TC_LAUNCH
     LAUNCH_CHECK();
     return VIASD_OK;
 }
