@@ -27,7 +27,7 @@ constexpr int MAX_SMS = 160;            // workspace is sized without asking the
 constexpr int MAX_GEMM_CTAS = 2 * MAX_SMS;
 
 size_t part_bytes_for(const viasd_config &c) {
-    const size_t R = (size_t)c.max_batch * c.max_query;
+    const size_t R = (size_t)2 * c.max_batch * c.max_query;
     // attention split-KV partials: up to 16 key ranges of (head_dim + 2) floats per (row, head)
     size_t att = R * c.n_heads * 16 * (size_t)(c.head_dim + 2) * sizeof(float);
     const size_t cap = (size_t)256 << 20;
@@ -37,7 +37,7 @@ size_t part_bytes_for(const viasd_config &c) {
 // One layout routine serves both the size query (base = null) and the real carve.
 size_t carve(const viasd_config &c, char *base, Workspace *ws) {
     Carver cv{base, 0};
-    const size_t R = (size_t)c.max_batch * c.max_query, es = elem_size(c.dtype);
+    const size_t R = (size_t)2 * c.max_batch * c.max_query, es = elem_size(c.dtype);   // two row streams
     const size_t qd = (size_t)c.n_heads * c.head_dim, kvd = (size_t)c.n_kv_heads * c.head_dim;
     Workspace w;
     w.rope_cos = cv.take<float>((size_t)c.max_ctx * (c.head_dim / 2) * 4);
@@ -152,20 +152,30 @@ int run_gemm(viasd_model *m, const GemmCall &g, int rows, cudaStream_t st) {
 
 // Tensor-core path with fused epilogues: per layer QKV (+RMS scale, rotary, KV append) -> attention ->
 // O (+residual, next-norm preparation) -> gate/up (+RMS scale, SwiGLU) -> down (+residual, next-norm preparation).
-int forward_fused(viasd_model *m, const viasd_cache *cache, const viasd_draft *d, bool slim, float *logits, cudaStream_t st) {
+// mode 0: full verifier q; mode 1: slim verifier q' (routed layers only); mode 2: both in one sweep over the
+// layers.  In mode 2 the block rows exist twice, [full stream; slim stream]: a routed layer's weights are streamed
+// once and applied to both streams, an unrouted layer runs on the full stream only.  Results are those of the two
+// separate passes; only the weight traffic of the routed layers is shared.
+int forward_sweep(viasd_model *m, const viasd_cache *cache, const viasd_draft *d, int mode, float *logits_full,
+                  float *logits_slim, cudaStream_t st) {
     const viasd_config &c = m->cfg;
     const int B = d->batch, M = d->n_nodes + 1, rows = B * M;
     const int qd = c.n_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
-    void *kc = slim ? cache->k_slim : cache->k_full, *vc = slim ? cache->v_slim : cache->v_full;
-    const int n_run = slim ? m->n_routed : c.n_layers;
     const size_t R = m->ws.rows_alloc;
+    const bool dual = mode == 2;
     int rc;
-    auto layer_id = [&](int ord) { return slim ? m->routed[ord] : ord; };
-    // common part of a launch description; rows beyond 128 go in chunks
-    auto gemm = [&](int cls, TcLaunch L, const ActMaps &xm) -> int {
-        return timed(m, cls, st, [&]() -> int {
-            for (int row0 = 0; row0 < rows; row0 += 128) {
-                const int nr = rows - row0 < 128 ? rows - row0 : 128, nt = tc_pick_nt(nr);
+    // layers this sweep visits, and for each whether the slim stream takes part
+    const int n_run = mode == 1 ? m->n_routed : c.n_layers;
+    auto layer_id = [&](int it) { return mode == 1 ? m->routed[it] : it; };
+    auto routed_ord = [&](int l) { for (int o = 0; o < m->n_routed; ++o) if (m->routed[o] == l) return o; return -1; };
+    auto next_slim_gain = [&](int l) -> const float * {       // gain of the slim stream's next norm1 after layer l
+        for (int o = 0; o < m->n_routed; ++o) if (m->routed[o] > l) return m->norm1[m->routed[o]];
+        return m->final_norm;
+    };
+    auto gemm = [&](TcLaunch L, const ActMaps &xm, int nrows) -> int {
+        return timed(m, VIASD_T_GEMM, st, [&]() -> int {
+            for (int row0 = 0; row0 < nrows; row0 += 128) {
+                const int nr = nrows - row0 < 128 ? nrows - row0 : 128, nt = tc_pick_nt(nr);
                 const int ni = nt == 16 ? 0 : nt == 32 ? 1 : nt == 64 ? 2 : 3;
                 L.map_x = &xm.map[ni]; L.x_box_rows = xm.box_rows[ni];
                 L.has_lo = 1; L.lo_row_offset = (int)R;
@@ -173,6 +183,7 @@ int forward_fused(viasd_model *m, const viasd_cache *cache, const viasd_draft *d
                 L.scratch = m->ws.gemm_scratch; L.counters = m->ws.gemm_counters; L.status = &m->ws.stats->device_status;
                 L.sm_count = m->sm_count;
                 L.ssq_stride = (int)R; L.inv_d = 1.0f / (float)c.d_model; L.eps = c.rms_eps;
+                L.split_row = dual ? rows : 0;
                 int r2 = launch_gemm_tc(L, st);
                 if (r2) return r2;
             }
@@ -183,10 +194,21 @@ int forward_fused(viasd_model *m, const viasd_cache *cache, const viasd_draft *d
     const int ssq_n = (c.d_model / 128) * 4;
 
     if ((rc = timed(m, VIASD_T_EMBED, st, [&] { return launch_prep(m, cache, d, st); }))) return rc;
-    if ((rc = timed(m, VIASD_T_EMBED, st, [&] { return launch_embed_norm(m, m->norm1[layer_id(0)], rows, st); }))) return rc;
-    for (int ord = 0; ord < n_run; ++ord) {
-        const int l = layer_id(ord);
+    if (dual) {
+        if ((rc = timed(m, VIASD_T_EMBED, st, [&] { return launch_embed_norm2(m, m->norm1[0], m->norm1[m->routed[0]], rows, st); })))
+            return rc;
+    } else {
+        if ((rc = timed(m, VIASD_T_EMBED, st, [&] { return launch_embed_norm(m, m->norm1[layer_id(0)], rows, st); }))) return rc;
+    }
+    for (int it = 0; it < n_run; ++it) {
+        const int l = layer_id(it);
+        const int so = routed_ord(l);                          // slim ordinal of this layer, -1 if unrouted
+        const bool both = dual && so >= 0;
+        const int nrows = both ? 2 * rows : rows;
         const LayerMaps &lm = m->lmaps[l];
+        // cache and layer ordinal of the first stream
+        void *kc = mode == 1 ? cache->k_slim : cache->k_full, *vc = mode == 1 ? cache->v_slim : cache->v_full;
+        const int ord = mode == 1 ? it : l;
         {   // QKV: scale by 1/rms, rotate q and k, append k and v to the cache
             TcLaunch L; memset(&L, 0, sizeof(L));
             wseg(L, 0, lm.wq, qd); wseg(L, 1, lm.wk, kvd); wseg(L, 2, lm.wv, kvd); L.n_seg = 3;
@@ -195,37 +217,46 @@ int forward_fused(viasd_model *m, const viasd_cache *cache, const viasd_draft *d
             L.q_out = m->ws.q; L.kc = kc; L.vc = vc; L.cosv = m->ws.rope_cos; L.sinv = m->ws.rope_sin;
             L.len_eff = m->ws.len_eff; L.depth = m->ws.tree->depth; L.rope_M = M; L.rope_H = c.n_heads; L.rope_Hkv = c.n_kv_heads;
             L.max_batch = c.max_batch; L.max_ctx = c.max_ctx; L.layer_ord = ord;
-            if ((rc = gemm(VIASD_T_GEMM, L, m->maps_a))) return rc;
+            L.kc2 = cache->k_slim; L.vc2 = cache->v_slim; L.layer_ord2 = so;
+            if ((rc = gemm(L, m->maps_a, nrows))) return rc;
         }
-        if ((rc = timed(m, VIASD_T_ATTENTION, st, [&] { return launch_attention(m, kc, vc, slim, ord, B, M, st); }))) return rc;
+        if (both) {
+            if ((rc = timed(m, VIASD_T_ATTENTION, st, [&] { return launch_attention_dual(m, cache->k_full, cache->v_full, l,
+                    cache->k_slim, cache->v_slim, so, B, M, st); }))) return rc;
+        } else {
+            if ((rc = timed(m, VIASD_T_ATTENTION, st, [&] { return launch_attention(m, kc, vc, mode == 1, ord, B, M, st); })))
+                return rc;
+        }
         {   // O projection into the residual; prepare the input of the post-attention norm
             TcLaunch L; memset(&L, 0, sizeof(L));
             wseg(L, 0, lm.wo, c.d_model); L.n_seg = 1;
             L.k = qd; L.epi = EPI_ADD_NORM; L.out_f32 = m->ws.h; L.ld_out = c.d_model;
             L.next_gain = m->norm2[l]; L.next_act = m->ws.a; L.next_plane = R * c.d_model; L.ssq_out = m->ws.ssq;
-            if ((rc = gemm(VIASD_T_GEMM, L, m->maps_attn))) return rc;
+            if ((rc = gemm(L, m->maps_attn, nrows))) return rc;
         }
         {   // gate / up with SwiGLU
             TcLaunch L; memset(&L, 0, sizeof(L));
             wseg(L, 0, lm.wg, c.d_ff); wseg(L, 1, lm.wu, c.d_ff); L.n_seg = 2;
             L.k = c.d_model; L.epi = EPI_SWIGLU; L.out_act = m->ws.act; L.act_plane = R * c.d_ff; L.ld_out = c.d_ff;
             L.ssq_in = m->ws.ssq; L.ssq_in_n = ssq_n;
-            if ((rc = gemm(VIASD_T_GEMM, L, m->maps_a))) return rc;
+            if ((rc = gemm(L, m->maps_a, nrows))) return rc;
         }
-        {   // down projection into the residual; prepare the input of the next norm (next layer's or the final one)
+        {   // down projection into the residual; prepare the input of each stream's next norm
             TcLaunch L; memset(&L, 0, sizeof(L));
             wseg(L, 0, lm.wd, c.d_model); L.n_seg = 1;
             L.k = c.d_ff; L.epi = EPI_ADD_NORM; L.out_f32 = m->ws.h; L.ld_out = c.d_model;
-            L.next_gain = ord + 1 < n_run ? m->norm1[layer_id(ord + 1)] : m->final_norm;
+            L.next_gain = it + 1 < n_run ? m->norm1[layer_id(it + 1)] : m->final_norm;
+            L.next_gain2 = both ? next_slim_gain(l) : nullptr;
             L.next_act = m->ws.a; L.next_plane = R * c.d_model; L.ssq_out = m->ws.ssq;
-            if ((rc = gemm(VIASD_T_GEMM, L, m->maps_act))) return rc;
+            if ((rc = gemm(L, m->maps_act, nrows))) return rc;
         }
     }
     TcLaunch L; memset(&L, 0, sizeof(L));
     wseg(L, 0, m->head_map, c.vocab); L.n_seg = 1;
-    L.k = c.d_model; L.epi = EPI_STORE; L.out_f32 = logits; L.ld_out = c.vocab;
+    L.k = c.d_model; L.epi = EPI_STORE; L.out_f32 = mode == 1 ? logits_slim : logits_full; L.out_f32_2 = logits_slim;
+    L.ld_out = c.vocab;
     L.ssq_in = m->ws.ssq; L.ssq_in_n = ssq_n;
-    return gemm(VIASD_T_GEMM, L, m->maps_a);
+    return gemm(L, m->maps_a, dual ? 2 * rows : rows);
 }
 
 // One pass of the sub-network made of `layers` (all of them for q, the routed ones for q').
@@ -234,7 +265,7 @@ int forward(viasd_model *m, const viasd_cache *cache, const viasd_draft *d, bool
     int rc;
     if ((rc = check_draft(m, d)) || (rc = check_cache(cache))) return rc;
     if (!logits) return VIASD_EINVAL;
-    if (m->fused) return forward_fused(m, cache, d, slim, logits, st);
+    if (m->fused) return forward_sweep(m, cache, d, slim ? 1 : 0, slim ? nullptr : logits, slim ? logits : nullptr, st);
     const viasd_config &c = m->cfg;
     const int B = d->batch, M = d->n_nodes + 1, rows = B * M;
     const int qd = c.n_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
@@ -447,6 +478,13 @@ int viasd_verify_step(viasd_model *m, viasd_cache *cache, const viasd_draft *dra
     int rc;
     if (!slim_logits || !full_logits) return VIASD_EINVAL;
     if ((rc = check_params(params))) return rc;
+    if (m && m->fused) {
+        // both verifiers in one sweep over the layers (routed layers' weights are read once for both)
+        if ((rc = check_draft(m, draft)) || (rc = check_cache(cache))) return rc;
+        if ((rc = forward_sweep(m, cache, draft, 2, full_logits, slim_logits, (cudaStream_t)stream))) return rc;
+        if ((rc = viasd_tier_accept(m, draft, params, slim_logits, full_logits, 3, result, stream))) return rc;
+        return viasd_kv_commit(m, cache, draft, result, stream);
+    }
     if (params->conf_source == 0) {
         if ((rc = viasd_tier_accept(m, draft, params, nullptr, nullptr, 1, result, stream))) return rc;
         if ((rc = viasd_slim_forward(m, cache, draft, slim_logits, stream))) return rc;

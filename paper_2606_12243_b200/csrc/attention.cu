@@ -175,7 +175,7 @@ int launch_attention(viasd_model *m, const void *kc, const void *vc, bool slim, 
         if (nsplit > 16) nsplit = 16;
         size_t per_split = (size_t)batch * c.n_heads * M * (c.head_dim + 2) * sizeof(float);
         while (nsplit > 1 && per_split * nsplit > m->ws.part_bytes) --nsplit;
-        int rc = launch_attention_mma(m, kc, vc, slim, layer_ord, batch, M, nsplit, st);
+        int rc = launch_attention_mma(m, kc, vc, slim, layer_ord, nullptr, nullptr, 0, 1, batch, M, nsplit, st);
         if (rc || nsplit == 1) return rc;
         attention_combine_kernel<__nv_bfloat16, 128><<<dim3(batch * M, c.n_heads), 128, 0, st>>>(
             (__nv_bfloat16 *)m->ws.attn, m->ws.rows_alloc * (size_t)c.n_heads * 128, m->ws.part, M, c.n_heads, nsplit);
@@ -191,4 +191,24 @@ int launch_attention(viasd_model *m, const void *kc, const void *vc, bool slim, 
         if (c.head_dim == 128) return run<__nv_bfloat16, 128>(m, kc, vc, layer_ord, batch, M, nsplit, st);
     }
     return VIASD_EINVAL;
+}
+
+// Both verifiers in one launch: the full stream's rows against the full cache, the slim stream's rows against the
+// slim cache (tensor-core kernel only).
+int launch_attention_dual(viasd_model *m, const void *kf, const void *vf, int layer_full, const void *ks, const void *vs,
+                          int ord_slim, int batch, int M, cudaStream_t st) {
+    const viasd_config &c = m->cfg;
+    const int ctas = batch * c.n_kv_heads;                  // same key ranges as the one-stream launch: same bits
+    int nsplit = (m->sm_count + ctas - 1) / ctas;
+    const int max_tiles = (c.max_ctx + 127) / 128;
+    if (nsplit > max_tiles) nsplit = max_tiles;
+    if (nsplit > 16) nsplit = 16;
+    size_t per_split = (size_t)2 * batch * c.n_heads * M * (c.head_dim + 2) * sizeof(float);
+    while (nsplit > 1 && per_split * nsplit > m->ws.part_bytes) --nsplit;
+    int rc = launch_attention_mma(m, kf, vf, false, layer_full, ks, vs, ord_slim, 2, batch, M, nsplit, st);
+    if (rc || nsplit == 1) return rc;
+    attention_combine_kernel<__nv_bfloat16, 128><<<dim3(2 * batch * M, c.n_heads), 128, 0, st>>>(
+        (__nv_bfloat16 *)m->ws.attn, m->ws.rows_alloc * (size_t)c.n_heads * 128, m->ws.part, M, c.n_heads, nsplit);
+    LAUNCH_CHECK();
+    return VIASD_OK;
 }

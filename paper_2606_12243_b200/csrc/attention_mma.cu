@@ -90,6 +90,7 @@ struct AttnArgs {
     const TreeInfo *tree;
     int *status;
     int M, H, Hkv, max_batch, max_ctx, layer_ord, nsplit, mt;   // mt = query tiles of 16 rows
+    int batch, layer_ord2;      // second row stream (blockIdx.z = 1): rows batch*M.., its own cache and layer ordinal
     float scale;
 };
 
@@ -188,13 +189,16 @@ __device__ __forceinline__ void tile_step(uint32_t qhi, uint32_t qlo, int mrow0,
 // KEYSPLIT: warps split the keys of a stage (query tiles <= 2); else warps split the query tiles (<= 8)
 template <bool KEYSPLIT>
 __global__ void __launch_bounds__(WARPS * 32)
-attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const AttnArgs a) {
+attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                     const __grid_constant__ CUtensorMap map_k2, const __grid_constant__ CUtensorMap map_v2, const AttnArgs a) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) unsigned long long bars[NSTAGE];
     constexpr int MTW = 2;                                   // query tiles per warp at most
     PDL_TRIGGER();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int b = blockIdx.x / a.Hkv, g = blockIdx.x % a.Hkv, split = blockIdx.y;
+    const int b = blockIdx.x / a.Hkv, g = blockIdx.x % a.Hkv, split = blockIdx.y, stream = blockIdx.z;
+    const int be = stream * a.batch + b;                     // row block of this (stream, sequence)
+    const CUtensorMap *mk = stream ? &map_k2 : &map_k, *mv = stream ? &map_v2 : &map_v;
     const int grp = a.H / a.Hkv, QR = grp * a.M, QRP = a.mt * 16;
     const int n_ctx = a.len_eff[b], Tk = n_ctx + a.M;
     int chunk = (Tk + a.nsplit - 1) / a.nsplit;
@@ -212,16 +216,16 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     // first rows of this (layer, sequence, kv head) in the cache viewed as a 2-D tensor [rows, HD]
-    const int row_base = ((a.layer_ord * a.max_batch + b) * a.Hkv + g) * a.max_ctx;
+    const int row_base = (((stream ? a.layer_ord2 : a.layer_ord) * a.max_batch + b) * a.Hkv + g) * a.max_ctx;
     auto issue = [&](int tile) {
         const int st = tile % NSTAGE;
         const uint32_t bar = smem_u32(&bars[st]), dst = base + st * STAGE_BYTES;
         const int y = row_base + k_begin + tile * TKEYS;
         mbar_expect_tx(bar, STAGE_BYTES);
-        tma_load_2d(dst, &map_k, bar, 0, y);
-        tma_load_2d(dst + HALF_BYTES, &map_k, bar, 64, y);
-        tma_load_2d(dst + 2 * HALF_BYTES, &map_v, bar, 0, y);
-        tma_load_2d(dst + 3 * HALF_BYTES, &map_v, bar, 64, y);
+        tma_load_2d(dst, mk, bar, 0, y);
+        tma_load_2d(dst + HALF_BYTES, mk, bar, 64, y);
+        tma_load_2d(dst + 2 * HALF_BYTES, mv, bar, 0, y);
+        tma_load_2d(dst + 3 * HALF_BYTES, mv, bar, 64, y);
     };
     __syncthreads();
     if (threadIdx.x == 0) for (int t = 0; t < NSTAGE && t < n_tiles; ++t) issue(t);
@@ -232,7 +236,7 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
         float x0 = 0.f, x1 = 0.f;
         if (row < QR) {
             const int h = g * grp + row / a.M, i = row % a.M;
-            const float2 v = *reinterpret_cast<const float2 *>(a.q + ((size_t)(b * a.M + i) * a.H + h) * HD + d2);
+            const float2 v = *reinterpret_cast<const float2 *>(a.q + ((size_t)(be * a.M + i) * a.H + h) * HD + d2);
             x0 = v.x * a.scale; x1 = v.y * a.scale;
         }
         uint32_t hi, lo;
@@ -330,9 +334,9 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             const float inv = 1.f / l;
 #pragma unroll
             for (int e = 0; e < HD / 32; ++e)
-                store_act<__nv_bfloat16>(a.out, a.out_plane, ((size_t)(b * a.M + i) * a.H + h) * HD + lane + 32 * e, acc[e] * inv);
+                store_act<__nv_bfloat16>(a.out, a.out_plane, ((size_t)(be * a.M + i) * a.H + h) * HD + lane + 32 * e, acc[e] * inv);
         } else {
-            float *dst = a.part + ((((size_t)b * a.H + h) * a.M + i) * a.nsplit + split) * (HD + 2);
+            float *dst = a.part + ((((size_t)be * a.H + h) * a.M + i) * a.nsplit + split) * (HD + 2);
 #pragma unroll
             for (int e = 0; e < HD / 32; ++e) dst[lane + 32 * e] = acc[e];
             if (lane == 0) { dst[HD] = mmax; dst[HD + 1] = l; }
@@ -348,16 +352,29 @@ int attention_mma_supported(const viasd_model *m, int M) {
     return c.dtype == 1 && c.head_dim == HD && (c.n_heads / c.n_kv_heads) * M <= 128 && m->use_tc;
 }
 
-int launch_attention_mma(viasd_model *m, const void *kc, const void *vc, bool slim, int layer_ord, int batch, int M,
-                         int nsplit, cudaStream_t st) {
+static int cache_maps(viasd_model *m, CacheMaps &cm, const void *kc, const void *vc, int n_layers) {
+    if (cm.k_ptr == kc && cm.v_ptr == vc) return VIASD_OK;
+    const viasd_config &c = m->cfg;
+    const uint64_t rows = (uint64_t)n_layers * c.max_batch * c.n_kv_heads * c.max_ctx;
+    int rc;
+    if ((rc = tc_make_map(&cm.k, kc, rows, HD, TKEYS))) return rc;
+    if ((rc = tc_make_map(&cm.v, vc, rows, HD, TKEYS))) return rc;
+    cm.k_ptr = kc; cm.v_ptr = vc;
+    return VIASD_OK;
+}
+
+// streams = 1: one cache (full or slim).  streams = 2: rows [0, batch*M) against the full cache at layer_ord and
+// rows [batch*M, 2*batch*M) against the slim cache at layer_ord2, in one launch.
+int launch_attention_mma(viasd_model *m, const void *kc, const void *vc, bool slim, int layer_ord, const void *kc2,
+                         const void *vc2, int layer_ord2, int streams, int batch, int M, int nsplit, cudaStream_t st) {
     const viasd_config &c = m->cfg;
     CacheMaps &cm = slim ? m->cmaps_slim : m->cmaps_full;
-    if (cm.k_ptr != kc || cm.v_ptr != vc) {
-        const uint64_t rows = (uint64_t)(slim ? m->n_routed : c.n_layers) * c.max_batch * c.n_kv_heads * c.max_ctx;
-        int rc;
-        if ((rc = tc_make_map(&cm.k, kc, rows, HD, TKEYS))) return rc;
-        if ((rc = tc_make_map(&cm.v, vc, rows, HD, TKEYS))) return rc;
-        cm.k_ptr = kc; cm.v_ptr = vc;
+    int rc;
+    if ((rc = cache_maps(m, cm, kc, vc, slim ? m->n_routed : c.n_layers))) return rc;
+    CacheMaps *cm2 = &cm;
+    if (streams == 2) {
+        cm2 = &m->cmaps_slim;
+        if ((rc = cache_maps(m, *cm2, kc2, vc2, m->n_routed))) return rc;
     }
     const int grp = c.n_heads / c.n_kv_heads, mt = (grp * M + 15) / 16;
     AttnArgs a;
@@ -366,6 +383,7 @@ int launch_attention_mma(viasd_model *m, const void *kc, const void *vc, bool sl
     a.len_eff = m->ws.len_eff; a.tree = m->ws.tree; a.status = &m->ws.stats->device_status;
     a.M = M; a.H = c.n_heads; a.Hkv = c.n_kv_heads; a.max_batch = c.max_batch; a.max_ctx = c.max_ctx;
     a.layer_ord = layer_ord; a.nsplit = nsplit; a.mt = mt; a.scale = 1.0f / sqrtf((float)HD);
+    a.batch = batch; a.layer_ord2 = layer_ord2;
     const size_t q_bytes = (size_t)mt * 16 * 256 * 2;
     const size_t smem = 1024 + NSTAGE * STAGE_BYTES + q_bytes;
     static bool attr_done = false;
@@ -374,9 +392,9 @@ int launch_attention_mma(viasd_model *m, const void *kc, const void *vc, bool sl
         CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
         attr_done = true;
     }
-    dim3 grid(batch * c.n_kv_heads, nsplit);
-    if (mt <= 2) attention_mma_kernel<true><<<grid, WARPS * 32, smem, st>>>(cm.k, cm.v, a);
-    else attention_mma_kernel<false><<<grid, WARPS * 32, smem, st>>>(cm.k, cm.v, a);
+    dim3 grid(batch * c.n_kv_heads, nsplit, streams);
+    if (mt <= 2) attention_mma_kernel<true><<<grid, WARPS * 32, smem, st>>>(cm.k, cm.v, cm2->k, cm2->v, a);
+    else attention_mma_kernel<false><<<grid, WARPS * 32, smem, st>>>(cm.k, cm.v, cm2->k, cm2->v, a);
     LAUNCH_CHECK();
     return VIASD_OK;
 }

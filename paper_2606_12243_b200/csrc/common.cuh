@@ -140,8 +140,11 @@ int launch_attention(viasd_model *m, const void *kc, const void *vc, bool slim, 
                      cudaStream_t st);
 // attention_mma.cu
 int attention_mma_supported(const viasd_model *m, int M);
-int launch_attention_mma(viasd_model *m, const void *kc, const void *vc, bool slim, int layer_ord, int batch, int M,
-                         int nsplit, cudaStream_t st);
+int launch_attention_mma(viasd_model *m, const void *kc, const void *vc, bool slim, int layer_ord, const void *kc2,
+                         const void *vc2, int layer_ord2, int streams, int batch, int M, int nsplit, cudaStream_t st);
+int launch_attention_dual(viasd_model *m, const void *kf, const void *vf, int layer_full, const void *ks, const void *vs,
+                          int ord_slim, int batch, int M, cudaStream_t st);
+int launch_embed_norm2(const viasd_model *m, const float *gain_full, const float *gain_slim, int rows, cudaStream_t st);
 
 // tier_accept.cu
 int launch_tier(const viasd_model *m, const viasd_draft *d, const viasd_params *p, const float *slim_logits,

@@ -168,18 +168,20 @@ __device__ __forceinline__ void finish_chunk(const TcParams &p, int tile, int f,
     const int n = nbase + nin;
     if (EPI == EPI_STORE) {
         if (!valid) return;
-        float *dst = p.out_f32 + (size_t)(p.row0 + r0) * p.ld_out + n;
-        if (p.epi == EPI_ADD) {
 #pragma unroll
-            for (int j = 0; j < CH; ++j) if (j < nrow) dst[(size_t)j * p.ld_out] += g[j];
-        } else {
-#pragma unroll
-            for (int j = 0; j < CH; ++j) if (j < nrow) dst[(size_t)j * p.ld_out] = g[j];
+        for (int j = 0; j < CH; ++j) {
+            if (j < nrow) {
+                const int row = p.row0 + r0 + j;          // the second stream's rows go to the second output
+                float *dst = row < p.split_row ? p.out_f32 + (size_t)row * p.ld_out + n
+                                               : p.out_f32_2 + (size_t)(row - p.split_row) * p.ld_out + n;
+                if (p.epi == EPI_ADD) *dst += g[j]; else *dst = g[j];
+            }
         }
     } else if (EPI == EPI_ADD_NORM) {
         // residual update, plus what the next RMSNorm needs: h * gain as hi/lo planes and partial sums of h^2.
         // Loads first, then arithmetic, then stores: the CH rows cost one memory round trip.
-        const float gain = valid ? p.next_gain[n] : 0.f;
+        const float gain_a = valid ? p.next_gain[n] : 0.f;
+        const float gain_b = (valid && p.next_gain2) ? p.next_gain2[n] : gain_a;
         float *hp = p.out_f32 + (size_t)(p.row0 + r0) * p.ld_out + n;
         __nv_bfloat16 *ap = p.next_act + (size_t)(p.row0 + r0) * p.ld_out + n;
         float v[CH];
@@ -189,7 +191,8 @@ __device__ __forceinline__ void finish_chunk(const TcParams &p, int tile, int f,
         for (int j = 0; j < CH; ++j) {
             if (valid && j < nrow) {
                 hp[(size_t)j * p.ld_out] = v[j];
-                store_act<__nv_bfloat16>(ap, p.next_plane, (size_t)j * p.ld_out, v[j] * gain);
+                store_act<__nv_bfloat16>(ap, p.next_plane, (size_t)j * p.ld_out,
+                                         v[j] * (p.row0 + r0 + j < p.split_row ? gain_a : gain_b));
             }
             v[j] *= v[j];
         }
@@ -227,12 +230,13 @@ __device__ __forceinline__ void finish_chunk(const TcParams &p, int tile, int f,
 #pragma unroll
             for (int j = 0; j < CH; ++j) if (j < nrow) dst[(size_t)j * p.rope_H * TILE_F] = g[j];
         } else {
-            __nv_bfloat16 *cache = s == 1 ? p.kc : p.vc;
 #pragma unroll
             for (int j = 0; j < CH; ++j) {
                 if (j < nrow) {
                     const int4 rm = rowmeta[r0 + j];
-                    cache[((((size_t)p.layer_ord * p.max_batch + rm.z) * p.rope_Hkv + head) * p.max_ctx + rm.y) * TILE_F + f] =
+                    __nv_bfloat16 *cache = rm.w ? (s == 1 ? p.kc2 : p.vc2) : (s == 1 ? p.kc : p.vc);
+                    const int lo = rm.w ? p.layer_ord2 : p.layer_ord;
+                    cache[((((size_t)lo * p.max_batch + rm.z) * p.rope_Hkv + head) * p.max_ctx + rm.y) * TILE_F + f] =
                         __float2bfloat16_rn(g[j]);
                 }
             }
@@ -396,9 +400,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
         }
         if (EPI == EPI_QKV_ROPE) {
             if (et < p.rows) {
-                const int row = p.row0 + et, b = row / p.rope_M, i = row - b * p.rope_M;
+                // rows are laid out [stream][sequence][block row]; stream 1 (rows >= split_row) is the slim verifier
+                const int row = p.row0 + et, stream = row >= p.split_row ? 1 : 0, rs = row - stream * p.split_row;
+                const int b = rs / p.rope_M, i = rs - b * p.rope_M;
                 const int n_ctx = p.len_eff[b];
-                rowmeta[et] = make_int4(n_ctx + p.depth[i], n_ctx + i, b, 0);
+                rowmeta[et] = make_int4(n_ctx + p.depth[i], n_ctx + i, b, stream);
             }
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -601,6 +607,9 @@ int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {
     p.q_out = L.q_out; p.kc = (__nv_bfloat16 *)L.kc; p.vc = (__nv_bfloat16 *)L.vc; p.cosv = L.cosv; p.sinv = L.sinv;
     p.len_eff = L.len_eff; p.depth = L.depth; p.rope_M = L.rope_M; p.rope_H = L.rope_H; p.rope_Hkv = L.rope_Hkv;
     p.max_batch = L.max_batch; p.max_ctx = L.max_ctx; p.layer_ord = L.layer_ord;
+    p.split_row = L.split_row > 0 ? L.split_row : 0x7fffffff;
+    p.out_f32_2 = L.out_f32_2; p.next_gain2 = L.next_gain2; p.kc2 = (__nv_bfloat16 *)L.kc2; p.vc2 = (__nv_bfloat16 *)L.vc2;
+    p.layer_ord2 = L.layer_ord2;
     const int units = p.n_tiles * p.k_tiles;
     if (units <= 0) return VIASD_OK;
     int ctas_per_sm = 1;

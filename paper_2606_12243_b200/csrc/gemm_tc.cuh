@@ -29,6 +29,8 @@ struct TcParams {                       // kernel argument block
     // EPI_QKV_ROPE
     float *q_out; __nv_bfloat16 *kc, *vc; const float *cosv, *sinv; const int *len_eff, *depth;
     int rope_M, rope_H, rope_Hkv, max_batch, max_ctx, layer_ord;
+    // two row streams in one launch (full verifier rows first, slim verifier rows from split_row on)
+    int split_row, layer_ord2; float *out_f32_2; const float *next_gain2; __nv_bfloat16 *kc2, *vc2;
 };
 
 struct TcLaunch {                       // host-side description of one GEMM
@@ -55,6 +57,7 @@ struct TcLaunch {                       // host-side description of one GEMM
     // EPI_QKV_ROPE
     float *q_out; void *kc, *vc; const float *cosv, *sinv; const int *len_eff, *depth;
     int rope_M, rope_H, rope_Hkv, max_batch, max_ctx, layer_ord;
+    int split_row, layer_ord2; float *out_f32_2; const float *next_gain2; void *kc2, *vc2;
 };
 
 // 2-D bf16 tensor [rows, k] row-major -> TMA map with a (64 x box_rows) box and the 128-byte swizzle

@@ -112,6 +112,35 @@ int launch_embed_norm(const viasd_model *m, const float *gain, int rows, cudaStr
     return VIASD_OK;
 }
 
+// Two row streams from the same block rows: rows [0, rows) prepared for the full verifier's first layer,
+// rows [rows, 2*rows) for the slim verifier's first routed layer (their first norms differ).
+__global__ void __launch_bounds__(256)
+embed_norm2_kernel(float *h, __nv_bfloat16 *a, size_t plane, float *ssq, int ssq_stride, const __nv_bfloat16 *E,
+                   const float *gain_full, const float *gain_slim, const int *row_tok, int d, int rows) {
+    const int r = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    PDL_TRIGGER();
+    const float *gain = r < rows ? gain_full : gain_slim;
+    const __nv_bfloat16 *src = E + (size_t)row_tok[r < rows ? r : r - rows] * d;
+    for (int base = 0; base < d; base += 256) {
+        const int i = base + warp * 32 + lane;
+        if (base + warp * 32 < d) {
+            const float v = __bfloat162float(src[i]);
+            h[(size_t)r * d + i] = v;
+            store_act<__nv_bfloat16>(a, plane, (size_t)r * d + i, v * gain[i]);
+            const float sq = warp_sum(v * v);
+            if (lane == 0) ssq[(size_t)(i >> 5) * ssq_stride + r] = sq;
+        }
+    }
+}
+
+int launch_embed_norm2(const viasd_model *m, const float *gain_full, const float *gain_slim, int rows, cudaStream_t st) {
+    embed_norm2_kernel<<<2 * rows, 256, 0, st>>>(m->ws.h, (__nv_bfloat16 *)m->ws.a, m->ws.rows_alloc * m->cfg.d_model,
+                                                 m->ws.ssq, (int)m->ws.rows_alloc, (const __nv_bfloat16 *)m->embed, gain_full,
+                                                 gain_slim, m->ws.row_tok, m->cfg.d_model, rows);
+    LAUNCH_CHECK();
+    return VIASD_OK;
+}
+
 int launch_embed(const viasd_model *m, int rows, cudaStream_t st) {
     if (m->cfg.dtype == 0)
         embed_kernel<float><<<rows, 256, 0, st>>>(m->ws.h, (const float *)m->embed, m->ws.row_tok, m->cfg.d_model);
