@@ -288,24 +288,31 @@ def run_ours(args, wl) -> None:
 
     peak, peak_kind = measured_peaks()
     sb = RL.step_bytes(wl)
+    # verify_step streams every layer's weights once and applies the routed layers to both row streams, so the
+    # bytes its GEMM launches move are the "shared" figure; the two-separate-passes figure is reported beside it
     gemm_ms = timing["gemm"]["ms"] / n_timed
-    gemm_gbs = sb["gemm"] / 1e9 / (gemm_ms * 1e-3) if gemm_ms > 0 else 0.0
-    step_gbs = sb["total"] / 1e9 / (ms_step * 1e-3)
+    gemm_gbs = sb["gemm_shared"] / 1e9 / (gemm_ms * 1e-3) if gemm_ms > 0 else 0.0
+    step_gbs = sb["total_shared"] / 1e9 / (ms_step * 1e-3)
+    step_gbs_sep = sb["total"] / 1e9 / (ms_step * 1e-3)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.shape.dtype,
         "data": "synthetic",
         "config": {"workload": wl.name, "batch": wl.batch, "ctx": wl.ctx, "draft_nodes": wl.n_nodes,
                    "routed_layers": wl.n_routed, "layers": wl.shape.n_layers, "mode": wl.mode,
-                   "l2": "inputs larger than L2: the step streams %.1f GB of weights" % (sb["gemm"] / 1e9),
+                   "l2": "inputs larger than L2: the step streams %.1f GB of weights" % (sb["gemm_shared"] / 1e9),
                    "replicas": world},
         "roofline": {"bound": "hbm", "kernel": "projection GEMMs (all launches of the step)",
                      "achieved": gemm_gbs, "peak": peak, "peak_kind": peak_kind + " copy bandwidth",
                      "unit": "GB/s", "frac": gemm_gbs / peak, "traffic": None,
-                     "algorithmic_bytes_per_step": sb["gemm"], "ms_per_step": gemm_ms,
-                     "launches_per_step": timing["gemm"]["launches"] // n_timed},
-        "step_roofline": {"algorithmic_bytes": sb["total"], "achieved_gbs": step_gbs,
+                     "algorithmic_bytes_per_step": sb["gemm_shared"], "ms_per_step": gemm_ms,
+                     "launches_per_step": timing["gemm"]["launches"] // n_timed,
+                     "note": "per-launch events serialise the launches (no overlap between kernels), so this is a lower "
+                             "bound on what the same kernels reach inside the untimed step"},
+        "step_roofline": {"algorithmic_bytes": sb["total_shared"], "achieved_gbs": step_gbs,
                           "frac_of_measured": step_gbs / peak, "frac_of_8tbs": step_gbs / HBM_NOMINAL_GBS,
+                          "algorithmic_bytes_two_separate_passes": sb["total"],
+                          "achieved_gbs_two_separate_passes": step_gbs_sep,
                           "tensor_frac": sb["flops"] / (ms_step * 1e-3) / 1.67e15},
         "kernel_ms_per_step": {k: v["ms"] / n_timed for k, v in timing.items() if isinstance(v, dict)},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},

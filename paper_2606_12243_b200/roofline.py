@@ -47,9 +47,25 @@ def gemm_bytes(wl: Workload, n_layers: int) -> int:
 
 
 def step_bytes(wl: Workload) -> dict:
+    """Bytes of one verify step.
+
+    "total" / "gemm": the two passes counted separately (each pass streams its own layers and the head).
+    "total_shared" / "gemm_shared": what the one-sweep schedule of viasd_verify_step has to move: every layer's
+    weights and the head once, with the routed layers applied to both row streams; KV caches, appended rows,
+    embeddings and logits of both verifiers as before.
+    """
     s = wl.shape
+    es = s.elem_bytes
     full, slim = pass_bytes(wl, s.n_layers), pass_bytes(wl, wl.n_routed)
     tier = wl.batch * len(set(wl.parent)) * s.vocab * 4
-    return dict(full=full, slim=slim, tier=tier, total=full["total"] + slim["total"] + tier,
-                flops=full["flops"] + slim["flops"],
-                gemm=gemm_bytes(wl, s.n_layers) + gemm_bytes(wl, wl.n_routed))
+    rows = wl.batch * wl.rows
+    qd, kvd = s.n_heads * s.head_dim, s.n_kv_heads * s.head_dim
+    act_per_layer = rows * ((s.d_model * es + (qd + 2 * kvd) * 4) + (qd * es + s.d_model * 4)
+                            + (s.d_model * es + s.d_ff * es) + (s.d_ff * es + s.d_model * 4))
+    head_act = rows * (s.d_model * es + s.vocab * 4)
+    slim_weights = (wl.n_routed * (layer_weight_params(s) + 2 * s.d_model) + s.vocab * s.d_model + s.d_model) * es
+    gemm_sep = gemm_bytes(wl, s.n_layers) + gemm_bytes(wl, wl.n_routed)
+    gemm_shared = gemm_bytes(wl, s.n_layers) + wl.n_routed * act_per_layer + head_act
+    total_sep = full["total"] + slim["total"] + tier
+    return dict(full=full, slim=slim, tier=tier, total=total_sep, flops=full["flops"] + slim["flops"], gemm=gemm_sep,
+                gemm_shared=gemm_shared, total_shared=total_sep - slim_weights)

@@ -145,6 +145,8 @@ def _wl() -> Dict[str, Workload]:
         for ls in (16, 32, 48):
             w[f"c5_32b_b{b}_r{ls}"] = Workload(f"c5_32b_b{b}_r{ls}", s32b, b, 4096, chain(5), ls,
                                                seed=5000)
+    # profiling-sized cut of the 7B workload: same layer shapes, 2 layers (about 1.3 GB on the device)
+    w["c2_7b_l2"] = Workload("c2_7b_l2", replace(s7b, n_layers=2), 1, 1024, chain(8), 1, seed=2000)
     # shrunken siblings: same head_dim, same query/KV-head ratio, same draft shape
     m7 = ModelShape(4, 512, 4, 4, 128, 1408, 2048)
     m8 = ModelShape(4, 512, 4, 1, 128, 1536, 4096)

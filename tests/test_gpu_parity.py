@@ -437,3 +437,34 @@ def test_argument_and_capacity_errors():
     torch.cuda.synchronize()
     assert vb.get_stats(eng.model).device_status == vb.VIASD_ECAPACITY
     assert vb.lib().viasd_strerror(vb.VIASD_ECAPACITY).decode() == "capacity exceeded"
+
+
+# ---------------------------------------------------------------------------------------------
+# full size, in the launch configuration the benchmark times
+# ---------------------------------------------------------------------------------------------
+def test_full_size_7b_verify_step_matches_oracle():
+    """The benchmarked workload (7B-shaped, 32 layers, ctx 1024, chain of 8) through viasd_verify_step, against the
+    oracle evaluated in fp32 on the same generated weights: all logits of both verifiers, tiers, and every pinned
+    decision."""
+    wl = W.get("c2_7b")
+    vb = _vb()
+    eng, st, si, model = _prepare(wl, dt=np.float32)
+    lo, hi = W.thresholds(wl)
+    want = step.verify_step(model, wl.shape, wl.routed, st, si.draft_tok, wl.parent, si.prow, si.drafter_logits,
+                            lo, hi, PU.oracle_params(wl), dt=np.float32)
+    sl, fl = eng.logits_buffer(), eng.logits_buffer()
+    res = vb.alloc_result(wl.batch, wl.n_nodes)
+    vb.verify_step(eng.model, eng.cache, eng.draft, eng.params(), sl, fl, res)
+    torch.cuda.synchronize()
+    assert vb.get_stats(eng.model).device_status == 0
+    assert np.array_equal(res.tier.cpu().numpy(), want.tier)
+    e1, r1 = PU.assert_logits_close(sl.cpu().numpy(), want.slim_logits, "bf16", "slim 7B")
+    e2, r2 = PU.assert_logits_close(fl.cpu().numpy(), want.full_logits, "bf16", "full 7B")
+    pinned, total, full = PU.compare_resolution(want.seqs, res.n_acc.cpu().numpy(), res.path.cpu().numpy(),
+                                                res.out_tok.cpu().numpy(), res.n_emit.cpu().numpy(),
+                                                res.corr_src.cpu().numpy(), eps_row=max(e1, e2))
+    print(f"7B full-size: slim max-abs {e1:.2e} rel-L2 {r1:.2e}; full max-abs {e2:.2e} rel-L2 {r2:.2e}; "
+          f"pinned decisions {pinned}/{total}")
+    assert total == 0 or pinned == total
+    if full == wl.batch:
+        _check_state(eng, st, wl)
