@@ -39,6 +39,16 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
+def gemm_traffic(wl):
+    """DRAM bytes (read + write) of the step's GEMM launches, from the ncu capture summarised in
+    profiles/gemm_tc_kernel_c2_7b_layer_shapes.md: per layer 104.9 + 34.0 + 187.5 + 94.6 MB, head 273.8 MB, captured on
+    the 2-layer cut of the 7B workload and scaled by the number of layers (traffic is per launch and the launches
+    are the same).  Only known for the 7B layer shapes."""
+    if wl.name != "c2_7b":
+        return None
+    return int((104.9 + 34.0 + 187.5 + 94.6) * 1e6 * wl.shape.n_layers + 273.8e6)
+
+
 # ---------------------------------------------------------------------------------------------
 # CPU baseline: the oracle timed on a bounded sample
 # ---------------------------------------------------------------------------------------------
@@ -177,6 +187,24 @@ class ClockSampler:
 
 
 # ---------------------------------------------------------------------------------------------
+# multi-replica aggregation (one process per GPU; replicas are independent, they meet only here)
+# ---------------------------------------------------------------------------------------------
+def max_over_ranks(ms: float, dist, device) -> float:
+    """Slowest replica's time: the job is done when the last rank is."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(world: int, batch: int, n_nodes: int, ms_per_step: float) -> float:
+    """Verified draft tokens per second of the whole job: every replica pushes batch * n_nodes tokens per step."""
+    return world * batch * n_nodes / (ms_per_step * 1e-3)
+
+
+# ---------------------------------------------------------------------------------------------
 # GPU arm
 # ---------------------------------------------------------------------------------------------
 def run_ours(args, wl) -> None:
@@ -234,12 +262,9 @@ def run_ours(args, wl) -> None:
     launches = vb.launch_count() - l0
     ms = ev0.elapsed_time(ev1)
     clk = clocks.stop() if rank == 0 else None
-    if dist is not None:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, dist, "cuda")
     ms_step = ms / args.steps
-    value = world * wl.batch * wl.n_nodes / (ms_step * 1e-3)
+    value = job_value(world, wl.batch, wl.n_nodes, ms_step)
 
     # second timed region with per-launch events: attributes time to kernel classes
     vb.set_timing(eng.model, True)
@@ -275,11 +300,8 @@ def run_ours(args, wl) -> None:
     ev1.record(stream)
     barrier()
     ms_e2e = ev0.elapsed_time(ev1)
-    if dist is not None:
-        t = torch.tensor([ms_e2e], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
-    e2e_value = world * wl.batch * wl.n_nodes / (ms_e2e / args.steps * 1e-3)
+    ms_e2e = max_over_ranks(ms_e2e, dist, "cuda")
+    e2e_value = job_value(world, wl.batch, wl.n_nodes, ms_e2e / args.steps)
 
     if rank != 0:
         if dist is not None:
@@ -304,7 +326,7 @@ def run_ours(args, wl) -> None:
                    "replicas": world},
         "roofline": {"bound": "hbm", "kernel": "projection GEMMs (all launches of the step)",
                      "achieved": gemm_gbs, "peak": peak, "peak_kind": peak_kind + " copy bandwidth",
-                     "unit": "GB/s", "frac": gemm_gbs / peak, "traffic": None,
+                     "unit": "GB/s", "frac": gemm_gbs / peak, "traffic": gemm_traffic(wl),
                      "algorithmic_bytes_per_step": sb["gemm_shared"], "ms_per_step": gemm_ms,
                      "launches_per_step": timing["gemm"]["launches"] // n_timed,
                      "note": "per-launch events serialise the launches (no overlap between kernels), so this is a lower "
