@@ -163,24 +163,50 @@ int attention_nsplit(const viasd_model *m, int batch, int M) {
     return nsplit;
 }
 
+// Key ranges per (sequence, kv head) for the tensor-core kernel, from a small cost model: items are dealt to
+// CTAs in equal contiguous shares, each item costs a fixed part (query staging, merge, partial) plus its tiles,
+// and every extra range adds merge work.  Depends on batch, heads and M only, so the one-stream and the two-stream
+// launch cut the keys at the same places and produce the same bits.
+static int mma_nsplit(const viasd_model *m, int batch, int M, int streams) {
+    const viasd_config &c = m->cfg;
+    const int base = batch * c.n_kv_heads, sms = m->sm_count;
+    const int mt = ((c.n_heads / c.n_kv_heads) * M + 15) / 16;
+    const int tiles = (c.max_ctx + 127) / 128;
+    int max_s = tiles < 16 ? tiles : 16;
+    const double t_tile = 0.5 + 0.8 * mt, t_item = 3.0;
+    int best = 1;
+    double best_cost = 1e30;
+    for (int s = 1; s <= max_s; ++s) {
+        const int n = base * s, ipc = (n + sms - 1) / sms;
+        const int tpi = ((tiles + s - 1) / s);
+        const double cost = ipc * (tpi * t_tile + t_item) + 0.15 * s;
+        if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
+    }
+    size_t per_split = (size_t)streams * batch * c.n_heads * M * (c.head_dim + 2) * sizeof(float);
+    while (best > 1 && per_split * best > m->ws.part_bytes) --best;
+    return best;
+}
+
+// merge of the key ranges: inside the attention kernel when there is little to merge, else its own kernel
+static int mma_attention(viasd_model *m, const void *kc, const void *vc, bool slim, int layer_ord, const void *kc2,
+                         const void *vc2, int layer_ord2, int streams, int batch, int M, cudaStream_t st) {
+    const viasd_config &c = m->cfg;
+    const int nsplit = mma_nsplit(m, batch, M, streams);
+    const int QR = (c.n_heads / c.n_kv_heads) * M;
+    const bool fuse = nsplit > 1 && QR * nsplit <= 160;
+    int rc = launch_attention_mma(m, kc, vc, slim, layer_ord, kc2, vc2, layer_ord2, streams, batch, M, nsplit, fuse ? 1 : 0, st);
+    if (rc || nsplit == 1 || fuse) return rc;
+    attention_combine_kernel<__nv_bfloat16, 128><<<dim3(streams * batch * M, c.n_heads), 128, 0, st>>>(
+        (__nv_bfloat16 *)m->ws.attn, m->ws.rows_alloc * (size_t)c.n_heads * 128, m->ws.part, M, c.n_heads, nsplit);
+    LAUNCH_CHECK();
+    return VIASD_OK;
+}
+
 int launch_attention(viasd_model *m, const void *kc, const void *vc, bool slim, int layer_ord, int batch, int M,
                      cudaStream_t st) {
     const viasd_config &c = m->cfg;
     if (attention_mma_supported(m, M)) {
-        // tensor-core kernel: one CTA per (sequence, kv head, key range of whole 128-key tiles)
-        const int ctas = batch * c.n_kv_heads;
-        int nsplit = (m->sm_count + ctas - 1) / ctas;
-        const int max_tiles = (c.max_ctx + 127) / 128;
-        if (nsplit > max_tiles) nsplit = max_tiles;
-        if (nsplit > 16) nsplit = 16;
-        size_t per_split = (size_t)batch * c.n_heads * M * (c.head_dim + 2) * sizeof(float);
-        while (nsplit > 1 && per_split * nsplit > m->ws.part_bytes) --nsplit;
-        int rc = launch_attention_mma(m, kc, vc, slim, layer_ord, nullptr, nullptr, 0, 1, batch, M, nsplit, st);
-        if (rc || nsplit == 1) return rc;
-        attention_combine_kernel<__nv_bfloat16, 128><<<dim3(batch * M, c.n_heads), 128, 0, st>>>(
-            (__nv_bfloat16 *)m->ws.attn, m->ws.rows_alloc * (size_t)c.n_heads * 128, m->ws.part, M, c.n_heads, nsplit);
-        LAUNCH_CHECK();
-        return VIASD_OK;
+        return mma_attention(m, kc, vc, slim, layer_ord, nullptr, nullptr, 0, 1, batch, M, st);
     }
     int nsplit = attention_nsplit(m, batch, M);
     if (c.dtype == 0) {
@@ -198,17 +224,5 @@ int launch_attention(viasd_model *m, const void *kc, const void *vc, bool slim, 
 int launch_attention_dual(viasd_model *m, const void *kf, const void *vf, int layer_full, const void *ks, const void *vs,
                           int ord_slim, int batch, int M, cudaStream_t st) {
     const viasd_config &c = m->cfg;
-    const int ctas = batch * c.n_kv_heads;                  // same key ranges as the one-stream launch: same bits
-    int nsplit = (m->sm_count + ctas - 1) / ctas;
-    const int max_tiles = (c.max_ctx + 127) / 128;
-    if (nsplit > max_tiles) nsplit = max_tiles;
-    if (nsplit > 16) nsplit = 16;
-    size_t per_split = (size_t)2 * batch * c.n_heads * M * (c.head_dim + 2) * sizeof(float);
-    while (nsplit > 1 && per_split * nsplit > m->ws.part_bytes) --nsplit;
-    int rc = launch_attention_mma(m, kf, vf, false, layer_full, ks, vs, ord_slim, 2, batch, M, nsplit, st);
-    if (rc || nsplit == 1) return rc;
-    attention_combine_kernel<__nv_bfloat16, 128><<<dim3(2 * batch * M, c.n_heads), 128, 0, st>>>(
-        (__nv_bfloat16 *)m->ws.attn, m->ws.rows_alloc * (size_t)c.n_heads * 128, m->ws.part, M, c.n_heads, nsplit);
-    LAUNCH_CHECK();
-    return VIASD_OK;
+    return mma_attention(m, kf, vf, false, layer_full, ks, vs, ord_slim, 2, batch, M, st);
 }

@@ -51,6 +51,7 @@ struct Workspace {                      // pointers into the caller's workspace 
     float *gemm_scratch;                // partial tiles of split GEMM work (tcgen05 kernel)
     int *gemm_counters;                 // per-tile arrival counters, zero between launches
     size_t n_counters;
+    int *attn_counters;                 // [2 * max_batch * Hkv] key-range arrivals per (sequence, kv head)
     float *ssq;                         // [(d / 128) * 4][R] partial sums of h^2 for the fused RMSNorm
 };
 
@@ -141,7 +142,8 @@ int launch_attention(viasd_model *m, const void *kc, const void *vc, bool slim, 
 // attention_mma.cu
 int attention_mma_supported(const viasd_model *m, int M);
 int launch_attention_mma(viasd_model *m, const void *kc, const void *vc, bool slim, int layer_ord, const void *kc2,
-                         const void *vc2, int layer_ord2, int streams, int batch, int M, int nsplit, cudaStream_t st);
+                         const void *vc2, int layer_ord2, int streams, int batch, int M, int nsplit, int fuse_merge,
+                         cudaStream_t st);
 int launch_attention_dual(viasd_model *m, const void *kf, const void *vf, int layer_full, const void *ks, const void *vs,
                           int ord_slim, int batch, int M, cudaStream_t st);
 int launch_embed_norm2(const viasd_model *m, const float *gain_full, const float *gain_slim, int rows, cudaStream_t st);

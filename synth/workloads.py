@@ -147,6 +147,7 @@ def _wl() -> Dict[str, Workload]:
                                                seed=5000)
     # profiling-sized cut of the 7B workload: same layer shapes, 2 layers (about 1.3 GB on the device)
     w["c2_7b_l2"] = Workload("c2_7b_l2", replace(s7b, n_layers=2), 1, 1024, chain(8), 1, seed=2000)
+    w["c4_13b_l2"] = Workload("c4_13b_l2", replace(s13b, n_layers=2), 8, 4096, chain(6), 1, quantiles=(0.30, 0.70), seed=4000)
     # shrunken siblings: same head_dim, same query/KV-head ratio, same draft shape
     m7 = ModelShape(4, 512, 4, 4, 128, 1408, 2048)
     m8 = ModelShape(4, 512, 4, 1, 128, 1536, 4096)
