@@ -20,6 +20,7 @@
 // last CTA to finish one of them (an atomic counter; nobody waits).  The only waits are on TMA arrival and are
 // bounded.
 #include "common.cuh"
+#include <stdlib.h>
 
 namespace {
 
@@ -110,7 +111,7 @@ __device__ __forceinline__ float ex2(float x) {            // 2^x, hardware appr
 // One warp, one 16-row query tile, SUBK (16 or 32) keys starting at key index jbase (tile-relative row r0).
 // The query fragments live in registers; scores are in log2 units (the query was scaled by log2(e) / sqrt(hd)).
 // MASKED: the keys reach past the committed context or past the end of the range.
-template <int SUBK, bool PLO, bool MASKED>
+template <int SUBK, bool PLO, bool QLO, bool MASKED>
 __device__ __forceinline__ void tile_step(const uint32_t (&qh)[8][4], const uint32_t (&ql)[8][4], uint32_t kst, uint32_t vst,
                                           int r0, int lane, int jbase, int n_ctx, int k_end, unsigned long long anc0,
                                           unsigned long long anc1, float (&mrun)[2], float (&lrun)[2], float (&o)[16][4]) {
@@ -132,8 +133,10 @@ __device__ __forceinline__ void tile_step(const uint32_t (&qh)[8][4], const uint
         // independent accumulators first with the hi part of Q, then with the lo part
 #pragma unroll
         for (int np = 0; np < NS / 2; ++np) { mma16816(s[np * 2], qh[ks], b[np][0], b[np][1]); mma16816(s[np * 2 + 1], qh[ks], b[np][2], b[np][3]); }
+        if (QLO) {
 #pragma unroll
-        for (int np = 0; np < NS / 2; ++np) { mma16816(s[np * 2], ql[ks], b[np][0], b[np][1]); mma16816(s[np * 2 + 1], ql[ks], b[np][2], b[np][3]); }
+            for (int np = 0; np < NS / 2; ++np) { mma16816(s[np * 2], ql[ks], b[np][0], b[np][1]); mma16816(s[np * 2 + 1], ql[ks], b[np][2], b[np][3]); }
+        }
     }
     // mask, online softmax (rows g and g + 8 of the tile; columns 8n + 2t, 8n + 2t + 1)
     float mx[2] = {-INFINITY, -INFINITY};
@@ -168,7 +171,10 @@ __device__ __forceinline__ void tile_step(const uint32_t (&qh)[8][4], const uint
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const float m = mrun[e >> 1];
-            const float p = (MASKED && s[n][e] == -INFINITY) ? 0.f : ex2(s[n][e] - m);
+            float p = (MASKED && s[n][e] == -INFINITY) ? 0.f : ex2(s[n][e] - m);
+            // without the lo part the MMA sees bf16(p): normalise by the sum of those same rounded values, or the
+            // rounding of near-equal weights would not cancel
+            if (!PLO) p = __bfloat162float(__float2bfloat16_rn(p));
             s[n][e] = p;
             rs[e >> 1] += p;
         }
@@ -227,8 +233,8 @@ __device__ __forceinline__ Item decode_item(const AttnArgs &a, int item) {
     return it;
 }
 
-// PLO: use the lo part of the probabilities too (few query rows: the extra MMAs are free)
-template <bool PLO>
+// PLO / QLO: use the lo parts of the probabilities / of the query too
+template <bool PLO, bool QLO>
 __global__ void __launch_bounds__(WARPS * 32)
 attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                      const __grid_constant__ CUtensorMap map_k2, const __grid_constant__ CUtensorMap map_v2, const AttnArgs a) {
@@ -340,18 +346,18 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
                     const int r0 = kgroup * 16, jb = j0 + r0;
                     if (jb < it.k_end) {
                         if (jb + 16 <= it.n_ctx && jb + 16 <= it.k_end)
-                            tile_step<16, PLO, false>(qh, ql, kst, vst, r0, lane, jb, it.n_ctx, it.k_end, anc[0], anc[1], mrun, lrun, o);
+                            tile_step<16, PLO, QLO, false>(qh, ql, kst, vst, r0, lane, jb, it.n_ctx, it.k_end, anc[0], anc[1], mrun, lrun, o);
                         else
-                            tile_step<16, PLO, true>(qh, ql, kst, vst, r0, lane, jb, it.n_ctx, it.k_end, anc[0], anc[1], mrun, lrun, o);
+                            tile_step<16, PLO, QLO, true>(qh, ql, kst, vst, r0, lane, jb, it.n_ctx, it.k_end, anc[0], anc[1], mrun, lrun, o);
                     }
                 } else {
                     for (int sub = 0; sub < kg_keys; sub += 32) {
                         const int r0 = kgroup * kg_keys + sub, jb = j0 + r0;
                         if (jb < it.k_end) {
                             if (jb + 32 <= it.n_ctx && jb + 32 <= it.k_end)
-                                tile_step<32, PLO, false>(qh, ql, kst, vst, r0, lane, jb, it.n_ctx, it.k_end, anc[0], anc[1], mrun, lrun, o);
+                                tile_step<32, PLO, QLO, false>(qh, ql, kst, vst, r0, lane, jb, it.n_ctx, it.k_end, anc[0], anc[1], mrun, lrun, o);
                             else
-                                tile_step<32, PLO, true>(qh, ql, kst, vst, r0, lane, jb, it.n_ctx, it.k_end, anc[0], anc[1], mrun, lrun, o);
+                                tile_step<32, PLO, QLO, true>(qh, ql, kst, vst, r0, lane, jb, it.n_ctx, it.k_end, anc[0], anc[1], mrun, lrun, o);
                         }
                     }
                 }
@@ -521,15 +527,19 @@ int launch_attention_mma(viasd_model *m, const void *kc, const void *vc, bool sl
     const size_t smem = 1024 + a.nstage * (size_t)STAGE_BYTES + q_bytes + osm_bytes;
     static bool attr_done = false;
     if (!attr_done) {
-        CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
-        CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
+        CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
+        CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
+        CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
         attr_done = true;
     }
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
     pdl_config(cfg, attr, dim3(grid), dim3(WARPS * 32), smem, st);
-    if (mt <= 2) CUDA_TRY(cudaLaunchKernelEx(&cfg, attention_mma_kernel<true>, cm.k, cm.v, cm2->k, cm2->v, a));
-    else CUDA_TRY(cudaLaunchKernelEx(&cfg, attention_mma_kernel<false>, cm.k, cm.v, cm2->k, cm2->v, a));
+    static int lo_mode = -1;                 // VIASD_ATTN_LO: 2 = hi/lo for Q and P, 1 = hi/lo for Q only, 0 = plain bf16
+    if (lo_mode < 0) { const char *e = getenv("VIASD_ATTN_LO"); lo_mode = e ? atoi(e) : 2; }
+    if (lo_mode >= 2) CUDA_TRY(cudaLaunchKernelEx(&cfg, attention_mma_kernel<true, true>, cm.k, cm.v, cm2->k, cm2->v, a));
+    else if (lo_mode == 1) CUDA_TRY(cudaLaunchKernelEx(&cfg, attention_mma_kernel<false, true>, cm.k, cm.v, cm2->k, cm2->v, a));
+    else CUDA_TRY(cudaLaunchKernelEx(&cfg, attention_mma_kernel<false, false>, cm.k, cm.v, cm2->k, cm2->v, a));
     LAUNCH_CHECK();
     return VIASD_OK;
 }
