@@ -21,236 +21,16 @@
 #include "gemm_tc.cuh"
 #include <stdlib.h>
 
+#include "gemm_tc_device.cuh"
+
 namespace {
-
-constexpr int TILE_F = 128;          // output features per tile (MMA M)
-constexpr int TILE_K = 64;           // bf16 per k-block: 128 bytes, one swizzle row
-constexpr int MAX_STAGES = 12;
-constexpr int THREADS = 192;
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about two seconds
-
-// ---- PTX wrappers ---------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.b32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait.  Returns false when the limit expired or another role of this CTA already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    int spins = 0;
-    while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 255) == 0) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
-                *abort_flag = 1;
-                atomicExch(status, VIASD_EDEVICE);
-                return false;
-            }
-        }
-    }
-    return true;
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-constexpr int CH = 8;                // token rows per epilogue chunk
-__device__ __forceinline__ void tc_ld8(uint32_t taddr, float (&v)[CH]) {
-    uint32_t r[8];
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-                 : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
-}
-
-// K-major operand tile, 128-byte swizzle, rows 128 bytes apart, 8-row groups 1024 bytes apart
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
-    return (uint64_t)((addr >> 4) & 0x3FFF) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
-}
-
-#ifdef VIASD_TC_TRACE
-__device__ long long g_tc_trace[160 * 8];
-#define TRACE(slot) do { if (p.trace_on) g_tc_trace[blockIdx.x * 8 + (slot)] = clock64(); } while (0)
-#define DBG(p, bit) ((p).dbg & (bit))
-__device__ unsigned long long g_tc_span[8192 * 2];       // per launch: earliest CTA start, latest CTA end (globaltimer ns)
-__device__ __forceinline__ unsigned long long gtimer() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define SPAN_BEGIN(p) do { if (threadIdx.x == 0) atomicMin(&g_tc_span[((p).launch_idx & 8191) * 2], gtimer()); } while (0)
-#define SPAN_END(p) do { if (threadIdx.x == 0) atomicMax(&g_tc_span[((p).launch_idx & 8191) * 2 + 1], gtimer()); } while (0)
-#else
-#define SPAN_BEGIN(p) do { } while (0)
-#define SPAN_END(p) do { } while (0)
-#define DBG(p, bit) 0
-#define TRACE(slot) do { } while (0)
-#endif
-
-struct Seg { int tile, ka, kb; };      // one contiguous piece of this CTA's unit range inside a tile
-
-__device__ __forceinline__ bool next_seg(int &u, int u1, int k_tiles, Seg &s) {
-    if (u >= u1) return false;
-    s.tile = u / k_tiles;
-    s.ka = u - s.tile * k_tiles;
-    s.kb = min(k_tiles, s.ka + (u1 - u));
-    u += s.kb - s.ka;
-    return true;
-}
-
-// Epilogue for CH token rows r0..r0+CH-1 of one tile; thread f holds the full-K sums g (and u for the gate/up
-// pair) of output feature f.  Called by all 128 epilogue threads together.  The epilogue kind is a template
-// parameter so that each kernel carries one short epilogue: this code runs once per tile, straight from the
-// instruction cache's cold side, and its size is what its latency is made of.
-template <int EPI>
-__device__ __forceinline__ void finish_chunk(const TcParams &p, int tile, int f, int r0, float (&g)[CH], float (&uu)[CH],
-                                             float *xch, const float *inv_sh, const int4 *rowmeta, int lane) {
-    constexpr bool DUAL = EPI == EPI_SWIGLU;
-    if (EPI == EPI_STORE || EPI == EPI_SWIGLU || EPI == EPI_QKV_ROPE) {
-        if (p.ssq_in) {                   // the input was h * gain without its RMS factor: apply it per row here
-#pragma unroll
-            for (int j = 0; j < CH; ++j) {
-                const float sc = inv_sh[min(r0 + j, 127)];
-                g[j] *= sc;
-                if (DUAL) uu[j] *= sc;
-            }
-        }
-    }
-    const int nrow = min(CH, p.rows - r0);
-    if (DUAL) {
-        const int n = tile * TILE_F + f;
-        if (n >= p.seg_n[0]) return;
-        __nv_bfloat16 *dst = p.out_act + (size_t)(p.row0 + r0) * p.ld_out + n;
-#pragma unroll
-        for (int j = 0; j < CH; ++j) {
-            if (j < nrow) {
-                const float sg = g[j] / (1.f + __expf(-g[j]));
-                store_act<__nv_bfloat16>(dst, p.act_plane, (size_t)j * p.ld_out, sg * uu[j]);
-            }
-        }
-        return;
-    }
-    int s = 0, t0 = 0, nbase = 0;
-    while (s < 2 && tile >= p.seg_tile_end[s]) { t0 = p.seg_tile_end[s]; nbase += p.seg_n[s]; ++s; }
-    const int nin = (tile - t0) * TILE_F + f;
-    const bool valid = nin < p.seg_n[s];
-    const int n = nbase + nin;
-    if (EPI == EPI_STORE) {
-        if (!valid) return;
-#pragma unroll
-        for (int j = 0; j < CH; ++j) {
-            if (j < nrow) {
-                const int row = p.row0 + r0 + j;          // the second stream's rows go to the second output
-                float *dst = row < p.split_row ? p.out_f32 + (size_t)row * p.ld_out + n
-                                               : p.out_f32_2 + (size_t)(row - p.split_row) * p.ld_out + n;
-                if (p.epi == EPI_ADD) *dst += g[j]; else *dst = g[j];
-            }
-        }
-    } else if (EPI == EPI_ADD_NORM) {
-        // residual update, plus what the next RMSNorm needs: h * gain as hi/lo planes and partial sums of h^2.
-        // Loads first, then arithmetic, then stores: the CH rows cost one memory round trip.
-        const float gain_a = valid ? p.next_gain[n] : 0.f;
-        const float gain_b = (valid && p.next_gain2) ? p.next_gain2[n] : gain_a;
-        float *hp = p.out_f32 + (size_t)(p.row0 + r0) * p.ld_out + n;
-        __nv_bfloat16 *ap = p.next_act + (size_t)(p.row0 + r0) * p.ld_out + n;
-        float v[CH];
-#pragma unroll
-        for (int j = 0; j < CH; ++j) v[j] = (valid && j < nrow) ? __ldcg(hp + (size_t)j * p.ld_out) + g[j] : 0.f;
-#pragma unroll
-        for (int j = 0; j < CH; ++j) {
-            if (valid && j < nrow) {
-                hp[(size_t)j * p.ld_out] = v[j];
-                store_act<__nv_bfloat16>(ap, p.next_plane, (size_t)j * p.ld_out,
-                                         v[j] * (p.row0 + r0 + j < p.split_row ? gain_a : gain_b));
-            }
-            v[j] *= v[j];
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1)
-#pragma unroll
-            for (int j = 0; j < CH; ++j) v[j] += __shfl_xor_sync(0xffffffffu, v[j], o);
-        if (lane < nrow) {
-            float mine = v[0];
-#pragma unroll
-            for (int j = 1; j < CH; ++j) mine = lane == j ? v[j] : mine;
-            p.ssq_out[((size_t)tile * 4 + (f >> 5)) * p.ssq_stride + p.row0 + r0 + lane] = mine;
-        }
-    } else {   // EPI_QKV_ROPE: one tile is one head of 128 dims; rotate pairs (p, p + 64), write q / K cache / V cache
-#pragma unroll
-        for (int j = 0; j < CH; ++j) xch[j * TILE_F + f] = g[j];
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        const int head = tile - t0, pidx = f & 63;
-        if (s < 2) {
-            float c[CH], sn[CH];
-#pragma unroll
-            for (int j = 0; j < CH; ++j) {
-                const int pos = rowmeta[min(r0 + j, 127)].x;
-                c[j] = p.cosv[(size_t)pos * 64 + pidx];
-                sn[j] = p.sinv[(size_t)pos * 64 + pidx];
-            }
-#pragma unroll
-            for (int j = 0; j < CH; ++j) {
-                const float other = xch[j * TILE_F + (f ^ 64)];
-                g[j] = f < 64 ? g[j] * c[j] - other * sn[j] : g[j] * c[j] + other * sn[j];
-            }
-        }
-        if (s == 0) {
-            float *dst = p.q_out + ((size_t)(p.row0 + r0) * p.rope_H + head) * TILE_F + f;
-#pragma unroll
-            for (int j = 0; j < CH; ++j) if (j < nrow) dst[(size_t)j * p.rope_H * TILE_F] = g[j];
-        } else {
-#pragma unroll
-            for (int j = 0; j < CH; ++j) {
-                if (j < nrow) {
-                    const int4 rm = rowmeta[r0 + j];
-                    __nv_bfloat16 *cache = rm.w ? (s == 1 ? p.kc2 : p.vc2) : (s == 1 ? p.kc : p.vc);
-                    const int lo = rm.w ? p.layer_ord2 : p.layer_ord;
-                    cache[((((size_t)lo * p.max_batch + rm.z) * p.rope_Hkv + head) * p.max_ctx + rm.y) * TILE_F + f] =
-                        __float2bfloat16_rn(g[j]);
-                }
-            }
-        }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-    }
-}
 
 template <int EPI>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
                const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_x, const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) unsigned long long bars[2 * MAX_STAGES + 4];
+    __shared__ __align__(8) unsigned long long bars[2 * MAX_STAGES + 5];
     __shared__ uint32_t tmem_base_sh;
     __shared__ int abort_sh, last_sh;
     __shared__ float inv_sh[128];                       // per-row 1/rms of the input (fused RMSNorm)
@@ -271,12 +51,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
     auto empty_bar = [&](int s) { return smem_u32(&bars[MAX_STAGES + s]); };
     auto tfull_bar = [&](int b) { return smem_u32(&bars[2 * MAX_STAGES + b]); };
     auto tempty_bar = [&](int b) { return smem_u32(&bars[2 * MAX_STAGES + 2 + b]); };
+    const uint32_t gather_bar = smem_u32(&bars[2 * MAX_STAGES + 4]);
     const int NB = p.has_lo ? 2 * NT : NT;                  // MMA N: hi and lo token columns side by side
     const uint32_t acc_cols = NACC * NB;                    // TMEM columns per accumulator buffer
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+        mbar_init(gather_bar, 128);
         abort_sh = 0;
         last_sh = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -331,7 +113,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                              "r"(DUAL ? 2 * p.a_tx[0] : p.a_tx[sidx]) : "memory");
                 load_w(it, mw, wrow, kt);
             }
+            TRACE(2);
             asm volatile("griddepcontrol.wait;" ::: "memory");
+            TRACE(3);
             for (int it = 0; it < pre; ++it) {
                 unit(it, mw, wrow, kt, sidx);
                 mbar_expect_tx(full_bar(it), 2 * p.b_tx);
@@ -361,6 +145,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                 for (int kt = sg.ka; kt < sg.kb; ++kt, ++it) {
                     const int st = it % S;
                     if (!(ok = mbar_wait(full_bar(st), (it / S) & 1, &abort_sh, p.status))) break;
+                    if (it == 0) TRACE(4);
                     tc_fence_after();
                     const uint32_t base = smem_base + st * stage_bytes;
                     // the hi tile is followed by the lo tile: together one K-major operand of NB rows
@@ -376,131 +161,224 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                 if (ok) tc_commit(tfull_bar(buf));          // accumulator complete
                 ++acc_it;
             }
-            TRACE(3);
+            TRACE(5);
         }
     } else {
         // ---------------- epilogue (warps 2..5 <-> TMEM lane quarters 2,3,0,1) ----------------
-        asm volatile("griddepcontrol.wait;" ::: "memory");     // outputs, scratch and counters belong to the chain
         const int quarter = warp & 3;
-        const int f = quarter * 32 + lane;                  // feature lane inside the tile
+        const int f = quarter * 32 + lane;                  // feature lane inside the tile, as TMEM lanes map to warps
         const int et = threadIdx.x - 64;                    // 0..127 among epilogue threads
         const size_t slot_floats = (size_t)NACC * NT * TILE_F;
         // per-row tables (all 128 entries defined: chunks read a few rows past p.rows and discard them)
         inv_sh[et] = 0.f;
         rowmeta[et] = make_int4(0, 0, 0, 0);
         asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (p.ssq_in) {
-            // 1/rms per input row: a warp sums the row's partial sums of squares (fixed order: reproducible)
-            for (int r = (et >> 5); r < p.rows; r += 4) {
-                float ss = 0.f;
-                for (int j = lane; j < p.ssq_in_n; j += 32) ss += __ldcg(p.ssq_in + (size_t)j * p.ssq_stride + p.row0 + r);
-                ss = warp_sum(ss);
-                if (lane == 0) inv_sh[r] = rsqrtf(ss * p.inv_d + p.eps);
-            }
-        }
-        if (EPI == EPI_QKV_ROPE) {
-            if (et < p.rows) {
-                // rows are laid out [stream][sequence][block row]; stream 1 (rows >= split_row) is the slim verifier
-                const int row = p.row0 + et, stream = row >= p.split_row ? 1 : 0, rs = row - stream * p.split_row;
-                const int b = rs / p.rope_M, i = rs - b * p.rope_M;
-                const int n_ctx = p.len_eff[b];
-                rowmeta[et] = make_int4(n_ctx + p.depth[i], n_ctx + i, b, stream);
-            }
-        }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+
+        // A tile is finished from one of three sources: the accumulator in TMEM (this CTA held all of K), the
+        // partials staged in shared memory, or the partials read straight from global memory.  All three feed ONE
+        // copy of the epilogue code, and that copy runs once "dry" (no row is live, nothing is stored) before
+        // the kernel waits for its predecessor: the epilogue otherwise runs exactly once per CTA, at the very end,
+        // from a cold instruction cache while HBM is saturated, and those instruction misses were the tail.
+        enum { SRC_DRY, SRC_TMEM, SRC_SMEM, SRC_GLOBAL };
         int acc_it = 0, u = u_begin, seg_i = 0;
         Seg sg;
-        bool ok = true;
-        while (ok && next_seg(u, u_end, p.k_tiles, sg)) {
-            const int buf = acc_it % p.acc_bufs;
-            if (!(ok = mbar_wait(tfull_bar(buf), (acc_it / p.acc_bufs) & 1, &abort_sh, p.status))) break;
-            tc_fence_after();
-            const bool whole = sg.ka == 0 && sg.kb == p.k_tiles;
-            const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * acc_cols;
-            // partial of a split tile: slot 0 if the tile is the first one this CTA touches, else slot 1
-            float *slot = p.scratch + ((size_t)blockIdx.x * 2 + (seg_i == 0 ? 0 : 1)) * slot_floats;
-            for (int c = 0; c < p.rows; c += CH) {           // padding rows beyond p.rows are never read
-                float g[CH], uu[CH];
-                tc_ld8(t0 + c, g);
-                if (DUAL) tc_ld8(t0 + NB + c, uu);
-                if (p.has_lo) {                              // add the product with the lo plane
-                    float lo[CH];
-                    tc_ld8(t0 + NT + c, lo);
-#pragma unroll
-                    for (int j = 0; j < CH; ++j) g[j] += lo[j];
-                    if (DUAL) {
-                        tc_ld8(t0 + NB + NT + c, lo);
-#pragma unroll
-                        for (int j = 0; j < CH; ++j) uu[j] += lo[j];
-                    }
-                }
-                if (whole) {
-                    finish_chunk<EPI>(p, sg.tile, f, c, g, uu, xch, inv_sh, rowmeta, lane);
+        sg.tile = (u_end - 1) / p.k_tiles; sg.ka = 0; sg.kb = 0;   // dry pass: the tile this CTA is most likely to finish
+        bool ok = true, dry = true;
+        while (ok) {
+            int src = SRC_DRY, buf = 0, first_cta = 0, last_cta = 0;
+            uint32_t t0 = 0;
+            const float *parts = nullptr, *aux = nullptr;
+            if (!dry) {
+                if (!next_seg(u, u_end, p.k_tiles, sg)) break;
+                buf = acc_it % p.acc_bufs;
+                if (!(ok = mbar_wait(tfull_bar(buf), (acc_it / p.acc_bufs) & 1, &abort_sh, p.status))) break;
+                if (et == 0) TRACE(6);
+                tc_fence_after();
+                t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * acc_cols;
+                if (sg.ka == 0 && sg.kb == p.k_tiles) {
+                    src = SRC_TMEM;
                 } else {
+                    // partial of a split tile: slot 0 if the tile is the first one this CTA touches, else slot 1
+                    float *slot = p.scratch + ((size_t)blockIdx.x * 2 + (seg_i == 0 ? 0 : 1)) * slot_floats;
+                    for (int c = 0; c < p.rows; c += CH) {       // padding rows beyond p.rows are never read
+                        float g[CH], uu[CH];
+                        tc_ld8(t0 + c, g);
+                        if (DUAL) tc_ld8(t0 + NB + c, uu);
+                        if (p.has_lo) {                          // add the product with the lo plane
+                            float lo[CH];
+                            tc_ld8(t0 + NT + c, lo);
 #pragma unroll
-                    for (int j = 0; j < CH; ++j) {
-                        slot[(size_t)(c + j) * TILE_F + f] = g[j];
-                        if (DUAL) slot[(size_t)(NT + c + j) * TILE_F + f] = uu[j];
+                            for (int j = 0; j < CH; ++j) g[j] += lo[j];
+                            if (DUAL) {
+                                tc_ld8(t0 + NB + NT + c, lo);
+#pragma unroll
+                                for (int j = 0; j < CH; ++j) uu[j] += lo[j];
+                            }
+                        }
+#pragma unroll
+                        for (int j = 0; j < CH; ++j) {
+                            slot[(size_t)(c + j) * TILE_F + f] = g[j];
+                            if (DUAL) slot[(size_t)(NT + c + j) * TILE_F + f] = uu[j];
+                        }
+                    }
+                    if (et == 0) TRACE(7);
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tempty_bar(buf));   // accumulator buffer may be overwritten
+                    // publish the partial; the last contributor of the tile sums all of them in CTA order
+                    __threadfence();
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    first_cta = (sg.tile * p.k_tiles) / p.units_per_cta;
+                    last_cta = ((sg.tile + 1) * p.k_tiles - 1) / p.units_per_cta;
+                    if (et == 0) {
+                        const int old = atomicAdd(&p.counters[sg.tile], 1);
+                        last_sh = (old == last_cta - first_cta) ? 1 : 0;
+                        if (last_sh) p.counters[sg.tile] = 0;   // ready for the next launch
+                    }
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    if (et == 0) TRACE(8);
+                    const bool last = last_sh != 0;
+                    asm volatile("bar.sync 1, 128;" ::: "memory");   // last_sh is reused by the next split tile
+                    if (!last) { ++acc_it; ++seg_i; continue; }
+                    __threadfence();
+                    if (et == 0) TRACE(13);
+                    src = SRC_GLOBAL;
+                    // Staged gather: when this is the CTA's last piece of work the shared-memory ring is idle, so
+                    // all partials (and the rows the epilogue would otherwise fetch chunk by chunk) come in with
+                    // one round of bulk copies.  Same sums in the same order as the direct path.
+                    const int n_c = last_cta - first_cta + 1;
+                    const uint32_t part_bytes = (uint32_t)p.rows * TILE_F * 4;
+                    if (u >= u_end && (uint32_t)(n_c * NACC + 1) * part_bytes <= (uint32_t)S * stage_bytes) {
+                        const uint32_t aux_sh = smem_base, part_sh = smem_base + part_bytes;
+                        int aux_kind = 0;                    // 1: residual rows, 2: rotary tables
+                        if (EPI == EPI_ADD_NORM && (sg.tile + 1) * TILE_F <= p.seg_n[0]) aux_kind = 1;
+                        if (EPI == EPI_QKV_ROPE && sg.tile < p.seg_tile_end[1]) aux_kind = 2;
+                        const bool has_part = et < n_c * NACC, has_aux = aux_kind && et < p.rows;
+                        asm volatile("fence.proxy.async.global;" ::: "memory");
+                        if (has_part || has_aux) {
+                            mbar_expect_tx(gather_bar, (has_part ? part_bytes : 0u) + (has_aux ? TILE_F * 4u : 0u));
+                            if (has_part) {
+                                const int c = first_cta + et / NACC, half = et - (et / NACC) * NACC;
+                                const int c_first_tile = (c * p.units_per_cta) / p.k_tiles;
+                                const float *from = p.scratch + ((size_t)c * 2 + (c_first_tile == sg.tile ? 0 : 1)) * slot_floats +
+                                                    (size_t)half * NT * TILE_F;
+                                bulk_load(part_sh + (uint32_t)et * part_bytes, from, part_bytes, gather_bar);
+                            }
+                            if (has_aux) {
+                                const uint32_t dst = aux_sh + (uint32_t)et * TILE_F * 4;
+                                if (aux_kind == 1) {
+                                    bulk_load(dst, p.out_f32 + (size_t)(p.row0 + et) * p.ld_out + sg.tile * TILE_F, TILE_F * 4, gather_bar);
+                                } else {
+                                    const int pos = rowmeta[et].x;
+                                    bulk_load(dst, p.cosv + (size_t)pos * 64, 256, gather_bar);
+                                    bulk_load(dst + 256, p.sinv + (size_t)pos * 64, 256, gather_bar);
+                                }
+                            }
+                        } else {
+                            mbar_arrive(gather_bar);
+                        }
+                        if (!(ok = mbar_wait(gather_bar, 0, &abort_sh, p.status))) break;
+                        if (et == 0) TRACE(14);
+                        parts = reinterpret_cast<const float *>(smem_raw + (part_sh - smem_u32(smem_raw)));
+                        if (aux_kind) aux = reinterpret_cast<const float *>(smem_raw + (aux_sh - smem_u32(smem_raw)));
+                        src = SRC_SMEM;
                     }
                 }
             }
-            if (et == 0) TRACE(2);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(buf));   // accumulator buffer may be overwritten
-            if (!whole) {
-                // publish the partial; the last contributor of the tile sums all of them in CTA order
-                __threadfence();
-                asm volatile("bar.sync 1, 128;" ::: "memory");
-                if (et == 0) {
-                    const int first_cta = (sg.tile * p.k_tiles) / p.units_per_cta;
-                    const int last_cta = ((sg.tile + 1) * p.k_tiles - 1) / p.units_per_cta;
-                    const int old = atomicAdd(&p.counters[sg.tile], 1);
-                    last_sh = (old == last_cta - first_cta) ? 1 : 0;
-                    if (last_sh) p.counters[sg.tile] = 0;   // ready for the next launch
-                }
-                asm volatile("bar.sync 1, 128;" ::: "memory");
-                if (et == 0) TRACE(5);
-                if (last_sh) {
-                    __threadfence();
-                    const int first_cta = (sg.tile * p.k_tiles) / p.units_per_cta;
-                    const int last_cta = ((sg.tile + 1) * p.k_tiles - 1) / p.units_per_cta;
-                    for (int r0 = 0; r0 < p.rows; r0 += CH) {
-                        float g[CH], uu[CH];
+
+            // ---- the one finishing loop
+            const int fe = src == SRC_TMEM ? f : et;
+            const int rows_live = dry ? 0 : p.rows, rows_loop = dry ? CH : p.rows, plane = p.rows * TILE_F;
+#pragma unroll 1
+            for (int r0 = 0; r0 < rows_loop; r0 += CH) {
+                float g[CH], uu[CH];
 #pragma unroll
-                        for (int j = 0; j < CH; ++j) { g[j] = 0.f; uu[j] = 0.f; }
-                        // contributors four at a time: all their loads are in flight before the first add, and the
-                        // sums still run in CTA order
-                        for (int c0 = first_cta; c0 <= last_cta; c0 += 4) {
-                            float pg[4][CH], pu[4][CH];
+                for (int j = 0; j < CH; ++j) { g[j] = 0.f; uu[j] = 0.f; }
+                if (src == SRC_TMEM) {
+                    tc_ld8(t0 + r0, g);
+                    if (DUAL) tc_ld8(t0 + NB + r0, uu);
+                    if (p.has_lo) {
+                        float lo[CH];
+                        tc_ld8(t0 + NT + r0, lo);
 #pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                const int c = c0 + q;
-                                const bool on = c <= last_cta;
-                                const int c_first_tile = (c * p.units_per_cta) / p.k_tiles;
-                                const float *src = p.scratch + ((size_t)(on ? c : first_cta) * 2 + (c_first_tile == sg.tile ? 0 : 1)) *
-                                                   slot_floats + (size_t)r0 * TILE_F + et;
+                        for (int j = 0; j < CH; ++j) g[j] += lo[j];
+                        if (DUAL) {
+                            tc_ld8(t0 + NB + NT + r0, lo);
 #pragma unroll
-                                for (int j = 0; j < CH; ++j) {     // slots are NT >= rows + CH - 1 rows deep: in bounds
-                                    pg[q][j] = on ? __ldcg(src + (size_t)j * TILE_F) : 0.f;
-                                    if (DUAL) pu[q][j] = on ? __ldcg(src + (size_t)(NT + j) * TILE_F) : 0.f;
-                                }
-                            }
-#pragma unroll
-                            for (int q = 0; q < 4; ++q)
-#pragma unroll
-                                for (int j = 0; j < CH; ++j) { g[j] += pg[q][j]; if (DUAL) uu[j] += pu[q][j]; }
+                            for (int j = 0; j < CH; ++j) uu[j] += lo[j];
                         }
-                        if (et == 0) TRACE(6);
-                        finish_chunk<EPI>(p, sg.tile, et, r0, g, uu, xch, inv_sh, rowmeta, lane);
-                        if (et == 0) TRACE(1);
+                    }
+                } else if (src == SRC_SMEM) {
+                    for (int c = 0; c <= last_cta - first_cta; ++c) {
+#pragma unroll
+                        for (int j = 0; j < CH; ++j) {
+                            const int r = min(r0 + j, p.rows - 1);        // rows past the end are discarded
+                            g[j] += parts[(c * NACC) * plane + r * TILE_F + et];
+                            if (DUAL) uu[j] += parts[(c * NACC + 1) * plane + r * TILE_F + et];
+                        }
+                    }
+                } else if (src == SRC_GLOBAL) {
+                    // contributors four at a time: all their loads are in flight before the first add, and the
+                    // sums still run in CTA order
+                    for (int c0 = first_cta; c0 <= last_cta; c0 += 4) {
+                        float pg[4][CH], pu[4][CH];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const int c = c0 + q;
+                            const bool on = c <= last_cta;
+                            const int c_first_tile = (c * p.units_per_cta) / p.k_tiles;
+                            const float *from = p.scratch + ((size_t)(on ? c : first_cta) * 2 + (c_first_tile == sg.tile ? 0 : 1)) *
+                                                slot_floats + (size_t)r0 * TILE_F + et;
+#pragma unroll
+                            for (int j = 0; j < CH; ++j) {     // slots are NT >= rows + CH - 1 rows deep: in bounds
+                                pg[q][j] = on ? __ldcg(from + (size_t)j * TILE_F) : 0.f;
+                                if (DUAL) pu[q][j] = on ? __ldcg(from + (size_t)(NT + j) * TILE_F) : 0.f;
+                            }
+                        }
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+#pragma unroll
+                            for (int j = 0; j < CH; ++j) { g[j] += pg[q][j]; if (DUAL) uu[j] += pu[q][j]; }
                     }
                 }
-                asm volatile("bar.sync 1, 128;" ::: "memory");   // last_sh is reused by the next split tile
+                if (et == 0 && r0 == 0) TRACE(9);
+                finish_chunk<EPI>(p, sg.tile, fe, r0, g, uu, xch, inv_sh, rowmeta, lane, aux, rows_live);
+                if (et == 0 && r0 == 0) TRACE(15);
+            }
+
+            if (dry) {
+                dry = false;
+                asm volatile("griddepcontrol.wait;" ::: "memory");     // outputs, scratch and counters belong to the chain
+                if (p.ssq_in) {
+                    // 1/rms per input row: a warp sums the row's partial sums of squares (fixed order: reproducible)
+                    for (int r = (et >> 5); r < p.rows; r += 4) {
+                        float ss = 0.f;
+                        for (int j = lane; j < p.ssq_in_n; j += 32) ss += __ldcg(p.ssq_in + (size_t)j * p.ssq_stride + p.row0 + r);
+                        ss = warp_sum(ss);
+                        if (lane == 0) inv_sh[r] = rsqrtf(ss * p.inv_d + p.eps);
+                    }
+                }
+                if (EPI == EPI_QKV_ROPE) {
+                    if (et < p.rows) {
+                        // rows are laid out [stream][sequence][block row]; stream 1 (rows >= split_row) is the slim verifier
+                        const int row = p.row0 + et, stream = row >= p.split_row ? 1 : 0, rs = row - stream * p.split_row;
+                        const int b = rs / p.rope_M, i = rs - b * p.rope_M;
+                        const int n_ctx = p.len_eff[b];
+                        rowmeta[et] = make_int4(n_ctx + p.depth[i], n_ctx + i, b, stream);
+                    }
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                continue;
+            }
+            if (src == SRC_TMEM) {
+                if (et == 0) TRACE(7);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty_bar(buf));   // accumulator buffer may be overwritten
             }
             ++acc_it;
             ++seg_i;
-            if (et == 0) TRACE(4);
+            if (et == 0) TRACE(10);
         }
     }
 
@@ -513,7 +391,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
     }
     tc_fence_before();
     __syncthreads();
-    if (threadIdx.x == 0) TRACE(7);
+    if (threadIdx.x == 0) { TRACE(11); TRACE_SM(); }
     SPAN_END(p);
     if (warp == 1) {
         tc_fence_after();
@@ -550,7 +428,7 @@ int tc_make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t k, u
 
 #ifdef VIASD_TC_TRACE
 extern "C" int viasd_debug_trace(long long *host_out) {
-    return (int)cudaMemcpyFromSymbol(host_out, g_tc_trace, sizeof(long long) * 160 * 8);
+    return (int)cudaMemcpyFromSymbol(host_out, g_tc_trace, sizeof(long long) * 160 * 16);
 }
 static int g_span_launches = 0;
 extern "C" int viasd_debug_span_reset(void) {
@@ -574,8 +452,8 @@ size_t tc_scratch_floats(int sm_count, int nt, bool dual) { return (size_t)sm_co
 
 int tc_tiles(int n) { return (n + TILE_F - 1) / TILE_F; }
 
-int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {
-    TcParams p;
+// TcLaunch (host description) -> TcParams (kernel argument block), schedule fields left to the caller
+void tc_fill_params(const TcLaunch &L, TcParams &p) {
     memset(&p, 0, sizeof(p));
     const bool dual = L.epi == EPI_SWIGLU;
     p.nt = L.nt;
@@ -610,6 +488,12 @@ int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {
     p.split_row = L.split_row > 0 ? L.split_row : 0x7fffffff;
     p.out_f32_2 = L.out_f32_2; p.next_gain2 = L.next_gain2; p.kc2 = (__nv_bfloat16 *)L.kc2; p.vc2 = (__nv_bfloat16 *)L.vc2;
     p.layer_ord2 = L.layer_ord2;
+}
+
+int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {
+    TcParams p;
+    tc_fill_params(L, p);
+    const bool dual = L.epi == EPI_SWIGLU;
     const int units = p.n_tiles * p.k_tiles;
     if (units <= 0) return VIASD_OK;
     int ctas_per_sm = 1;

@@ -67,3 +67,5 @@ uint32_t tc_box_rows(uint64_t tensor_rows, uint32_t want);
 size_t tc_scratch_floats(int sm_count, int nt, bool dual);
 int tc_tiles(int n);
 int launch_gemm_tc(const TcLaunch &L, cudaStream_t st);
+void tc_fill_params(const TcLaunch &L, TcParams &p);
+

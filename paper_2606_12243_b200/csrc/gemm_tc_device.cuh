@@ -1,0 +1,254 @@
+// Device-side pieces shared by the tcgen05 GEMM kernels: PTX wrappers (mbarrier, TMA, tcgen05), the shared-memory
+// operand descriptor, the unit-range walk of the stream-K schedule and the fused epilogues.
+#pragma once
+#include "common.cuh"
+#include "gemm_tc.cuh"
+
+namespace {
+
+constexpr int TILE_F = 128;          // output features per tile (MMA M)
+constexpr int TILE_K = 64;           // bf16 per k-block: 128 bytes, one swizzle row
+constexpr int MAX_STAGES = 12;
+constexpr int THREADS = 192;
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about two seconds
+
+// ---- PTX wrappers ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the limit expired or another role of this CTA already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    int spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 255) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+                *abort_flag = 1;
+                atomicExch(status, VIASD_EDEVICE);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+
+// plain (untiled) bulk copy global -> shared; both addresses 16-byte aligned, size a multiple of 16 bytes
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+constexpr int CH = 8;                // token rows per epilogue chunk
+__device__ __forceinline__ void tc_ld8(uint32_t taddr, float (&v)[CH]) {
+    uint32_t r[8];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// K-major operand tile, 128-byte swizzle, rows 128 bytes apart, 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+    return (uint64_t)((addr >> 4) & 0x3FFF) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+
+#ifdef VIASD_TC_TRACE
+__device__ long long g_tc_trace[160 * 16];                // per CTA of the traced launch: globaltimer ns at 16 points
+#define TRACE(slot) do { if (p.trace_on) { unsigned long long t_; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_)); \
+                                           g_tc_trace[blockIdx.x * 16 + (slot)] = (long long)t_; } } while (0)
+#define TRACE_SM() do { if (p.trace_on) { unsigned sm_; asm volatile("mov.u32 %0, %smid;" : "=r"(sm_)); g_tc_trace[blockIdx.x * 16 + 12] = sm_; } } while (0)
+#define DBG(p, bit) ((p).dbg & (bit))
+__device__ unsigned long long g_tc_span[8192 * 2];       // per launch: earliest CTA start, latest CTA end (globaltimer ns)
+__device__ __forceinline__ unsigned long long gtimer() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define SPAN_BEGIN(p) do { if (threadIdx.x == 0) atomicMin(&g_tc_span[((p).launch_idx & 8191) * 2], gtimer()); } while (0)
+#define SPAN_END(p) do { if (threadIdx.x == 0) atomicMax(&g_tc_span[((p).launch_idx & 8191) * 2 + 1], gtimer()); } while (0)
+#else
+#define SPAN_BEGIN(p) do { } while (0)
+#define SPAN_END(p) do { } while (0)
+#define DBG(p, bit) 0
+#define TRACE(slot) do { } while (0)
+#define TRACE_SM() do { } while (0)
+#endif
+
+struct Seg { int tile, ka, kb; };      // one contiguous piece of this CTA's unit range inside a tile
+
+__device__ __forceinline__ bool next_seg(int &u, int u1, int k_tiles, Seg &s) {
+    if (u >= u1) return false;
+    s.tile = u / k_tiles;
+    s.ka = u - s.tile * k_tiles;
+    s.kb = min(k_tiles, s.ka + (u1 - u));
+    u += s.kb - s.ka;
+    return true;
+}
+
+// Epilogue for CH token rows r0..r0+CH-1 of one tile; thread f holds the full-K sums g (and u for the gate/up
+// pair) of output feature f.  Called by all 128 epilogue threads together.  The epilogue kind is a template
+// parameter so that each kernel carries one short epilogue: this code runs once per tile, straight from the
+// instruction cache's cold side, and its size is what its latency is made of.
+template <int EPI>
+__device__ __forceinline__ void finish_chunk(const TcParams &p, int tile, int f, int r0, float (&g)[CH], float (&uu)[CH],
+                                             float *xch, const float *inv_sh, const int4 *rowmeta, int lane,
+                                             const float *aux, int rows_live) {
+    // aux: null, or [rows][128] floats already in shared memory - the residual row of this tile (EPI_ADD_NORM),
+    // or the row's 64 cosines followed by its 64 sines (EPI_QKV_ROPE) - so that no chunk waits for global memory.
+    // rows_live: rows r0.. below it are written (p.rows, or 0 for the dry pass that only warms the instruction cache)
+    constexpr bool DUAL = EPI == EPI_SWIGLU;
+    if (EPI == EPI_STORE || EPI == EPI_SWIGLU || EPI == EPI_QKV_ROPE) {
+        if (p.ssq_in) {                   // the input was h * gain without its RMS factor: apply it per row here
+#pragma unroll
+            for (int j = 0; j < CH; ++j) {
+                const float sc = inv_sh[min(r0 + j, 127)];
+                g[j] *= sc;
+                if (DUAL) uu[j] *= sc;
+            }
+        }
+    }
+    const int nrow = min(CH, rows_live - r0);
+    if (DUAL) {
+        const int n = tile * TILE_F + f;
+        if (n >= p.seg_n[0]) return;
+        __nv_bfloat16 *dst = p.out_act + (size_t)(p.row0 + r0) * p.ld_out + n;
+#pragma unroll
+        for (int j = 0; j < CH; ++j) {
+            if (j < nrow) {
+                const float sg = g[j] / (1.f + __expf(-g[j]));
+                store_act<__nv_bfloat16>(dst, p.act_plane, (size_t)j * p.ld_out, sg * uu[j]);
+            }
+        }
+        return;
+    }
+    int s = 0, t0 = 0, nbase = 0;
+    while (s < 2 && tile >= p.seg_tile_end[s]) { t0 = p.seg_tile_end[s]; nbase += p.seg_n[s]; ++s; }
+    const int nin = (tile - t0) * TILE_F + f;
+    const bool valid = nin < p.seg_n[s];
+    const int n = nbase + nin;
+    if (EPI == EPI_STORE) {
+        if (!valid) return;
+#pragma unroll
+        for (int j = 0; j < CH; ++j) {
+            if (j < nrow) {
+                const int row = p.row0 + r0 + j;          // the second stream's rows go to the second output
+                float *dst = row < p.split_row ? p.out_f32 + (size_t)row * p.ld_out + n
+                                               : p.out_f32_2 + (size_t)(row - p.split_row) * p.ld_out + n;
+                if (p.epi == EPI_ADD) *dst += g[j]; else *dst = g[j];
+            }
+        }
+    } else if (EPI == EPI_ADD_NORM) {
+        // residual update, plus what the next RMSNorm needs: h * gain as hi/lo planes and partial sums of h^2.
+        // Loads first, then arithmetic, then stores: the CH rows cost one memory round trip.
+        const float gain_a = valid ? p.next_gain[n] : 0.f;
+        const float gain_b = (valid && p.next_gain2) ? p.next_gain2[n] : gain_a;
+        float *hp = p.out_f32 + (size_t)(p.row0 + r0) * p.ld_out + n;
+        __nv_bfloat16 *ap = p.next_act + (size_t)(p.row0 + r0) * p.ld_out + n;
+        float v[CH];
+#ifdef VIASD_TC_TRACE
+        asm volatile("" :: "f"(gain_a), "f"(gain_b));
+        if (f == 0 && r0 == 0) TRACE(2);
+#endif
+#pragma unroll
+        for (int j = 0; j < CH; ++j)
+            v[j] = (valid && j < nrow) ? (aux ? aux[(r0 + j) * TILE_F + f] : __ldcg(hp + (size_t)j * p.ld_out)) + g[j] : 0.f;
+#ifdef VIASD_TC_TRACE
+        asm volatile("" :: "f"(v[0]), "f"(v[7]));
+        if (f == 0 && r0 == 0) TRACE(3);
+#endif
+#pragma unroll
+        for (int j = 0; j < CH; ++j) {
+            if (valid && j < nrow) {
+                hp[(size_t)j * p.ld_out] = v[j];
+                store_act<__nv_bfloat16>(ap, p.next_plane, (size_t)j * p.ld_out,
+                                         v[j] * (p.row0 + r0 + j < p.split_row ? gain_a : gain_b));
+            }
+            v[j] *= v[j];
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+            for (int j = 0; j < CH; ++j) v[j] += __shfl_xor_sync(0xffffffffu, v[j], o);
+        if (lane < nrow) {
+            float mine = v[0];
+#pragma unroll
+            for (int j = 1; j < CH; ++j) mine = lane == j ? v[j] : mine;
+            p.ssq_out[((size_t)tile * 4 + (f >> 5)) * p.ssq_stride + p.row0 + r0 + lane] = mine;
+        }
+    } else {   // EPI_QKV_ROPE: one tile is one head of 128 dims; rotate pairs (p, p + 64), write q / K cache / V cache
+#pragma unroll
+        for (int j = 0; j < CH; ++j) xch[j * TILE_F + f] = g[j];
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        const int head = tile - t0, pidx = f & 63;
+        if (s < 2) {
+            float c[CH], sn[CH];
+#pragma unroll
+            for (int j = 0; j < CH; ++j) {
+                const int pos = rowmeta[min(r0 + j, 127)].x;
+                const float *ar = aux + min(r0 + j, p.rows - 1) * TILE_F + pidx;
+                c[j] = aux ? ar[0] : p.cosv[(size_t)pos * 64 + pidx];
+                sn[j] = aux ? ar[64] : p.sinv[(size_t)pos * 64 + pidx];
+            }
+#pragma unroll
+            for (int j = 0; j < CH; ++j) {
+                const float other = xch[j * TILE_F + (f ^ 64)];
+                g[j] = f < 64 ? g[j] * c[j] - other * sn[j] : g[j] * c[j] + other * sn[j];
+            }
+        }
+        if (s == 0) {
+            float *dst = p.q_out + ((size_t)(p.row0 + r0) * p.rope_H + head) * TILE_F + f;
+#pragma unroll
+            for (int j = 0; j < CH; ++j) if (j < nrow) dst[(size_t)j * p.rope_H * TILE_F] = g[j];
+        } else {
+#pragma unroll
+            for (int j = 0; j < CH; ++j) {
+                if (j < nrow) {
+                    const int4 rm = rowmeta[r0 + j];
+                    __nv_bfloat16 *cache = rm.w ? (s == 1 ? p.kc2 : p.vc2) : (s == 1 ? p.kc : p.vc);
+                    const int lo = rm.w ? p.layer_ord2 : p.layer_ord;
+                    cache[((((size_t)lo * p.max_batch + rm.z) * p.rope_Hkv + head) * p.max_ctx + rm.y) * TILE_F + f] =
+                        __float2bfloat16_rn(g[j]);
+                }
+            }
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+    }
+}
+
+}  // namespace
