@@ -81,7 +81,7 @@ typedef struct {
     const int *draft_tok;              /* [B, N] */
     const int *parent;                 /* [N] parent node, -1 = child of the pending token; parents first */
     const int *prow;                   /* [N] drafter-logit row the node was drafted from */
-    int n_prows;                       /* R */
+    int n_prows;                       /* R, 1..64 (one drafter row per distinct parent at most) */
     const float *drafter_logits;       /* [B, R, vocab] */
 } viasd_draft;
 

@@ -56,7 +56,7 @@ size_t carve(const viasd_config &c, char *base, Workspace *ws) {
     w.row_tok = cv.take<int>(R * 4);
     w.tree = cv.take<TreeInfo>(sizeof(TreeInfo));
     w.stats = cv.take<DeviceStats>(sizeof(DeviceStats));
-    w.accept_scratch = cv.take<float>((size_t)c.max_batch * 3 * c.vocab * 4);
+    w.accept_scratch = cv.take<float>(((size_t)c.max_batch * 3 * c.vocab + (size_t)c.max_batch * 9 * VIASD_MAX_ROWS_PER_SEQ) * 4);
     {
         const int nt = tc_pick_nt(R < 128 ? (int)R : 128);
         w.gemm_scratch = cv.take<float>(tc_scratch_floats(MAX_GEMM_CTAS, nt, true) * 4);

@@ -47,7 +47,7 @@ struct Workspace {                      // pointers into the caller's workspace 
     int *row_tok;                       // [R] token id per row
     TreeInfo *tree;
     DeviceStats *stats;
-    float *accept_scratch;              // [B, 3, V] sampling-mode distributions
+    float *accept_scratch;              // [B, 3, V] sampling-mode distributions, then [3][B, 3, 64] row statistics
     float *gemm_scratch;                // partial tiles of split GEMM work (tcgen05 kernel)
     int *gemm_counters;                 // per-tile arrival counters, zero between launches
     size_t n_counters;

@@ -507,7 +507,9 @@ int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {
     const size_t stage = (size_t)nacc * TILE_F * TILE_K * 2 + 2 * (size_t)L.nt * TILE_K * 2;
     // a ring of about 100 KB keeps HBM busy (deeper rings measured no faster) and lets the CTA of the next
     // kernel in the stream become resident beside this one, so that its weight prefetch overlaps this tail
-    int stages = (int)((size_t)104 * 1024 / stage);
+    static int ring_kb = -1;
+    if (ring_kb < 0) { const char *e = getenv("VIASD_TC_RING_KB"); ring_kb = e ? atoi(e) : 200; }
+    int stages = (int)((size_t)ring_kb * 1024 / stage);
     if (stages < 2) stages = 2;
     if (stages > MAX_STAGES) stages = MAX_STAGES;
 #ifdef VIASD_TC_TRACE

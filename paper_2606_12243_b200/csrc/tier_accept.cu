@@ -8,8 +8,10 @@
 // one CTA per sequence walks the draft from the pending token: children of the current row are tried in
 // index order; tier-0 children are taken at once, tier-1 children are judged by q', tier-2 children by
 // q.  The first row where no child passes ends the walk and the strongest judge that rejected there
-// emits the replacement token.  The walk is sequential over depth; every test is a reduction over the
-// vocabulary done by the whole CTA.
+// emits the replacement token.  The walk is sequential over depth, so everything that can be known before
+// it is: a row-statistics kernel (one CTA per logits row, all rows at once) leaves each row's maximum,
+// argmax and softmax denominator, which makes every first test at a position O(1).  Only a rejection in
+// sampling mode (residual, Eq. A.3) and the final draw still sweep the vocabulary inside the walk.
 #include "common.cuh"
 
 namespace {
@@ -113,8 +115,64 @@ tier_kernel(unsigned char *__restrict__ tier, float *__restrict__ conf, DeviceSt
     if (gr == 0 && b == 0 && threadIdx.x == 0) atomicAdd(&stats->steps, 1ull);
 }
 
+// ---- row statistics ---------------------------------------------------------------------------
+// grid (rows, B, 3): kind 0 = drafter rows [B, R, V], 1 = slim [B, M, V], 2 = full [B, M, V].
+// Per row: max, argmax (lowest index on ties) and, when want_z, sum exp((l - max) / T).
+constexpr int RS_STRIDE = VIASD_MAX_ROWS_PER_SEQ;
+struct RowStats { float *mx; int *arg; float *z; };       // each [B, 3, RS_STRIDE]
+
+__global__ void __launch_bounds__(512)
+row_stats_kernel(RowStats rs, const float *__restrict__ drafter, const float *__restrict__ slim,
+                 const float *__restrict__ full, int R, int M, int V, float inv_temp, int want_z) {
+    __shared__ float sh[32];
+    __shared__ MaxIdx shm[32];
+    const int kind = blockIdx.z, b = blockIdx.y, r = blockIdx.x;
+    const float *base = kind == 0 ? drafter : (kind == 1 ? slim : full);
+    const int rows = kind == 0 ? R : M;
+    if (!base || r >= rows) return;
+    const float *row = base + ((size_t)b * rows + r) * V;
+    const bool vec = (V & 3) == 0 && ((uintptr_t)row & 15) == 0;
+    MaxIdx best; best.v = -INFINITY; best.i = 0x7fffffff;
+    if (vec) {
+        const float4 *r4 = reinterpret_cast<const float4 *>(row);
+        for (int i = threadIdx.x; i < V / 4; i += blockDim.x) {
+            const float4 v = r4[i];
+            MaxIdx c;
+            c.v = v.x; c.i = 4 * i; best = better(best, c);
+            c.v = v.y; c.i = 4 * i + 1; best = better(best, c);
+            c.v = v.z; c.i = 4 * i + 2; best = better(best, c);
+            c.v = v.w; c.i = 4 * i + 3; best = better(best, c);
+        }
+    } else {
+        for (int i = threadIdx.x; i < V; i += blockDim.x) { MaxIdx c; c.v = row[i]; c.i = i; best = better(best, c); }
+    }
+    best = block_argmax(best, shm);
+    float z = 0.f;
+    if (want_z) {
+        const float mx = best.v;
+        if (vec) {
+            const float4 *r4 = reinterpret_cast<const float4 *>(row);
+            for (int i = threadIdx.x; i < V / 4; i += blockDim.x) {
+                const float4 v = r4[i];
+                z += expf((v.x - mx) * inv_temp) + expf((v.y - mx) * inv_temp) + expf((v.z - mx) * inv_temp) +
+                     expf((v.w - mx) * inv_temp);
+            }
+        } else {
+            for (int i = threadIdx.x; i < V; i += blockDim.x) z += expf((row[i] - mx) * inv_temp);
+        }
+        z = block_sum(z, sh);
+    }
+    if (threadIdx.x == 0) {
+        const size_t o = ((size_t)b * 3 + kind) * RS_STRIDE + r;
+        rs.mx[o] = best.v;
+        rs.arg[o] = best.i == 0x7fffffff ? 0 : best.i;
+        rs.z[o] = z;
+    }
+}
+
 // ---- accept kernel ----------------------------------------------------------------------------
 struct AcceptArgs {
+    RowStats rs;
     const float *slim, *full, *drafter;      // [B, M, V], [B, M, V], [B, R, V]
     const int *draft_tok, *prow;             // [B, N], [N]
     const unsigned char *tier;               // [B, N]
@@ -130,18 +188,10 @@ struct AcceptArgs {
     unsigned long long seed, step;
 };
 
-// numerators of softmax(l / T) into dst, returns their sum
-__device__ float softmax_numerators(float *dst, const float *row, int V, float inv_temp, float *sh) {
-    float mx = -INFINITY;
-    for (int i = threadIdx.x; i < V; i += blockDim.x) mx = fmaxf(mx, row[i]);
-    mx = block_max(mx, sh);
-    float s = 0.f;
-    for (int i = threadIdx.x; i < V; i += blockDim.x) {
-        float e = expf((row[i] - mx) * inv_temp);
-        dst[i] = e;
-        s += e;
-    }
-    return block_sum(s, sh);
+// numerators of softmax(l / T) into dst (the row maximum comes from the row statistics)
+__device__ void softmax_numerators(float *dst, const float *row, int V, float inv_temp, float mx) {
+    for (int i = threadIdx.x; i < V; i += blockDim.x) dst[i] = expf((row[i] - mx) * inv_temp);
+    __syncthreads();
 }
 
 // argmax_v (log w[v] - log(-log u_v)): a draw from w / sum(w)
@@ -159,22 +209,17 @@ __device__ int gumbel_argmax(const float *w, int V, unsigned long long key, int 
     return best.i == 0x7fffffff ? 0 : best.i;
 }
 
-__device__ int row_argmax(const float *row, int V, MaxIdx *shm) {
-    MaxIdx best; best.v = -INFINITY; best.i = 0x7fffffff;
-    for (int i = threadIdx.x; i < V; i += blockDim.x) { MaxIdx c; c.v = row[i]; c.i = i; best = better(best, c); }
-    best = block_argmax(best, shm);
-    return best.i == 0x7fffffff ? 0 : best.i;
-}
-
 __global__ void __launch_bounds__(ACC_THREADS)
 accept_kernel(AcceptArgs a) {
-    __shared__ float sh[32];
     __shared__ MaxIdx shm[32];
+    __shared__ float sh[32];
     const int b = blockIdx.x, N = a.N, M = N + 1, V = a.V;
     const TreeInfo *tree = a.tree;
     const bool sampling = a.mode == 1;
     float *P[3] = {a.scratch + ((size_t)b * 3 + 0) * V, a.scratch + ((size_t)b * 3 + 1) * V,
                    a.scratch + ((size_t)b * 3 + 2) * V};
+    const float *st_mx = a.rs.mx + (size_t)b * 3 * RS_STRIDE, *st_z = a.rs.z + (size_t)b * 3 * RS_STRIDE;
+    const int *st_arg = a.rs.arg + (size_t)b * 3 * RS_STRIDE;
     const unsigned long long k_acc = stream_key(a.seed, a.step, b, 0), k_gum = stream_key(a.seed, a.step, b, 1);
     for (int n = threadIdx.x; n < N; n += blockDim.x) a.judge[b * N + n] = 0;
     __syncthreads();
@@ -182,23 +227,24 @@ accept_kernel(AcceptArgs a) {
     int cur = 0, n_acc = 0, corr = -1, corr_src = 0;
     while (true) {
         int c = tree->first_child[cur];
-        const float *Lrow[3] = {nullptr, a.slim + ((size_t)b * M + cur) * V, a.full + ((size_t)b * M + cur) * V};
         if (c < 0) {                                             // leaf: whole path accepted
             if (a.emit_bonus) {
                 if (sampling) {
-                    softmax_numerators(P[2], Lrow[2], V, a.inv_temp, sh);
-                    __syncthreads();
+                    softmax_numerators(P[2], a.full + ((size_t)b * M + cur) * V, V, a.inv_temp, st_mx[2 * RS_STRIDE + cur]);
                     corr = gumbel_argmax(P[2], V, k_gum, cur, shm);
                 } else {
-                    corr = row_argmax(Lrow[2], V, shm);
+                    corr = st_arg[2 * RS_STRIDE + cur];
                 }
                 corr_src = 2;
             }
             break;
         }
-        float Z[3] = {0.f, 0.f, 0.f};
-        bool have[3] = {false, false, false};
-        float rowmax[3] = {0.f, 0.f, 0.f};
+        // the three distributions of this position: 0 = proposal (drafter row), 1 = q', 2 = q.  Each starts as
+        // "row + statistics" and is written out as numerators (mat) only once a residual has to be formed.
+        const float *row[3] = {nullptr, a.slim + ((size_t)b * M + cur) * V, a.full + ((size_t)b * M + cur) * V};
+        float mx[3] = {0.f, st_mx[1 * RS_STRIDE + cur], st_mx[2 * RS_STRIDE + cur]};
+        float Z[3] = {0.f, st_z[1 * RS_STRIDE + cur], st_z[2 * RS_STRIDE + cur]};
+        bool mat[3] = {false, false, false};
         int failed = 0, taken = -1, taken_tier = 0;
         for (; c >= 0; c = tree->next_sibling[c]) {
             const int t = a.tier[b * N + c];
@@ -211,27 +257,19 @@ accept_kernel(AcceptArgs a) {
             }
             bool pass;
             if (!sampling) {
-                if (!have[t]) {
-                    float mx = -INFINITY;
-                    for (int i = threadIdx.x; i < V; i += blockDim.x) mx = fmaxf(mx, Lrow[t][i]);
-                    rowmax[t] = block_max(mx, sh);
-                    have[t] = true;
-                }
-                pass = (Lrow[t][v] - rowmax[t]) >= a.log_acc_rel[t];
+                pass = (row[t][v] - mx[t]) >= a.log_acc_rel[t];
             } else {
-                if (!have[0]) {
-                    const float *prow_logits = a.drafter + ((size_t)b * a.R + a.prow[c]) * V;
-                    Z[0] = softmax_numerators(P[0], prow_logits, V, a.inv_temp, sh);
-                    have[0] = true;
+                if (!row[0]) {
+                    const int pr = a.prow[c];
+                    row[0] = a.drafter + ((size_t)b * a.R + pr) * V;
+                    mx[0] = st_mx[pr];
+                    Z[0] = st_z[pr];
                 }
-                if (!have[t]) {
-                    Z[t] = softmax_numerators(P[t], Lrow[t], V, a.inv_temp, sh);
-                    have[t] = true;
-                }
-                __syncthreads();
                 const float u = unit_f32(k_acc, (unsigned long long)c);
-                const float lp = logf(P[0][v] / Z[0]);
-                const float lj = logf(P[t][v] / Z[t]);
+                const float pv = mat[0] ? P[0][v] : expf((row[0][v] - mx[0]) * a.inv_temp);
+                const float jv = mat[t] ? P[t][v] : expf((row[t][v] - mx[t]) * a.inv_temp);
+                const float lp = logf(pv / Z[0]);
+                const float lj = logf(jv / Z[t]);
                 pass = (logf(u) + a.log1m_alpha + lp) < lj;       // u < j(v) / ((1 - alpha) p(v)), Eq. A.2
             }
             if (pass) {
@@ -244,6 +282,9 @@ accept_kernel(AcceptArgs a) {
             if (sampling) {
                 // Eq. A.3 round by round: the rejecting judge becomes its residual against the proposal
                 // (kept as is if the residual vanishes); the rejected token leaves the proposal.
+                __syncthreads();                                  // every thread has read P[.][v] above
+                if (!mat[t]) { softmax_numerators(P[t], row[t], V, a.inv_temp, mx[t]); mat[t] = true; }
+                if (!mat[0]) { softmax_numerators(P[0], row[0], V, a.inv_temp, mx[0]); mat[0] = true; }
                 const float sj = a.inv_beta / Z[t], sp = 1.f / Z[0];
                 float s = 0.f;
                 for (int i = threadIdx.x; i < V; i += blockDim.x) s += fmaxf(0.f, P[t][i] * sj - P[0][i] * sp);
@@ -277,7 +318,7 @@ accept_kernel(AcceptArgs a) {
             __syncthreads();
             corr = gumbel_argmax(P[failed], V, k_gum, cur, shm);
         } else {
-            corr = row_argmax(Lrow[failed], V, shm);
+            corr = st_arg[failed * RS_STRIDE + cur];
         }
         break;
     }
@@ -338,7 +379,18 @@ int launch_accept(const viasd_model *m, const viasd_draft *d, const viasd_params
                   const float *full_logits, viasd_result *r, cudaStream_t st) {
     tree_only_kernel<<<1, 32, 0, st>>>(m->ws.tree, m->ws.stats, d->parent, d->n_nodes);
     LAUNCH_CHECK();
+    if (d->n_prows > RS_STRIDE) return VIASD_EINVAL;
     AcceptArgs a;
+    {
+        // row statistics live behind the three distribution buffers
+        float *base = m->ws.accept_scratch + (size_t)m->cfg.max_batch * 3 * m->cfg.vocab;
+        const size_t n = (size_t)m->cfg.max_batch * 3 * RS_STRIDE;
+        a.rs.mx = base; a.rs.arg = reinterpret_cast<int *>(base + n); a.rs.z = base + 2 * n;
+        const int M = d->n_nodes + 1, rows = M > d->n_prows ? M : d->n_prows;
+        row_stats_kernel<<<dim3(rows, d->batch, 3), 512, 0, st>>>(a.rs, p->mode == 1 ? d->drafter_logits : nullptr, slim_logits,
+            full_logits, d->n_prows, M, m->cfg.vocab, 1.0f / p->temperature, p->mode == 1);
+        LAUNCH_CHECK();
+    }
     a.slim = slim_logits; a.full = full_logits; a.drafter = d->drafter_logits;
     a.draft_tok = d->draft_tok; a.prow = d->prow; a.tier = r->tier; a.tree = m->ws.tree;
     a.scratch = m->ws.accept_scratch;
