@@ -193,7 +193,7 @@ static int mma_attention(viasd_model *m, const void *kc, const void *vc, bool sl
     const viasd_config &c = m->cfg;
     const int nsplit = mma_nsplit(m, batch, M, streams);
     const int QR = (c.n_heads / c.n_kv_heads) * M;
-    const bool fuse = nsplit > 1 && QR * nsplit <= 160;
+    const bool fuse = nsplit > 1 && nsplit <= 32 && QR * nsplit <= 160;
     int rc = launch_attention_mma(m, kc, vc, slim, layer_ord, kc2, vc2, layer_ord2, streams, batch, M, nsplit, fuse ? 1 : 0, st);
     if (rc || nsplit == 1 || fuse) return rc;
     attention_combine_kernel<__nv_bfloat16, 128><<<dim3(streams * batch * M, c.n_heads), 128, 0, st>>>(

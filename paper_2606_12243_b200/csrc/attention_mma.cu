@@ -21,6 +21,7 @@
 // bounded.
 #include "common.cuh"
 #include <stdlib.h>
+#include <stdio.h>
 
 namespace {
 
@@ -100,6 +101,7 @@ struct AttnArgs {
     int streams, n_items, items_per_cta, fuse_merge, nstage, mt_eff;
     int *counters;              // [streams * batch * Hkv] arrivals per (sequence, kv head), zero between launches
     float scale;
+    int trace_on;               // trace builds only
 };
 
 __device__ __forceinline__ float ex2(float x) {            // 2^x, hardware approximation (2 ulp)
@@ -233,6 +235,14 @@ __device__ __forceinline__ Item decode_item(const AttnArgs &a, int item) {
     return it;
 }
 
+#ifdef VIASD_TC_TRACE
+__device__ long long g_at_trace[160 * 16];
+#define ATRACE(slot) do { if (a.trace_on && threadIdx.x == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_)); \
+                                             g_at_trace[blockIdx.x * 16 + (slot)] = (long long)t_; } } while (0)
+#else
+#define ATRACE(slot) do { } while (0)
+#endif
+
 // PLO / QLO: use the lo parts of the probabilities / of the query too
 template <bool PLO, bool QLO>
 __global__ void __launch_bounds__(WARPS * 32)
@@ -243,6 +253,10 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
     __shared__ int last_sh;
     constexpr int ROWF = HD + 2;
     PDL_TRIGGER();
+    ATRACE(0);
+#ifdef VIASD_TC_TRACE
+    if (a.trace_on && threadIdx.x == 0) { g_at_trace[blockIdx.x * 16 + 10] = 0; g_at_trace[blockIdx.x * 16 + 11] = 0; }
+#endif
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int NSTAGE = a.nstage;
     const int grp = a.H / a.Hkv, QR = grp * a.M, QRP = a.mt * 16;
@@ -286,7 +300,9 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
         // committed context does not change during the pass: ask for it before waiting for the previous kernel
         while (p_count < NSTAGE && issue_next(true)) { }
     }
+    ATRACE(1);
     PDL_WAIT();
+    ATRACE(2);
     if (threadIdx.x == 0) while (p_count < NSTAGE && issue_next(false)) { }
 
     uint32_t qh[8][4], ql[8][4];                             // this warp's query tile, hi and lo, as MMA A fragments
@@ -298,22 +314,32 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
         if (it.be != q_be || it.g != q_g) {
             // stage the query rows of this (sequence, kv head) as bf16 hi / lo, pre-scaled
             __syncthreads();
-            for (int idx = threadIdx.x; idx < QRP * (HD / 2); idx += blockDim.x) {
-                const int row = idx / (HD / 2), d2 = (idx % (HD / 2)) * 2;
-                float x0 = 0.f, x1 = 0.f;
-                if (row < QR) {
-                    const int h = it.g * grp + row / a.M, i = row % a.M;
-                    const float2 v = *reinterpret_cast<const float2 *>(a.q + ((size_t)(it.be * a.M + i) * a.H + h) * HD + d2);
-                    x0 = v.x * a.scale; x1 = v.y * a.scale;
+            // four elements per thread at a time, loads first: the staging costs one memory round trip per batch
+            for (int idx0 = threadIdx.x; idx0 < QRP * (HD / 2); idx0 += 4 * blockDim.x) {
+                float2 v[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int idx = idx0 + q * blockDim.x, row = idx / (HD / 2), d2 = (idx % (HD / 2)) * 2;
+                    v[q] = make_float2(0.f, 0.f);
+                    if (idx < QRP * (HD / 2) && row < QR) {
+                        const int h = it.g * grp + row / a.M, i = row % a.M;
+                        v[q] = __ldcg(reinterpret_cast<const float2 *>(a.q + ((size_t)(it.be * a.M + i) * a.H + h) * HD + d2));
+                    }
                 }
-                uint32_t hi, lo;
-                split2(x0, x1, hi, lo);
-                const uint32_t off = qoff(row, d2 >> 3) + (d2 & 7) * 2;
-                *reinterpret_cast<uint32_t *>(gen_base + (qhi - base) + off) = hi;
-                *reinterpret_cast<uint32_t *>(gen_base + (qlo - base) + off) = lo;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int idx = idx0 + q * blockDim.x, row = idx / (HD / 2), d2 = (idx % (HD / 2)) * 2;
+                    if (idx >= QRP * (HD / 2)) continue;
+                    uint32_t hi, lo;
+                    split2(v[q].x * a.scale, v[q].y * a.scale, hi, lo);
+                    const uint32_t off = qoff(row, d2 >> 3) + (d2 & 7) * 2;
+                    *reinterpret_cast<uint32_t *>(gen_base + (qhi - base) + off) = hi;
+                    *reinterpret_cast<uint32_t *>(gen_base + (qlo - base) + off) = lo;
+                }
             }
             __syncthreads();
             q_be = it.be; q_g = it.g;
+            if (item == i0) ATRACE(3);
             if (active) {
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
@@ -337,8 +363,16 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
 
         for (int tile = 0; tile < it.n_tiles; ++tile, ++c_count) {
             const int st = c_count % NSTAGE;
+#ifdef VIASD_TC_TRACE
+            unsigned long long tw0_ = 0; if (a.trace_on && threadIdx.x == 0) asm volatile("mov.u64 %0, %globaltimer;" : "=l"(tw0_));
+#endif
             ok = mbar_wait(smem_u32(&bars[st]), (c_count / NSTAGE) & 1, a.status);
+#ifdef VIASD_TC_TRACE
+            if (a.trace_on && threadIdx.x == 0) { unsigned long long tw1_; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(tw1_));
+                g_at_trace[blockIdx.x * 16 + 10] += (long long)(tw1_ - tw0_); g_at_trace[blockIdx.x * 16 + 11] += 1; }
+#endif
             if (!__syncthreads_and(ok)) { ok = false; break; }   // leave together if any thread gave up
+            if (item == i0 && tile == 0) ATRACE(4);
             const uint32_t kst = base + st * STAGE_BYTES, vst = kst + 2 * HALF_BYTES;
             const int j0 = it.k_begin + tile * TKEYS;
             if (active) {
@@ -366,6 +400,7 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             if (threadIdx.x == 0) issue_next(false);
         }
         if (!ok) break;
+        if (item == i0) ATRACE(5);
 
         // ---- end of the item: merge the key groups of each query tile pairwise, in registers ----
         // (the fragment layouts match lane for lane, so the exchange buffer is just each lane's values)
@@ -405,6 +440,7 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             }
         }
         const bool single = a.nsplit == 1;
+        if (item == i0) ATRACE(6);
         if (active && kgroup == 0) {
             // this warp now holds its query tile for the whole key range: write it from registers
 #pragma unroll
@@ -440,24 +476,34 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
                 if (last_sh) a.counters[it.be * a.Hkv + it.g] = 0;
             }
             __syncthreads();
+            if (item == i0) ATRACE(7);
             if (last_sh) {
                 __threadfence();
                 for (int row = warp; row < QR; row += WARPS) {
                     const int h = it.g * grp + row / a.M, i = row % a.M;
                     const float *src = a.part + (((size_t)it.be * a.H + h) * a.M + i) * (size_t)a.nsplit * ROWF;
-                    float mmax = -INFINITY;
-                    for (int s2 = 0; s2 < a.nsplit; ++s2) mmax = fmaxf(mmax, __ldcg(src + (size_t)s2 * ROWF + HD));
-                    float den = 0.f, num[HD / 32];
+                    // lane s holds range s's (max, sum); the weights go round by shuffle (nsplit <= 32 when fused)
+                    float ms = -INFINITY, ls = 0.f;
+                    if (lane < a.nsplit) { ms = __ldcg(src + (size_t)lane * ROWF + HD); ls = __ldcg(src + (size_t)lane * ROWF + HD + 1); }
+                    float num[HD / 32];
 #pragma unroll
                     for (int e = 0; e < HD / 32; ++e) num[e] = 0.f;
-                    for (int s2 = 0; s2 < a.nsplit; ++s2) {
-                        const float *p = src + (size_t)s2 * ROWF;
-                        const float ms = __ldcg(p + HD);
-                        if (ms == -INFINITY) continue;
-                        const float w = expf(ms - mmax);
-                        den = fmaf(__ldcg(p + HD + 1), w, den);
+                    const float mmax = warp_max(ms);
+                    const float w = (ms == -INFINITY) ? 0.f : expf(ms - mmax);
+                    const float den = warp_sum(ls * w);
+                    for (int s0 = 0; s0 < a.nsplit; s0 += 4) {
+                        float v[4][HD / 32];
 #pragma unroll
-                        for (int e = 0; e < HD / 32; ++e) num[e] = fmaf(__ldcg(p + lane + 32 * e), w, num[e]);
+                        for (int q = 0; q < 4; ++q)
+#pragma unroll
+                            for (int e = 0; e < HD / 32; ++e)
+                                v[q][e] = s0 + q < a.nsplit ? __ldcg(src + (size_t)(s0 + q) * ROWF + lane + 32 * e) : 0.f;
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const float wq = __shfl_sync(0xffffffffu, w, (s0 + q) & 31);
+#pragma unroll
+                            for (int e = 0; e < HD / 32; ++e) num[e] = fmaf(v[q][e], s0 + q < a.nsplit ? wq : 0.f, num[e]);
+                        }
                     }
                     const float inv = 1.f / den;
 #pragma unroll
@@ -468,7 +514,9 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             }
             __syncthreads();
         }
+        ATRACE(8);
     }
+    ATRACE(9);
 }
 
 }  // namespace
@@ -507,6 +555,7 @@ int launch_attention_mma(viasd_model *m, const void *kc, const void *vc, bool sl
     const int grp = c.n_heads / c.n_kv_heads, mt = (grp * M + 15) / 16;
     const int mt_eff = mt <= 1 ? 1 : mt <= 2 ? 2 : mt <= 4 ? 4 : 8;
     AttnArgs a;
+    a.trace_on = 0;
     a.q = m->ws.q; a.part = m->ws.part; a.out = (__nv_bfloat16 *)m->ws.attn;
     a.out_plane = m->ws.rows_alloc * (size_t)c.n_heads * HD;
     a.len_eff = m->ws.len_eff; a.tree = m->ws.tree; a.status = &m->ws.stats->device_status;
@@ -516,6 +565,15 @@ int launch_attention_mma(viasd_model *m, const void *kc, const void *vc, bool sl
     a.counters = m->ws.attn_counters;
     a.fuse_merge = fuse_merge;
     a.mt_eff = mt_eff;
+#ifdef VIASD_TC_TRACE
+    {
+        static int n_launch = 0;
+        const char *e = getenv("VIASD_AT_TRACE_IDX");
+        a.trace_on = e && atoi(e) == n_launch ? 1 : 0;
+        if (a.trace_on) fprintf(stderr, "attention trace: nsplit %d fuse %d streams %d mt %d\n", nsplit, fuse_merge, streams, mt);
+        if (e && atoi(e) < 0) n_launch = 0; else ++n_launch;
+    }
+#endif
     a.n_items = streams * batch * c.n_kv_heads * nsplit;
     int grid = a.n_items < m->sm_count ? a.n_items : m->sm_count;
     a.items_per_cta = (a.n_items + grid - 1) / grid;
@@ -543,3 +601,9 @@ int launch_attention_mma(viasd_model *m, const void *kc, const void *vc, bool sl
     LAUNCH_CHECK();
     return VIASD_OK;
 }
+
+#ifdef VIASD_TC_TRACE
+extern "C" int viasd_debug_attn_trace(long long *host_out) {
+    return (int)cudaMemcpyFromSymbol(host_out, g_at_trace, sizeof(long long) * 160 * 16);
+}
+#endif
