@@ -4,6 +4,8 @@
 // query rows), keeps an online softmax per query row and writes unnormalised partials; a second
 // kernel merges the key ranges.
 #include "common.cuh"
+#include <string.h>
+#include <stdlib.h>
 
 namespace {
 
@@ -167,22 +169,24 @@ int attention_nsplit(const viasd_model *m, int batch, int M) {
 // CTAs in equal contiguous shares, each item costs a fixed part (query staging, merge, partial) plus its tiles,
 // and every extra range adds merge work.  Depends on batch, heads and M only, so the one-stream and the two-stream
 // launch cut the keys at the same places and produce the same bits.
-static int mma_nsplit(const viasd_model *m, int batch, int M, int streams) {
+static int mma_nsplit(const viasd_model *m, int batch, int M, int streams, bool tc, int reps) {
     const viasd_config &c = m->cfg;
     const int base = batch * c.n_kv_heads, sms = m->sm_count;
     const int mt = ((c.n_heads / c.n_kv_heads) * M + 15) / 16;
     const int tiles = (c.max_ctx + 127) / 128;
-    int max_s = tiles < 16 ? tiles : 16;
-    const double t_tile = 0.5 + 0.8 * mt, t_item = 3.0;
+    int max_s = tiles < 16 / reps ? tiles : 16 / reps;          // the partial buffer holds 16 ranges per (row, head)
+    if (max_s < 1) max_s = 1;
+    // microseconds, roughly: the tcgen05 kernel's tile does not depend on the number of query tiles
+    const double t_tile = tc ? 0.7 : 0.5 + 0.8 * mt, t_item = tc ? 4.0 : 3.0;
     int best = 1;
     double best_cost = 1e30;
     for (int s = 1; s <= max_s; ++s) {
         const int n = base * s, ipc = (n + sms - 1) / sms;
         const int tpi = ((tiles + s - 1) / s);
-        const double cost = ipc * (tpi * t_tile + t_item) + 0.15 * s;
+        const double cost = ipc * (tpi * t_tile + t_item) + 0.15 * s * reps;
         if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
     }
-    size_t per_split = (size_t)streams * batch * c.n_heads * M * (c.head_dim + 2) * sizeof(float);
+    size_t per_split = (size_t)streams * batch * c.n_heads * M * (c.head_dim + 2) * sizeof(float) * reps;
     while (best > 1 && per_split * best > m->ws.part_bytes) --best;
     return best;
 }
@@ -191,13 +195,18 @@ static int mma_nsplit(const viasd_model *m, int batch, int M, int streams) {
 static int mma_attention(viasd_model *m, const void *kc, const void *vc, bool slim, int layer_ord, const void *kc2,
                          const void *vc2, int layer_ord2, int streams, int batch, int M, cudaStream_t st) {
     const viasd_config &c = m->cfg;
-    const int nsplit = mma_nsplit(m, batch, M, streams);
+    static int use_tc = -1;                  // VIASD_ATTN=tc selects the tcgen05 kernel with query rows on TMEM lanes
+    if (use_tc < 0) { const char *e = getenv("VIASD_ATTN"); use_tc = e && strcmp(e, "tc") == 0; }
     const int QR = (c.n_heads / c.n_kv_heads) * M;
-    const bool fuse = nsplit > 1 && nsplit <= 32 && QR * nsplit <= 160;
-    int rc = launch_attention_mma(m, kc, vc, slim, layer_ord, kc2, vc2, layer_ord2, streams, batch, M, nsplit, fuse ? 1 : 0, st);
-    if (rc || nsplit == 1 || fuse) return rc;
+    const int reps = use_tc ? attention_tc_replicas(QR) : 1;
+    const int nsplit = mma_nsplit(m, batch, M, streams, use_tc != 0, reps);
+    const int n_part = nsplit * reps;        // key ranges per (row, head) that have to be merged
+    const bool fuse = n_part > 1 && n_part <= 32 && QR * n_part <= 160;
+    int rc = use_tc ? launch_attention_tc(m, kc, vc, slim, layer_ord, kc2, vc2, layer_ord2, streams, batch, M, nsplit, fuse ? 1 : 0, st)
+                    : launch_attention_mma(m, kc, vc, slim, layer_ord, kc2, vc2, layer_ord2, streams, batch, M, nsplit, fuse ? 1 : 0, st);
+    if (rc || n_part == 1 || fuse) return rc;
     attention_combine_kernel<__nv_bfloat16, 128><<<dim3(streams * batch * M, c.n_heads), 128, 0, st>>>(
-        (__nv_bfloat16 *)m->ws.attn, m->ws.rows_alloc * (size_t)c.n_heads * 128, m->ws.part, M, c.n_heads, nsplit);
+        (__nv_bfloat16 *)m->ws.attn, m->ws.rows_alloc * (size_t)c.n_heads * 128, m->ws.part, M, c.n_heads, n_part);
     LAUNCH_CHECK();
     return VIASD_OK;
 }
