@@ -195,15 +195,27 @@ static int mma_nsplit(const viasd_model *m, int batch, int M, int streams, bool 
 static int mma_attention(viasd_model *m, const void *kc, const void *vc, bool slim, int layer_ord, const void *kc2,
                          const void *vc2, int layer_ord2, int streams, int batch, int M, cudaStream_t st) {
     const viasd_config &c = m->cfg;
-    static int use_tc = -1;                  // VIASD_ATTN=tc selects the tcgen05 kernel with query rows on TMEM lanes
-    if (use_tc < 0) { const char *e = getenv("VIASD_ATTN"); use_tc = e && strcmp(e, "tc") == 0; }
+    // VIASD_ATTN: "mma" = mma.sync kernel, "tc" = tcgen05 with query rows on the TMEM lanes, "tk" = tcgen05 with keys on
+    // the lanes (few query rows only).  Default: tk where it applies, else mma.
+    static int kind = -1;                    // 0 mma, 1 tc, 2 tk, 3 default
+    if (kind < 0) {
+        const char *e = getenv("VIASD_ATTN");
+        kind = !e ? 3 : strcmp(e, "mma") == 0 ? 0 : strcmp(e, "tc") == 0 ? 1 : strcmp(e, "tk") == 0 ? 2 : 3;
+    }
     const int QR = (c.n_heads / c.n_kv_heads) * M;
-    const int reps = use_tc ? attention_tc_replicas(QR) : 1;
-    const int nsplit = mma_nsplit(m, batch, M, streams, use_tc != 0, reps);
+    // keys-on-lanes pays off when a CTA streams many tiles; with a handful per CTA (one short sequence) the
+    // mma.sync kernel's shorter latency chain wins
+    const long long tiles_total = (long long)streams * batch * c.n_kv_heads * ((c.max_ctx + 127) / 128);
+    int use = kind == 3 ? (attention_tk_supported(QR) && tiles_total >= 8LL * m->sm_count ? 2 : 0) : kind;
+    if (use == 2 && !attention_tk_supported(QR)) use = 0;
+    const int reps = use == 1 ? attention_tc_replicas(QR) : 1;
+    const int nsplit = mma_nsplit(m, batch, M, streams, use != 0, reps);
     const int n_part = nsplit * reps;        // key ranges per (row, head) that have to be merged
     const bool fuse = n_part > 1 && n_part <= 32 && QR * n_part <= 160;
-    int rc = use_tc ? launch_attention_tc(m, kc, vc, slim, layer_ord, kc2, vc2, layer_ord2, streams, batch, M, nsplit, fuse ? 1 : 0, st)
-                    : launch_attention_mma(m, kc, vc, slim, layer_ord, kc2, vc2, layer_ord2, streams, batch, M, nsplit, fuse ? 1 : 0, st);
+    int rc;
+    if (use == 2) rc = launch_attention_tk(m, kc, vc, slim, layer_ord, kc2, vc2, layer_ord2, streams, batch, M, nsplit, fuse ? 1 : 0, st);
+    else if (use == 1) rc = launch_attention_tc(m, kc, vc, slim, layer_ord, kc2, vc2, layer_ord2, streams, batch, M, nsplit, fuse ? 1 : 0, st);
+    else rc = launch_attention_mma(m, kc, vc, slim, layer_ord, kc2, vc2, layer_ord2, streams, batch, M, nsplit, fuse ? 1 : 0, st);
     if (rc || n_part == 1 || fuse) return rc;
     attention_combine_kernel<__nv_bfloat16, 128><<<dim3(streams * batch * M, c.n_heads), 128, 0, st>>>(
         (__nv_bfloat16 *)m->ws.attn, m->ws.rows_alloc * (size_t)c.n_heads * 128, m->ws.part, M, c.n_heads, n_part);

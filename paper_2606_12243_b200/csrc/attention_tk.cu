@@ -1,0 +1,618 @@
+// Block attention on tcgen05 for few query rows (at most 32 per kv head): keys on the TMEM lanes.
+//
+// With 5-27 query rows an MMA whose M dimension is the query rows would be almost all padding.  Here the
+// roles are swapped, as in the projection GEMMs: the 128 keys of a tile are the MMA's M dimension and the
+// query rows its N dimension,
+//
+//   S^T[128 keys, rows] = K Q^T      A = K tile exactly as its TMA box lands (K-major, 128-byte swizzle)
+//                                    B = Q, hi rows then lo rows (N = 2 x rows: x = hi + lo to ~16 bits)
+//   O^T[128 dims, rows] += V^T P^T   A = V tile as it lands, read MN-major (the keys are the contraction)
+//                                    B = P^T, hi rows then lo rows, written by the softmax threads into
+//                                        shared memory in the swizzled K-major layout
+//
+// so a tile costs 16 MMAs of 128 x N x 16 with N = 16..64 instead of 32 of 128 x 128 x 16.
+// A softmax thread owns a key (a TMEM lane) and sees all query rows of it.  Row maxima are exchanged once per
+// tile (warp shuffles, then four values per row through shared memory and one barrier of the four warps); the
+// running maximum only moves when a tile exceeds it by 2^8, so rescaling O^T in TMEM is rare, and every thread
+// takes that decision from the same exchanged values.  Row sums stay per thread until the item ends.
+//
+// Warp roles (192 threads): warp 0 requests K/V tiles by TMA into a ring that runs across the CTA's items,
+// warp 1 owns TMEM and issues the MMAs, warps 2-5 stage Q, run the softmax and write the result.
+// TMEM: S^T double-buffered (2 x 64 columns), O^T (64 columns).
+// Every wait is bounded: on expiry the CTA records VIASD_EDEVICE, lets its copies land and leaves.
+#include "common.cuh"
+#include "tc_ptx.cuh"
+#include <stdlib.h>
+
+namespace {
+
+constexpr int HD = 128;                        // head dimension
+constexpr int TKEYS = 128;                     // keys per tile
+constexpr int HALF_BYTES = TKEYS * 128;        // 128 keys x 64 dims of bf16, as one TMA box lands
+constexpr int STAGE_BYTES = 4 * HALF_BYTES;    // K dims 0..63, K dims 64..127, V dims 0..63, V dims 64..127
+constexpr int TK_THREADS = 192;
+constexpr int TK_MAX_STAGE = 3;
+constexpr int ROWF = HD + 2;                   // partial row: 128 numerators, max (natural-log units), sum
+constexpr float RESCALE_GAP = 8.f;             // log2 units
+constexpr uint32_t TM_S = 0, TM_O = 128;       // TMEM column offsets: S^T buffers at 0 and 64, O^T at 128
+
+struct AttnTkArgs {
+    const float *q;             // [rows, H * HD] rotated queries
+    float *part;                // [b][h][i][split][HD + 2]
+    __nv_bfloat16 *out;         // attention output planes (hi, lo)
+    size_t out_plane;
+    const int *len_eff;
+    const TreeInfo *tree;
+    int *status;
+    int M, H, Hkv, max_batch, max_ctx, layer_ord, nsplit;
+    int batch, layer_ord2;      // second row stream: rows batch*M.., its own cache and layer ordinal
+    int streams, n_items, items_per_cta, fuse_merge, nstage;
+    int *counters;              // arrivals per (stream, sequence, kv head), zero between launches
+    float scale;                // log2(e) / sqrt(hd)
+    int trace_on;               // trace builds only
+};
+
+struct Item { int be, b, g, stream, split, n_ctx, k_begin, k_end, n_tiles, row_base; };
+
+__device__ __forceinline__ Item decode_item(const AttnTkArgs &a, int item) {
+    Item it;
+    it.split = item % a.nsplit;
+    const int bg = item / a.nsplit;
+    it.g = bg % a.Hkv;
+    it.be = bg / a.Hkv;
+    it.stream = it.be / a.batch;
+    it.b = it.be - it.stream * a.batch;
+    it.n_ctx = a.len_eff[it.b];
+    const int Tk = it.n_ctx + a.M;
+    int chunk = (Tk + a.nsplit - 1) / a.nsplit;
+    chunk = (chunk + TKEYS - 1) / TKEYS * TKEYS;
+    it.k_begin = it.split * chunk;
+    it.k_end = min(Tk, it.k_begin + chunk);
+    it.n_tiles = it.k_end > it.k_begin ? (it.k_end - it.k_begin + TKEYS - 1) / TKEYS : 0;
+    it.row_base = (((it.stream ? a.layer_ord2 : a.layer_ord) * a.max_batch + it.b) * a.Hkv + it.g) * a.max_ctx;
+    return it;
+}
+
+__device__ __forceinline__ float ex2(float x) {            // 2^x, hardware approximation (2 ulp)
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// MN-major operand tile with the 128-byte swizzle: 64 contiguous elements along MN per row of 128 bytes,
+// 8 rows (8 steps of the contraction) per 1024-byte group; groups `sbo` bytes apart along the contraction,
+// 64-element blocks `lbo` bytes apart along MN.
+__device__ __forceinline__ uint64_t smem_desc_mn(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+    return (uint64_t)((addr >> 4) & 0x3FFF) | ((uint64_t)((lbo >> 4) & 0x3FFF) << 16) | ((uint64_t)((sbo >> 4) & 0x3FFF) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+          "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// hi + lo columns of one accumulator row: v[r] = column r + column NR + r
+template <int NR>
+__device__ __forceinline__ void load_rows(uint32_t taddr, float (&v)[NR]) {
+    float t[2 * NR];
+#pragma unroll
+    for (int c = 0; c < 2 * NR / 16; ++c) {
+        uint32_t r[16];
+        tc_ld16(taddr + c * 16, r);
+#pragma unroll
+        for (int e = 0; e < 16; ++e) t[c * 16 + e] = __uint_as_float(r[e]);
+    }
+#pragma unroll
+    for (int r = 0; r < NR; ++r) v[r] = t[r] + t[NR + r];
+}
+
+// byte offset of element (row, col) in a K-major tile of 128-byte rows with the 128-byte swizzle; col in bf16 units < 64
+__device__ __forceinline__ uint32_t sw_off(uint32_t row, uint32_t col) {
+    return row * 128u + ((((col >> 3) ^ (row & 7u))) << 4) + (col & 7u) * 2u;
+}
+
+#ifdef VIASD_TC_TRACE
+__device__ long long g_atk_trace[160 * 16];
+__device__ __forceinline__ long long gt_now() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return (long long)t; }
+#define ATK_ON (a.trace_on && et == 0)
+#define ATK_MARK(slot) do { if (ATK_ON) g_atk_trace[blockIdx.x * 16 + (slot)] = gt_now(); } while (0)
+#define ATK_T0() long long tt_ = ATK_ON ? gt_now() : 0
+#define ATK_ADD(slot) do { if (ATK_ON) { long long n_ = gt_now(); g_atk_trace[blockIdx.x * 16 + (slot)] += n_ - tt_; tt_ = n_; } } while (0)
+#else
+#define ATK_MARK(slot) do { } while (0)
+#define ATK_T0() do { } while (0)
+#define ATK_ADD(slot) do { } while (0)
+#endif
+
+template <int NR>                                           // query rows per kv head rounded up to 8, 16 or 32
+__global__ void __launch_bounds__(TK_THREADS, 1)
+attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                    const __grid_constant__ CUtensorMap map_k2, const __grid_constant__ CUtensorMap map_v2, const AttnTkArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) unsigned long long bars[2 * TK_MAX_STAGE + 10];
+    __shared__ uint32_t tmem_base_sh;
+    __shared__ int abort_sh, last_sh;
+    __shared__ float wmax_sh[2][4][NR];                     // per tile parity, per warp: row maxima of its 32 keys
+    __shared__ float lsum_sh[4][NR];                        // per warp: row sums, once per item
+    __shared__ unsigned long long anc_sh[VIASD_MAX_ROWS_PER_SEQ];
+
+    constexpr int NC = 2 * NR;                              // MMA N: hi rows then lo rows
+    constexpr uint32_t QCH = (uint32_t)NC * 128u;           // one 64-wide chunk of an [NC rows] operand
+    PDL_TRIGGER();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int NSTAGE = a.nstage;
+    const int grp = a.H / a.Hkv, QR = grp * a.M;
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t qsm = base, psm = base + 2 * QCH, ring = base + 6 * QCH;   // Q (2 chunks), P^T (2 buffers x 2 chunks), ring
+    uint8_t *gen = smem_raw + (base - smem_u32(smem_raw));
+    auto full_bar = [&](int s) { return smem_u32(&bars[s]); };
+    auto empty_bar = [&](int s) { return smem_u32(&bars[TK_MAX_STAGE + s]); };
+    auto sfull_bar = [&](int b) { return smem_u32(&bars[2 * TK_MAX_STAGE + b]); };
+    auto pfull_bar = [&](int b) { return smem_u32(&bars[2 * TK_MAX_STAGE + 2 + b]); };
+    auto pvdone_bar = [&](int b) { return smem_u32(&bars[2 * TK_MAX_STAGE + 4 + b]); };
+    const uint32_t ofree_bar = smem_u32(&bars[2 * TK_MAX_STAGE + 6]), qfull_bar = smem_u32(&bars[2 * TK_MAX_STAGE + 7]);
+    const uint32_t wg_bar = smem_u32(&bars[2 * TK_MAX_STAGE + 8]);      // the softmax warps among themselves (bounded)
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NSTAGE; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(sfull_bar(b), 1); mbar_init(pfull_bar(b), 4); mbar_init(pvdone_bar(b), 1); }
+        mbar_init(ofree_bar, 4);
+        mbar_init(qfull_bar, 4);
+        mbar_init(wg_bar, 128);
+        abort_sh = 0;
+        last_sh = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_sh)), "r"(256) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_sh;
+    const int i0 = blockIdx.x * a.items_per_cta, i1 = min(a.n_items, i0 + a.items_per_cta);
+
+    if (warp == 0) {
+        // ---------------- TMA producer: the CTA's (item, tile) list, flattened ----------------
+        if (lane == 0) {
+            int p_item = i0, p_tile = 0, p_count = 0;
+            bool ok = true;
+            Item pit = i0 < i1 ? decode_item(a, i0) : Item{};
+            auto issue_next = [&](bool context_only) -> bool {  // false: nothing (more) to request under this condition
+                while (p_item < i1 && p_tile >= pit.n_tiles) { ++p_item; p_tile = 0; if (p_item < i1) pit = decode_item(a, p_item); }
+                if (p_item >= i1) return false;
+                const int k0 = pit.k_begin + p_tile * TKEYS;
+                if (context_only && k0 + TKEYS > pit.n_ctx) return false;   // this tile holds rows the previous kernel writes
+                const int st = p_count % NSTAGE;
+                if (p_count >= NSTAGE && !(ok = mbar_wait(empty_bar(st), ((p_count / NSTAGE) & 1) ^ 1, &abort_sh, a.status))) return false;
+                const uint32_t bar = full_bar(st), dst = ring + st * STAGE_BYTES;
+                const CUtensorMap *mk = pit.stream ? &map_k2 : &map_k, *mv = pit.stream ? &map_v2 : &map_v;
+                const int y = pit.row_base + k0;
+                mbar_expect_tx(bar, STAGE_BYTES);
+                tma_load_2d(dst, mk, bar, 0, y);
+                tma_load_2d(dst + HALF_BYTES, mk, bar, 64, y);
+                tma_load_2d(dst + 2 * HALF_BYTES, mv, bar, 0, y);
+                tma_load_2d(dst + 3 * HALF_BYTES, mv, bar, 64, y);
+                ++p_tile; ++p_count;
+                return true;
+            };
+            // committed context does not change during the pass: ask for it before waiting for the previous kernel
+            while (p_count < NSTAGE && issue_next(true)) { }
+            PDL_WAIT();
+            while (ok && issue_next(false)) { }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NC >> 3) << 17) | ((128u >> 4) << 24);
+            const uint32_t idesc_pv = idesc | (1u << 15);                 // A (the V tile) is MN-major
+            int c_tile = 0, n_q = 0, o_uses = 0, q_be = -1, q_g = -1;   // c_tile: tiles of earlier items (ring and buffer phase)
+            bool ok = true;
+            // tile g (counted over the whole CTA) uses stage g % NSTAGE, S^T buffer g & 1 and P^T buffer g & 1
+            auto issue_qk = [&](int g) -> bool {
+                const int st = g % NSTAGE, sb = g & 1;
+                if (!mbar_wait(full_bar(st), (g / NSTAGE) & 1, &abort_sh, a.status)) return false;
+                tc_fence_after();
+                const uint32_t kst = ring + st * STAGE_BYTES, d = tmem + TM_S + sb * 64;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)
+                    tc_mma(d, smem_desc(kst + (ks >> 2) * HALF_BYTES + (ks & 3) * 32), smem_desc(qsm + (ks >> 2) * QCH + (ks & 3) * 32),
+                           idesc, ks > 0 ? 1u : 0u);
+                tc_commit(sfull_bar(sb));
+                return true;
+            };
+            for (int item = i0; item < i1 && ok; ++item) {
+                const Item it = decode_item(a, item);
+                if (it.be != q_be || it.g != q_g) {
+                    if (!(ok = mbar_wait(qfull_bar, n_q & 1, &abort_sh, a.status))) break;
+                    ++n_q; q_be = it.be; q_g = it.g;
+                }
+                if (it.n_tiles == 0) continue;
+                // issue order S(0), S(1), O(0), S(2), O(1), ...: S(t + 2) is only issued once the softmax of tile t has
+                // read its buffer (it arrived on p_full(t)), and its completion implies that O(t) has read P^T(t)
+                if (!(ok = issue_qk(c_tile))) break;
+                if (it.n_tiles > 1 && !(ok = issue_qk(c_tile + 1))) break;
+                for (int t = 0; t < it.n_tiles; ++t) {
+                    const int g = c_tile + t, sb = g & 1, st = g % NSTAGE;
+                    if (t == 0 && o_uses > 0 && !(ok = mbar_wait(ofree_bar, (o_uses - 1) & 1, &abort_sh, a.status))) break;
+                    if (!(ok = mbar_wait(pfull_bar(sb), (g >> 1) & 1, &abort_sh, a.status))) break;
+                    tc_fence_after();
+                    const uint32_t vst = ring + st * STAGE_BYTES + 2 * HALF_BYTES, pb = psm + sb * 2 * QCH;
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)                        // 16 keys per step: two 8-key groups of 1024 bytes
+                        tc_mma(tmem + TM_O, smem_desc_mn(vst + kk * 2048, HALF_BYTES, 1024),
+                               smem_desc(pb + (kk >> 2) * QCH + (kk & 3) * 32), idesc_pv, (t > 0 || kk > 0) ? 1u : 0u);
+                    tc_commit(empty_bar(st));                             // the stage is free once these MMAs have read it
+                    tc_commit(pvdone_bar(sb));
+                    if (t + 2 < it.n_tiles && !(ok = issue_qk(g + 2))) break;
+                }
+                c_tile += it.n_tiles;
+                ++o_uses;
+            }
+        }
+    } else {
+        // ---------------- softmax / epilogue (warps 2..5 <-> TMEM lane quarters 2,3,0,1): one thread, one key (later one dim) ----------------
+        const int quarter = warp & 3, kl = quarter * 32 + lane, et = threadIdx.x - 64;   // kl: key of the tile / dim of O^T
+        const uint32_t tlane = tmem + ((uint32_t)(quarter * 32) << 16);
+#ifdef VIASD_TC_TRACE
+        if (ATK_ON) for (int z = 0; z < 16; ++z) g_atk_trace[blockIdx.x * 16 + z] = 0;
+#endif
+        ATK_MARK(0);
+        int s_cnt = 0, q_be = -1, q_g = -1, wg_phase = 0;        // s_cnt: tiles this CTA has finished (buffer phase)
+        bool ok = true;
+        auto wg_sync = [&]() -> bool {
+            mbar_arrive(wg_bar);
+            const bool done = mbar_wait(wg_bar, wg_phase & 1, &abort_sh, a.status);
+            ++wg_phase;
+            return done;
+        };
+        // The loop starts with a dry item: one tile and one result on whatever TMEM holds, no waits on the other
+        // roles, nothing stored.  A launch runs this code only a few times per CTA, and the first time through comes
+        // from a cold instruction cache (several microseconds); the dry item takes that hit before the kernel's
+        // predecessor has finished.
+        for (int item = i0 - 1; item < i1 && ok; ++item) {
+            const bool dry = item < i0;
+            if (item == i0) {
+                PDL_WAIT();
+                ATK_MARK(1);
+#ifdef VIASD_TC_TRACE
+                if (ATK_ON) for (int z = 3; z < 12; ++z) g_atk_trace[blockIdx.x * 16 + z] = 0;
+#endif
+                if (et < a.M) anc_sh[et] = a.tree->anc[et];
+                if (!(ok = wg_sync())) break;                         // anc_sh is visible
+            }
+            Item it;
+            if (dry) {
+                it.be = it.b = it.g = it.stream = it.split = it.row_base = it.k_begin = 0;
+                it.n_ctx = it.k_end = TKEYS; it.n_tiles = 1;
+            } else {
+                it = decode_item(a, item);
+            }
+            const int QRW = dry ? 0 : QR;                              // rows whose result is written
+            if (dry || it.be != q_be || it.g != q_g) {
+                // stage the query rows of this (sequence, kv head): rows 0..NR-1 the hi parts, NR..2NR-1 the lo parts,
+                // pre-scaled, in the K-major 128-byte-swizzled layout the MMA reads; loads first
+                for (int idx0 = et; idx0 < NR * (HD / 2); idx0 += 4 * 128) {
+                    float2 v[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int idx = idx0 + q * 128, r = idx / (HD / 2), d2 = (idx % (HD / 2)) * 2;
+                        v[q] = make_float2(0.f, 0.f);
+                        if (idx < NR * (HD / 2) && r < QR) {
+                            const int h = it.g * grp + r / a.M, i = r % a.M;
+                            v[q] = __ldcg(reinterpret_cast<const float2 *>(a.q + ((size_t)(it.be * a.M + i) * a.H + h) * HD + d2));
+                        }
+                    }
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int idx = idx0 + q * 128, r = idx / (HD / 2), d2 = (idx % (HD / 2)) * 2;
+                        if (idx >= NR * (HD / 2)) continue;
+                        const float x0 = v[q].x * a.scale, x1 = v[q].y * a.scale;
+                        const __nv_bfloat162 hi = __floats2bfloat162_rn(x0, x1);
+                        const __nv_bfloat162 lo = __floats2bfloat162_rn(x0 - __low2float(hi), x1 - __high2float(hi));
+                        uint8_t *chunk = gen + (uint32_t)(d2 >> 6) * QCH;
+                        *reinterpret_cast<__nv_bfloat162 *>(chunk + sw_off(r, d2 & 63)) = hi;
+                        *reinterpret_cast<__nv_bfloat162 *>(chunk + sw_off(NR + r, d2 & 63)) = lo;
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> the MMA's reads
+                __syncwarp();
+                if (lane == 0 && !dry) mbar_arrive(qfull_bar);
+                if (!dry) { q_be = it.be; q_g = it.g; }
+                if (item == i0) ATK_MARK(2);
+            }
+            float m_run[NR], l_run[NR];
+#pragma unroll
+            for (int r = 0; r < NR; ++r) { m_run[r] = -INFINITY; l_run[r] = 0.f; }
+
+            for (int t = 0; t < it.n_tiles; ++t) {
+                const int sb = s_cnt & 1;
+                ATK_T0();
+                if (!dry && !(ok = mbar_wait(sfull_bar(sb), (s_cnt >> 1) & 1, &abort_sh, a.status))) break;
+                tc_fence_after();
+                ATK_ADD(3);
+                float s[NR];
+                load_rows<NR>(tlane + TM_S + sb * 64, s);
+                // visibility: past the key range nothing; in the committed context everything; among the block's own
+                // rows only the ancestors of the query's node
+                const int j = it.k_begin + t * TKEYS + kl;
+                if (j >= it.k_end) {
+#pragma unroll
+                    for (int r = 0; r < NR; ++r) s[r] = -INFINITY;
+                } else if (j >= it.n_ctx) {
+                    const int tb = j - it.n_ctx;
+#pragma unroll
+                    for (int r = 0; r < NR; ++r) if (!((anc_sh[r % a.M] >> tb) & 1ull)) s[r] = -INFINITY;
+                }
+                ATK_ADD(4);
+                // row maxima: over the warp's 32 keys by shuffle, over the four warps through shared memory
+                {
+                    float mine = -INFINITY;
+#pragma unroll
+                    for (int r = 0; r < NR; ++r) {
+                        const float wm = warp_max(s[r]);
+                        if (lane == (r & 31)) mine = wm;
+                    }
+                    if (lane < NR) wmax_sh[sb][quarter][lane] = mine;
+                }
+                ATK_ADD(5);
+                if (!(ok = wg_sync())) break;
+                ATK_ADD(6);
+                float corr[NR];
+                bool moved = false;
+#pragma unroll
+                for (int r = 0; r < NR; ++r) {
+                    const float mt = fmaxf(fmaxf(wmax_sh[sb][0][r], wmax_sh[sb][1][r]), fmaxf(wmax_sh[sb][2][r], wmax_sh[sb][3][r]));
+                    corr[r] = 1.f;
+                    if (mt > m_run[r] + RESCALE_GAP) {                 // also the first tile with a visible key (m_run = -inf)
+                        if (m_run[r] != -INFINITY) { corr[r] = ex2(m_run[r] - mt); moved = true; }
+                        m_run[r] = mt;
+                    }
+                }
+                if (moved && !dry) {
+                    // rare: a running maximum moved.  Every thread sees the same maxima, so all four warps come here
+                    // together; O^T is rescaled once the previous tile's MMAs have written it.
+                    if (!(ok = mbar_wait(pvdone_bar(sb ^ 1), ((s_cnt - 1) >> 1) & 1, &abort_sh, a.status))) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int c = 0; c < NC / 16; ++c) {
+                        uint32_t w[16];
+                        tc_ld16(tlane + TM_O + c * 16, w);
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) w[e] = __float_as_uint(__uint_as_float(w[e]) * corr[(c * 16 + e) % NR]);
+                        tc_st16(tlane + TM_O + c * 16, w);
+                    }
+                    tc_wait_st();
+                }
+                ATK_ADD(7);
+                // weights of this key for every row; P^T (hi rows, lo rows) into shared memory for the MMA
+                uint8_t *pchunk = gen + 2 * QCH + (uint32_t)sb * 2 * QCH + (uint32_t)(kl >> 6) * QCH;
+#pragma unroll
+                for (int r = 0; r < NR; ++r) {
+                    const float p = ex2(s[r] - (m_run[r] == -INFINITY ? 0.f : m_run[r]));   // masked scores are -inf: weight 0
+                    l_run[r] = l_run[r] * corr[r] + p;
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(p), lo = __float2bfloat16_rn(p - __bfloat162float(hi));
+                    *reinterpret_cast<__nv_bfloat16 *>(pchunk + sw_off(r, kl & 63)) = hi;
+                    *reinterpret_cast<__nv_bfloat16 *>(pchunk + sw_off(NR + r, kl & 63)) = lo;
+                }
+                ATK_ADD(8);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> the MMA's reads
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0 && !dry) mbar_arrive(pfull_bar(sb));     // S^T is read, P^T (and the rescaled O^T) are in place
+                if (!dry) ++s_cnt;
+                ATK_ADD(9);
+#ifdef VIASD_TC_TRACE
+                if (ATK_ON && !dry) g_atk_trace[blockIdx.x * 16 + 10] += 1;
+#endif
+            }
+            if (!ok) break;
+            ATK_T0();
+            // ---- the item's result ----
+            // row sums: per warp by shuffle, across the warps through shared memory
+            {
+                float mine = 0.f;
+#pragma unroll
+                for (int r = 0; r < NR; ++r) {
+                    const float ws = warp_sum(l_run[r]);
+                    if (lane == (r & 31)) mine = ws;
+                }
+                if (lane < NR) lsum_sh[quarter][lane] = mine;
+            }
+            // the last MMA into O^T of the item (and with it all earlier ones) is complete
+            if (!dry && it.n_tiles > 0 && !(ok = mbar_wait(pvdone_bar((s_cnt - 1) & 1), ((s_cnt - 1) >> 1) & 1, &abort_sh, a.status))) break;
+            tc_fence_after();
+            if (!(ok = wg_sync())) break;
+            float o[NR];
+            if (it.n_tiles > 0) {
+                load_rows<NR>(tlane + TM_O, o);
+            } else {
+#pragma unroll
+                for (int r = 0; r < NR; ++r) o[r] = 0.f;
+            }
+            const bool single = a.nsplit == 1;
+#pragma unroll
+            for (int r = 0; r < NR; ++r) {
+                if (r < QRW) {
+                    const float l = lsum_sh[0][r] + lsum_sh[1][r] + lsum_sh[2][r] + lsum_sh[3][r];
+                    const int h = it.g * grp + r / a.M, node = r % a.M;
+                    if (single) {
+                        store_act<__nv_bfloat16>(a.out, a.out_plane, ((size_t)(it.be * a.M + node) * a.H + h) * HD + kl, o[r] / l);
+                    } else {
+                        float *pdst = a.part + ((((size_t)it.be * a.H + h) * a.M + node) * a.nsplit + it.split) * ROWF;
+                        pdst[kl] = o[r];
+                        if (kl == 0) { pdst[HD] = m_run[r] * 0.6931471805599453f; pdst[HD + 1] = l; }   // natural-log units
+                    }
+                }
+            }
+            if (!dry && it.n_tiles > 0) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(ofree_bar);                 // the next item may overwrite O^T
+            }
+            if (!dry && !single && a.fuse_merge) {
+                // last key range of this (sequence, kv head) to finish merges all of them, in range order
+                __threadfence();
+                if (!(ok = wg_sync())) break;
+                if (et == 0) {
+                    const int old = atomicAdd(&a.counters[it.be * a.Hkv + it.g], 1);
+                    last_sh = old == a.nsplit - 1;
+                    if (last_sh) a.counters[it.be * a.Hkv + it.g] = 0;
+                }
+                if (!(ok = wg_sync())) break;
+                if (last_sh) {
+                    __threadfence();
+                    for (int r = warp - 2; r < QR; r += 4) {
+                        const int hh = it.g * grp + r / a.M, i = r % a.M;
+                        const float *src = a.part + (((size_t)it.be * a.H + hh) * a.M + i) * (size_t)a.nsplit * ROWF;
+                        // lane s holds range s's (max, sum); the weights go round by shuffle (at most 32 ranges when fused)
+                        float ms = -INFINITY, ls = 0.f;
+                        if (lane < a.nsplit) { ms = __ldcg(src + (size_t)lane * ROWF + HD); ls = __ldcg(src + (size_t)lane * ROWF + HD + 1); }
+                        float num[HD / 32];
+#pragma unroll
+                        for (int e = 0; e < HD / 32; ++e) num[e] = 0.f;
+                        const float mmax = warp_max(ms);
+                        const float w = (ms == -INFINITY) ? 0.f : expf(ms - mmax);
+                        const float den = warp_sum(ls * w);
+                        for (int s0 = 0; s0 < a.nsplit; s0 += 4) {
+                            float v[4][HD / 32];
+#pragma unroll
+                            for (int q = 0; q < 4; ++q)
+#pragma unroll
+                                for (int e = 0; e < HD / 32; ++e)
+                                    v[q][e] = s0 + q < a.nsplit ? __ldcg(src + (size_t)(s0 + q) * ROWF + lane + 32 * e) : 0.f;
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const float wq = __shfl_sync(0xffffffffu, w, (s0 + q) & 31);
+#pragma unroll
+                                for (int e = 0; e < HD / 32; ++e) num[e] = fmaf(v[q][e], s0 + q < a.nsplit ? wq : 0.f, num[e]);
+                            }
+                        }
+                        const float invd = 1.f / den;
+#pragma unroll
+                        for (int e = 0; e < HD / 32; ++e)
+                            store_act<__nv_bfloat16>(a.out, a.out_plane, ((size_t)(it.be * a.M + i) * a.H + hh) * HD + lane + 32 * e,
+                                                     num[e] * invd);
+                    }
+                }
+                if (!(ok = wg_sync())) break;                          // last_sh and lsum_sh are reused by the next item
+            } else {
+                if (!(ok = wg_sync())) break;                          // lsum_sh is reused by the next item
+            }
+            ATK_ADD(11);
+        }
+    }
+
+    // ---------------- teardown ----------------
+    __syncwarp();
+#ifdef VIASD_TC_TRACE
+    if (a.trace_on && threadIdx.x == 64) g_atk_trace[blockIdx.x * 16 + 12] = gt_now();
+#endif
+    if (abort_sh && threadIdx.x == 0) {
+        // give copies and MMAs that are still in flight time to land before shared memory and TMEM go away
+        const long long t0 = clock64();
+        while (clock64() - t0 < 400000) { }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256) : "memory");
+    }
+}
+
+}  // namespace
+
+int attention_tk_supported(int query_rows) { return query_rows <= 32; }
+
+// tensor maps over the caches are rebuilt only when the caller's pointers change
+static int cache_maps_tk(viasd_model *m, CacheMaps &cm, const void *kc, const void *vc, int n_layers) {
+    if (cm.k_ptr == kc && cm.v_ptr == vc) return VIASD_OK;
+    const viasd_config &c = m->cfg;
+    const uint64_t rows = (uint64_t)n_layers * c.max_batch * c.n_kv_heads * c.max_ctx;
+    int rc;
+    if ((rc = tc_make_map(&cm.k, kc, rows, HD, TKEYS))) return rc;
+    if ((rc = tc_make_map(&cm.v, vc, rows, HD, TKEYS))) return rc;
+    cm.k_ptr = kc; cm.v_ptr = vc;
+    return VIASD_OK;
+}
+
+// streams = 1: one cache (full or slim).  streams = 2: rows [0, batch*M) against the full cache at layer_ord and
+// rows [batch*M, 2*batch*M) against the slim cache at layer_ord2, in one launch.
+int launch_attention_tk(viasd_model *m, const void *kc, const void *vc, bool slim, int layer_ord, const void *kc2,
+                        const void *vc2, int layer_ord2, int streams, int batch, int M, int nsplit, int fuse_merge,
+                        cudaStream_t st) {
+    const viasd_config &c = m->cfg;
+    CacheMaps &cm = slim ? m->cmaps_slim : m->cmaps_full;
+    int rc;
+    if ((rc = cache_maps_tk(m, cm, kc, vc, slim ? m->n_routed : c.n_layers))) return rc;
+    CacheMaps *cm2 = &cm;
+    if (streams == 2) {
+        cm2 = &m->cmaps_slim;
+        if ((rc = cache_maps_tk(m, *cm2, kc2, vc2, m->n_routed))) return rc;
+    }
+    const int grp = c.n_heads / c.n_kv_heads, QR = grp * M;
+    if (QR > 32) return VIASD_EINVAL;
+    const int nr = QR <= 8 ? 8 : QR <= 16 ? 16 : 32;
+    AttnTkArgs a;
+    a.trace_on = 0;
+#ifdef VIASD_TC_TRACE
+    {
+        static int n_launch = 0;
+        const char *e = getenv("VIASD_AT_TRACE_IDX");
+        a.trace_on = e && atoi(e) == n_launch ? 1 : 0;
+        if (e && atoi(e) < 0) n_launch = 0; else ++n_launch;
+    }
+#endif
+    a.q = m->ws.q; a.part = m->ws.part; a.out = (__nv_bfloat16 *)m->ws.attn;
+    a.out_plane = m->ws.rows_alloc * (size_t)c.n_heads * HD;
+    a.len_eff = m->ws.len_eff; a.tree = m->ws.tree; a.status = &m->ws.stats->device_status;
+    a.M = M; a.H = c.n_heads; a.Hkv = c.n_kv_heads; a.max_batch = c.max_batch; a.max_ctx = c.max_ctx;
+    a.layer_ord = layer_ord; a.nsplit = nsplit; a.scale = 1.4426950408889634f / sqrtf((float)HD);   // log2(e) / sqrt(hd)
+    a.batch = batch; a.layer_ord2 = layer_ord2; a.streams = streams;
+    a.counters = m->ws.attn_counters;
+    a.fuse_merge = fuse_merge;
+    a.n_items = streams * batch * c.n_kv_heads * nsplit;
+    int grid = a.n_items < m->sm_count ? a.n_items : m->sm_count;
+    a.items_per_cta = (a.n_items + grid - 1) / grid;
+    grid = (a.n_items + a.items_per_cta - 1) / a.items_per_cta;
+    const size_t op_bytes = 6 * (size_t)(2 * nr) * 128;            // Q (2 chunks) and two P^T buffers (2 chunks each)
+    a.nstage = 1024 + op_bytes + 3 * (size_t)STAGE_BYTES <= 220 * 1024 ? 3 : 2;
+    const size_t smem = 1024 + op_bytes + a.nstage * (size_t)STAGE_BYTES;
+    static bool attr_done = false;
+    if (!attr_done) {
+        CUDA_TRY(cudaFuncSetAttribute(attention_tk_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+        CUDA_TRY(cudaFuncSetAttribute(attention_tk_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+        CUDA_TRY(cudaFuncSetAttribute(attention_tk_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+        attr_done = true;
+    }
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    pdl_config(cfg, attr, dim3(grid), dim3(TK_THREADS), smem, st);
+    if (nr == 8) CUDA_TRY(cudaLaunchKernelEx(&cfg, attention_tk_kernel<8>, cm.k, cm.v, cm2->k, cm2->v, a));
+    else if (nr == 16) CUDA_TRY(cudaLaunchKernelEx(&cfg, attention_tk_kernel<16>, cm.k, cm.v, cm2->k, cm2->v, a));
+    else CUDA_TRY(cudaLaunchKernelEx(&cfg, attention_tk_kernel<32>, cm.k, cm.v, cm2->k, cm2->v, a));
+    LAUNCH_CHECK();
+    return VIASD_OK;
+}
+
+#ifdef VIASD_TC_TRACE
+extern "C" int viasd_debug_attn_tk_trace(long long *host_out) {
+    return (int)cudaMemcpyFromSymbol(host_out, g_atk_trace, sizeof(long long) * 160 * 16);
+}
+#endif

@@ -148,6 +148,10 @@ int attention_tc_replicas(int query_rows);
 int launch_attention_tc(viasd_model *m, const void *kc, const void *vc, bool slim, int layer_ord, const void *kc2,
                          const void *vc2, int layer_ord2, int streams, int batch, int M, int nsplit, int fuse_merge,
                          cudaStream_t st);
+int attention_tk_supported(int query_rows);
+int launch_attention_tk(viasd_model *m, const void *kc, const void *vc, bool slim, int layer_ord, const void *kc2,
+                         const void *vc2, int layer_ord2, int streams, int batch, int M, int nsplit, int fuse_merge,
+                         cudaStream_t st);
 int launch_attention_dual(viasd_model *m, const void *kf, const void *vf, int layer_full, const void *ks, const void *vs,
                           int ord_slim, int batch, int M, cudaStream_t st);
 int launch_embed_norm2(const viasd_model *m, const float *gain_full, const float *gain_slim, int rows, cudaStream_t st);

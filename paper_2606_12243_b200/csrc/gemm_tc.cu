@@ -239,7 +239,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                     if (et == 0) TRACE(8);
                     const bool last = last_sh != 0;
                     asm volatile("bar.sync 1, 128;" ::: "memory");   // last_sh is reused by the next split tile
-                    if (!last) { ++acc_it; ++seg_i; continue; }
+                    if (!last || DBG(p, 1)) { ++acc_it; ++seg_i; continue; }   // (measurement knob: no finishing at all)
                     __threadfence();
                     if (et == 0) TRACE(13);
                     src = SRC_GLOBAL;
@@ -288,7 +288,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
 
             // ---- the one finishing loop
             const int fe = src == SRC_TMEM ? f : et;
-            const int rows_live = dry ? 0 : p.rows, rows_loop = dry ? CH : p.rows, plane = p.rows * TILE_F;
+            const int rows_live = dry ? 0 : p.rows, rows_loop = dry ? (DBG(p, 2) ? 0 : CH) : p.rows, plane = p.rows * TILE_F;
 #pragma unroll 1
             for (int r0 = 0; r0 < rows_loop; r0 += CH) {
                 float g[CH], uu[CH];
