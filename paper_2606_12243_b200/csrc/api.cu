@@ -483,8 +483,8 @@ int viasd_verify_step(viasd_model *m, viasd_cache *cache, const viasd_draft *dra
     // Both verifiers in one sweep over the layers (routed layers' weights are read once for both) while the two
     // row streams together still fit one 128-column MMA with hi/lo planes; beyond that the step is no longer bound
     // by the weight stream alone and the passes run one after the other.
-    static int dual_max = -1;                // VIASD_DUAL_MAX: most rows (both streams together) the one-sweep schedule takes
-    if (dual_max < 0) { const char *e = getenv("VIASD_DUAL_MAX"); dual_max = e ? atoi(e) : 64; }
+    int dual_max = 64;                       // VIASD_DUAL_MAX: most rows (both streams together) the one-sweep schedule takes
+    if (const char *e = getenv("VIASD_DUAL_MAX")) dual_max = atoi(e);
     if (m && m->fused && draft && 2 * draft->batch * (draft->n_nodes + 1) <= dual_max) {
         if ((rc = check_draft(m, draft)) || (rc = check_cache(cache))) return rc;
         if ((rc = forward_sweep(m, cache, draft, 2, full_logits, slim_logits, (cudaStream_t)stream))) return rc;

@@ -197,11 +197,8 @@ static int mma_attention(viasd_model *m, const void *kc, const void *vc, bool sl
     const viasd_config &c = m->cfg;
     // VIASD_ATTN: "mma" = mma.sync kernel, "tc" = tcgen05 with query rows on the TMEM lanes, "tk" = tcgen05 with keys on
     // the lanes (few query rows only).  Default: tk where it applies, else mma.
-    static int kind = -1;                    // 0 mma, 1 tc, 2 tk, 3 default
-    if (kind < 0) {
-        const char *e = getenv("VIASD_ATTN");
-        kind = !e ? 3 : strcmp(e, "mma") == 0 ? 0 : strcmp(e, "tc") == 0 ? 1 : strcmp(e, "tk") == 0 ? 2 : 3;
-    }
+    int kind = 3;                            // 0 mma, 1 tc, 2 tk, 3 default (read per call: a test may switch kernels)
+    if (const char *e = getenv("VIASD_ATTN")) kind = strcmp(e, "mma") == 0 ? 0 : strcmp(e, "tc") == 0 ? 1 : strcmp(e, "tk") == 0 ? 2 : 3;
     const int QR = (c.n_heads / c.n_kv_heads) * M;
     // keys-on-lanes pays off when a CTA streams many tiles; with a handful per CTA (one short sequence) the
     // mma.sync kernel's shorter latency chain wins

@@ -73,6 +73,20 @@ FORWARD_CASES = ["c1_tiny", "tiny_tree_f32", "mini_7b", "mini_8b_tree", "mini_13
 
 @pytest.mark.parametrize("name", FORWARD_CASES)
 def test_forward_logits_and_appended_kv(name):
+    _check_forward(name)
+
+
+# The attention kernel is chosen by problem size (mma.sync for short single sequences, tcgen05 with keys on the TMEM
+# lanes when a CTA streams many tiles); the small parity cases would otherwise only ever see the first.  "tk" needs at
+# most 32 query rows per kv head, "tc" (query rows on the lanes) takes up to 128.
+@pytest.mark.parametrize("name,kernel", [("mini_7b", "tk"), ("mini_13b", "tk"), ("mini_32b_b3", "tk"), ("mini_7b", "tc"),
+                                         ("mini_8b_tree", "tc"), ("mini_32b", "tc")])
+def test_forward_with_each_attention_kernel(name, kernel, monkeypatch):
+    monkeypatch.setenv("VIASD_ATTN", kernel)
+    _check_forward(name)
+
+
+def _check_forward(name):
     wl = W.get(name)
     vb = _vb()
     eng, st, si, model = _prepare(wl)
@@ -285,6 +299,20 @@ STEP_CASES = ["c1_tiny", "tiny_tree_f32", "mini_7b", "mini_8b_tree", "mini_8b_tr
 
 @pytest.mark.parametrize("name", STEP_CASES)
 def test_verify_step_matches_oracle(name):
+    _check_verify_step(name)
+
+
+# both row streams in one attention launch, with the kernels the small cases do not pick by themselves; and the
+# one-sweep schedule with more than 64 rows (token tiles of 128)
+@pytest.mark.parametrize("name,env", [("mini_7b", {"VIASD_ATTN": "tk"}), ("mini_7b", {"VIASD_ATTN": "tc"}),
+                                      ("mini_13b", {"VIASD_ATTN": "tk", "VIASD_DUAL_MAX": "128"})])
+def test_verify_step_with_each_attention_kernel(name, env, monkeypatch):
+    for k, v in env.items():
+        monkeypatch.setenv(k, v)
+    _check_verify_step(name)
+
+
+def _check_verify_step(name):
     wl = W.get(name)
     vb = _vb()
     eng, st, si, model = _prepare(wl)
