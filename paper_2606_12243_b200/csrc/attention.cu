@@ -241,6 +241,5 @@ int launch_attention(viasd_model *m, const void *kc, const void *vc, bool slim, 
 // slim cache (tensor-core kernel only).
 int launch_attention_dual(viasd_model *m, const void *kf, const void *vf, int layer_full, const void *ks, const void *vs,
                           int ord_slim, int batch, int M, cudaStream_t st) {
-    const viasd_config &c = m->cfg;
     return mma_attention(m, kf, vf, false, layer_full, ks, vs, ord_slim, 2, batch, M, st);
 }

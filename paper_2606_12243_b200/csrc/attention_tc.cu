@@ -310,7 +310,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         const int quarter = warp & 3, trow = quarter * 32 + lane, et = threadIdx.x - 64;
         const int rep = trow / a.rows_per_rep, row = trow - rep * a.rows_per_rep;     // replica, query row
         const bool live = row < QR, warp_live = (quarter * 32) % a.rows_per_rep < QR;
-        const int KR = TKEYS / a.reps, key0 = rep * KR, n_chunk = KR / 32;              // this replica's keys of a tile
+        const int KR = TKEYS / a.reps, key0 = rep * KR;                                // this replica's keys of a tile
         const uint32_t tlane = tmem + ((uint32_t)(quarter * 32) << 16);
 #ifdef VIASD_TC_TRACE
         if (ATC_ON) for (int z = 0; z < 13; ++z) g_atc_trace[blockIdx.x * 16 + z] = 0;

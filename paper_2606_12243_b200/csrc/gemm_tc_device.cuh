@@ -75,10 +75,15 @@ __device__ __forceinline__ void finish_chunk(const TcParams &p, int tile, int f,
         }
     }
     const int nrow = min(CH, rows_live - r0);
+    // dry pass: nothing is stored, but the lines (and pages) the real pass will write are asked for, so that its
+    // first stores do not start with address-translation misses
+    const bool touch = rows_live == 0 && (f & 31) == 0;
+    auto want = [](const void *ptr) { asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr)); };
     if (DUAL) {
         const int n = tile * TILE_F + f;
         if (n >= p.seg_n[0]) return;
         __nv_bfloat16 *dst = p.out_act + (size_t)(p.row0 + r0) * p.ld_out + n;
+        if (touch) { want(dst); want(dst + p.act_plane); }
 #pragma unroll
         for (int j = 0; j < CH; ++j) {
             if (j < nrow) {
@@ -95,6 +100,7 @@ __device__ __forceinline__ void finish_chunk(const TcParams &p, int tile, int f,
     const int n = nbase + nin;
     if (EPI == EPI_STORE) {
         if (!valid) return;
+        if (touch) want(p.out_f32 + (size_t)(p.row0 + r0) * p.ld_out + n);
 #pragma unroll
         for (int j = 0; j < CH; ++j) {
             if (j < nrow) {
@@ -111,6 +117,7 @@ __device__ __forceinline__ void finish_chunk(const TcParams &p, int tile, int f,
         const float gain_b = (valid && p.next_gain2) ? p.next_gain2[n] : gain_a;
         float *hp = p.out_f32 + (size_t)(p.row0 + r0) * p.ld_out + n;
         __nv_bfloat16 *ap = p.next_act + (size_t)(p.row0 + r0) * p.ld_out + n;
+        if (touch) { want(hp); want(ap); want(ap + p.next_plane); want(p.ssq_out + ((size_t)tile * 4 + (f >> 5)) * p.ssq_stride + p.row0 + r0); }
         float v[CH];
 #ifdef VIASD_TC_TRACE
         asm volatile("" :: "f"(gain_a), "f"(gain_b));
@@ -161,6 +168,10 @@ __device__ __forceinline__ void finish_chunk(const TcParams &p, int tile, int f,
                 const float other = xch[j * TILE_F + (f ^ 64)];
                 g[j] = f < 64 ? g[j] * c[j] - other * sn[j] : g[j] * c[j] + other * sn[j];
             }
+        }
+        if (touch) {
+            if (s == 0) want(p.q_out + ((size_t)(p.row0 + r0) * p.rope_H + head) * TILE_F + f);
+            else want((s == 1 ? p.kc : p.vc) + ((((size_t)p.layer_ord * p.max_batch) * p.rope_Hkv + head) * p.max_ctx) * TILE_F + f);
         }
         if (s == 0) {
             float *dst = p.q_out + ((size_t)(p.row0 + r0) * p.rope_H + head) * TILE_F + f;
