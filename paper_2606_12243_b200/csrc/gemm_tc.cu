@@ -188,6 +188,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
             int src = SRC_DRY, buf = 0, first_cta = 0, last_cta = 0;
             uint32_t t0 = 0;
             const float *parts = nullptr, *aux = nullptr;
+            int stage_rows = 0, aux_kind = 0;                // staged gather: rows per round; 1: residual rows, 2: rotary tables
             if (dry) {
                 // the dry pass sums one "contributor" out of whatever the ring holds, so that the staged path's code is warm too
                 src = SRC_SMEM;
@@ -247,54 +248,66 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                     __threadfence();
                     if (et == 0) TRACE(13);
                     src = SRC_GLOBAL;
-                    // Staged gather: when this is the CTA's last piece of work the shared-memory ring is idle, so
-                    // all partials (and the rows the epilogue would otherwise fetch chunk by chunk) come in with
-                    // one round of bulk copies.  Same sums in the same order as the direct path.
+                    // Staged gather: when this is the CTA's last piece of work the shared-memory ring is idle, so the
+                    // partials (and the rows the epilogue would otherwise fetch chunk by chunk) come in by bulk copies,
+                    // as many rows per round as the ring holds.  Same sums in the same order as the direct path.
                     const int n_c = last_cta - first_cta + 1;
-                    const uint32_t part_bytes = (uint32_t)p.rows * TILE_F * 4;
-                    if (u >= u_end && (uint32_t)(n_c * NACC + 1) * part_bytes <= (uint32_t)S * stage_bytes) {
-                        const uint32_t aux_sh = smem_base, part_sh = smem_base + part_bytes;
-                        int aux_kind = 0;                    // 1: residual rows, 2: rotary tables
+                    const int fit = (int)(((uint32_t)S * stage_bytes) / ((uint32_t)(n_c * NACC + 1) * TILE_F * 4u)) / CH * CH;
+                    if (u >= u_end && fit >= CH) {
+                        stage_rows = fit < p.rows ? fit : (p.rows + CH - 1) / CH * CH;
                         if (EPI == EPI_ADD_NORM && (sg.tile + 1) * TILE_F <= p.seg_n[0]) aux_kind = 1;
                         if (EPI == EPI_QKV_ROPE && sg.tile < p.seg_tile_end[1]) aux_kind = 2;
-                        const bool has_part = et < n_c * NACC, has_aux = aux_kind && et < p.rows;
-                        asm volatile("fence.proxy.async.global;" ::: "memory");
-                        if (has_part || has_aux) {
-                            mbar_expect_tx(gather_bar, (has_part ? part_bytes : 0u) + (has_aux ? TILE_F * 4u : 0u));
-                            if (has_part) {
-                                const int c = first_cta + et / NACC, half = et - (et / NACC) * NACC;
-                                const int c_first_tile = (c * p.units_per_cta) / p.k_tiles;
-                                const float *from = p.scratch + ((size_t)c * 2 + (c_first_tile == sg.tile ? 0 : 1)) * slot_floats +
-                                                    (size_t)half * NT * TILE_F;
-                                bulk_load(part_sh + (uint32_t)et * part_bytes, from, part_bytes, gather_bar);
-                            }
-                            if (has_aux) {
-                                const uint32_t dst = aux_sh + (uint32_t)et * TILE_F * 4;
-                                if (aux_kind == 1) {
-                                    bulk_load(dst, p.out_f32 + (size_t)(p.row0 + et) * p.ld_out + sg.tile * TILE_F, TILE_F * 4, gather_bar);
-                                } else {
-                                    const int pos = rowmeta[et].x;
-                                    bulk_load(dst, p.cosv + (size_t)pos * 64, 256, gather_bar);
-                                    bulk_load(dst + 256, p.sinv + (size_t)pos * 64, 256, gather_bar);
-                                }
-                            }
-                        } else {
-                            mbar_arrive(gather_bar);
-                        }
-                        if (!(ok = mbar_wait(gather_bar, 0, &abort_sh, p.status))) break;
-                        if (et == 0) TRACE(14);
-                        parts = reinterpret_cast<const float *>(smem_raw + (part_sh - smem_u32(smem_raw)));
-                        if (aux_kind) aux = reinterpret_cast<const float *>(smem_raw + (aux_sh - smem_u32(smem_raw)));
                         src = SRC_SMEM;
                     }
                 }
             }
 
-            // ---- the one finishing loop
+            // ---- the one finishing loop, over blocks of rows (one block unless the gather is staged in rounds)
             const int fe = src == SRC_TMEM ? f : et;
-            const int rows_live = dry ? 0 : p.rows, rows_loop = dry ? (DBG(p, 2) ? 0 : CH) : p.rows, plane = p.rows * TILE_F;
+            const int rows_live = dry ? 0 : p.rows, rows_loop = dry ? (DBG(p, 2) ? 0 : CH) : p.rows;
+            const int blk_rows = stage_rows ? stage_rows : (rows_loop > 0 ? rows_loop : 1);
+            const int plane = stage_rows ? stage_rows * TILE_F : p.rows * TILE_F;     // floats between contributors in shared memory
+            int round = 0;
 #pragma unroll 1
-            for (int r0 = 0; r0 < rows_loop; r0 += CH) {
+            for (int blk0 = 0; blk0 < rows_loop && ok; blk0 += blk_rows, ++round) {
+            const int blk_end = min(rows_loop, blk0 + blk_rows);
+            if (stage_rows) {
+                // rows blk0 .. blk_end-1 of every contributor (and of the epilogue's own inputs) into the ring
+                const int nr = min(p.rows, blk_end) - blk0, n_c = last_cta - first_cta + 1;
+                const uint32_t row_bytes = TILE_F * 4u, aux_sh = smem_base, part_sh = smem_base + (uint32_t)stage_rows * row_bytes;
+                if (round > 0) asm volatile("bar.sync 1, 128;" ::: "memory");    // everyone is done with the previous round's rows
+                const bool has_part = et < n_c * NACC, has_aux = aux_kind && et < nr;
+                asm volatile("fence.proxy.async.global;" ::: "memory");
+                if (has_part || has_aux) {
+                    mbar_expect_tx(gather_bar, (has_part ? (uint32_t)nr * row_bytes : 0u) + (has_aux ? row_bytes : 0u));
+                    if (has_part) {
+                        const int c = first_cta + et / NACC, half = et - (et / NACC) * NACC;
+                        const int c_first_tile = (c * p.units_per_cta) / p.k_tiles;
+                        const float *from = p.scratch + ((size_t)c * 2 + (c_first_tile == sg.tile ? 0 : 1)) * slot_floats +
+                                            (size_t)half * NT * TILE_F + (size_t)blk0 * TILE_F;
+                        bulk_load(part_sh + (uint32_t)et * (uint32_t)stage_rows * row_bytes, from, (uint32_t)nr * row_bytes, gather_bar);
+                    }
+                    if (has_aux) {
+                        const uint32_t dst = aux_sh + (uint32_t)et * row_bytes;
+                        if (aux_kind == 1) {
+                            bulk_load(dst, p.out_f32 + (size_t)(p.row0 + blk0 + et) * p.ld_out + sg.tile * TILE_F, row_bytes, gather_bar);
+                        } else {
+                            const int pos = rowmeta[blk0 + et].x;
+                            bulk_load(dst, p.cosv + (size_t)pos * 64, 256, gather_bar);
+                            bulk_load(dst + 256, p.sinv + (size_t)pos * 64, 256, gather_bar);
+                        }
+                    }
+                } else {
+                    mbar_arrive(gather_bar);
+                }
+                if (!(ok = mbar_wait(gather_bar, round & 1, &abort_sh, p.status))) break;
+                if (et == 0) TRACE(14);
+                parts = reinterpret_cast<const float *>(smem_raw + (part_sh - smem_u32(smem_raw)));
+                // finish_chunk indexes the epilogue's rows by their number in the launch: shift the base by the block start
+                if (aux_kind) aux = reinterpret_cast<const float *>(smem_raw + (aux_sh - smem_u32(smem_raw))) - (size_t)blk0 * TILE_F;
+            }
+#pragma unroll 1
+            for (int r0 = blk0; r0 < blk_end; r0 += CH) {
                 float g[CH], uu[CH];
 #pragma unroll
                 for (int j = 0; j < CH; ++j) { g[j] = 0.f; uu[j] = 0.f; }
@@ -316,7 +329,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                     for (int c = 0; c <= last_cta - first_cta; ++c) {
 #pragma unroll
                         for (int j = 0; j < CH; ++j) {
-                            const int r = min(r0 + j, p.rows - 1);        // rows past the end are discarded
+                            const int r = min(r0 + j, p.rows - 1) - blk0;  // row inside the staged block; rows past the end are discarded
                             g[j] += parts[(c * NACC) * plane + r * TILE_F + et];
                             if (DUAL) uu[j] += parts[(c * NACC + 1) * plane + r * TILE_F + et];
                         }
@@ -349,6 +362,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                 finish_chunk<EPI>(p, sg.tile, fe, r0, g, uu, xch, inv_sh, rowmeta, lane, aux, rows_live);
                 if (et == 0 && r0 == 0) TRACE(15);
             }
+            }   // blocks of rows
 
             if (dry) {
                 dry = false;
