@@ -10,8 +10,11 @@
 //
 // Persistent stream-K schedule: the (tile, k-block) units of the whole GEMM are cut into one contiguous
 // range per CTA, so every SM streams the same number of bytes whatever the shape.  A CTA that holds all
-// k-blocks of a tile finishes it from TMEM; otherwise it writes an fp32 partial and the last CTA to
-// arrive at the tile (an atomic counter, no waiting) sums the partials in CTA order - bit-reproducible.
+// k-blocks of a tile finishes it from TMEM; otherwise it writes an fp32 partial and counts itself in.  The
+// contributors that end their range inside the tile then share its finishing: each waits (bounded) for the
+// count to be complete, pulls its slice of the token rows of every partial into the idle shared-memory ring
+// with bulk copies and sums them in CTA order - bit-reproducible whoever does it.  A contributor that
+// continues into the next tile never waits, so waits cannot chain.
 //
 // Warp roles (192 threads): warp 0 issues TMA loads into a ring of stages, warp 1 allocates TMEM and
 // issues tcgen05.mma, warps 2-5 read the accumulators (tcgen05.ld) and run the epilogue.  Accumulators
@@ -32,7 +35,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) unsigned long long bars[2 * MAX_STAGES + 5];
     __shared__ uint32_t tmem_base_sh;
-    __shared__ int abort_sh, last_sh;
+    __shared__ int abort_sh;
     __shared__ float inv_sh[128];                       // per-row 1/rms of the input (fused RMSNorm)
     __shared__ float xch[CH * TILE_F];                  // rotary partner exchange
     __shared__ int4 rowmeta[128];                       // per token row: rotary position, cache slot, sequence
@@ -60,7 +63,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
         for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
         mbar_init(gather_bar, 128);
         abort_sh = 0;
-        last_sh = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -189,6 +191,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
             uint32_t t0 = 0;
             const float *parts = nullptr, *aux = nullptr;
             int stage_rows = 0, aux_kind = 0;                // staged gather: rows per round; 1: residual rows, 2: rotary tables
+            int row_begin = 0, row_end = p.rows;             // the rows this CTA finishes
             if (dry) {
                 // the dry pass sums one "contributor" out of whatever the ring holds, so that the staged path's code is warm too
                 src = SRC_SMEM;
@@ -230,31 +233,49 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(tempty_bar(buf));   // accumulator buffer may be overwritten
-                    // publish the partial; the last contributor of the tile sums all of them in CTA order
+                    // Publish the partial.  The contributors for which this tile is the last piece of work then share
+                    // its finishing: each waits (bounded) until every contributor has arrived and finishes its own
+                    // slice of the token rows, summing the partials in CTA order.  A contributor that goes on into the
+                    // next tile only arrives and never waits, so no wait depends on another wait.
                     __threadfence();
                     asm volatile("bar.sync 1, 128;" ::: "memory");
                     first_cta = (sg.tile * p.k_tiles) / p.units_per_cta;
                     last_cta = ((sg.tile + 1) * p.k_tiles - 1) / p.units_per_cta;
+                    if (et == 0) atomicAdd(&p.counters[sg.tile], 1);                  // low half: arrivals
+                    if (u < u_end) { ++acc_it; ++seg_i; continue; }
+                    const int n_c = last_cta - first_cta + 1;
+                    const int last_range_end = min(total_units, (last_cta + 1) * p.units_per_cta);
+                    const int n_fin = n_c - (last_range_end > (sg.tile + 1) * p.k_tiles ? 1 : 0);
                     if (et == 0) {
-                        const int old = atomicAdd(&p.counters[sg.tile], 1);
-                        last_sh = (old == last_cta - first_cta) ? 1 : 0;
-                        if (last_sh) p.counters[sg.tile] = 0;   // ready for the next launch
+                        volatile int *ctr = p.counters + sg.tile;
+                        const long long w0 = clock64();
+                        while ((*ctr & 0xffff) < n_c) {
+                            if (abort_sh || clock64() - w0 > WAIT_LIMIT_CYCLES) { abort_sh = 1; atomicExch(p.status, VIASD_EDEVICE); break; }
+                            __nanosleep(64);
+                        }
+                        // high half: finishers that have seen all arrivals; the last of them leaves the counter at zero
+                        if (!abort_sh && (atomicAdd(&p.counters[sg.tile], 1 << 16) >> 16) == n_fin - 1) atomicExch(&p.counters[sg.tile], 0);
                     }
                     asm volatile("bar.sync 1, 128;" ::: "memory");
                     if (et == 0) TRACE(8);
-                    const bool last = last_sh != 0;
-                    asm volatile("bar.sync 1, 128;" ::: "memory");   // last_sh is reused by the next split tile
-                    if (!last || DBG(p, 1)) { ++acc_it; ++seg_i; continue; }   // (measurement knob: no finishing at all)
+                    if (abort_sh) { ok = false; break; }
                     __threadfence();
                     if (et == 0) TRACE(13);
+                    {
+                        // this finisher's rows: whole chunks, dealt in order of CTA number
+                        const int n_chunks = (p.rows + CH - 1) / CH, per = (n_chunks + n_fin - 1) / n_fin;
+                        const int mine = blockIdx.x - first_cta;
+                        row_begin = min(p.rows, mine * per * CH);
+                        row_end = min(p.rows, (mine + 1) * per * CH);
+                    }
                     src = SRC_GLOBAL;
                     // Staged gather: when this is the CTA's last piece of work the shared-memory ring is idle, so the
                     // partials (and the rows the epilogue would otherwise fetch chunk by chunk) come in by bulk copies,
                     // as many rows per round as the ring holds.  Same sums in the same order as the direct path.
-                    const int n_c = last_cta - first_cta + 1;
                     const int fit = (int)(((uint32_t)S * stage_bytes) / ((uint32_t)(n_c * NACC + 1) * TILE_F * 4u)) / CH * CH;
-                    if (u >= u_end && fit >= CH) {
-                        stage_rows = fit < p.rows ? fit : (p.rows + CH - 1) / CH * CH;
+                    if (fit >= CH && row_end > row_begin) {
+                        const int my_rows = (row_end - row_begin + CH - 1) / CH * CH;
+                        stage_rows = fit < my_rows ? fit : my_rows;
                         if (EPI == EPI_ADD_NORM && (sg.tile + 1) * TILE_F <= p.seg_n[0]) aux_kind = 1;
                         if (EPI == EPI_QKV_ROPE && sg.tile < p.seg_tile_end[1]) aux_kind = 2;
                         src = SRC_SMEM;
@@ -264,12 +285,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
 
             // ---- the one finishing loop, over blocks of rows (one block unless the gather is staged in rounds)
             const int fe = src == SRC_TMEM ? f : et;
-            const int rows_live = dry ? 0 : p.rows, rows_loop = dry ? (DBG(p, 2) ? 0 : CH) : p.rows;
+            const int rows_live = dry ? 0 : p.rows, rows_loop = dry ? (DBG(p, 2) ? 0 : CH) : row_end;
             const int blk_rows = stage_rows ? stage_rows : (rows_loop > 0 ? rows_loop : 1);
             const int plane = stage_rows ? stage_rows * TILE_F : p.rows * TILE_F;     // floats between contributors in shared memory
             int round = 0;
 #pragma unroll 1
-            for (int blk0 = 0; blk0 < rows_loop && ok; blk0 += blk_rows, ++round) {
+            for (int blk0 = dry ? 0 : row_begin; blk0 < rows_loop && ok; blk0 += blk_rows, ++round) {
             const int blk_end = min(rows_loop, blk0 + blk_rows);
             if (stage_rows) {
                 // rows blk0 .. blk_end-1 of every contributor (and of the epilogue's own inputs) into the ring
