@@ -185,6 +185,21 @@ int viasd_gemm(const void *x, const void *w, float *y, int rows, int n, int k, i
  * Errors: EINVAL (null / misaligned pointer, k not a multiple of 8), ECAPACITY, ECUDA, EUNSUPPORTED. */
 int viasd_gemm_static(const void *x, const void *w, float *y, int rows, int n, int k, void *stream);
 
+/* KL-style verification cost of a judge distribution against a proposal, per row (Eq. 11), and its sum over the
+ * rows given (block cost, Eq. 10).  With q = softmax(judge_logits / temperature), p = softmax(proposal_logits /
+ * temperature), z1 = log(1 - alpha) + log p - log q, z2 = log(beta) + log p - log q:
+ *     cost_rows[r] = sum_v p(v) phi(z1(v)) + sum_v q(v) phi(z2(v))
+ * margin 0: phi(z) = max(0, z) (Eq. 11); margin 1: phi(z) = tau log(1 + exp(z / tau)) (App. F), which lies
+ * between the margin-0 value and that value plus 2 tau log 2 (F.8).  The cost of a layer mask z over a window of
+ * decoding steps (Eq. 12) is this call with the full verifier's logits as judge and the slim verifier's as
+ * proposal; the gain of the routed path over the direct one (Sec. 2.2) is cost(q, p) - cost(u, p) - cost(q, u).
+ * judge_logits, proposal_logits: device, fp32 [rows, vocab] row-major, read only.  cost_rows: device, [rows],
+ * written.  cost_total: device, one float, written with the sum of cost_rows in row order; may be NULL.
+ * Asynchronous on `stream`; allocates nothing.  Errors: EINVAL (null pointer, rows or vocab < 1, temperature <= 0,
+ * alpha outside [0, 1), beta <= 0, unknown margin, tau <= 0 with margin 1), ECUDA. */
+int viasd_kl_cost(const float *judge_logits, const float *proposal_logits, int rows, int vocab, float temperature,
+                  float alpha, float beta, int margin, float tau, float *cost_rows, float *cost_total, void *stream);
+
 /* Measurement hooks (the paper has no counterpart; they exist so that a benchmark can attribute time).
  * viasd_launch_count: kernels launched by this library in this process so far.
  * viasd_set_timing(on): when on, every launch of the forward / tier / accept / commit path is bracketed by

@@ -21,7 +21,7 @@ VIASD_OK, VIASD_EINVAL, VIASD_ECAPACITY, VIASD_ECUDA, VIASD_EDEVICE, VIASD_EUNSU
 EXPORTS = ["viasd_workspace_bytes", "viasd_init_model", "viasd_full_forward", "viasd_slim_forward",
            "viasd_tier_accept", "viasd_kv_commit", "viasd_verify_step", "viasd_get_stats",
            "viasd_free_model", "viasd_strerror", "viasd_last_cuda_error", "viasd_gemm_scratch_bytes",
-           "viasd_gemm", "viasd_gemm_static", "viasd_launch_count", "viasd_set_timing", "viasd_get_timing"]
+           "viasd_gemm", "viasd_gemm_static", "viasd_kl_cost", "viasd_launch_count", "viasd_set_timing", "viasd_get_timing"]
 
 TIMING_CLASSES = ["gemm", "attention", "norm", "rope", "embed", "tier_accept", "commit"]
 
@@ -114,6 +114,8 @@ def lib() -> C.CDLL:
         l.viasd_gemm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int,
                                  C.c_void_p, C.c_size_t, C.c_void_p]
         l.viasd_gemm_static.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p]
+        l.viasd_kl_cost.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_float, C.c_float, C.c_float, C.c_int,
+                                    C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]
         l.viasd_launch_count.restype = C.c_ulonglong
         l.viasd_set_timing.argtypes = [C.c_void_p, C.c_int]
         l.viasd_get_timing.argtypes = [C.c_void_p, C.POINTER(Timing), C.c_void_p]
@@ -289,6 +291,22 @@ def get_timing(m: Model, stream=None) -> dict:
     out = {n: {"ms": t.ms[i], "launches": int(t.launches[i])} for i, n in enumerate(TIMING_CLASSES)}
     out["dropped"] = int(t.dropped)
     return out
+
+
+def kl_cost(judge_logits: torch.Tensor, proposal_logits: torch.Tensor, alpha: float = 0.0, beta: float = 1.0,
+            temperature: float = 1.0, margin: int = 0, tau: float = 1.0, stream=None):
+    """viasd_kl_cost: per-row KL-style cost of the judge against the proposal (Eq. 11) and its sum (Eq. 10).
+
+    fp32 [rows, V] device tensors -> (cost_rows [rows], cost_total [1]), both fp32 device tensors.
+    """
+    assert judge_logits.dtype == torch.float32 and proposal_logits.dtype == torch.float32
+    assert judge_logits.is_contiguous() and proposal_logits.is_contiguous() and judge_logits.shape == proposal_logits.shape
+    rows, vocab = judge_logits.shape
+    out = torch.empty(rows, dtype=torch.float32, device=judge_logits.device)
+    total = torch.empty(1, dtype=torch.float32, device=judge_logits.device)
+    _check(lib().viasd_kl_cost(_ptr(judge_logits), _ptr(proposal_logits), rows, vocab, temperature, alpha, beta,
+                               int(margin), tau, _ptr(out), _ptr(total), _stream(stream)), "viasd_kl_cost")
+    return out, total
 
 
 def gemm_static(x: torch.Tensor, w: torch.Tensor, y: torch.Tensor, stream=None) -> None:

@@ -496,3 +496,37 @@ def test_full_size_7b_verify_step_matches_oracle():
     assert total == 0 or pinned == total
     if full == wl.batch:
         _check_state(eng, st, wl)
+
+
+# ---------------------------------------------------------------------------------------------
+# KL-style cost kernel (Eq. 10-11, App. F)
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("rows,vocab", [(1, 7), (5, 1000), (9, 32000), (27, 4097)])
+def test_kl_cost_matches_oracle(rows, vocab):
+    from oracle import cost
+    vb = _vb()
+    seed = 9000 + rows
+    judge = synth.normal_f32(seed, 1, (rows, vocab), 2.0)
+    prop = synth.normal_f32(seed, 2, (rows, vocab), 2.0)
+    prop[0] = judge[0]                                                  # equal rows cost nothing
+    tj, tp = torch.from_numpy(judge).cuda(), torch.from_numpy(prop).cuda()
+    for kw in (dict(), dict(alpha=0.2, beta=0.7), dict(alpha=0.1, beta=1.5, temperature=0.8),
+               dict(margin=1, tau=0.5), dict(alpha=0.3, margin=1, tau=0.05)):
+        got, total = vb.kl_cost(tj, tp, **kw)
+        torch.cuda.synchronize()
+        okw = dict(kw)
+        if okw.pop("margin", 0) == 1:
+            okw["phi"] = "softplus"
+        want = cost.step_cost(judge, prop, **okw)
+        g = got.cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(g - want) <= 2e-4 * np.maximum(1.0, np.abs(want))), (kw, g, want)
+        assert abs(float(total.item()) - want.sum()) <= 2e-4 * max(1.0, abs(want.sum())) * rows
+        if not kw:
+            assert g[0] <= 1e-6
+    # argument errors launch nothing
+    lib = vb.lib()
+    assert lib.viasd_kl_cost(tj.data_ptr(), tp.data_ptr(), rows, vocab, 1.0, 1.0, 1.0, 0, 1.0, got.data_ptr(), None, None) \
+        == vb.VIASD_EINVAL
+    assert lib.viasd_kl_cost(tj.data_ptr(), tp.data_ptr(), rows, vocab, 0.0, 0.0, 1.0, 0, 1.0, got.data_ptr(), None, None) \
+        == vb.VIASD_EINVAL
+    assert lib.viasd_kl_cost(None, tp.data_ptr(), rows, vocab, 1.0, 0.0, 1.0, 0, 1.0, got.data_ptr(), None, None) == vb.VIASD_EINVAL
