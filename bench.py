@@ -238,10 +238,12 @@ def run_ours(args, wl) -> None:
     len0, pend0 = eng.len.clone(), eng.pending.clone()
     stream = torch.cuda.current_stream()
 
+    pkw = dict(conf_source=1, strict_break=1) if args.gate == "slim" else {}
+
     def one_step(i):
         eng.len.copy_(len0, non_blocking=True)            # bench-only: rewind the cache instead of refilling it
         eng.pending.copy_(pend0, non_blocking=True)
-        vb.verify_step(eng.model, eng.cache, eng.draft, eng.params(step=i), sl, fl, res)
+        vb.verify_step(eng.model, eng.cache, eng.draft, eng.params(step=i, **pkw), sl, fl, res)
 
     for i in range(args.warmup):
         one_step(i)
@@ -287,7 +289,7 @@ def run_ours(args, wl) -> None:
         eng.draft_tok.copy_(h_tok, non_blocking=True)
         eng.drafter_logits.copy_(h_logits, non_blocking=True)
         eng.pending.copy_(h_pend, non_blocking=True)
-        vb.verify_step(eng.model, eng.cache, eng.draft, eng.params(step=i), sl, fl, res)
+        vb.verify_step(eng.model, eng.cache, eng.draft, eng.params(step=i, **pkw), sl, fl, res)
         h_out.copy_(res.out_tok, non_blocking=True)
         h_ne.copy_(res.n_emit, non_blocking=True)
         stream.synchronize()
@@ -321,7 +323,7 @@ def run_ours(args, wl) -> None:
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.shape.dtype,
         "data": "synthetic",
         "config": {"workload": wl.name, "batch": wl.batch, "ctx": wl.ctx, "draft_nodes": wl.n_nodes,
-                   "routed_layers": wl.n_routed, "layers": wl.shape.n_layers, "mode": wl.mode,
+                   "routed_layers": wl.n_routed, "layers": wl.shape.n_layers, "mode": wl.mode, "gate": args.gate,
                    "l2": "inputs larger than L2: the step streams %.1f GB of weights" % (sb["gemm_shared"] / 1e9),
                    "replicas": world},
         "roofline": {"bound": "hbm", "kernel": "projection GEMMs (all launches of the step)",
@@ -360,6 +362,9 @@ def main() -> None:
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2_7b")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--gate", default="drafter", choices=["drafter", "slim"],
+                    help="whose confidence sets the tiers: the drafter's (default, the configuration the metric is quoted on) "
+                         "or the slim verifier's with a tier-1 acceptance ending the block (Algorithm 2 as printed)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     from synth import workloads as W

@@ -530,3 +530,38 @@ def test_kl_cost_matches_oracle(rows, vocab):
     assert lib.viasd_kl_cost(tj.data_ptr(), tp.data_ptr(), rows, vocab, 0.0, 0.0, 1.0, 0, 1.0, got.data_ptr(), None, None) \
         == vb.VIASD_EINVAL
     assert lib.viasd_kl_cost(None, tp.data_ptr(), rows, vocab, 1.0, 0.0, 1.0, 0, 1.0, got.data_ptr(), None, None) == vb.VIASD_EINVAL
+
+
+# ---------------------------------------------------------------------------------------------
+# Algorithm 2 as printed: the slim verifier's own confidence gates the tiers, a tier-1 acceptance ends the block
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("name", ["mini_7b", "mini_8b_tree_greedy", "mini_13b"])
+def test_verify_step_in_algorithm_2_mode(name):
+    wl = W.get(name)
+    vb = _vb()
+    eng, st, si, model = _prepare(wl)
+    lo, hi = W.thresholds(wl)
+    want = step.verify_step(model, wl.shape, wl.routed, st, si.draft_tok, wl.parent, si.prow, si.drafter_logits,
+                            lo, hi, PU.oracle_params(wl, strict_break=True), conf_source=1)
+    sl, fl = eng.logits_buffer(), eng.logits_buffer()
+    res = vb.alloc_result(wl.batch, wl.n_nodes)
+    vb.verify_step(eng.model, eng.cache, eng.draft, eng.params(conf_source=1, strict_break=1), sl, fl, res)
+    torch.cuda.synchronize()
+    assert vb.get_stats(eng.model).device_status == 0
+    e1, _ = PU.assert_logits_close(sl.cpu().numpy(), want.slim_logits, wl.shape.dtype, "slim")
+    e2, _ = PU.assert_logits_close(fl.cpu().numpy(), want.full_logits, wl.shape.dtype, "full")
+    # the tier of a node is pinned when its confidence is further from both thresholds than the logit error allows
+    got_tier = res.tier.cpu().numpy()
+    margin = np.minimum(np.abs(want.conf - lo), np.abs(want.conf - hi))
+    pinned = margin > 4 * e1
+    assert pinned.mean() > 0.5
+    assert np.array_equal(got_tier[pinned], want.tier[pinned])
+    # confidence itself: one subtraction on logits that agree to e1
+    assert np.abs(res.conf.cpu().numpy() - want.conf).max() <= 2 * e1 + 1e-6
+    if np.array_equal(got_tier, want.tier):
+        pinned_d, total, full = PU.compare_resolution(want.seqs, res.n_acc.cpu().numpy(), res.path.cpu().numpy(),
+                                                      res.out_tok.cpu().numpy(), res.n_emit.cpu().numpy(),
+                                                      res.corr_src.cpu().numpy(), eps_row=max(e1, e2))
+        assert total == 0 or pinned_d / total > 0.6, (pinned_d, total)
+        if full == wl.batch:
+            _check_state(eng, st, wl)
