@@ -356,27 +356,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                         }
                     }
                 } else if (src == SRC_GLOBAL) {
-                    // contributors four at a time: all their loads are in flight before the first add, and the
-                    // sums still run in CTA order
-                    for (int c0 = first_cta; c0 <= last_cta; c0 += 4) {
-                        float pg[4][CH], pu[4][CH];
+                    // rare (a tile shared by more CTAs than the ring can stage a chunk of): plain loads, contributor by
+                    // contributor, kept small on purpose - the size of this loop's code is part of every launch's tail
+#pragma unroll 1
+                    for (int c = first_cta; c <= last_cta; ++c) {
+                        const int c_first_tile = (c * p.units_per_cta) / p.k_tiles;
+                        const float *from = p.scratch + ((size_t)c * 2 + (c_first_tile == sg.tile ? 0 : 1)) * slot_floats +
+                                            (size_t)r0 * TILE_F + et;
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const int c = c0 + q;
-                            const bool on = c <= last_cta;
-                            const int c_first_tile = (c * p.units_per_cta) / p.k_tiles;
-                            const float *from = p.scratch + ((size_t)(on ? c : first_cta) * 2 + (c_first_tile == sg.tile ? 0 : 1)) *
-                                                slot_floats + (size_t)r0 * TILE_F + et;
-#pragma unroll
-                            for (int j = 0; j < CH; ++j) {     // slots are NT >= rows + CH - 1 rows deep: in bounds
-                                pg[q][j] = on ? __ldcg(from + (size_t)j * TILE_F) : 0.f;
-                                if (DUAL) pu[q][j] = on ? __ldcg(from + (size_t)(NT + j) * TILE_F) : 0.f;
-                            }
+                        for (int j = 0; j < CH; ++j) {         // slots are NT >= rows + CH - 1 rows deep: in bounds
+                            g[j] += __ldcg(from + (size_t)j * TILE_F);
+                            if (DUAL) uu[j] += __ldcg(from + (size_t)(NT + j) * TILE_F);
                         }
-#pragma unroll
-                        for (int q = 0; q < 4; ++q)
-#pragma unroll
-                            for (int j = 0; j < CH; ++j) { g[j] += pg[q][j]; if (DUAL) uu[j] += pu[q][j]; }
                     }
                 }
                 if (et == 0 && r0 == 0) TRACE(9);
