@@ -5,18 +5,23 @@
 // vocabulary once and serves every node gated by that row.
 //
 // Accept kernel (Algorithm 2, per-position loop; Algorithm 1, what is appended; App. A, Eq. A.2-A.3):
-// one CTA per sequence walks the draft from the pending token: children of the current row are tried in
+// one CTA per sequence (a cluster of eight when it samples over a large vocabulary) walks the draft from the pending token: children of the current row are tried in
 // index order; tier-0 children are taken at once, tier-1 children are judged by q', tier-2 children by
 // q.  The first row where no child passes ends the walk and the strongest judge that rejected there
 // emits the replacement token.  The walk is sequential over depth, so everything that can be known before
 // it is: a row-statistics kernel (one CTA per logits row, all rows at once) leaves each row's maximum,
 // argmax and softmax denominator, which makes every first test at a position O(1).  Only a rejection in
-// sampling mode (residual, Eq. A.3) and the final draw still sweep the vocabulary inside the walk.
+// sampling mode (residual, Eq. A.3: two sweeps) and the final draw still sweep the vocabulary inside the walk;
+// the CTAs of a cluster share each sweep and combine their block results through distributed shared memory in rank
+// order, so all of them hold the same values and walk the same way.
 #include "common.cuh"
+#include <string.h>
+#include <stdlib.h>
 
 namespace {
 
 constexpr int ACC_THREADS = 512;
+constexpr int ACC_TEAM = 8;               // CTAs per sequence in sampling mode (a portable cluster size)
 
 // ---- counter-based uniforms -------------------------------------------------------------------
 __device__ __forceinline__ unsigned long long mix64(unsigned long long z) {
@@ -188,16 +193,66 @@ struct AcceptArgs {
     unsigned long long seed, step;
 };
 
-// numerators of softmax(l / T) into dst (the row maximum comes from the row statistics)
-__device__ void softmax_numerators(float *dst, const float *row, int V, float inv_temp, float mx) {
-    for (int i = threadIdx.x; i < V; i += blockDim.x) dst[i] = expf((row[i] - mx) * inv_temp);
+// ---- the CTAs of a sequence (a thread-block cluster in sampling mode, else one CTA) ---------------------
+// Each CTA sweeps its share of the vocabulary (indices strided by CTAs x threads); block results are combined through
+// distributed shared memory in rank order, so every CTA holds the same value and takes the same branches.
+struct Team {
+    unsigned rank, size;
+    float *slot_f;              // [2] own slots, double-buffered by phase
+    MaxIdx *slot_m;             // [2]
+    int phase;
+};
+__device__ __forceinline__ void team_barrier() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t remote_addr(const void *own, unsigned rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"((uint32_t)__cvta_generic_to_shared(own)), "r"(rank));
+    return r;
+}
+__device__ float team_sum(float x, float *sh, Team &tm) {
+    x = block_sum(x, sh);
+    if (tm.size == 1) return x;
+    float *slot = tm.slot_f + (tm.phase & 1);
+    if (threadIdx.x == 0) *slot = x;
+    team_barrier();
+    float r = 0.f;
+    for (unsigned k = 0; k < tm.size; ++k) {
+        float v;
+        asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote_addr(slot, k)));
+        r += v;
+    }
+    ++tm.phase;
+    return r;
+}
+__device__ MaxIdx team_argmax(MaxIdx x, MaxIdx *shm, Team &tm) {
+    x = block_argmax(x, shm);
+    if (tm.size == 1) return x;
+    MaxIdx *slot = tm.slot_m + (tm.phase & 1);
+    if (threadIdx.x == 0) *slot = x;
+    team_barrier();
+    MaxIdx r; r.v = -INFINITY; r.i = 0x7fffffff;
+    for (unsigned k = 0; k < tm.size; ++k) {
+        MaxIdx y;
+        const uint32_t ra = remote_addr(slot, k);
+        asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(y.v) : "r"(ra));
+        asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(y.i) : "r"(ra + 4));
+        r = better(r, y);
+    }
+    ++tm.phase;
+    return r;
+}
+
+// numerators of softmax(l / T) into dst (the row maximum comes from the row statistics); this CTA's share
+__device__ void softmax_numerators(float *dst, const float *row, int V, float inv_temp, float mx, const Team &tm) {
+    for (int i = tm.rank * blockDim.x + threadIdx.x; i < V; i += tm.size * blockDim.x) dst[i] = expf((row[i] - mx) * inv_temp);
     __syncthreads();
 }
 
 // argmax_v (log w[v] - log(-log u_v)): a draw from w / sum(w)
-__device__ int gumbel_argmax(const float *w, int V, unsigned long long key, int row, MaxIdx *shm) {
+__device__ int gumbel_argmax(const float *w, int V, unsigned long long key, int row, MaxIdx *shm, Team &tm) {
     MaxIdx best; best.v = -INFINITY; best.i = 0x7fffffff;
-    for (int i = threadIdx.x; i < V; i += blockDim.x) {
+    for (int i = tm.rank * blockDim.x + threadIdx.x; i < V; i += tm.size * blockDim.x) {
         float wi = w[i];
         if (wi > 0.f) {
             float u = unit_f32(key, ((unsigned long long)row << 32) + (unsigned long long)i);
@@ -205,7 +260,7 @@ __device__ int gumbel_argmax(const float *w, int V, unsigned long long key, int 
             best = better(best, c);
         }
     }
-    best = block_argmax(best, shm);
+    best = team_argmax(best, shm, tm);
     return best.i == 0x7fffffff ? 0 : best.i;
 }
 
@@ -213,7 +268,14 @@ __global__ void __launch_bounds__(ACC_THREADS)
 accept_kernel(AcceptArgs a) {
     __shared__ MaxIdx shm[32];
     __shared__ float sh[32];
-    const int b = blockIdx.x, N = a.N, M = N + 1, V = a.V;
+    __shared__ float slot_f[2];
+    __shared__ MaxIdx slot_m[2];
+    Team tm;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(tm.rank));
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(tm.size));
+    tm.slot_f = slot_f; tm.slot_m = slot_m; tm.phase = 0;
+    const bool lead = tm.rank == 0 && threadIdx.x == 0;       // the one thread that writes the results
+    const int b = blockIdx.x / tm.size, N = a.N, M = N + 1, V = a.V;
     const TreeInfo *tree = a.tree;
     const bool sampling = a.mode == 1;
     float *P[3] = {a.scratch + ((size_t)b * 3 + 0) * V, a.scratch + ((size_t)b * 3 + 1) * V,
@@ -221,7 +283,7 @@ accept_kernel(AcceptArgs a) {
     const float *st_mx = a.rs.mx + (size_t)b * 3 * RS_STRIDE, *st_z = a.rs.z + (size_t)b * 3 * RS_STRIDE;
     const int *st_arg = a.rs.arg + (size_t)b * 3 * RS_STRIDE;
     const unsigned long long k_acc = stream_key(a.seed, a.step, b, 0), k_gum = stream_key(a.seed, a.step, b, 1);
-    for (int n = threadIdx.x; n < N; n += blockDim.x) a.judge[b * N + n] = 0;
+    if (tm.rank == 0) for (int n = threadIdx.x; n < N; n += blockDim.x) a.judge[b * N + n] = 0;
     __syncthreads();
 
     int cur = 0, n_acc = 0, corr = -1, corr_src = 0;
@@ -230,8 +292,8 @@ accept_kernel(AcceptArgs a) {
         if (c < 0) {                                             // leaf: whole path accepted
             if (a.emit_bonus) {
                 if (sampling) {
-                    softmax_numerators(P[2], a.full + ((size_t)b * M + cur) * V, V, a.inv_temp, st_mx[2 * RS_STRIDE + cur]);
-                    corr = gumbel_argmax(P[2], V, k_gum, cur, shm);
+                    softmax_numerators(P[2], a.full + ((size_t)b * M + cur) * V, V, a.inv_temp, st_mx[2 * RS_STRIDE + cur], tm);
+                    corr = gumbel_argmax(P[2], V, k_gum, cur, shm, tm);
                 } else {
                     corr = st_arg[2 * RS_STRIDE + cur];
                 }
@@ -252,7 +314,7 @@ accept_kernel(AcceptArgs a) {
             v = min(max(v, 0), V - 1);
             if (t == 0) {
                 taken = c; taken_tier = 0;
-                if (threadIdx.x == 0) a.judge[b * N + c] = 1;
+                if (lead) a.judge[b * N + c] = 1;
                 break;
             }
             bool pass;
@@ -266,40 +328,49 @@ accept_kernel(AcceptArgs a) {
                     Z[0] = st_z[pr];
                 }
                 const float u = unit_f32(k_acc, (unsigned long long)c);
-                const float pv = mat[0] ? P[0][v] : expf((row[0][v] - mx[0]) * a.inv_temp);
-                const float jv = mat[t] ? P[t][v] : expf((row[t][v] - mx[t]) * a.inv_temp);
+                const float pv = mat[0] ? __ldcg(&P[0][v]) : expf((row[0][v] - mx[0]) * a.inv_temp);
+                const float jv = mat[t] ? __ldcg(&P[t][v]) : expf((row[t][v] - mx[t]) * a.inv_temp);
                 const float lp = logf(pv / Z[0]);
                 const float lj = logf(jv / Z[t]);
                 pass = (logf(u) + a.log1m_alpha + lp) < lj;       // u < j(v) / ((1 - alpha) p(v)), Eq. A.2
             }
             if (pass) {
                 taken = c; taken_tier = t;
-                if (threadIdx.x == 0) a.judge[b * N + c] = (unsigned char)(1 | (t << 4));
+                if (lead) a.judge[b * N + c] = (unsigned char)(1 | (t << 4));
                 break;
             }
-            if (threadIdx.x == 0) a.judge[b * N + c] = (unsigned char)(2 | (t << 4));
+            if (lead) a.judge[b * N + c] = (unsigned char)(2 | (t << 4));
             failed = max(failed, t);
             if (sampling) {
-                // Eq. A.3 round by round: the rejecting judge becomes its residual against the proposal
-                // (kept as is if the residual vanishes); the rejected token leaves the proposal.
+                // Eq. A.3 round by round: the rejecting judge becomes its residual against the proposal (kept as is if
+                // the residual vanishes); the rejected token leaves the proposal.  Two sweeps of the vocabulary: the
+                // residual's mass, then both distributions written out (from the logits the first time at a position).
                 __syncthreads();                                  // every thread has read P[.][v] above
-                if (!mat[t]) { softmax_numerators(P[t], row[t], V, a.inv_temp, mx[t]); mat[t] = true; }
-                if (!mat[0]) { softmax_numerators(P[0], row[0], V, a.inv_temp, mx[0]); mat[0] = true; }
                 const float sj = a.inv_beta / Z[t], sp = 1.f / Z[0];
+                const bool mt = mat[t], m0 = mat[0];
+                const float *rt = row[t], *r0 = row[0];
+                const float mxt = mx[t], mx0 = mx[0];
                 float s = 0.f;
-                for (int i = threadIdx.x; i < V; i += blockDim.x) s += fmaxf(0.f, P[t][i] * sj - P[0][i] * sp);
-                s = block_sum(s, sh);
-                if (s > 0.f) {
-                    for (int i = threadIdx.x; i < V; i += blockDim.x) P[t][i] = fmaxf(0.f, P[t][i] * sj - P[0][i] * sp);
-                    Z[t] = s;
+                for (int i = tm.rank * blockDim.x + threadIdx.x; i < V; i += tm.size * blockDim.x) {
+                    const float jt = mt ? P[t][i] : expf((rt[i] - mxt) * a.inv_temp);
+                    const float pr = m0 ? P[0][i] : expf((r0[i] - mx0) * a.inv_temp);
+                    s += fmaxf(0.f, jt * sj - pr * sp);
                 }
-                __syncthreads();
-                if (threadIdx.x == 0) P[0][v] = 0.f;
-                __syncthreads();
+                s = team_sum(s, sh, tm);
                 float z = 0.f;
-                for (int i = threadIdx.x; i < V; i += blockDim.x) z += P[0][i];
-                z = block_sum(z, sh);
+                for (int i = tm.rank * blockDim.x + threadIdx.x; i < V; i += tm.size * blockDim.x) {
+                    const float jt = mt ? P[t][i] : expf((rt[i] - mxt) * a.inv_temp);
+                    const float pr = m0 ? P[0][i] : expf((r0[i] - mx0) * a.inv_temp);
+                    P[t][i] = s > 0.f ? fmaxf(0.f, jt * sj - pr * sp) : jt;
+                    const float keep = i == v ? 0.f : pr;
+                    P[0][i] = keep;
+                    z += keep;
+                }
+                z = team_sum(z, sh, tm);                          // (its barrier also publishes the arrays to the other CTAs)
+                mat[t] = true; mat[0] = true;
+                if (s > 0.f) Z[t] = s;
                 if (z > 0.f) Z[0] = z;
+                __syncthreads();
             }
         }
         if (taken >= 0) {
@@ -308,7 +379,7 @@ accept_kernel(AcceptArgs a) {
                 corr_src = 1;
                 break;
             }
-            if (threadIdx.x == 0) a.path[b * N + n_acc] = taken;
+            if (lead) a.path[b * N + n_acc] = taken;
             ++n_acc;
             cur = taken + 1;
             continue;
@@ -316,14 +387,14 @@ accept_kernel(AcceptArgs a) {
         corr_src = failed;
         if (sampling) {
             __syncthreads();
-            corr = gumbel_argmax(P[failed], V, k_gum, cur, shm);
+            corr = gumbel_argmax(P[failed], V, k_gum, cur, shm, tm);
         } else {
             corr = st_arg[failed * RS_STRIDE + cur];
         }
         break;
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
+    if (lead) {
         int ne = 0;
         for (int j = 0; j < n_acc; ++j) {
             int node = a.path[b * N + j];
@@ -336,6 +407,7 @@ accept_kernel(AcceptArgs a) {
         atomicAdd(&a.stats->emitted, (unsigned long long)ne);
         atomicAdd(&a.stats->accepted, (unsigned long long)n_acc);
     }
+    if (tm.size > 1) team_barrier();          // no CTA leaves while another may still read its slots
 }
 
 // the accept kernel needs the tree layout but no cache: build it here when called on its own
@@ -403,7 +475,20 @@ int launch_accept(const viasd_model *m, const viasd_draft *d, const viasd_params
     a.inv_beta = 1.0f / p->beta;
     for (int i = 0; i < 3; ++i) a.log_acc_rel[i] = p->log_acc_rel[i];
     a.seed = p->seed; a.step = p->step;
-    accept_kernel<<<d->batch, ACC_THREADS, 0, st>>>(a);
+    // sampling over a large vocabulary: a cluster of CTAs per sequence shares every sweep of the vocabulary
+    int team = (p->mode == 1 && m->cfg.vocab >= 16384) ? ACC_TEAM : 1;
+    if (const char *e = getenv("VIASD_ACCEPT_TEAM")) { const int t = atoi(e); if (t == 1 || t == 2 || t == 4 || t == 8) team = t; }
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(d->batch * team);
+    cfg.blockDim = dim3(ACC_THREADS);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = team; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = team > 1 ? 1 : 0;
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, accept_kernel, a));
     LAUNCH_CHECK();
     return VIASD_OK;
 }

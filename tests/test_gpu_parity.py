@@ -222,6 +222,22 @@ def test_accept_sampling_on_oracle_logits(name):
     assert full >= 0.9 * nseq, (full, nseq)
 
 
+# the accept walk runs as a cluster of CTAs per sequence when it samples over a large vocabulary; the small cases
+# force that, and one case has the 8B-shaped vocabulary and tree themselves
+@pytest.mark.parametrize("name,team", [("mini_8b_tree", "8"), ("mini_32b", "4"), ("mini_7b", "2")])
+def test_accept_sampling_as_a_cluster(name, team, monkeypatch):
+    monkeypatch.setenv("VIASD_ACCEPT_TEAM", team)
+    wl = replace(W.get(name), mode="sampling")
+    pinned, total, full, nseq = _accept_case(wl, "sampling", 905)
+    assert full >= 0.9 * nseq, (full, nseq)
+
+
+def test_accept_sampling_full_vocabulary_tree():
+    wl = W.get("c3_8b_tree_b1")
+    pinned, total, full, nseq = _accept_case(replace(wl, batch=2), "sampling", 906, n_steps=2)
+    assert full >= 0.75 * nseq, (full, nseq)
+
+
 def test_accept_options_on_oracle_logits():
     wl = replace(W.get("mini_8b_tree"), mode="greedy")
     for pk in (dict(emit_bonus=True), dict(strict_break=True), dict(log_acc_rel=(0.0, -0.7, -0.3))):
