@@ -178,12 +178,18 @@ static int mma_nsplit(const viasd_model *m, int batch, int M, int streams, bool 
     if (max_s < 1) max_s = 1;
     // microseconds, roughly: the tcgen05 kernel's tile does not depend on the number of query tiles
     const double t_tile = tc ? 0.7 : 0.5 + 0.8 * mt, t_item = tc ? 4.0 : 3.0;
+    // One choice for the whole model, whichever call runs (the cuts must not depend on it): the routed layers are
+    // charged as two-stream launches, as the verify step runs them, the others as one-stream launches.
+    const int n_dual = m->n_routed, n_single = c.n_layers - m->n_routed;
     int best = 1;
     double best_cost = 1e30;
     for (int s = 1; s <= max_s; ++s) {
-        const int n = base * s, ipc = (n + sms - 1) / sms;
         const int tpi = ((tiles + s - 1) / s);
-        const double cost = ipc * (tpi * t_tile + t_item) + 0.15 * s * reps;
+        double cost = 0.15 * s * reps * (n_dual + n_single);
+        for (int st2 = 1; st2 <= 2; ++st2) {
+            const int n = base * s * st2, ipc = (n + sms - 1) / sms;
+            cost += (st2 == 2 ? n_dual : n_single) * ipc * (tpi * t_tile + t_item);
+        }
         if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
     }
     size_t per_split = (size_t)streams * batch * c.n_heads * M * (c.head_dim + 2) * sizeof(float) * reps;
