@@ -41,12 +41,12 @@ def measured_peaks():
 
 def gemm_traffic(wl):
     """DRAM bytes (read + write) of the step's GEMM launches, from the ncu capture of the GEMM kernel at 7B layer
-    shapes whose summary is kept under profiles/: per layer 105.1 + 34.0 + 185.5 + 94.6 MB, head 271.4 MB, captured on
+    shapes whose summary is kept under profiles/: per layer 105.8 + 34.1 + 185.6 + 95.5 MB, head 270.8 MB, captured on
     the 2-layer cut of the 7B workload and scaled by the number of layers (traffic is per launch and the launches
     are the same).  Only known for the 7B layer shapes."""
     if wl.name != "c2_7b":
         return None
-    return int((105.1 + 34.0 + 185.5 + 94.6) * 1e6 * wl.shape.n_layers + 271.4e6)
+    return int((105.8 + 34.1 + 185.6 + 95.5) * 1e6 * wl.shape.n_layers + 270.8e6)
 
 
 # ---------------------------------------------------------------------------------------------
