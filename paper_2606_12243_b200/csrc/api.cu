@@ -132,7 +132,7 @@ int run_gemm(viasd_model *m, const GemmCall &g, int rows, cudaStream_t st) {
     for (int row0 = 0; row0 < rows; row0 += 128) {
         const int nr = rows - row0 < 128 ? rows - row0 : 128;
         const int nt = tc_pick_nt(nr);
-        const int ni = nt == 16 ? 0 : nt == 32 ? 1 : nt == 64 ? 2 : 3;
+        const int ni = nt / 16 - 1;
         TcLaunch L;
         memset(&L, 0, sizeof(L));
         for (int i = 0; i < g.count; ++i) { L.map_w[i] = &g.wmap[i]->map; L.seg_n[i] = g.n[i]; L.w_box_rows[i] = g.wmap[i]->box_rows; }
@@ -177,7 +177,7 @@ int forward_sweep(viasd_model *m, const viasd_cache *cache, const viasd_draft *d
         return timed(m, VIASD_T_GEMM, st, [&]() -> int {
             for (int row0 = 0; row0 < nrows; row0 += 128) {
                 const int nr = nrows - row0 < 128 ? nrows - row0 : 128, nt = tc_pick_nt(nr);
-                const int ni = nt == 16 ? 0 : nt == 32 ? 1 : nt == 64 ? 2 : 3;
+                const int ni = nt / 16 - 1;
                 L.map_x = &xm.map[ni]; L.x_box_rows = xm.box_rows[ni];
                 L.has_lo = 1; L.lo_row_offset = (int)R;
                 L.rows = nr; L.row0 = row0; L.nt = nt;
@@ -401,9 +401,8 @@ int viasd_init_model(const viasd_config *cfg, const viasd_weights *w, const unsi
         }
         if (!rc) rc = wm(m->head_map, m->lm_head, cfg->vocab, d);
         auto am = [&](ActMaps &o, const void *base, uint64_t k) {
-            const int nts[4] = {16, 32, 64, 128};
-            for (int i = 0; i < 4; ++i) {
-                o.box_rows[i] = tc_box_rows(2 * R, nts[i]);
+            for (int i = 0; i < 8; ++i) {
+                o.box_rows[i] = tc_box_rows(2 * R, 16 * (i + 1));
                 int r2 = tc_make_map(&o.map[i], base, 2 * R, k, o.box_rows[i]);
                 if (r2) return r2;
             }
@@ -481,9 +480,9 @@ int viasd_verify_step(viasd_model *m, viasd_cache *cache, const viasd_draft *dra
     if (!slim_logits || !full_logits) return VIASD_EINVAL;
     if ((rc = check_params(params))) return rc;
     // Both verifiers in one sweep over the layers (routed layers' weights are read once for both) while the two
-    // row streams together still fit one 128-column MMA with hi/lo planes; beyond that the step is no longer bound
-    // by the weight stream alone and the passes run one after the other.
-    int dual_max = 64;                       // VIASD_DUAL_MAX: most rows (both streams together) the one-sweep schedule takes
+    // row streams together fit one launch (128 token rows: an MMA of 256 columns with the hi/lo planes); beyond
+    // that a sweep would stream every routed layer twice anyway, and the passes run one after the other.
+    int dual_max = 128;                      // VIASD_DUAL_MAX: most rows (both streams together) the one-sweep schedule takes
     if (const char *e = getenv("VIASD_DUAL_MAX")) dual_max = atoi(e);
     if (m && m->fused && draft && 2 * draft->batch * (draft->n_nodes + 1) <= dual_max) {
         if ((rc = check_draft(m, draft)) || (rc = check_cache(cache))) return rc;

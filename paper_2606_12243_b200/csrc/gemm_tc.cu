@@ -474,7 +474,8 @@ extern "C" int viasd_debug_span_read(unsigned long long *host_out, int *n_launch
 }
 #endif
 
-int tc_pick_nt(int rows) { return rows <= 16 ? 16 : rows <= 32 ? 32 : rows <= 64 ? 64 : 128; }
+// token-tile width: the rows rounded up to the MMA's N granularity of 16 (at most 128)
+int tc_pick_nt(int rows) { const int nt = (rows + 15) / 16 * 16; return nt < 16 ? 16 : nt > 128 ? 128 : nt; }
 
 uint32_t tc_box_rows(uint64_t tensor_rows, uint32_t want) { return tensor_rows < want ? (uint32_t)tensor_rows : want; }
 

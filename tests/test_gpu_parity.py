@@ -318,10 +318,10 @@ def test_verify_step_matches_oracle(name):
     _check_verify_step(name)
 
 
-# both row streams in one attention launch, with the kernels the small cases do not pick by themselves; and the
-# one-sweep schedule with more than 64 rows (token tiles of 128)
+# both row streams in one attention launch, with the kernels the small cases do not pick by themselves; and
+# separate passes where the default would be one sweep
 @pytest.mark.parametrize("name,env", [("mini_7b", {"VIASD_ATTN": "tk"}), ("mini_7b", {"VIASD_ATTN": "tc"}),
-                                      ("mini_13b", {"VIASD_ATTN": "tk", "VIASD_DUAL_MAX": "128"})])
+                                      ("mini_13b", {"VIASD_ATTN": "tk", "VIASD_DUAL_MAX": "64"})])
 def test_verify_step_with_each_attention_kernel(name, env, monkeypatch):
     for k, v in env.items():
         monkeypatch.setenv(k, v)
