@@ -58,7 +58,7 @@ size_t carve(const viasd_config &c, char *base, Workspace *ws) {
     w.stats = cv.take<DeviceStats>(sizeof(DeviceStats));
     w.accept_scratch = cv.take<float>(((size_t)c.max_batch * 3 * c.vocab + (size_t)c.max_batch * 9 * VIASD_MAX_ROWS_PER_SEQ) * 4);
     {
-        const int nt = tc_pick_nt(R < 128 ? (int)R : 128);
+        const int nt = tc_pick_nt(R < 128 ? (int)R : 128, true);
         w.gemm_scratch = cv.take<float>(tc_scratch_floats(MAX_GEMM_CTAS, nt, true) * 4);
         size_t widest = (size_t)c.vocab;
         if (qd + 2 * kvd > widest) widest = qd + 2 * kvd;
@@ -131,8 +131,8 @@ int run_gemm(viasd_model *m, const GemmCall &g, int rows, cudaStream_t st) {
     }
     for (int row0 = 0; row0 < rows; row0 += 128) {
         const int nr = rows - row0 < 128 ? rows - row0 : 128;
-        const int nt = tc_pick_nt(nr);
-        const int ni = nt / 16 - 1;
+        const int nt = tc_pick_nt(nr, true);
+        const int ni = nt / 8 - 1;
         TcLaunch L;
         memset(&L, 0, sizeof(L));
         for (int i = 0; i < g.count; ++i) { L.map_w[i] = &g.wmap[i]->map; L.seg_n[i] = g.n[i]; L.w_box_rows[i] = g.wmap[i]->box_rows; }
@@ -176,8 +176,8 @@ int forward_sweep(viasd_model *m, const viasd_cache *cache, const viasd_draft *d
     auto gemm = [&](TcLaunch L, const ActMaps &xm, int nrows) -> int {
         return timed(m, VIASD_T_GEMM, st, [&]() -> int {
             for (int row0 = 0; row0 < nrows; row0 += 128) {
-                const int nr = nrows - row0 < 128 ? nrows - row0 : 128, nt = tc_pick_nt(nr);
-                const int ni = nt / 16 - 1;
+                const int nr = nrows - row0 < 128 ? nrows - row0 : 128, nt = tc_pick_nt(nr, true);
+                const int ni = nt / 8 - 1;
                 L.map_x = &xm.map[ni]; L.x_box_rows = xm.box_rows[ni];
                 L.has_lo = 1; L.lo_row_offset = (int)R;
                 L.rows = nr; L.row0 = row0; L.nt = nt;
@@ -401,8 +401,8 @@ int viasd_init_model(const viasd_config *cfg, const viasd_weights *w, const unsi
         }
         if (!rc) rc = wm(m->head_map, m->lm_head, cfg->vocab, d);
         auto am = [&](ActMaps &o, const void *base, uint64_t k) {
-            for (int i = 0; i < 8; ++i) {
-                o.box_rows[i] = tc_box_rows(2 * R, 16 * (i + 1));
+            for (int i = 0; i < 16; ++i) {
+                o.box_rows[i] = tc_box_rows(2 * R, 8 * (i + 1));
                 int r2 = tc_make_map(&o.map[i], base, 2 * R, k, o.box_rows[i]);
                 if (r2) return r2;
             }
@@ -571,7 +571,7 @@ int viasd_get_timing(viasd_model *m, viasd_timing *out, void *stream) {
 size_t viasd_gemm_scratch_bytes(int rows, int n, int k) {
     (void)k;
     if (rows < 1 || n < 1) return 256;
-    const int nt = tc_pick_nt(rows < 128 ? rows : 128);
+    const int nt = tc_pick_nt(rows < 128 ? rows : 128, false);
     // [tile counters | one status word] then the partial-tile slots
     return align_up((size_t)(tc_tiles(n) + 1) * 4, 256) + tc_scratch_floats(MAX_GEMM_CTAS, nt, false) * 4;
 }
@@ -601,7 +601,7 @@ int viasd_gemm(const void *x, const void *w, float *y, int rows, int n, int k, i
     if ((rc = tc_make_map(&mw, w, n, k, wbox))) return rc;
     for (int row0 = 0; row0 < rows; row0 += 128) {
         const int nr = rows - row0 < 128 ? rows - row0 : 128;
-        const int nt = tc_pick_nt(nr);
+        const int nt = tc_pick_nt(nr, false);
         const uint32_t xbox = tc_box_rows(rows, nt);
         if ((rc = tc_make_map(&mx, x, rows, k, xbox))) return rc;
         TcLaunch L;

@@ -56,7 +56,7 @@ struct Workspace {                      // pointers into the caller's workspace 
 };
 
 struct WMap { CUtensorMap map; uint32_t box_rows; };        // TMA view of one weight matrix
-struct ActMaps { CUtensorMap map[8]; uint32_t box_rows[8]; }; // TMA views of an activation buffer, NT = 16, 32, ..., 128
+struct ActMaps { CUtensorMap map[16]; uint32_t box_rows[16]; }; // TMA views of an activation buffer, NT = 8, 16, ..., 128
 struct LayerMaps { WMap wq, wk, wv, wo, wg, wu, wd; };
 struct CacheMaps { CUtensorMap k, v; const void *k_ptr, *v_ptr; };   // TMA views of one model's KV cache
 

@@ -474,8 +474,11 @@ extern "C" int viasd_debug_span_read(unsigned long long *host_out, int *n_launch
 }
 #endif
 
-// token-tile width: the rows rounded up to the MMA's N granularity of 16 (at most 128)
-int tc_pick_nt(int rows) { const int nt = (rows + 15) / 16 * 16; return nt < 16 ? 16 : nt > 128 ? 128 : nt; }
+// token-tile width: the MMA's N (2 x NT with the hi / lo planes side by side, else NT) comes in multiples of 16
+int tc_pick_nt(int rows, bool has_lo) {
+    const int g = has_lo ? 8 : 16, nt = (rows + g - 1) / g * g;
+    return nt < 16 ? 16 : nt > 128 ? 128 : nt;
+}
 
 uint32_t tc_box_rows(uint64_t tensor_rows, uint32_t want) { return tensor_rows < want ? (uint32_t)tensor_rows : want; }
 

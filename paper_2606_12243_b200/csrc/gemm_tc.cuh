@@ -62,7 +62,7 @@ struct TcLaunch {                       // host-side description of one GEMM
 
 // 2-D bf16 tensor [rows, k] row-major -> TMA map with a (64 x box_rows) box and the 128-byte swizzle
 int tc_make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t k, uint32_t box_rows);
-int tc_pick_nt(int rows);
+int tc_pick_nt(int rows, bool has_lo);
 uint32_t tc_box_rows(uint64_t tensor_rows, uint32_t want);
 size_t tc_scratch_floats(int sm_count, int nt, bool dual);
 int tc_tiles(int n);
