@@ -586,3 +586,42 @@ def test_verify_step_in_algorithm_2_mode(name):
         assert total == 0 or pinned_d / total > 0.6, (pinned_d, total)
         if full == wl.batch:
             _check_state(eng, st, wl)
+
+
+# ---------------------------------------------------------------------------------------------
+# edges of the block shape: the most rows a sequence may have, a one-node draft, an empty committed context
+# ---------------------------------------------------------------------------------------------
+def _edge_tree63():
+    # 63 nodes, 64 rows: a chain of 9 with six children hanging off every chain node
+    par = list(range(-1, 8))
+    for c in range(9):
+        par += [c] * 6
+    assert len(par) == 63
+    return tuple(par)
+
+
+@pytest.mark.parametrize("name,parent,ctx", [("mini_7b", W.chain(63), 300), ("mini_8b_tree_greedy", _edge_tree63(), 200),
+                                             ("mini_13b", W.chain(1), 517), ("mini_7b", W.chain(8), 0),
+                                             ("mini_8b_tree", W.small_tree(), 0)])
+def test_verify_step_edge_shapes(name, parent, ctx):
+    base = W.get(name)
+    wl = replace(base, parent=parent, ctx=ctx, real_prefill=False)
+    vb = _vb()
+    eng, st, si, model = _prepare(wl)
+    lo, hi = W.thresholds(wl)
+    want = step.verify_step(model, wl.shape, wl.routed, st, si.draft_tok, wl.parent, si.prow, si.drafter_logits,
+                            lo, hi, PU.oracle_params(wl))
+    sl, fl = eng.logits_buffer(), eng.logits_buffer()
+    res = vb.alloc_result(wl.batch, wl.n_nodes)
+    vb.verify_step(eng.model, eng.cache, eng.draft, eng.params(), sl, fl, res)
+    torch.cuda.synchronize()
+    assert vb.get_stats(eng.model).device_status == 0
+    assert np.array_equal(res.tier.cpu().numpy(), want.tier)
+    e1, _ = PU.assert_logits_close(sl.cpu().numpy(), want.slim_logits, wl.shape.dtype, "slim")
+    e2, _ = PU.assert_logits_close(fl.cpu().numpy(), want.full_logits, wl.shape.dtype, "full")
+    pinned, total, full = PU.compare_resolution(want.seqs, res.n_acc.cpu().numpy(), res.path.cpu().numpy(),
+                                                res.out_tok.cpu().numpy(), res.n_emit.cpu().numpy(),
+                                                res.corr_src.cpu().numpy(), eps_row=max(e1, e2))
+    assert total == 0 or pinned / total > 0.5, (pinned, total)
+    if full == wl.batch:
+        _check_state(eng, st, wl)
