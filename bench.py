@@ -331,8 +331,9 @@ def run_ours(args, wl) -> None:
                      "unit": "GB/s", "frac": gemm_gbs / peak, "traffic": gemm_traffic(wl),
                      "algorithmic_bytes_per_step": sb["gemm_shared"], "ms_per_step": gemm_ms,
                      "launches_per_step": timing["gemm"]["launches"] // n_timed,
-                     "note": "per-launch events serialise the launches (no overlap between kernels), so this is a lower "
-                             "bound on what the same kernels reach inside the untimed step"},
+                     "note": "one CUDA-event pair per run of consecutive GEMM launches (the four projections between two "
+                             "attention calls, which keep their programmatic overlap); the runs are cut off from the "
+                             "attention kernels around them, so this is a lower bound on the untimed step"},
         "step_roofline": {"algorithmic_bytes": sb["total_shared"], "achieved_gbs": step_gbs,
                           "frac_of_measured": step_gbs / peak, "frac_of_8tbs": step_gbs / HBM_NOMINAL_GBS,
                           "algorithmic_bytes_two_separate_passes": sb["total"],

@@ -202,8 +202,9 @@ int viasd_kl_cost(const float *judge_logits, const float *proposal_logits, int r
 
 /* Measurement hooks (the paper has no counterpart; they exist so that a benchmark can attribute time).
  * viasd_launch_count: kernels launched by this library in this process so far.
- * viasd_set_timing(on): when on, every launch of the forward / tier / accept / commit path is bracketed by
- * CUDA events on the caller's stream (a few thousand launches are kept; later ones are dropped).
+ * viasd_set_timing(on): when on, every run of consecutive launches of one kernel class in the forward / tier /
+ * accept / commit path is bracketed by one pair of CUDA events on the caller's stream (the launches inside a run
+ * keep their programmatic overlap; a few thousand runs are kept, later ones are dropped).
  * viasd_get_timing: synchronises `stream`, sums the recorded intervals per kernel class into `out`
  * (VIASD_T_COUNT entries each) and clears the record. */
 enum { VIASD_T_GEMM = 0, VIASD_T_ATTENTION, VIASD_T_NORM, VIASD_T_ROPE, VIASD_T_EMBED, VIASD_T_TIER_ACCEPT,

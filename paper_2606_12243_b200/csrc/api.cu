@@ -77,13 +77,15 @@ template <typename F>
 int timed(viasd_model *m, int cls, cudaStream_t st, F &&f) {
     KernelTimer &t = m->timer;
     if (!t.on) return f();
+    if (t.open >= 0 && t.cls[t.open] == cls) { ++t.cnt[t.open]; return f(); }     // the run goes on
+    if (t.open >= 0) { CUDA_TRY(cudaEventRecord(t.end[t.open], st)); t.open = -1; }
     if (t.n >= KernelTimer::CAP) { ++t.dropped; return f(); }
     const int i = t.n++;
     t.cls[i] = cls;
+    t.cnt[i] = 1;
     CUDA_TRY(cudaEventRecord(t.beg[i], st));
-    int rc = f();
-    CUDA_TRY(cudaEventRecord(t.end[i], st));
-    return rc;
+    t.open = i;
+    return f();
 }
 
 int check_config(const viasd_config *c) {
@@ -434,6 +436,7 @@ void viasd_free_model(viasd_model *m) {
     delete[] m->timer.beg;
     delete[] m->timer.end;
     delete[] m->timer.cls;
+    delete[] m->timer.cnt;
     delete m;
 }
 
@@ -540,6 +543,7 @@ int viasd_set_timing(viasd_model *m, int on) {
         t.beg = new cudaEvent_t[KernelTimer::CAP];
         t.end = new cudaEvent_t[KernelTimer::CAP];
         t.cls = new int[KernelTimer::CAP];
+        t.cnt = new int[KernelTimer::CAP];
         for (t.created = 0; t.created < KernelTimer::CAP; ++t.created) {
             CUDA_TRY(cudaEventCreate(&t.beg[t.created]));
             CUDA_TRY(cudaEventCreate(&t.end[t.created]));
@@ -547,6 +551,7 @@ int viasd_set_timing(viasd_model *m, int on) {
     }
     t.on = on != 0;
     t.n = 0;
+    t.open = -1;
     t.dropped = 0;
     return VIASD_OK;
 }
@@ -554,13 +559,14 @@ int viasd_set_timing(viasd_model *m, int on) {
 int viasd_get_timing(viasd_model *m, viasd_timing *out, void *stream) {
     if (!m || !out) return VIASD_EINVAL;
     KernelTimer &t = m->timer;
+    if (t.open >= 0) { CUDA_TRY(cudaEventRecord(t.end[t.open], (cudaStream_t)stream)); t.open = -1; }
     CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
     memset(out, 0, sizeof(*out));
     for (int i = 0; i < t.n; ++i) {
         float ms = 0.f;
         CUDA_TRY(cudaEventElapsedTime(&ms, t.beg[i], t.end[i]));
         out->ms[t.cls[i]] += ms;
-        out->launches[t.cls[i]] += 1;
+        out->launches[t.cls[i]] += t.cnt[i];
     }
     out->dropped = t.dropped;
     t.n = 0;

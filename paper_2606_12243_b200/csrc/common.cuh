@@ -60,11 +60,14 @@ struct ActMaps { CUtensorMap map[16]; uint32_t box_rows[16]; }; // TMA views of 
 struct LayerMaps { WMap wq, wk, wv, wo, wg, wu, wd; };
 struct CacheMaps { CUtensorMap k, v; const void *k_ptr, *v_ptr; };   // TMA views of one model's KV cache
 
-struct KernelTimer {                    // optional per-launch CUDA-event record (measurement only)
+// Optional CUDA-event record (measurement only).  A run of consecutive launches of one class shares one pair of
+// events, so that the launches inside it keep their programmatic overlap: an event between two kernels would
+// serialise them, and what is timed then is not what runs.
+struct KernelTimer {
     static constexpr int CAP = 8192;
     cudaEvent_t *beg, *end;
-    int *cls;
-    int n, created;
+    int *cls, *cnt;                     // class and number of calls of each recorded run
+    int n, created, open;               // open: index of the run that has no end event yet, or -1
     long long dropped;
     bool on;
 };
