@@ -83,6 +83,33 @@ __global__ void embed_kernel(float *h, const T *E, const int *row_tok, int d) {
     for (int i = threadIdx.x; i < d; i += blockDim.x) h[(size_t)r * d + i] = to_f32<T>(src[i]);
 }
 
+// One embedding row by one CTA of 8 warps: h = E[tok], a = hi/lo(h * gain), sums of h^2 per 32 features.
+// The row and the gains are loaded in batches of eight independent loads per thread: the embedding rows are cold in
+// HBM, and one load per loop trip made this kernel a chain of memory round trips.
+__device__ __forceinline__ void embed_row(float *h, __nv_bfloat16 *a, size_t plane, float *ssq, int ssq_stride,
+                                          const __nv_bfloat16 *src, const float *gain, int r, int d, int warp, int lane) {
+    for (int base0 = 0; base0 < d; base0 += 8 * 256) {
+        float v[8], g[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int base = base0 + j * 256, i = base + warp * 32 + lane;   // d is a multiple of 128: whole warps stay in range
+            const bool on = base + warp * 32 < d;
+            v[j] = on ? __bfloat162float(src[i]) : 0.f;
+            g[j] = on ? gain[i] : 0.f;
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int base = base0 + j * 256, i = base + warp * 32 + lane;
+            if (base + warp * 32 < d) {
+                h[(size_t)r * d + i] = v[j];
+                store_act<__nv_bfloat16>(a, plane, (size_t)r * d + i, v[j] * g[j]);
+                const float sq = warp_sum(v[j] * v[j]);
+                if (lane == 0) ssq[(size_t)(i >> 5) * ssq_stride + r] = sq;   // (tile * 4 + quarter) == feature / 32
+            }
+        }
+    }
+}
+
 // Embedding gather fused with the preparation of the first RMSNorm of the pass (tensor-core path):
 // h = E[tok]; a = hi/lo(h * gain); partial sums of h^2 per 32 features in the layout the GEMM epilogue reads.
 __global__ void __launch_bounds__(256)
@@ -91,17 +118,7 @@ embed_norm_kernel(float *h, __nv_bfloat16 *a, size_t plane, float *ssq, int ssq_
     const int r = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     PDL_TRIGGER();
     const __nv_bfloat16 *src = E + (size_t)row_tok[r] * d;
-    for (int base = 0; base < d; base += 256) {
-        const int i = base + warp * 32 + lane;            // d is a multiple of 128: whole warps stay in range
-        float v = 0.f;
-        if (base + warp * 32 < d) {
-            v = __bfloat162float(src[i]);
-            h[(size_t)r * d + i] = v;
-            store_act<__nv_bfloat16>(a, plane, (size_t)r * d + i, v * gain[i]);
-            const float sq = warp_sum(v * v);
-            if (lane == 0) ssq[(size_t)(i >> 5) * ssq_stride + r] = sq;   // (tile * 4 + quarter) == feature / 32
-        }
-    }
+    embed_row(h, a, plane, ssq, ssq_stride, src, gain, r, d, warp, lane);
 }
 
 int launch_embed_norm(const viasd_model *m, const float *gain, int rows, cudaStream_t st) {
@@ -121,16 +138,7 @@ embed_norm2_kernel(float *h, __nv_bfloat16 *a, size_t plane, float *ssq, int ssq
     PDL_TRIGGER();
     const float *gain = r < rows ? gain_full : gain_slim;
     const __nv_bfloat16 *src = E + (size_t)row_tok[r < rows ? r : r - rows] * d;
-    for (int base = 0; base < d; base += 256) {
-        const int i = base + warp * 32 + lane;
-        if (base + warp * 32 < d) {
-            const float v = __bfloat162float(src[i]);
-            h[(size_t)r * d + i] = v;
-            store_act<__nv_bfloat16>(a, plane, (size_t)r * d + i, v * gain[i]);
-            const float sq = warp_sum(v * v);
-            if (lane == 0) ssq[(size_t)(i >> 5) * ssq_stride + r] = sq;
-        }
-    }
+    embed_row(h, a, plane, ssq, ssq_stride, src, gain, r, d, warp, lane);
 }
 
 int launch_embed_norm2(const viasd_model *m, const float *gain_full, const float *gain_slim, int rows, cudaStream_t st) {
