@@ -448,8 +448,8 @@ int viasd_slim_forward(viasd_model *m, const viasd_cache *cache, const viasd_dra
     return forward(m, cache, draft, true, logits, (cudaStream_t)stream);
 }
 
-int viasd_tier_accept(viasd_model *m, const viasd_draft *draft, const viasd_params *params, const float *slim_logits,
-                      const float *full_logits, int phase, viasd_result *result, void *stream) {
+static int tier_accept_impl(viasd_model *m, const viasd_draft *draft, const viasd_params *params, const float *slim_logits,
+                           const float *full_logits, int phase, viasd_result *result, bool tree_ready, void *stream) {
     int rc;
     if ((rc = check_draft(m, draft)) || (rc = check_params(params))) return rc;
     if (phase < 1 || phase > 3) return VIASD_EINVAL;
@@ -463,9 +463,14 @@ int viasd_tier_accept(viasd_model *m, const viasd_draft *draft, const viasd_para
     if (phase & 2) {
         if (!slim_logits || !full_logits) return VIASD_EINVAL;
         if ((rc = timed(m, VIASD_T_TIER_ACCEPT, st, [&] { return launch_accept(m, draft, params, slim_logits, full_logits,
-                                                                          result, st); }))) return rc;
+                                                                          result, tree_ready, st); }))) return rc;
     }
     return VIASD_OK;
+}
+
+int viasd_tier_accept(viasd_model *m, const viasd_draft *draft, const viasd_params *params, const float *slim_logits,
+                      const float *full_logits, int phase, viasd_result *result, void *stream) {
+    return tier_accept_impl(m, draft, params, slim_logits, full_logits, phase, result, false, stream);
 }
 
 int viasd_kv_commit(viasd_model *m, viasd_cache *cache, const viasd_draft *draft, const viasd_result *result,
@@ -490,7 +495,7 @@ int viasd_verify_step(viasd_model *m, viasd_cache *cache, const viasd_draft *dra
     if (m && m->fused && draft && 2 * draft->batch * (draft->n_nodes + 1) <= dual_max) {
         if ((rc = check_draft(m, draft)) || (rc = check_cache(cache))) return rc;
         if ((rc = forward_sweep(m, cache, draft, 2, full_logits, slim_logits, (cudaStream_t)stream))) return rc;
-        if ((rc = viasd_tier_accept(m, draft, params, slim_logits, full_logits, 3, result, stream))) return rc;
+        if ((rc = tier_accept_impl(m, draft, params, slim_logits, full_logits, 3, result, true, stream))) return rc;
         return viasd_kv_commit(m, cache, draft, result, stream);
     }
     if (params->conf_source == 0) {
@@ -501,7 +506,7 @@ int viasd_verify_step(viasd_model *m, viasd_cache *cache, const viasd_draft *dra
         if ((rc = viasd_tier_accept(m, draft, params, slim_logits, nullptr, 1, result, stream))) return rc;
     }
     if ((rc = viasd_full_forward(m, cache, draft, full_logits, stream))) return rc;
-    if ((rc = viasd_tier_accept(m, draft, params, slim_logits, full_logits, 2, result, stream))) return rc;
+    if ((rc = tier_accept_impl(m, draft, params, slim_logits, full_logits, 2, result, true, stream))) return rc;
     return viasd_kv_commit(m, cache, draft, result, stream);
 }
 

@@ -163,7 +163,7 @@ int launch_embed_norm2(const viasd_model *m, const float *gain_full, const float
 int launch_tier(const viasd_model *m, const viasd_draft *d, const viasd_params *p, const float *slim_logits,
                 viasd_result *r, cudaStream_t st);
 int launch_accept(const viasd_model *m, const viasd_draft *d, const viasd_params *p, const float *slim_logits,
-                  const float *full_logits, viasd_result *r, cudaStream_t st);
+                  const float *full_logits, viasd_result *r, bool tree_ready, cudaStream_t st);
 
 // ---------------------------------------------------------------------------------------------
 // small device helpers

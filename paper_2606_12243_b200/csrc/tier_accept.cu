@@ -448,9 +448,11 @@ int launch_tier(const viasd_model *m, const viasd_draft *d, const viasd_params *
 }
 
 int launch_accept(const viasd_model *m, const viasd_draft *d, const viasd_params *p, const float *slim_logits,
-                  const float *full_logits, viasd_result *r, cudaStream_t st) {
-    tree_only_kernel<<<1, 32, 0, st>>>(m->ws.tree, m->ws.stats, d->parent, d->n_nodes);
-    LAUNCH_CHECK();
+                  const float *full_logits, viasd_result *r, bool tree_ready, cudaStream_t st) {
+    if (!tree_ready) {                       // a forward pass of the same call has laid the tree out already
+        tree_only_kernel<<<1, 32, 0, st>>>(m->ws.tree, m->ws.stats, d->parent, d->n_nodes);
+        LAUNCH_CHECK();
+    }
     if (d->n_prows > RS_STRIDE) return VIASD_EINVAL;
     AcceptArgs a;
     {
