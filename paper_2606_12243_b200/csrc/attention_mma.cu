@@ -300,6 +300,15 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
         // committed context does not change during the pass: ask for it before waiting for the previous kernel
         while (p_count < NSTAGE && issue_next(true)) { }
     }
+    // the first item's description and its rows' ancestor sets come from the pass's preparation kernel, long done:
+    // fetch them now, not after the dependency wait, where every dependent global load is a microsecond on the path
+    const Item first_item = i0 < i1 ? decode_item(a, i0) : Item{};
+    unsigned long long anc_first[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const int row = (warp & (a.mt_eff - 1)) * 16 + (lane >> 2) + r * 8;
+        anc_first[r] = row < (a.H / a.Hkv) * a.M ? a.tree->anc[row % a.M] : 0ull;
+    }
     ATRACE(1);
     PDL_WAIT();
     ATRACE(2);
@@ -310,7 +319,7 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
     int q_be = -1, q_g = -1;
     bool ok = true;
     for (int item = i0; item < i1 && ok; ++item) {
-        const Item it = decode_item(a, item);
+        const Item it = item == i0 ? first_item : decode_item(a, item);
         if (it.be != q_be || it.g != q_g) {
             // stage the query rows of this (sequence, kv head) as bf16 hi / lo, pre-scaled
             __syncthreads();
@@ -354,7 +363,7 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
             const int row = mtile * 16 + (lane >> 2) + r * 8;
-            anc[r] = (active && row < QR) ? a.tree->anc[row % a.M] : 0ull;
+            anc[r] = !(active && row < QR) ? 0ull : item == i0 ? anc_first[r] : a.tree->anc[row % a.M];
         }
 #pragma unroll
         for (int n = 0; n < 16; ++n)
