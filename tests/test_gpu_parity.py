@@ -351,8 +351,9 @@ def _check_verify_step(name):
         _check_state(eng, st, wl)
 
 
-def test_step_pieces_equal_fused_call():
-    wl = W.get("mini_8b_tree")
+@pytest.mark.parametrize("name", ["mini_8b_tree", "mini_7b", "mini_13b"])
+def test_step_pieces_equal_fused_call(name):
+    wl = W.get(name)
     vb = _vb()
     outs = []
     for fused in (True, False):
