@@ -380,12 +380,37 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                 dry = false;
                 asm volatile("griddepcontrol.wait;" ::: "memory");     // outputs, scratch and counters belong to the chain
                 if (p.ssq_in) {
-                    // 1/rms per input row: a warp sums the row's partial sums of squares (fixed order: reproducible)
-                    for (int r = (et >> 5); r < p.rows; r += 4) {
-                        float ss = 0.f;
-                        for (int j = lane; j < p.ssq_in_n; j += 32) ss += __ldcg(p.ssq_in + (size_t)j * p.ssq_stride + p.row0 + r);
-                        ss = warp_sum(ss);
-                        if (lane == 0) inv_sh[r] = rsqrtf(ss * p.inv_d + p.eps);
+                    // 1/rms per input row from the row's partial sums of squares, always in one order: 32 lane-strided
+                    // sub-sums, then the shuffle tree's pairing (16, 8, 4, 2, 1) - reproducible whatever the row count.
+                    if (p.rows > 32) {
+                        // a thread per row: adjacent threads read adjacent floats, 32 independent loads at a time.  A
+                        // warp per row (below) is a chain of dependent, uncoalesced loads, a microsecond per row, which
+                        // at a hundred rows outlasted the streaming of the weights.
+                        const float *from = p.ssq_in + p.row0 + min(et, p.rows - 1);
+                        float acc[32];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+#pragma unroll 1
+                        for (int j0 = 0; j0 < p.ssq_in_n; j0 += 32) {
+                            float v[32];
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) v[i] = j0 + i < p.ssq_in_n ? __ldcg(from + (size_t)(j0 + i) * p.ssq_stride) : 0.f;
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) acc[i] += v[i];
+                        }
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+                            for (int i = 0; i < o; ++i) acc[i] += acc[i + o];
+                        }
+                        if (et < p.rows) inv_sh[et] = rsqrtf(acc[0] * p.inv_d + p.eps);
+                    } else {
+                        for (int r = (et >> 5); r < p.rows; r += 4) {
+                            float ss = 0.f;
+                            for (int j = lane; j < p.ssq_in_n; j += 32) ss += __ldcg(p.ssq_in + (size_t)j * p.ssq_stride + p.row0 + r);
+                            ss = warp_sum(ss);
+                            if (lane == 0) inv_sh[r] = rsqrtf(ss * p.inv_d + p.eps);
+                        }
                     }
                 }
                 if (EPI == EPI_QKV_ROPE) {
