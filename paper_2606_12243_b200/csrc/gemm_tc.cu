@@ -16,8 +16,8 @@
 // with bulk copies and sums them in CTA order - bit-reproducible whoever does it.  A contributor that
 // continues into the next tile never waits, so waits cannot chain.
 //
-// Warp roles (192 threads): warp 0 issues TMA loads into a ring of stages, warp 1 allocates TMEM and
-// issues tcgen05.mma, warps 2-5 read the accumulators (tcgen05.ld) and run the epilogue.  Accumulators
+// Warp roles (320 threads): warp 0 issues TMA loads into a ring of stages, warp 1 allocates TMEM and
+// issues tcgen05.mma, warps 2-9 read the accumulators (tcgen05.ld) and run the epilogue.  Accumulators
 // are double-buffered in TMEM so the epilogue of one tile overlaps the main loop of the next.
 // Every wait is bounded: on expiry the CTA records VIASD_EDEVICE, lets its copies land and leaves.
 #include "common.cuh"
@@ -28,8 +28,8 @@
 
 namespace {
 
-template <int EPI>
-__global__ void __launch_bounds__(THREADS, 1)
+template <int EPI, int GROUPS>
+__global__ void __launch_bounds__(64 + 128 * GROUPS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
                const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_x, const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -37,7 +37,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
     __shared__ uint32_t tmem_base_sh;
     __shared__ int abort_sh;
     __shared__ float inv_sh[128];                       // per-row 1/rms of the input (fused RMSNorm)
-    __shared__ float xch[CH * TILE_F];                  // rotary partner exchange
+    __shared__ float xch[GROUPS * CH * TILE_F];         // rotary partner exchange, one buffer per epilogue group
     __shared__ int4 rowmeta[128];                       // per token row: rotary position, cache slot, sequence
 
     constexpr bool DUAL = EPI == EPI_SWIGLU;
@@ -60,8 +60,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
-        mbar_init(gather_bar, 128);
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), GROUPS * 4); }
+        mbar_init(gather_bar, GROUPS * 128);
         abort_sh = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -166,15 +166,31 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
             TRACE(5);
         }
     } else {
-        // ---------------- epilogue (warps 2..5 <-> TMEM lane quarters 2,3,0,1) ----------------
+        // ---------------- epilogue (warps 2..5 and 6..9 <-> TMEM lane quarters 2,3,0,1) ----------------
+        // One or two groups of 128 threads (the launch decides: the second group pays at wide token tiles, where the
+        // finishing is many chunks long, and costs a little at narrow ones); wherever rows are handled chunk by
+        // chunk, the groups take the chunks in turn.
         const int quarter = warp & 3;
         const int f = quarter * 32 + lane;                  // feature lane inside the tile, as TMEM lanes map to warps
-        const int et = threadIdx.x - 64;                    // 0..127 among epilogue threads
+        const int et_all = threadIdx.x - 64;                // 0..255 among epilogue threads
+        const int group = GROUPS > 1 ? et_all >> 7 : 0, et = GROUPS > 1 ? (et_all & 127) : et_all;   // et: the thread's number in its group = its feature in staged tiles
+        constexpr int epi_threads = GROUPS * 128, n_groups = GROUPS;
         const size_t slot_floats = (size_t)NACC * NT * TILE_F;
         // per-row tables (all 128 entries defined: chunks read a few rows past p.rows and discard them)
         inv_sh[et] = 0.f;
         rowmeta[et] = make_int4(0, 0, 0, 0);
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(epi_threads) : "memory");
+        // The tile this CTA's range ends in is the one it will help to finish: what that epilogue reads from
+        // weights (not from the kernel before) is fetched now, off the critical path.
+        const int last_tile = (u_end - 1) / p.k_tiles;
+        float2 last_gain = make_float2(0.f, 0.f);
+        if (EPI == EPI_ADD_NORM) {
+            const int n = last_tile * TILE_F + et;
+            if (n < p.seg_n[0]) {
+                last_gain.x = __ldg(p.next_gain + n);
+                last_gain.y = p.next_gain2 ? __ldg(p.next_gain2 + n) : last_gain.x;
+            }
+        }
 
         // A tile is finished from one of three sources: the accumulator in TMEM (this CTA held all of K), the
         // partials staged in shared memory, or the partials read straight from global memory.  All three feed ONE
@@ -184,7 +200,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
         enum { SRC_DRY, SRC_TMEM, SRC_SMEM, SRC_GLOBAL };
         int acc_it = 0, u = u_begin, seg_i = 0;
         Seg sg;
-        sg.tile = (u_end - 1) / p.k_tiles; sg.ka = 0; sg.kb = 0;   // dry pass: the tile this CTA is most likely to finish
+        sg.tile = last_tile; sg.ka = 0; sg.kb = 0;                 // dry pass: the tile this CTA is most likely to finish
         bool ok = true, dry = true;
         while (ok) {
             int src = SRC_DRY, buf = 0, first_cta = 0, last_cta = 0;
@@ -208,7 +224,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                 } else {
                     // partial of a split tile: slot 0 if the tile is the first one this CTA touches, else slot 1
                     float *slot = p.scratch + ((size_t)blockIdx.x * 2 + (seg_i == 0 ? 0 : 1)) * slot_floats;
-                    for (int c = 0; c < p.rows; c += CH) {       // padding rows beyond p.rows are never read
+                    for (int c = group * CH; c < p.rows; c += n_groups * CH) {   // padding rows beyond p.rows are never read
                         float g[CH], uu[CH];
                         tc_ld8(t0 + c, g);
                         if (DUAL) tc_ld8(t0 + NB + c, uu);
@@ -238,15 +254,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                     // slice of the token rows, summing the partials in CTA order.  A contributor that goes on into the
                     // next tile only arrives and never waits, so no wait depends on another wait.
                     __threadfence();
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    asm volatile("bar.sync 1, %0;" ::"n"(epi_threads) : "memory");
                     first_cta = (sg.tile * p.k_tiles) / p.units_per_cta;
                     last_cta = ((sg.tile + 1) * p.k_tiles - 1) / p.units_per_cta;
-                    if (et == 0) atomicAdd(&p.counters[sg.tile], 1);                  // low half: arrivals
+                    if (et_all == 0) atomicAdd(&p.counters[sg.tile], 1);              // low half: arrivals
                     if (u < u_end) { ++acc_it; ++seg_i; continue; }
                     const int n_c = last_cta - first_cta + 1;
                     const int last_range_end = min(total_units, (last_cta + 1) * p.units_per_cta);
                     const int n_fin = n_c - (last_range_end > (sg.tile + 1) * p.k_tiles ? 1 : 0);
-                    if (et == 0) {
+                    if (et_all == 0) {
                         volatile int *ctr = p.counters + sg.tile;
                         const long long w0 = clock64();
                         while ((*ctr & 0xffff) < n_c) {
@@ -256,7 +272,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                         // high half: finishers that have seen all arrivals; the last of them leaves the counter at zero
                         if (!abort_sh && (atomicAdd(&p.counters[sg.tile], 1 << 16) >> 16) == n_fin - 1) atomicExch(&p.counters[sg.tile], 0);
                     }
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    asm volatile("bar.sync 1, %0;" ::"n"(epi_threads) : "memory");
                     if (et == 0) TRACE(8);
                     if (abort_sh) { ok = false; break; }
                     __threadfence();
@@ -296,17 +312,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                 // rows blk0 .. blk_end-1 of every contributor (and of the epilogue's own inputs) into the ring
                 const int nr = min(p.rows, blk_end) - blk0, n_c = last_cta - first_cta + 1;
                 const uint32_t row_bytes = TILE_F * 4u, aux_sh = smem_base, part_sh = smem_base + (uint32_t)stage_rows * row_bytes;
-                if (round > 0) asm volatile("bar.sync 1, 128;" ::: "memory");    // everyone is done with the previous round's rows
-                const bool has_part = et < n_c * NACC, has_aux = aux_kind && et < nr;
+                if (round > 0) asm volatile("bar.sync 1, %0;" ::"n"(epi_threads) : "memory");    // everyone is done with the previous round's rows
+                const bool has_part = et_all < n_c * NACC, has_aux = aux_kind && et_all < nr;   // nr <= 128: first group
                 asm volatile("fence.proxy.async.global;" ::: "memory");
                 if (has_part || has_aux) {
                     mbar_expect_tx(gather_bar, (has_part ? (uint32_t)nr * row_bytes : 0u) + (has_aux ? row_bytes : 0u));
                     if (has_part) {
-                        const int c = first_cta + et / NACC, half = et - (et / NACC) * NACC;
+                        const int c = first_cta + et_all / NACC, half = et_all - (et_all / NACC) * NACC;
                         const int c_first_tile = (c * p.units_per_cta) / p.k_tiles;
                         const float *from = p.scratch + ((size_t)c * 2 + (c_first_tile == sg.tile ? 0 : 1)) * slot_floats +
                                             (size_t)half * NT * TILE_F + (size_t)blk0 * TILE_F;
-                        bulk_load(part_sh + (uint32_t)et * (uint32_t)stage_rows * row_bytes, from, (uint32_t)nr * row_bytes, gather_bar);
+                        bulk_load(part_sh + (uint32_t)et_all * (uint32_t)stage_rows * row_bytes, from, (uint32_t)nr * row_bytes, gather_bar);
                     }
                     if (has_aux) {
                         const uint32_t dst = aux_sh + (uint32_t)et * row_bytes;
@@ -328,7 +344,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                 if (aux_kind) aux = reinterpret_cast<const float *>(smem_raw + (aux_sh - smem_u32(smem_raw))) - (size_t)blk0 * TILE_F;
             }
 #pragma unroll 1
-            for (int r0 = blk0; r0 < blk_end; r0 += CH) {
+            for (int r0 = blk0 + group * CH; r0 < blk_end; r0 += n_groups * CH) {
                 float g[CH], uu[CH];
 #pragma unroll
                 for (int j = 0; j < CH; ++j) { g[j] = 0.f; uu[j] = 0.f; }
@@ -370,9 +386,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                         }
                     }
                 }
-                if (et == 0 && r0 == 0) TRACE(9);
-                finish_chunk<EPI>(p, sg.tile, fe, r0, g, uu, xch, inv_sh, rowmeta, lane, aux, rows_live);
-                if (et == 0 && r0 == 0) TRACE(15);
+                if (et == 0 && r0 == row_begin) TRACE(9);
+                finish_chunk<EPI, GROUPS>(p, sg.tile, fe, r0, g, uu, xch + group * (CH * TILE_F), inv_sh, rowmeta, lane, aux, rows_live,
+                                  src != SRC_TMEM && sg.tile == last_tile, last_gain, GROUPS > 1 ? 2 + group : 1);
+                if (et == 0 && r0 == row_begin) TRACE(15);
             }
             }   // blocks of rows
 
@@ -383,6 +400,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                     // 1/rms per input row from the row's partial sums of squares, always in one order: 32 lane-strided
                     // sub-sums, then the shuffle tree's pairing (16, 8, 4, 2, 1) - reproducible whatever the row count.
                     if (p.rows > 32) {
+                      if (group == 0) {
                         // a thread per row: adjacent threads read adjacent floats, 32 independent loads at a time.  A
                         // warp per row (below) is a chain of dependent, uncoalesced loads, a microsecond per row, which
                         // at a hundred rows outlasted the streaming of the weights.
@@ -404,8 +422,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                             for (int i = 0; i < o; ++i) acc[i] += acc[i + o];
                         }
                         if (et < p.rows) inv_sh[et] = rsqrtf(acc[0] * p.inv_d + p.eps);
+                      }
                     } else {
-                        for (int r = (et >> 5); r < p.rows; r += 4) {
+                        for (int r = (et_all >> 5); r < p.rows; r += n_groups * 4) {
                             float ss = 0.f;
                             for (int j = lane; j < p.ssq_in_n; j += 32) ss += __ldcg(p.ssq_in + (size_t)j * p.ssq_stride + p.row0 + r);
                             ss = warp_sum(ss);
@@ -414,7 +433,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                     }
                 }
                 if (EPI == EPI_QKV_ROPE) {
-                    if (et < p.rows) {
+                    if (et_all < p.rows) {
                         // rows are laid out [stream][sequence][block row]; stream 1 (rows >= split_row) is the slim verifier
                         const int row = p.row0 + et, stream = row >= p.split_row ? 1 : 0, rs = row - stream * p.split_row;
                         const int b = rs / p.rope_M, i = rs - b * p.rope_M;
@@ -422,7 +441,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                         rowmeta[et] = make_int4(n_ctx + p.depth[i], n_ctx + i, b, stream);
                     }
                 }
-                asm volatile("bar.sync 1, 128;" ::: "memory");
+                asm volatile("bar.sync 1, %0;" ::"n"(epi_threads) : "memory");
                 continue;
             }
             if (src == SRC_TMEM) {
@@ -588,16 +607,20 @@ int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {
     const CUtensorMap &w0 = *L.map_w[0], &w1 = *L.map_w[L.n_seg > 1 ? 1 : 0], &w2 = *L.map_w[L.n_seg > 2 ? 2 : 0];
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
-    pdl_config(cfg, attr, dim3(grid), dim3(THREADS), smem, st);
-    static bool attr_done[4] = {false, false, false, false};
-#define TC_LAUNCH(IDX, KIND)                                                                                          \
+    // a second epilogue group above token tiles of 48 (VIASD_TC_EPI_GROUPS overrides)
+    static const int groups_env = getenv("VIASD_TC_EPI_GROUPS") ? atoi(getenv("VIASD_TC_EPI_GROUPS")) : 0;
+    const int groups = groups_env == 1 || groups_env == 2 ? groups_env : (p.nt > 48 ? 2 : 1);
+    pdl_config(cfg, attr, dim3(grid), dim3(64 + 128 * groups), smem, st);
+    static bool attr_done[8] = {false, false, false, false, false, false, false, false};
+#define TC_LAUNCH_G(IDX, KIND, G)                                                                                     \
     do {                                                                                                              \
         if (!attr_done[IDX]) {                                                                                        \
-            CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, 208 * 1024)); \
+            CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<KIND, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, 208 * 1024)); \
             attr_done[IDX] = true;                                                                                    \
         }                                                                                                             \
-        CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<KIND>, w0, w1, w2, *L.map_x, p));                            \
+        CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<KIND, G>, w0, w1, w2, *L.map_x, p));                         \
     } while (0)
+#define TC_LAUNCH(IDX, KIND) do { if (groups == 2) TC_LAUNCH_G(IDX + 4, KIND, 2); else TC_LAUNCH_G(IDX, KIND, 1); } while (0)
     switch (L.epi) {
     case EPI_SWIGLU: TC_LAUNCH(0, EPI_SWIGLU); break;
     case EPI_ADD_NORM: TC_LAUNCH(1, EPI_ADD_NORM); break;
@@ -605,6 +628,7 @@ int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {
     default: TC_LAUNCH(3, EPI_STORE); break;          // EPI_STORE and EPI_ADD share one kernel
     }
 #undef TC_LAUNCH
+#undef TC_LAUNCH_G
     LAUNCH_CHECK();
     return VIASD_OK;
 }

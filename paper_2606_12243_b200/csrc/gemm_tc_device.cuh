@@ -10,7 +10,6 @@ namespace {
 constexpr int TILE_F = 128;          // output features per tile (MMA M)
 constexpr int TILE_K = 64;           // bf16 per k-block: 128 bytes, one swizzle row
 constexpr int MAX_STAGES = 12;
-constexpr int THREADS = 192;
 
 constexpr int CH = 8;                // token rows per epilogue chunk
 __device__ __forceinline__ void tc_ld8(uint32_t taddr, float (&v)[CH]) {
@@ -56,13 +55,15 @@ __device__ __forceinline__ bool next_seg(int &u, int u1, int k_tiles, Seg &s) {
 // pair) of output feature f.  Called by all 128 epilogue threads together.  The epilogue kind is a template
 // parameter so that each kernel carries one short epilogue: this code runs once per tile, straight from the
 // instruction cache's cold side, and its size is what its latency is made of.
-template <int EPI>
+template <int EPI, int GROUPS>
 __device__ __forceinline__ void finish_chunk(const TcParams &p, int tile, int f, int r0, float (&g)[CH], float (&uu)[CH],
                                              float *xch, const float *inv_sh, const int4 *rowmeta, int lane,
-                                             const float *aux, int rows_live) {
+                                             const float *aux, int rows_live, bool have_gain, float2 gain, int group_bar) {
     // aux: null, or [rows][128] floats already in shared memory - the residual row of this tile (EPI_ADD_NORM),
     // or the row's 64 cosines followed by its 64 sines (EPI_QKV_ROPE) - so that no chunk waits for global memory.
     // rows_live: rows r0.. below it are written (p.rows, or 0 for the dry pass that only warms the instruction cache)
+    // have_gain / gain: the next norm's gains of feature f, fetched by the caller long before (EPI_ADD_NORM)
+    // group_bar: the named barrier of the calling group of 128 threads; xch is that group's exchange buffer
     constexpr bool DUAL = EPI == EPI_SWIGLU;
     if (EPI == EPI_STORE || EPI == EPI_SWIGLU || EPI == EPI_QKV_ROPE) {
         if (p.ssq_in) {                   // the input was h * gain without its RMS factor: apply it per row here
@@ -113,8 +114,10 @@ __device__ __forceinline__ void finish_chunk(const TcParams &p, int tile, int f,
     } else if (EPI == EPI_ADD_NORM) {
         // residual update, plus what the next RMSNorm needs: h * gain as hi/lo planes and partial sums of h^2.
         // Loads first, then arithmetic, then stores: the CH rows cost one memory round trip.
-        const float gain_a = valid ? p.next_gain[n] : 0.f;
-        const float gain_b = (valid && p.next_gain2) ? p.next_gain2[n] : gain_a;
+        // fetched here, the two gains are a round trip to L2 at the head of every chunk (the stores in between keep
+        // the compiler from hoisting them): a microsecond on the launch's critical path
+        const float gain_a = have_gain ? gain.x : (valid ? p.next_gain[n] : 0.f);
+        const float gain_b = have_gain ? gain.y : ((valid && p.next_gain2) ? p.next_gain2[n] : gain_a);
         float *hp = p.out_f32 + (size_t)(p.row0 + r0) * p.ld_out + n;
         __nv_bfloat16 *ap = p.next_act + (size_t)(p.row0 + r0) * p.ld_out + n;
         if (touch) { want(hp); want(ap); want(ap + p.next_plane); want(p.ssq_out + ((size_t)tile * 4 + (f >> 5)) * p.ssq_stride + p.row0 + r0); }
@@ -152,7 +155,7 @@ __device__ __forceinline__ void finish_chunk(const TcParams &p, int tile, int f,
     } else {   // EPI_QKV_ROPE: one tile is one head of 128 dims; rotate pairs (p, p + 64), write q / K cache / V cache
 #pragma unroll
         for (int j = 0; j < CH; ++j) xch[j * TILE_F + f] = g[j];
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (GROUPS == 1) asm volatile("bar.sync 1, 128;" ::: "memory"); else asm volatile("bar.sync %0, 128;" ::"r"(group_bar) : "memory");
         const int head = tile - t0, pidx = f & 63;
         if (s < 2) {
             float c[CH], sn[CH];
@@ -189,7 +192,7 @@ __device__ __forceinline__ void finish_chunk(const TcParams &p, int tile, int f,
                 }
             }
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (GROUPS == 1) asm volatile("bar.sync 1, 128;" ::: "memory"); else asm volatile("bar.sync %0, 128;" ::"r"(group_bar) : "memory");
     }
 }
 
