@@ -147,6 +147,9 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     __shared__ int abort_sh, last_sh;
     __shared__ float wmax_sh[2][4][NR];                     // per tile parity, per warp: row maxima of its 32 keys
     __shared__ float lsum_sh[4][NR];                        // per warp: row sums, once per item
+    __shared__ float mref_sh[4][NR];                        // per warp (each keeps its own copy): the rows' running maxima, 0 while none
+    __shared__ float corr_sh[4][NR];                        // per warp: rescale factors of a tile in which a maximum moved
+    __shared__ float mraw_sh[NR];                           // the rows' running maxima at the end of an item (-inf: no visible key)
     __shared__ unsigned long long anc_sh[VIASD_MAX_ROWS_PER_SEQ];
 
     constexpr int NC = 2 * NR;                              // MMA N: hi rows then lo rows
@@ -336,9 +339,13 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 if (!dry) { q_be = it.be; q_g = it.g; }
                 if (item == i0) ATK_MARK(2);
             }
-            float m_run[NR], l_run[NR];
+            // Lane r of every warp keeps row r's running maximum (the four warps compute the same values); the other
+            // lanes read it, as the exponent's reference, from the warp's copy in shared memory.
+            float m_lane = -INFINITY, l_run[NR];
 #pragma unroll
-            for (int r = 0; r < NR; ++r) { m_run[r] = -INFINITY; l_run[r] = 0.f; }
+            for (int r = 0; r < NR; ++r) l_run[r] = 0.f;
+            if (lane < NR) mref_sh[quarter][lane] = 0.f;
+            __syncwarp();
 
             for (int t = 0; t < it.n_tiles; ++t) {
                 const int sb = s_cnt & 1;
@@ -360,52 +367,63 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     for (int r = 0; r < NR; ++r) if (!((anc_sh[r % a.M] >> tb) & 1ull)) s[r] = -INFINITY;
                 }
                 ATK_ADD(4);
-                // row maxima: over the warp's 32 keys by shuffle, over the four warps through shared memory
+                // row maxima: over the warp's 32 keys by one warp-wide reduction per row (lane r keeps row r's), over the
+                // four warps through shared memory
                 {
                     float mine = -INFINITY;
 #pragma unroll
                     for (int r = 0; r < NR; ++r) {
-                        const float wm = warp_max(s[r]);
-                        if (lane == (r & 31)) mine = wm;
+                        float wm;
+                        asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(wm) : "f"(s[r]));
+                        if (lane == r) mine = wm;
                     }
                     if (lane < NR) wmax_sh[sb][quarter][lane] = mine;
                 }
                 ATK_ADD(5);
                 if (!(ok = wg_sync())) break;
                 ATK_ADD(6);
-                float corr[NR];
-                bool moved = false;
-#pragma unroll
-                for (int r = 0; r < NR; ++r) {
-                    const float mt = fmaxf(fmaxf(wmax_sh[sb][0][r], wmax_sh[sb][1][r]), fmaxf(wmax_sh[sb][2][r], wmax_sh[sb][3][r]));
-                    corr[r] = 1.f;
-                    if (mt > m_run[r] + RESCALE_GAP) {                 // also the first tile with a visible key (m_run = -inf)
-                        if (m_run[r] != -INFINITY) { corr[r] = ex2(m_run[r] - mt); moved = true; }
-                        m_run[r] = mt;
+                bool moved_l = false;
+                if (lane < NR) {
+                    const float mt = fmaxf(fmaxf(wmax_sh[sb][0][lane], wmax_sh[sb][1][lane]), fmaxf(wmax_sh[sb][2][lane], wmax_sh[sb][3][lane]));
+                    float corr = 1.f;
+                    if (mt > m_lane + RESCALE_GAP) {                   // also the first tile with a visible key (m_lane = -inf)
+                        if (m_lane != -INFINITY) { corr = ex2(m_lane - mt); moved_l = true; }
+                        m_lane = mt;
+                        mref_sh[quarter][lane] = mt;
                     }
+                    corr_sh[quarter][lane] = corr;
                 }
-                if (moved && !dry) {
-                    // rare: a running maximum moved.  Every thread sees the same maxima, so all four warps come here
+                const bool moved = __any_sync(0xffffffffu, moved_l);
+                __syncwarp();
+                if (moved) {
+                    // rare: a running maximum moved.  Every warp sees the same maxima, so all four come here
                     // together; O^T is rescaled once the previous tile's MMAs have written it.
-                    if (!(ok = mbar_wait(pvdone_bar(sb ^ 1), ((s_cnt - 1) >> 1) & 1, &abort_sh, a.status))) break;
-                    tc_fence_after();
 #pragma unroll
-                    for (int c = 0; c < NC / 16; ++c) {
-                        uint32_t w[16];
-                        tc_ld16(tlane + TM_O + c * 16, w);
+                    for (int r = 0; r < NR; ++r) l_run[r] *= corr_sh[quarter][r];
+                    if (!dry) {
+                        if (!(ok = mbar_wait(pvdone_bar(sb ^ 1), ((s_cnt - 1) >> 1) & 1, &abort_sh, a.status))) break;
+                        tc_fence_after();
 #pragma unroll
-                        for (int e = 0; e < 16; ++e) w[e] = __float_as_uint(__uint_as_float(w[e]) * corr[(c * 16 + e) % NR]);
-                        tc_st16(tlane + TM_O + c * 16, w);
+                        for (int c = 0; c < NC / 16; ++c) {
+                            uint32_t w[16];
+                            tc_ld16(tlane + TM_O + c * 16, w);
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) w[e] = __float_as_uint(__uint_as_float(w[e]) * corr_sh[quarter][(c * 16 + e) % NR]);
+                            tc_st16(tlane + TM_O + c * 16, w);
+                        }
+                        tc_wait_st();
                     }
-                    tc_wait_st();
                 }
                 ATK_ADD(7);
                 // weights of this key for every row; P^T (hi rows, lo rows) into shared memory for the MMA
                 uint8_t *pchunk = gen + 2 * QCH + (uint32_t)sb * 2 * QCH + (uint32_t)(kl >> 6) * QCH;
+                float mref[NR];                                  // read before the stores below: they could alias, which would
+#pragma unroll                                                   // put every one of these loads behind the previous row's stores
+                for (int r = 0; r < NR; ++r) mref[r] = mref_sh[quarter][r];
 #pragma unroll
                 for (int r = 0; r < NR; ++r) {
-                    const float p = ex2(s[r] - (m_run[r] == -INFINITY ? 0.f : m_run[r]));   // masked scores are -inf: weight 0
-                    l_run[r] = l_run[r] * corr[r] + p;
+                    const float p = ex2(s[r] - mref[r]);                   // masked scores are -inf: weight 0
+                    l_run[r] += p;
                     const __nv_bfloat16 hi = __float2bfloat16_rn(p), lo = __float2bfloat16_rn(p - __bfloat162float(hi));
                     *reinterpret_cast<__nv_bfloat16 *>(pchunk + sw_off(r, kl & 63)) = hi;
                     *reinterpret_cast<__nv_bfloat16 *>(pchunk + sw_off(NR + r, kl & 63)) = lo;
@@ -433,6 +451,7 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     if (lane == (r & 31)) mine = ws;
                 }
                 if (lane < NR) lsum_sh[quarter][lane] = mine;
+                if (quarter == 0 && lane < NR) mraw_sh[lane] = m_lane;
             }
             // the last MMA into O^T of the item (and with it all earlier ones) is complete
             if (!dry && it.n_tiles > 0 && !(ok = mbar_wait(pvdone_bar((s_cnt - 1) & 1), ((s_cnt - 1) >> 1) & 1, &abort_sh, a.status))) break;
@@ -456,7 +475,7 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     } else {
                         float *pdst = a.part + ((((size_t)it.be * a.H + h) * a.M + node) * a.nsplit + it.split) * ROWF;
                         pdst[kl] = o[r];
-                        if (kl == 0) { pdst[HD] = m_run[r] * 0.6931471805599453f; pdst[HD + 1] = l; }   // natural-log units
+                        if (kl == 0) { pdst[HD] = mraw_sh[r] * 0.6931471805599453f; pdst[HD + 1] = l; }   // natural-log units
                     }
                 }
             }
