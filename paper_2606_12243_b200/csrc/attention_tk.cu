@@ -29,7 +29,7 @@ namespace {
 constexpr int HD = 128;                        // head dimension
 constexpr int TKEYS = 128;                     // keys per tile
 constexpr int HALF_BYTES = TKEYS * 128;        // 128 keys x 64 dims of bf16, as one TMA box lands
-constexpr int STAGE_BYTES = 4 * HALF_BYTES;    // K dims 0..63, K dims 64..127, V dims 0..63, V dims 64..127
+constexpr int SLOT_BYTES = 2 * HALF_BYTES;     // one tile of K or of V: dims 0..63, dims 64..127
 constexpr int TK_THREADS = 192;
 constexpr int TK_MAX_STAGE = 3;
 constexpr int ROWF = HD + 2;                   // partial row: 128 numerators, max (natural-log units), sum
@@ -46,7 +46,7 @@ struct AttnTkArgs {
     int *status;
     int M, H, Hkv, max_batch, max_ctx, layer_ord, nsplit;
     int batch, layer_ord2;      // second row stream: rows batch*M.., its own cache and layer ordinal
-    int streams, n_items, items_per_cta, fuse_merge, nstage;
+    int streams, n_items, items_per_cta, fuse_merge, nk, nv;   // nk, nv: ring slots for K tiles and for V tiles
     int *counters;              // arrivals per (stream, sequence, kv head), zero between launches
     float scale;                // log2(e) / sqrt(hd)
     int trace_on;               // trace builds only
@@ -142,7 +142,7 @@ __global__ void __launch_bounds__(TK_THREADS, 1)
 attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                     const __grid_constant__ CUtensorMap map_k2, const __grid_constant__ CUtensorMap map_v2, const AttnTkArgs a) {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) unsigned long long bars[2 * TK_MAX_STAGE + 10];
+    __shared__ __align__(8) unsigned long long bars[4 * TK_MAX_STAGE + 10];
     __shared__ uint32_t tmem_base_sh;
     __shared__ int abort_sh, last_sh;
     __shared__ float wmax_sh[2][4][NR];                     // per tile parity, per warp: row maxima of its 32 keys
@@ -153,24 +153,29 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     __shared__ unsigned long long anc_sh[VIASD_MAX_ROWS_PER_SEQ];
 
     constexpr int NC = 2 * NR;                              // MMA N: hi rows then lo rows
+    constexpr bool SPLIT = NR == 32;                        // K and V tiles in rings of their own (else a slot holds a tile's K and V)
     constexpr uint32_t QCH = (uint32_t)NC * 128u;           // one 64-wide chunk of an [NC rows] operand
     PDL_TRIGGER();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int NSTAGE = a.nstage;
+    const int NK = a.nk, NV = a.nv;
     const int grp = a.H / a.Hkv, QR = grp * a.M;
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t qsm = base, psm = base + 2 * QCH, ring = base + 6 * QCH;   // Q (2 chunks), P^T (2 buffers x 2 chunks), ring
     uint8_t *gen = smem_raw + (base - smem_u32(smem_raw));
-    auto full_bar = [&](int s) { return smem_u32(&bars[s]); };
-    auto empty_bar = [&](int s) { return smem_u32(&bars[TK_MAX_STAGE + s]); };
-    auto sfull_bar = [&](int b) { return smem_u32(&bars[2 * TK_MAX_STAGE + b]); };
-    auto pfull_bar = [&](int b) { return smem_u32(&bars[2 * TK_MAX_STAGE + 2 + b]); };
-    auto pvdone_bar = [&](int b) { return smem_u32(&bars[2 * TK_MAX_STAGE + 4 + b]); };
-    const uint32_t ofree_bar = smem_u32(&bars[2 * TK_MAX_STAGE + 6]), qfull_bar = smem_u32(&bars[2 * TK_MAX_STAGE + 7]);
-    const uint32_t wg_bar = smem_u32(&bars[2 * TK_MAX_STAGE + 8]);      // the softmax warps among themselves (bounded)
+    // K tiles and V tiles have rings of their own: a K slot is free as soon as S^T = K Q^T has read it, long before the
+    // tile's V, so the next K tiles are on their way while the softmax of the current one runs
+    auto fullk_bar = [&](int s) { return smem_u32(&bars[s]); };
+    auto emptyk_bar = [&](int s) { return smem_u32(&bars[TK_MAX_STAGE + s]); };
+    auto fullv_bar = [&](int s) { return smem_u32(&bars[2 * TK_MAX_STAGE + s]); };
+    auto emptyv_bar = [&](int s) { return smem_u32(&bars[3 * TK_MAX_STAGE + s]); };
+    auto sfull_bar = [&](int b) { return smem_u32(&bars[4 * TK_MAX_STAGE + b]); };
+    auto pfull_bar = [&](int b) { return smem_u32(&bars[4 * TK_MAX_STAGE + 2 + b]); };
+    auto pvdone_bar = [&](int b) { return smem_u32(&bars[4 * TK_MAX_STAGE + 4 + b]); };
+    const uint32_t ofree_bar = smem_u32(&bars[4 * TK_MAX_STAGE + 6]), qfull_bar = smem_u32(&bars[4 * TK_MAX_STAGE + 7]);
+    const uint32_t wg_bar = smem_u32(&bars[4 * TK_MAX_STAGE + 8]);      // the softmax warps among themselves (bounded)
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < NSTAGE; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int s = 0; s < TK_MAX_STAGE; ++s) { mbar_init(fullk_bar(s), 1); mbar_init(emptyk_bar(s), 1); mbar_init(fullv_bar(s), 1); mbar_init(emptyv_bar(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(sfull_bar(b), 1); mbar_init(pfull_bar(b), 4); mbar_init(pvdone_bar(b), 1); }
         mbar_init(ofree_bar, 4);
         mbar_init(qfull_bar, 4);
@@ -193,31 +198,77 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     if (warp == 0) {
         // ---------------- TMA producer: the CTA's (item, tile) list, flattened ----------------
         if (lane == 0) {
-            int p_item = i0, p_tile = 0, p_count = 0;
-            bool ok = true;
-            Item pit = i0 < i1 ? decode_item(a, i0) : Item{};
-            auto issue_next = [&](bool context_only) -> bool {  // false: nothing (more) to request under this condition
-                while (p_item < i1 && p_tile >= pit.n_tiles) { ++p_item; p_tile = 0; if (p_item < i1) pit = decode_item(a, p_item); }
-                if (p_item >= i1) return false;
-                const int k0 = pit.k_begin + p_tile * TKEYS;
-                if (context_only && k0 + TKEYS > pit.n_ctx) return false;   // this tile holds rows the previous kernel writes
-                const int st = p_count % NSTAGE;
-                if (p_count >= NSTAGE && !(ok = mbar_wait(empty_bar(st), ((p_count / NSTAGE) & 1) ^ 1, &abort_sh, a.status))) return false;
-                const uint32_t bar = full_bar(st), dst = ring + st * STAGE_BYTES;
-                const CUtensorMap *mk = pit.stream ? &map_k2 : &map_k, *mv = pit.stream ? &map_v2 : &map_v;
-                const int y = pit.row_base + k0;
-                mbar_expect_tx(bar, STAGE_BYTES);
-                tma_load_2d(dst, mk, bar, 0, y);
-                tma_load_2d(dst + HALF_BYTES, mk, bar, 64, y);
-                tma_load_2d(dst + 2 * HALF_BYTES, mv, bar, 0, y);
-                tma_load_2d(dst + 3 * HALF_BYTES, mv, bar, 64, y);
-                ++p_tile; ++p_count;
-                return true;
+            if constexpr (!SPLIT) {
+                // few query rows: a tile's K and V share a ring slot and are requested together
+                int p_item = i0, p_tile = 0, p_count = 0;
+                bool ok = true;
+                Item pit = i0 < i1 ? decode_item(a, i0) : Item{};
+                auto issue_next = [&](bool context_only) -> bool {  // false: nothing (more) to request under this condition
+                    while (p_item < i1 && p_tile >= pit.n_tiles) { ++p_item; p_tile = 0; if (p_item < i1) pit = decode_item(a, p_item); }
+                    if (p_item >= i1) return false;
+                    const int k0 = pit.k_begin + p_tile * TKEYS;
+                    if (context_only && k0 + TKEYS > pit.n_ctx) return false;   // this tile holds rows the previous kernel writes
+                    const int st = p_count % NK;
+                    if (p_count >= NK && !(ok = mbar_wait(emptyk_bar(st), ((p_count / NK) & 1) ^ 1, &abort_sh, a.status))) return false;
+                    const uint32_t bar = fullk_bar(st), dst = ring + st * 2 * SLOT_BYTES;
+                    const CUtensorMap *mk = pit.stream ? &map_k2 : &map_k, *mv = pit.stream ? &map_v2 : &map_v;
+                    const int y = pit.row_base + k0;
+                    mbar_expect_tx(bar, 2 * SLOT_BYTES);
+                    tma_load_2d(dst, mk, bar, 0, y);
+                    tma_load_2d(dst + HALF_BYTES, mk, bar, 64, y);
+                    tma_load_2d(dst + 2 * HALF_BYTES, mv, bar, 0, y);
+                    tma_load_2d(dst + 3 * HALF_BYTES, mv, bar, 64, y);
+                    ++p_tile; ++p_count;
+                    return true;
+                };
+                // committed context does not change during the pass: ask for it before waiting for the previous kernel
+                while (p_count < NK && issue_next(true)) { }
+                PDL_WAIT();
+                while (ok && issue_next(false)) { }
+            } else {
+            struct Cursor { int item, tile, count; Item it; };
+            Cursor ck{i0, 0, 0, i0 < i1 ? decode_item(a, i0) : Item{}}, cv = ck;
+            // 1: requested; 0: the slot is still being read; -1: nothing (more) to request under this condition
+            auto request = [&](Cursor &c, bool is_v, bool context_only, bool block) -> int {
+                while (c.item < i1 && c.tile >= c.it.n_tiles) { ++c.item; c.tile = 0; if (c.item < i1) c.it = decode_item(a, c.item); }
+                if (c.item >= i1) return -1;
+                const int k0 = c.it.k_begin + c.tile * TKEYS;
+                if (context_only && k0 + TKEYS > c.it.n_ctx) return -1;     // this tile holds rows the previous kernel writes
+                const int n = is_v ? NV : NK, st = c.count % n;
+                if (c.count >= n) {
+                    const uint32_t eb = is_v ? emptyv_bar(st) : emptyk_bar(st), par = ((c.count / n) & 1) ^ 1;
+                    if (block) { if (!mbar_wait(eb, par, &abort_sh, a.status)) return -1; }
+                    else if (!mbar_test(eb, par)) return 0;
+                }
+                const uint32_t bar = is_v ? fullv_bar(st) : fullk_bar(st), dst = ring + (uint32_t)(is_v ? NK + st : st) * SLOT_BYTES;
+                const CUtensorMap *mp = is_v ? (c.it.stream ? &map_v2 : &map_v) : (c.it.stream ? &map_k2 : &map_k);
+                const int y = c.it.row_base + k0;
+                mbar_expect_tx(bar, SLOT_BYTES);
+                tma_load_2d(dst, mp, bar, 0, y);
+                tma_load_2d(dst + HALF_BYTES, mp, bar, 64, y);
+                ++c.tile; ++c.count;
+                return 1;
             };
             // committed context does not change during the pass: ask for it before waiting for the previous kernel
-            while (p_count < NSTAGE && issue_next(true)) { }
+            while (ck.count < NK && request(ck, false, true, false) == 1) { }
+            while (cv.count < NV && request(cv, true, true, false) == 1) { }
             PDL_WAIT();
-            while (ok && issue_next(false)) { }
+            // K first, then V, whichever has a free slot; bounded like every wait: no request for too long ends the CTA
+            long long t_last = clock64();
+            int rk = 0, rv = 0;
+            while (rk >= 0 || rv >= 0) {
+                if (rk >= 0) rk = request(ck, false, false, false);
+                if (rv >= 0) rv = request(cv, true, false, false);
+                if (rk == 1 || rv == 1) { t_last = clock64(); continue; }
+                if (*(volatile int *)&abort_sh) break;
+                if (clock64() - t_last > WAIT_LIMIT_CYCLES) { abort_sh = 1; atomicExch(a.status, VIASD_EDEVICE); break; }
+                // nothing to request right now: sleep on the slot that frees first (K's while K has tiles left); the
+                // hardware wakes the thread when the phase completes or after its own short limit (a suspend-time
+                // hint woke it late, not early: 0.25 us per tile)
+                if (rk == 0) mbar_try_wait(emptyk_bar(ck.count % NK), ((ck.count / NK) & 1) ^ 1);
+                else mbar_try_wait(emptyv_bar(cv.count % NV), ((cv.count / NV) & 1) ^ 1);
+            }
+            }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
@@ -226,16 +277,17 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             const uint32_t idesc_pv = idesc | (1u << 15);                 // A (the V tile) is MN-major
             int c_tile = 0, n_q = 0, o_uses = 0, q_be = -1, q_g = -1;   // c_tile: tiles of earlier items (ring and buffer phase)
             bool ok = true;
-            // tile g (counted over the whole CTA) uses stage g % NSTAGE, S^T buffer g & 1 and P^T buffer g & 1
+            // tile g (counted over the whole CTA) uses K slot g % NK, V slot g % NV, S^T buffer g & 1 and P^T buffer g & 1
             auto issue_qk = [&](int g) -> bool {
-                const int st = g % NSTAGE, sb = g & 1;
-                if (!mbar_wait(full_bar(st), (g / NSTAGE) & 1, &abort_sh, a.status)) return false;
+                const int st = g % NK, sb = g & 1;
+                if (!mbar_wait(fullk_bar(st), (g / NK) & 1, &abort_sh, a.status)) return false;
                 tc_fence_after();
-                const uint32_t kst = ring + st * STAGE_BYTES, d = tmem + TM_S + sb * 64;
+                const uint32_t kst = ring + st * (SPLIT ? 1 : 2) * SLOT_BYTES, d = tmem + TM_S + sb * 64;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)
                     tc_mma(d, smem_desc(kst + (ks >> 2) * HALF_BYTES + (ks & 3) * 32), smem_desc(qsm + (ks >> 2) * QCH + (ks & 3) * 32),
                            idesc, ks > 0 ? 1u : 0u);
+                if (SPLIT) tc_commit(emptyk_bar(st));                     // the K slot is free once these MMAs have read it
                 tc_commit(sfull_bar(sb));
                 return true;
             };
@@ -251,16 +303,18 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 if (!(ok = issue_qk(c_tile))) break;
                 if (it.n_tiles > 1 && !(ok = issue_qk(c_tile + 1))) break;
                 for (int t = 0; t < it.n_tiles; ++t) {
-                    const int g = c_tile + t, sb = g & 1, st = g % NSTAGE;
+                    const int g = c_tile + t, sb = g & 1, st = g % NV;
                     if (t == 0 && o_uses > 0 && !(ok = mbar_wait(ofree_bar, (o_uses - 1) & 1, &abort_sh, a.status))) break;
+                    if (SPLIT && !(ok = mbar_wait(fullv_bar(st), (g / NV) & 1, &abort_sh, a.status))) break;
                     if (!(ok = mbar_wait(pfull_bar(sb), (g >> 1) & 1, &abort_sh, a.status))) break;
                     tc_fence_after();
-                    const uint32_t vst = ring + st * STAGE_BYTES + 2 * HALF_BYTES, pb = psm + sb * 2 * QCH;
+                    const uint32_t vst = SPLIT ? ring + (uint32_t)(NK + st) * SLOT_BYTES : ring + (uint32_t)(2 * st + 1) * SLOT_BYTES;
+                    const uint32_t pb = psm + sb * 2 * QCH;
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk)                        // 16 keys per step: two 8-key groups of 1024 bytes
                         tc_mma(tmem + TM_O, smem_desc_mn(vst + kk * 2048, HALF_BYTES, 1024),
                                smem_desc(pb + (kk >> 2) * QCH + (kk & 3) * 32), idesc_pv, (t > 0 || kk > 0) ? 1u : 0u);
-                    tc_commit(empty_bar(st));                             // the stage is free once these MMAs have read it
+                    tc_commit(SPLIT ? emptyv_bar(st) : emptyk_bar(st));   // the slot is free once these MMAs have read it
                     tc_commit(pvdone_bar(sb));
                     if (t + 2 < it.n_tiles && !(ok = issue_qk(g + 2))) break;
                 }
@@ -611,13 +665,24 @@ int launch_attention_tk(viasd_model *m, const void *kc, const void *vc, bool sli
     a.items_per_cta = (a.n_items + grid - 1) / grid;
     grid = (a.n_items + a.items_per_cta - 1) / a.items_per_cta;
     const size_t op_bytes = 6 * (size_t)(2 * nr) * 128;            // Q (2 chunks) and two P^T buffers (2 chunks each)
-    a.nstage = 1024 + op_bytes + 3 * (size_t)STAGE_BYTES <= 220 * 1024 ? 3 : 2;
-    const size_t smem = 1024 + op_bytes + a.nstage * (size_t)STAGE_BYTES;
+    // 32 query rows: the softmax of a tile is long, so K tiles get slots of their own, released by S^T = K Q^T, and the
+    // tile after next is on its way meanwhile.  With fewer rows this measured slower than a slot per (K, V) pair.
+    const size_t smem_max = 222 * 1024;
+    size_t smem;
+    if (nr == 32) {
+        int slots = (int)((smem_max - 1024 - op_bytes) / SLOT_BYTES);
+        if (slots > 2 * TK_MAX_STAGE) slots = 2 * TK_MAX_STAGE;
+        a.nk = (slots + 1) / 2; a.nv = slots / 2;
+        smem = 1024 + op_bytes + (size_t)slots * SLOT_BYTES;
+    } else {
+        a.nk = a.nv = 1024 + op_bytes + 3 * (size_t)(2 * SLOT_BYTES) <= 220 * 1024 ? 3 : 2;
+        smem = 1024 + op_bytes + a.nk * (size_t)(2 * SLOT_BYTES);
+    }
     static bool attr_done = false;
     if (!attr_done) {
-        CUDA_TRY(cudaFuncSetAttribute(attention_tk_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
-        CUDA_TRY(cudaFuncSetAttribute(attention_tk_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
-        CUDA_TRY(cudaFuncSetAttribute(attention_tk_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+        CUDA_TRY(cudaFuncSetAttribute(attention_tk_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024));
+        CUDA_TRY(cudaFuncSetAttribute(attention_tk_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024));
+        CUDA_TRY(cudaFuncSetAttribute(attention_tk_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024));
         attr_done = true;
     }
     cudaLaunchConfig_t cfg;
