@@ -216,7 +216,18 @@ static int mma_attention(viasd_model *m, const void *kc, const void *vc, bool sl
     const int n_part = nsplit * reps;        // key ranges per (row, head) that have to be merged
     const bool fuse = n_part > 1 && n_part <= 32 && QR * n_part <= 160;
     int rc;
-    if (use == 2) rc = launch_attention_tk(m, kc, vc, slim, layer_ord, kc2, vc2, layer_ord2, streams, batch, M, nsplit, fuse ? 1 : 0, st);
+    if (use == 2) {
+        // The keys-on-lanes kernel deals tiles, not key ranges, evenly to the CTAs (nsplit 0) when the partial buffer
+        // has its 16 slots per (row, head): whole (sequence, head) items leave SMs idle (320 items on 148 SMs: a
+        // quarter of them).  Its merges are then always fused.  Not with more than 16 query rows per kv head: there an
+        // item's fixed cost (staging 32 rows of queries, 32 rows of results) is worth a dozen tiles, and the extra
+        // item per CTA cost more than the balance won (32B batch-16 step 36.5 -> 39.0 ms).  VIASD_TK_FLAT=0/1 overrides.
+        const char *e = getenv("VIASD_TK_FLAT");
+        const size_t need = (size_t)streams * batch * c.n_heads * M * 16 * (c.head_dim + 2) * sizeof(float);
+        if ((e ? atoi(e) != 0 : QR <= 16) && need <= m->ws.part_bytes)
+            return launch_attention_tk(m, kc, vc, slim, layer_ord, kc2, vc2, layer_ord2, streams, batch, M, 0, 1, st);
+        rc = launch_attention_tk(m, kc, vc, slim, layer_ord, kc2, vc2, layer_ord2, streams, batch, M, nsplit, fuse ? 1 : 0, st);
+    }
     else if (use == 1) rc = launch_attention_tc(m, kc, vc, slim, layer_ord, kc2, vc2, layer_ord2, streams, batch, M, nsplit, fuse ? 1 : 0, st);
     else rc = launch_attention_mma(m, kc, vc, slim, layer_ord, kc2, vc2, layer_ord2, streams, batch, M, nsplit, fuse ? 1 : 0, st);
     if (rc || n_part == 1 || fuse) return rc;

@@ -47,16 +47,18 @@ struct AttnTkArgs {
     int M, H, Hkv, max_batch, max_ctx, layer_ord, nsplit;
     int batch, layer_ord2;      // second row stream: rows batch*M.., its own cache and layer ordinal
     int streams, n_items, items_per_cta, fuse_merge, nk, nv;   // nk, nv: ring slots for K tiles and for V tiles
+    int flat, part_slots;       // flat: tiles (not key ranges) are dealt evenly to the CTAs; part_slots: partial slots per (row, head)
     int *counters;              // arrivals per (stream, sequence, kv head), zero between launches
     float scale;                // log2(e) / sqrt(hd)
     int trace_on;               // trace builds only
 };
 
-struct Item { int be, b, g, stream, split, n_ctx, k_begin, k_end, n_tiles, row_base; };
+struct Item { int be, b, g, stream, split, n_split, n_ctx, k_begin, k_end, n_tiles, row_base; };   // split of n_split key ranges of the pair
 
 __device__ __forceinline__ Item decode_item(const AttnTkArgs &a, int item) {
     Item it;
     it.split = item % a.nsplit;
+    it.n_split = a.nsplit;
     const int bg = item / a.nsplit;
     it.g = bg % a.Hkv;
     it.be = bg / a.Hkv;
@@ -71,6 +73,46 @@ __device__ __forceinline__ Item decode_item(const AttnTkArgs &a, int item) {
     it.n_tiles = it.k_end > it.k_begin ? (it.k_end - it.k_begin + TKEYS - 1) / TKEYS : 0;
     it.row_base = (((it.stream ? a.layer_ord2 : a.layer_ord) * a.max_batch + it.b) * a.Hkv + it.g) * a.max_ctx;
     return it;
+}
+
+// The CTA's work list, one item after the other.  Two ways of cutting the work:
+//  - a.flat == 0: every (sequence, kv head) pair is cut into a.nsplit key ranges, and the ranges are dealt to the CTAs
+//    in equal contiguous shares (whole items: 320 items on 148 SMs leave a quarter of the SMs idle);
+//  - a.flat == 1: the tiles of all pairs of a row stream, laid end to end, are cut into one range of `per` tiles per
+//    CTA; a pair that straddles a cut gets one key range per CTA it reaches.  The cuts depend on the lengths, the
+//    number of kv heads and the grid only, so a one-stream launch and a two-stream launch (each CTA takes its
+//    range of both streams) cut the same pairs at the same keys and produce the same bits.
+struct ItemSrc { int item, i1, s, b, g, off; };
+__device__ __forceinline__ void src_init(const AttnTkArgs &a, ItemSrc &c) {
+    c.item = blockIdx.x * a.items_per_cta;
+    c.i1 = min(a.n_items, c.item + a.items_per_cta);
+    c.s = c.b = c.g = c.off = 0;
+}
+__device__ __forceinline__ bool next_item(const AttnTkArgs &a, int per, ItemSrc &c, Item &it) {
+    if (!a.flat) {
+        if (c.item >= c.i1) return false;
+        it = decode_item(a, c.item++);
+        return true;
+    }
+    const int lo = blockIdx.x * per, hi = lo + per;
+    while (c.s < a.streams) {
+        if (c.b >= a.batch || c.off >= hi) { ++c.s; c.b = c.g = c.off = 0; continue; }   // done with this stream
+        const int n_ctx = a.len_eff[c.b], Tk = n_ctx + a.M, tb = (Tk + TKEYS - 1) / TKEYS;
+        if (c.off + a.Hkv * tb <= lo) { c.off += a.Hkv * tb; ++c.b; c.g = 0; continue; }    // this sequence ends before the range
+        if (c.g == 0 && c.off < lo) c.g = (lo - c.off) / tb;                                // its first pair that reaches into the range
+        const int p_lo = c.off + c.g * tb;
+        if (c.g >= a.Hkv) { c.off += a.Hkv * tb; ++c.b; c.g = 0; continue; }
+        if (p_lo >= hi) { ++c.s; c.b = c.g = c.off = 0; continue; }
+        const int p_hi = p_lo + tb, t0 = max(lo, p_lo) - p_lo, t1 = min(hi, p_hi) - p_lo;
+        const int first = p_lo / per, last = (p_hi - 1) / per;
+        it.b = c.b; it.stream = c.s; it.be = c.s * a.batch + c.b; it.g = c.g;
+        it.split = (int)blockIdx.x - first; it.n_split = last - first + 1;
+        it.n_ctx = n_ctx; it.k_begin = t0 * TKEYS; it.k_end = min(Tk, t1 * TKEYS); it.n_tiles = t1 - t0;
+        it.row_base = (((c.s ? a.layer_ord2 : a.layer_ord) * a.max_batch + c.b) * a.Hkv + c.g) * a.max_ctx;
+        ++c.g;
+        return true;
+    }
+    return false;
 }
 
 __device__ __forceinline__ float ex2(float x) {            // 2^x, hardware approximation (2 ulp)
@@ -144,9 +186,8 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) unsigned long long bars[4 * TK_MAX_STAGE + 10];
     __shared__ uint32_t tmem_base_sh;
-    __shared__ int abort_sh, last_sh;
+    __shared__ int abort_sh, last_sh, per_sh;
     __shared__ float wmax_sh[2][4][NR];                     // per tile parity, per warp: row maxima of its 32 keys
-    __shared__ float lsum_sh[4][NR];                        // per warp: row sums, once per item
     __shared__ float mref_sh[4][NR];                        // per warp (each keeps its own copy): the rows' running maxima, 0 while none
     __shared__ float corr_sh[4][NR];                        // per warp: rescale factors of a tile in which a maximum moved
     __shared__ float mraw_sh[NR];                           // the rows' running maxima at the end of an item (-inf: no visible key)
@@ -185,6 +226,12 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    if (threadIdx.x == 64) {
+        // tiles per CTA when the tiles are dealt evenly: a pair may not be cut into more ranges than it has partial slots
+        int T = 0, tmax = 1;
+        if (a.flat) for (int b = 0; b < a.batch; ++b) { const int tb = (a.len_eff[b] + a.M + TKEYS - 1) / TKEYS; T += a.Hkv * tb; tmax = max(tmax, tb); }
+        per_sh = max(max((T + (int)gridDim.x - 1) / (int)gridDim.x, (tmax + a.part_slots - 2) / (a.part_slots - 1)), 1);
+    }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_sh)), "r"(256) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -193,19 +240,22 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_base_sh;
-    const int i0 = blockIdx.x * a.items_per_cta, i1 = min(a.n_items, i0 + a.items_per_cta);
+    const int per = per_sh;
 
     if (warp == 0) {
         // ---------------- TMA producer: the CTA's (item, tile) list, flattened ----------------
         if (lane == 0) {
             if constexpr (!SPLIT) {
                 // few query rows: a tile's K and V share a ring slot and are requested together
-                int p_item = i0, p_tile = 0, p_count = 0;
+                int p_tile = 0, p_count = 0;
                 bool ok = true;
-                Item pit = i0 < i1 ? decode_item(a, i0) : Item{};
+                ItemSrc src;
+                src_init(a, src);
+                Item pit;
+                bool p_more = next_item(a, per, src, pit);
                 auto issue_next = [&](bool context_only) -> bool {  // false: nothing (more) to request under this condition
-                    while (p_item < i1 && p_tile >= pit.n_tiles) { ++p_item; p_tile = 0; if (p_item < i1) pit = decode_item(a, p_item); }
-                    if (p_item >= i1) return false;
+                    while (p_more && p_tile >= pit.n_tiles) { p_tile = 0; p_more = next_item(a, per, src, pit); }
+                    if (!p_more) return false;
                     const int k0 = pit.k_begin + p_tile * TKEYS;
                     if (context_only && k0 + TKEYS > pit.n_ctx) return false;   // this tile holds rows the previous kernel writes
                     const int st = p_count % NK;
@@ -226,20 +276,20 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 PDL_WAIT();
                 while (ok && issue_next(false)) { }
             } else {
-            struct Cursor { int item, tile, count; Item it; };
-            Cursor ck{i0, 0, 0, i0 < i1 ? decode_item(a, i0) : Item{}}, cv = ck;
+            struct Cursor { ItemSrc src; bool more; int tile, count; Item it; };
+            Cursor ck;
+            src_init(a, ck.src);
+            ck.tile = ck.count = 0;
+            ck.more = next_item(a, per, ck.src, ck.it);
+            Cursor cv = ck;
             // 1: requested; 0: the slot is still being read; -1: nothing (more) to request under this condition
-            auto request = [&](Cursor &c, bool is_v, bool context_only, bool block) -> int {
-                while (c.item < i1 && c.tile >= c.it.n_tiles) { ++c.item; c.tile = 0; if (c.item < i1) c.it = decode_item(a, c.item); }
-                if (c.item >= i1) return -1;
+            auto request = [&](Cursor &c, bool is_v, bool context_only) -> int {
+                while (c.more && c.tile >= c.it.n_tiles) { c.tile = 0; c.more = next_item(a, per, c.src, c.it); }
+                if (!c.more) return -1;
                 const int k0 = c.it.k_begin + c.tile * TKEYS;
                 if (context_only && k0 + TKEYS > c.it.n_ctx) return -1;     // this tile holds rows the previous kernel writes
                 const int n = is_v ? NV : NK, st = c.count % n;
-                if (c.count >= n) {
-                    const uint32_t eb = is_v ? emptyv_bar(st) : emptyk_bar(st), par = ((c.count / n) & 1) ^ 1;
-                    if (block) { if (!mbar_wait(eb, par, &abort_sh, a.status)) return -1; }
-                    else if (!mbar_test(eb, par)) return 0;
-                }
+                if (c.count >= n && !mbar_test(is_v ? emptyv_bar(st) : emptyk_bar(st), ((c.count / n) & 1) ^ 1)) return 0;
                 const uint32_t bar = is_v ? fullv_bar(st) : fullk_bar(st), dst = ring + (uint32_t)(is_v ? NK + st : st) * SLOT_BYTES;
                 const CUtensorMap *mp = is_v ? (c.it.stream ? &map_v2 : &map_v) : (c.it.stream ? &map_k2 : &map_k);
                 const int y = c.it.row_base + k0;
@@ -250,15 +300,15 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 return 1;
             };
             // committed context does not change during the pass: ask for it before waiting for the previous kernel
-            while (ck.count < NK && request(ck, false, true, false) == 1) { }
-            while (cv.count < NV && request(cv, true, true, false) == 1) { }
+            while (ck.count < NK && request(ck, false, true) == 1) { }
+            while (cv.count < NV && request(cv, true, true) == 1) { }
             PDL_WAIT();
             // K first, then V, whichever has a free slot; bounded like every wait: no request for too long ends the CTA
             long long t_last = clock64();
             int rk = 0, rv = 0;
             while (rk >= 0 || rv >= 0) {
-                if (rk >= 0) rk = request(ck, false, false, false);
-                if (rv >= 0) rv = request(cv, true, false, false);
+                if (rk >= 0) rk = request(ck, false, false);
+                if (rv >= 0) rv = request(cv, true, false);
                 if (rk == 1 || rv == 1) { t_last = clock64(); continue; }
                 if (*(volatile int *)&abort_sh) break;
                 if (clock64() - t_last > WAIT_LIMIT_CYCLES) { abort_sh = 1; atomicExch(a.status, VIASD_EDEVICE); break; }
@@ -291,8 +341,10 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 tc_commit(sfull_bar(sb));
                 return true;
             };
-            for (int item = i0; item < i1 && ok; ++item) {
-                const Item it = decode_item(a, item);
+            ItemSrc src;
+            src_init(a, src);
+            Item it;
+            while (ok && next_item(a, per, src, it)) {
                 if (it.be != q_be || it.g != q_g) {
                     if (!(ok = mbar_wait(qfull_bar, n_q & 1, &abort_sh, a.status))) break;
                     ++n_q; q_be = it.be; q_g = it.g;
@@ -342,9 +394,18 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         // roles, nothing stored.  A launch runs this code only a few times per CTA, and the first time through comes
         // from a cold instruction cache (several microseconds); the dry item takes that hit before the kernel's
         // predecessor has finished.
-        for (int item = i0 - 1; item < i1 && ok; ++item) {
-            const bool dry = item < i0;
-            if (item == i0) {
+        ItemSrc src;
+        src_init(a, src);
+        for (int n_item = -1; ok; ++n_item) {
+            const bool dry = n_item < 0;
+            Item it;
+            if (dry) {
+                it.be = it.b = it.g = it.stream = it.split = it.row_base = it.k_begin = 0;
+                it.n_ctx = it.k_end = TKEYS; it.n_tiles = 1; it.n_split = 1;
+            } else if (!next_item(a, per, src, it)) {
+                break;
+            }
+            if (n_item == 0) {
                 PDL_WAIT();
                 ATK_MARK(1);
 #ifdef VIASD_TC_TRACE
@@ -352,13 +413,6 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 #endif
                 if (et < a.M) anc_sh[et] = a.tree->anc[et];
                 if (!(ok = wg_sync())) break;                         // anc_sh is visible
-            }
-            Item it;
-            if (dry) {
-                it.be = it.b = it.g = it.stream = it.split = it.row_base = it.k_begin = 0;
-                it.n_ctx = it.k_end = TKEYS; it.n_tiles = 1;
-            } else {
-                it = decode_item(a, item);
             }
             const int QRW = dry ? 0 : QR;                              // rows whose result is written
             if (dry || it.be != q_be || it.g != q_g) {
@@ -391,7 +445,7 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 __syncwarp();
                 if (lane == 0 && !dry) mbar_arrive(qfull_bar);
                 if (!dry) { q_be = it.be; q_g = it.g; }
-                if (item == i0) ATK_MARK(2);
+                if (n_item == 0) ATK_MARK(2);
             }
             // Lane r of every warp keeps row r's running maximum (the four warps compute the same values); the other
             // lanes read it, as the exponent's reference, from the warp's copy in shared memory.
@@ -496,21 +550,11 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             if (!ok) break;
             ATK_T0();
             // ---- the item's result ----
-            // row sums: per warp by shuffle, across the warps through shared memory
-            {
-                float mine = 0.f;
-#pragma unroll
-                for (int r = 0; r < NR; ++r) {
-                    const float ws = warp_sum(l_run[r]);
-                    if (lane == (r & 31)) mine = ws;
-                }
-                if (lane < NR) lsum_sh[quarter][lane] = mine;
-                if (quarter == 0 && lane < NR) mraw_sh[lane] = m_lane;
-            }
+            if (quarter == 0 && lane < NR) mraw_sh[lane] = m_lane;
             // the last MMA into O^T of the item (and with it all earlier ones) is complete
             if (!dry && it.n_tiles > 0 && !(ok = mbar_wait(pvdone_bar((s_cnt - 1) & 1), ((s_cnt - 1) >> 1) & 1, &abort_sh, a.status))) break;
             tc_fence_after();
-            if (!(ok = wg_sync())) break;
+            ATK_ADD(13);
             float o[NR];
             if (it.n_tiles > 0) {
                 load_rows<NR>(tlane + TM_O, o);
@@ -518,21 +562,43 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 #pragma unroll
                 for (int r = 0; r < NR; ++r) o[r] = 0.f;
             }
-            const bool single = a.nsplit == 1;
+            const bool single = it.n_split == 1;
+            ATK_ADD(15);
+            // O^T and every thread's share of the row sums go through shared memory (the P^T buffers are idle: the item's
+            // last MMA has read them) as [row][dim] and [row][key lane], and whole warps finish the rows in a rolled loop.
+            // Unrolled over 32 rows, the sums and the stores were kilobytes of code run once per item: fetched cold, with
+            // HBM saturated, they took 25 us.
+            float *osm = reinterpret_cast<float *>(gen + 2 * QCH), *lsm = osm + NR * HD;
 #pragma unroll
-            for (int r = 0; r < NR; ++r) {
-                if (r < QRW) {
-                    const float l = lsum_sh[0][r] + lsum_sh[1][r] + lsum_sh[2][r] + lsum_sh[3][r];
-                    const int h = it.g * grp + r / a.M, node = r % a.M;
-                    if (single) {
-                        store_act<__nv_bfloat16>(a.out, a.out_plane, ((size_t)(it.be * a.M + node) * a.H + h) * HD + kl, o[r] / l);
-                    } else {
-                        float *pdst = a.part + ((((size_t)it.be * a.H + h) * a.M + node) * a.nsplit + it.split) * ROWF;
-                        pdst[kl] = o[r];
-                        if (kl == 0) { pdst[HD] = mraw_sh[r] * 0.6931471805599453f; pdst[HD + 1] = l; }   // natural-log units
+            for (int r = 0; r < NR; ++r) { osm[r * HD + kl] = o[r]; lsm[r * HD + kl] = l_run[r]; }
+            if (!(ok = wg_sync())) break;
+            const int rows_out = dry ? 1 : QR;                          // the dry item runs the loop's code once, without the stores
+#pragma unroll 1
+            for (int r = warp - 2; r < rows_out; r += 4) {
+                const float *lr = lsm + r * HD + lane;
+                const float l = warp_sum((lr[0] + lr[32]) + (lr[64] + lr[96]));
+                const float4 v = *reinterpret_cast<const float4 *>(osm + r * HD + lane * 4);
+                const int hq = r / a.M, h = it.g * grp + hq, node = r - hq * a.M;
+                if (single) {
+                    const float x0 = v.x / l, x1 = v.y / l, x2 = v.z / l, x3 = v.w / l;
+                    const __nv_bfloat162 h01 = __floats2bfloat162_rn(x0, x1), h23 = __floats2bfloat162_rn(x2, x3);
+                    const __nv_bfloat162 l01 = __floats2bfloat162_rn(x0 - __low2float(h01), x1 - __high2float(h01));
+                    const __nv_bfloat162 l23 = __floats2bfloat162_rn(x2 - __low2float(h23), x3 - __high2float(h23));
+                    __nv_bfloat16 *dst = a.out + ((size_t)(it.be * a.M + node) * a.H + h) * HD + lane * 4;
+                    if (!dry) {
+                        *reinterpret_cast<uint2 *>(dst) = make_uint2(*reinterpret_cast<const uint32_t *>(&h01), *reinterpret_cast<const uint32_t *>(&h23));
+                        if (a.out_plane)
+                            *reinterpret_cast<uint2 *>(dst + a.out_plane) =
+                                make_uint2(*reinterpret_cast<const uint32_t *>(&l01), *reinterpret_cast<const uint32_t *>(&l23));
                     }
+                } else if (!dry) {
+                    float *pdst = a.part + ((((size_t)it.be * a.H + h) * a.M + node) * a.part_slots + it.split) * ROWF;
+                    *reinterpret_cast<float2 *>(pdst + lane * 4) = make_float2(v.x, v.y);       // rows are 8-byte aligned (HD + 2 floats)
+                    *reinterpret_cast<float2 *>(pdst + lane * 4 + 2) = make_float2(v.z, v.w);
+                    if (lane == 0) { pdst[HD] = mraw_sh[r] * 0.6931471805599453f; pdst[HD + 1] = l; }   // natural-log units
                 }
             }
+            ATK_ADD(14);
             if (!dry && it.n_tiles > 0) {
                 tc_fence_before();
                 __syncwarp();
@@ -544,7 +610,7 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 if (!(ok = wg_sync())) break;
                 if (et == 0) {
                     const int old = atomicAdd(&a.counters[it.be * a.Hkv + it.g], 1);
-                    last_sh = old == a.nsplit - 1;
+                    last_sh = old == it.n_split - 1;
                     if (last_sh) a.counters[it.be * a.Hkv + it.g] = 0;
                 }
                 if (!(ok = wg_sync())) break;
@@ -552,28 +618,28 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     __threadfence();
                     for (int r = warp - 2; r < QR; r += 4) {
                         const int hh = it.g * grp + r / a.M, i = r % a.M;
-                        const float *src = a.part + (((size_t)it.be * a.H + hh) * a.M + i) * (size_t)a.nsplit * ROWF;
+                        const float *psrc = a.part + (((size_t)it.be * a.H + hh) * a.M + i) * (size_t)a.part_slots * ROWF;
                         // lane s holds range s's (max, sum); the weights go round by shuffle (at most 32 ranges when fused)
                         float ms = -INFINITY, ls = 0.f;
-                        if (lane < a.nsplit) { ms = __ldcg(src + (size_t)lane * ROWF + HD); ls = __ldcg(src + (size_t)lane * ROWF + HD + 1); }
+                        if (lane < it.n_split) { ms = __ldcg(psrc + (size_t)lane * ROWF + HD); ls = __ldcg(psrc + (size_t)lane * ROWF + HD + 1); }
                         float num[HD / 32];
 #pragma unroll
                         for (int e = 0; e < HD / 32; ++e) num[e] = 0.f;
                         const float mmax = warp_max(ms);
                         const float w = (ms == -INFINITY) ? 0.f : expf(ms - mmax);
                         const float den = warp_sum(ls * w);
-                        for (int s0 = 0; s0 < a.nsplit; s0 += 4) {
+                        for (int s0 = 0; s0 < it.n_split; s0 += 4) {
                             float v[4][HD / 32];
 #pragma unroll
                             for (int q = 0; q < 4; ++q)
 #pragma unroll
                                 for (int e = 0; e < HD / 32; ++e)
-                                    v[q][e] = s0 + q < a.nsplit ? __ldcg(src + (size_t)(s0 + q) * ROWF + lane + 32 * e) : 0.f;
+                                    v[q][e] = s0 + q < it.n_split ? __ldcg(psrc + (size_t)(s0 + q) * ROWF + lane + 32 * e) : 0.f;
 #pragma unroll
                             for (int q = 0; q < 4; ++q) {
                                 const float wq = __shfl_sync(0xffffffffu, w, (s0 + q) & 31);
 #pragma unroll
-                                for (int e = 0; e < HD / 32; ++e) num[e] = fmaf(v[q][e], s0 + q < a.nsplit ? wq : 0.f, num[e]);
+                                for (int e = 0; e < HD / 32; ++e) num[e] = fmaf(v[q][e], s0 + q < it.n_split ? wq : 0.f, num[e]);
                             }
                         }
                         const float invd = 1.f / den;
@@ -583,9 +649,9 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                                                      num[e] * invd);
                     }
                 }
-                if (!(ok = wg_sync())) break;                          // last_sh and lsum_sh are reused by the next item
+                if (!(ok = wg_sync())) break;                          // last_sh and the staged rows are reused by the next item
             } else {
-                if (!(ok = wg_sync())) break;                          // lsum_sh is reused by the next item
+                if (!(ok = wg_sync())) break;                          // the staged rows are overwritten by the next item's P^T
             }
             ATK_ADD(11);
         }
@@ -660,10 +726,18 @@ int launch_attention_tk(viasd_model *m, const void *kc, const void *vc, bool sli
     a.batch = batch; a.layer_ord2 = layer_ord2; a.streams = streams;
     a.counters = m->ws.attn_counters;
     a.fuse_merge = fuse_merge;
-    a.n_items = streams * batch * c.n_kv_heads * nsplit;
-    int grid = a.n_items < m->sm_count ? a.n_items : m->sm_count;
-    a.items_per_cta = (a.n_items + grid - 1) / grid;
-    grid = (a.n_items + a.items_per_cta - 1) / a.items_per_cta;
+    int grid;
+    if (nsplit <= 0) {
+        // tiles dealt evenly: one range per CTA and row stream, cut by the kernel from the lengths; merges are fused
+        a.flat = 1; a.part_slots = 16; a.nsplit = 1; a.fuse_merge = 1; a.n_items = 0; a.items_per_cta = 0;
+        grid = m->sm_count;
+    } else {
+        a.flat = 0; a.part_slots = nsplit;
+        a.n_items = streams * batch * c.n_kv_heads * nsplit;
+        grid = a.n_items < m->sm_count ? a.n_items : m->sm_count;
+        a.items_per_cta = (a.n_items + grid - 1) / grid;
+        grid = (a.n_items + a.items_per_cta - 1) / a.items_per_cta;
+    }
     const size_t op_bytes = 6 * (size_t)(2 * nr) * 128;            // Q (2 chunks) and two P^T buffers (2 chunks each)
     // 32 query rows: the softmax of a tile is long, so K tiles get slots of their own, released by S^T = K Q^T, and the
     // tile after next is on its way meanwhile.  With fewer rows this measured slower than a slot per (K, V) pair.
