@@ -477,17 +477,18 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
         }
         if (!single && a.fuse_merge) {
             // last key range of this (sequence, kv head) to finish merges all of them, in range order
-            __threadfence();
+            // (one acquire-release atomic after the barrier instead of a fence per thread on both sides: the barrier
+            // orders the CTA's stores before it, and the release is cumulative)
             __syncthreads();
             if (threadIdx.x == 0) {
-                const int old = atomicAdd(&a.counters[it.be * a.Hkv + it.g], 1);
+                int old;
+                asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(a.counters + it.be * a.Hkv + it.g) : "memory");
                 last_sh = old == a.nsplit - 1;
                 if (last_sh) a.counters[it.be * a.Hkv + it.g] = 0;
             }
             __syncthreads();
             if (item == i0) ATRACE(7);
             if (last_sh) {
-                __threadfence();
                 for (int row = warp; row < QR; row += WARPS) {
                     const int h = it.g * grp + row / a.M, i = row % a.M;
                     const float *src = a.part + (((size_t)it.be * a.H + h) * a.M + i) * (size_t)a.nsplit * ROWF;

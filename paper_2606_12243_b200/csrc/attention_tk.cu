@@ -606,16 +606,16 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             }
             if (!dry && !single && a.fuse_merge) {
                 // last key range of this (sequence, kv head) to finish merges all of them, in range order
-                __threadfence();
+                // (one acquire-release atomic after the barrier instead of a fence per thread on both sides)
                 if (!(ok = wg_sync())) break;
                 if (et == 0) {
-                    const int old = atomicAdd(&a.counters[it.be * a.Hkv + it.g], 1);
+                    int old;
+                    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(a.counters + it.be * a.Hkv + it.g) : "memory");
                     last_sh = old == it.n_split - 1;
                     if (last_sh) a.counters[it.be * a.Hkv + it.g] = 0;
                 }
                 if (!(ok = wg_sync())) break;
                 if (last_sh) {
-                    __threadfence();
                     for (int r = warp - 2; r < QR; r += 4) {
                         const int hh = it.g * grp + r / a.M, i = r % a.M;
                         const float *psrc = a.part + (((size_t)it.be * a.H + hh) * a.M + i) * (size_t)a.part_slots * ROWF;

@@ -253,19 +253,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                     // its finishing: each waits (bounded) until every contributor has arrived and finishes its own
                     // slice of the token rows, summing the partials in CTA order.  A contributor that goes on into the
                     // next tile only arrives and never waits, so no wait depends on another wait.
-                    __threadfence();
+                    // (release / acquire: the barrier orders the group's stores before its first thread's release, which
+                    // is cumulative; a fence per thread on both sides was a microsecond of the launch's tail)
                     asm volatile("bar.sync 1, %0;" ::"n"(epi_threads) : "memory");
                     first_cta = (sg.tile * p.k_tiles) / p.units_per_cta;
                     last_cta = ((sg.tile + 1) * p.k_tiles - 1) / p.units_per_cta;
-                    if (et_all == 0) atomicAdd(&p.counters[sg.tile], 1);              // low half: arrivals
+                    if (et_all == 0) asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(p.counters + sg.tile) : "memory");   // low half: arrivals
                     if (u < u_end) { ++acc_it; ++seg_i; continue; }
                     const int n_c = last_cta - first_cta + 1;
                     const int last_range_end = min(total_units, (last_cta + 1) * p.units_per_cta);
                     const int n_fin = n_c - (last_range_end > (sg.tile + 1) * p.k_tiles ? 1 : 0);
                     if (et_all == 0) {
-                        volatile int *ctr = p.counters + sg.tile;
+                        const int *ctr = p.counters + sg.tile;
+                        auto arrived = [&]() { int v; asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory"); return v & 0xffff; };
                         const long long w0 = clock64();
-                        while ((*ctr & 0xffff) < n_c) {
+                        while (arrived() < n_c) {
                             if (abort_sh || clock64() - w0 > WAIT_LIMIT_CYCLES) { abort_sh = 1; atomicExch(p.status, VIASD_EDEVICE); break; }
                             __nanosleep(64);
                         }
@@ -275,7 +277,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                     asm volatile("bar.sync 1, %0;" ::"n"(epi_threads) : "memory");
                     if (et == 0) TRACE(8);
                     if (abort_sh) { ok = false; break; }
-                    __threadfence();
                     if (et == 0) TRACE(13);
                     {
                         // this finisher's rows: whole chunks, dealt in order of CTA number
