@@ -731,6 +731,7 @@ int launch_attention_tk(viasd_model *m, const void *kc, const void *vc, bool sli
         // tiles dealt evenly: one range per CTA and row stream, cut by the kernel from the lengths; merges are fused
         a.flat = 1; a.part_slots = 16; a.nsplit = 1; a.fuse_merge = 1; a.n_items = 0; a.items_per_cta = 0;
         grid = m->sm_count;
+        if (const char *e = getenv("VIASD_TK_GRID")) { const int v = atoi(e); if (v >= 1 && v < grid) grid = v; }   // tests: long ranges per CTA on small cases
     } else {
         a.flat = 0; a.part_slots = nsplit;
         a.n_items = streams * batch * c.n_kv_heads * nsplit;

@@ -328,6 +328,59 @@ def test_verify_step_with_each_attention_kernel(name, env, monkeypatch):
     _check_verify_step(name)
 
 
+# Sequences of different lengths in one batch.  The attention kernels deal key ranges or tiles to CTAs from the
+# committed lengths (the keys-on-lanes kernel cuts the tiles of all (sequence, head) pairs, laid end to end, into
+# equal ranges), so lengths that need 5, 6 and 7 tiles of 128 keys check those cuts against the oracle.  The extra
+# committed rows hold random bf16-exact keys and values, the same on both sides.  VIASD_TK_GRID shrinks the grid, so that
+# a CTA's range runs over several pairs, whole and cut, as it does at full size.
+@pytest.mark.parametrize("env", [{}, {"VIASD_ATTN": "tk"}, {"VIASD_ATTN": "tk", "VIASD_TK_FLAT": "0"},
+                                 {"VIASD_ATTN": "tk", "VIASD_DUAL_MAX": "64"}, {"VIASD_ATTN": "tk", "VIASD_TK_GRID": "7"},
+                                 {"VIASD_ATTN": "tk", "VIASD_TK_GRID": "3", "VIASD_DUAL_MAX": "64"}, {"VIASD_ATTN": "tc"},
+                                 {"VIASD_ATTN": "mma"}])
+def test_verify_step_with_ragged_lengths(env, monkeypatch):
+    for k, v in env.items():
+        monkeypatch.setenv(k, v)
+    wl = W.get("mini_13b")
+    extra = [0, 130, 7, 260, 1, 128, 64, 200]
+    assert wl.batch == len(extra) and not wl.real_prefill
+    vb = _vb()
+    eng, st, si, model = _prepare(wl, extra=max(extra) + 8)
+    rng = np.random.default_rng(7)
+    for cache, kc, vc in ((st.full, eng.k_full, eng.v_full), (st.slim, eng.k_slim, eng.v_slim)):
+        for o in range(cache.n_layers):
+            for b, e in enumerate(extra):
+                if e == 0:
+                    continue
+                for own, dev in ((cache.k[o], kc), (cache.v[o], vc)):
+                    t = torch.from_numpy(rng.standard_normal((own.shape[1], e, own.shape[3])).astype(np.float32)).to(torch.bfloat16)
+                    own[b, :, :e] = t.float().numpy()
+                    dev[o, b, :, wl.ctx:wl.ctx + e] = t.to(dev.device)
+    for b, e in enumerate(extra):
+        st.lens[b] += e
+        st.tokens[b] = [0] * e
+    eng.len.copy_(torch.from_numpy(st.lens.astype(np.int32)))
+    tiles = sorted(set((int(n) + wl.rows + 127) // 128 for n in st.lens))
+    assert len(tiles) >= 3, tiles
+    lo, hi = W.thresholds(wl)
+    want = step.verify_step(model, wl.shape, wl.routed, st, si.draft_tok, wl.parent, si.prow, si.drafter_logits,
+                            lo, hi, PU.oracle_params(wl))
+    sl, fl = eng.logits_buffer(), eng.logits_buffer()
+    res = vb.alloc_result(wl.batch, wl.n_nodes)
+    vb.verify_step(eng.model, eng.cache, eng.draft, eng.params(), sl, fl, res)
+    torch.cuda.synchronize()
+    assert vb.get_stats(eng.model).device_status == 0
+    assert np.array_equal(res.tier.cpu().numpy(), want.tier)
+    e1, _ = PU.assert_logits_close(sl.cpu().numpy(), want.slim_logits, wl.shape.dtype, "slim")
+    e2, _ = PU.assert_logits_close(fl.cpu().numpy(), want.full_logits, wl.shape.dtype, "full")
+    pinned, total, full = PU.compare_resolution(want.seqs, res.n_acc.cpu().numpy(), res.path.cpu().numpy(),
+                                                res.out_tok.cpu().numpy(), res.n_emit.cpu().numpy(),
+                                                res.corr_src.cpu().numpy(), eps_row=max(e1, e2))
+    assert total == 0 or pinned / total > 0.6, (pinned, total)
+    if full == wl.batch:
+        assert eng.len.cpu().tolist() == [int(x) for x in st.lens]
+        assert eng.pending.cpu().tolist() == [int(x) for x in st.pending]
+
+
 def _check_verify_step(name):
     wl = W.get(name)
     vb = _vb()
