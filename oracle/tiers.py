@@ -27,6 +27,9 @@ replacement token (argmax, or a draw from norm(max(0, j/beta - p))).  The
 accepted path plus that token are emitted; if every level was accepted nothing
 is added unless emit_bonus asks for a token from q at the leaf.
 
+Region masses (Eq. B.4-B.10): the probability, under the proposal, that a drafted token falls in region A, B, C;
+as sums over the vocabulary they are what the empirical tier frequencies converge to.
+
 Random numbers: a counter-based hash of (seed, step, sequence, stream, index);
 categorical draws use the Gumbel-max form so that no prefix sum is involved.
 """
@@ -103,6 +106,25 @@ def tier_rule(conf_logits: np.ndarray, draft_tok: np.ndarray, src_row: Sequence[
             d[b, n] = log_confidence(conf_logits[b, src_row[n]], int(draft_tok[b, n]))
             tier[b, n] = tier_of(d[b, n], log_tau_lo, log_tau_hi)
     return tier, d
+
+
+def region_masses(gate_logits: np.ndarray, proposal_logits: np.ndarray, log_tau_lo: float, log_tau_hi: float,
+                  temperature: float = 1.0) -> np.ndarray:
+    """(delta_p, delta_1bar, delta_2) per row (Eq. B.8-B.10): how much of the proposal p = softmax(proposal / T) lies on
+    the tokens that the gating row places in region A, B and C (Eq. B.1-B.3).  [..., V] x2 -> [..., 3].
+
+    A token's region is decided exactly as tier_of decides a drafted token's: d = l[u] - max l in the fp32 the logits
+    are stored in, compared with the fp32 log thresholds.  The masses are sums of p in float64.
+    """
+    g = np.asarray(gate_logits, dtype=np.float32)
+    d = g - g.max(axis=-1, keepdims=True)
+    in_a = d >= np.float32(log_tau_hi)
+    in_b = ~in_a & (d >= np.float32(log_tau_lo))
+    z = np.asarray(proposal_logits, dtype=np.float64) / float(temperature)
+    z = z - z.max(axis=-1, keepdims=True)
+    p = np.exp(z)
+    p = p / p.sum(axis=-1, keepdims=True)
+    return np.stack([(p * in_a).sum(axis=-1), (p * in_b).sum(axis=-1), (p * ~(in_a | in_b)).sum(axis=-1)], axis=-1)
 
 
 def quantile_thresholds(d: np.ndarray, q_lo: float, q_hi: float):
