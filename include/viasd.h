@@ -200,6 +200,20 @@ int viasd_gemm_static(const void *x, const void *w, float *y, int rows, int n, i
 int viasd_kl_cost(const float *judge_logits, const float *proposal_logits, int rows, int vocab, float temperature,
                   float alpha, float beta, int margin, float tau, float *cost_rows, float *cost_total, void *stream);
 
+/* Region masses (Eq. B.8-B.10; regions of Eq. B.1-B.3): per row, how much of the proposal distribution
+ * p = softmax(proposal_logits / temperature) lies on the tokens that the gating row places in region A (accepted
+ * outright), B (left to the slim verifier) and C (escalated to the full verifier):
+ *     mass[r][0] = delta_p     = sum_u p(u) [d(u) >= log_tau_hi]
+ *     mass[r][1] = delta_1-bar = sum_u p(u) [log_tau_lo <= d(u) < log_tau_hi]
+ *     mass[r][2] = delta_2     = sum_u p(u) [d(u) < log_tau_lo],        d(u) = gate_logits[r][u] - max_w gate_logits[r][w]
+ * with d taken in fp32 exactly as the tier step takes it for a drafted token, so these are the probabilities, under
+ * v ~ p, of the three tiers (Eq. B.4-B.6) and the weights of the output mixture of Eq. B.7.
+ * gate_logits, proposal_logits: device, fp32 [rows, vocab] row-major, read only.  mass: device, [rows, 3], written.
+ * mean: device, 3 floats, written with the mean of the rows in row order; may be NULL.  Asynchronous on `stream`;
+ * allocates nothing.  Errors: EINVAL (null pointer, rows or vocab < 1, temperature <= 0, log_tau_lo > log_tau_hi), ECUDA. */
+int viasd_region_mass(const float *gate_logits, const float *proposal_logits, int rows, int vocab, float temperature,
+                      float log_tau_hi, float log_tau_lo, float *mass, float *mean, void *stream);
+
 /* Measurement hooks (the paper has no counterpart; they exist so that a benchmark can attribute time).
  * viasd_launch_count: kernels launched by this library in this process so far.
  * viasd_set_timing(on): when on, every run of consecutive launches of one kernel class in the forward / tier /

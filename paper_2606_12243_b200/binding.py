@@ -21,7 +21,7 @@ VIASD_OK, VIASD_EINVAL, VIASD_ECAPACITY, VIASD_ECUDA, VIASD_EDEVICE, VIASD_EUNSU
 EXPORTS = ["viasd_workspace_bytes", "viasd_init_model", "viasd_full_forward", "viasd_slim_forward",
            "viasd_tier_accept", "viasd_kv_commit", "viasd_verify_step", "viasd_get_stats",
            "viasd_free_model", "viasd_strerror", "viasd_last_cuda_error", "viasd_gemm_scratch_bytes",
-           "viasd_gemm", "viasd_gemm_static", "viasd_kl_cost", "viasd_launch_count", "viasd_set_timing", "viasd_get_timing"]
+           "viasd_gemm", "viasd_gemm_static", "viasd_kl_cost", "viasd_region_mass", "viasd_launch_count", "viasd_set_timing", "viasd_get_timing"]
 
 TIMING_CLASSES = ["gemm", "attention", "norm", "rope", "embed", "tier_accept", "commit"]
 
@@ -116,6 +116,8 @@ def lib() -> C.CDLL:
         l.viasd_gemm_static.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p]
         l.viasd_kl_cost.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_float, C.c_float, C.c_float, C.c_int,
                                     C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]
+        l.viasd_region_mass.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_float, C.c_float, C.c_float,
+                                        C.c_void_p, C.c_void_p, C.c_void_p]
         l.viasd_launch_count.restype = C.c_ulonglong
         l.viasd_set_timing.argtypes = [C.c_void_p, C.c_int]
         l.viasd_get_timing.argtypes = [C.c_void_p, C.POINTER(Timing), C.c_void_p]
@@ -307,6 +309,22 @@ def kl_cost(judge_logits: torch.Tensor, proposal_logits: torch.Tensor, alpha: fl
     _check(lib().viasd_kl_cost(_ptr(judge_logits), _ptr(proposal_logits), rows, vocab, temperature, alpha, beta,
                                int(margin), tau, _ptr(out), _ptr(total), _stream(stream)), "viasd_kl_cost")
     return out, total
+
+
+def region_mass(gate_logits: torch.Tensor, proposal_logits: torch.Tensor, log_tau_hi: float, log_tau_lo: float,
+                temperature: float = 1.0, stream=None):
+    """viasd_region_mass: mass of the proposal on the gate's regions A, B, C per row (Eq. B.8-B.10) and its mean.
+
+    fp32 [rows, V] device tensors -> (mass [rows, 3], mean [3]), both fp32 device tensors.
+    """
+    assert gate_logits.dtype == torch.float32 and proposal_logits.dtype == torch.float32
+    assert gate_logits.is_contiguous() and proposal_logits.is_contiguous() and gate_logits.shape == proposal_logits.shape
+    rows, vocab = gate_logits.shape
+    mass = torch.empty((rows, 3), dtype=torch.float32, device=gate_logits.device)
+    mean = torch.empty(3, dtype=torch.float32, device=gate_logits.device)
+    _check(lib().viasd_region_mass(_ptr(gate_logits), _ptr(proposal_logits), rows, vocab, temperature, log_tau_hi,
+                                   log_tau_lo, _ptr(mass), _ptr(mean), _stream(stream)), "viasd_region_mass")
+    return mass, mean
 
 
 def gemm_static(x: torch.Tensor, w: torch.Tensor, y: torch.Tensor, stream=None) -> None:

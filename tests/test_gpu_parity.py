@@ -284,6 +284,56 @@ def test_sampling_draws_follow_the_judge_distribution():
 
 
 # ---------------------------------------------------------------------------------------------
+# region masses (Eq. B.8-B.10)
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("rows,vocab,temperature", [(1, 7, 1.0), (5, 1000, 1.0), (9, 32000, 0.7), (3, 128256, 1.0)])
+def test_region_mass_matches_oracle(rows, vocab, temperature):
+    vb = _vb()
+    rng = np.random.default_rng(rows * 1000 + vocab)
+    gate = (rng.standard_normal((rows, vocab)) * 2.0).astype(np.float32)
+    prop = (rng.standard_normal((rows, vocab)) * 2.0).astype(np.float32)
+    prop[:, :3] += 3.0
+    lo, hi = float(np.log(0.02)), float(np.log(0.3))
+    want = tiers.region_masses(gate, prop, lo, hi, temperature)
+    mass, mean = vb.region_mass(torch.from_numpy(gate).cuda(), torch.from_numpy(prop).cuda(), hi, lo, temperature)
+    torch.cuda.synchronize()
+    got = mass.cpu().numpy()
+    # the region of every token is decided in the same fp32 on both sides; the masses are fp32 sums against float64
+    assert np.abs(got - want).max() <= 2e-5, np.abs(got - want).max()
+    assert np.abs(got.sum(axis=-1) - 1.0).max() <= 1e-5
+    assert np.abs(mean.cpu().numpy() - want.mean(axis=0)).max() <= 2e-5
+
+
+def test_region_masses_are_what_the_tier_kernel_converges_to():
+    # tiers of tokens drawn from the proposal (Eq. B.4-B.6), counted by the tier kernel, against the masses of the same
+    # gate row from the region-mass kernel (Eq. B.8-B.10)
+    vb = _vb()
+    B, V = 64, 1024
+    wl = replace(W.get("c1_tiny"), batch=B, parent=W.chain(4))
+    eng = _tier_only_engine(wl)
+    si = W.step_inputs(wl)
+    si.drafter_logits[:] = si.drafter_logits[0, 0]                 # one gate row, which is also the proposal
+    gate = si.drafter_logits[0, 0]
+    p = tiers.softmax64(gate, 1.0)
+    lo, hi = W.thresholds(wl)
+    g = torch.from_numpy(gate[None].copy()).cuda()
+    mass, _ = vb.region_mass(g, g, float(hi), float(lo))
+    m = mass.cpu().numpy()[0].astype(np.float64)
+    rng = np.random.default_rng(5)
+    counts, n = np.zeros(3), 0
+    for it in range(30):
+        si.draft_tok[:] = rng.choice(V, size=si.draft_tok.shape, p=p)
+        eng.set_inputs(si)
+        res = vb.alloc_result(B, wl.n_nodes)
+        vb.tier_accept(eng.model, eng.draft, eng.params(step=it), None, None, 1, res)
+        t = res.tier.cpu().numpy().ravel()
+        counts += np.bincount(t, minlength=3)
+        n += t.size
+    freq = counts / n
+    assert np.all(np.abs(freq - m) < 4.0 * np.sqrt(m * (1 - m) / n) + 2e-4), (freq, m)
+
+
+# ---------------------------------------------------------------------------------------------
 # whole step and multi-step loop
 # ---------------------------------------------------------------------------------------------
 def _check_state(eng, st, wl, check_cache=True):
