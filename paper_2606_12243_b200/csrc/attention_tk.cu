@@ -228,9 +228,13 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     }
     if (threadIdx.x == 64) {
         // tiles per CTA when the tiles are dealt evenly: a pair may not be cut into more ranges than it has partial slots
-        int T = 0, tmax = 1;
-        if (a.flat) for (int b = 0; b < a.batch; ++b) { const int tb = (a.len_eff[b] + a.M + TKEYS - 1) / TKEYS; T += a.Hkv * tb; tmax = max(tmax, tb); }
-        per_sh = max(max((T + (int)gridDim.x - 1) / (int)gridDim.x, (tmax + a.part_slots - 2) / (a.part_slots - 1)), 1);
+        int per = 1;
+        if (a.flat) {
+            int T = 0, tmax = 1;
+            for (int b = 0; b < a.batch; ++b) { const int tb = (a.len_eff[b] + a.M + TKEYS - 1) / TKEYS; T += a.Hkv * tb; tmax = max(tmax, tb); }
+            per = max(max((T + (int)gridDim.x - 1) / (int)gridDim.x, (tmax + a.part_slots - 2) / (a.part_slots - 1)), 1);
+        }
+        per_sh = per;
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_sh)), "r"(256) : "memory");
