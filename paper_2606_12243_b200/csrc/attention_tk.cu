@@ -30,7 +30,7 @@ constexpr int HD = 128;                        // head dimension
 constexpr int TKEYS = 128;                     // keys per tile
 constexpr int HALF_BYTES = TKEYS * 128;        // 128 keys x 64 dims of bf16, as one TMA box lands
 constexpr int SLOT_BYTES = 2 * HALF_BYTES;     // one tile of K or of V: dims 0..63, dims 64..127
-constexpr int TK_THREADS = 192;
+constexpr int TK_THREADS = 192;                 // two service warps and four softmax warps (eight at 32 query rows)
 constexpr int TK_MAX_STAGE = 3;
 constexpr int ROWF = HD + 2;                   // partial row: 128 numerators, max (natural-log units), sum
 constexpr float RESCALE_GAP = 8.f;             // log2 units
@@ -146,9 +146,17 @@ __device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&r)[16])
 }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// hi + lo columns of one accumulator row: v[r] = column r + column NR + r
-template <int NR>
-__device__ __forceinline__ void load_rows(uint32_t taddr, float (&v)[NR]) {
+// hi + lo columns of RG accumulator rows: v[i] = column row0 + i plus column NR + row0 + i
+template <int NR, int RG>
+__device__ __forceinline__ void load_rows(uint32_t taddr, int row0, float (&v)[RG]) {
+    if constexpr (RG == 16 && NR == 32) {
+        uint32_t hi[16], lo[16];
+        tc_ld16(taddr + row0, hi);
+        tc_ld16(taddr + NR + row0, lo);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(hi[i]) + __uint_as_float(lo[i]);
+        return;
+    }
     float t[2 * NR];
 #pragma unroll
     for (int c = 0; c < 2 * NR / 16; ++c) {
@@ -158,7 +166,7 @@ __device__ __forceinline__ void load_rows(uint32_t taddr, float (&v)[NR]) {
         for (int e = 0; e < 16; ++e) t[c * 16 + e] = __uint_as_float(r[e]);
     }
 #pragma unroll
-    for (int r = 0; r < NR; ++r) v[r] = t[r] + t[NR + r];
+    for (int r = 0; r < RG; ++r) v[r] = t[r] + t[NR + r];
 }
 
 // byte offset of element (row, col) in a K-major tile of 128-byte rows with the 128-byte swizzle; col in bf16 units < 64
@@ -180,16 +188,18 @@ __device__ __forceinline__ long long gt_now() { unsigned long long t; asm volati
 #endif
 
 template <int NR>                                           // query rows per kv head rounded up to 8, 16 or 32
-__global__ void __launch_bounds__(TK_THREADS, 1)
+__global__ void __launch_bounds__(NR == 32 ? TK_THREADS + 128 : TK_THREADS, 1)
 attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                     const __grid_constant__ CUtensorMap map_k2, const __grid_constant__ CUtensorMap map_v2, const AttnTkArgs a) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) unsigned long long bars[4 * TK_MAX_STAGE + 10];
     __shared__ uint32_t tmem_base_sh;
     __shared__ int abort_sh, last_sh, per_sh;
-    __shared__ float wmax_sh[2][4][NR];                     // per tile parity, per warp: row maxima of its 32 keys
-    __shared__ float mref_sh[4][NR];                        // per warp (each keeps its own copy): the rows' running maxima, 0 while none
-    __shared__ float corr_sh[4][NR];                        // per warp: rescale factors of a tile in which a maximum moved
+    constexpr int SG = NR == 32 ? 2 : 1;                    // groups of four softmax warps; a group takes RG of the query rows
+    constexpr int RG = NR / SG, SW = 4 * SG, ST = 128 * SG; // rows per group, softmax warps, softmax threads
+    __shared__ float wmax_sh[2][4][NR];                     // per tile parity, per lane quarter: row maxima of its 32 keys
+    __shared__ float mref_sh[SW][RG];                        // per warp (each keeps its own copy): the rows' running maxima, 0 while none
+    __shared__ float corr_sh[SW][RG];                        // per warp: rescale factors of a tile in which a maximum moved
     __shared__ float mraw_sh[NR];                           // the rows' running maxima at the end of an item (-inf: no visible key)
     __shared__ unsigned long long anc_sh[VIASD_MAX_ROWS_PER_SEQ];
 
@@ -217,10 +227,10 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < TK_MAX_STAGE; ++s) { mbar_init(fullk_bar(s), 1); mbar_init(emptyk_bar(s), 1); mbar_init(fullv_bar(s), 1); mbar_init(emptyv_bar(s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(sfull_bar(b), 1); mbar_init(pfull_bar(b), 4); mbar_init(pvdone_bar(b), 1); }
-        mbar_init(ofree_bar, 4);
-        mbar_init(qfull_bar, 4);
-        mbar_init(wg_bar, 128);
+        for (int b = 0; b < 2; ++b) { mbar_init(sfull_bar(b), 1); mbar_init(pfull_bar(b), SW); mbar_init(pvdone_bar(b), 1); }
+        mbar_init(ofree_bar, SW);
+        mbar_init(qfull_bar, SW);
+        mbar_init(wg_bar, ST);
         abort_sh = 0;
         last_sh = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -380,7 +390,10 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         }
     } else {
         // ---------------- softmax / epilogue (warps 2..5 <-> TMEM lane quarters 2,3,0,1): one thread, one key (later one dim) ----------------
+        // With 32 query rows a second group of four warps (6..9, the same lane quarters) takes rows 16..31: the softmax
+        // of a tile is then half as long per thread, and two warps per scheduler hide each other's latencies.
         const int quarter = warp & 3, kl = quarter * 32 + lane, et = threadIdx.x - 64;   // kl: key of the tile / dim of O^T
+        const int sw = warp - 2, row0 = (sw >> 2) * RG;            // softmax warp number; first query row of its group
         const uint32_t tlane = tmem + ((uint32_t)(quarter * 32) << 16);
 #ifdef VIASD_TC_TRACE
         if (ATK_ON) for (int z = 0; z < 16; ++z) g_atk_trace[blockIdx.x * 16 + z] = 0;
@@ -418,15 +431,14 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 if (et < a.M) anc_sh[et] = a.tree->anc[et];
                 if (!(ok = wg_sync())) break;                         // anc_sh is visible
             }
-            const int QRW = dry ? 0 : QR;                              // rows whose result is written
             if (dry || it.be != q_be || it.g != q_g) {
                 // stage the query rows of this (sequence, kv head): rows 0..NR-1 the hi parts, NR..2NR-1 the lo parts,
                 // pre-scaled, in the K-major 128-byte-swizzled layout the MMA reads; loads first
-                for (int idx0 = et; idx0 < NR * (HD / 2); idx0 += 4 * 128) {
+                for (int idx0 = et; idx0 < NR * (HD / 2); idx0 += 4 * ST) {
                     float2 v[4];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
-                        const int idx = idx0 + q * 128, r = idx / (HD / 2), d2 = (idx % (HD / 2)) * 2;
+                        const int idx = idx0 + q * ST, r = idx / (HD / 2), d2 = (idx % (HD / 2)) * 2;
                         v[q] = make_float2(0.f, 0.f);
                         if (idx < NR * (HD / 2) && r < QR) {
                             const int h = it.g * grp + r / a.M, i = r % a.M;
@@ -435,7 +447,7 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     }
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
-                        const int idx = idx0 + q * 128, r = idx / (HD / 2), d2 = (idx % (HD / 2)) * 2;
+                        const int idx = idx0 + q * ST, r = idx / (HD / 2), d2 = (idx % (HD / 2)) * 2;
                         if (idx >= NR * (HD / 2)) continue;
                         const float x0 = v[q].x * a.scale, x1 = v[q].y * a.scale;
                         const __nv_bfloat162 hi = __floats2bfloat162_rn(x0, x1);
@@ -453,10 +465,10 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             }
             // Lane r of every warp keeps row r's running maximum (the four warps compute the same values); the other
             // lanes read it, as the exponent's reference, from the warp's copy in shared memory.
-            float m_lane = -INFINITY, l_run[NR];
+            float m_lane = -INFINITY, l_run[RG];
 #pragma unroll
-            for (int r = 0; r < NR; ++r) l_run[r] = 0.f;
-            if (lane < NR) mref_sh[quarter][lane] = 0.f;
+            for (int r = 0; r < RG; ++r) l_run[r] = 0.f;
+            if (lane < RG) mref_sh[sw][lane] = 0.f;
             __syncwarp();
 
             for (int t = 0; t < it.n_tiles; ++t) {
@@ -465,18 +477,18 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 if (!dry && !(ok = mbar_wait(sfull_bar(sb), (s_cnt >> 1) & 1, &abort_sh, a.status))) break;
                 tc_fence_after();
                 ATK_ADD(3);
-                float s[NR];
-                load_rows<NR>(tlane + TM_S + sb * 64, s);
+                float s[RG];
+                load_rows<NR, RG>(tlane + TM_S + sb * 64, row0, s);
                 // visibility: past the key range nothing; in the committed context everything; among the block's own
                 // rows only the ancestors of the query's node
                 const int j = it.k_begin + t * TKEYS + kl;
                 if (j >= it.k_end) {
 #pragma unroll
-                    for (int r = 0; r < NR; ++r) s[r] = -INFINITY;
+                    for (int r = 0; r < RG; ++r) s[r] = -INFINITY;
                 } else if (j >= it.n_ctx) {
                     const int tb = j - it.n_ctx;
 #pragma unroll
-                    for (int r = 0; r < NR; ++r) if (!((anc_sh[r % a.M] >> tb) & 1ull)) s[r] = -INFINITY;
+                    for (int r = 0; r < RG; ++r) if (!((anc_sh[(row0 + r) % a.M] >> tb) & 1ull)) s[r] = -INFINITY;
                 }
                 ATK_ADD(4);
                 // row maxima: over the warp's 32 keys by one warp-wide reduction per row (lane r keeps row r's), over the
@@ -484,26 +496,27 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 {
                     float mine = -INFINITY;
 #pragma unroll
-                    for (int r = 0; r < NR; ++r) {
+                    for (int r = 0; r < RG; ++r) {
                         float wm;
                         asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(wm) : "f"(s[r]));
                         if (lane == r) mine = wm;
                     }
-                    if (lane < NR) wmax_sh[sb][quarter][lane] = mine;
+                    if (lane < RG) wmax_sh[sb][quarter][row0 + lane] = mine;
                 }
                 ATK_ADD(5);
                 if (!(ok = wg_sync())) break;
                 ATK_ADD(6);
                 bool moved_l = false;
-                if (lane < NR) {
-                    const float mt = fmaxf(fmaxf(wmax_sh[sb][0][lane], wmax_sh[sb][1][lane]), fmaxf(wmax_sh[sb][2][lane], wmax_sh[sb][3][lane]));
+                if (lane < RG) {
+                    const int rr = row0 + lane;
+                    const float mt = fmaxf(fmaxf(wmax_sh[sb][0][rr], wmax_sh[sb][1][rr]), fmaxf(wmax_sh[sb][2][rr], wmax_sh[sb][3][rr]));
                     float corr = 1.f;
                     if (mt > m_lane + RESCALE_GAP) {                   // also the first tile with a visible key (m_lane = -inf)
                         if (m_lane != -INFINITY) { corr = ex2(m_lane - mt); moved_l = true; }
                         m_lane = mt;
-                        mref_sh[quarter][lane] = mt;
+                        mref_sh[sw][lane] = mt;
                     }
-                    corr_sh[quarter][lane] = corr;
+                    corr_sh[sw][lane] = corr;
                 }
                 const bool moved = __any_sync(0xffffffffu, moved_l);
                 __syncwarp();
@@ -511,17 +524,18 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     // rare: a running maximum moved.  Every warp sees the same maxima, so all four come here
                     // together; O^T is rescaled once the previous tile's MMAs have written it.
 #pragma unroll
-                    for (int r = 0; r < NR; ++r) l_run[r] *= corr_sh[quarter][r];
+                    for (int r = 0; r < RG; ++r) l_run[r] *= corr_sh[sw][r];
                     if (!dry) {
                         if (!(ok = mbar_wait(pvdone_bar(sb ^ 1), ((s_cnt - 1) >> 1) & 1, &abort_sh, a.status))) break;
                         tc_fence_after();
 #pragma unroll
-                        for (int c = 0; c < NC / 16; ++c) {
+                        for (int c = 0; c < 2 * RG / 16; ++c) {             // this group's hi columns, then its lo columns
+                            const uint32_t col = RG == 8 ? 0u : (uint32_t)(c * NR + row0);
                             uint32_t w[16];
-                            tc_ld16(tlane + TM_O + c * 16, w);
+                            tc_ld16(tlane + TM_O + col, w);
 #pragma unroll
-                            for (int e = 0; e < 16; ++e) w[e] = __float_as_uint(__uint_as_float(w[e]) * corr_sh[quarter][(c * 16 + e) % NR]);
-                            tc_st16(tlane + TM_O + c * 16, w);
+                            for (int e = 0; e < 16; ++e) w[e] = __float_as_uint(__uint_as_float(w[e]) * corr_sh[sw][(c * 16 + e) % RG]);
+                            tc_st16(tlane + TM_O + col, w);
                         }
                         tc_wait_st();
                     }
@@ -529,16 +543,16 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 ATK_ADD(7);
                 // weights of this key for every row; P^T (hi rows, lo rows) into shared memory for the MMA
                 uint8_t *pchunk = gen + 2 * QCH + (uint32_t)sb * 2 * QCH + (uint32_t)(kl >> 6) * QCH;
-                float mref[NR];                                  // read before the stores below: they could alias, which would
+                float mref[RG];                                  // read before the stores below: they could alias, which would
 #pragma unroll                                                   // put every one of these loads behind the previous row's stores
-                for (int r = 0; r < NR; ++r) mref[r] = mref_sh[quarter][r];
+                for (int r = 0; r < RG; ++r) mref[r] = mref_sh[sw][r];
 #pragma unroll
-                for (int r = 0; r < NR; ++r) {
+                for (int r = 0; r < RG; ++r) {
                     const float p = ex2(s[r] - mref[r]);                   // masked scores are -inf: weight 0
                     l_run[r] += p;
                     const __nv_bfloat16 hi = __float2bfloat16_rn(p), lo = __float2bfloat16_rn(p - __bfloat162float(hi));
-                    *reinterpret_cast<__nv_bfloat16 *>(pchunk + sw_off(r, kl & 63)) = hi;
-                    *reinterpret_cast<__nv_bfloat16 *>(pchunk + sw_off(NR + r, kl & 63)) = lo;
+                    *reinterpret_cast<__nv_bfloat16 *>(pchunk + sw_off(row0 + r, kl & 63)) = hi;
+                    *reinterpret_cast<__nv_bfloat16 *>(pchunk + sw_off(NR + row0 + r, kl & 63)) = lo;
                 }
                 ATK_ADD(8);
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> the MMA's reads
@@ -554,17 +568,17 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             if (!ok) break;
             ATK_T0();
             // ---- the item's result ----
-            if (quarter == 0 && lane < NR) mraw_sh[lane] = m_lane;
+            if (quarter == 0 && lane < RG) mraw_sh[row0 + lane] = m_lane;
             // the last MMA into O^T of the item (and with it all earlier ones) is complete
             if (!dry && it.n_tiles > 0 && !(ok = mbar_wait(pvdone_bar((s_cnt - 1) & 1), ((s_cnt - 1) >> 1) & 1, &abort_sh, a.status))) break;
             tc_fence_after();
             ATK_ADD(13);
-            float o[NR];
+            float o[RG];
             if (it.n_tiles > 0) {
-                load_rows<NR>(tlane + TM_O, o);
+                load_rows<NR, RG>(tlane + TM_O, row0, o);
             } else {
 #pragma unroll
-                for (int r = 0; r < NR; ++r) o[r] = 0.f;
+                for (int r = 0; r < RG; ++r) o[r] = 0.f;
             }
             const bool single = it.n_split == 1;
             ATK_ADD(15);
@@ -574,11 +588,11 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             // HBM saturated, they took 25 us.
             float *osm = reinterpret_cast<float *>(gen + 2 * QCH), *lsm = osm + NR * HD;
 #pragma unroll
-            for (int r = 0; r < NR; ++r) { osm[r * HD + kl] = o[r]; lsm[r * HD + kl] = l_run[r]; }
+            for (int r = 0; r < RG; ++r) { osm[(row0 + r) * HD + kl] = o[r]; lsm[(row0 + r) * HD + kl] = l_run[r]; }
             if (!(ok = wg_sync())) break;
             const int rows_out = dry ? 1 : QR;                          // the dry item runs the loop's code once, without the stores
 #pragma unroll 1
-            for (int r = warp - 2; r < rows_out; r += 4) {
+            for (int r = sw; r < rows_out; r += SW) {
                 const float *lr = lsm + r * HD + lane;
                 const float l = warp_sum((lr[0] + lr[32]) + (lr[64] + lr[96]));
                 const float4 v = *reinterpret_cast<const float4 *>(osm + r * HD + lane * 4);
@@ -620,7 +634,7 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 }
                 if (!(ok = wg_sync())) break;
                 if (last_sh) {
-                    for (int r = warp - 2; r < QR; r += 4) {
+                    for (int r = sw; r < QR; r += SW) {
                         const int hh = it.g * grp + r / a.M, i = r % a.M;
                         const float *psrc = a.part + (((size_t)it.be * a.H + hh) * a.M + i) * (size_t)a.part_slots * ROWF;
                         // lane s holds range s's (max, sum); the weights go round by shuffle (at most 32 ranges when fused)
@@ -766,7 +780,7 @@ int launch_attention_tk(viasd_model *m, const void *kc, const void *vc, bool sli
     }
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
-    pdl_config(cfg, attr, dim3(grid), dim3(TK_THREADS), smem, st);
+    pdl_config(cfg, attr, dim3(grid), dim3(nr == 32 ? TK_THREADS + 128 : TK_THREADS), smem, st);
     if (nr == 8) CUDA_TRY(cudaLaunchKernelEx(&cfg, attention_tk_kernel<8>, cm.k, cm.v, cm2->k, cm2->v, a));
     else if (nr == 16) CUDA_TRY(cudaLaunchKernelEx(&cfg, attention_tk_kernel<16>, cm.k, cm.v, cm2->k, cm2->v, a));
     else CUDA_TRY(cudaLaunchKernelEx(&cfg, attention_tk_kernel<32>, cm.k, cm.v, cm2->k, cm2->v, a));
