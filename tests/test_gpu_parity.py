@@ -454,6 +454,35 @@ def _check_verify_step(name):
         _check_state(eng, st, wl)
 
 
+# The split tiles of the GEMMs and the key ranges of the attention kernels are handed from CTA to CTA through global
+# memory (a release on a counter, an acquire by the CTA that finishes).  A hand-over that was not ordered would show
+# as a rare difference between runs: the same step, many times, must give the same bits.
+@pytest.mark.parametrize("name,env", [("mini_7b", {}), ("mini_13b", {"VIASD_ATTN": "tk"}), ("mini_32b_b3", {"VIASD_ATTN": "tk"}),
+                                      ("mini_8b_tree", {}), ("mini_7b", {"VIASD_ATTN": "tk", "VIASD_TK_GRID": "7"})])
+def test_repeated_verify_steps_are_bit_identical(name, env, monkeypatch):
+    for k, v in env.items():
+        monkeypatch.setenv(k, v)
+    wl = W.get(name)
+    vb = _vb()
+    eng, st, si, model = _prepare(wl)
+    sl, fl = eng.logits_buffer(), eng.logits_buffer()
+    res = vb.alloc_result(wl.batch, wl.n_nodes)
+    len0, pend0 = eng.len.clone(), eng.pending.clone()
+    ref = None
+    for it in range(300):
+        eng.len.copy_(len0)
+        eng.pending.copy_(pend0)
+        vb.verify_step(eng.model, eng.cache, eng.draft, eng.params(), sl, fl, res)
+        if it % 20 == 0 or it == 299:
+            torch.cuda.synchronize()
+            cur = (sl.clone(), fl.clone(), res.out_tok.clone(), res.n_emit.clone())
+            if ref is None:
+                ref = cur
+            else:
+                assert all(torch.equal(a, b) for a, b in zip(ref, cur)), it
+    assert vb.get_stats(eng.model).device_status == 0
+
+
 @pytest.mark.parametrize("name", ["mini_8b_tree", "mini_7b", "mini_13b"])
 def test_step_pieces_equal_fused_call(name):
     wl = W.get(name)
