@@ -169,9 +169,9 @@ int attention_nsplit(const viasd_model *m, int batch, int M) {
 // CTAs in equal contiguous shares, each item costs a fixed part (query staging, merge, partial) plus its tiles,
 // and every extra range adds merge work.  Depends on batch, heads and M only, so the one-stream and the two-stream
 // launch cut the keys at the same places and produce the same bits.
-static int mma_nsplit(const viasd_model *m, int batch, int M, int streams, bool tc, int reps) {
+static int mma_nsplit(const viasd_model *m, int batch, int M, int streams, bool tc, int reps, int subs) {
     const viasd_config &c = m->cfg;
-    const int base = batch * c.n_kv_heads, sms = m->sm_count;
+    const int base = batch * c.n_kv_heads * subs, sms = m->sm_count;      // subs: items per kv head (keys-on-lanes kernel)
     const int mt = ((c.n_heads / c.n_kv_heads) * M + 15) / 16;
     const int tiles = (c.max_ctx + 127) / 128;
     int max_s = tiles < 16 / reps ? tiles : 16 / reps;          // the partial buffer holds 16 ranges per (row, head)
@@ -209,12 +209,14 @@ static int mma_attention(viasd_model *m, const void *kc, const void *vc, bool sl
     // keys-on-lanes pays off when a CTA streams many tiles; with a handful per CTA (one short sequence) the
     // mma.sync kernel's shorter latency chain wins
     const long long tiles_total = (long long)streams * batch * c.n_kv_heads * ((c.max_ctx + 127) / 128);
-    int use = kind == 3 ? (attention_tk_supported(QR) && tiles_total >= 8LL * m->sm_count ? 2 : 0) : kind;
-    if (use == 2 && !attention_tk_supported(QR)) use = 0;
+    const int grp = c.n_heads / c.n_kv_heads, hpi = attention_tk_heads_per_item(grp, M);
+    const int subs = hpi ? grp / hpi : 1, QRi = hpi * M;       // keys-on-lanes: items per kv head, query rows per item
+    int use = kind == 3 ? (hpi && tiles_total * subs >= 8LL * m->sm_count ? 2 : 0) : kind;
+    if (use == 2 && !hpi) use = 0;
     const int reps = use == 1 ? attention_tc_replicas(QR) : 1;
-    const int nsplit = mma_nsplit(m, batch, M, streams, use != 0, reps);
+    const int nsplit = mma_nsplit(m, batch, M, streams, use != 0, reps, use == 2 ? subs : 1);
     const int n_part = nsplit * reps;        // key ranges per (row, head) that have to be merged
-    const bool fuse = n_part > 1 && n_part <= 32 && QR * n_part <= 160;
+    const bool fuse = n_part > 1 && n_part <= 32 && (use == 2 ? QRi : QR) * n_part <= 160;
     int rc;
     if (use == 2) {
         // The keys-on-lanes kernel deals tiles, not key ranges, evenly to the CTAs (nsplit 0) when the partial buffer
@@ -224,7 +226,7 @@ static int mma_attention(viasd_model *m, const void *kc, const void *vc, bool sl
         // item per CTA cost more than the balance won (32B batch-16 step 36.5 -> 39.0 ms).  VIASD_TK_FLAT=0/1 overrides.
         const char *e = getenv("VIASD_TK_FLAT");
         const size_t need = (size_t)streams * batch * c.n_heads * M * 16 * (c.head_dim + 2) * sizeof(float);
-        if ((e ? atoi(e) != 0 : QR <= 16) && need <= m->ws.part_bytes)
+        if ((e ? atoi(e) != 0 : QR <= 16) && subs == 1 && need <= m->ws.part_bytes)
             return launch_attention_tk(m, kc, vc, slim, layer_ord, kc2, vc2, layer_ord2, streams, batch, M, 0, 1, st);
         rc = launch_attention_tk(m, kc, vc, slim, layer_ord, kc2, vc2, layer_ord2, streams, batch, M, nsplit, fuse ? 1 : 0, st);
     }

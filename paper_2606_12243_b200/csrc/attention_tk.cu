@@ -47,6 +47,8 @@ struct AttnTkArgs {
     int M, H, Hkv, max_batch, max_ctx, layer_ord, nsplit;
     int batch, layer_ord2;      // second row stream: rows batch*M.., its own cache and layer ordinal
     int streams, n_items, items_per_cta, fuse_merge, nk, nv;   // nk, nv: ring slots for K tiles and for V tiles
+    int subs;                   // item groups per kv head: with more than 32 query rows per kv head, the query heads of a
+                                // kv head are dealt to `subs` items (each streams the K/V tiles again, from L2)
     int flat, part_slots;       // flat: tiles (not key ranges) are dealt evenly to the CTAs; part_slots: partial slots per (row, head)
     int *counters;              // arrivals per (stream, sequence, kv head), zero between launches
     float scale;                // log2(e) / sqrt(hd)
@@ -60,8 +62,8 @@ __device__ __forceinline__ Item decode_item(const AttnTkArgs &a, int item) {
     it.split = item % a.nsplit;
     it.n_split = a.nsplit;
     const int bg = item / a.nsplit;
-    it.g = bg % a.Hkv;
-    it.be = bg / a.Hkv;
+    it.g = bg % (a.Hkv * a.subs);                  // group of query heads: kv head it.g / subs, part it.g % subs of its heads
+    it.be = bg / (a.Hkv * a.subs);
     it.stream = it.be / a.batch;
     it.b = it.be - it.stream * a.batch;
     it.n_ctx = a.len_eff[it.b];
@@ -71,7 +73,7 @@ __device__ __forceinline__ Item decode_item(const AttnTkArgs &a, int item) {
     it.k_begin = it.split * chunk;
     it.k_end = min(Tk, it.k_begin + chunk);
     it.n_tiles = it.k_end > it.k_begin ? (it.k_end - it.k_begin + TKEYS - 1) / TKEYS : 0;
-    it.row_base = (((it.stream ? a.layer_ord2 : a.layer_ord) * a.max_batch + it.b) * a.Hkv + it.g) * a.max_ctx;
+    it.row_base = (((it.stream ? a.layer_ord2 : a.layer_ord) * a.max_batch + it.b) * a.Hkv + it.g / a.subs) * a.max_ctx;
     return it;
 }
 
@@ -94,21 +96,21 @@ __device__ __forceinline__ bool next_item(const AttnTkArgs &a, int per, ItemSrc 
         it = decode_item(a, c.item++);
         return true;
     }
-    const int lo = blockIdx.x * per, hi = lo + per;
+    const int lo = blockIdx.x * per, hi = lo + per, HkvV = a.Hkv * a.subs;
     while (c.s < a.streams) {
         if (c.b >= a.batch || c.off >= hi) { ++c.s; c.b = c.g = c.off = 0; continue; }   // done with this stream
         const int n_ctx = a.len_eff[c.b], Tk = n_ctx + a.M, tb = (Tk + TKEYS - 1) / TKEYS;
-        if (c.off + a.Hkv * tb <= lo) { c.off += a.Hkv * tb; ++c.b; c.g = 0; continue; }    // this sequence ends before the range
+        if (c.off + HkvV * tb <= lo) { c.off += HkvV * tb; ++c.b; c.g = 0; continue; }      // this sequence ends before the range
         if (c.g == 0 && c.off < lo) c.g = (lo - c.off) / tb;                                // its first pair that reaches into the range
         const int p_lo = c.off + c.g * tb;
-        if (c.g >= a.Hkv) { c.off += a.Hkv * tb; ++c.b; c.g = 0; continue; }
+        if (c.g >= HkvV) { c.off += HkvV * tb; ++c.b; c.g = 0; continue; }
         if (p_lo >= hi) { ++c.s; c.b = c.g = c.off = 0; continue; }
         const int p_hi = p_lo + tb, t0 = max(lo, p_lo) - p_lo, t1 = min(hi, p_hi) - p_lo;
         const int first = p_lo / per, last = (p_hi - 1) / per;
         it.b = c.b; it.stream = c.s; it.be = c.s * a.batch + c.b; it.g = c.g;
         it.split = (int)blockIdx.x - first; it.n_split = last - first + 1;
         it.n_ctx = n_ctx; it.k_begin = t0 * TKEYS; it.k_end = min(Tk, t1 * TKEYS); it.n_tiles = t1 - t0;
-        it.row_base = (((c.s ? a.layer_ord2 : a.layer_ord) * a.max_batch + c.b) * a.Hkv + c.g) * a.max_ctx;
+        it.row_base = (((c.s ? a.layer_ord2 : a.layer_ord) * a.max_batch + c.b) * a.Hkv + c.g / a.subs) * a.max_ctx;
         ++c.g;
         return true;
     }
@@ -209,7 +211,7 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     PDL_TRIGGER();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int NK = a.nk, NV = a.nv;
-    const int grp = a.H / a.Hkv, QR = grp * a.M;
+    const int HkvV = a.Hkv * a.subs, grp = a.H / HkvV, QR = grp * a.M;   // query heads and rows per item group
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t qsm = base, psm = base + 2 * QCH, ring = base + 6 * QCH;   // Q (2 chunks), P^T (2 buffers x 2 chunks), ring
     uint8_t *gen = smem_raw + (base - smem_u32(smem_raw));
@@ -241,7 +243,7 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         int per = 1;
         if (a.flat) {
             int T = 0, tmax = 1;
-            for (int b = 0; b < a.batch; ++b) { const int tb = (a.len_eff[b] + a.M + TKEYS - 1) / TKEYS; T += a.Hkv * tb; tmax = max(tmax, tb); }
+            for (int b = 0; b < a.batch; ++b) { const int tb = (a.len_eff[b] + a.M + TKEYS - 1) / TKEYS; T += a.Hkv * a.subs * tb; tmax = max(tmax, tb); }
             per = max(max((T + (int)gridDim.x - 1) / (int)gridDim.x, (tmax + a.part_slots - 2) / (a.part_slots - 1)), 1);
         }
         per_sh = per;
@@ -628,9 +630,9 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 if (!(ok = wg_sync())) break;
                 if (et == 0) {
                     int old;
-                    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(a.counters + it.be * a.Hkv + it.g) : "memory");
+                    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(a.counters + it.be * HkvV + it.g) : "memory");
                     last_sh = old == it.n_split - 1;
-                    if (last_sh) a.counters[it.be * a.Hkv + it.g] = 0;
+                    if (last_sh) a.counters[it.be * HkvV + it.g] = 0;
                 }
                 if (!(ok = wg_sync())) break;
                 if (last_sh) {
@@ -695,7 +697,15 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 
 }  // namespace
 
-int attention_tk_supported(int query_rows) { return query_rows <= 32; }
+// Query heads of a kv head that one item takes: as many as fit 32 rows (a divisor of the group, at most 4 items per
+// kv head: the arrival counters have four slots per (sequence, kv head)).  0: the kernel does not take this shape.
+int attention_tk_heads_per_item(int group_heads, int M) {
+    if (M > 32 || M < 1) return 0;
+    for (int hpi = group_heads; hpi >= 1; --hpi)
+        if (group_heads % hpi == 0 && hpi * M <= 32) return group_heads / hpi <= 4 ? hpi : 0;
+    return 0;
+}
+int attention_tk_supported(int group_heads, int M) { return attention_tk_heads_per_item(group_heads, M) > 0; }
 
 // tensor maps over the caches are rebuilt only when the caller's pointers change
 static int cache_maps_tk(viasd_model *m, CacheMaps &cm, const void *kc, const void *vc, int n_layers) {
@@ -723,8 +733,9 @@ int launch_attention_tk(viasd_model *m, const void *kc, const void *vc, bool sli
         cm2 = &m->cmaps_slim;
         if ((rc = cache_maps_tk(m, *cm2, kc2, vc2, m->n_routed))) return rc;
     }
-    const int grp = c.n_heads / c.n_kv_heads, QR = grp * M;
-    if (QR > 32) return VIASD_EINVAL;
+    const int grp = c.n_heads / c.n_kv_heads, hpi = attention_tk_heads_per_item(grp, M);
+    if (hpi == 0) return VIASD_EINVAL;
+    const int QR = hpi * M, subs = grp / hpi;                      // rows per item; items per kv head
     const int nr = QR <= 8 ? 8 : QR <= 16 ? 16 : 32;
     AttnTkArgs a;
     a.trace_on = 0;
@@ -739,7 +750,7 @@ int launch_attention_tk(viasd_model *m, const void *kc, const void *vc, bool sli
     a.q = m->ws.q; a.part = m->ws.part; a.out = (__nv_bfloat16 *)m->ws.attn;
     a.out_plane = m->ws.rows_alloc * (size_t)c.n_heads * HD;
     a.len_eff = m->ws.len_eff; a.tree = m->ws.tree; a.status = &m->ws.stats->device_status;
-    a.M = M; a.H = c.n_heads; a.Hkv = c.n_kv_heads; a.max_batch = c.max_batch; a.max_ctx = c.max_ctx;
+    a.M = M; a.H = c.n_heads; a.Hkv = c.n_kv_heads; a.subs = subs; a.max_batch = c.max_batch; a.max_ctx = c.max_ctx;
     a.layer_ord = layer_ord; a.nsplit = nsplit; a.scale = 1.4426950408889634f / sqrtf((float)HD);   // log2(e) / sqrt(hd)
     a.batch = batch; a.layer_ord2 = layer_ord2; a.streams = streams;
     a.counters = m->ws.attn_counters;
@@ -752,7 +763,7 @@ int launch_attention_tk(viasd_model *m, const void *kc, const void *vc, bool sli
         if (const char *e = getenv("VIASD_TK_GRID")) { const int v = atoi(e); if (v >= 1 && v < grid) grid = v; }   // tests: long ranges per CTA on small cases
     } else {
         a.flat = 0; a.part_slots = nsplit;
-        a.n_items = streams * batch * c.n_kv_heads * nsplit;
+        a.n_items = streams * batch * c.n_kv_heads * subs * nsplit;
         grid = a.n_items < m->sm_count ? a.n_items : m->sm_count;
         a.items_per_cta = (a.n_items + grid - 1) / grid;
         grid = (a.n_items + a.items_per_cta - 1) / a.items_per_cta;

@@ -151,7 +151,8 @@ int attention_tc_replicas(int query_rows);
 int launch_attention_tc(viasd_model *m, const void *kc, const void *vc, bool slim, int layer_ord, const void *kc2,
                          const void *vc2, int layer_ord2, int streams, int batch, int M, int nsplit, int fuse_merge,
                          cudaStream_t st);
-int attention_tk_supported(int query_rows);
+int attention_tk_heads_per_item(int group_heads, int M);
+int attention_tk_supported(int group_heads, int M);
 int launch_attention_tk(viasd_model *m, const void *kc, const void *vc, bool slim, int layer_ord, const void *kc2,
                          const void *vc2, int layer_ord2, int streams, int batch, int M, int nsplit, int fuse_merge,
                          cudaStream_t st);

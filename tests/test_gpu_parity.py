@@ -78,8 +78,10 @@ def test_forward_logits_and_appended_kv(name):
 
 # The attention kernel is chosen by problem size (mma.sync for short single sequences, tcgen05 with keys on the TMEM
 # lanes when a CTA streams many tiles); the small parity cases would otherwise only ever see the first.  "tk" needs at
-# most 32 query rows per kv head, "tc" (query rows on the lanes) takes up to 128.
-@pytest.mark.parametrize("name,kernel", [("mini_7b", "tk"), ("mini_13b", "tk"), ("mini_32b_b3", "tk"), ("mini_7b", "tc"),
+# most 32 query rows per item (a tree of 27 rows with four query heads per kv head becomes four items per kv head),
+# "tc" (query rows on the lanes) takes up to 128.
+@pytest.mark.parametrize("name,kernel", [("mini_7b", "tk"), ("mini_13b", "tk"), ("mini_32b_b3", "tk"), ("mini_8b_tree", "tk"),
+                                         ("mini_7b", "tc"),
                                          ("mini_8b_tree", "tc"), ("mini_32b", "tc")])
 def test_forward_with_each_attention_kernel(name, kernel, monkeypatch):
     monkeypatch.setenv("VIASD_ATTN", kernel)
@@ -371,7 +373,8 @@ def test_verify_step_matches_oracle(name):
 # both row streams in one attention launch, with the kernels the small cases do not pick by themselves; and
 # separate passes where the default would be one sweep
 @pytest.mark.parametrize("name,env", [("mini_7b", {"VIASD_ATTN": "tk"}), ("mini_7b", {"VIASD_ATTN": "tc"}),
-                                      ("mini_13b", {"VIASD_ATTN": "tk", "VIASD_DUAL_MAX": "64"})])
+                                      ("mini_13b", {"VIASD_ATTN": "tk", "VIASD_DUAL_MAX": "64"}),
+                                      ("mini_8b_tree", {"VIASD_ATTN": "tk"}), ("mini_8b_tree", {"VIASD_ATTN": "tk", "VIASD_DUAL_MAX": "16"})])
 def test_verify_step_with_each_attention_kernel(name, env, monkeypatch):
     for k, v in env.items():
         monkeypatch.setenv(k, v)
@@ -458,7 +461,8 @@ def _check_verify_step(name):
 # memory (a release on a counter, an acquire by the CTA that finishes).  A hand-over that was not ordered would show
 # as a rare difference between runs: the same step, many times, must give the same bits.
 @pytest.mark.parametrize("name,env", [("mini_7b", {}), ("mini_13b", {"VIASD_ATTN": "tk"}), ("mini_32b_b3", {"VIASD_ATTN": "tk"}),
-                                      ("mini_8b_tree", {}), ("mini_7b", {"VIASD_ATTN": "tk", "VIASD_TK_GRID": "7"})])
+                                      ("mini_8b_tree", {}), ("mini_8b_tree", {"VIASD_ATTN": "tk"}),
+                                      ("mini_7b", {"VIASD_ATTN": "tk", "VIASD_TK_GRID": "7"})])
 def test_repeated_verify_steps_are_bit_identical(name, env, monkeypatch):
     for k, v in env.items():
         monkeypatch.setenv(k, v)
