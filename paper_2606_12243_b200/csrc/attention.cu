@@ -169,7 +169,7 @@ int attention_nsplit(const viasd_model *m, int batch, int M) {
 // CTAs in equal contiguous shares, each item costs a fixed part (query staging, merge, partial) plus its tiles,
 // and every extra range adds merge work.  Depends on batch, heads and M only, so the one-stream and the two-stream
 // launch cut the keys at the same places and produce the same bits.
-static int mma_nsplit(const viasd_model *m, int batch, int M, int streams, bool tc, int reps, int subs) {
+static int mma_nsplit(const viasd_model *m, int batch, int M, int streams, bool tc, int reps, int subs, int tk_rows) {
     const viasd_config &c = m->cfg;
     const int base = batch * c.n_kv_heads * subs, sms = m->sm_count;      // subs: items per kv head (keys-on-lanes kernel)
     const int mt = ((c.n_heads / c.n_kv_heads) * M + 15) / 16;
@@ -177,7 +177,10 @@ static int mma_nsplit(const viasd_model *m, int batch, int M, int streams, bool 
     int max_s = tiles < 16 / reps ? tiles : 16 / reps;          // the partial buffer holds 16 ranges per (row, head)
     if (max_s < 1) max_s = 1;
     // microseconds, roughly: the tcgen05 kernel's tile does not depend on the number of query tiles
-    const double t_tile = tc ? 0.7 : 0.5 + 0.8 * mt, t_item = tc ? 4.0 : 3.0;
+    // (keys-on-lanes kernel, measured: a tile costs its softmax chain, 1.1 - 1.8 us with 8 - 32 rows per item, an item
+    // 5 - 10 us of query staging, result rows and merge)
+    const double t_tile = tk_rows > 16 ? 1.8 : tk_rows > 8 ? 1.3 : tk_rows > 0 ? 1.1 : tc ? 0.7 : 0.5 + 0.8 * mt;
+    const double t_item = tk_rows > 16 ? 8.0 : tk_rows > 0 ? 5.0 : tc ? 4.0 : 3.0;
     // One choice for the whole model, whichever call runs (the cuts must not depend on it): the routed layers are
     // charged as two-stream launches, as the verify step runs them, the others as one-stream launches.
     const int n_dual = m->n_routed, n_single = c.n_layers - m->n_routed;
@@ -192,6 +195,7 @@ static int mma_nsplit(const viasd_model *m, int batch, int M, int streams, bool 
         }
         if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
     }
+    if (const char *e = getenv("VIASD_ATTN_NSPLIT")) { const int v = atoi(e); if (v >= 1 && v <= max_s) best = v; }   // measurement
     size_t per_split = (size_t)streams * batch * c.n_heads * M * (c.head_dim + 2) * sizeof(float) * reps;
     while (best > 1 && per_split * best > m->ws.part_bytes) --best;
     return best;
@@ -211,10 +215,12 @@ static int mma_attention(viasd_model *m, const void *kc, const void *vc, bool sl
     const long long tiles_total = (long long)streams * batch * c.n_kv_heads * ((c.max_ctx + 127) / 128);
     const int grp = c.n_heads / c.n_kv_heads, hpi = attention_tk_heads_per_item(grp, M);
     const int subs = hpi ? grp / hpi : 1, QRi = hpi * M;       // keys-on-lanes: items per kv head, query rows per item
-    int use = kind == 3 ? (hpi && tiles_total * subs >= 8LL * m->sm_count ? 2 : 0) : kind;
+    // (with more than 32 query rows per kv head the mma.sync kernel has one key group per query tile and is bound by
+    // its MMA issue: there the keys-on-lanes kernel wins from two tiles per SM on)
+    int use = kind == 3 ? (hpi && tiles_total * subs >= (subs > 1 ? 2LL : 8LL) * m->sm_count ? 2 : 0) : kind;
     if (use == 2 && !hpi) use = 0;
     const int reps = use == 1 ? attention_tc_replicas(QR) : 1;
-    const int nsplit = mma_nsplit(m, batch, M, streams, use != 0, reps, use == 2 ? subs : 1);
+    const int nsplit = mma_nsplit(m, batch, M, streams, use != 0, reps, use == 2 ? subs : 1, use == 2 ? QRi : 0);
     const int n_part = nsplit * reps;        // key ranges per (row, head) that have to be merged
     const bool fuse = n_part > 1 && n_part <= 32 && (use == 2 ? QRi : QR) * n_part <= 160;
     int rc;

@@ -51,7 +51,7 @@ struct Workspace {                      // pointers into the caller's workspace 
     float *gemm_scratch;                // partial tiles of split GEMM work (tcgen05 kernel)
     int *gemm_counters;                 // per-tile arrival counters, zero between launches
     size_t n_counters;
-    int *attn_counters;                 // [2 * max_batch * Hkv] key-range arrivals per (sequence, kv head)
+    int *attn_counters;                 // [2 * max_batch * Hkv * 4] key-range arrivals per (stream, sequence, kv head, group of query heads)
     float *ssq;                         // [(d / 128) * 4][R] partial sums of h^2 for the fused RMSNorm
 };
 

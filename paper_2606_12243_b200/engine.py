@@ -42,7 +42,9 @@ class Engine:
         mask = [1 if l in set(self.routed) else 0 for l in range(s.n_layers)]
         nbytes = vb.workspace_bytes(self.cfg, len(self.routed))
         assert nbytes > 0, "configuration rejected by viasd_workspace_bytes"
-        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=device)
+        # Poisoned on purpose (every float a NaN, every counter -1): the library has to initialise what it relies on,
+        # and recycled device memory is not zero.
+        self.workspace = torch.full((nbytes,), 0xFF, dtype=torch.uint8, device=device)
         self.model = vb.init_model(self.cfg, self.embed, self.lm_head, self.final_norm, self.layers, mask,
                                    self.workspace)
         kv = lambda nl: torch.zeros((nl, wl.batch, s.n_kv_heads, self.max_ctx, s.head_dim), dtype=self.tdtype,
