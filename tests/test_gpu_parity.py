@@ -623,12 +623,13 @@ def test_argument_and_capacity_errors():
 # ---------------------------------------------------------------------------------------------
 # full size, in the launch configuration the benchmark times
 # ---------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("name", ["c2_7b", "c3_8b_tree_b1", "c4_13b"])
+@pytest.mark.parametrize("name", ["c2_7b", "c3_8b_tree_b1", "c3_8b_tree", "c4_13b"])
 def test_full_size_verify_step_matches_oracle(name):
     """Full-size workloads through viasd_verify_step, in the launch configuration the benchmark times, against the
     oracle evaluated in fp32 on the same generated weights: all logits of both verifiers, tiers, and every pinned
     decision.  c2_7b is the benchmarked workload (chain of 8, one sweep for both verifiers, mma.sync attention);
-    c3_8b_tree_b1 has the 26-node tree, grouped heads, the 128k vocabulary and sampling (cluster accept walk);
+    c3_8b_tree_b1 has the 26-node tree, grouped heads, the 128k vocabulary and sampling (cluster accept walk; one sweep,
+    keys-on-lanes attention with four items per kv head); c3_8b_tree is the same at batch 4 (108 rows: separate passes);
     c4_13b has 8 sequences of 4096 tokens (separate passes, tcgen05 keys-on-lanes attention)."""
     wl = W.get(name)
     vb = _vb()
