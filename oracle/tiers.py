@@ -10,7 +10,7 @@ region A (accept) c >= tau_hi, region B (slim verifier decides) tau_lo <= c <
 tau_hi, region C (escalate to the full verifier) c < tau_lo.  With logits the
 test is d = l[v] - max_u l[u] compared with log tau; the log thresholds are the
 inputs, so the decision is one fp32 subtraction and a comparison.
-Readings taken where the paper leaves a choice (all listed in the design notes):
+Readings taken where the paper leaves a choice:
 thresholds are given directly as tau_hi >= tau_lo; the gating distribution is
 the drafter's (conf_source 0) or the slim verifier's at the parent row
 (conf_source 1, Algorithm 2 as printed).

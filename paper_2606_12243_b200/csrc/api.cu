@@ -64,7 +64,7 @@ size_t carve(const viasd_config &c, char *base, Workspace *ws) {
         if (qd + 2 * kvd > widest) widest = qd + 2 * kvd;
         if ((size_t)c.d_ff > widest) widest = c.d_ff;
         w.ssq = cv.take<float>((size_t)(c.d_model / 128 + 1) * 4 * R * 4);
-        w.attn_counters = cv.take<int>((size_t)2 * c.max_batch * c.n_kv_heads * 4);
+        w.attn_counters = cv.take<int>(attn_counter_count(c.max_batch, c.n_kv_heads) * sizeof(int));
         w.n_counters = widest / 128 + 8;
         w.gemm_counters = cv.take<int>(w.n_counters * 4);
     }
@@ -417,7 +417,7 @@ int viasd_init_model(const viasd_config *cfg, const viasd_weights *w, const unsi
     }
     cudaError_t e = cudaMemset(m->ws.stats, 0, sizeof(DeviceStats));
     if (e == cudaSuccess) e = cudaMemset(m->ws.gemm_counters, 0, m->ws.n_counters * 4);
-    if (e == cudaSuccess) e = cudaMemset(m->ws.attn_counters, 0, (size_t)2 * cfg->max_batch * cfg->n_kv_heads * 4 * sizeof(int));   // four counters per (stream, sequence, kv head)
+    if (e == cudaSuccess) e = cudaMemset(m->ws.attn_counters, 0, attn_counter_count(cfg->max_batch, cfg->n_kv_heads) * sizeof(int));
     if (e == cudaSuccess) { rc = launch_rope_table(m, 0); if (rc == VIASD_OK) e = cudaDeviceSynchronize(); }
     if (e != cudaSuccess) { g_last_cuda_error = (int)e; rc = VIASD_ECUDA; }
     if (rc) { viasd_free_model(m); return rc; }

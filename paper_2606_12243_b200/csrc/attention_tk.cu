@@ -702,7 +702,7 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 int attention_tk_heads_per_item(int group_heads, int M) {
     if (M > 32 || M < 1) return 0;
     for (int hpi = group_heads; hpi >= 1; --hpi)
-        if (group_heads % hpi == 0 && hpi * M <= 32) return group_heads / hpi <= 4 ? hpi : 0;
+        if (group_heads % hpi == 0 && hpi * M <= 32) return group_heads / hpi <= VIASD_ATTN_ITEMS_PER_KV_HEAD ? hpi : 0;
     return 0;
 }
 int attention_tk_supported(int group_heads, int M) { return attention_tk_heads_per_item(group_heads, M) > 0; }

@@ -8,6 +8,12 @@
 #include "gemm_tc.cuh"
 
 #define VIASD_MAX_ROWS_PER_SEQ 64
+// Arrival counters of the attention kernels: one per (stream, sequence, kv head, item of that kv head).  The
+// keys-on-lanes kernel deals the query heads of a kv head to at most this many items.
+#define VIASD_ATTN_ITEMS_PER_KV_HEAD 4
+inline size_t attn_counter_count(int max_batch, int n_kv_heads) {
+    return (size_t)2 * max_batch * n_kv_heads * VIASD_ATTN_ITEMS_PER_KV_HEAD;
+}
 
 // ---------------------------------------------------------------------------------------------
 // device-side records kept in the workspace
@@ -51,7 +57,7 @@ struct Workspace {                      // pointers into the caller's workspace 
     float *gemm_scratch;                // partial tiles of split GEMM work (tcgen05 kernel)
     int *gemm_counters;                 // per-tile arrival counters, zero between launches
     size_t n_counters;
-    int *attn_counters;                 // [2 * max_batch * Hkv * 4] key-range arrivals per (stream, sequence, kv head, group of query heads)
+    int *attn_counters;                 // [attn_counter_count()] key-range arrivals per (stream, sequence, kv head, group of query heads)
     float *ssq;                         // [(d / 128) * 4][R] partial sums of h^2 for the fused RMSNorm
 };
 

@@ -22,6 +22,13 @@ def to_device(a: np.ndarray, device="cuda") -> torch.Tensor:
 
 
 class Engine:
+    GUARD = 8192                         # bytes of poisoned memory kept on either side of the workspace
+
+    def guards_intact(self) -> bool:
+        off = self.workspace.data_ptr() - self._ws_block.data_ptr()
+        before, after = self._ws_block[:off], self._ws_block[off + self.workspace.numel():]
+        return bool((before == 0xFF).all().item()) and bool((after == 0xFF).all().item())
+
     def __init__(self, wl: W.Workload, device="cuda", max_query: Optional[int] = None,
                  extra_ctx: int = 0, fill_context: bool = True):
         self.wl, self.device = wl, device
@@ -44,7 +51,11 @@ class Engine:
         assert nbytes > 0, "configuration rejected by viasd_workspace_bytes"
         # Poisoned on purpose (every float a NaN, every counter -1): the library has to initialise what it relies on,
         # and recycled device memory is not zero.
-        self.workspace = torch.full((nbytes,), 0xFF, dtype=torch.uint8, device=device)
+        # The library gets exactly the bytes it asked for, cut out of the middle of a larger block whose two ends
+        # serve as guard zones: anything written outside the workspace shows in guards_intact().
+        self._ws_block = torch.full((nbytes + 2 * self.GUARD,), 0xFF, dtype=torch.uint8, device=device)
+        off = (-self._ws_block.data_ptr()) % 256 + self.GUARD // 2
+        self.workspace = self._ws_block[off:off + nbytes]
         self.model = vb.init_model(self.cfg, self.embed, self.lm_head, self.final_norm, self.layers, mask,
                                    self.workspace)
         kv = lambda nl: torch.zeros((nl, wl.batch, s.n_kv_heads, self.max_ctx, s.head_dim), dtype=self.tdtype,

@@ -1,7 +1,7 @@
 """Helpers shared by the GPU parity tests: run the oracle on a workload, compare under the margin rule."""
 from __future__ import annotations
 
-from typing import List, Optional
+from typing import List, Optional, Sequence
 
 import numpy as np
 
@@ -43,26 +43,60 @@ def assert_logits_close(got, want, dtype: str, what: str = "logits"):
     return ma, rl
 
 
-def compare_resolution(seqs: List[tiers.SeqResult], n_acc, path, out_tok, n_emit, corr_src, eps_row: float):
+def pinned_prefix(s: tiers.SeqResult, eps_row: float):
+    """How far one sequence's result is fixed by the margin rule.
+
+    Walks the oracle's decisions in order and stops at the first whose margin does not exceed 4 * eps_row.
+    Returns (number of leading decisions that are pinned, number of path nodes fixed by them, whether every
+    decision is pinned).  The decisions before the first unpinned one at block row r fix the accepted path up
+    to the node that owns row r (node r - 1; nothing when r is the pending token's row).
+    """
+    n_pinned = 0
+    for dcs in s.decisions:
+        if dcs.margin > 4.0 * eps_row:
+            n_pinned += 1
+            continue
+        k = 0 if dcs.row == 0 else s.path.index(dcs.row - 1) + 1
+        return n_pinned, k, False
+    return n_pinned, s.n_acc, True
+
+
+def compare_resolution(seqs: List[tiers.SeqResult], n_acc, path, out_tok, n_emit, corr_src, eps_row: float,
+                       only: Optional[Sequence[int]] = None):
     """Margin rule: a decision is pinned when its oracle margin exceeds 4 * eps_row (eps_row = observed
-    max-abs logit difference).  Walk the oracle's decisions in order; everything up to the first unpinned
-    one must match exactly.  Returns (pinned decisions, total decisions, fully compared sequences)."""
+    max-abs logit difference).  Per sequence the oracle's decisions are walked in order; the accepted path
+    and the emitted tokens up to the first unpinned decision must match exactly (the whole result when
+    every decision is pinned).  ``only`` restricts the comparison to those sequences (the others count as
+    not compared).  Returns (pinned leading decisions, total decisions, sequences compared to the end)."""
     pinned = total = full = 0
     for b, s in enumerate(seqs):
-        ok_all = True
-        n_ok_path = 0          # accepted prefix known to be pinned
-        for dcs in s.decisions:
-            total += 1
-            if dcs.margin > 4.0 * eps_row:
-                pinned += 1
-            else:
-                ok_all = False
-                break
+        if only is not None and b not in only:
+            total += len(s.decisions)
+            continue
+        total += len(s.decisions)
+        n_pin, k, ok_all = pinned_prefix(s, eps_row)
+        pinned += n_pin
+        got_path = [int(x) for x in path[b][:int(n_acc[b])]]
+        got_tok = [int(x) for x in out_tok[b][:int(n_emit[b])]]
+        # the fixed prefix: the device accepted at least these nodes, in this order, and emitted their tokens
+        assert int(n_acc[b]) >= k, (b, int(n_acc[b]), k)
+        assert got_path[:k] == s.path[:k], (b, got_path, s.path, k)
+        assert got_tok[:k] == s.out_tok[:k], (b, got_tok, s.out_tok, k)
         if ok_all:
             full += 1
             assert int(n_acc[b]) == s.n_acc, (b, int(n_acc[b]), s.n_acc)
-            assert [int(x) for x in path[b][:s.n_acc]] == s.path, b
+            assert got_path == s.path, (b, got_path, s.path)
             assert int(n_emit[b]) == len(s.out_tok), b
-            assert [int(x) for x in out_tok[b][:len(s.out_tok)]] == s.out_tok, (b, out_tok[b], s.out_tok)
+            assert got_tok == s.out_tok, (b, got_tok, s.out_tok)
             assert int(corr_src[b]) == s.corr_src, b
     return pinned, total, full
+
+
+def assert_pinned(what: str, pinned: int, total: int, full: int, n_seq: int, min_frac: float, min_full: int):
+    """The share of decisions the margin rule fixes is a property of the workload (logit spread against the
+    bf16 path's error), so its floor is set per case from what is observed, less a margin; the message
+    carries the counts either way."""
+    msg = f"{what}: pinned decisions {pinned}/{total}, sequences compared to the end {full}/{n_seq}"
+    print("PINNED " + msg)
+    assert total == 0 or pinned / total >= min_frac, msg
+    assert full >= min_full, msg

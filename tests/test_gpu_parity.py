@@ -13,6 +13,10 @@ pytestmark = pytest.mark.gpu
 
 torch = pytest.importorskip("torch")
 
+# Least share of decisions the margin rule must fix (pinned leading decisions / all decisions) wherever the bf16 path's
+# logits decide; set from the shares observed on these workloads less a margin (printed by PU.assert_pinned).
+FLOOR_FRAC = 0.6
+
 
 def _engine(wl, **kw):
     from paper_2606_12243_b200.engine import Engine
@@ -44,7 +48,8 @@ def _prepare(wl, dt=np.float64, extra=0, step_no=0):
 # ---------------------------------------------------------------------------------------------
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 @pytest.mark.parametrize("rows,n,k", [(1, 64, 64), (5, 1024, 256), (9, 4096, 512), (9, 1000, 1408), (27, 776, 4096),
-                                      (56, 520, 640), (64, 256, 11008), (96, 384, 1024), (108, 2048, 512)])
+                                      (56, 520, 640), (64, 256, 11008), (96, 384, 1024), (108, 2048, 512),
+                                      (9, 512, 1000), (20, 300, 8), (33, 129, 72)])      # k not a multiple of the 64-wide k-block
 def test_gemm_matches_matmul(dtype, rows, n, k):
     vb = _vb()
     from paper_2606_12243_b200.engine import to_device
@@ -428,7 +433,7 @@ def test_verify_step_with_ragged_lengths(env, monkeypatch):
     pinned, total, full = PU.compare_resolution(want.seqs, res.n_acc.cpu().numpy(), res.path.cpu().numpy(),
                                                 res.out_tok.cpu().numpy(), res.n_emit.cpu().numpy(),
                                                 res.corr_src.cpu().numpy(), eps_row=max(e1, e2))
-    assert total == 0 or pinned / total > 0.6, (pinned, total)
+    PU.assert_pinned("ragged mini_13b", pinned, total, full, wl.batch, FLOOR_FRAC, wl.batch // 2)
     if full == wl.batch:
         assert eng.len.cpu().tolist() == [int(x) for x in st.lens]
         assert eng.pending.cpu().tolist() == [int(x) for x in st.pending]
@@ -438,6 +443,7 @@ def _check_verify_step(name):
     wl = W.get(name)
     vb = _vb()
     eng, st, si, model = _prepare(wl)
+    assert eng.guards_intact(), "viasd_init_model wrote outside the workspace it was given"
     lo, hi = W.thresholds(wl)
     want = step.verify_step(model, wl.shape, wl.routed, st, si.draft_tok, wl.parent, si.prow, si.drafter_logits,
                             lo, hi, PU.oracle_params(wl))
@@ -452,9 +458,30 @@ def _check_verify_step(name):
     pinned, total, full = PU.compare_resolution(want.seqs, res.n_acc.cpu().numpy(), res.path.cpu().numpy(),
                                                 res.out_tok.cpu().numpy(), res.n_emit.cpu().numpy(),
                                                 res.corr_src.cpu().numpy(), eps_row=max(e1, e2))
-    assert total == 0 or pinned / total > 0.6, (pinned, total)
+    PU.assert_pinned(name, pinned, total, full, wl.batch, FLOOR_FRAC, wl.batch // 2)
+    assert eng.guards_intact(), "a verify step wrote outside the workspace"
     if full == wl.batch:
         _check_state(eng, st, wl)
+
+
+@pytest.mark.parametrize("name", ["mini_13b", "mini_8b_tree", "mini_32b_b3"])
+def test_workspace_of_exactly_the_queried_size_is_enough(name):
+    """viasd_workspace_bytes() is a promise: the library is handed exactly that many bytes, poisoned, between two
+    poisoned guard zones, and neither viasd_init_model nor a verify step (a batch-8 multi-head shape; grouped heads with
+    four attention items per kv head; a batch of three) may touch the guards."""
+    wl = W.get(name)
+    vb = _vb()
+    eng = _engine(wl)
+    assert eng.workspace.numel() == vb.workspace_bytes(eng.cfg, len(eng.routed))
+    assert eng.guards_intact()
+    eng.set_inputs(W.step_inputs(wl))
+    sl, fl = eng.logits_buffer(), eng.logits_buffer()
+    res = vb.alloc_result(wl.batch, wl.n_nodes)
+    for i in range(2):
+        vb.verify_step(eng.model, eng.cache, eng.draft, eng.params(step=i), sl, fl, res)
+    torch.cuda.synchronize()
+    assert vb.get_stats(eng.model).device_status == 0
+    assert eng.guards_intact()
 
 
 # The split tiles of the GEMMs and the key ranges of the attention kernels are handed from CTA to CTA through global
@@ -648,11 +675,9 @@ def test_full_size_verify_step_matches_oracle(name):
     pinned, total, full = PU.compare_resolution(want.seqs, res.n_acc.cpu().numpy(), res.path.cpu().numpy(),
                                                 res.out_tok.cpu().numpy(), res.n_emit.cpu().numpy(),
                                                 res.corr_src.cpu().numpy(), eps_row=max(e1, e2))
-    print(f"{name} full-size: slim max-abs {e1:.2e} rel-L2 {r1:.2e}; full max-abs {e2:.2e} rel-L2 {r2:.2e}; "
-          f"pinned decisions {pinned}/{total}, sequences compared to the end {full}/{wl.batch}")
-    # every sequence whose decisions are all pinned was compared exactly inside compare_resolution
-    assert total == 0 or pinned / total > 0.6, (pinned, total)
-    assert full >= (wl.batch + 1) // 2
+    print(f"{name} full-size: slim max-abs {e1:.2e} rel-L2 {r1:.2e}; full max-abs {e2:.2e} rel-L2 {r2:.2e}")
+    # every sequence is compared up to its first unpinned decision inside compare_resolution
+    PU.assert_pinned(f"{name} full-size", pinned, total, full, wl.batch, FLOOR_FRAC, (wl.batch + 1) // 2)
     if full == wl.batch:
         _check_state(eng, st, wl)
 
@@ -717,13 +742,14 @@ def test_verify_step_in_algorithm_2_mode(name):
     assert np.array_equal(got_tier[pinned], want.tier[pinned])
     # confidence itself: one subtraction on logits that agree to e1
     assert np.abs(res.conf.cpu().numpy() - want.conf).max() <= 2 * e1 + 1e-6
-    if np.array_equal(got_tier, want.tier):
-        pinned_d, total, full = PU.compare_resolution(want.seqs, res.n_acc.cpu().numpy(), res.path.cpu().numpy(),
-                                                      res.out_tok.cpu().numpy(), res.n_emit.cpu().numpy(),
-                                                      res.corr_src.cpu().numpy(), eps_row=max(e1, e2))
-        assert total == 0 or pinned_d / total > 0.6, (pinned_d, total)
-        if full == wl.batch:
-            _check_state(eng, st, wl)
+    # the walk of a sequence is compared when all of its tiers came out as the oracle's
+    same = [b for b in range(wl.batch) if np.array_equal(got_tier[b], want.tier[b])]
+    pinned_d, total, full = PU.compare_resolution(want.seqs, res.n_acc.cpu().numpy(), res.path.cpu().numpy(),
+                                                  res.out_tok.cpu().numpy(), res.n_emit.cpu().numpy(),
+                                                  res.corr_src.cpu().numpy(), eps_row=max(e1, e2), only=same)
+    PU.assert_pinned(f"{name} (Algorithm 2 mode)", pinned_d, total, full, wl.batch, 0.5 if len(same) == wl.batch else 0.0, 0)
+    if full == wl.batch:
+        _check_state(eng, st, wl)
 
 
 # ---------------------------------------------------------------------------------------------
@@ -760,6 +786,6 @@ def test_verify_step_edge_shapes(name, parent, ctx):
     pinned, total, full = PU.compare_resolution(want.seqs, res.n_acc.cpu().numpy(), res.path.cpu().numpy(),
                                                 res.out_tok.cpu().numpy(), res.n_emit.cpu().numpy(),
                                                 res.corr_src.cpu().numpy(), eps_row=max(e1, e2))
-    assert total == 0 or pinned / total > 0.5, (pinned, total)
+    PU.assert_pinned(f"edge {name} {len(parent)} nodes ctx {ctx}", pinned, total, full, wl.batch, 0.5, 0)
     if full == wl.batch:
         _check_state(eng, st, wl)

@@ -431,6 +431,35 @@ def test_resolve_sampling_monte_carlo_matches_judges():
     assert r.out_tok == [3] and r.n_acc == 1 and r.corr_src == 0
 
 
+def test_sampling_bonus_token_is_a_draw_from_the_full_verifier_at_the_leaf():
+    """emit_bonus in sampling mode: when the whole draft is accepted, one more token is drawn from q at
+    the last accepted row (not the pending row, not q')."""
+    rng = np.random.default_rng(5)
+    V, n_trials = 6, 20000
+    q_root, q_leaf, qs = _rand_dist(rng, V), _rand_dist(rng, V), _rand_dist(rng, V)
+    assert np.abs(q_root - q_leaf).max() > 0.1 and np.abs(qs - q_leaf).max() > 0.1
+    fl = np.stack([_fake_logits(q_root), _fake_logits(q_leaf)])
+    sl = np.stack([_fake_logits(qs)] * 2)
+    dl = np.zeros((1, V))
+    cnt = np.zeros(V)
+    for i in range(n_trials):
+        P = tiers.Params(mode="sampling", seed=77, step=i, emit_bonus=True)
+        r = tiers.resolve_sequence(0, [2], (-1,), (0,), (0,), dl, sl, fl, P)      # tier 0: always accepted
+        assert r.n_acc == 1 and r.out_tok[0] == 2 and len(r.out_tok) == 2 and r.corr_src == 2
+        cnt[r.out_tok[1]] += 1
+    assert np.abs(cnt / n_trials - q_leaf).max() < 0.012, (cnt / n_trials, q_leaf)
+    # a temperature reshapes the draw: T = 2 gives softmax(log q / 2)
+    t2 = np.sqrt(q_leaf) / np.sqrt(q_leaf).sum()
+    cnt = np.zeros(V)
+    for i in range(n_trials):
+        P = tiers.Params(mode="sampling", seed=78, step=i, emit_bonus=True, temperature=2.0)
+        cnt[tiers.resolve_sequence(0, [2], (-1,), (0,), (0,), dl, sl, fl, P).out_tok[1]] += 1
+    assert np.abs(cnt / n_trials - t2).max() < 0.012
+    # without the flag nothing is added
+    r = tiers.resolve_sequence(0, [2], (-1,), (0,), (0,), dl, sl, fl, tiers.Params(mode="sampling"))
+    assert r.out_tok == [2] and r.corr_src == 0
+
+
 def test_uniform_hash_statistics_and_streams():
     k = tiers.stream_key(1, 2, 3, tiers.STREAM_GUMBEL)
     u = tiers.unit_vec(k, 5 << 32, 200000)
@@ -603,3 +632,81 @@ def test_tree_commit_moves_accepted_rows():
         for l in range(c.n_layers):
             assert np.allclose(c.k[l][0, :, :6], c2.k[l][0, :, :6], atol=1e-10)
             assert np.allclose(c.v[l][0, :, :6], c2.v[l][0, :, :6], atol=1e-10)
+
+
+# --------------------------------------------------------------------------
+# Algorithm 2 as printed: the slim verifier's own confidence gates the tiers
+# --------------------------------------------------------------------------
+def _uniform_attention_logits(E, toks, n_layers, eps):
+    """Closed form of the _OneLayerIdentity model on a chain: every layer adds to row i the mean of the
+    normalised rows 0..i; the head is the identity, so the logits are the final norm of the stream."""
+    nrm = lambda x: x / np.sqrt((x * x).mean(-1, keepdims=True) + eps)
+    h = E[toks].astype(np.float64)
+    for _ in range(n_layers):
+        a = nrm(h)
+        h = h + np.stack([a[:i + 1].mean(0) for i in range(len(toks))])
+    return nrm(h)
+
+
+def test_algorithm_2_gate_reads_the_slim_verifier_at_the_parent_row():
+    """conf_source 1 through oracle.step.verify_step: a drafted token is placed by q'_{t+j}, the slim
+    verifier's distribution that predicts its position (the row of its parent), with M' the maximum
+    of that row (App. B, Eq. B.1-B.3; Algorithm 2, the per-position loop), and with strict_break the
+    block ends exactly as the printed loop says.  The expected values come from the closed form of a
+    model with uniform attention and from the loop of Algorithm 2 written out here."""
+    s = W.ModelShape(2, 8, 2, 2, 4, 4, 8, dtype="f32")
+    rng = np.random.default_rng(3)
+    E = (rng.standard_normal((8, 8)) * 1.5).astype(np.float32)
+    wts = _OneLayerIdentity(s, E)
+    K, B = 3, 40
+    log_lo, log_hi = np.log(0.3), np.log(0.75)
+    routed = [0]
+    seen_regions, seen_ends, discriminating = set(), set(), 0
+    pend = rng.integers(0, 8, size=B)
+    draft = rng.integers(0, 8, size=(B, K))
+    st = step.new_state(s, 1, B, 16)
+    st.pending[:] = pend
+    dl = rng.standard_normal((B, K, 8)).astype(np.float32)           # drafter logits: must not be what gates
+    out = step.verify_step(wts, s, routed, st, draft, W.chain(K), tuple(range(K)), dl, log_lo, log_hi,
+                           tiers.Params(strict_break=True), conf_source=1, do_commit=False)
+    region = lambda d: 0 if d >= np.float32(log_hi) else (1 if d >= np.float32(log_lo) else 2)
+    for b in range(B):
+        toks = np.concatenate([[pend[b]], draft[b]])
+        S = _uniform_attention_logits(E, toks, 1, s.rms_eps)          # q' = layer 0 only
+        F = _uniform_attention_logits(E, toks, 2, s.rms_eps)          # q = both layers
+        assert np.allclose(out.slim_logits[b], S, atol=1e-9) and np.allclose(out.full_logits[b], F, atol=1e-9)
+        S32 = S.astype(np.float32)
+        want_tier = []
+        for j in range(K):
+            d_parent = np.float32(S32[j][draft[b, j]] - S32[j].max())         # row j predicts draft j
+            d_own = np.float32(S32[j + 1][draft[b, j]] - S32[j + 1].max())    # the node's own row: the wrong one
+            d_full = np.float32(F[j][draft[b, j]] - F[j].max())
+            d_draft = np.float32(dl[b, j][draft[b, j]] - dl[b, j].max())
+            want_tier.append(region(d_parent))
+            discriminating += (region(d_own) != region(d_parent)) + (region(d_full) != region(d_parent)) \
+                + (region(d_draft) != region(d_parent))
+            assert out.conf[b, j] == d_parent
+        assert list(out.tier[b]) == want_tier, (b, list(out.tier[b]), want_tier)
+        seen_regions.update(want_tier)
+        # Algorithm 2, lines of the per-position loop, greedy: accept in region A; in region B rewrite with q'
+        # and break; in region C ask q, accept if it agrees, else rewrite with q and break
+        emitted, src = [], 0
+        for j in range(K):
+            x = int(draft[b, j])
+            if want_tier[j] == 0:
+                emitted.append(x)
+                continue
+            judge = S if want_tier[j] == 1 else F
+            if int(np.argmax(judge[j])) == x:                        # cannot happen in region B: x is below the mode
+                emitted.append(x)
+                assert want_tier[j] == 2
+                continue
+            emitted.append(int(np.argmax(judge[j])))
+            src = want_tier[j]
+            break
+        r = out.seqs[b]
+        assert r.out_tok == emitted and r.corr_src == src, (b, r.out_tok, emitted, r.corr_src, src)
+        assert r.n_acc == len(emitted) - (1 if src else 0)
+        seen_ends.add(src)
+    assert seen_regions == {0, 1, 2} and seen_ends == {0, 1, 2}
+    assert discriminating > 20          # the other candidate rows would have placed many tokens elsewhere
