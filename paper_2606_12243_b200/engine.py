@@ -30,7 +30,11 @@ class Engine:
         return bool((before == 0xFF).all().item()) and bool((after == 0xFF).all().item())
 
     def __init__(self, wl: W.Workload, device="cuda", max_query: Optional[int] = None,
-                 extra_ctx: int = 0, fill_context: bool = True):
+                 extra_ctx: int = 0, fill_context=True, weights_from: Optional["Engine"] = None):
+        """fill_context: True = the generator's committed context (what the parity tests compare against);
+        "device" = values of the same distribution drawn on the device (timing sweeps over caches of tens of
+        GB, where only the shape matters); False = leave the caches empty.
+        weights_from: another engine of the same model shape and seed whose weight tensors are reused."""
         self.wl, self.device = wl, device
         s = wl.shape
         self.tdtype = torch.float32 if s.dtype == "f32" else torch.bfloat16
@@ -38,13 +42,19 @@ class Engine:
         self.max_ctx = wl.ctx + max(self.max_query, wl.rows) + extra_ctx
         self.cfg = vb.make_config(s.n_layers, s.d_model, s.n_heads, s.n_kv_heads, s.head_dim, s.d_ff, s.vocab,
                                   s.dtype, wl.batch, self.max_ctx, self.max_query, s.rms_eps, s.rope_theta)
-        gen = W.Model(wl)
-        self.embed = to_device(gen.tensor(-1, "embed"), device)
-        self.lm_head = to_device(gen.tensor(-1, "lm_head"), device)
-        self.final_norm = to_device(gen.tensor(-1, "final_norm"), device)
-        self.layers: List[Dict[str, torch.Tensor]] = []
-        for l in range(s.n_layers):
-            self.layers.append({k: to_device(v, device) for k, v in gen.layer(l).items()})
+        if weights_from is not None:
+            o = weights_from.wl
+            assert (o.shape, o.seed, o.weight_sigma, o.gain_jitter) == (s, wl.seed, wl.weight_sigma, wl.gain_jitter)
+            self.embed, self.lm_head, self.final_norm = weights_from.embed, weights_from.lm_head, weights_from.final_norm
+            self.layers: List[Dict[str, torch.Tensor]] = weights_from.layers
+        else:
+            gen = W.Model(wl)
+            self.embed = to_device(gen.tensor(-1, "embed"), device)
+            self.lm_head = to_device(gen.tensor(-1, "lm_head"), device)
+            self.final_norm = to_device(gen.tensor(-1, "final_norm"), device)
+            self.layers = []
+            for l in range(s.n_layers):
+                self.layers.append({k: to_device(v, device) for k, v in gen.layer(l).items()})
         self.routed = wl.routed
         mask = [1 if l in set(self.routed) else 0 for l in range(s.n_layers)]
         nbytes = vb.workspace_bytes(self.cfg, len(self.routed))
@@ -67,7 +77,9 @@ class Engine:
         self.tokens = torch.zeros((wl.batch, self.max_ctx), dtype=torch.int32, device=device)
         self.cache = vb.make_cache(self.k_full, self.v_full, self.k_slim, self.v_slim, self.len, self.pending,
                                    self.tokens)
-        if fill_context and not wl.real_prefill and wl.ctx > 0:
+        if fill_context == "device" and wl.ctx > 0:
+            self.fill_random_context()
+        elif fill_context and not wl.real_prefill and wl.ctx > 0:
             self.fill_synthetic_context()
         self.draft = None
         self.inputs = None
@@ -81,6 +93,16 @@ class Engine:
                 kc[o, :, :, :wl.ctx] = to_device(W.context_kv(wl, cache_id, o, 0), self.device)
                 vc[o, :, :, :wl.ctx] = to_device(W.context_kv(wl, cache_id, o, 1), self.device)
         self.len.fill_(wl.ctx)
+
+    def fill_random_context(self) -> None:
+        """Committed context drawn on the device, N(0, kv_sigma) like the generator's: for timing only."""
+        g = torch.Generator(device=self.device)
+        g.manual_seed(self.wl.seed)
+        sigma = W.kv_sigma(self.wl)
+        for t in (self.k_full, self.v_full, self.k_slim, self.v_slim):
+            for o in range(t.shape[0]):
+                t[o, :, :, :self.wl.ctx].normal_(0.0, sigma, generator=g)
+        self.len.fill_(self.wl.ctx)
 
     def prefill(self, prompt: np.ndarray) -> None:
         """Push a prompt [B, T] through both models with the library's own forward + commit calls."""

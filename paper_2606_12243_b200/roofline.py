@@ -69,3 +69,46 @@ def step_bytes(wl: Workload) -> dict:
     total_sep = full["total"] + slim["total"] + tier
     return dict(full=full, slim=slim, tier=tier, total=total_sep, flops=full["flops"] + slim["flops"], gemm=gemm_sep,
                 gemm_shared=gemm_shared, total_shared=total_sep - slim_weights)
+
+
+def call_bytes(wl: Workload) -> dict:
+    """Algorithmic bytes of the two small calls.  tier_accept: the tier kernel reads every gating row once, the row
+    statistics read every drafter / slim / full logits row once (the accept walk then works from the statistics).
+    kv_commit: at most depth-of-tree rows of K and V per layer and kv head move (read + write), in both caches."""
+    s = wl.shape
+    R = len(set(wl.parent))
+    tier_accept = wl.batch * R * s.vocab * 4 + (2 * wl.batch * wl.rows + wl.batch * R) * s.vocab * 4
+    depth = {-1: 0}
+    for n, p in enumerate(wl.parent):
+        depth[n] = depth[p] + 1
+    kv_commit = 2 * (s.n_layers + wl.n_routed) * wl.batch * max(depth.values()) * 2 * s.n_kv_heads * s.head_dim * s.elem_bytes
+    return dict(tier_accept=tier_accept, kv_commit=kv_commit)
+
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of gemm_tc_kernel, in MB, from the ncu
+# captures summarised under profiles/ (gemm_tc_kernel_*_layer_shapes.md), keyed by (output features, input features)
+# of the launch: QKV, O, gate/up (both matrices), down, head.  The weights are all but a per cent of it at the token
+# rows of these workloads (activation tiles hit in L2), so one figure serves launches of 9 to 54 rows.
+NCU_GEMM_TRAFFIC_MB = {
+    # 7B layer shapes (captured with 18 token rows)
+    (12288, 4096): 105.2, (4096, 4096): 34.1, (22016, 4096): 185.3, (4096, 11008): 96.6, (32000, 4096): 271.6,
+}
+
+
+def gemm_traffic(wl: Workload):
+    """Measured DRAM bytes of the step's GEMM launches: per-launch ncu figures of the workload's layer shapes scaled
+    by the launches of the step (traffic is per launch, and every layer launches the same shapes).  None when a
+    shape of this workload has no capture."""
+    s = wl.shape
+    qd, kvd = s.n_heads * s.head_dim, s.n_kv_heads * s.head_dim
+    shapes = [(qd + 2 * kvd, s.d_model), (s.d_model, qd), (2 * s.d_ff, s.d_model), (s.d_model, s.d_ff)]
+    one_sweep = 2 * wl.batch * wl.rows <= 128
+    layer_launches = s.n_layers if one_sweep else s.n_layers + wl.n_routed
+    head_launches = 1 if one_sweep else 2
+    total = 0.0
+    for n, k in shapes + [(s.vocab, s.d_model)]:
+        t = NCU_GEMM_TRAFFIC_MB.get((n, k))
+        if t is None:
+            return None
+        total += t * (head_launches if n == s.vocab else layer_launches)
+    return int(total * 1e6)

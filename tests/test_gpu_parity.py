@@ -15,7 +15,12 @@ torch = pytest.importorskip("torch")
 
 # Least share of decisions the margin rule must fix (pinned leading decisions / all decisions) wherever the bf16 path's
 # logits decide; set from the shares observed on these workloads less a margin (printed by PU.assert_pinned).
-FLOOR_FRAC = 0.6
+FLOOR_FRAC = 0.85       # observed: 0.90 (16 sequences of the shrunken 32B shape) to 1.0
+
+
+def _floor_full(batch):
+    """Least number of sequences that must be compared to their end (observed: 13 of 16, 7 of 8, else all)."""
+    return -(-3 * batch // 4)
 
 
 def _engine(wl, **kw):
@@ -433,7 +438,7 @@ def test_verify_step_with_ragged_lengths(env, monkeypatch):
     pinned, total, full = PU.compare_resolution(want.seqs, res.n_acc.cpu().numpy(), res.path.cpu().numpy(),
                                                 res.out_tok.cpu().numpy(), res.n_emit.cpu().numpy(),
                                                 res.corr_src.cpu().numpy(), eps_row=max(e1, e2))
-    PU.assert_pinned("ragged mini_13b", pinned, total, full, wl.batch, FLOOR_FRAC, wl.batch // 2)
+    PU.assert_pinned("ragged mini_13b", pinned, total, full, wl.batch, FLOOR_FRAC, _floor_full(wl.batch))
     if full == wl.batch:
         assert eng.len.cpu().tolist() == [int(x) for x in st.lens]
         assert eng.pending.cpu().tolist() == [int(x) for x in st.pending]
@@ -458,7 +463,7 @@ def _check_verify_step(name):
     pinned, total, full = PU.compare_resolution(want.seqs, res.n_acc.cpu().numpy(), res.path.cpu().numpy(),
                                                 res.out_tok.cpu().numpy(), res.n_emit.cpu().numpy(),
                                                 res.corr_src.cpu().numpy(), eps_row=max(e1, e2))
-    PU.assert_pinned(name, pinned, total, full, wl.batch, FLOOR_FRAC, wl.batch // 2)
+    PU.assert_pinned(name, pinned, total, full, wl.batch, FLOOR_FRAC, _floor_full(wl.batch))
     assert eng.guards_intact(), "a verify step wrote outside the workspace"
     if full == wl.batch:
         _check_state(eng, st, wl)
@@ -477,7 +482,9 @@ def test_workspace_of_exactly_the_queried_size_is_enough(name):
     eng.set_inputs(W.step_inputs(wl))
     sl, fl = eng.logits_buffer(), eng.logits_buffer()
     res = vb.alloc_result(wl.batch, wl.n_nodes)
+    len0 = eng.len.clone()
     for i in range(2):
+        eng.len.copy_(len0)                 # the cache has room for one block beyond the context
         vb.verify_step(eng.model, eng.cache, eng.draft, eng.params(step=i), sl, fl, res)
     torch.cuda.synchronize()
     assert vb.get_stats(eng.model).device_status == 0
@@ -677,7 +684,7 @@ def test_full_size_verify_step_matches_oracle(name):
                                                 res.corr_src.cpu().numpy(), eps_row=max(e1, e2))
     print(f"{name} full-size: slim max-abs {e1:.2e} rel-L2 {r1:.2e}; full max-abs {e2:.2e} rel-L2 {r2:.2e}")
     # every sequence is compared up to its first unpinned decision inside compare_resolution
-    PU.assert_pinned(f"{name} full-size", pinned, total, full, wl.batch, FLOOR_FRAC, (wl.batch + 1) // 2)
+    PU.assert_pinned(f"{name} full-size", pinned, total, full, wl.batch, FLOOR_FRAC, _floor_full(wl.batch))
     if full == wl.batch:
         _check_state(eng, st, wl)
 
@@ -747,7 +754,7 @@ def test_verify_step_in_algorithm_2_mode(name):
     pinned_d, total, full = PU.compare_resolution(want.seqs, res.n_acc.cpu().numpy(), res.path.cpu().numpy(),
                                                   res.out_tok.cpu().numpy(), res.n_emit.cpu().numpy(),
                                                   res.corr_src.cpu().numpy(), eps_row=max(e1, e2), only=same)
-    PU.assert_pinned(f"{name} (Algorithm 2 mode)", pinned_d, total, full, wl.batch, 0.5 if len(same) == wl.batch else 0.0, 0)
+    PU.assert_pinned(f"{name} (Algorithm 2 mode)", pinned_d, total, full, wl.batch, FLOOR_FRAC if len(same) == wl.batch else 0.0, 0)
     if full == wl.batch:
         _check_state(eng, st, wl)
 
@@ -786,6 +793,6 @@ def test_verify_step_edge_shapes(name, parent, ctx):
     pinned, total, full = PU.compare_resolution(want.seqs, res.n_acc.cpu().numpy(), res.path.cpu().numpy(),
                                                 res.out_tok.cpu().numpy(), res.n_emit.cpu().numpy(),
                                                 res.corr_src.cpu().numpy(), eps_row=max(e1, e2))
-    PU.assert_pinned(f"edge {name} {len(parent)} nodes ctx {ctx}", pinned, total, full, wl.batch, 0.5, 0)
+    PU.assert_pinned(f"edge {name} {len(parent)} nodes ctx {ctx}", pinned, total, full, wl.batch, 0.7, wl.batch // 2)
     if full == wl.batch:
         _check_state(eng, st, wl)
