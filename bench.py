@@ -308,17 +308,19 @@ class Bench:
 
     def kv_commit(self, i):
         e = self.eng
-        self.rewind()
         self.vb.kv_commit(e.model, e.cache, e.draft, self.res)
 
     def time_each(self, fn, n: int, warmup: int = 3):
-        """n individually timed calls (one event pair each) -> (median ms, min ms)."""
+        """n individually timed calls (one event pair each; the cache is rewound before each, outside the pair)
+        -> (median ms, min ms)."""
         torch = self.torch
         for i in range(warmup):
+            self.rewind()
             fn(i)
         ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
         torch.cuda.synchronize()
         for i, (a, b) in enumerate(ev):
+            self.rewind()
             a.record(self.stream)
             fn(i)
             b.record(self.stream)

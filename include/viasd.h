@@ -143,18 +143,42 @@ int viasd_tier_accept(viasd_model *m, const viasd_draft *draft, const viasd_para
                       const float *slim_logits, const float *full_logits, int phase, viasd_result *result,
                       void *stream);
 
-/* Commit: move the accepted path's K/V rows to slots len+1.., len += n_emit, pending = last emitted
- * token, committed ids appended to cache.tokens.  Rejected rows are left beyond len (rollback). */
+/* Commit (Algorithm 1, the lines after the prefix is chosen: append the accepted prefix and the regenerated
+ * token, discard the remaining suffix, advance t; Sec. 3.5 step 4): move the accepted path's K/V rows to
+ * slots len+1.., len += n_emit, pending = last emitted token, committed ids appended to cache.tokens.
+ * Rejected rows are left beyond len: rollback is not keeping them. */
 int viasd_kv_commit(viasd_model *m, viasd_cache *cache, const viasd_draft *draft, const viasd_result *result,
                     void *stream);
 
-/* tier -> slim forward -> full forward -> accept -> commit, identical to calling the pieces.
- * slim_logits / full_logits: caller's buffers [B, M, vocab], filled as a side effect. */
+/* tier -> slim forward -> full forward -> accept -> commit, identical to calling the pieces (one decoding
+ * cycle: Algorithm 1, body of the loop; Algorithm 2 from the parallel run of q' to the append).
+ * slim_logits / full_logits: caller's buffers [B, M, vocab], filled as a side effect; both are required (the
+ * workspace holds no logits: at the largest geometries they would be over a gigabyte). */
 int viasd_verify_step(viasd_model *m, viasd_cache *cache, const viasd_draft *draft, const viasd_params *params,
                       float *slim_logits, float *full_logits, viasd_result *result, void *stream);
 
 /* Copies the device counters out; synchronises `stream`. */
 int viasd_get_stats(viasd_model *m, viasd_stats *host_out, void *stream);
+
+/* Tuning switches of one handle (the paper has no counterpart).  The defaults are what the benchmark measures; the
+ * tests use the switches to force every kernel onto every shape.  Takes effect from the next call on; results stay
+ * within the stated tolerances under every setting, but their last bits may change with it.
+ * Errors: EINVAL (null handle, unknown option, value out of range). */
+enum {
+    VIASD_OPT_ATTENTION_KERNEL = 0,    /* 0 choose by shape (default), 1 mma.sync, 2 tcgen05 with query rows on the
+                                          TMEM lanes, 3 tcgen05 with keys on the lanes (where the shape allows) */
+    VIASD_OPT_ATTENTION_SPLITS,        /* key ranges per (sequence, kv head), 1..16; 0 = cost model (default) */
+    VIASD_OPT_ATTENTION_LO,            /* mma.sync kernel: hi/lo split of queries and probabilities 2 (default),
+                                          queries only 1, neither 0 (fails the logit tolerance at full size) */
+    VIASD_OPT_ACCEPT_TEAM,             /* CTAs per sequence in the accept walk: 1, 2, 4, 8; 0 = by mode and vocabulary */
+    VIASD_OPT_DUAL_MAX_ROWS,           /* most token rows (both verifiers together) that viasd_verify_step runs as one
+                                          sweep over the layers, 0..128 (default 128); above it the passes run in turn */
+    VIASD_OPT_TK_GRID,                 /* keys-on-lanes attention with tiles dealt evenly: CTAs to use; 0 = one per SM */
+    VIASD_OPT_TK_FLAT,                 /* keys-on-lanes attention: deal tiles 1, key ranges 0; -1 = by shape (default) */
+    VIASD_OPT_GEMM_RING_KB,            /* stream-K GEMM: shared-memory ring in KB, 32..200; 0 = default (200) */
+    VIASD_OPT_GEMM_EPI_GROUPS          /* stream-K GEMM: groups of four epilogue warps, 1 or 2; 0 = by token tile */
+};
+int viasd_set_option(viasd_model *m, int option, int value);
 
 void viasd_free_model(viasd_model *m);
 const char *viasd_strerror(int code);

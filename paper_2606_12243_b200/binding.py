@@ -21,7 +21,12 @@ VIASD_OK, VIASD_EINVAL, VIASD_ECAPACITY, VIASD_ECUDA, VIASD_EDEVICE, VIASD_EUNSU
 EXPORTS = ["viasd_workspace_bytes", "viasd_init_model", "viasd_full_forward", "viasd_slim_forward",
            "viasd_tier_accept", "viasd_kv_commit", "viasd_verify_step", "viasd_get_stats",
            "viasd_free_model", "viasd_strerror", "viasd_last_cuda_error", "viasd_gemm_scratch_bytes",
-           "viasd_gemm", "viasd_gemm_static", "viasd_kl_cost", "viasd_region_mass", "viasd_launch_count", "viasd_set_timing", "viasd_get_timing"]
+           "viasd_gemm", "viasd_gemm_static", "viasd_kl_cost", "viasd_region_mass", "viasd_launch_count", "viasd_set_timing", "viasd_get_timing",
+           "viasd_set_option"]
+
+OPTIONS = {"attention_kernel": 0, "attention_splits": 1, "attention_lo": 2, "accept_team": 3, "dual_max_rows": 4,
+           "tk_grid": 5, "tk_flat": 6, "gemm_ring_kb": 7, "gemm_epi_groups": 8}
+ATTENTION_KERNELS = {"auto": 0, "mma": 1, "tc": 2, "tk": 3}
 
 TIMING_CLASSES = ["gemm", "attention", "norm", "rope", "embed", "tier_accept", "commit"]
 
@@ -118,6 +123,7 @@ def lib() -> C.CDLL:
                                     C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]
         l.viasd_region_mass.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_float, C.c_float, C.c_float,
                                         C.c_void_p, C.c_void_p, C.c_void_p]
+        l.viasd_set_option.argtypes = [C.c_void_p, C.c_int, C.c_int]
         l.viasd_launch_count.restype = C.c_ulonglong
         l.viasd_set_timing.argtypes = [C.c_void_p, C.c_int]
         l.viasd_get_timing.argtypes = [C.c_void_p, C.POINTER(Timing), C.c_void_p]
@@ -277,6 +283,13 @@ def gemm(x: torch.Tensor, w: torch.Tensor, y: torch.Tensor, scratch: torch.Tenso
     dtype = 0 if x.dtype == torch.float32 else 1
     _check(lib().viasd_gemm(_ptr(x), _ptr(w), _ptr(y), rows, n, k, dtype, _ptr(scratch),
                             scratch.numel() * scratch.element_size(), _stream(stream)), "viasd_gemm")
+
+
+def set_option(m: Model, option: str, value) -> None:
+    """viasd_set_option by name; attention_kernel also takes "auto" / "mma" / "tc" / "tk"."""
+    if option == "attention_kernel" and isinstance(value, str):
+        value = ATTENTION_KERNELS[value]
+    _check(lib().viasd_set_option(m.handle, OPTIONS[option], int(value)), "viasd_set_option")
 
 
 def launch_count() -> int:

@@ -88,6 +88,22 @@ int timed(viasd_model *m, int cls, cudaStream_t st, F &&f) {
     return f();
 }
 
+int env_int(const char *name, int dflt) { const char *e = getenv(name); return e && *e ? atoi(e) : dflt; }
+
+// Initial option values: the defaults, or what the VIASD_* environment variables say (read here, once per model).
+void default_options(ModelOptions &o) {
+    o.attn_kernel = 0;
+    if (const char *e = getenv("VIASD_ATTN")) o.attn_kernel = strcmp(e, "mma") == 0 ? 1 : strcmp(e, "tc") == 0 ? 2 : strcmp(e, "tk") == 0 ? 3 : 0;
+    o.attn_splits = env_int("VIASD_ATTN_NSPLIT", 0);
+    o.attn_lo = env_int("VIASD_ATTN_LO", 2);
+    o.accept_team = env_int("VIASD_ACCEPT_TEAM", 0);
+    o.dual_max_rows = env_int("VIASD_DUAL_MAX", 128);
+    o.tk_grid = env_int("VIASD_TK_GRID", 0);
+    o.tk_flat = env_int("VIASD_TK_FLAT", -1);
+    o.ring_kb = env_int("VIASD_TC_RING_KB", 0);
+    o.epi_groups = env_int("VIASD_TC_EPI_GROUPS", 0);
+}
+
 int check_config(const viasd_config *c) {
     if (!c) return VIASD_EINVAL;
     if (c->n_layers < 1 || c->n_layers > 512 || c->d_model < 8 || c->n_heads < 1 || c->n_kv_heads < 1) return VIASD_EINVAL;
@@ -147,6 +163,7 @@ int run_gemm(viasd_model *m, const GemmCall &g, int rows, cudaStream_t st) {
         L.out_f32 = g.out_f32; L.out_act = g.out_act; L.act_plane = g.act_plane; L.ld_out = g.ld_out;
         L.scratch = m->ws.gemm_scratch; L.counters = m->ws.gemm_counters; L.status = &m->ws.stats->device_status;
         L.sm_count = m->sm_count;
+        L.ring_kb = m->opt.ring_kb; L.epi_groups = m->opt.epi_groups;
         int rc = launch_gemm_tc(L, st);
         if (rc) return rc;
     }
@@ -185,6 +202,7 @@ int forward_sweep(viasd_model *m, const viasd_cache *cache, const viasd_draft *d
                 L.rows = nr; L.row0 = row0; L.nt = nt;
                 L.scratch = m->ws.gemm_scratch; L.counters = m->ws.gemm_counters; L.status = &m->ws.stats->device_status;
                 L.sm_count = m->sm_count;
+                L.ring_kb = m->opt.ring_kb; L.epi_groups = m->opt.epi_groups;
                 L.ssq_stride = (int)R; L.inv_d = 1.0f / (float)c.d_model; L.eps = c.rms_eps;
                 L.split_row = dual ? rows : 0;
                 int r2 = launch_gemm_tc(L, st);
@@ -354,6 +372,7 @@ int viasd_init_model(const viasd_config *cfg, const viasd_weights *w, const unsi
     viasd_model *m = new (std::nothrow) viasd_model();
     if (!m) return VIASD_EINVAL;
     memset(&m->timer, 0, sizeof(m->timer));
+    default_options(m->opt);
     m->cfg = *cfg;
     m->sm_count = prop.multiProcessorCount;
     m->n_routed = 0;
@@ -490,9 +509,7 @@ int viasd_verify_step(viasd_model *m, viasd_cache *cache, const viasd_draft *dra
     // Both verifiers in one sweep over the layers (routed layers' weights are read once for both) while the two
     // row streams together fit one launch (128 token rows: an MMA of 256 columns with the hi/lo planes); beyond
     // that a sweep would stream every routed layer twice anyway, and the passes run one after the other.
-    int dual_max = 128;                      // VIASD_DUAL_MAX: most rows (both streams together) the one-sweep schedule takes
-    if (const char *e = getenv("VIASD_DUAL_MAX")) dual_max = atoi(e);
-    if (m && m->fused && draft && 2 * draft->batch * (draft->n_nodes + 1) <= dual_max) {
+    if (m && m->fused && draft && 2 * draft->batch * (draft->n_nodes + 1) <= m->opt.dual_max_rows) {
         if ((rc = check_draft(m, draft)) || (rc = check_cache(cache))) return rc;
         if ((rc = forward_sweep(m, cache, draft, 2, full_logits, slim_logits, (cudaStream_t)stream))) return rc;
         if ((rc = tier_accept_impl(m, draft, params, slim_logits, full_logits, 3, result, true, stream))) return rc;
@@ -522,6 +539,24 @@ int viasd_get_stats(viasd_model *m, viasd_stats *host_out, void *stream) {
     host_out->device_status = s.device_status;
     host_out->need_slim = s.need_slim;
     host_out->need_full = s.need_full;
+    return VIASD_OK;
+}
+
+int viasd_set_option(viasd_model *m, int option, int value) {
+    if (!m) return VIASD_EINVAL;
+    ModelOptions &o = m->opt;
+    switch (option) {
+    case VIASD_OPT_ATTENTION_KERNEL: if (value < 0 || value > 3) return VIASD_EINVAL; o.attn_kernel = value; break;
+    case VIASD_OPT_ATTENTION_SPLITS: if (value < 0 || value > 16) return VIASD_EINVAL; o.attn_splits = value; break;
+    case VIASD_OPT_ATTENTION_LO: if (value < 0 || value > 2) return VIASD_EINVAL; o.attn_lo = value; break;
+    case VIASD_OPT_ACCEPT_TEAM: if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8) return VIASD_EINVAL; o.accept_team = value; break;
+    case VIASD_OPT_DUAL_MAX_ROWS: if (value < 0 || value > 128) return VIASD_EINVAL; o.dual_max_rows = value; break;
+    case VIASD_OPT_TK_GRID: if (value < 0) return VIASD_EINVAL; o.tk_grid = value; break;
+    case VIASD_OPT_TK_FLAT: if (value < -1 || value > 1) return VIASD_EINVAL; o.tk_flat = value; break;
+    case VIASD_OPT_GEMM_RING_KB: if (value != 0 && (value < 32 || value > 200)) return VIASD_EINVAL; o.ring_kb = value; break;
+    case VIASD_OPT_GEMM_EPI_GROUPS: if (value < 0 || value > 2) return VIASD_EINVAL; o.epi_groups = value; break;
+    default: return VIASD_EINVAL;
+    }
     return VIASD_OK;
 }
 

@@ -195,7 +195,7 @@ static int mma_nsplit(const viasd_model *m, int batch, int M, int streams, bool 
         }
         if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
     }
-    if (const char *e = getenv("VIASD_ATTN_NSPLIT")) { const int v = atoi(e); if (v >= 1 && v <= max_s) best = v; }   // measurement
+    if (m->opt.attn_splits >= 1 && m->opt.attn_splits <= max_s) best = m->opt.attn_splits;
     size_t per_split = (size_t)streams * batch * c.n_heads * M * (c.head_dim + 2) * sizeof(float) * reps;
     while (best > 1 && per_split * best > m->ws.part_bytes) --best;
     return best;
@@ -205,10 +205,9 @@ static int mma_nsplit(const viasd_model *m, int batch, int M, int streams, bool 
 static int mma_attention(viasd_model *m, const void *kc, const void *vc, bool slim, int layer_ord, const void *kc2,
                          const void *vc2, int layer_ord2, int streams, int batch, int M, cudaStream_t st) {
     const viasd_config &c = m->cfg;
-    // VIASD_ATTN: "mma" = mma.sync kernel, "tc" = tcgen05 with query rows on the TMEM lanes, "tk" = tcgen05 with keys on
-    // the lanes (few query rows only).  Default: tk where it applies, else mma.
-    int kind = 3;                            // 0 mma, 1 tc, 2 tk, 3 default (read per call: a test may switch kernels)
-    if (const char *e = getenv("VIASD_ATTN")) kind = strcmp(e, "mma") == 0 ? 0 : strcmp(e, "tc") == 0 ? 1 : strcmp(e, "tk") == 0 ? 2 : 3;
+    // Which kernel (VIASD_OPT_ATTENTION_KERNEL): the mma.sync kernel, tcgen05 with the query rows on the TMEM lanes, or
+    // tcgen05 with the keys on the lanes (few query rows only).  Default: keys-on-lanes where it applies, else mma.sync.
+    const int kind = m->opt.attn_kernel == 1 ? 0 : m->opt.attn_kernel == 2 ? 1 : m->opt.attn_kernel == 3 ? 2 : 3;   // 0 mma, 1 tc, 2 tk, 3 default
     const int QR = (c.n_heads / c.n_kv_heads) * M;
     // keys-on-lanes pays off when a CTA streams many tiles; with a handful per CTA (one short sequence) the
     // mma.sync kernel's shorter latency chain wins
@@ -229,10 +228,9 @@ static int mma_attention(viasd_model *m, const void *kc, const void *vc, bool sl
         // has its 16 slots per (row, head): whole (sequence, head) items leave SMs idle (320 items on 148 SMs: a
         // quarter of them).  Its merges are then always fused.  Not with more than 16 query rows per kv head: there an
         // item's fixed cost (staging 32 rows of queries, 32 rows of results) is worth a dozen tiles, and the extra
-        // item per CTA cost more than the balance won (32B batch-16 step 36.5 -> 39.0 ms).  VIASD_TK_FLAT=0/1 overrides.
-        const char *e = getenv("VIASD_TK_FLAT");
+        // item per CTA cost more than the balance won (32B batch-16 step 36.5 -> 39.0 ms).  VIASD_OPT_TK_FLAT overrides.
         const size_t need = (size_t)streams * batch * c.n_heads * M * 16 * (c.head_dim + 2) * sizeof(float);
-        if ((e ? atoi(e) != 0 : QR <= 16) && subs == 1 && need <= m->ws.part_bytes)
+        if ((m->opt.tk_flat >= 0 ? m->opt.tk_flat != 0 : QR <= 16) && subs == 1 && need <= m->ws.part_bytes)
             return launch_attention_tk(m, kc, vc, slim, layer_ord, kc2, vc2, layer_ord2, streams, batch, M, 0, 1, st);
         rc = launch_attention_tk(m, kc, vc, slim, layer_ord, kc2, vc2, layer_ord2, streams, batch, M, nsplit, fuse ? 1 : 0, st);
     }

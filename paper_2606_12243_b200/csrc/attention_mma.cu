@@ -593,18 +593,16 @@ int launch_attention_mma(viasd_model *m, const void *kc, const void *vc, bool sl
     // three stages (two tiles in flight while one is consumed) when the rest of the CTA's shared memory allows
     a.nstage = 1024 + 3 * (size_t)STAGE_BYTES + q_bytes + osm_bytes <= 226 * 1024 ? 3 : 2;
     const size_t smem = 1024 + a.nstage * (size_t)STAGE_BYTES + q_bytes + osm_bytes;
-    static bool attr_done = false;
-    if (!attr_done) {
+    static bool attr_done[64];
+    if (first_use_on_device(attr_done)) {
         CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
         CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
         CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
-        attr_done = true;
     }
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
     pdl_config(cfg, attr, dim3(grid), dim3(WARPS * 32), smem, st);
-    static int lo_mode = -1;                 // VIASD_ATTN_LO: 2 = hi/lo for Q and P, 1 = hi/lo for Q only, 0 = plain bf16
-    if (lo_mode < 0) { const char *e = getenv("VIASD_ATTN_LO"); lo_mode = e ? atoi(e) : 2; }
+    const int lo_mode = m->opt.attn_lo;      // 2 = hi/lo for Q and P, 1 = hi/lo for Q only, 0 = plain bf16
     if (lo_mode >= 2) CUDA_TRY(cudaLaunchKernelEx(&cfg, attention_mma_kernel<true, true>, cm.k, cm.v, cm2->k, cm2->v, a));
     else if (lo_mode == 1) CUDA_TRY(cudaLaunchKernelEx(&cfg, attention_mma_kernel<false, true>, cm.k, cm.v, cm2->k, cm2->v, a));
     else CUDA_TRY(cudaLaunchKernelEx(&cfg, attention_mma_kernel<false, false>, cm.k, cm.v, cm2->k, cm2->v, a));

@@ -645,10 +645,9 @@ int launch_attention_tc(viasd_model *m, const void *kc, const void *vc, bool sli
     const size_t q_bytes = a.q_bytes;
     a.nstage = 1024 + q_bytes + 3 * (size_t)STAGE_BYTES <= 220 * 1024 ? 3 : 2;
     const size_t smem = 1024 + q_bytes + a.nstage * (size_t)STAGE_BYTES;
-    static bool attr_done = false;
-    if (!attr_done) {
+    static bool attr_done[64];
+    if (first_use_on_device(attr_done)) {
         CUDA_TRY(cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
-        attr_done = true;
     }
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];

@@ -760,7 +760,7 @@ int launch_attention_tk(viasd_model *m, const void *kc, const void *vc, bool sli
         // tiles dealt evenly: one range per CTA and row stream, cut by the kernel from the lengths; merges are fused
         a.flat = 1; a.part_slots = 16; a.nsplit = 1; a.fuse_merge = 1; a.n_items = 0; a.items_per_cta = 0;
         grid = m->sm_count;
-        if (const char *e = getenv("VIASD_TK_GRID")) { const int v = atoi(e); if (v >= 1 && v < grid) grid = v; }   // tests: long ranges per CTA on small cases
+        if (m->opt.tk_grid >= 1 && m->opt.tk_grid < grid) grid = m->opt.tk_grid;     // tests: long ranges per CTA on small cases
     } else {
         a.flat = 0; a.part_slots = nsplit;
         a.n_items = streams * batch * c.n_kv_heads * subs * nsplit;
@@ -782,12 +782,11 @@ int launch_attention_tk(viasd_model *m, const void *kc, const void *vc, bool sli
         a.nk = a.nv = 1024 + op_bytes + 3 * (size_t)(2 * SLOT_BYTES) <= 220 * 1024 ? 3 : 2;
         smem = 1024 + op_bytes + a.nk * (size_t)(2 * SLOT_BYTES);
     }
-    static bool attr_done = false;
-    if (!attr_done) {
+    static bool attr_done[64];
+    if (first_use_on_device(attr_done)) {
         CUDA_TRY(cudaFuncSetAttribute(attention_tk_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024));
         CUDA_TRY(cudaFuncSetAttribute(attention_tk_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024));
         CUDA_TRY(cudaFuncSetAttribute(attention_tk_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024));
-        attr_done = true;
     }
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];

@@ -78,8 +78,23 @@ struct KernelTimer {
     bool on;
 };
 
+// Tuning switches of one model (viasd_set_option; the VIASD_* environment variables give their initial values, read
+// once in viasd_init_model).  The defaults are what is measured; tests use them to force every kernel onto every shape.
+struct ModelOptions {
+    int attn_kernel;        // VIASD_OPT_ATTENTION_KERNEL: 0 choose by shape, 1 mma.sync, 2 tcgen05 rows-on-lanes, 3 tcgen05 keys-on-lanes
+    int attn_splits;        // VIASD_OPT_ATTENTION_SPLITS: key ranges per (sequence, kv head); 0 = cost model
+    int attn_lo;            // VIASD_OPT_ATTENTION_LO: mma.sync kernel, hi/lo split of Q and P (2), of Q only (1), none (0)
+    int accept_team;        // VIASD_OPT_ACCEPT_TEAM: CTAs per sequence in the accept walk; 0 = by mode and vocabulary
+    int dual_max_rows;      // VIASD_OPT_DUAL_MAX_ROWS: most rows (both verifiers) the one-sweep schedule takes
+    int tk_grid;            // VIASD_OPT_TK_GRID: CTAs of the keys-on-lanes kernel when tiles are dealt evenly; 0 = one per SM
+    int tk_flat;            // VIASD_OPT_TK_FLAT: deal tiles (1) or key ranges (0); -1 = by shape
+    int ring_kb;            // VIASD_OPT_GEMM_RING_KB: shared-memory ring of the stream-K GEMM
+    int epi_groups;         // VIASD_OPT_GEMM_EPI_GROUPS: groups of four epilogue warps; 0 = by token tile
+};
+
 struct viasd_model {
     KernelTimer timer;
+    ModelOptions opt;
     viasd_config cfg;
     int n_routed;
     int routed[512];                    // routed layer ids, increasing
@@ -107,6 +122,16 @@ extern unsigned long long g_launch_count;
         if (e__ != cudaSuccess) { g_last_cuda_error = (int)e__; return VIASD_ECUDA; } \
     } while (0)
 #define LAUNCH_CHECK() do { ++g_launch_count; CUDA_TRY(cudaGetLastError()); } while (0)
+
+// cudaFuncSetAttribute applies to the current device only: remembers, per device, whether a launcher has set its
+// kernels' attributes there.  Returns true the first time it is asked about (flags, current device).
+inline bool first_use_on_device(bool (&flags)[64]) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;     // unknown: set them again, which is harmless
+    const bool first = !flags[dev];
+    flags[dev] = true;
+    return first;
+}
 
 // Programmatic dependent launch: a kernel launched with this configuration may begin (prologue, weight
 // prefetch) while the kernel before it in the stream is still finishing; it must execute griddepcontrol.wait

@@ -584,10 +584,9 @@ int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {
     grid = (units + p.units_per_cta - 1) / p.units_per_cta;
     const int nacc = dual ? 2 : 1;
     const size_t stage = (size_t)nacc * TILE_F * TILE_K * 2 + 2 * (size_t)L.nt * TILE_K * 2;
-    // a ring of about 100 KB keeps HBM busy (deeper rings measured no faster) and lets the CTA of the next
-    // kernel in the stream become resident beside this one, so that its weight prefetch overlaps this tail
-    static int ring_kb = -1;
-    if (ring_kb < 0) { const char *e = getenv("VIASD_TC_RING_KB"); ring_kb = e ? atoi(e) : 200; }
+    // The depth of the ring bounds the streaming rate (bytes in flight per SM): 200 KB, one CTA per SM, measured
+    // faster than 100 KB with the next kernel's CTA resident beside this one.
+    const int ring_kb = L.ring_kb > 0 ? L.ring_kb : 200;
     int stages = (int)((size_t)ring_kb * 1024 / stage);
     if (stages < 2) stages = 2;
     if (stages > MAX_STAGES) stages = MAX_STAGES;
@@ -608,16 +607,18 @@ int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {
     const CUtensorMap &w0 = *L.map_w[0], &w1 = *L.map_w[L.n_seg > 1 ? 1 : 0], &w2 = *L.map_w[L.n_seg > 2 ? 2 : 0];
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
-    // a second epilogue group above token tiles of 48 (VIASD_TC_EPI_GROUPS overrides)
-    static const int groups_env = getenv("VIASD_TC_EPI_GROUPS") ? atoi(getenv("VIASD_TC_EPI_GROUPS")) : 0;
-    const int groups = groups_env == 1 || groups_env == 2 ? groups_env : (p.nt > 48 ? 2 : 1);
+    // a second epilogue group above token tiles of 48 unless the caller says otherwise
+    const int groups = L.epi_groups == 1 || L.epi_groups == 2 ? L.epi_groups : (p.nt > 48 ? 2 : 1);
     pdl_config(cfg, attr, dim3(grid), dim3(64 + 128 * groups), smem, st);
-    static bool attr_done[8] = {false, false, false, false, false, false, false, false};
+    static bool attr_done[64][8];            // the attribute belongs to a (kernel, device) pair
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return VIASD_EUNSUPPORTED;
 #define TC_LAUNCH_G(IDX, KIND, G)                                                                                     \
     do {                                                                                                              \
-        if (!attr_done[IDX]) {                                                                                        \
+        if (!attr_done[dev][IDX]) {                                                                                   \
             CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<KIND, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, 208 * 1024)); \
-            attr_done[IDX] = true;                                                                                    \
+            attr_done[dev][IDX] = true;                                                                               \
         }                                                                                                             \
         CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<KIND, G>, w0, w1, w2, *L.map_x, p));                         \
     } while (0)

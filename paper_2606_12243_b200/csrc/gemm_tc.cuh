@@ -58,6 +58,7 @@ struct TcLaunch {                       // host-side description of one GEMM
     float *q_out; void *kc, *vc; const float *cosv, *sinv; const int *len_eff, *depth;
     int rope_M, rope_H, rope_Hkv, max_batch, max_ctx, layer_ord;
     int split_row, layer_ord2; float *out_f32_2; const float *next_gain2; void *kc2, *vc2;
+    int ring_kb, epi_groups;            // stream-K kernel: ring size and epilogue groups; 0 = defaults (200 KB; by token tile)
 };
 
 // 2-D bf16 tensor [rows, k] row-major -> TMA map with a (64 x box_rows) box and the 128-byte swizzle
@@ -67,5 +68,6 @@ uint32_t tc_box_rows(uint64_t tensor_rows, uint32_t want);
 size_t tc_scratch_floats(int sm_count, int nt, bool dual);
 int tc_tiles(int n);
 int launch_gemm_tc(const TcLaunch &L, cudaStream_t st);
+
 void tc_fill_params(const TcLaunch &L, TcParams &p);
 

@@ -479,7 +479,7 @@ int launch_accept(const viasd_model *m, const viasd_draft *d, const viasd_params
     a.seed = p->seed; a.step = p->step;
     // sampling over a large vocabulary: a cluster of CTAs per sequence shares every sweep of the vocabulary
     int team = (p->mode == 1 && m->cfg.vocab >= 16384) ? ACC_TEAM : 1;
-    if (const char *e = getenv("VIASD_ACCEPT_TEAM")) { const int t = atoi(e); if (t == 1 || t == 2 || t == 4 || t == 8) team = t; }
+    { const int t = m->opt.accept_team; if (t == 1 || t == 2 || t == 4 || t == 8) team = t; }
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(d->batch * team);

@@ -657,14 +657,17 @@ def test_argument_and_capacity_errors():
 # ---------------------------------------------------------------------------------------------
 # full size, in the launch configuration the benchmark times
 # ---------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("name", ["c2_7b", "c3_8b_tree_b1", "c3_8b_tree", "c4_13b"])
+@pytest.mark.parametrize("name", ["c2_7b", "c3_8b_tree_b1", "c3_8b_tree", "c4_13b", "c5_32b_b1_r16", "c5_32b_b16_r32"])
 def test_full_size_verify_step_matches_oracle(name):
     """Full-size workloads through viasd_verify_step, in the launch configuration the benchmark times, against the
     oracle evaluated in fp32 on the same generated weights: all logits of both verifiers, tiers, and every pinned
     decision.  c2_7b is the benchmarked workload (chain of 8, one sweep for both verifiers, mma.sync attention);
     c3_8b_tree_b1 has the 26-node tree, grouped heads, the 128k vocabulary and sampling (cluster accept walk; one sweep,
     keys-on-lanes attention with four items per kv head); c3_8b_tree is the same at batch 4 (108 rows: separate passes);
-    c4_13b has 8 sequences of 4096 tokens (separate passes, tcgen05 keys-on-lanes attention)."""
+    c4_13b has 8 sequences of 4096 tokens (separate passes, tcgen05 keys-on-lanes attention); the 32B-shaped model
+    (64 layers, d_ff 27648, vocabulary 152064, 40 query / 8 kv heads at 4096 tokens) runs at batch 1 with 16 layers
+    routed (6 rows, one sweep) and at batch 16 with 32 routed (96 rows per verifier: separate passes, token tiles of 96,
+    keys-on-lanes items of 30 rows).  Every logit of both verifiers is compared in all cases."""
     wl = W.get(name)
     vb = _vb()
     eng, st, si, model = _prepare(wl, dt=np.float32)
