@@ -74,6 +74,9 @@ typedef struct {
     int *len;                  /* [batch] committed length, shared by both caches */
     int *pending;              /* [batch] last emitted token */
     int *tokens;               /* [batch, max_ctx] committed token ids, or NULL */
+    int *len_full;             /* [batch] how far the full verifier's cache is complete (<= len), or NULL.  Only the
+                                  routed execution policy lets it fall behind len; viasd_kv_commit sets it to the new
+                                  len whenever the full verifier's pass ran in the step it commits. */
 } viasd_cache;
 
 typedef struct {
@@ -94,7 +97,15 @@ typedef struct {
     float log_acc_rel[3];              /* greedy gate per tier: accept if l[v] - max l >= this; 0 = argmax */
     int strict_break;                  /* 1: an accepted tier-1 token still ends the block (Alg. 2 as printed) */
     int emit_bonus;                    /* 1: when the whole path is accepted, add a token from q at the leaf */
-    int policy;                        /* 0: both passes always run (the only policy implemented) */
+    int policy;                        /* 0: both passes run in every step.  1: routed execution (viasd_verify_step only;
+                                          the point of the method, Sec. 1 and Eq. B.20): q' runs in every step, q only when
+                                          the walk reaches a tier-2 node before the first break or a bonus token is due.  A
+                                          skipped pass leaves q's cache short of the emitted tokens; the next pass of q
+                                          replays the last G = max_query - (n_nodes + 1) committed tokens in front of the
+                                          block, so a pass is skipped only while the backlog fits G, and every sequence
+                                          must hold at least G committed tokens.  Needs cache.tokens and cache.len_full, a
+                                          bf16 model with head_dim 128, and max_query > n_nodes + 1.  Emitted tokens are
+                                          those of policy 0; full_logits is left untouched by a step that skips q. */
     unsigned long long seed, step;     /* counter-based random numbers for sampling mode */
 } viasd_params;
 
@@ -116,6 +127,8 @@ typedef struct {
     unsigned long long accepted;       /* draft nodes accepted */
     int device_status;                 /* 0 or a VIASD_E* code recorded by a kernel */
     int need_slim, need_full;          /* last tier pass: any node in tier 1 / tier 2 */
+    int full_ran;                      /* 1 if the full verifier's pass of the last step ran (always, under policy 0) */
+    unsigned long long full_skipped;   /* committed steps whose full pass the routed execution policy skipped */
 } viasd_stats;
 
 /* Bytes of workspace viasd_init_model needs for this geometry. */
@@ -237,6 +250,17 @@ int viasd_kl_cost(const float *judge_logits, const float *proposal_logits, int r
  * allocates nothing.  Errors: EINVAL (null pointer, rows or vocab < 1, temperature <= 0, log_tau_lo > log_tau_hi), ECUDA. */
 int viasd_region_mass(const float *gate_logits, const float *proposal_logits, int rows, int vocab, float temperature,
                       float log_tau_hi, float log_tau_lo, float *mass, float *mean, void *stream);
+
+/* Self-test of the failure path (the paper has no counterpart).  Every wait inside the kernels of this library - on a
+ * TMA arrival, on a tensor-core commit, on another CTA's partial results - is bounded: when its limit expires the
+ * waiting kernel records VIASD_EDEVICE in a status word and returns by itself, so that the context stays usable and
+ * the next viasd_get_stats reports the failure.  Ordinary runs never take that path; this hook does, harmlessly: it
+ * launches one CTA that waits, through the same routine with a limit of limit_us microseconds (1..100000), on a
+ * barrier nothing arrives at.
+ * status: device, one int, written with VIASD_EDEVICE when the wait has expired.  waited_cycles: device, one 64-bit
+ * integer or NULL, written with the SM cycles the wait lasted (-1 if it did not expire).  Asynchronous on `stream`.
+ * Errors: EINVAL, ECUDA. */
+int viasd_selftest_wait_expiry(int *status, int limit_us, long long *waited_cycles, void *stream);
 
 /* Measurement hooks (the paper has no counterpart; they exist so that a benchmark can attribute time).
  * viasd_launch_count: kernels launched by this library in this process so far.

@@ -22,7 +22,7 @@ EXPORTS = ["viasd_workspace_bytes", "viasd_init_model", "viasd_full_forward", "v
            "viasd_tier_accept", "viasd_kv_commit", "viasd_verify_step", "viasd_get_stats",
            "viasd_free_model", "viasd_strerror", "viasd_last_cuda_error", "viasd_gemm_scratch_bytes",
            "viasd_gemm", "viasd_gemm_static", "viasd_kl_cost", "viasd_region_mass", "viasd_launch_count", "viasd_set_timing", "viasd_get_timing",
-           "viasd_set_option"]
+           "viasd_set_option", "viasd_selftest_wait_expiry"]
 
 OPTIONS = {"attention_kernel": 0, "attention_splits": 1, "attention_lo": 2, "accept_team": 3, "dual_max_rows": 4,
            "tk_grid": 5, "tk_flat": 6, "gemm_ring_kb": 7, "gemm_epi_groups": 8}
@@ -55,7 +55,8 @@ class Weights(C.Structure):
 
 
 class Cache(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in ("k_full", "v_full", "k_slim", "v_slim", "len", "pending", "tokens")]
+    _fields_ = [(n, C.c_void_p) for n in ("k_full", "v_full", "k_slim", "v_slim", "len", "pending", "tokens",
+                                          "len_full")]
 
 
 class Draft(C.Structure):
@@ -78,7 +79,7 @@ class Result(C.Structure):
 class Stats(C.Structure):
     _fields_ = [("steps", C.c_ulonglong), ("tier_count", C.c_ulonglong * 3), ("emitted", C.c_ulonglong),
                 ("accepted", C.c_ulonglong), ("device_status", C.c_int), ("need_slim", C.c_int),
-                ("need_full", C.c_int)]
+                ("need_full", C.c_int), ("full_ran", C.c_int), ("full_skipped", C.c_ulonglong)]
 
 
 class Timing(C.Structure):
@@ -124,6 +125,7 @@ def lib() -> C.CDLL:
         l.viasd_region_mass.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_float, C.c_float, C.c_float,
                                         C.c_void_p, C.c_void_p, C.c_void_p]
         l.viasd_set_option.argtypes = [C.c_void_p, C.c_int, C.c_int]
+        l.viasd_selftest_wait_expiry.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
         l.viasd_launch_count.restype = C.c_ulonglong
         l.viasd_set_timing.argtypes = [C.c_void_p, C.c_int]
         l.viasd_get_timing.argtypes = [C.c_void_p, C.POINTER(Timing), C.c_void_p]
@@ -193,9 +195,10 @@ def init_model(cfg: Config, embed: torch.Tensor, lm_head: torch.Tensor, final_no
     return Model(out.value, cfg, (embed, lm_head, final_norm, layers, workspace))
 
 
-def make_cache(k_full, v_full, k_slim, v_slim, length, pending, tokens=None) -> Cache:
-    c = Cache(_ptr(k_full), _ptr(v_full), _ptr(k_slim), _ptr(v_slim), _ptr(length), _ptr(pending), _ptr(tokens))
-    c._keep = (k_full, v_full, k_slim, v_slim, length, pending, tokens)
+def make_cache(k_full, v_full, k_slim, v_slim, length, pending, tokens=None, len_full=None) -> Cache:
+    c = Cache(_ptr(k_full), _ptr(v_full), _ptr(k_slim), _ptr(v_slim), _ptr(length), _ptr(pending), _ptr(tokens),
+              _ptr(len_full))
+    c._keep = (k_full, v_full, k_slim, v_slim, length, pending, tokens, len_full)
     return c
 
 
@@ -208,9 +211,9 @@ def make_draft(draft_tok, parent, prow, n_prows: int, drafter_logits) -> Draft:
 
 def make_params(log_tau_lo: float, log_tau_hi: float, mode: int = 0, temperature: float = 1.0, alpha: float = 0.0,
                 beta: float = 1.0, conf_source: int = 0, log_acc_rel=(0.0, 0.0, 0.0), strict_break: int = 0,
-                emit_bonus: int = 0, seed: int = 0, step: int = 0) -> Params:
+                emit_bonus: int = 0, seed: int = 0, step: int = 0, policy: int = 0) -> Params:
     return Params(log_tau_hi, log_tau_lo, conf_source, mode, temperature, alpha, beta,
-                  (C.c_float * 3)(*log_acc_rel), strict_break, emit_bonus, 0, seed, step)
+                  (C.c_float * 3)(*log_acc_rel), strict_break, emit_bonus, policy, seed, step)
 
 
 @dataclass
@@ -290,6 +293,14 @@ def set_option(m: Model, option: str, value) -> None:
     if option == "attention_kernel" and isinstance(value, str):
         value = ATTENTION_KERNELS[value]
     _check(lib().viasd_set_option(m.handle, OPTIONS[option], int(value)), "viasd_set_option")
+
+
+def selftest_wait_expiry(status: torch.Tensor, limit_us: int, waited_cycles: Optional[torch.Tensor] = None,
+                         stream=None) -> None:
+    """viasd_selftest_wait_expiry: status int32[1], waited_cycles int64[1] or None (device tensors)."""
+    assert status.dtype == torch.int32 and (waited_cycles is None or waited_cycles.dtype == torch.int64)
+    _check(lib().viasd_selftest_wait_expiry(_ptr(status), int(limit_us), _ptr(waited_cycles), _stream(stream)),
+           "viasd_selftest_wait_expiry")
 
 
 def launch_count() -> int:

@@ -64,6 +64,8 @@ size_t carve(const viasd_config &c, char *base, Workspace *ws) {
         if (qd + 2 * kvd > widest) widest = qd + 2 * kvd;
         if ((size_t)c.d_ff > widest) widest = c.d_ff;
         w.ssq = cv.take<float>((size_t)(c.d_model / 128 + 1) * 4 * R * 4);
+        w.a_head = cv.take<void>(R * c.d_model * 4);
+        w.ssq_head = cv.take<float>((size_t)(c.d_model / 128 + 1) * 4 * R * 4);
         w.attn_counters = cv.take<int>(attn_counter_count(c.max_batch, c.n_kv_heads) * sizeof(int));
         w.n_counters = widest / 128 + 8;
         w.gemm_counters = cv.take<int>(w.n_counters * 4);
@@ -176,10 +178,12 @@ int run_gemm(viasd_model *m, const GemmCall &g, int rows, cudaStream_t st) {
 // layers.  In mode 2 the block rows exist twice, [full stream; slim stream]: a routed layer's weights are streamed
 // once and applied to both streams, an unrouted layer runs on the full stream only.  Results are those of the two
 // separate passes; only the weight traffic of the routed layers is shared.
+// replay > 0 (mode 0 only, routed execution policy): every sequence's block is extended in front by its last `replay`
+// committed tokens (see prep_replay_kernel); the logits written are those of the block's own rows.
 int forward_sweep(viasd_model *m, const viasd_cache *cache, const viasd_draft *d, int mode, float *logits_full,
-                  float *logits_slim, cudaStream_t st) {
+                  float *logits_slim, cudaStream_t st, int replay = 0) {
     const viasd_config &c = m->cfg;
-    const int B = d->batch, M = d->n_nodes + 1, rows = B * M;
+    const int B = d->batch, M = d->n_nodes + 1 + replay, rows = B * M;
     const int qd = c.n_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
     const size_t R = m->ws.rows_alloc;
     const bool dual = mode == 2;
@@ -203,6 +207,7 @@ int forward_sweep(viasd_model *m, const viasd_cache *cache, const viasd_draft *d
                 L.scratch = m->ws.gemm_scratch; L.counters = m->ws.gemm_counters; L.status = &m->ws.stats->device_status;
                 L.sm_count = m->sm_count;
                 L.ring_kb = m->opt.ring_kb; L.epi_groups = m->opt.epi_groups;
+                L.run_flag = m->run_flag;
                 L.ssq_stride = (int)R; L.inv_d = 1.0f / (float)c.d_model; L.eps = c.rms_eps;
                 L.split_row = dual ? rows : 0;
                 int r2 = launch_gemm_tc(L, st);
@@ -214,7 +219,8 @@ int forward_sweep(viasd_model *m, const viasd_cache *cache, const viasd_draft *d
     auto wseg = [&](TcLaunch &L, int i, const WMap &w, int n) { L.map_w[i] = &w.map; L.seg_n[i] = n; L.w_box_rows[i] = w.box_rows; };
     const int ssq_n = (c.d_model / 128) * 4;
 
-    if ((rc = timed(m, VIASD_T_EMBED, st, [&] { return launch_prep(m, cache, d, st); }))) return rc;
+    if ((rc = timed(m, VIASD_T_EMBED, st, [&] { return replay ? launch_prep_replay(m, cache, d, replay, st)
+                                                              : launch_prep(m, cache, d, mode != 1, st); }))) return rc;
     if (dual) {
         if ((rc = timed(m, VIASD_T_EMBED, st, [&] { return launch_embed_norm2(m, m->norm1[0], m->norm1[m->routed[0]], rows, st); })))
             return rc;
@@ -239,6 +245,7 @@ int forward_sweep(viasd_model *m, const viasd_cache *cache, const viasd_draft *d
             L.len_eff = m->ws.len_eff; L.depth = m->ws.tree->depth; L.rope_M = M; L.rope_H = c.n_heads; L.rope_Hkv = c.n_kv_heads;
             L.max_batch = c.max_batch; L.max_ctx = c.max_ctx; L.layer_ord = ord;
             L.kc2 = cache->k_slim; L.vc2 = cache->v_slim; L.layer_ord2 = so;
+            L.kv_keep = replay ? cache->len_full : nullptr;
             if ((rc = gemm(L, m->maps_a, nrows))) return rc;
         }
         if (both) {
@@ -277,6 +284,12 @@ int forward_sweep(viasd_model *m, const viasd_cache *cache, const viasd_draft *d
     L.k = c.d_model; L.epi = EPI_STORE; L.out_f32 = mode == 1 ? logits_slim : logits_full; L.out_f32_2 = logits_slim;
     L.ld_out = c.vocab;
     L.ssq_in = m->ws.ssq; L.ssq_in_n = ssq_n;
+    if (replay) {
+        // the head runs on the block's own rows only, packed into a buffer of their own
+        if ((rc = timed(m, VIASD_T_EMBED, st, [&] { return launch_compact_head_rows(m, B, M - replay, replay, st); }))) return rc;
+        L.ssq_in = m->ws.ssq_head;
+        return gemm(L, m->maps_head, B * (M - replay));
+    }
     return gemm(L, m->maps_a, dual ? 2 * rows : rows);
 }
 
@@ -295,7 +308,7 @@ int forward(viasd_model *m, const viasd_cache *cache, const viasd_draft *d, bool
     const size_t R = m->ws.rows_alloc;
     const size_t pa = c.dtype ? R * c.d_model : 0, pq = c.dtype ? R * qd : 0, pf = c.dtype ? R * c.d_ff : 0;
 
-    if ((rc = timed(m, VIASD_T_EMBED, st, [&] { return launch_prep(m, cache, d, st); }))) return rc;
+    if ((rc = timed(m, VIASD_T_EMBED, st, [&] { return launch_prep(m, cache, d, !slim, st); }))) return rc;
     if ((rc = timed(m, VIASD_T_EMBED, st, [&] { return launch_embed(m, rows, st); }))) return rc;
     for (int ord = 0; ord < n_run; ++ord) {
         const int l = slim ? m->routed[ord] : ord;
@@ -331,7 +344,7 @@ int check_params(const viasd_params *p) {
     if (p->mode != 0 && p->mode != 1) return VIASD_EINVAL;
     if (p->mode == 1 && !(p->temperature > 0.f)) return VIASD_EINVAL;
     if (!(p->alpha >= 0.f && p->alpha < 1.f) || !(p->beta > 0.f)) return VIASD_EINVAL;
-    if (p->policy != 0) return VIASD_EINVAL;
+    if (p->policy != 0 && p->policy != 1) return VIASD_EINVAL;
     return VIASD_OK;
 }
 
@@ -432,9 +445,12 @@ int viasd_init_model(const viasd_config *cfg, const viasd_weights *w, const unsi
         if (!rc) rc = am(m->maps_a, m->ws.a, d);
         if (!rc) rc = am(m->maps_attn, m->ws.attn, qd);
         if (!rc) rc = am(m->maps_act, m->ws.act, ff);
+        if (!rc) rc = am(m->maps_head, m->ws.a_head, d);
         if (rc) { viasd_free_model(m); return rc; }
     }
+    m->run_flag = nullptr;
     cudaError_t e = cudaMemset(m->ws.stats, 0, sizeof(DeviceStats));
+    if (e == cudaSuccess) { const int one = 1; e = cudaMemcpy(&m->ws.stats->full_ran, &one, sizeof(int), cudaMemcpyHostToDevice); }
     if (e == cudaSuccess) e = cudaMemset(m->ws.gemm_counters, 0, m->ws.n_counters * 4);
     if (e == cudaSuccess) e = cudaMemset(m->ws.attn_counters, 0, attn_counter_count(cfg->max_batch, cfg->n_kv_heads) * sizeof(int));
     if (e == cudaSuccess) { rc = launch_rope_table(m, 0); if (rc == VIASD_OK) e = cudaDeviceSynchronize(); }
@@ -501,11 +517,47 @@ int viasd_kv_commit(viasd_model *m, viasd_cache *cache, const viasd_draft *draft
     return timed(m, VIASD_T_COMMIT, st, [&] { return launch_commit(m, cache, draft, result, st); });
 }
 
+// Routed execution policy (policy 1): the full verifier is invoked only when the walk needs it.
+//   tier -> slim pass -> probe (the accept walk on q' alone; raises the device flag when a tier-2 node is reached
+//   before the first break, a bonus token is due, or the backlog would outgrow the replay window) -> full pass, every
+//   kernel of which leaves at once when the flag is zero -> accept -> commit (len_full follows len only if q ran).
+// The full pass is a replay pass: the block is extended in front by the last G = max_query - M committed tokens, which
+// closes whatever gap skipped passes left in q's cache; q' keeps its cache current in every step.  No host decision,
+// no device-to-host traffic.  Results are those of policy 0 (the passes compute the same distributions).
+static int verify_step_routed(viasd_model *m, viasd_cache *cache, const viasd_draft *draft, const viasd_params *params,
+                              float *slim_logits, float *full_logits, viasd_result *result, void *stream) {
+    int rc;
+    if ((rc = check_draft(m, draft)) || (rc = check_cache(cache))) return rc;
+    if (!m->fused || !cache->len_full || !cache->tokens) return VIASD_EINVAL;
+    const int M = draft->n_nodes + 1, G = m->cfg.max_query - M;
+    if (G < 1) return VIASD_ECAPACITY;                        // no room for replayed rows: size max_query above M
+    cudaStream_t st = (cudaStream_t)stream;
+    int *flag = &m->ws.stats->full_ran;
+    if (params->conf_source == 0) {
+        if ((rc = viasd_tier_accept(m, draft, params, nullptr, nullptr, 1, result, stream))) return rc;
+        if ((rc = forward_sweep(m, cache, draft, 1, nullptr, slim_logits, st))) return rc;
+    } else {
+        if ((rc = forward_sweep(m, cache, draft, 1, nullptr, slim_logits, st))) return rc;
+        if ((rc = viasd_tier_accept(m, draft, params, slim_logits, nullptr, 1, result, stream))) return rc;
+    }
+    CUDA_TRY(cudaMemsetAsync(flag, 0, sizeof(int), st));
+    AcceptProbe probe{G, flag, cache->len, cache->len_full};
+    if ((rc = timed(m, VIASD_T_TIER_ACCEPT, st, [&] { return launch_accept(m, draft, params, slim_logits, nullptr, result,
+                                                                      true, st, &probe); }))) return rc;
+    m->run_flag = flag;
+    rc = forward_sweep(m, cache, draft, 0, full_logits, nullptr, st, G);
+    m->run_flag = nullptr;
+    if (rc) return rc;
+    if ((rc = tier_accept_impl(m, draft, params, slim_logits, full_logits, 2, result, false, stream))) return rc;
+    return viasd_kv_commit(m, cache, draft, result, stream);
+}
+
 int viasd_verify_step(viasd_model *m, viasd_cache *cache, const viasd_draft *draft, const viasd_params *params,
                       float *slim_logits, float *full_logits, viasd_result *result, void *stream) {
     int rc;
     if (!slim_logits || !full_logits) return VIASD_EINVAL;
     if ((rc = check_params(params))) return rc;
+    if (params->policy == 1) return verify_step_routed(m, cache, draft, params, slim_logits, full_logits, result, stream);
     // Both verifiers in one sweep over the layers (routed layers' weights are read once for both) while the two
     // row streams together fit one launch (128 token rows: an MMA of 256 columns with the hi/lo planes); beyond
     // that a sweep would stream every routed layer twice anyway, and the passes run one after the other.
@@ -539,6 +591,8 @@ int viasd_get_stats(viasd_model *m, viasd_stats *host_out, void *stream) {
     host_out->device_status = s.device_status;
     host_out->need_slim = s.need_slim;
     host_out->need_full = s.need_full;
+    host_out->full_ran = s.full_ran;
+    host_out->full_skipped = s.full_skipped;
     return VIASD_OK;
 }
 

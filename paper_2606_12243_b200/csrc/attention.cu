@@ -17,7 +17,9 @@ template <typename T, int HD>
 __global__ void __launch_bounds__(ATT_WARPS * 32)
 attention_split_kernel(float *__restrict__ part, const float *__restrict__ q, const T *__restrict__ kc,
                        const T *__restrict__ vc, const int *__restrict__ len_eff, const TreeInfo *__restrict__ tree,
-                       int M, int H, int Hkv, int max_batch, int max_ctx, int layer_ord, int nsplit, float scale) {
+                       int M, int H, int Hkv, int max_batch, int max_ctx, int layer_ord, int nsplit, float scale,
+                       const int *run_flag) {
+    RUN_FLAG_EXIT(run_flag);
     __shared__ float Qs[QG][HD];
     __shared__ float Ks[TK][HD + 1];
     __shared__ float Vs[TK][HD];
@@ -109,7 +111,8 @@ attention_split_kernel(float *__restrict__ part, const float *__restrict__ q, co
 
 template <typename T, int HD>
 __global__ void attention_combine_kernel(T *__restrict__ out, size_t plane, const float *__restrict__ part, int M, int H,
-                                         int nsplit) {
+                                         int nsplit, const int *run_flag) {
+    RUN_FLAG_EXIT(run_flag);
     const int r = blockIdx.x, h = blockIdx.y;        // r = b * M + i
     PDL_TRIGGER();
     const int b = r / M, i = r % M;
@@ -139,10 +142,10 @@ int run(const viasd_model *m, const void *kc, const void *vc, int layer_ord, int
     dim3 grid(batch * c.n_kv_heads, nsplit, qgroups);
     attention_split_kernel<T, HD><<<grid, ATT_WARPS * 32, 0, st>>>(m->ws.part, m->ws.q, (const T *)kc,
         (const T *)vc, m->ws.len_eff, m->ws.tree, M, c.n_heads, c.n_kv_heads, c.max_batch, c.max_ctx, layer_ord, nsplit,
-        1.0f / sqrtf((float)HD));
+        1.0f / sqrtf((float)HD), m->run_flag);
     LAUNCH_CHECK();
     attention_combine_kernel<T, HD><<<dim3(batch * M, c.n_heads), HD < 128 ? HD : 128, 0, st>>>((T *)m->ws.attn,
-        sizeof(T) == 2 ? m->ws.rows_alloc * (size_t)c.n_heads * HD : 0, m->ws.part, M, c.n_heads, nsplit);
+        sizeof(T) == 2 ? m->ws.rows_alloc * (size_t)c.n_heads * HD : 0, m->ws.part, M, c.n_heads, nsplit, m->run_flag);
     LAUNCH_CHECK();
     return VIASD_OK;
 }
@@ -238,7 +241,7 @@ static int mma_attention(viasd_model *m, const void *kc, const void *vc, bool sl
     else rc = launch_attention_mma(m, kc, vc, slim, layer_ord, kc2, vc2, layer_ord2, streams, batch, M, nsplit, fuse ? 1 : 0, st);
     if (rc || n_part == 1 || fuse) return rc;
     attention_combine_kernel<__nv_bfloat16, 128><<<dim3(streams * batch * M, c.n_heads), 128, 0, st>>>(
-        (__nv_bfloat16 *)m->ws.attn, m->ws.rows_alloc * (size_t)c.n_heads * 128, m->ws.part, M, c.n_heads, n_part);
+        (__nv_bfloat16 *)m->ws.attn, m->ws.rows_alloc * (size_t)c.n_heads * 128, m->ws.part, M, c.n_heads, n_part, m->run_flag);
     LAUNCH_CHECK();
     return VIASD_OK;
 }

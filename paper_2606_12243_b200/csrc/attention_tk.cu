@@ -44,6 +44,7 @@ struct AttnTkArgs {
     const int *len_eff;
     const TreeInfo *tree;
     int *status;
+    const int *run_flag;        // null, or a device flag: the kernel leaves at once when it is zero
     int M, H, Hkv, max_batch, max_ctx, layer_ord, nsplit;
     int batch, layer_ord2;      // second row stream: rows batch*M.., its own cache and layer ordinal
     int streams, n_items, items_per_cta, fuse_merge, nk, nv;   // nk, nv: ring slots for K tiles and for V tiles
@@ -208,6 +209,7 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     constexpr int NC = 2 * NR;                              // MMA N: hi rows then lo rows
     constexpr bool SPLIT = NR == 32;                        // K and V tiles in rings of their own (else a slot holds a tile's K and V)
     constexpr uint32_t QCH = (uint32_t)NC * 128u;           // one 64-wide chunk of an [NC rows] operand
+    RUN_FLAG_EXIT(a.run_flag);
     PDL_TRIGGER();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int NK = a.nk, NV = a.nv;
@@ -749,7 +751,7 @@ int launch_attention_tk(viasd_model *m, const void *kc, const void *vc, bool sli
 #endif
     a.q = m->ws.q; a.part = m->ws.part; a.out = (__nv_bfloat16 *)m->ws.attn;
     a.out_plane = m->ws.rows_alloc * (size_t)c.n_heads * HD;
-    a.len_eff = m->ws.len_eff; a.tree = m->ws.tree; a.status = &m->ws.stats->device_status;
+    a.len_eff = m->ws.len_eff; a.tree = m->ws.tree; a.status = &m->ws.stats->device_status; a.run_flag = m->run_flag;
     a.M = M; a.H = c.n_heads; a.Hkv = c.n_kv_heads; a.subs = subs; a.max_batch = c.max_batch; a.max_ctx = c.max_ctx;
     a.layer_ord = layer_ord; a.nsplit = nsplit; a.scale = 1.4426950408889634f / sqrtf((float)HD);   // log2(e) / sqrt(hd)
     a.batch = batch; a.layer_ord2 = layer_ord2; a.streams = streams;

@@ -33,6 +33,8 @@ struct DeviceStats {
     unsigned long long accepted;
     int device_status;
     int need_slim, need_full;
+    int full_ran;                       // the full verifier's pass of the current step ran (its cache holds the block's rows)
+    unsigned long long full_skipped;    // steps whose full pass the routed execution policy skipped
 };
 
 struct Workspace {                      // pointers into the caller's workspace block
@@ -59,6 +61,7 @@ struct Workspace {                      // pointers into the caller's workspace 
     size_t n_counters;
     int *attn_counters;                 // [attn_counter_count()] key-range arrivals per (stream, sequence, kv head, group of query heads)
     float *ssq;                         // [(d / 128) * 4][R] partial sums of h^2 for the fused RMSNorm
+    void *a_head; float *ssq_head;      // the block's own rows of `a` and `ssq`, compacted for the output head after a replay pass
 };
 
 struct WMap { CUtensorMap map; uint32_t box_rows; };        // TMA view of one weight matrix
@@ -111,6 +114,8 @@ struct viasd_model {
     WMap head_map;
     ActMaps maps_a, maps_attn, maps_act;
     CacheMaps cmaps_full, cmaps_slim;
+    ActMaps maps_head;                  // TMA views of the compacted head input (routed execution policy)
+    const int *run_flag;                // non-null while the launches of a conditional pass are being enqueued
 };
 
 // error helpers -------------------------------------------------------------------------------
@@ -146,6 +151,11 @@ inline void pdl_config(cudaLaunchConfig_t &cfg, cudaLaunchAttribute *attr, dim3 
     cfg.attrs = attr;
     cfg.numAttrs = g_use_pdl ? 1 : 0;
 }
+// A pass that runs only when a device flag says so (the full verifier's pass under the routed execution policy): every
+// kernel of it takes the flag's address and leaves at once when the flag is zero.  The flag is written by a kernel that
+// has completed before the pass's first kernel starts (the pass opens with ordinary, fully ordered launches), so
+// reading it ahead of the dependency wait is safe.
+#define RUN_FLAG_EXIT(ptr) do { if ((ptr) != nullptr && *reinterpret_cast<const volatile int *>(ptr) == 0) return; } while (0)
 #define PDL_WAIT() asm volatile("griddepcontrol.wait;" ::: "memory")
 #define PDL_TRIGGER() asm volatile("griddepcontrol.launch_dependents;" ::: "memory")
 
@@ -154,7 +164,9 @@ inline void pdl_config(cudaLaunchConfig_t &cfg, cudaLaunchAttribute *attr, dim3 
 // ---------------------------------------------------------------------------------------------
 // misc.cu
 int launch_rope_table(const viasd_model *m, cudaStream_t st);
-int launch_prep(const viasd_model *m, const viasd_cache *c, const viasd_draft *d, cudaStream_t st);
+int launch_prep(const viasd_model *m, const viasd_cache *c, const viasd_draft *d, bool full_pass, cudaStream_t st);
+int launch_prep_replay(const viasd_model *m, const viasd_cache *c, const viasd_draft *d, int G, cudaStream_t st);
+int launch_compact_head_rows(const viasd_model *m, int batch, int M, int G, cudaStream_t st);
 int launch_embed(const viasd_model *m, int rows, cudaStream_t st);
 int launch_embed_norm(const viasd_model *m, const float *gain, int rows, cudaStream_t st);
 int launch_rmsnorm(const viasd_model *m, const float *gain, int rows, cudaStream_t st);
@@ -194,8 +206,11 @@ int launch_embed_norm2(const viasd_model *m, const float *gain_full, const float
 // tier_accept.cu
 int launch_tier(const viasd_model *m, const viasd_draft *d, const viasd_params *p, const float *slim_logits,
                 viasd_result *r, cudaStream_t st);
+// probe != null: the walk on the slim verifier's logits alone, deciding whether the full verifier's pass is needed
+struct AcceptProbe { int replay_rows; int *need_full; const int *len, *len_full; };
 int launch_accept(const viasd_model *m, const viasd_draft *d, const viasd_params *p, const float *slim_logits,
-                  const float *full_logits, viasd_result *r, bool tree_ready, cudaStream_t st);
+                  const float *full_logits, viasd_result *r, bool tree_ready, cudaStream_t st,
+                  const AcceptProbe *probe = nullptr);
 
 // ---------------------------------------------------------------------------------------------
 // small device helpers

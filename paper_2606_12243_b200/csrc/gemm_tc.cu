@@ -41,6 +41,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
     __shared__ int4 rowmeta[128];                       // per token row: rotary position, cache slot, sequence
 
     constexpr bool DUAL = EPI == EPI_SWIGLU;
+    RUN_FLAG_EXIT(p.run_flag);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may start its prologue
     if (threadIdx.x == 0) TRACE(0);
@@ -439,7 +440,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                         const int row = p.row0 + et, stream = row >= p.split_row ? 1 : 0, rs = row - stream * p.split_row;
                         const int b = rs / p.rope_M, i = rs - b * p.rope_M;
                         const int n_ctx = p.len_eff[b];
-                        rowmeta[et] = make_int4(n_ctx + p.depth[i], n_ctx + i, b, stream);
+                        // replay pass: rows that fall on slots the cache already holds are recomputed but not stored
+                        const int slot = (p.kv_keep && n_ctx + i < p.kv_keep[b]) ? -1 : n_ctx + i;
+                        rowmeta[et] = make_int4(n_ctx + p.depth[i], slot, b, stream);
                     }
                 }
                 asm volatile("bar.sync 1, %0;" ::"n"(epi_threads) : "memory");
@@ -567,6 +570,8 @@ void tc_fill_params(const TcLaunch &L, TcParams &p) {
     p.split_row = L.split_row > 0 ? L.split_row : 0x7fffffff;
     p.out_f32_2 = L.out_f32_2; p.next_gain2 = L.next_gain2; p.kc2 = (__nv_bfloat16 *)L.kc2; p.vc2 = (__nv_bfloat16 *)L.vc2;
     p.layer_ord2 = L.layer_ord2;
+    p.run_flag = L.run_flag;
+    p.kv_keep = L.kv_keep;
 }
 
 int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {

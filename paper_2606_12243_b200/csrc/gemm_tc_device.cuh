@@ -183,8 +183,8 @@ __device__ __forceinline__ void finish_chunk(const TcParams &p, int tile, int f,
         } else {
 #pragma unroll
             for (int j = 0; j < CH; ++j) {
-                if (j < nrow) {
-                    const int4 rm = rowmeta[r0 + j];
+                const int4 rm = rowmeta[min(r0 + j, 127)];
+                if (j < nrow && rm.y >= 0) {
                     __nv_bfloat16 *cache = rm.w ? (s == 1 ? p.kc2 : p.vc2) : (s == 1 ? p.kc : p.vc);
                     const int lo = rm.w ? p.layer_ord2 : p.layer_ord;
                     cache[((((size_t)lo * p.max_batch + rm.z) * p.rope_Hkv + head) * p.max_ctx + rm.y) * TILE_F + f] =

@@ -30,10 +30,11 @@ int launch_rope_table(const viasd_model *m, cudaStream_t st) {
 // ---------------------------------------------------------------------------------------------
 __global__ void prep_kernel(TreeInfo *tree, int *len_eff, int *row_tok, DeviceStats *stats, const int *len,
                             const int *pending, const int *draft_tok, const int *parent, int B, int N,
-                            int max_ctx, int vocab) {
+                            int max_ctx, int vocab, int full_pass) {
     const int M = N + 1;
     PDL_TRIGGER();
     if (threadIdx.x == 0) {
+        if (full_pass) stats->full_ran = 1;                     // the full verifier's cache receives this block's rows
         int last_child[VIASD_MAX_ROWS_PER_SEQ];
         for (int i = 0; i < M; ++i) { tree->first_child[i] = -1; tree->next_sibling[i] = -1; last_child[i] = -1; }
         tree->anc[0] = 1ull;
@@ -65,9 +66,85 @@ __global__ void prep_kernel(TreeInfo *tree, int *len_eff, int *row_tok, DeviceSt
     }
 }
 
-int launch_prep(const viasd_model *m, const viasd_cache *c, const viasd_draft *d, cudaStream_t st) {
+int launch_prep(const viasd_model *m, const viasd_cache *c, const viasd_draft *d, bool full_pass, cudaStream_t st) {
     prep_kernel<<<1, 128, 0, st>>>(m->ws.tree, m->ws.len_eff, m->ws.row_tok, m->ws.stats, c->len, c->pending,
-                                   d->draft_tok, d->parent, d->batch, d->n_nodes, m->cfg.max_ctx, m->cfg.vocab);
+                                   d->draft_tok, d->parent, d->batch, d->n_nodes, m->cfg.max_ctx, m->cfg.vocab,
+                                   full_pass ? 1 : 0);
+    LAUNCH_CHECK();
+    return VIASD_OK;
+}
+
+// Preparation of a replay pass (routed execution policy): the block of every sequence is extended, in front, by its
+// last G committed tokens, so that the rows are
+//     row 0 .. G-1 : tokens[len - G .. len - 1]  (a chain; row 0 plays the pending token's part)
+//     row G        : the pending token
+//     row G+1+n    : draft node n (its parent moved along)
+// against a context of len - G rows.  The full verifier recomputes K/V of the G committed tokens (the same values
+// where its cache had them, the missing ones where a skipped pass left a gap) on its way to the block's own rows.
+__global__ void prep_replay_kernel(TreeInfo *tree, int *len_eff, int *row_tok, DeviceStats *stats, const int *len,
+                                   const int *pending, const int *draft_tok, const int *parent, const int *tokens,
+                                   int B, int N, int G, int max_ctx, int vocab, const int *run_flag) {
+    RUN_FLAG_EXIT(run_flag);
+    const int Mx = G + N + 1;
+    if (threadIdx.x == 0) {
+        stats->full_ran = 1;
+        tree->anc[0] = 1ull;
+        tree->depth[0] = 0;
+        for (int i = 0; i < Mx; ++i) { tree->first_child[i] = -1; tree->next_sibling[i] = -1; }
+        for (int e = 0; e < G + N; ++e) {                       // extended node e is row e + 1
+            int p = e < G ? e - 1 : parent[e - G];
+            if (e >= G) {
+                if (p < -1 || p >= e - G) { stats->device_status = VIASD_EDEVICE; p = -1; }
+                p = p < 0 ? G - 1 : G + p;
+            }
+            const int pr = p + 1, i = e + 1;
+            tree->anc[i] = tree->anc[pr] | (1ull << i);
+            tree->depth[i] = tree->depth[pr] + 1;
+        }
+        tree->is_chain = 0;
+    }
+    for (int b = threadIdx.x; b < B; b += blockDim.x) {
+        const int l = len[b] - G;
+        const int c = min(max(l, 0), max_ctx - Mx);
+        if (c != l) stats->device_status = VIASD_ECAPACITY;     // fewer than G committed tokens, or no room for the rows
+        len_eff[b] = c;
+    }
+    for (int r = threadIdx.x; r < B * Mx; r += blockDim.x) {
+        const int b = r / Mx, i = r % Mx;
+        const int base = max(len[b] - G, 0);
+        int t = i < G ? tokens[(size_t)b * max_ctx + min(base + i, max_ctx - 1)] : i == G ? pending[b] : draft_tok[b * N + i - G - 1];
+        if (t < 0 || t >= vocab) { stats->device_status = VIASD_EDEVICE; t = 0; }
+        row_tok[r] = t;
+    }
+}
+
+int launch_prep_replay(const viasd_model *m, const viasd_cache *c, const viasd_draft *d, int G, cudaStream_t st) {
+    prep_replay_kernel<<<1, 128, 0, st>>>(m->ws.tree, m->ws.len_eff, m->ws.row_tok, m->ws.stats, c->len, c->pending,
+                                          d->draft_tok, d->parent, c->tokens, d->batch, d->n_nodes, G, m->cfg.max_ctx,
+                                          m->cfg.vocab, m->run_flag);
+    LAUNCH_CHECK();
+    return VIASD_OK;
+}
+
+// The block's own rows (the last M of every sequence's G + M) of the head's input and of its row statistics, packed
+// for the output head: row b * (G + M) + G + i -> row b * M + i.  One CTA per row.
+__global__ void compact_head_rows_kernel(__nv_bfloat16 *dst, const __nv_bfloat16 *src, size_t plane, float *ssq_dst,
+                                         const float *ssq_src, int ssq_stride, int ssq_n, int d, int M, int G,
+                                         const int *run_flag) {
+    RUN_FLAG_EXIT(run_flag);
+    PDL_TRIGGER();
+    const int r = blockIdx.x, b = r / M, i = r % M, from = b * (G + M) + G + i;
+    const uint4 *s0 = reinterpret_cast<const uint4 *>(src + (size_t)from * d), *s1 = reinterpret_cast<const uint4 *>(src + plane + (size_t)from * d);
+    uint4 *d0 = reinterpret_cast<uint4 *>(dst + (size_t)r * d), *d1 = reinterpret_cast<uint4 *>(dst + plane + (size_t)r * d);
+    for (int c = threadIdx.x; c < d / 8; c += blockDim.x) { d0[c] = s0[c]; d1[c] = s1[c]; }
+    for (int e = threadIdx.x; e < ssq_n; e += blockDim.x) ssq_dst[(size_t)e * ssq_stride + r] = ssq_src[(size_t)e * ssq_stride + from];
+}
+
+int launch_compact_head_rows(const viasd_model *m, int batch, int M, int G, cudaStream_t st) {
+    const viasd_config &c = m->cfg;
+    compact_head_rows_kernel<<<batch * M, 128, 0, st>>>((__nv_bfloat16 *)m->ws.a_head, (const __nv_bfloat16 *)m->ws.a,
+        m->ws.rows_alloc * (size_t)c.d_model, m->ws.ssq_head, m->ws.ssq, (int)m->ws.rows_alloc, (c.d_model / 128) * 4,
+        c.d_model, M, G, m->run_flag);
     LAUNCH_CHECK();
     return VIASD_OK;
 }
@@ -114,7 +191,8 @@ __device__ __forceinline__ void embed_row(float *h, __nv_bfloat16 *a, size_t pla
 // h = E[tok]; a = hi/lo(h * gain); partial sums of h^2 per 32 features in the layout the GEMM epilogue reads.
 __global__ void __launch_bounds__(256)
 embed_norm_kernel(float *h, __nv_bfloat16 *a, size_t plane, float *ssq, int ssq_stride, const __nv_bfloat16 *E,
-                  const float *gain, const int *row_tok, int d) {
+                  const float *gain, const int *row_tok, int d, const int *run_flag) {
+    RUN_FLAG_EXIT(run_flag);
     const int r = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     PDL_TRIGGER();
     const __nv_bfloat16 *src = E + (size_t)row_tok[r] * d;
@@ -124,7 +202,7 @@ embed_norm_kernel(float *h, __nv_bfloat16 *a, size_t plane, float *ssq, int ssq_
 int launch_embed_norm(const viasd_model *m, const float *gain, int rows, cudaStream_t st) {
     embed_norm_kernel<<<rows, 256, 0, st>>>(m->ws.h, (__nv_bfloat16 *)m->ws.a, m->ws.rows_alloc * m->cfg.d_model, m->ws.ssq,
                                             (int)m->ws.rows_alloc, (const __nv_bfloat16 *)m->embed, gain, m->ws.row_tok,
-                                            m->cfg.d_model);
+                                            m->cfg.d_model, m->run_flag);
     LAUNCH_CHECK();
     return VIASD_OK;
 }
@@ -273,8 +351,9 @@ int launch_rope_append(const viasd_model *m, void *kc, void *vc, int layer_ord, 
 template <typename T>
 __global__ void commit_move_kernel(T *kf, T *vf, T *ks, T *vs, const int *len_eff, const int *n_acc,
                                    const int *path, int N, int L, int Ls, int Hkv, int hd, int max_batch,
-                                   int max_ctx) {
+                                   int max_ctx, const DeviceStats *stats) {
     int layer = blockIdx.x, b = blockIdx.y, g = blockIdx.z;
+    if (layer < L && !stats->full_ran) return;                  // the full verifier's cache did not receive this block
     T *kc = layer < L ? kf : ks;
     T *vc = layer < L ? vf : vs;
     int lo = layer < L ? layer : layer - L;
@@ -294,12 +373,16 @@ __global__ void commit_move_kernel(T *kf, T *vf, T *ks, T *vs, const int *len_ef
     }
 }
 
-__global__ void commit_advance_kernel(int *len, int *pending, int *tokens, const int *len_eff, const int *n_emit,
-                                      const int *out_tok, int B, int N, int max_ctx) {
+__global__ void commit_advance_kernel(int *len, int *len_full, int *pending, int *tokens, const int *len_eff,
+                                      const int *n_emit, const int *out_tok, int B, int N, int max_ctx,
+                                      DeviceStats *stats) {
     int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
     int n = len_eff[b];
     int ne = min(max(n_emit[b], 0), N + 1);
+    // the full verifier's cache is complete up to the new length exactly when its pass ran in this step
+    if (len_full && stats->full_ran) len_full[b] = n + ne;
+    if (b == 0 && !stats->full_ran) ++stats->full_skipped;
     if (ne == 0) return;
     if (tokens) {
         tokens[(size_t)b * max_ctx + n] = pending[b];
@@ -312,21 +395,22 @@ __global__ void commit_advance_kernel(int *len, int *pending, int *tokens, const
 int launch_commit(const viasd_model *m, viasd_cache *c, const viasd_draft *d, const viasd_result *r,
                   cudaStream_t st) {
     const viasd_config &cf = m->cfg;
-    int rc = launch_prep(m, c, d, st);
+    int rc = launch_prep(m, c, d, false, st);
     if (rc) return rc;
     dim3 grid(cf.n_layers + m->n_routed, d->batch, cf.n_kv_heads);
     int threads = cf.head_dim < 32 ? 32 : (cf.head_dim > 256 ? 256 : cf.head_dim);
     if (cf.dtype == 0)
         commit_move_kernel<float><<<grid, threads, 0, st>>>((float *)c->k_full, (float *)c->v_full, (float *)c->k_slim,
             (float *)c->v_slim, m->ws.len_eff, r->n_acc, r->path, d->n_nodes, cf.n_layers, m->n_routed, cf.n_kv_heads,
-            cf.head_dim, cf.max_batch, cf.max_ctx);
+            cf.head_dim, cf.max_batch, cf.max_ctx, m->ws.stats);
     else
         commit_move_kernel<__nv_bfloat16><<<grid, threads, 0, st>>>((__nv_bfloat16 *)c->k_full,
             (__nv_bfloat16 *)c->v_full, (__nv_bfloat16 *)c->k_slim, (__nv_bfloat16 *)c->v_slim, m->ws.len_eff, r->n_acc,
-            r->path, d->n_nodes, cf.n_layers, m->n_routed, cf.n_kv_heads, cf.head_dim, cf.max_batch, cf.max_ctx);
+            r->path, d->n_nodes, cf.n_layers, m->n_routed, cf.n_kv_heads, cf.head_dim, cf.max_batch, cf.max_ctx, m->ws.stats);
     LAUNCH_CHECK();
-    commit_advance_kernel<<<(d->batch + 63) / 64, 64, 0, st>>>(c->len, c->pending, c->tokens, m->ws.len_eff,
-                                                               r->n_emit, r->out_tok, d->batch, d->n_nodes, cf.max_ctx);
+    commit_advance_kernel<<<(d->batch + 63) / 64, 64, 0, st>>>(c->len, c->len_full, c->pending, c->tokens, m->ws.len_eff,
+                                                               r->n_emit, r->out_tok, d->batch, d->n_nodes, cf.max_ctx,
+                                                               m->ws.stats);
     LAUNCH_CHECK();
     return VIASD_OK;
 }

@@ -191,6 +191,13 @@ struct AcceptArgs {
     float inv_temp, log1m_alpha, inv_beta;
     float log_acc_rel[3];
     unsigned long long seed, step;
+    // Probe (routed execution policy): the same walk on the slim verifier's logits alone.  It stops where the full
+    // verifier's judgment (a tier-2 node, or the bonus token at a leaf) would be needed and raises *need_full; it also
+    // raises it when a sequence's backlog (len - len_full) plus this step's tokens would outgrow the replay window.
+    // Writes no result.
+    int probe, replay_rows;
+    int *need_full;
+    const int *len, *len_full;
 };
 
 // ---- the CTAs of a sequence (a thread-block cluster in sampling mode, else one CTA) ---------------------
@@ -283,13 +290,15 @@ accept_kernel(AcceptArgs a) {
     const float *st_mx = a.rs.mx + (size_t)b * 3 * RS_STRIDE, *st_z = a.rs.z + (size_t)b * 3 * RS_STRIDE;
     const int *st_arg = a.rs.arg + (size_t)b * 3 * RS_STRIDE;
     const unsigned long long k_acc = stream_key(a.seed, a.step, b, 0), k_gum = stream_key(a.seed, a.step, b, 1);
-    if (tm.rank == 0) for (int n = threadIdx.x; n < N; n += blockDim.x) a.judge[b * N + n] = 0;
+    if (tm.rank == 0 && !a.probe) for (int n = threadIdx.x; n < N; n += blockDim.x) a.judge[b * N + n] = 0;
     __syncthreads();
 
     int cur = 0, n_acc = 0, corr = -1, corr_src = 0;
+    bool needs_q = false;
     while (true) {
         int c = tree->first_child[cur];
         if (c < 0) {                                             // leaf: whole path accepted
+            if (a.emit_bonus && a.probe) { needs_q = true; break; }
             if (a.emit_bonus) {
                 if (sampling) {
                     softmax_numerators(P[2], a.full + ((size_t)b * M + cur) * V, V, a.inv_temp, st_mx[2 * RS_STRIDE + cur], tm);
@@ -314,9 +323,10 @@ accept_kernel(AcceptArgs a) {
             v = min(max(v, 0), V - 1);
             if (t == 0) {
                 taken = c; taken_tier = 0;
-                if (lead) a.judge[b * N + c] = 1;
+                if (lead && !a.probe) a.judge[b * N + c] = 1;
                 break;
             }
+            if (t == 2 && a.probe) { needs_q = true; break; }     // from here on the walk depends on q
             bool pass;
             if (!sampling) {
                 pass = (row[t][v] - mx[t]) >= a.log_acc_rel[t];
@@ -336,10 +346,10 @@ accept_kernel(AcceptArgs a) {
             }
             if (pass) {
                 taken = c; taken_tier = t;
-                if (lead) a.judge[b * N + c] = (unsigned char)(1 | (t << 4));
+                if (lead && !a.probe) a.judge[b * N + c] = (unsigned char)(1 | (t << 4));
                 break;
             }
-            if (lead) a.judge[b * N + c] = (unsigned char)(2 | (t << 4));
+            if (lead && !a.probe) a.judge[b * N + c] = (unsigned char)(2 | (t << 4));
             failed = max(failed, t);
             if (sampling) {
                 // Eq. A.3 round by round: the rejecting judge becomes its residual against the proposal (kept as is if
@@ -373,13 +383,14 @@ accept_kernel(AcceptArgs a) {
                 __syncthreads();
             }
         }
+        if (needs_q) break;
         if (taken >= 0) {
             if (a.strict_break && taken_tier == 1) {
                 corr = min(max(a.draft_tok[b * N + taken], 0), V - 1);
                 corr_src = 1;
                 break;
             }
-            if (lead) a.path[b * N + n_acc] = taken;
+            if (lead && !a.probe) a.path[b * N + n_acc] = taken;
             ++n_acc;
             cur = taken + 1;
             continue;
@@ -394,6 +405,16 @@ accept_kernel(AcceptArgs a) {
         break;
     }
     __syncthreads();
+    if (a.probe) {
+        if (lead) {
+            // tokens this step emits if q is not asked: the accepted nodes and the replacement (or nothing at a leaf)
+            const int ne = n_acc + (corr >= 0 ? 1 : 0);
+            const bool room = a.len[b] - a.len_full[b] + ne <= a.replay_rows && a.len[b] >= a.replay_rows;
+            if (needs_q || !room) atomicExch(a.need_full, 1);
+        }
+        if (tm.size > 1) team_barrier();
+        return;
+    }
     if (lead) {
         int ne = 0;
         for (int j = 0; j < n_acc; ++j) {
@@ -448,7 +469,7 @@ int launch_tier(const viasd_model *m, const viasd_draft *d, const viasd_params *
 }
 
 int launch_accept(const viasd_model *m, const viasd_draft *d, const viasd_params *p, const float *slim_logits,
-                  const float *full_logits, viasd_result *r, bool tree_ready, cudaStream_t st) {
+                  const float *full_logits, viasd_result *r, bool tree_ready, cudaStream_t st, const AcceptProbe *probe) {
     if (!tree_ready) {                       // a forward pass of the same call has laid the tree out already
         tree_only_kernel<<<1, 32, 0, st>>>(m->ws.tree, m->ws.stats, d->parent, d->n_nodes);
         LAUNCH_CHECK();
@@ -477,6 +498,11 @@ int launch_accept(const viasd_model *m, const viasd_draft *d, const viasd_params
     a.inv_beta = 1.0f / p->beta;
     for (int i = 0; i < 3; ++i) a.log_acc_rel[i] = p->log_acc_rel[i];
     a.seed = p->seed; a.step = p->step;
+    a.probe = probe ? 1 : 0;
+    a.replay_rows = probe ? probe->replay_rows : 0;
+    a.need_full = probe ? probe->need_full : nullptr;
+    a.len = probe ? probe->len : nullptr;
+    a.len_full = probe ? probe->len_full : nullptr;
     // sampling over a large vocabulary: a cluster of CTAs per sequence shares every sweep of the vocabulary
     int team = (p->mode == 1 && m->cfg.vocab >= 16384) ? ACC_TEAM : 1;
     { const int t = m->opt.accept_team; if (t == 1 || t == 2 || t == 4 || t == 8) team = t; }

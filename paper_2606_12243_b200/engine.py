@@ -75,8 +75,9 @@ class Engine:
         self.len = torch.zeros(wl.batch, dtype=torch.int32, device=device)
         self.pending = torch.zeros(wl.batch, dtype=torch.int32, device=device)
         self.tokens = torch.zeros((wl.batch, self.max_ctx), dtype=torch.int32, device=device)
+        self.len_full = torch.zeros(wl.batch, dtype=torch.int32, device=device)
         self.cache = vb.make_cache(self.k_full, self.v_full, self.k_slim, self.v_slim, self.len, self.pending,
-                                   self.tokens)
+                                   self.tokens, self.len_full)
         if fill_context == "device" and wl.ctx > 0:
             self.fill_random_context()
         elif fill_context and not wl.real_prefill and wl.ctx > 0:
@@ -93,6 +94,7 @@ class Engine:
                 kc[o, :, :, :wl.ctx] = to_device(W.context_kv(wl, cache_id, o, 0), self.device)
                 vc[o, :, :, :wl.ctx] = to_device(W.context_kv(wl, cache_id, o, 1), self.device)
         self.len.fill_(wl.ctx)
+        self.len_full.fill_(wl.ctx)
 
     def fill_random_context(self) -> None:
         """Committed context drawn on the device, N(0, kv_sigma) like the generator's: for timing only."""
@@ -103,6 +105,7 @@ class Engine:
             for o in range(t.shape[0]):
                 t[o, :, :, :self.wl.ctx].normal_(0.0, sigma, generator=g)
         self.len.fill_(self.wl.ctx)
+        self.len_full.fill_(self.wl.ctx)
 
     def prefill(self, prompt: np.ndarray) -> None:
         """Push a prompt [B, T] through both models with the library's own forward + commit calls."""

@@ -655,6 +655,98 @@ def test_argument_and_capacity_errors():
 
 
 # ---------------------------------------------------------------------------------------------
+# failure path: a bounded wait that runs out
+# ---------------------------------------------------------------------------------------------
+def test_expired_wait_is_reported_and_the_context_stays_usable():
+    """The bounded wait of the tcgen05 kernels on a barrier nothing arrives at: the kernel returns by itself after the
+    limit (1 ms here, 2 s in the kernels), the status word reads VIASD_EDEVICE, and the library keeps working."""
+    vb = _vb()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    waited = torch.zeros(1, dtype=torch.int64, device="cuda")
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    vb.selftest_wait_expiry(status, 1000, waited)
+    e1.record()
+    torch.cuda.synchronize()
+    assert int(status.item()) == vb.VIASD_EDEVICE
+    assert int(waited.item()) > 0
+    assert 0.5 <= e0.elapsed_time(e1) <= 50.0, e0.elapsed_time(e1)       # about the limit: neither at once nor the 2 s default
+    with pytest.raises(vb.ViasdError):
+        vb.selftest_wait_expiry(status, 0)
+    _check_verify_step("mini_7b")                                          # an ordinary step afterwards: status 0, parity
+
+
+# ---------------------------------------------------------------------------------------------
+# routed execution policy: the full verifier runs only when the walk needs it
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("name,replay", [("mini_7b", 18), ("mini_8b_tree_greedy", 12), ("mini_13b", 14)])
+def test_routed_policy_emits_what_running_both_passes_emits(name, replay):
+    """A decoding loop under policy 1 (q' in every step, q only when a tier-2 node is reached before the first break,
+    its cache caught up by replaying the last committed tokens) against the same loop under policy 0 and against the
+    oracle, with thresholds that leave most blocks to tiers 0 and 1: same tiers, same accepted paths, same emitted
+    tokens in every step; q's pass skipped in some steps and run in others; q''s cache identical, q's cache equal as
+    far as it is complete and complete again after a pass of q."""
+    wl = W.get(name)
+    vb = _vb()
+    n_steps, M = 12, wl.rows
+    model = W.Model(wl, keep=True)
+    st = PU.oracle_state(wl, np.float64, extra=n_steps * M)
+    engs = [_engine(wl, max_query=M + replay, extra_ctx=n_steps * M) for _ in range(2)]
+    # thresholds at the 5th / 50th percentile of the drafted tokens' log-confidence over the steps of this loop
+    inputs = [W.step_inputs(wl, i) for i in range(n_steps)]
+    d_all = np.concatenate([tiers.tier_rule(si.drafter_logits, si.draft_tok, si.prow, 0.0, 0.0)[1].ravel() for si in inputs])
+    lo, hi = tiers.quantile_thresholds(d_all, 0.05, 0.50)
+    st.pending[:] = inputs[0].pending
+    for e in engs:
+        e.set_inputs(inputs[0])
+    bufs = [(e.logits_buffer(), e.logits_buffer(), vb.alloc_result(wl.batch, wl.n_nodes)) for e in engs]
+    ran, max_err = [], 0.0
+    for i, si in enumerate(inputs):
+        want = step.verify_step(model, wl.shape, wl.routed, st, si.draft_tok, wl.parent, si.prow, si.drafter_logits,
+                                float(lo), float(hi), PU.oracle_params(wl, i))
+        for pol, (e, (sl, fl, res)) in enumerate(zip(engs, bufs)):
+            e.set_inputs(si, set_pending=False)
+            vb.verify_step(e.model, e.cache, e.draft, e.params(step=i, log_tau_lo=float(lo), log_tau_hi=float(hi), policy=pol),
+                           sl, fl, res)
+        torch.cuda.synchronize()
+        stats = vb.get_stats(engs[1].model)
+        assert stats.device_status == 0 and vb.get_stats(engs[0].model).device_status == 0
+        ran.append(stats.full_ran)
+        (sl0, fl0, r0), (sl1, fl1, r1) = bufs
+        assert np.array_equal(r0.tier.cpu().numpy(), want.tier) and torch.equal(r0.tier, r1.tier)
+        assert torch.equal(sl0, sl1), "the slim verifier's pass does not depend on the policy"
+        for a, b in ((r0.n_acc, r1.n_acc), (r0.n_emit, r1.n_emit), (r0.corr_src, r1.corr_src)):
+            assert torch.equal(a, b), (i, a, b)
+        for b in range(wl.batch):
+            ne = int(r0.n_emit[b])
+            assert r0.out_tok[b, :ne].tolist() == r1.out_tok[b, :ne].tolist(), (i, b)
+            assert r0.path[b, :int(r0.n_acc[b])].tolist() == r1.path[b, :int(r1.n_acc[b])].tolist()
+        e1, _ = PU.assert_logits_close(sl1.cpu().numpy(), want.slim_logits, wl.shape.dtype, "slim")
+        if stats.full_ran:
+            e2, _ = PU.assert_logits_close(fl1.cpu().numpy(), want.full_logits, wl.shape.dtype, "full (replay pass)")
+            max_err = max(max_err, e2)
+        # the oracle's emitted tokens, wherever its decisions are pinned
+        PU.compare_resolution(want.seqs, r1.n_acc.cpu().numpy(), r1.path.cpu().numpy(), r1.out_tok.cpu().numpy(),
+                              r1.n_emit.cpu().numpy(), r1.corr_src.cpu().numpy(), eps_row=max(e1, max_err, 1e-3))
+        assert torch.equal(engs[0].len, engs[1].len) and torch.equal(engs[0].pending, engs[1].pending)
+        assert bool((engs[1].len_full <= engs[1].len).all())
+        if stats.full_ran:
+            assert torch.equal(engs[1].len_full, engs[1].len)
+    assert 0 < sum(ran) < n_steps, f"q ran in steps {ran}: the loop must cover both a skipped and an executed pass"
+    assert vb.get_stats(engs[1].model).full_skipped == n_steps - sum(ran)
+    assert vb.get_stats(engs[0].model).full_skipped == 0
+    # caches: q' identical; q equal up to where policy 1 has it complete (values recomputed by a replay pass may differ
+    # in the last bf16 bit from the ones a sequential pass stored)
+    assert torch.equal(engs[0].k_slim, engs[1].k_slim) and torch.equal(engs[0].v_slim, engs[1].v_slim)
+    for b in range(wl.batch):
+        n = int(engs[1].len_full[b])
+        for c0, c1 in ((engs[0].k_full, engs[1].k_full), (engs[0].v_full, engs[1].v_full)):
+            a, bb = c0[:, b, :, :n].float(), c1[:, b, :, :n].float()
+            assert float((a - bb).abs().max()) <= 2.0 ** -7 * max(1.0, float(a.abs().max()))
+    print(f"{name}: full verifier ran in {sum(ran)} of {n_steps} steps")
+
+
+# ---------------------------------------------------------------------------------------------
 # full size, in the launch configuration the benchmark times
 # ---------------------------------------------------------------------------------------------
 @pytest.mark.parametrize("name", ["c2_7b", "c3_8b_tree_b1", "c3_8b_tree", "c4_13b", "c5_32b_b1_r16", "c5_32b_b16_r32"])
