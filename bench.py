@@ -266,14 +266,14 @@ class Bench:
     """One workload resident in HBM and the five calls of the path, each timed with CUDA events on the stream
     the library launches on."""
 
-    def __init__(self, wl, rank: int = 0, gate: str = "drafter", weights_from=None, fill_context=True):
+    def __init__(self, wl, rank: int = 0, gate: str = "drafter", weights_from=None, fill_context=True, **engine_kw):
         import torch
         from synth import workloads as W
         from paper_2606_12243_b200 import binding as vb
         from paper_2606_12243_b200.engine import Engine
         self.torch, self.vb, self.wl = torch, vb, wl
         self.eng = Engine(wl, weights_from=weights_from.eng if weights_from is not None else None,
-                          fill_context=fill_context)
+                          fill_context=fill_context, **engine_kw)
         self.eng.set_inputs(W.step_inputs(wl, step=rank))      # every rank: its own seed-shifted inputs, same shapes
         self.sl, self.fl = self.eng.logits_buffer(), self.eng.logits_buffer()
         self.res = vb.alloc_result(wl.batch, wl.n_nodes)
@@ -359,6 +359,52 @@ def per_call(b: Bench, n: int, peak: float, tf_peak: float) -> dict:
     return out
 
 
+def run_routed_policy(weights_from: Bench, n_steps: int = 48, replay: int = 18) -> dict:
+    """Decoding loops of n_steps verify steps on the 7B-shaped workload with thresholds at the 5th / 50th percentile
+    of drafter confidence (most drafted tokens in tiers 0 and 1), once with both passes in every step (policy 0) and
+    once with routed execution (policy 1: the full verifier only when the walk needs it, up to `replay` committed
+    tokens replayed when it does).  Eight input sets, resident on the device, are used in turn; the cache grows as
+    tokens are committed.  Reports ms per step of each loop and the share of steps in which the full verifier ran."""
+    import torch
+    from synth import workloads as W
+    from paper_2606_12243_b200 import binding as vb
+    wl = W.get("c2_7b_routed")
+    out = {"config": config_of(wl, replay_rows=replay, steps=n_steps)}
+    for policy in (0, 1):
+        b = Bench(wl, weights_from=weights_from, fill_context="device", max_query=wl.rows + replay,
+                  extra_ctx=(n_steps + 4) * wl.rows)
+        e = b.eng
+        sets = []
+        for k in range(8):
+            e.set_inputs(W.step_inputs(wl, step=k), set_pending=(k == 0))
+            sets.append(e.draft)
+        torch.cuda.synchronize()
+
+        def loop(n, first):
+            for i in range(n):
+                vb.verify_step(e.model, e.cache, sets[(first + i) % 8], e.params(step=first + i, policy=policy), b.sl, b.fl, b.res)
+
+        loop(4, 0)                                              # warm-up steps, committed like the rest
+        torch.cuda.synchronize()
+        s0 = vb.get_stats(e.model)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(b.stream)
+        loop(n_steps, 4)
+        ev1.record(b.stream)
+        torch.cuda.synchronize()
+        s1 = vb.get_stats(e.model)
+        skipped = int(s1.full_skipped - s0.full_skipped)
+        out[f"policy_{policy}"] = {"ms_per_step": ev0.elapsed_time(ev1) / n_steps,
+                                   "full_pass_share": (n_steps - skipped) / n_steps,
+                                   "tokens_emitted_per_step": float(s1.emitted - s0.emitted) / n_steps,
+                                   "tier_share": [float(s1.tier_count[i] - s0.tier_count[i]) /
+                                                  max(1.0, float(sum(s1.tier_count) - sum(s0.tier_count))) for i in range(3)],
+                                   "device_status_ok": s1.device_status == 0}
+        del b, e, sets
+    out["speedup_of_policy_1"] = out["policy_0"]["ms_per_step"] / out["policy_1"]["ms_per_step"]
+    return out
+
+
 def run_sweep(main: Bench, peak: float, tf_peak: float, n: int) -> dict:
     """The other benchmark configurations, one after the other (weights of a model shape are uploaded once and
     shared by its workloads; committed context drawn on the device): step, full pass and slim pass each."""
@@ -391,6 +437,8 @@ def run_sweep(main: Bench, peak: float, tf_peak: float, n: int) -> dict:
         rec["verified_tokens_per_s"] = wl.batch * wl.n_nodes / (rec["verify_step"]["ms_median"] * 1e-3)
         rec["device_status_ok"] = b.status_ok()
         out[name] = rec
+        if name == "c2_7b":
+            out["routed_policy_7b"] = run_routed_policy(b)
         if share is None:
             holder = b
         del b

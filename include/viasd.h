@@ -86,6 +86,12 @@ typedef struct {
     const int *prow;                   /* [N] drafter-logit row the node was drafted from */
     int n_prows;                       /* R, 1..64 (one drafter row per distinct parent at most) */
     const float *drafter_logits;       /* [B, R, vocab] */
+    int per_sequence;                  /* 0: one tree for the whole batch (parent and prow are [N]).  1: every sequence
+                                          brings its own tree, which may change from call to call (dynamic drafts):
+                                          parent and prow are [B, N]; a sequence that uses fewer than N nodes marks the
+                                          others with parent -2 (they are nobody's children; their rows are computed and
+                                          ignored).  Sequences are independent, so the result of each is the result of
+                                          a batch-of-one call with its tree. */
 } viasd_draft;
 
 typedef struct {

@@ -61,7 +61,7 @@ class Cache(C.Structure):
 
 class Draft(C.Structure):
     _fields_ = [("batch", C.c_int), ("n_nodes", C.c_int), ("draft_tok", C.c_void_p), ("parent", C.c_void_p),
-                ("prow", C.c_void_p), ("n_prows", C.c_int), ("drafter_logits", C.c_void_p)]
+                ("prow", C.c_void_p), ("n_prows", C.c_int), ("drafter_logits", C.c_void_p), ("per_sequence", C.c_int)]
 
 
 class Params(C.Structure):
@@ -203,8 +203,11 @@ def make_cache(k_full, v_full, k_slim, v_slim, length, pending, tokens=None, len
 
 
 def make_draft(draft_tok, parent, prow, n_prows: int, drafter_logits) -> Draft:
+    """parent / prow of shape [N] (one tree for the batch) or [B, N] (a tree per sequence)."""
     B, N = draft_tok.shape
-    d = Draft(B, N, _ptr(draft_tok), _ptr(parent), _ptr(prow), n_prows, _ptr(drafter_logits))
+    per_seq = int(parent.dim() == 2)
+    assert tuple(parent.shape) == ((B, N) if per_seq else (N,)) and tuple(prow.shape) == tuple(parent.shape)
+    d = Draft(B, N, _ptr(draft_tok), _ptr(parent), _ptr(prow), n_prows, _ptr(drafter_logits), per_seq)
     d._keep = (draft_tok, parent, prow, drafter_logits)
     return d
 

@@ -54,7 +54,7 @@ size_t carve(const viasd_config &c, char *base, Workspace *ws) {
     w.part = cv.take<float>(w.part_bytes);
     w.len_eff = cv.take<int>((size_t)c.max_batch * 4);
     w.row_tok = cv.take<int>(R * 4);
-    w.tree = cv.take<TreeInfo>(sizeof(TreeInfo));
+    w.tree = cv.take<TreeInfo>(sizeof(TreeInfo) * (size_t)c.max_batch);
     w.stats = cv.take<DeviceStats>(sizeof(DeviceStats));
     w.accept_scratch = cv.take<float>(((size_t)c.max_batch * 3 * c.vocab + (size_t)c.max_batch * 9 * VIASD_MAX_ROWS_PER_SEQ) * 4);
     {
@@ -242,7 +242,7 @@ int forward_sweep(viasd_model *m, const viasd_cache *cache, const viasd_draft *d
             L.k = c.d_model; L.epi = EPI_QKV_ROPE; L.ld_out = qd + 2 * kvd;
             L.ssq_in = m->ws.ssq; L.ssq_in_n = ssq_n;
             L.q_out = m->ws.q; L.kc = kc; L.vc = vc; L.cosv = m->ws.rope_cos; L.sinv = m->ws.rope_sin;
-            L.len_eff = m->ws.len_eff; L.depth = m->ws.tree->depth; L.rope_M = M; L.rope_H = c.n_heads; L.rope_Hkv = c.n_kv_heads;
+            L.len_eff = m->ws.len_eff; L.depth = m->ws.tree->depth; L.tree_stride = (int)(sizeof(TreeInfo) / sizeof(int)); L.rope_M = M; L.rope_H = c.n_heads; L.rope_Hkv = c.n_kv_heads;
             L.max_batch = c.max_batch; L.max_ctx = c.max_ctx; L.layer_ord = ord;
             L.kc2 = cache->k_slim; L.vc2 = cache->v_slim; L.layer_ord2 = so;
             L.kv_keep = replay ? cache->len_full : nullptr;

@@ -55,7 +55,7 @@ attention_split_kernel(float *__restrict__ part, const float *__restrict__ q, co
     for (int r = 0; r < 2; ++r) {
         int qidx = qg * QG + warp * 2 + r;
         qrow[r] = qidx < QR ? qidx : -1;
-        anc[r] = qidx < QR ? tree->anc[qidx % M] : 0ull;
+        anc[r] = qidx < QR ? tree[b].anc[qidx % M] : 0ull;
     }
     const size_t cbase = (((size_t)layer_ord * max_batch + b) * Hkv + g) * (size_t)max_ctx * HD;
 

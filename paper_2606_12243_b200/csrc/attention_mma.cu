@@ -309,7 +309,7 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
         const int row = (warp & (a.mt_eff - 1)) * 16 + (lane >> 2) + r * 8;
-        anc_first[r] = row < (a.H / a.Hkv) * a.M ? a.tree->anc[row % a.M] : 0ull;
+        anc_first[r] = row < (a.H / a.Hkv) * a.M ? a.tree[first_item.b].anc[row % a.M] : 0ull;
     }
     ATRACE(1);
     PDL_WAIT();
@@ -365,7 +365,7 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
             const int row = mtile * 16 + (lane >> 2) + r * 8;
-            anc[r] = !(active && row < QR) ? 0ull : item == i0 ? anc_first[r] : a.tree->anc[row % a.M];
+            anc[r] = !(active && row < QR) ? 0ull : item == i0 ? anc_first[r] : a.tree[it.b].anc[row % a.M];
         }
 #pragma unroll
         for (int n = 0; n < 16; ++n)

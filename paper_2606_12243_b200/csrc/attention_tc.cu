@@ -367,7 +367,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 if (item == i0) ATC_MARK(2);
             }
             const int h = it.g * grp + row / a.M, node = row % a.M;
-            const unsigned long long anc = live ? a.tree->anc[node] : 0ull;
+            const unsigned long long anc = live ? a.tree[it.b].anc[node] : 0ull;
             float m_run = -INFINITY, l_run = 0.f;
 
             for (int t = 0; t < it.n_tiles; ++t, ++s_cnt) {

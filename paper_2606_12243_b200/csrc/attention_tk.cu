@@ -404,6 +404,7 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 #endif
         ATK_MARK(0);
         int s_cnt = 0, q_be = -1, q_g = -1, wg_phase = 0;        // s_cnt: tiles this CTA has finished (buffer phase)
+        int anc_b = -1;                                          // sequence whose ancestor sets anc_sh holds
         bool ok = true;
         auto wg_sync = [&]() -> bool {
             mbar_arrive(wg_bar);
@@ -432,8 +433,13 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 #ifdef VIASD_TC_TRACE
                 if (ATK_ON) for (int z = 3; z < 12; ++z) g_atk_trace[blockIdx.x * 16 + z] = 0;
 #endif
-                if (et < a.M) anc_sh[et] = a.tree->anc[et];
+            }
+            if (!dry && it.b != anc_b) {
+                // the ancestor sets of this sequence's draft tree (every sequence may have its own)
+                if (n_item > 0 && !(ok = wg_sync())) break;           // nobody reads the previous sequence's sets any more
+                if (et < a.M) anc_sh[et] = a.tree[it.b].anc[et];
                 if (!(ok = wg_sync())) break;                         // anc_sh is visible
+                anc_b = it.b;
             }
             if (dry || it.be != q_be || it.g != q_g) {
                 // stage the query rows of this (sequence, kv head): rows 0..NR-1 the hi parts, NR..2NR-1 the lo parts,

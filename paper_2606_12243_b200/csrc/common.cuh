@@ -18,7 +18,7 @@ inline size_t attn_counter_count(int max_batch, int n_kv_heads) {
 // ---------------------------------------------------------------------------------------------
 // device-side records kept in the workspace
 // ---------------------------------------------------------------------------------------------
-struct TreeInfo {                       // rebuilt from `parent` at the start of every pass
+struct TreeInfo {                       // one per sequence, rebuilt from `parent` at the start of every pass
     unsigned long long anc[VIASD_MAX_ROWS_PER_SEQ];   // bit r set: row r is on the root path of row i
     int depth[VIASD_MAX_ROWS_PER_SEQ];
     int first_child[VIASD_MAX_ROWS_PER_SEQ];          // per row: first child node or -1
@@ -53,7 +53,7 @@ struct Workspace {                      // pointers into the caller's workspace 
     size_t part_bytes;
     int *len_eff;                       // [B] committed length clamped to the cache capacity
     int *row_tok;                       // [R] token id per row
-    TreeInfo *tree;
+    TreeInfo *tree;                     // [max_batch]: every sequence has its own draft tree (copies when the call shares one)
     DeviceStats *stats;
     float *accept_scratch;              // [B, 3, V] sampling-mode distributions, then [3][B, 3, 64] row statistics
     float *gemm_scratch;                // partial tiles of split GEMM work (tcgen05 kernel)
@@ -117,6 +117,33 @@ struct viasd_model {
     ActMaps maps_head;                  // TMA views of the compacted head input (routed execution policy)
     const int *run_flag;                // non-null while the launches of a conditional pass are being enqueued
 };
+
+#ifdef __CUDACC__
+// Lays out one sequence's draft tree: ancestor sets, depths, child lists.  parent[n] = -1: child of the pending token;
+// -2: the node is unused (a sequence with fewer nodes than the call's N): it is nobody's child and nothing attends to it.
+__device__ inline void build_tree(TreeInfo *tree, const int *parent, int N, DeviceStats *stats) {
+    const int M = N + 1;
+    int last_child[VIASD_MAX_ROWS_PER_SEQ];
+    for (int i = 0; i < M; ++i) { tree->first_child[i] = -1; tree->next_sibling[i] = -1; last_child[i] = -1; }
+    tree->anc[0] = 1ull;
+    tree->depth[0] = 0;
+    int chain = 1;
+    for (int n = 0; n < N; ++n) {
+        int p = parent[n];
+        const int i = n + 1;
+        if (p == -2) { tree->anc[i] = 1ull << i; tree->depth[i] = 0; chain = 0; continue; }
+        if (p < -1 || p >= n) { stats->device_status = VIASD_EDEVICE; p = -1; }
+        if (p != n - 1) chain = 0;
+        const int pr = p + 1;
+        tree->anc[i] = tree->anc[pr] | (1ull << i);
+        tree->depth[i] = tree->depth[pr] + 1;
+        if (last_child[pr] < 0) tree->first_child[pr] = n; else tree->next_sibling[last_child[pr]] = n;
+        last_child[pr] = n;
+    }
+    tree->is_chain = chain;
+}
+
+#endif
 
 // error helpers -------------------------------------------------------------------------------
 extern int g_last_cuda_error;

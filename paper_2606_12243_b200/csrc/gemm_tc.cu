@@ -442,7 +442,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                         const int n_ctx = p.len_eff[b];
                         // replay pass: rows that fall on slots the cache already holds are recomputed but not stored
                         const int slot = (p.kv_keep && n_ctx + i < p.kv_keep[b]) ? -1 : n_ctx + i;
-                        rowmeta[et] = make_int4(n_ctx + p.depth[i], slot, b, stream);
+                        rowmeta[et] = make_int4(n_ctx + p.depth[(size_t)b * p.tree_stride + i], slot, b, stream);
                     }
                 }
                 asm volatile("bar.sync 1, %0;" ::"n"(epi_threads) : "memory");
@@ -566,7 +566,7 @@ void tc_fill_params(const TcLaunch &L, TcParams &p) {
     p.next_gain = L.next_gain; p.next_act = (__nv_bfloat16 *)L.next_act; p.next_plane = L.next_plane; p.ssq_out = L.ssq_out;
     p.q_out = L.q_out; p.kc = (__nv_bfloat16 *)L.kc; p.vc = (__nv_bfloat16 *)L.vc; p.cosv = L.cosv; p.sinv = L.sinv;
     p.len_eff = L.len_eff; p.depth = L.depth; p.rope_M = L.rope_M; p.rope_H = L.rope_H; p.rope_Hkv = L.rope_Hkv;
-    p.max_batch = L.max_batch; p.max_ctx = L.max_ctx; p.layer_ord = L.layer_ord;
+    p.max_batch = L.max_batch; p.max_ctx = L.max_ctx; p.layer_ord = L.layer_ord; p.tree_stride = L.tree_stride;
     p.split_row = L.split_row > 0 ? L.split_row : 0x7fffffff;
     p.out_f32_2 = L.out_f32_2; p.next_gain2 = L.next_gain2; p.kc2 = (__nv_bfloat16 *)L.kc2; p.vc2 = (__nv_bfloat16 *)L.vc2;
     p.layer_ord2 = L.layer_ord2;

@@ -29,6 +29,7 @@ struct TcParams {                       // kernel argument block
     // EPI_QKV_ROPE
     float *q_out; __nv_bfloat16 *kc, *vc; const float *cosv, *sinv; const int *len_eff, *depth;
     int rope_M, rope_H, rope_Hkv, max_batch, max_ctx, layer_ord;
+    int tree_stride;                    // ints between the depth tables of consecutive sequences
     // two row streams in one launch (full verifier rows first, slim verifier rows from split_row on)
     int split_row, layer_ord2; float *out_f32_2; const float *next_gain2; __nv_bfloat16 *kc2, *vc2;
     const int *run_flag;                // null, or a device flag: the kernel leaves at once when it is zero
@@ -58,7 +59,7 @@ struct TcLaunch {                       // host-side description of one GEMM
     const float *next_gain; void * next_act; size_t next_plane; float *ssq_out;
     // EPI_QKV_ROPE
     float *q_out; void *kc, *vc; const float *cosv, *sinv; const int *len_eff, *depth;
-    int rope_M, rope_H, rope_Hkv, max_batch, max_ctx, layer_ord;
+    int rope_M, rope_H, rope_Hkv, max_batch, max_ctx, layer_ord, tree_stride;
     int split_row, layer_ord2; float *out_f32_2; const float *next_gain2; void *kc2, *vc2;
     const int *run_flag, *kv_keep;
     int ring_kb, epi_groups;            // stream-K kernel: ring size and epilogue groups; 0 = defaults (200 KB; by token tile)

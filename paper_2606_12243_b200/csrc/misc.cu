@@ -28,31 +28,15 @@ int launch_rope_table(const viasd_model *m, cudaStream_t st) {
 // ---------------------------------------------------------------------------------------------
 // per-pass preparation
 // ---------------------------------------------------------------------------------------------
+// parent: [N] shared by the batch, or [B, N] when per_seq
 __global__ void prep_kernel(TreeInfo *tree, int *len_eff, int *row_tok, DeviceStats *stats, const int *len,
-                            const int *pending, const int *draft_tok, const int *parent, int B, int N,
+                            const int *pending, const int *draft_tok, const int *parent, int per_seq, int B, int N,
                             int max_ctx, int vocab, int full_pass) {
     const int M = N + 1;
     PDL_TRIGGER();
-    if (threadIdx.x == 0) {
-        if (full_pass) stats->full_ran = 1;                     // the full verifier's cache receives this block's rows
-        int last_child[VIASD_MAX_ROWS_PER_SEQ];
-        for (int i = 0; i < M; ++i) { tree->first_child[i] = -1; tree->next_sibling[i] = -1; last_child[i] = -1; }
-        tree->anc[0] = 1ull;
-        tree->depth[0] = 0;
-        int chain = 1;
-        for (int n = 0; n < N; ++n) {
-            int p = parent[n];
-            if (p < -1 || p >= n) { stats->device_status = VIASD_EDEVICE; p = -1; }
-            if (p != n - 1) chain = 0;
-            int pr = p + 1, i = n + 1;
-            tree->anc[i] = tree->anc[pr] | (1ull << i);
-            tree->depth[i] = tree->depth[pr] + 1;
-            if (last_child[pr] < 0) tree->first_child[pr] = n; else tree->next_sibling[last_child[pr]] = n;
-            last_child[pr] = n;
-        }
-        tree->is_chain = chain;
-    }
+    if (threadIdx.x == 0 && full_pass) stats->full_ran = 1;     // the full verifier's cache receives this block's rows
     for (int b = threadIdx.x; b < B; b += blockDim.x) {
+        build_tree(tree + b, parent + (per_seq ? (size_t)b * N : 0), N, stats);
         int l = len[b];
         int c = min(max(l, 0), max_ctx - M);
         if (c != l) stats->device_status = VIASD_ECAPACITY;
@@ -68,8 +52,8 @@ __global__ void prep_kernel(TreeInfo *tree, int *len_eff, int *row_tok, DeviceSt
 
 int launch_prep(const viasd_model *m, const viasd_cache *c, const viasd_draft *d, bool full_pass, cudaStream_t st) {
     prep_kernel<<<1, 128, 0, st>>>(m->ws.tree, m->ws.len_eff, m->ws.row_tok, m->ws.stats, c->len, c->pending,
-                                   d->draft_tok, d->parent, d->batch, d->n_nodes, m->cfg.max_ctx, m->cfg.vocab,
-                                   full_pass ? 1 : 0);
+                                   d->draft_tok, d->parent, d->per_sequence, d->batch, d->n_nodes, m->cfg.max_ctx,
+                                   m->cfg.vocab, full_pass ? 1 : 0);
     LAUNCH_CHECK();
     return VIASD_OK;
 }
@@ -82,28 +66,30 @@ int launch_prep(const viasd_model *m, const viasd_cache *c, const viasd_draft *d
 // against a context of len - G rows.  The full verifier recomputes K/V of the G committed tokens (the same values
 // where its cache had them, the missing ones where a skipped pass left a gap) on its way to the block's own rows.
 __global__ void prep_replay_kernel(TreeInfo *tree, int *len_eff, int *row_tok, DeviceStats *stats, const int *len,
-                                   const int *pending, const int *draft_tok, const int *parent, const int *tokens,
-                                   int B, int N, int G, int max_ctx, int vocab, const int *run_flag) {
+                                   const int *pending, const int *draft_tok, const int *parent, int per_seq,
+                                   const int *tokens, int B, int N, int G, int max_ctx, int vocab, const int *run_flag) {
     RUN_FLAG_EXIT(run_flag);
     const int Mx = G + N + 1;
-    if (threadIdx.x == 0) {
-        stats->full_ran = 1;
-        tree->anc[0] = 1ull;
-        tree->depth[0] = 0;
-        for (int i = 0; i < Mx; ++i) { tree->first_child[i] = -1; tree->next_sibling[i] = -1; }
+    if (threadIdx.x == 0) stats->full_ran = 1;
+    for (int b = threadIdx.x; b < B; b += blockDim.x) {
+        TreeInfo *t = tree + b;
+        const int *par = parent + (per_seq ? (size_t)b * N : 0);
+        t->anc[0] = 1ull;
+        t->depth[0] = 0;
+        for (int i = 0; i < Mx; ++i) { t->first_child[i] = -1; t->next_sibling[i] = -1; }
         for (int e = 0; e < G + N; ++e) {                       // extended node e is row e + 1
-            int p = e < G ? e - 1 : parent[e - G];
+            int p = e < G ? e - 1 : par[e - G];
+            const int i = e + 1;
             if (e >= G) {
+                if (p == -2) { t->anc[i] = 1ull << i; t->depth[i] = 0; continue; }
                 if (p < -1 || p >= e - G) { stats->device_status = VIASD_EDEVICE; p = -1; }
                 p = p < 0 ? G - 1 : G + p;
             }
-            const int pr = p + 1, i = e + 1;
-            tree->anc[i] = tree->anc[pr] | (1ull << i);
-            tree->depth[i] = tree->depth[pr] + 1;
+            const int pr = p + 1;
+            t->anc[i] = t->anc[pr] | (1ull << i);
+            t->depth[i] = t->depth[pr] + 1;
         }
-        tree->is_chain = 0;
-    }
-    for (int b = threadIdx.x; b < B; b += blockDim.x) {
+        t->is_chain = 0;
         const int l = len[b] - G;
         const int c = min(max(l, 0), max_ctx - Mx);
         if (c != l) stats->device_status = VIASD_ECAPACITY;     // fewer than G committed tokens, or no room for the rows
@@ -120,8 +106,8 @@ __global__ void prep_replay_kernel(TreeInfo *tree, int *len_eff, int *row_tok, D
 
 int launch_prep_replay(const viasd_model *m, const viasd_cache *c, const viasd_draft *d, int G, cudaStream_t st) {
     prep_replay_kernel<<<1, 128, 0, st>>>(m->ws.tree, m->ws.len_eff, m->ws.row_tok, m->ws.stats, c->len, c->pending,
-                                          d->draft_tok, d->parent, c->tokens, d->batch, d->n_nodes, G, m->cfg.max_ctx,
-                                          m->cfg.vocab, m->run_flag);
+                                          d->draft_tok, d->parent, d->per_sequence, c->tokens, d->batch, d->n_nodes, G,
+                                          m->cfg.max_ctx, m->cfg.vocab, m->run_flag);
     LAUNCH_CHECK();
     return VIASD_OK;
 }
@@ -303,7 +289,7 @@ __global__ void rope_append_kernel(float *q_out, T *kc, T *vc, const float *qkv,
     int b = r / M, i = r % M;
     int half = hd >> 1;
     int n = len_eff[b];
-    int pos = n + tree->depth[i], slot = n + i;
+    int pos = n + tree[b].depth[i], slot = n + i;
     const float *src = qkv + (size_t)r * (H + 2 * Hkv) * hd + (size_t)head * hd;
     for (int p = threadIdx.x; p < half; p += blockDim.x) {
         float x1 = src[p], x2 = src[p + half];

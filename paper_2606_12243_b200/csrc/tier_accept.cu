@@ -88,10 +88,11 @@ __device__ float block_max(float x, float *sh) {
 __global__ void __launch_bounds__(256)
 tier_kernel(unsigned char *__restrict__ tier, float *__restrict__ conf, DeviceStats *stats,
             const float *__restrict__ gate_logits, const int *__restrict__ draft_tok, const int *__restrict__ prow,
-            const int *__restrict__ parent, int conf_source, int rows_per_seq, int N, int V, float log_tau_lo,
+            const int *__restrict__ parent, int per_seq, int conf_source, int rows_per_seq, int N, int V, float log_tau_lo,
             float log_tau_hi) {
     __shared__ float sh[32];
     const int gr = blockIdx.x, b = blockIdx.y;
+    if (per_seq) { prow += (size_t)b * N; parent += (size_t)b * N; }     // every sequence has its own tree
     const float *row = gate_logits + ((size_t)b * rows_per_seq + gr) * V;
     float mx = -INFINITY;
     if ((V & 3) == 0 && ((uintptr_t)row & 15) == 0) {
@@ -105,6 +106,10 @@ tier_kernel(unsigned char *__restrict__ tier, float *__restrict__ conf, DeviceSt
     }
     mx = block_max(mx, sh);
     for (int n = threadIdx.x; n < N; n += blockDim.x) {
+        if (parent[n] == -2) {                                   // unused node of this sequence's tree
+            if (gr == 0) { tier[b * N + n] = 0; conf[b * N + n] = 0.f; }
+            continue;
+        }
         int g = conf_source == 0 ? prow[n] : parent[n] + 1;
         if (g != gr) continue;
         int t = draft_tok[b * N + n];
@@ -195,6 +200,7 @@ struct AcceptArgs {
     // verifier's judgment (a tier-2 node, or the bonus token at a leaf) would be needed and raises *need_full; it also
     // raises it when a sequence's backlog (len - len_full) plus this step's tokens would outgrow the replay window.
     // Writes no result.
+    int per_seq;                             // prow is [B, N] and every sequence has its own tree
     int probe, replay_rows;
     int *need_full;
     const int *len, *len_full;
@@ -283,7 +289,8 @@ accept_kernel(AcceptArgs a) {
     tm.slot_f = slot_f; tm.slot_m = slot_m; tm.phase = 0;
     const bool lead = tm.rank == 0 && threadIdx.x == 0;       // the one thread that writes the results
     const int b = blockIdx.x / tm.size, N = a.N, M = N + 1, V = a.V;
-    const TreeInfo *tree = a.tree;
+    const TreeInfo *tree = a.tree + b;
+    const int *prow = a.prow + (a.per_seq ? (size_t)b * N : 0);
     const bool sampling = a.mode == 1;
     float *P[3] = {a.scratch + ((size_t)b * 3 + 0) * V, a.scratch + ((size_t)b * 3 + 1) * V,
                    a.scratch + ((size_t)b * 3 + 2) * V};
@@ -332,7 +339,7 @@ accept_kernel(AcceptArgs a) {
                 pass = (row[t][v] - mx[t]) >= a.log_acc_rel[t];
             } else {
                 if (!row[0]) {
-                    const int pr = a.prow[c];
+                    const int pr = prow[c];
                     row[0] = a.drafter + ((size_t)b * a.R + pr) * V;
                     mx[0] = st_mx[pr];
                     Z[0] = st_z[pr];
@@ -432,25 +439,8 @@ accept_kernel(AcceptArgs a) {
 }
 
 // the accept kernel needs the tree layout but no cache: build it here when called on its own
-__global__ void tree_only_kernel(TreeInfo *tree, DeviceStats *stats, const int *parent, int N) {
-    if (threadIdx.x != 0) return;
-    const int M = N + 1;
-    int last_child[VIASD_MAX_ROWS_PER_SEQ];
-    for (int i = 0; i < M; ++i) { tree->first_child[i] = -1; tree->next_sibling[i] = -1; last_child[i] = -1; }
-    tree->anc[0] = 1ull;
-    tree->depth[0] = 0;
-    int chain = 1;
-    for (int n = 0; n < N; ++n) {
-        int p = parent[n];
-        if (p < -1 || p >= n) { stats->device_status = VIASD_EDEVICE; p = -1; }
-        if (p != n - 1) chain = 0;
-        int pr = p + 1, i = n + 1;
-        tree->anc[i] = tree->anc[pr] | (1ull << i);
-        tree->depth[i] = tree->depth[pr] + 1;
-        if (last_child[pr] < 0) tree->first_child[pr] = n; else tree->next_sibling[last_child[pr]] = n;
-        last_child[pr] = n;
-    }
-    tree->is_chain = chain;
+__global__ void tree_only_kernel(TreeInfo *tree, DeviceStats *stats, const int *parent, int per_seq, int B, int N) {
+    for (int b = threadIdx.x; b < B; b += blockDim.x) build_tree(tree + b, parent + (per_seq ? (size_t)b * N : 0), N, stats);
 }
 
 }  // namespace
@@ -463,7 +453,7 @@ int launch_tier(const viasd_model *m, const viasd_draft *d, const viasd_params *
     const int rows = p->conf_source == 0 ? d->n_prows : M;
     if (!gate) return VIASD_EINVAL;
     tier_kernel<<<dim3(rows, d->batch), 256, 0, st>>>(r->tier, r->conf, m->ws.stats, gate, d->draft_tok, d->prow,
-        d->parent, p->conf_source, rows, d->n_nodes, m->cfg.vocab, p->log_tau_lo, p->log_tau_hi);
+        d->parent, d->per_sequence, p->conf_source, rows, d->n_nodes, m->cfg.vocab, p->log_tau_lo, p->log_tau_hi);
     LAUNCH_CHECK();
     return VIASD_OK;
 }
@@ -471,7 +461,7 @@ int launch_tier(const viasd_model *m, const viasd_draft *d, const viasd_params *
 int launch_accept(const viasd_model *m, const viasd_draft *d, const viasd_params *p, const float *slim_logits,
                   const float *full_logits, viasd_result *r, bool tree_ready, cudaStream_t st, const AcceptProbe *probe) {
     if (!tree_ready) {                       // a forward pass of the same call has laid the tree out already
-        tree_only_kernel<<<1, 32, 0, st>>>(m->ws.tree, m->ws.stats, d->parent, d->n_nodes);
+        tree_only_kernel<<<1, 64, 0, st>>>(m->ws.tree, m->ws.stats, d->parent, d->per_sequence, d->batch, d->n_nodes);
         LAUNCH_CHECK();
     }
     if (d->n_prows > RS_STRIDE) return VIASD_EINVAL;
@@ -498,6 +488,7 @@ int launch_accept(const viasd_model *m, const viasd_draft *d, const viasd_params
     a.inv_beta = 1.0f / p->beta;
     for (int i = 0; i < 3; ++i) a.log_acc_rel[i] = p->log_acc_rel[i];
     a.seed = p->seed; a.step = p->step;
+    a.per_seq = d->per_sequence;
     a.probe = probe ? 1 : 0;
     a.replay_rows = probe ? probe->replay_rows : 0;
     a.need_full = probe ? probe->need_full : nullptr;

@@ -145,8 +145,12 @@ def _wl() -> Dict[str, Workload]:
         for ls in (16, 32, 48):
             w[f"c5_32b_b{b}_r{ls}"] = Workload(f"c5_32b_b{b}_r{ls}", s32b, b, 4096, chain(5), ls,
                                                seed=5000)
+    # the 7B workload with thresholds that leave most drafted tokens to tiers 0 and 1 (quantiles 0.05 / 0.50): the case the
+    # routed execution policy is for; 18 committed tokens can be replayed (max_query 27)
+    w["c2_7b_routed"] = replace(w["c2_7b"], name="c2_7b_routed", quantiles=(0.05, 0.50))
     # profiling-sized cut of the 7B workload: same layer shapes, 2 layers (about 1.3 GB on the device)
     w["c2_7b_l2"] = Workload("c2_7b_l2", replace(s7b, n_layers=2), 1, 1024, chain(8), 1, seed=2000)
+    w["c3_8b_tree_b1_l2"] = Workload("c3_8b_tree_b1_l2", replace(s8b, n_layers=2), 1, 2048, tree26(), 1, mode="sampling", seed=3000)
     w["c4_13b_l2"] = Workload("c4_13b_l2", replace(s13b, n_layers=2), 8, 4096, chain(6), 1, quantiles=(0.30, 0.70), seed=4000)
     # shrunken siblings: same head_dim, same query/KV-head ratio, same draft shape
     m7 = ModelShape(4, 512, 4, 4, 128, 1408, 2048)

@@ -655,6 +655,89 @@ def test_argument_and_capacity_errors():
 
 
 # ---------------------------------------------------------------------------------------------
+# a draft tree per sequence (dynamic drafts)
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("name", ["mini_8b_tree_greedy", "mini_8b_tree"])
+def test_verify_step_with_a_tree_per_sequence(name):
+    """per_sequence = 1: the four sequences of the batch bring four different trees - the 26-node tree, a chain of 26,
+    a star (26 children of the pending token) and a 7-node tree with the other 19 nodes unused - and each must come out
+    as the oracle's batch-of-one step with its tree: logits of both verifiers, tiers, decisions, committed state."""
+    base = W.get(name)
+    assert base.batch == 4 and base.n_nodes == 26
+    trees = [W.tree26(), W.chain(26), tuple([-1] * 26), W.small_tree() + (-2,) * 19]
+    vb = _vb()
+    N, B, V = 26, 4, base.shape.vocab
+    si = W.step_inputs(base)
+    prows = [W.drafter_rows([p for p in t if p != -2]) for t in trees]
+    R = max(r for _, r in prows)
+    prow = np.zeros((B, N), dtype=np.int32)
+    for b, (pr, _) in enumerate(prows):
+        prow[b, :len(pr)] = pr
+    tok = si.draft_tok.copy()
+    for b, t in enumerate(trees):                     # siblings carry distinct ids
+        seen = {}
+        for n, p in enumerate(t):
+            if p == -2:
+                continue
+            sset = seen.setdefault(p, set())
+            while int(tok[b, n]) in sset:
+                tok[b, n] = (tok[b, n] + 1) % V
+            sset.add(int(tok[b, n]))
+    dl = synth.normal_f32(base.seed, 777, (B, R, V), base.logit_sigma)
+    for b, t in enumerate(trees):
+        for n, p in enumerate(t):
+            if p != -2:
+                dl[b, prow[b, n], tok[b, n]] += np.float32(base.plant)
+    lo, hi = W.thresholds(base)
+    eng = _engine(base)
+    eng.pending.copy_(torch.from_numpy(si.pending.astype(np.int32)))
+    parent_dev = torch.from_numpy(np.array(trees, dtype=np.int32)).cuda()
+    keep = (torch.from_numpy(tok.astype(np.int32)).cuda(), parent_dev, torch.from_numpy(prow).cuda(), torch.from_numpy(dl).cuda())
+    draft = vb.make_draft(keep[0], keep[1], keep[2], R, keep[3])
+    sl, fl = eng.logits_buffer(), eng.logits_buffer()
+    res = vb.alloc_result(B, N)
+    len0 = eng.len.clone()
+    vb.verify_step(eng.model, eng.cache, draft, eng.params(), sl, fl, res)
+    torch.cuda.synchronize()
+    assert vb.get_stats(eng.model).device_status == 0
+    model = W.Model(base, keep=True)
+    pinned_all = total_all = full_all = 0
+    for b, t in enumerate(trees):
+        live = [n for n, p in enumerate(t) if p != -2]
+        tb = tuple(t[n] for n in live)                                   # unused nodes come last: indices stay
+        one = replace(base, batch=1, parent=tb)
+        st = step.new_state(one.shape, one.n_routed, 1, one.ctx + N + 1, np.float64, base_len=one.ctx,
+                            base_full=lambda o, w, b=b: W.context_kv(base, 0, o, w)[b:b + 1],
+                            base_slim=lambda o, w, b=b: W.context_kv(base, 1, o, w)[b:b + 1])
+        st.pending[:] = si.pending[b]
+        P = replace(PU.oracle_params(base), seed=base.seed)
+        # the oracle numbers sequences from 0: give it this sequence's random-number stream
+        want = _oracle_step_for_sequence(model, one, st, tok[b:b + 1, live], prow[b, live], dl[b:b + 1], lo, hi, P, b)
+        rows = [0] + [n + 1 for n in live]
+        e1, _ = PU.assert_logits_close(sl[b, rows].cpu().numpy(), want.slim_logits[0], base.shape.dtype, f"slim seq {b}")
+        e2, _ = PU.assert_logits_close(fl[b, rows].cpu().numpy(), want.full_logits[0], base.shape.dtype, f"full seq {b}")
+        assert np.array_equal(res.tier[b, live].cpu().numpy(), want.tier[0])
+        p_, t_, f_ = PU.compare_resolution(want.seqs, res.n_acc[b:b + 1].cpu().numpy(), res.path[b:b + 1].cpu().numpy(),
+                                           res.out_tok[b:b + 1].cpu().numpy(), res.n_emit[b:b + 1].cpu().numpy(),
+                                           res.corr_src[b:b + 1].cpu().numpy(), eps_row=max(e1, e2))
+        pinned_all += p_; total_all += t_; full_all += f_
+        if f_ == 1:
+            assert int(eng.len[b]) == int(len0[b]) + len(want.seqs[0].out_tok)
+            assert int(eng.pending[b]) == want.seqs[0].out_tok[-1]
+    PU.assert_pinned(f"{name} with a tree per sequence", pinned_all, total_all, full_all, B, 0.7, 2)
+
+
+def _oracle_step_for_sequence(model, one, st, tok, prow, dl, lo, hi, P, b):
+    """The oracle's step for one sequence of a batch: resolve_sequence draws its random numbers by sequence number."""
+    rows = step.block_rows(st.pending, tok)
+    slim = decoder.forward(model, one.shape, one.routed, st.slim, st.lens, rows, one.parent)
+    tier, conf = tiers.tier_rule(dl, tok, prow, lo, hi)
+    full = decoder.forward(model, one.shape, range(one.shape.n_layers), st.full, st.lens, rows, one.parent)
+    seq = tiers.resolve_sequence(b, tok[0], one.parent, prow, tier[0], dl[0], slim[0], full[0], P)
+    return step.StepOut(tier, conf, slim, full, [seq])
+
+
+# ---------------------------------------------------------------------------------------------
 # failure path: a bounded wait that runs out
 # ---------------------------------------------------------------------------------------------
 def test_expired_wait_is_reported_and_the_context_stays_usable():
