@@ -210,6 +210,11 @@ int viasd_last_cuda_error(void);
 size_t viasd_gemm_scratch_bytes(int rows, int n, int k);
 int viasd_gemm(const void *x, const void *w, float *y, int rows, int n, int k, int dtype, void *scratch,
                size_t scratch_bytes, void *stream);
+/* The calls above are asynchronous, so a device-side failure (a bounded wait of the kernel that expired) cannot come
+ * back as their return value: it is recorded in a status word inside the scratch.  This reads it: *host_out =
+ * VIASD_OK or VIASD_EDEVICE for the last viasd_gemm call that used `scratch` with this n (bf16 only; the fp32 kernel
+ * has no waits).  Synchronises `stream`. */
+int viasd_gemm_status(const void *scratch, int n, int *host_out, void *stream);
 
 /* Same product as viasd_gemm for bf16 operands (y[rows, n] = x[rows, k] * W[n, k]^T, fp32 y) for callers that
  * cannot allocate device memory and therefore have no scratch to hand over: a serving process that gave all
@@ -227,6 +232,9 @@ int viasd_gemm(const void *x, const void *w, float *y, int rows, int n, int k, i
  * streams, or different host threads) race on it and give wrong results; serialise them.
  * Errors: EINVAL (null / misaligned pointer, k not a multiple of 8), ECAPACITY, ECUDA, EUNSUPPORTED. */
 int viasd_gemm_static(const void *x, const void *w, float *y, int rows, int n, int k, void *stream);
+/* Status of the last viasd_gemm_static call on the current device: *host_out = VIASD_OK, or VIASD_EDEVICE when a
+ * bounded wait of its kernel expired (y is then incomplete).  Synchronises `stream`; allocates nothing. */
+int viasd_gemm_static_status(int *host_out, void *stream);
 
 /* KL-style verification cost of a judge distribution against a proposal, per row (Eq. 11), and its sum over the
  * rows given (block cost, Eq. 10).  With q = softmax(judge_logits / temperature), p = softmax(proposal_logits /

@@ -22,7 +22,7 @@ EXPORTS = ["viasd_workspace_bytes", "viasd_init_model", "viasd_full_forward", "v
            "viasd_tier_accept", "viasd_kv_commit", "viasd_verify_step", "viasd_get_stats",
            "viasd_free_model", "viasd_strerror", "viasd_last_cuda_error", "viasd_gemm_scratch_bytes",
            "viasd_gemm", "viasd_gemm_static", "viasd_kl_cost", "viasd_region_mass", "viasd_launch_count", "viasd_set_timing", "viasd_get_timing",
-           "viasd_set_option", "viasd_selftest_wait_expiry"]
+           "viasd_set_option", "viasd_selftest_wait_expiry", "viasd_gemm_status", "viasd_gemm_static_status"]
 
 OPTIONS = {"attention_kernel": 0, "attention_splits": 1, "attention_lo": 2, "accept_team": 3, "dual_max_rows": 4,
            "tk_grid": 5, "tk_flat": 6, "gemm_ring_kb": 7, "gemm_epi_groups": 8}
@@ -125,6 +125,8 @@ def lib() -> C.CDLL:
         l.viasd_region_mass.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_float, C.c_float, C.c_float,
                                         C.c_void_p, C.c_void_p, C.c_void_p]
         l.viasd_set_option.argtypes = [C.c_void_p, C.c_int, C.c_int]
+        l.viasd_gemm_status.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.c_void_p]
+        l.viasd_gemm_static_status.argtypes = [C.POINTER(C.c_int), C.c_void_p]
         l.viasd_selftest_wait_expiry.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
         l.viasd_launch_count.restype = C.c_ulonglong
         l.viasd_set_timing.argtypes = [C.c_void_p, C.c_int]
@@ -304,6 +306,18 @@ def selftest_wait_expiry(status: torch.Tensor, limit_us: int, waited_cycles: Opt
     assert status.dtype == torch.int32 and (waited_cycles is None or waited_cycles.dtype == torch.int64)
     _check(lib().viasd_selftest_wait_expiry(_ptr(status), int(limit_us), _ptr(waited_cycles), _stream(stream)),
            "viasd_selftest_wait_expiry")
+
+
+def gemm_status(scratch: torch.Tensor, n: int, stream=None) -> int:
+    out = C.c_int(0)
+    _check(lib().viasd_gemm_status(_ptr(scratch), n, C.byref(out), _stream(stream)), "viasd_gemm_status")
+    return out.value
+
+
+def gemm_static_status(stream=None) -> int:
+    out = C.c_int(0)
+    _check(lib().viasd_gemm_static_status(C.byref(out), _stream(stream)), "viasd_gemm_static_status")
+    return out.value
 
 
 def launch_count() -> int:

@@ -719,4 +719,14 @@ int viasd_gemm(const void *x, const void *w, float *y, int rows, int n, int k, i
     return VIASD_OK;
 }
 
+// What the last viasd_gemm call that used this scratch recorded (n as in that call): VIASD_OK, or VIASD_EDEVICE when
+// one of its bounded waits expired.  Synchronises `stream`.
+int viasd_gemm_status(const void *scratch, int n, int *host_out, void *stream) {
+    if (!scratch || !host_out || n < 1) return VIASD_EINVAL;
+    CUDA_TRY(cudaMemcpyAsync(host_out, (const int *)scratch + tc_tiles(n), sizeof(int), cudaMemcpyDeviceToHost,
+                             (cudaStream_t)stream));
+    CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    return VIASD_OK;
+}
+
 }  // extern "C"

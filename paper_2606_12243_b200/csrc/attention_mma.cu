@@ -102,7 +102,6 @@ struct AttnArgs {
     int streams, n_items, items_per_cta, fuse_merge, nstage, mt_eff;
     int *counters;              // [streams * batch * Hkv] arrivals per (sequence, kv head), zero between launches
     float scale;
-    int trace_on;               // trace builds only
 };
 
 __device__ __forceinline__ float ex2(float x) {            // 2^x, hardware approximation (2 ulp)
@@ -236,13 +235,6 @@ __device__ __forceinline__ Item decode_item(const AttnArgs &a, int item) {
     return it;
 }
 
-#ifdef VIASD_TC_TRACE
-__device__ long long g_at_trace[160 * 16];
-#define ATRACE(slot) do { if (a.trace_on && threadIdx.x == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_)); \
-                                             g_at_trace[blockIdx.x * 16 + (slot)] = (long long)t_; } } while (0)
-#else
-#define ATRACE(slot) do { } while (0)
-#endif
 
 // PLO / QLO: use the lo parts of the probabilities / of the query too
 template <bool PLO, bool QLO>
@@ -255,10 +247,6 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
     constexpr int ROWF = HD + 2;
     RUN_FLAG_EXIT(a.run_flag);
     PDL_TRIGGER();
-    ATRACE(0);
-#ifdef VIASD_TC_TRACE
-    if (a.trace_on && threadIdx.x == 0) { g_at_trace[blockIdx.x * 16 + 10] = 0; g_at_trace[blockIdx.x * 16 + 11] = 0; }
-#endif
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int NSTAGE = a.nstage;
     const int grp = a.H / a.Hkv, QR = grp * a.M, QRP = a.mt * 16;
@@ -311,9 +299,7 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
         const int row = (warp & (a.mt_eff - 1)) * 16 + (lane >> 2) + r * 8;
         anc_first[r] = row < (a.H / a.Hkv) * a.M ? a.tree[first_item.b].anc[row % a.M] : 0ull;
     }
-    ATRACE(1);
     PDL_WAIT();
-    ATRACE(2);
     if (threadIdx.x == 0) while (p_count < NSTAGE && issue_next(false)) { }
 
     uint32_t qh[8][4], ql[8][4];                             // this warp's query tile, hi and lo, as MMA A fragments
@@ -350,7 +336,6 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             }
             __syncthreads();
             q_be = it.be; q_g = it.g;
-            if (item == i0) ATRACE(3);
             if (active) {
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
@@ -374,16 +359,8 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
 
         for (int tile = 0; tile < it.n_tiles; ++tile, ++c_count) {
             const int st = c_count % NSTAGE;
-#ifdef VIASD_TC_TRACE
-            unsigned long long tw0_ = 0; if (a.trace_on && threadIdx.x == 0) asm volatile("mov.u64 %0, %globaltimer;" : "=l"(tw0_));
-#endif
             ok = mbar_wait(smem_u32(&bars[st]), (c_count / NSTAGE) & 1, a.status);
-#ifdef VIASD_TC_TRACE
-            if (a.trace_on && threadIdx.x == 0) { unsigned long long tw1_; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(tw1_));
-                g_at_trace[blockIdx.x * 16 + 10] += (long long)(tw1_ - tw0_); g_at_trace[blockIdx.x * 16 + 11] += 1; }
-#endif
             if (!__syncthreads_and(ok)) { ok = false; break; }   // leave together if any thread gave up
-            if (item == i0 && tile == 0) ATRACE(4);
             const uint32_t kst = base + st * STAGE_BYTES, vst = kst + 2 * HALF_BYTES;
             const int j0 = it.k_begin + tile * TKEYS;
             if (active) {
@@ -411,7 +388,6 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             if (threadIdx.x == 0) issue_next(false);
         }
         if (!ok) break;
-        if (item == i0) ATRACE(5);
 
         // ---- end of the item: merge the key groups of each query tile pairwise, in registers ----
         // (the fragment layouts match lane for lane, so the exchange buffer is just each lane's values)
@@ -451,7 +427,6 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             }
         }
         const bool single = a.nsplit == 1;
-        if (item == i0) ATRACE(6);
         if (active && kgroup == 0) {
             // this warp now holds its query tile for the whole key range: write it from registers
 #pragma unroll
@@ -489,7 +464,6 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
                 if (last_sh) a.counters[it.be * a.Hkv + it.g] = 0;
             }
             __syncthreads();
-            if (item == i0) ATRACE(7);
             if (last_sh) {
                 for (int row = warp; row < QR; row += WARPS) {
                     const int h = it.g * grp + row / a.M, i = row % a.M;
@@ -526,9 +500,7 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             }
             __syncthreads();
         }
-        ATRACE(8);
     }
-    ATRACE(9);
 }
 
 }  // namespace
@@ -567,7 +539,6 @@ int launch_attention_mma(viasd_model *m, const void *kc, const void *vc, bool sl
     const int grp = c.n_heads / c.n_kv_heads, mt = (grp * M + 15) / 16;
     const int mt_eff = mt <= 1 ? 1 : mt <= 2 ? 2 : mt <= 4 ? 4 : 8;
     AttnArgs a;
-    a.trace_on = 0;
     a.q = m->ws.q; a.part = m->ws.part; a.out = (__nv_bfloat16 *)m->ws.attn;
     a.out_plane = m->ws.rows_alloc * (size_t)c.n_heads * HD;
     a.len_eff = m->ws.len_eff; a.tree = m->ws.tree; a.status = &m->ws.stats->device_status; a.run_flag = m->run_flag;
@@ -577,15 +548,6 @@ int launch_attention_mma(viasd_model *m, const void *kc, const void *vc, bool sl
     a.counters = m->ws.attn_counters;
     a.fuse_merge = fuse_merge;
     a.mt_eff = mt_eff;
-#ifdef VIASD_TC_TRACE
-    {
-        static int n_launch = 0;
-        const char *e = getenv("VIASD_AT_TRACE_IDX");
-        a.trace_on = e && atoi(e) == n_launch ? 1 : 0;
-        if (a.trace_on) fprintf(stderr, "attention trace: nsplit %d fuse %d streams %d mt %d\n", nsplit, fuse_merge, streams, mt);
-        if (e && atoi(e) < 0) n_launch = 0; else ++n_launch;
-    }
-#endif
     a.n_items = streams * batch * c.n_kv_heads * nsplit;
     int grid = a.n_items < m->sm_count ? a.n_items : m->sm_count;
     a.items_per_cta = (a.n_items + grid - 1) / grid;
@@ -612,8 +574,3 @@ int launch_attention_mma(viasd_model *m, const void *kc, const void *vc, bool sl
     return VIASD_OK;
 }
 
-#ifdef VIASD_TC_TRACE
-extern "C" int viasd_debug_attn_trace(long long *host_out) {
-    return (int)cudaMemcpyFromSymbol(host_out, g_at_trace, sizeof(long long) * 160 * 16);
-}
-#endif

@@ -58,7 +58,6 @@ struct AttnTcArgs {
     uint32_t q_bytes;           // staged queries in all; the ring follows
     int *counters;              // arrivals per (stream, sequence, kv head), zero between launches
     float scale;                // log2(e) / sqrt(hd)
-    int trace_on;               // trace builds only
 };
 
 struct Item { int be, b, g, stream, split, n_ctx, k_begin, k_end, n_tiles, row_base; };
@@ -151,18 +150,6 @@ __device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&r)[16])
 }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-#ifdef VIASD_TC_TRACE
-__device__ long long g_atc_trace[160 * 16];
-__device__ __forceinline__ long long gt_now() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return (long long)t; }
-#define ATC_ON (a.trace_on && trow == 0)
-#define ATC_MARK(slot) do { if (ATC_ON) g_atc_trace[blockIdx.x * 16 + (slot)] = gt_now(); } while (0)
-#define ATC_T0() long long tt_ = ATC_ON ? gt_now() : 0
-#define ATC_ADD(slot) do { if (ATC_ON) { long long n_ = gt_now(); g_atc_trace[blockIdx.x * 16 + (slot)] += n_ - tt_; tt_ = n_; } } while (0)
-#else
-#define ATC_MARK(slot) do { } while (0)
-#define ATC_T0() do { } while (0)
-#define ATC_ADD(slot) do { } while (0)
-#endif
 
 __global__ void __launch_bounds__(AT_THREADS, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
@@ -244,21 +231,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         if (lane == 0) {
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TKEYS >> 3) << 17) | ((128u >> 4) << 24);
             const uint32_t idesc_pv = idesc | (1u << 16);                 // B (the V tile) is MN-major
-#ifdef VIASD_TC_TRACE
-            if (a.trace_on) { g_atc_trace[blockIdx.x * 16 + 13] = 0; g_atc_trace[blockIdx.x * 16 + 14] = 0; }
-#endif
             int c_tile = 0, n_q = 0, o_uses = 0, q_be = -1, q_g = -1;   // c_tile: tiles of earlier items (ring and buffer phase)
             bool ok = true;
             // tile g (counted over the whole CTA) uses stage g % NSTAGE and S / P buffer g & 1
             auto issue_qk = [&](int g) -> bool {
                 const int st = g % NSTAGE, sb = g & 1;
-#ifdef VIASD_TC_TRACE
-                long long tq0_ = a.trace_on ? gt_now() : 0;
-#endif
                 if (!mbar_wait(full_bar(st), (g / NSTAGE) & 1, &abort_sh, a.status)) return false;
-#ifdef VIASD_TC_TRACE
-                if (a.trace_on) g_atc_trace[blockIdx.x * 16 + 13] += gt_now() - tq0_;
-#endif
                 tc_fence_after();
                 const uint32_t kst = ring + st * STAGE_BYTES, d = tmem + TM_S + sb * 128;
 #pragma unroll
@@ -283,13 +261,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 for (int t = 0; t < it.n_tiles; ++t) {
                     const int g = c_tile + t, sb = g & 1, st = g % NSTAGE;
                     if (t == 0 && o_uses > 0 && !(ok = mbar_wait(ofree_bar, (o_uses - 1) & 1, &abort_sh, a.status))) break;
-#ifdef VIASD_TC_TRACE
-                    long long tp0_ = a.trace_on ? gt_now() : 0;
-#endif
                     if (!(ok = mbar_wait(pfull_bar(sb), (g >> 1) & 1, &abort_sh, a.status))) break;
-#ifdef VIASD_TC_TRACE
-                    if (a.trace_on) g_atc_trace[blockIdx.x * 16 + 14] += gt_now() - tp0_;
-#endif
                     tc_fence_after();
                     const uint32_t vst = ring + st * STAGE_BYTES + 2 * HALF_BYTES, pb = tmem + TM_S + sb * 128;
 #pragma unroll
@@ -314,12 +286,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         const bool live = row < QR, warp_live = (quarter * 32) % a.rows_per_rep < QR;
         const int KR = TKEYS / a.reps, key0 = rep * KR;                                // this replica's keys of a tile
         const uint32_t tlane = tmem + ((uint32_t)(quarter * 32) << 16);
-#ifdef VIASD_TC_TRACE
-        if (ATC_ON) for (int z = 0; z < 13; ++z) g_atc_trace[blockIdx.x * 16 + z] = 0;
-#endif
-        ATC_MARK(0);
         PDL_WAIT();
-        ATC_MARK(1);
         int s_cnt = 0, q_be = -1, q_g = -1, wg_phase = 0;        // s_cnt: tiles this CTA has finished (buffer phase)
         bool ok = true;
         auto wg_sync = [&]() -> bool {
@@ -364,7 +331,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 __syncwarp();
                 if (lane == 0) mbar_arrive(qfull_bar);
                 q_be = it.be; q_g = it.g;
-                if (item == i0) ATC_MARK(2);
             }
             const int h = it.g * grp + row / a.M, node = row % a.M;
             const unsigned long long anc = live ? a.tree[it.b].anc[node] : 0ull;
@@ -372,10 +338,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 
             for (int t = 0; t < it.n_tiles; ++t, ++s_cnt) {
                 const int sb = s_cnt & 1;
-                ATC_T0();
                 if (!(ok = mbar_wait(sfull_bar(sb), (s_cnt >> 1) & 1, &abort_sh, a.status))) break;
                 tc_fence_after();
-                ATC_ADD(3);
                 const int j0 = it.k_begin + t * TKEYS;
                 const bool masked = j0 + TKEYS > it.n_ctx || j0 + TKEYS > it.k_end;
                 const uint32_t tb = tlane + TM_S + sb * 128;               // this tile's S / P buffer, this warp's lanes
@@ -402,7 +366,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                         for (int e = 0; e < 16; ++e) m_tile = fmaxf(m_tile, ((vis >> e) & 1u) ? __uint_as_float(r[e]) : -INFINITY);
                     }
                 }
-                ATC_ADD(4);
                 float m_new = m_run, corr = 1.f;
                 if (live && m_tile > m_run + RESCALE_GAP) {            // also the first tile with a visible key (m_run = -inf)
                     m_new = m_tile;
@@ -422,7 +385,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                         tc_st32(tlane + TM_O + c * 32, r);
                     }
                 }
-                ATC_ADD(6);
                 // pass 2: weights and their row sum; P replaces S in place, per 16 keys 8 columns of bf16 pairs hi and
                 // 8 columns lo; the key columns of the other replicas are zeroed (their scores are not this row's business)
                 float l_tile = 0.f;
@@ -449,23 +411,17 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                         tc_st16(tb + c * 16, w);
                     }
                 }
-                ATC_ADD(7);
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(pfull_bar(sb));             // P (and the rescaled O) are in place
                 l_run = l_run * corr + l_tile;
                 m_run = m_new;
-                ATC_ADD(8);
-#ifdef VIASD_TC_TRACE
-                if (ATC_ON) g_atc_trace[blockIdx.x * 16 + 9] += 1;
-#endif
             }
             if (!ok) break;
             // the last P V of the item (and with it all earlier ones) has written O
             if (it.n_tiles > 0 && !(ok = mbar_wait(pvdone_bar((s_cnt - 1) & 1), ((s_cnt - 1) >> 1) & 1, &abort_sh, a.status))) break;
             tc_fence_after();
-            ATC_T0();
             // ---- the item's result: O row from TMEM (zeros for an empty key range) ----
             const int n_part = a.nsplit * a.reps;                      // key ranges to merge: CTAs x replicas
             const bool single = n_part == 1;
@@ -507,7 +463,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 __syncwarp();
                 if (lane == 0) mbar_arrive(ofree_bar);                 // the next item may overwrite O
             }
-            ATC_ADD(11);
             if (!single && a.fuse_merge) {
                 // last key range of this (sequence, kv head) to finish merges all of them, in range order
                 __threadfence();
@@ -555,15 +510,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 }
                 if (!(ok = wg_sync())) break;                          // last_sh is reused by the next item
             }
-            ATC_ADD(12);
         }
     }
 
     // ---------------- teardown ----------------
     __syncwarp();
-#ifdef VIASD_TC_TRACE
-    if (a.trace_on && threadIdx.x == 128) g_atc_trace[blockIdx.x * 16 + 10] = gt_now();
-#endif
     if (abort_sh && threadIdx.x == 0) {
         // give copies and MMAs that are still in flight time to land before shared memory and TMEM go away
         const long long t0 = clock64();
@@ -611,15 +562,6 @@ int launch_attention_tc(viasd_model *m, const void *kc, const void *vc, bool sli
     const int grp = c.n_heads / c.n_kv_heads, QR = grp * M;
     if (QR > 128) return VIASD_EINVAL;
     AttnTcArgs a;
-    a.trace_on = 0;
-#ifdef VIASD_TC_TRACE
-    {
-        static int n_launch = 0;
-        const char *e = getenv("VIASD_AT_TRACE_IDX");
-        a.trace_on = e && atoi(e) == n_launch ? 1 : 0;
-        if (e && atoi(e) < 0) n_launch = 0; else ++n_launch;
-    }
-#endif
     a.q = m->ws.q; a.part = m->ws.part; a.out = (__nv_bfloat16 *)m->ws.attn;
     a.out_plane = m->ws.rows_alloc * (size_t)c.n_heads * HD;
     a.len_eff = m->ws.len_eff; a.tree = m->ws.tree; a.status = &m->ws.stats->device_status; a.run_flag = m->run_flag;
@@ -659,8 +601,3 @@ int launch_attention_tc(viasd_model *m, const void *kc, const void *vc, bool sli
     return VIASD_OK;
 }
 
-#ifdef VIASD_TC_TRACE
-extern "C" int viasd_debug_attn_tc_trace(long long *host_out) {
-    return (int)cudaMemcpyFromSymbol(host_out, g_atc_trace, sizeof(long long) * 160 * 16);
-}
-#endif

@@ -53,7 +53,6 @@ struct AttnTkArgs {
     int flat, part_slots;       // flat: tiles (not key ranges) are dealt evenly to the CTAs; part_slots: partial slots per (row, head)
     int *counters;              // arrivals per (stream, sequence, kv head), zero between launches
     float scale;                // log2(e) / sqrt(hd)
-    int trace_on;               // trace builds only
 };
 
 struct Item { int be, b, g, stream, split, n_split, n_ctx, k_begin, k_end, n_tiles, row_base; };   // split of n_split key ranges of the pair
@@ -177,18 +176,6 @@ __device__ __forceinline__ uint32_t sw_off(uint32_t row, uint32_t col) {
     return row * 128u + ((((col >> 3) ^ (row & 7u))) << 4) + (col & 7u) * 2u;
 }
 
-#ifdef VIASD_TC_TRACE
-__device__ long long g_atk_trace[160 * 16];
-__device__ __forceinline__ long long gt_now() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return (long long)t; }
-#define ATK_ON (a.trace_on && et == 0)
-#define ATK_MARK(slot) do { if (ATK_ON) g_atk_trace[blockIdx.x * 16 + (slot)] = gt_now(); } while (0)
-#define ATK_T0() long long tt_ = ATK_ON ? gt_now() : 0
-#define ATK_ADD(slot) do { if (ATK_ON) { long long n_ = gt_now(); g_atk_trace[blockIdx.x * 16 + (slot)] += n_ - tt_; tt_ = n_; } } while (0)
-#else
-#define ATK_MARK(slot) do { } while (0)
-#define ATK_T0() do { } while (0)
-#define ATK_ADD(slot) do { } while (0)
-#endif
 
 template <int NR>                                           // query rows per kv head rounded up to 8, 16 or 32
 __global__ void __launch_bounds__(NR == 32 ? TK_THREADS + 128 : TK_THREADS, 1)
@@ -399,10 +386,6 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         const int quarter = warp & 3, kl = quarter * 32 + lane, et = threadIdx.x - 64;   // kl: key of the tile / dim of O^T
         const int sw = warp - 2, row0 = (sw >> 2) * RG;            // softmax warp number; first query row of its group
         const uint32_t tlane = tmem + ((uint32_t)(quarter * 32) << 16);
-#ifdef VIASD_TC_TRACE
-        if (ATK_ON) for (int z = 0; z < 16; ++z) g_atk_trace[blockIdx.x * 16 + z] = 0;
-#endif
-        ATK_MARK(0);
         int s_cnt = 0, q_be = -1, q_g = -1, wg_phase = 0;        // s_cnt: tiles this CTA has finished (buffer phase)
         int anc_b = -1;                                          // sequence whose ancestor sets anc_sh holds
         bool ok = true;
@@ -429,10 +412,6 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             }
             if (n_item == 0) {
                 PDL_WAIT();
-                ATK_MARK(1);
-#ifdef VIASD_TC_TRACE
-                if (ATK_ON) for (int z = 3; z < 12; ++z) g_atk_trace[blockIdx.x * 16 + z] = 0;
-#endif
             }
             if (!dry && it.b != anc_b) {
                 // the ancestor sets of this sequence's draft tree (every sequence may have its own)
@@ -471,7 +450,6 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 __syncwarp();
                 if (lane == 0 && !dry) mbar_arrive(qfull_bar);
                 if (!dry) { q_be = it.be; q_g = it.g; }
-                if (n_item == 0) ATK_MARK(2);
             }
             // Lane r of every warp keeps row r's running maximum (the four warps compute the same values); the other
             // lanes read it, as the exponent's reference, from the warp's copy in shared memory.
@@ -483,10 +461,8 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 
             for (int t = 0; t < it.n_tiles; ++t) {
                 const int sb = s_cnt & 1;
-                ATK_T0();
                 if (!dry && !(ok = mbar_wait(sfull_bar(sb), (s_cnt >> 1) & 1, &abort_sh, a.status))) break;
                 tc_fence_after();
-                ATK_ADD(3);
                 float s[RG];
                 load_rows<NR, RG>(tlane + TM_S + sb * 64, row0, s);
                 // visibility: past the key range nothing; in the committed context everything; among the block's own
@@ -500,7 +476,6 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 #pragma unroll
                     for (int r = 0; r < RG; ++r) if (!((anc_sh[(row0 + r) % a.M] >> tb) & 1ull)) s[r] = -INFINITY;
                 }
-                ATK_ADD(4);
                 // row maxima: over the warp's 32 keys by one warp-wide reduction per row (lane r keeps row r's), over the
                 // four warps through shared memory
                 {
@@ -513,9 +488,7 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     }
                     if (lane < RG) wmax_sh[sb][quarter][row0 + lane] = mine;
                 }
-                ATK_ADD(5);
                 if (!(ok = wg_sync())) break;
-                ATK_ADD(6);
                 bool moved_l = false;
                 if (lane < RG) {
                     const int rr = row0 + lane;
@@ -550,7 +523,6 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                         tc_wait_st();
                     }
                 }
-                ATK_ADD(7);
                 // weights of this key for every row; P^T (hi rows, lo rows) into shared memory for the MMA
                 uint8_t *pchunk = gen + 2 * QCH + (uint32_t)sb * 2 * QCH + (uint32_t)(kl >> 6) * QCH;
                 float mref[RG];                                  // read before the stores below: they could alias, which would
@@ -564,25 +536,18 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     *reinterpret_cast<__nv_bfloat16 *>(pchunk + sw_off(row0 + r, kl & 63)) = hi;
                     *reinterpret_cast<__nv_bfloat16 *>(pchunk + sw_off(NR + row0 + r, kl & 63)) = lo;
                 }
-                ATK_ADD(8);
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> the MMA's reads
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0 && !dry) mbar_arrive(pfull_bar(sb));     // S^T is read, P^T (and the rescaled O^T) are in place
                 if (!dry) ++s_cnt;
-                ATK_ADD(9);
-#ifdef VIASD_TC_TRACE
-                if (ATK_ON && !dry) g_atk_trace[blockIdx.x * 16 + 10] += 1;
-#endif
             }
             if (!ok) break;
-            ATK_T0();
             // ---- the item's result ----
             if (quarter == 0 && lane < RG) mraw_sh[row0 + lane] = m_lane;
             // the last MMA into O^T of the item (and with it all earlier ones) is complete
             if (!dry && it.n_tiles > 0 && !(ok = mbar_wait(pvdone_bar((s_cnt - 1) & 1), ((s_cnt - 1) >> 1) & 1, &abort_sh, a.status))) break;
             tc_fence_after();
-            ATK_ADD(13);
             float o[RG];
             if (it.n_tiles > 0) {
                 load_rows<NR, RG>(tlane + TM_O, row0, o);
@@ -591,7 +556,6 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 for (int r = 0; r < RG; ++r) o[r] = 0.f;
             }
             const bool single = it.n_split == 1;
-            ATK_ADD(15);
             // O^T and every thread's share of the row sums go through shared memory (the P^T buffers are idle: the item's
             // last MMA has read them) as [row][dim] and [row][key lane], and whole warps finish the rows in a rolled loop.
             // Unrolled over 32 rows, the sums and the stores were kilobytes of code run once per item: fetched cold, with
@@ -626,7 +590,6 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     if (lane == 0) { pdst[HD] = mraw_sh[r] * 0.6931471805599453f; pdst[HD + 1] = l; }   // natural-log units
                 }
             }
-            ATK_ADD(14);
             if (!dry && it.n_tiles > 0) {
                 tc_fence_before();
                 __syncwarp();
@@ -681,15 +644,11 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             } else {
                 if (!(ok = wg_sync())) break;                          // the staged rows are overwritten by the next item's P^T
             }
-            ATK_ADD(11);
         }
     }
 
     // ---------------- teardown ----------------
     __syncwarp();
-#ifdef VIASD_TC_TRACE
-    if (a.trace_on && threadIdx.x == 64) g_atk_trace[blockIdx.x * 16 + 12] = gt_now();
-#endif
     if (abort_sh && threadIdx.x == 0) {
         // give copies and MMAs that are still in flight time to land before shared memory and TMEM go away
         const long long t0 = clock64();
@@ -746,15 +705,6 @@ int launch_attention_tk(viasd_model *m, const void *kc, const void *vc, bool sli
     const int QR = hpi * M, subs = grp / hpi;                      // rows per item; items per kv head
     const int nr = QR <= 8 ? 8 : QR <= 16 ? 16 : 32;
     AttnTkArgs a;
-    a.trace_on = 0;
-#ifdef VIASD_TC_TRACE
-    {
-        static int n_launch = 0;
-        const char *e = getenv("VIASD_AT_TRACE_IDX");
-        a.trace_on = e && atoi(e) == n_launch ? 1 : 0;
-        if (e && atoi(e) < 0) n_launch = 0; else ++n_launch;
-    }
-#endif
     a.q = m->ws.q; a.part = m->ws.part; a.out = (__nv_bfloat16 *)m->ws.attn;
     a.out_plane = m->ws.rows_alloc * (size_t)c.n_heads * HD;
     a.len_eff = m->ws.len_eff; a.tree = m->ws.tree; a.status = &m->ws.stats->device_status; a.run_flag = m->run_flag;
@@ -806,8 +756,3 @@ int launch_attention_tk(viasd_model *m, const void *kc, const void *vc, bool sli
     return VIASD_OK;
 }
 
-#ifdef VIASD_TC_TRACE
-extern "C" int viasd_debug_attn_tk_trace(long long *host_out) {
-    return (int)cudaMemcpyFromSymbol(host_out, g_atk_trace, sizeof(long long) * 160 * 16);
-}
-#endif

@@ -13,6 +13,7 @@ constexpr int STATIC_CTAS = 160;                     // at most one CTA per SM i
 constexpr size_t STATIC_COUNTER_BYTES = (size_t)(STATIC_MAX_N / 128 + 64) * 4;          // tile counters + status word
 constexpr size_t STATIC_PARTIAL_BYTES = (size_t)STATIC_CTAS * 2 * 16 * 128 * 4;         // two partial-tile slots per CTA
 constexpr size_t STATIC_BYTES = STATIC_COUNTER_BYTES + STATIC_PARTIAL_BYTES;            // about 2.6 MB per device
+constexpr int STATIC_STATUS_WORD = STATIC_MAX_N / 128 + 63;                             // last word of the counter region
 
 // Lives in every device's copy of the module from load to exit.  In host code this name is only a handle
 // for the runtime's symbol lookup, not a device address.
@@ -61,8 +62,23 @@ extern "C" int viasd_gemm_static(const void *x, const void *w, float *y, int row
     L.rows = rows; L.row0 = 0; L.k = k; L.nt = 16; L.epi = EPI_STORE;
     L.out_f32 = y; L.ld_out = n;
     L.counters = (int *)base;
-    L.status = (int *)base + tc_tiles(n);
+    L.status = (int *)base + STATIC_STATUS_WORD;
     L.scratch = (float *)(base + STATIC_COUNTER_BYTES);
     L.sm_count = sms;
     return launch_gemm_tc(L, st);
+}
+
+// What the last viasd_gemm_static call on this device recorded: VIASD_OK, or VIASD_EDEVICE when one of its bounded
+// waits expired (y is then incomplete).  Synchronises `stream`; allocates nothing.
+extern "C" int viasd_gemm_static_status(int *host_out, void *stream) {
+    if (!host_out) return VIASD_EINVAL;
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= MAX_DEVICES) return VIASD_EUNSUPPORTED;
+    *host_out = VIASD_OK;
+    if (!g_scratch_ptr[dev]) return VIASD_OK;               // no call on this device yet
+    CUDA_TRY(cudaMemcpyAsync(host_out, (int *)g_scratch_ptr[dev] + STATIC_STATUS_WORD, sizeof(int), cudaMemcpyDeviceToHost,
+                             (cudaStream_t)stream));
+    CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    return VIASD_OK;
 }

@@ -44,8 +44,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
     RUN_FLAG_EXIT(p.run_flag);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may start its prologue
-    if (threadIdx.x == 0) TRACE(0);
-    SPAN_BEGIN(p);
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int NT = p.nt, S = p.stages;
     constexpr int NACC = DUAL ? 2 : 1;
@@ -76,7 +74,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_sh;
-    if (threadIdx.x == 0) TRACE(1);
 
     const int total_units = p.n_tiles * p.k_tiles;
     const int u_begin = blockIdx.x * p.units_per_cta;
@@ -116,9 +113,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                              "r"(DUAL ? 2 * p.a_tx[0] : p.a_tx[sidx]) : "memory");
                 load_w(it, mw, wrow, kt);
             }
-            TRACE(2);
             asm volatile("griddepcontrol.wait;" ::: "memory");
-            TRACE(3);
             for (int it = 0; it < pre; ++it) {
                 unit(it, mw, wrow, kt, sidx);
                 mbar_expect_tx(full_bar(it), 2 * p.b_tx);
@@ -148,7 +143,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                 for (int kt = sg.ka; kt < sg.kb; ++kt, ++it) {
                     const int st = it % S;
                     if (!(ok = mbar_wait(full_bar(st), (it / S) & 1, &abort_sh, p.status))) break;
-                    if (it == 0) TRACE(4);
                     tc_fence_after();
                     const uint32_t base = smem_base + st * stage_bytes;
                     // the hi tile is followed by the lo tile: together one K-major operand of NB rows
@@ -164,7 +158,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                 if (ok) tc_commit(tfull_bar(buf));          // accumulator complete
                 ++acc_it;
             }
-            TRACE(5);
         }
     } else {
         // ---------------- epilogue (warps 2..5 and 6..9 <-> TMEM lane quarters 2,3,0,1) ----------------
@@ -217,7 +210,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                 if (!next_seg(u, u_end, p.k_tiles, sg)) break;
                 buf = acc_it % p.acc_bufs;
                 if (!(ok = mbar_wait(tfull_bar(buf), (acc_it / p.acc_bufs) & 1, &abort_sh, p.status))) break;
-                if (et == 0) TRACE(6);
                 tc_fence_after();
                 t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * acc_cols;
                 if (sg.ka == 0 && sg.kb == p.k_tiles) {
@@ -246,7 +238,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                             if (DUAL) slot[(size_t)(NT + c + j) * TILE_F + f] = uu[j];
                         }
                     }
-                    if (et == 0) TRACE(7);
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(tempty_bar(buf));   // accumulator buffer may be overwritten
@@ -276,9 +267,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                         if (!abort_sh && (atomicAdd(&p.counters[sg.tile], 1 << 16) >> 16) == n_fin - 1) atomicExch(&p.counters[sg.tile], 0);
                     }
                     asm volatile("bar.sync 1, %0;" ::"n"(epi_threads) : "memory");
-                    if (et == 0) TRACE(8);
                     if (abort_sh) { ok = false; break; }
-                    if (et == 0) TRACE(13);
                     {
                         // this finisher's rows: whole chunks, dealt in order of CTA number
                         const int n_chunks = (p.rows + CH - 1) / CH, per = (n_chunks + n_fin - 1) / n_fin;
@@ -303,7 +292,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
 
             // ---- the one finishing loop, over blocks of rows (one block unless the gather is staged in rounds)
             const int fe = src == SRC_TMEM ? f : et;
-            const int rows_live = dry ? 0 : p.rows, rows_loop = dry ? (DBG(p, 2) ? 0 : CH) : row_end;
+            const int rows_live = dry ? 0 : p.rows, rows_loop = dry ? CH : row_end;
             const int blk_rows = stage_rows ? stage_rows : (rows_loop > 0 ? rows_loop : 1);
             const int plane = stage_rows ? stage_rows * TILE_F : p.rows * TILE_F;     // floats between contributors in shared memory
             int round = 0;
@@ -340,7 +329,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                     mbar_arrive(gather_bar);
                 }
                 if (!(ok = mbar_wait(gather_bar, round & 1, &abort_sh, p.status))) break;
-                if (et == 0) TRACE(14);
                 parts = reinterpret_cast<const float *>(smem_raw + (part_sh - smem_u32(smem_raw)));
                 // finish_chunk indexes the epilogue's rows by their number in the launch: shift the base by the block start
                 if (aux_kind) aux = reinterpret_cast<const float *>(smem_raw + (aux_sh - smem_u32(smem_raw))) - (size_t)blk0 * TILE_F;
@@ -388,10 +376,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                         }
                     }
                 }
-                if (et == 0 && r0 == row_begin) TRACE(9);
                 finish_chunk<EPI, GROUPS>(p, sg.tile, fe, r0, g, uu, xch + group * (CH * TILE_F), inv_sh, rowmeta, lane, aux, rows_live,
                                   src != SRC_TMEM && sg.tile == last_tile, last_gain, GROUPS > 1 ? 2 + group : 1);
-                if (et == 0 && r0 == row_begin) TRACE(15);
             }
             }   // blocks of rows
 
@@ -449,14 +435,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                 continue;
             }
             if (src == SRC_TMEM) {
-                if (et == 0) TRACE(7);
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(tempty_bar(buf));   // accumulator buffer may be overwritten
             }
             ++acc_it;
             ++seg_i;
-            if (et == 0) TRACE(10);
         }
     }
 
@@ -469,8 +453,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
     }
     tc_fence_before();
     __syncthreads();
-    if (threadIdx.x == 0) { TRACE(11); TRACE_SM(); }
-    SPAN_END(p);
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
@@ -504,23 +486,6 @@ int tc_make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t k, u
     return VIASD_OK;
 }
 
-#ifdef VIASD_TC_TRACE
-extern "C" int viasd_debug_trace(long long *host_out) {
-    return (int)cudaMemcpyFromSymbol(host_out, g_tc_trace, sizeof(long long) * 160 * 16);
-}
-static int g_span_launches = 0;
-extern "C" int viasd_debug_span_reset(void) {
-    static unsigned long long init[8192 * 2];
-    for (int i = 0; i < 8192; ++i) { init[2 * i] = ~0ull; init[2 * i + 1] = 0ull; }
-    g_span_launches = 0;
-    return (int)cudaMemcpyToSymbol(g_tc_span, init, sizeof(init));
-}
-extern "C" int viasd_debug_span_read(unsigned long long *host_out, int *n_launches, int *meta) {
-    *n_launches = g_span_launches;
-    (void)meta;
-    return (int)cudaMemcpyFromSymbol(host_out, g_tc_span, sizeof(unsigned long long) * 8192 * 2);
-}
-#endif
 
 // token-tile width: the MMA's N (2 x NT with the hi / lo planes side by side, else NT) comes in multiples of 16
 int tc_pick_nt(int rows, bool has_lo) {
@@ -581,9 +546,6 @@ int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {
     const int units = p.n_tiles * p.k_tiles;
     if (units <= 0) return VIASD_OK;
     int ctas_per_sm = 1;
-#ifdef VIASD_TC_TRACE
-    if (getenv("VIASD_TC_PER_SM")) ctas_per_sm = atoi(getenv("VIASD_TC_PER_SM"));
-#endif
     int grid = L.sm_count * ctas_per_sm < units ? L.sm_count * ctas_per_sm : units;
     p.units_per_cta = (units + grid - 1) / grid;
     grid = (units + p.units_per_cta - 1) / p.units_per_cta;
@@ -595,12 +557,6 @@ int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {
     int stages = (int)((size_t)ring_kb * 1024 / stage);
     if (stages < 2) stages = 2;
     if (stages > MAX_STAGES) stages = MAX_STAGES;
-#ifdef VIASD_TC_TRACE
-    if (getenv("VIASD_TC_DBG")) p.dbg = atoi(getenv("VIASD_TC_DBG"));
-    p.launch_idx = g_span_launches++;
-    p.trace_on = getenv("VIASD_TC_TRACE_IDX") ? (atoi(getenv("VIASD_TC_TRACE_IDX")) == p.launch_idx) : 1;
-    if (getenv("VIASD_TC_STAGES")) { int v = atoi(getenv("VIASD_TC_STAGES")); if (v >= 2 && v < stages) stages = v; }
-#endif
     if (stages < 2) return VIASD_EINVAL;
     p.stages = stages;
     // accumulators are double-buffered when two of them fit in the 512 TMEM columns

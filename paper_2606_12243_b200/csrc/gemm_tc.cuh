@@ -21,7 +21,6 @@ struct TcParams {                       // kernel argument block
     float *scratch;                     // [grid][2] partial-tile slots
     int *counters;                      // [n_tiles], zero between launches
     int *status;                        // device status word
-    int dbg, launch_idx, trace_on;      // measurement knobs, honoured by trace builds only
     // fused RMSNorm on the input side: per-row partial sums of squares written by the producer
     const float *ssq_in; int ssq_in_n, ssq_stride; float inv_d, eps;
     // EPI_ADD_NORM: what the next RMSNorm needs

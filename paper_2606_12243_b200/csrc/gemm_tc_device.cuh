@@ -1,4 +1,4 @@
-// Device-side pieces of the tcgen05 GEMM kernel: tile constants, trace macros, the unit-range walk of the stream-K
+// Device-side pieces of the tcgen05 GEMM kernel: tile constants, the unit-range walk of the stream-K
 // schedule and the fused epilogues.
 #pragma once
 #include "common.cuh"
@@ -22,23 +22,6 @@ __device__ __forceinline__ void tc_ld8(uint32_t taddr, float (&v)[CH]) {
     for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-#ifdef VIASD_TC_TRACE
-__device__ long long g_tc_trace[160 * 16];                // per CTA of the traced launch: globaltimer ns at 16 points
-#define TRACE(slot) do { if (p.trace_on) { unsigned long long t_; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_)); \
-                                           g_tc_trace[blockIdx.x * 16 + (slot)] = (long long)t_; } } while (0)
-#define TRACE_SM() do { if (p.trace_on) { unsigned sm_; asm volatile("mov.u32 %0, %smid;" : "=r"(sm_)); g_tc_trace[blockIdx.x * 16 + 12] = sm_; } } while (0)
-#define DBG(p, bit) ((p).dbg & (bit))
-__device__ unsigned long long g_tc_span[8192 * 2];       // per launch: earliest CTA start, latest CTA end (globaltimer ns)
-__device__ __forceinline__ unsigned long long gtimer() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define SPAN_BEGIN(p) do { if (threadIdx.x == 0) atomicMin(&g_tc_span[((p).launch_idx & 8191) * 2], gtimer()); } while (0)
-#define SPAN_END(p) do { if (threadIdx.x == 0) atomicMax(&g_tc_span[((p).launch_idx & 8191) * 2 + 1], gtimer()); } while (0)
-#else
-#define SPAN_BEGIN(p) do { } while (0)
-#define SPAN_END(p) do { } while (0)
-#define DBG(p, bit) 0
-#define TRACE(slot) do { } while (0)
-#define TRACE_SM() do { } while (0)
-#endif
 
 struct Seg { int tile, ka, kb; };      // one contiguous piece of this CTA's unit range inside a tile
 
@@ -122,17 +105,9 @@ __device__ __forceinline__ void finish_chunk(const TcParams &p, int tile, int f,
         __nv_bfloat16 *ap = p.next_act + (size_t)(p.row0 + r0) * p.ld_out + n;
         if (touch) { want(hp); want(ap); want(ap + p.next_plane); want(p.ssq_out + ((size_t)tile * 4 + (f >> 5)) * p.ssq_stride + p.row0 + r0); }
         float v[CH];
-#ifdef VIASD_TC_TRACE
-        asm volatile("" :: "f"(gain_a), "f"(gain_b));
-        if (f == 0 && r0 == 0) TRACE(2);
-#endif
 #pragma unroll
         for (int j = 0; j < CH; ++j)
             v[j] = (valid && j < nrow) ? (aux ? aux[(r0 + j) * TILE_F + f] : __ldcg(hp + (size_t)j * p.ld_out)) + g[j] : 0.f;
-#ifdef VIASD_TC_TRACE
-        asm volatile("" :: "f"(v[0]), "f"(v[7]));
-        if (f == 0 && r0 == 0) TRACE(3);
-#endif
 #pragma unroll
         for (int j = 0; j < CH; ++j) {
             if (valid && j < nrow) {

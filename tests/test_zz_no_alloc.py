@@ -25,6 +25,18 @@ def _operands(rows, n, k, seed):
 def test_static_scratch_gemm_matches_caller_scratch_gemm(rows, n, k):
     from paper_2606_12243_b200 import binding as vb
     mem_before = torch.cuda.memory_allocated()
+    # one call beforehand (the first call on a device looks up the array's address and loads the kernel), then the
+    # device's free memory must not move over a call: torch's counters cannot see an allocation made by the library
+    x, w = _operands(rows, n, k, seed=39)
+    y = torch.empty((rows, n), dtype=torch.float32, device="cuda")
+    vb.gemm_static(x, w, y)
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    vb.gemm_static(x, w, y)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before, "viasd_gemm_static allocated device memory"
+    assert vb.gemm_static_status() == vb.VIASD_OK
+    del x, w, y
     for call in range(2):                                   # second call starts from the first call's leftovers
         x, w = _operands(rows, n, k, seed=40 + call)
         want = torch.full((rows, n), float("nan"), dtype=torch.float32, device="cuda")
@@ -33,6 +45,7 @@ def test_static_scratch_gemm_matches_caller_scratch_gemm(rows, n, k):
         got = torch.full((rows, n), float("nan"), dtype=torch.float32, device="cuda")
         vb.gemm_static(x, w, got)
         torch.cuda.synchronize()
+        assert vb.gemm_static_status() == vb.VIASD_OK and vb.gemm_status(scratch, n) == vb.VIASD_OK
         ref = x.float().cpu().double().numpy() @ w.float().cpu().double().numpy().T
         # same kernel, same schedule: the two entry points agree to the GEMM tests' tolerance (in fact bit for bit)
         tol = 2e-6 * np.sqrt(k) * np.abs(ref).max() + 1e-6
