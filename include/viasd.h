@@ -38,6 +38,10 @@
 extern "C" {
 #endif
 
+/* Verifiers that may judge a drafted token in one step: the slim verifiers, weakest first, and the full verifier
+ * last.  The method as benchmarked has two (three tiers); Sec. 3.2 and Table 1 go up to five tiers. */
+#define VIASD_MAX_JUDGES 4
+
 enum {
     VIASD_OK = 0,
     VIASD_EINVAL = -1,        /* null or misaligned pointer, shape out of range */
@@ -161,6 +165,26 @@ int viasd_slim_forward(viasd_model *m, const viasd_cache *cache, const viasd_dra
 int viasd_tier_accept(viasd_model *m, const viasd_draft *draft, const viasd_params *params,
                       const float *slim_logits, const float *full_logits, int phase, viasd_result *result,
                       void *stream);
+
+/* The tiered rule with more than one slim verifier (the n-tier remark of Sec. 3.2; Table 1): n_judges verifiers
+ * u_1 ... u_n = q, each a routed sub-network of the next (its own handle with its own mask, workspace and slim cache
+ * over the same weights; its logits come from viasd_slim_forward on that handle, q's from viasd_full_forward).
+ * log_tau: host, [n_judges], descending: tier 0 (accepted outright) from log_tau[0] up, tier k (judged by verifier
+ * k, counted from 1) between log_tau[k] and log_tau[k-1], tier n_judges (judged by q) below log_tau[n_judges-1].
+ * judge_logits: host array of n_judges device pointers [B, M, vocab], weakest verifier first.  conf_source 1 gates
+ * with the weakest verifier's confidence.  The walk is that of viasd_tier_accept: a tier-k child is judged by
+ * verifier k (greedy: log_acc_rel[1] for the slim verifiers, [2] for q; sampling: Eq. A.2 / A.3 with that verifier as
+ * the judge), the strongest judge that rejected emits the replacement; result.corr_src and the tier bits of
+ * result.judge run from 1 to n_judges.  With n_judges = 2 this is viasd_tier_accept with log_tau = (hi, lo).
+ * params.log_tau_hi / log_tau_lo are ignored.  Phases and errors as viasd_tier_accept.
+ * Committing an n-tier step: viasd_kv_commit_slim on every slim verifier's handle but one, then viasd_kv_commit on
+ * the remaining handle (it also moves q's rows and advances len, pending and tokens, which the handles share). */
+int viasd_tier_accept_n(viasd_model *m, const viasd_draft *draft, const viasd_params *params, int n_judges,
+                        const float *log_tau, const float *const *judge_logits, int phase, viasd_result *result,
+                        void *stream);
+/* Moves the accepted path's rows in this handle's slim cache only (no length changes): see viasd_tier_accept_n. */
+int viasd_kv_commit_slim(viasd_model *m, viasd_cache *cache, const viasd_draft *draft, const viasd_result *result,
+                         void *stream);
 
 /* Commit (Algorithm 1, the lines after the prefix is chosen: append the accepted prefix and the regenerated
  * token, discard the remaining suffix, advance t; Sec. 3.5 step 4): move the accepted path's K/V rows to

@@ -95,6 +95,27 @@ def tier_of(d: np.float32, log_tau_lo: float, log_tau_hi: float) -> int:
     return 2
 
 
+def tier_of_n(d: np.float32, log_taus: Sequence[float]) -> int:
+    """More than one slim verifier (Sec. 3.2, the n-tier remark; Table 1): descending log thresholds cut the
+    confidence axis into len(log_taus) + 1 tiers, tier 0 accepted outright, tier k judged by verifier k, the
+    last tier by the full verifier."""
+    for k, t in enumerate(log_taus):
+        if d >= np.float32(t):
+            return k
+    return len(log_taus)
+
+
+def tier_rule_n(conf_logits: np.ndarray, draft_tok: np.ndarray, src_row: Sequence[int], log_taus: Sequence[float]):
+    B, N = draft_tok.shape
+    tier = np.zeros((B, N), dtype=np.uint8)
+    d = np.zeros((B, N), dtype=np.float32)
+    for b in range(B):
+        for n in range(N):
+            d[b, n] = log_confidence(conf_logits[b, src_row[n]], int(draft_tok[b, n]))
+            tier[b, n] = tier_of_n(d[b, n], log_taus)
+    return tier, d
+
+
 def tier_rule(conf_logits: np.ndarray, draft_tok: np.ndarray, src_row: Sequence[int],
               log_tau_lo: float, log_tau_hi: float):
     """conf_logits [B, R, V]; src_row[n] = which row gates node n.  Returns tier [B,N] u8, d [B,N] f32."""
@@ -218,6 +239,18 @@ def resolve_sequence(b: int, tok: Sequence[int], parent: Sequence[int], prow: Se
                      tier: Sequence[int], drafter_logits: np.ndarray, slim_logits: np.ndarray,
                      full_logits: np.ndarray, P: Params) -> SeqResult:
     """One sequence.  drafter_logits [R, V]; slim_logits / full_logits [M, V] (row 0 = pending)."""
+    return resolve_sequence_n(b, tok, parent, prow, tier, drafter_logits, [slim_logits, full_logits], P)
+
+
+def resolve_sequence_n(b: int, tok: Sequence[int], parent: Sequence[int], prow: Sequence[int],
+                       tier: Sequence[int], drafter_logits: np.ndarray, judge_logits: Sequence[np.ndarray],
+                       P: Params) -> SeqResult:
+    """The same walk with J = len(judge_logits) verifiers, weakest first and the full verifier last (Sec. 3.2,
+    n-tier remark): a tier-k child is judged by verifier k; J = 2 is the three-tier method.  The greedy gate of
+    the slim verifiers is log_acc_rel[1], the full verifier's log_acc_rel[2]."""
+    J = len(judge_logits)
+    full_logits = judge_logits[J - 1]
+    gate = lambda t: P.log_acc_rel[1] if t < J else P.log_acc_rel[2]
     N = len(parent)
     children = [[] for _ in range(N + 1)]
     for n, p in enumerate(parent):
@@ -226,7 +259,7 @@ def resolve_sequence(b: int, tok: Sequence[int], parent: Sequence[int], prow: Se
     sampling = P.mode == "sampling"
     k_acc = stream_key(P.seed, P.step, b, STREAM_ACCEPT)
     k_gum = stream_key(P.seed, P.step, b, STREAM_GUMBEL)
-    L = {1: slim_logits, 2: full_logits}
+    L = {k + 1: judge_logits[k] for k in range(J)}
     cur = 0
     corr = None
     while True:
@@ -238,12 +271,11 @@ def resolve_sequence(b: int, tok: Sequence[int], parent: Sequence[int], prow: Se
                 else:
                     row = np.asarray(full_logits[cur])
                     corr, gap = int(np.argmax(row)), _top2_gap(row)
-                res.corr_src = 2
-                res.decisions.append(Decision("draw", cur, 2, gap))
+                res.corr_src = J
+                res.decisions.append(Decision("draw", cur, J, gap))
             break
         if sampling:
-            r = {1: softmax64(slim_logits[cur], P.temperature),
-                 2: softmax64(full_logits[cur], P.temperature)}
+            r = {k: softmax64(L[k][cur], P.temperature) for k in L}
             ptil = softmax64(drafter_logits[prow[C[0]]], P.temperature)
         failed, taken = 0, None
         for c in C:
@@ -259,9 +291,9 @@ def resolve_sequence(b: int, tok: Sequence[int], parent: Sequence[int], prow: Se
                 margin = abs(float(lr - np.log(u)))
             else:
                 row = np.asarray(L[t][cur])
-                dlt = float(row[v] - row.max()) - float(P.log_acc_rel[t])
+                dlt = float(row[v] - row.max()) - float(gate(t))
                 ok = dlt >= 0.0
-                if P.log_acc_rel[t] == 0.0:               # argmax test: flip point is the runner-up
+                if gate(t) == 0.0:                        # argmax test: flip point is the runner-up
                     margin = _top2_gap(row) if ok else -dlt
                 else:
                     margin = abs(dlt)
@@ -278,9 +310,9 @@ def resolve_sequence(b: int, tok: Sequence[int], parent: Sequence[int], prow: Se
                 r[t] = residual(r[t], ptil, P.beta)
                 ptil = drop_token(ptil, v)
         if taken is not None:
-            if P.strict_break and int(tier[taken]) == 1:
-                corr, res.corr_src = int(tok[taken]), 1
-                res.judge[taken] = 1 | (1 << 4)
+            if P.strict_break and 1 <= int(tier[taken]) < J:
+                corr, res.corr_src = int(tok[taken]), int(tier[taken])
+                res.judge[taken] = 1 | (int(tier[taken]) << 4)
                 break
             res.path.append(taken)
             cur = taken + 1
@@ -296,6 +328,12 @@ def resolve_sequence(b: int, tok: Sequence[int], parent: Sequence[int], prow: Se
     res.n_acc = len(res.path)
     res.out_tok = [int(tok[n]) for n in res.path] + ([corr] if corr is not None else [])
     return res
+
+
+def resolve_n(draft_tok: np.ndarray, parent: Sequence[int], prow: Sequence[int], tier: np.ndarray,
+              drafter_logits: np.ndarray, judge_logits: Sequence[np.ndarray], P: Params) -> List[SeqResult]:
+    return [resolve_sequence_n(b, draft_tok[b], parent, prow, tier[b], drafter_logits[b],
+                               [j[b] for j in judge_logits], P) for b in range(draft_tok.shape[0])]
 
 
 def resolve(draft_tok: np.ndarray, parent: Sequence[int], prow: Sequence[int], tier: np.ndarray,

@@ -22,7 +22,8 @@ EXPORTS = ["viasd_workspace_bytes", "viasd_init_model", "viasd_full_forward", "v
            "viasd_tier_accept", "viasd_kv_commit", "viasd_verify_step", "viasd_get_stats",
            "viasd_free_model", "viasd_strerror", "viasd_last_cuda_error", "viasd_gemm_scratch_bytes",
            "viasd_gemm", "viasd_gemm_static", "viasd_kl_cost", "viasd_region_mass", "viasd_launch_count", "viasd_set_timing", "viasd_get_timing",
-           "viasd_set_option", "viasd_selftest_wait_expiry", "viasd_gemm_status", "viasd_gemm_static_status"]
+           "viasd_set_option", "viasd_selftest_wait_expiry", "viasd_gemm_status", "viasd_gemm_static_status",
+           "viasd_tier_accept_n", "viasd_kv_commit_slim"]
 
 OPTIONS = {"attention_kernel": 0, "attention_splits": 1, "attention_lo": 2, "accept_team": 3, "dual_max_rows": 4,
            "tk_grid": 5, "tk_flat": 6, "gemm_ring_kb": 7, "gemm_epi_groups": 8}
@@ -107,6 +108,9 @@ def lib() -> C.CDLL:
         l.viasd_tier_accept.argtypes = [C.c_void_p, C.POINTER(Draft), C.POINTER(Params), C.c_void_p, C.c_void_p,
                                         C.c_int, C.POINTER(Result), C.c_void_p]
         l.viasd_kv_commit.argtypes = [C.c_void_p, C.POINTER(Cache), C.POINTER(Draft), C.POINTER(Result), C.c_void_p]
+        l.viasd_kv_commit_slim.argtypes = l.viasd_kv_commit.argtypes
+        l.viasd_tier_accept_n.argtypes = [C.c_void_p, C.POINTER(Draft), C.POINTER(Params), C.c_int, C.POINTER(C.c_float),
+                                          C.POINTER(C.c_void_p), C.c_int, C.POINTER(Result), C.c_void_p]
         l.viasd_verify_step.argtypes = [C.c_void_p, C.POINTER(Cache), C.POINTER(Draft), C.POINTER(Params),
                                         C.c_void_p, C.c_void_p, C.POINTER(Result), C.c_void_p]
         l.viasd_get_stats.argtypes = [C.c_void_p, C.POINTER(Stats), C.c_void_p]
@@ -260,6 +264,24 @@ def tier_accept(m: Model, draft: Draft, params: Params, slim_logits, full_logits
     r = result.struct()
     _check(lib().viasd_tier_accept(m.handle, C.byref(draft), C.byref(params), _ptr(slim_logits), _ptr(full_logits),
                                    phase, C.byref(r), _stream(stream)), "viasd_tier_accept")
+
+
+def tier_accept_n(m: Model, draft: Draft, params: Params, log_tau: Sequence[float], judge_logits: Sequence[torch.Tensor],
+                  phase: int, result: ResultBuffers, stream=None) -> None:
+    """viasd_tier_accept_n: log_tau descending, judge_logits weakest verifier first and q last (None allowed in phase 1)."""
+    n = len(log_tau)
+    assert len(judge_logits) == n
+    r = result.struct()
+    taus = (C.c_float * n)(*[float(t) for t in log_tau])
+    ptrs = (C.c_void_p * n)(*[_ptr(t) for t in judge_logits])
+    _check(lib().viasd_tier_accept_n(m.handle, C.byref(draft), C.byref(params), n, taus, ptrs, phase, C.byref(r),
+                                     _stream(stream)), "viasd_tier_accept_n")
+
+
+def kv_commit_slim(m: Model, cache: Cache, draft: Draft, result: ResultBuffers, stream=None) -> None:
+    r = result.struct()
+    _check(lib().viasd_kv_commit_slim(m.handle, C.byref(cache), C.byref(draft), C.byref(r), _stream(stream)),
+           "viasd_kv_commit_slim")
 
 
 def kv_commit(m: Model, cache: Cache, draft: Draft, result: ResultBuffers, stream=None) -> None:

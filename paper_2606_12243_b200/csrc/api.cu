@@ -56,7 +56,8 @@ size_t carve(const viasd_config &c, char *base, Workspace *ws) {
     w.row_tok = cv.take<int>(R * 4);
     w.tree = cv.take<TreeInfo>(sizeof(TreeInfo) * (size_t)c.max_batch);
     w.stats = cv.take<DeviceStats>(sizeof(DeviceStats));
-    w.accept_scratch = cv.take<float>(((size_t)c.max_batch * 3 * c.vocab + (size_t)c.max_batch * 9 * VIASD_MAX_ROWS_PER_SEQ) * 4);
+    w.accept_scratch = cv.take<float>(((size_t)c.max_batch * (VIASD_MAX_JUDGES + 1) * c.vocab +
+                                       (size_t)c.max_batch * 3 * (VIASD_MAX_JUDGES + 1) * VIASD_MAX_ROWS_PER_SEQ) * 4);
     {
         const int nt = tc_pick_nt(R < 128 ? (int)R : 128, true);
         w.gemm_scratch = cv.take<float>(tc_scratch_floats(MAX_GEMM_CTAS, nt, true) * 4);
@@ -483,29 +484,53 @@ int viasd_slim_forward(viasd_model *m, const viasd_cache *cache, const viasd_dra
     return forward(m, cache, draft, true, logits, (cudaStream_t)stream);
 }
 
-static int tier_accept_impl(viasd_model *m, const viasd_draft *draft, const viasd_params *params, const float *slim_logits,
-                           const float *full_logits, int phase, viasd_result *result, bool tree_ready, void *stream) {
+static int tier_accept_set(viasd_model *m, const viasd_draft *draft, const viasd_params *params, const JudgeSet &js,
+                           int phase, viasd_result *result, bool tree_ready, void *stream) {
     int rc;
     if ((rc = check_draft(m, draft)) || (rc = check_params(params))) return rc;
     if (phase < 1 || phase > 3) return VIASD_EINVAL;
     if ((rc = check_result(result, phase))) return rc;
     if (draft->n_nodes < 1 || !draft->prow || !draft->drafter_logits || draft->n_prows < 1) return VIASD_EINVAL;
+    for (int k = 1; k < js.n; ++k) if (!(js.log_tau[k] <= js.log_tau[k - 1])) return VIASD_EINVAL;
     cudaStream_t st = (cudaStream_t)stream;
     if (phase & 1) {
-        if ((rc = timed(m, VIASD_T_TIER_ACCEPT, st, [&] { return launch_tier(m, draft, params, slim_logits, result, st); })))
-            return rc;
+        if ((rc = timed(m, VIASD_T_TIER_ACCEPT, st, [&] { return launch_tier(m, draft, params, js, result, st); }))) return rc;
     }
     if (phase & 2) {
-        if (!slim_logits || !full_logits) return VIASD_EINVAL;
-        if ((rc = timed(m, VIASD_T_TIER_ACCEPT, st, [&] { return launch_accept(m, draft, params, slim_logits, full_logits,
-                                                                          result, tree_ready, st); }))) return rc;
+        for (int k = 0; k < js.n; ++k) if (!js.logits[k]) return VIASD_EINVAL;
+        if ((rc = timed(m, VIASD_T_TIER_ACCEPT, st, [&] { return launch_accept(m, draft, params, js, result, tree_ready, st); })))
+            return rc;
     }
     return VIASD_OK;
+}
+
+static int tier_accept_impl(viasd_model *m, const viasd_draft *draft, const viasd_params *params, const float *slim_logits,
+                           const float *full_logits, int phase, viasd_result *result, bool tree_ready, void *stream) {
+    if (!params) return VIASD_EINVAL;
+    JudgeSet js{2, {slim_logits, full_logits}, {params->log_tau_hi, params->log_tau_lo}};
+    return tier_accept_set(m, draft, params, js, phase, result, tree_ready, stream);
 }
 
 int viasd_tier_accept(viasd_model *m, const viasd_draft *draft, const viasd_params *params, const float *slim_logits,
                       const float *full_logits, int phase, viasd_result *result, void *stream) {
     return tier_accept_impl(m, draft, params, slim_logits, full_logits, phase, result, false, stream);
+}
+
+int viasd_tier_accept_n(viasd_model *m, const viasd_draft *draft, const viasd_params *params, int n_judges,
+                        const float *log_tau, const float *const *judge_logits, int phase, viasd_result *result,
+                        void *stream) {
+    if (!params || n_judges < 1 || n_judges > VIASD_MAX_JUDGES || !log_tau || !judge_logits) return VIASD_EINVAL;
+    JudgeSet js;
+    js.n = n_judges;
+    for (int k = 0; k < VIASD_MAX_JUDGES; ++k) {
+        js.logits[k] = k < n_judges ? judge_logits[k] : nullptr;
+        js.log_tau[k] = k < n_judges ? log_tau[k] : 0.f;
+    }
+    // the thresholds of viasd_params play no part here, but its other fields are checked as usual
+    viasd_params p = *params;
+    p.log_tau_hi = js.log_tau[0];
+    p.log_tau_lo = js.log_tau[n_judges - 1];
+    return tier_accept_set(m, draft, &p, js, phase, result, false, stream);
 }
 
 int viasd_kv_commit(viasd_model *m, viasd_cache *cache, const viasd_draft *draft, const viasd_result *result,
@@ -514,7 +539,16 @@ int viasd_kv_commit(viasd_model *m, viasd_cache *cache, const viasd_draft *draft
     if ((rc = check_draft(m, draft)) || (rc = check_cache(cache))) return rc;
     if (!result || !result->n_acc || !result->path || !result->out_tok || !result->n_emit) return VIASD_EINVAL;
     cudaStream_t st = (cudaStream_t)stream;
-    return timed(m, VIASD_T_COMMIT, st, [&] { return launch_commit(m, cache, draft, result, st); });
+    return timed(m, VIASD_T_COMMIT, st, [&] { return launch_commit(m, cache, draft, result, false, st); });
+}
+
+int viasd_kv_commit_slim(viasd_model *m, viasd_cache *cache, const viasd_draft *draft, const viasd_result *result,
+                         void *stream) {
+    int rc;
+    if ((rc = check_draft(m, draft)) || (rc = check_cache(cache))) return rc;
+    if (!result || !result->n_acc || !result->path) return VIASD_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    return timed(m, VIASD_T_COMMIT, st, [&] { return launch_commit(m, cache, draft, result, true, st); });
 }
 
 // Routed execution policy (policy 1): the full verifier is invoked only when the walk needs it.
@@ -542,8 +576,9 @@ static int verify_step_routed(viasd_model *m, viasd_cache *cache, const viasd_dr
     }
     CUDA_TRY(cudaMemsetAsync(flag, 0, sizeof(int), st));
     AcceptProbe probe{G, flag, cache->len, cache->len_full};
-    if ((rc = timed(m, VIASD_T_TIER_ACCEPT, st, [&] { return launch_accept(m, draft, params, slim_logits, nullptr, result,
-                                                                      true, st, &probe); }))) return rc;
+    JudgeSet probe_set{2, {slim_logits, nullptr}, {params->log_tau_hi, params->log_tau_lo}};
+    if ((rc = timed(m, VIASD_T_TIER_ACCEPT, st, [&] { return launch_accept(m, draft, params, probe_set, result, true, st,
+                                                                      &probe); }))) return rc;
     m->run_flag = flag;
     rc = forward_sweep(m, cache, draft, 0, full_logits, nullptr, st, G);
     m->run_flag = nullptr;

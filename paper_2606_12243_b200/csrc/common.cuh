@@ -199,7 +199,7 @@ int launch_embed_norm(const viasd_model *m, const float *gain, int rows, cudaStr
 int launch_rmsnorm(const viasd_model *m, const float *gain, int rows, cudaStream_t st);
 int launch_rope_append(const viasd_model *m, void *kc, void *vc, int layer_ord, int batch, int M,
                        cudaStream_t st);
-int launch_commit(const viasd_model *m, viasd_cache *c, const viasd_draft *d, const viasd_result *r,
+int launch_commit(const viasd_model *m, viasd_cache *c, const viasd_draft *d, const viasd_result *r, bool slim_only,
                   cudaStream_t st);
 
 // gemm_rowwarp.cu -- generic CUDA-core GEMM (fp32 models; shapes the tensor-core kernels do not take)
@@ -231,13 +231,15 @@ int launch_attention_dual(viasd_model *m, const void *kf, const void *vf, int la
 int launch_embed_norm2(const viasd_model *m, const float *gain_full, const float *gain_slim, int rows, cudaStream_t st);
 
 // tier_accept.cu
-int launch_tier(const viasd_model *m, const viasd_draft *d, const viasd_params *p, const float *slim_logits,
-                viasd_result *r, cudaStream_t st);
+// The verifiers that may judge a drafted token, weakest first, q last (two for the three-tier method), with the
+// descending log thresholds that cut the confidence axis into n + 1 tiers.
+struct JudgeSet { int n; const float *logits[VIASD_MAX_JUDGES]; float log_tau[VIASD_MAX_JUDGES]; };
+int launch_tier(const viasd_model *m, const viasd_draft *d, const viasd_params *p, const JudgeSet &js, viasd_result *r,
+                cudaStream_t st);
 // probe != null: the walk on the slim verifier's logits alone, deciding whether the full verifier's pass is needed
 struct AcceptProbe { int replay_rows; int *need_full; const int *len, *len_full; };
-int launch_accept(const viasd_model *m, const viasd_draft *d, const viasd_params *p, const float *slim_logits,
-                  const float *full_logits, viasd_result *r, bool tree_ready, cudaStream_t st,
-                  const AcceptProbe *probe = nullptr);
+int launch_accept(const viasd_model *m, const viasd_draft *d, const viasd_params *p, const JudgeSet &js, viasd_result *r,
+                  bool tree_ready, cudaStream_t st, const AcceptProbe *probe = nullptr);
 
 // ---------------------------------------------------------------------------------------------
 // small device helpers

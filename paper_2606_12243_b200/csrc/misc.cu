@@ -337,8 +337,8 @@ int launch_rope_append(const viasd_model *m, void *kc, void *vc, int layer_ord, 
 template <typename T>
 __global__ void commit_move_kernel(T *kf, T *vf, T *ks, T *vs, const int *len_eff, const int *n_acc,
                                    const int *path, int N, int L, int Ls, int Hkv, int hd, int max_batch,
-                                   int max_ctx, const DeviceStats *stats) {
-    int layer = blockIdx.x, b = blockIdx.y, g = blockIdx.z;
+                                   int max_ctx, const DeviceStats *stats, int layer0) {
+    int layer = layer0 + blockIdx.x, b = blockIdx.y, g = blockIdx.z;
     if (layer < L && !stats->full_ran) return;                  // the full verifier's cache did not receive this block
     T *kc = layer < L ? kf : ks;
     T *vc = layer < L ? vf : vs;
@@ -378,22 +378,26 @@ __global__ void commit_advance_kernel(int *len, int *len_full, int *pending, int
     pending[b] = out_tok[b * (N + 1) + ne - 1];
 }
 
-int launch_commit(const viasd_model *m, viasd_cache *c, const viasd_draft *d, const viasd_result *r,
+// slim_only: move the accepted rows in this handle's slim cache and nothing else (lengths, pending token and token
+// list belong to the handle that commits last)
+int launch_commit(const viasd_model *m, viasd_cache *c, const viasd_draft *d, const viasd_result *r, bool slim_only,
                   cudaStream_t st) {
     const viasd_config &cf = m->cfg;
     int rc = launch_prep(m, c, d, false, st);
     if (rc) return rc;
-    dim3 grid(cf.n_layers + m->n_routed, d->batch, cf.n_kv_heads);
+    const int layer0 = slim_only ? cf.n_layers : 0;
+    dim3 grid(cf.n_layers + m->n_routed - layer0, d->batch, cf.n_kv_heads);
     int threads = cf.head_dim < 32 ? 32 : (cf.head_dim > 256 ? 256 : cf.head_dim);
     if (cf.dtype == 0)
         commit_move_kernel<float><<<grid, threads, 0, st>>>((float *)c->k_full, (float *)c->v_full, (float *)c->k_slim,
             (float *)c->v_slim, m->ws.len_eff, r->n_acc, r->path, d->n_nodes, cf.n_layers, m->n_routed, cf.n_kv_heads,
-            cf.head_dim, cf.max_batch, cf.max_ctx, m->ws.stats);
+            cf.head_dim, cf.max_batch, cf.max_ctx, m->ws.stats, layer0);
     else
         commit_move_kernel<__nv_bfloat16><<<grid, threads, 0, st>>>((__nv_bfloat16 *)c->k_full,
             (__nv_bfloat16 *)c->v_full, (__nv_bfloat16 *)c->k_slim, (__nv_bfloat16 *)c->v_slim, m->ws.len_eff, r->n_acc,
-            r->path, d->n_nodes, cf.n_layers, m->n_routed, cf.n_kv_heads, cf.head_dim, cf.max_batch, cf.max_ctx, m->ws.stats);
+            r->path, d->n_nodes, cf.n_layers, m->n_routed, cf.n_kv_heads, cf.head_dim, cf.max_batch, cf.max_ctx, m->ws.stats, layer0);
     LAUNCH_CHECK();
+    if (slim_only) return VIASD_OK;
     commit_advance_kernel<<<(d->batch + 63) / 64, 64, 0, st>>>(c->len, c->len_full, c->pending, c->tokens, m->ws.len_eff,
                                                                r->n_emit, r->out_tok, d->batch, d->n_nodes, cf.max_ctx,
                                                                m->ws.stats);

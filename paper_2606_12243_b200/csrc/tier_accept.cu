@@ -21,6 +21,8 @@
 namespace {
 
 constexpr int ACC_THREADS = 512;
+constexpr int MAXJ = VIASD_MAX_JUDGES;    // verifiers that may judge a drafted token (the last one is q); 2 for three tiers
+constexpr int KINDS = MAXJ + 1;           // distributions kept per position: the proposal and the judges
 constexpr int ACC_TEAM = 8;               // CTAs per sequence in sampling mode (a portable cluster size)
 
 // ---- counter-based uniforms -------------------------------------------------------------------
@@ -83,13 +85,15 @@ __device__ float block_max(float x, float *sh) {
 }
 
 // ---- tier kernel ------------------------------------------------------------------------------
+// n thresholds in descending order cut the log-confidence axis into n + 1 tiers: tier 0 (accepted outright) from
+// log_tau[0] up, tier k between log_tau[k] and log_tau[k - 1], tier n (the full verifier) below log_tau[n - 1].
+struct TierCuts { int n; float log_tau[MAXJ]; };
 // grid (gate rows per sequence, B).  conf_source 0: gate row of node n = prow[n], rows = drafter logits
 // [B, R, V]; conf_source 1: gate row = parent[n] + 1, rows = slim logits [B, M, V].
 __global__ void __launch_bounds__(256)
 tier_kernel(unsigned char *__restrict__ tier, float *__restrict__ conf, DeviceStats *stats,
             const float *__restrict__ gate_logits, const int *__restrict__ draft_tok, const int *__restrict__ prow,
-            const int *__restrict__ parent, int per_seq, int conf_source, int rows_per_seq, int N, int V, float log_tau_lo,
-            float log_tau_hi) {
+            const int *__restrict__ parent, int per_seq, int conf_source, int rows_per_seq, int N, int V, TierCuts cuts) {
     __shared__ float sh[32];
     const int gr = blockIdx.x, b = blockIdx.y;
     if (per_seq) { prow += (size_t)b * N; parent += (size_t)b * N; }     // every sequence has its own tree
@@ -115,29 +119,30 @@ tier_kernel(unsigned char *__restrict__ tier, float *__restrict__ conf, DeviceSt
         int t = draft_tok[b * N + n];
         t = min(max(t, 0), V - 1);
         float d = row[t] - mx;
-        int tr = d >= log_tau_hi ? 0 : (d >= log_tau_lo ? 1 : 2);
+        int tr = 0;                                              // thresholds descend: the first one d reaches names the tier
+        while (tr < cuts.n && d < cuts.log_tau[tr]) ++tr;
         tier[b * N + n] = (unsigned char)tr;
         conf[b * N + n] = d;
-        atomicAdd(&stats->tier_count[tr], 1ull);
-        if (tr == 1) stats->need_slim = 1;
-        if (tr == 2) stats->need_full = 1;
+        atomicAdd(&stats->tier_count[tr == 0 ? 0 : (tr == cuts.n ? 2 : 1)], 1ull);   // accepted / some slim verifier / q
+        if (tr > 0 && tr < cuts.n) stats->need_slim = 1;
+        if (tr == cuts.n) stats->need_full = 1;
     }
     if (gr == 0 && b == 0 && threadIdx.x == 0) atomicAdd(&stats->steps, 1ull);
 }
 
 // ---- row statistics ---------------------------------------------------------------------------
-// grid (rows, B, 3): kind 0 = drafter rows [B, R, V], 1 = slim [B, M, V], 2 = full [B, M, V].
+// grid (rows, B, 1 + judges): kind 0 = drafter rows [B, R, V], kind k = judge k's rows [B, M, V] (the last judge is q).
 // Per row: max, argmax (lowest index on ties) and, when want_z, sum exp((l - max) / T).
 constexpr int RS_STRIDE = VIASD_MAX_ROWS_PER_SEQ;
-struct RowStats { float *mx; int *arg; float *z; };       // each [B, 3, RS_STRIDE]
+struct RowStats { float *mx; int *arg; float *z; };       // each [B, KINDS, RS_STRIDE]
+struct RowPtrs { const float *p[KINDS]; };                // drafter logits, then each judge's
 
 __global__ void __launch_bounds__(512)
-row_stats_kernel(RowStats rs, const float *__restrict__ drafter, const float *__restrict__ slim,
-                 const float *__restrict__ full, int R, int M, int V, float inv_temp, int want_z) {
+row_stats_kernel(RowStats rs, RowPtrs src, int R, int M, int V, float inv_temp, int want_z) {
     __shared__ float sh[32];
     __shared__ MaxIdx shm[32];
     const int kind = blockIdx.z, b = blockIdx.y, r = blockIdx.x;
-    const float *base = kind == 0 ? drafter : (kind == 1 ? slim : full);
+    const float *base = src.p[kind];
     const int rows = kind == 0 ? R : M;
     if (!base || r >= rows) return;
     const float *row = base + ((size_t)b * rows + r) * V;
@@ -173,7 +178,7 @@ row_stats_kernel(RowStats rs, const float *__restrict__ drafter, const float *__
         z = block_sum(z, sh);
     }
     if (threadIdx.x == 0) {
-        const size_t o = ((size_t)b * 3 + kind) * RS_STRIDE + r;
+        const size_t o = ((size_t)b * KINDS + kind) * RS_STRIDE + r;
         rs.mx[o] = best.v;
         rs.arg[o] = best.i == 0x7fffffff ? 0 : best.i;
         rs.z[o] = z;
@@ -183,18 +188,20 @@ row_stats_kernel(RowStats rs, const float *__restrict__ drafter, const float *__
 // ---- accept kernel ----------------------------------------------------------------------------
 struct AcceptArgs {
     RowStats rs;
-    const float *slim, *full, *drafter;      // [B, M, V], [B, M, V], [B, R, V]
+    const float *judges[KINDS];              // [1..n_judges]: each judge's logits [B, M, V], weakest first, q last
+    const float *drafter;                    // [B, R, V]
+    int n_judges;
     const int *draft_tok, *prow;             // [B, N], [N]
     const unsigned char *tier;               // [B, N]
     const TreeInfo *tree;
-    float *scratch;                          // [B, 3, V]
+    float *scratch;                          // [B, KINDS, V]
     int *n_acc, *path, *out_tok, *n_emit, *corr_src;
     unsigned char *judge;
     DeviceStats *stats;
     int N, R, V;
     int mode, strict_break, emit_bonus;
     float inv_temp, log1m_alpha, inv_beta;
-    float log_acc_rel[3];
+    float log_acc_rel[KINDS];                // greedy gate per judging tier
     unsigned long long seed, step;
     // Probe (routed execution policy): the same walk on the slim verifier's logits alone.  It stops where the full
     // verifier's judgment (a tier-2 node, or the bonus token at a leaf) would be needed and raises *need_full; it also
@@ -292,10 +299,12 @@ accept_kernel(AcceptArgs a) {
     const TreeInfo *tree = a.tree + b;
     const int *prow = a.prow + (a.per_seq ? (size_t)b * N : 0);
     const bool sampling = a.mode == 1;
-    float *P[3] = {a.scratch + ((size_t)b * 3 + 0) * V, a.scratch + ((size_t)b * 3 + 1) * V,
-                   a.scratch + ((size_t)b * 3 + 2) * V};
-    const float *st_mx = a.rs.mx + (size_t)b * 3 * RS_STRIDE, *st_z = a.rs.z + (size_t)b * 3 * RS_STRIDE;
-    const int *st_arg = a.rs.arg + (size_t)b * 3 * RS_STRIDE;
+    const int J = a.n_judges;                                 // tier J is the full verifier's
+    float *P[KINDS];
+#pragma unroll
+    for (int k = 0; k < KINDS; ++k) P[k] = a.scratch + ((size_t)b * KINDS + k) * V;
+    const float *st_mx = a.rs.mx + (size_t)b * KINDS * RS_STRIDE, *st_z = a.rs.z + (size_t)b * KINDS * RS_STRIDE;
+    const int *st_arg = a.rs.arg + (size_t)b * KINDS * RS_STRIDE;
     const unsigned long long k_acc = stream_key(a.seed, a.step, b, 0), k_gum = stream_key(a.seed, a.step, b, 1);
     if (tm.rank == 0 && !a.probe) for (int n = threadIdx.x; n < N; n += blockDim.x) a.judge[b * N + n] = 0;
     __syncthreads();
@@ -308,24 +317,32 @@ accept_kernel(AcceptArgs a) {
             if (a.emit_bonus && a.probe) { needs_q = true; break; }
             if (a.emit_bonus) {
                 if (sampling) {
-                    softmax_numerators(P[2], a.full + ((size_t)b * M + cur) * V, V, a.inv_temp, st_mx[2 * RS_STRIDE + cur], tm);
-                    corr = gumbel_argmax(P[2], V, k_gum, cur, shm, tm);
+                    softmax_numerators(P[J], a.judges[J] + ((size_t)b * M + cur) * V, V, a.inv_temp, st_mx[J * RS_STRIDE + cur], tm);
+                    corr = gumbel_argmax(P[J], V, k_gum, cur, shm, tm);
                 } else {
-                    corr = st_arg[2 * RS_STRIDE + cur];
+                    corr = st_arg[J * RS_STRIDE + cur];
                 }
-                corr_src = 2;
+                corr_src = J;
             }
             break;
         }
-        // the three distributions of this position: 0 = proposal (drafter row), 1 = q', 2 = q.  Each starts as
-        // "row + statistics" and is written out as numerators (mat) only once a residual has to be formed.
-        const float *row[3] = {nullptr, a.slim + ((size_t)b * M + cur) * V, a.full + ((size_t)b * M + cur) * V};
-        float mx[3] = {0.f, st_mx[1 * RS_STRIDE + cur], st_mx[2 * RS_STRIDE + cur]};
-        float Z[3] = {0.f, st_z[1 * RS_STRIDE + cur], st_z[2 * RS_STRIDE + cur]};
-        bool mat[3] = {false, false, false};
+        // the distributions of this position: 0 = proposal (drafter row), k = judge k (the slim verifiers, then q).  Each
+        // starts as "row + statistics" and is written out as numerators (mat) only once a residual has to be formed.
+        const float *row[KINDS];
+        float mx[KINDS], Z[KINDS];
+        bool mat[KINDS];
+        row[0] = nullptr; mx[0] = 0.f; Z[0] = 0.f; mat[0] = false;
+#pragma unroll
+        for (int k = 1; k < KINDS; ++k) {
+            const bool on = k <= J && a.judges[k] != nullptr;
+            row[k] = on ? a.judges[k] + ((size_t)b * M + cur) * V : nullptr;
+            mx[k] = on ? st_mx[k * RS_STRIDE + cur] : 0.f;
+            Z[k] = on ? st_z[k * RS_STRIDE + cur] : 0.f;
+            mat[k] = false;
+        }
         int failed = 0, taken = -1, taken_tier = 0;
         for (; c >= 0; c = tree->next_sibling[c]) {
-            const int t = a.tier[b * N + c];
+            const int t = min((int)a.tier[b * N + c], J);
             int v = a.draft_tok[b * N + c];
             v = min(max(v, 0), V - 1);
             if (t == 0) {
@@ -333,7 +350,7 @@ accept_kernel(AcceptArgs a) {
                 if (lead && !a.probe) a.judge[b * N + c] = 1;
                 break;
             }
-            if (t == 2 && a.probe) { needs_q = true; break; }     // from here on the walk depends on q
+            if (t == J && a.probe) { needs_q = true; break; }     // from here on the walk depends on q
             bool pass;
             if (!sampling) {
                 pass = (row[t][v] - mx[t]) >= a.log_acc_rel[t];
@@ -392,9 +409,9 @@ accept_kernel(AcceptArgs a) {
         }
         if (needs_q) break;
         if (taken >= 0) {
-            if (a.strict_break && taken_tier == 1) {
+            if (a.strict_break && taken_tier >= 1 && taken_tier < J) {
                 corr = min(max(a.draft_tok[b * N + taken], 0), V - 1);
-                corr_src = 1;
+                corr_src = taken_tier;
                 break;
             }
             if (lead && !a.probe) a.path[b * N + n_acc] = taken;
@@ -445,21 +462,26 @@ __global__ void tree_only_kernel(TreeInfo *tree, DeviceStats *stats, const int *
 
 }  // namespace
 
-int launch_tier(const viasd_model *m, const viasd_draft *d, const viasd_params *p, const float *slim_logits,
-                viasd_result *r, cudaStream_t st) {
+int launch_tier(const viasd_model *m, const viasd_draft *d, const viasd_params *p, const JudgeSet &js, viasd_result *r,
+                cudaStream_t st) {
     const int M = d->n_nodes + 1;
+    if (js.n < 1 || js.n > MAXJ) return VIASD_EINVAL;
     CUDA_TRY(cudaMemsetAsync(&m->ws.stats->need_slim, 0, 2 * sizeof(int), st));
-    const float *gate = p->conf_source == 0 ? d->drafter_logits : slim_logits;
+    const float *gate = p->conf_source == 0 ? d->drafter_logits : js.logits[0];   // Alg. 2 gates with the slim(mest) verifier
     const int rows = p->conf_source == 0 ? d->n_prows : M;
     if (!gate) return VIASD_EINVAL;
+    TierCuts cuts;
+    cuts.n = js.n;
+    for (int k = 0; k < MAXJ; ++k) cuts.log_tau[k] = k < js.n ? js.log_tau[k] : 0.f;
     tier_kernel<<<dim3(rows, d->batch), 256, 0, st>>>(r->tier, r->conf, m->ws.stats, gate, d->draft_tok, d->prow,
-        d->parent, d->per_sequence, p->conf_source, rows, d->n_nodes, m->cfg.vocab, p->log_tau_lo, p->log_tau_hi);
+        d->parent, d->per_sequence, p->conf_source, rows, d->n_nodes, m->cfg.vocab, cuts);
     LAUNCH_CHECK();
     return VIASD_OK;
 }
 
-int launch_accept(const viasd_model *m, const viasd_draft *d, const viasd_params *p, const float *slim_logits,
-                  const float *full_logits, viasd_result *r, bool tree_ready, cudaStream_t st, const AcceptProbe *probe) {
+int launch_accept(const viasd_model *m, const viasd_draft *d, const viasd_params *p, const JudgeSet &js, viasd_result *r,
+                  bool tree_ready, cudaStream_t st, const AcceptProbe *probe) {
+    if (js.n < 1 || js.n > MAXJ) return VIASD_EINVAL;
     if (!tree_ready) {                       // a forward pass of the same call has laid the tree out already
         tree_only_kernel<<<1, 64, 0, st>>>(m->ws.tree, m->ws.stats, d->parent, d->per_sequence, d->batch, d->n_nodes);
         LAUNCH_CHECK();
@@ -467,16 +489,22 @@ int launch_accept(const viasd_model *m, const viasd_draft *d, const viasd_params
     if (d->n_prows > RS_STRIDE) return VIASD_EINVAL;
     AcceptArgs a;
     {
-        // row statistics live behind the three distribution buffers
-        float *base = m->ws.accept_scratch + (size_t)m->cfg.max_batch * 3 * m->cfg.vocab;
-        const size_t n = (size_t)m->cfg.max_batch * 3 * RS_STRIDE;
+        // row statistics live behind the distribution buffers
+        float *base = m->ws.accept_scratch + (size_t)m->cfg.max_batch * KINDS * m->cfg.vocab;
+        const size_t n = (size_t)m->cfg.max_batch * KINDS * RS_STRIDE;
         a.rs.mx = base; a.rs.arg = reinterpret_cast<int *>(base + n); a.rs.z = base + 2 * n;
         const int M = d->n_nodes + 1, rows = M > d->n_prows ? M : d->n_prows;
-        row_stats_kernel<<<dim3(rows, d->batch, 3), 512, 0, st>>>(a.rs, p->mode == 1 ? d->drafter_logits : nullptr, slim_logits,
-            full_logits, d->n_prows, M, m->cfg.vocab, 1.0f / p->temperature, p->mode == 1);
+        RowPtrs src;
+        src.p[0] = p->mode == 1 ? d->drafter_logits : nullptr;
+        for (int k = 1; k < KINDS; ++k) src.p[k] = k <= js.n ? js.logits[k - 1] : nullptr;
+        row_stats_kernel<<<dim3(rows, d->batch, js.n + 1), 512, 0, st>>>(a.rs, src, d->n_prows, M, m->cfg.vocab,
+                                                                         1.0f / p->temperature, p->mode == 1);
         LAUNCH_CHECK();
     }
-    a.slim = slim_logits; a.full = full_logits; a.drafter = d->drafter_logits;
+    a.judges[0] = nullptr;
+    for (int k = 1; k < KINDS; ++k) a.judges[k] = k <= js.n ? js.logits[k - 1] : nullptr;
+    a.n_judges = js.n;
+    a.drafter = d->drafter_logits;
     a.draft_tok = d->draft_tok; a.prow = d->prow; a.tier = r->tier; a.tree = m->ws.tree;
     a.scratch = m->ws.accept_scratch;
     a.n_acc = r->n_acc; a.path = r->path; a.out_tok = r->out_tok; a.n_emit = r->n_emit; a.corr_src = r->corr_src;
@@ -486,7 +514,8 @@ int launch_accept(const viasd_model *m, const viasd_draft *d, const viasd_params
     a.inv_temp = 1.0f / p->temperature;
     a.log1m_alpha = log1pf(-p->alpha);
     a.inv_beta = 1.0f / p->beta;
-    for (int i = 0; i < 3; ++i) a.log_acc_rel[i] = p->log_acc_rel[i];
+    // greedy gates: log_acc_rel[1] for every slim verifier, log_acc_rel[2] for q
+    for (int k = 0; k < KINDS; ++k) a.log_acc_rel[k] = k == 0 ? p->log_acc_rel[0] : k < js.n ? p->log_acc_rel[1] : p->log_acc_rel[2];
     a.seed = p->seed; a.step = p->step;
     a.per_seq = d->per_sequence;
     a.probe = probe ? 1 : 0;

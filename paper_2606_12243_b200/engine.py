@@ -30,11 +30,15 @@ class Engine:
         return bool((before == 0xFF).all().item()) and bool((after == 0xFF).all().item())
 
     def __init__(self, wl: W.Workload, device="cuda", max_query: Optional[int] = None,
-                 extra_ctx: int = 0, fill_context=True, weights_from: Optional["Engine"] = None):
+                 extra_ctx: int = 0, fill_context=True, weights_from: Optional["Engine"] = None,
+                 state_from: Optional["Engine"] = None):
         """fill_context: True = the generator's committed context (what the parity tests compare against);
         "device" = values of the same distribution drawn on the device (timing sweeps over caches of tens of
         GB, where only the shape matters); False = leave the caches empty.
-        weights_from: another engine of the same model shape and seed whose weight tensors are reused."""
+        weights_from: another engine of the same model shape and seed whose weight tensors are reused.
+        state_from: a handle for one more slim verifier of the same model (an n-tier step): the full verifier's
+        cache, lengths, pending tokens and token list are the other engine's; only the slim cache and the workspace
+        are this engine's own."""
         self.wl, self.device = wl, device
         s = wl.shape
         self.tdtype = torch.float32 if s.dtype == "f32" else torch.bfloat16
@@ -70,26 +74,34 @@ class Engine:
                                    self.workspace)
         kv = lambda nl: torch.zeros((nl, wl.batch, s.n_kv_heads, self.max_ctx, s.head_dim), dtype=self.tdtype,
                                     device=device)
-        self.k_full, self.v_full = kv(s.n_layers), kv(s.n_layers)
         self.k_slim, self.v_slim = kv(len(self.routed)), kv(len(self.routed))
-        self.len = torch.zeros(wl.batch, dtype=torch.int32, device=device)
-        self.pending = torch.zeros(wl.batch, dtype=torch.int32, device=device)
-        self.tokens = torch.zeros((wl.batch, self.max_ctx), dtype=torch.int32, device=device)
-        self.len_full = torch.zeros(wl.batch, dtype=torch.int32, device=device)
+        if state_from is not None:
+            o = state_from
+            assert o.max_ctx == self.max_ctx and o.wl.batch == wl.batch and o.wl.shape == s
+            self.k_full, self.v_full, self.len, self.pending = o.k_full, o.v_full, o.len, o.pending
+            self.tokens, self.len_full = o.tokens, o.len_full
+        else:
+            self.k_full, self.v_full = kv(s.n_layers), kv(s.n_layers)
+            self.len = torch.zeros(wl.batch, dtype=torch.int32, device=device)
+            self.pending = torch.zeros(wl.batch, dtype=torch.int32, device=device)
+            self.tokens = torch.zeros((wl.batch, self.max_ctx), dtype=torch.int32, device=device)
+            self.len_full = torch.zeros(wl.batch, dtype=torch.int32, device=device)
         self.cache = vb.make_cache(self.k_full, self.v_full, self.k_slim, self.v_slim, self.len, self.pending,
                                    self.tokens, self.len_full)
         if fill_context == "device" and wl.ctx > 0:
             self.fill_random_context()
         elif fill_context and not wl.real_prefill and wl.ctx > 0:
-            self.fill_synthetic_context()
+            self.fill_synthetic_context(slim_only=state_from is not None)
         self.draft = None
         self.inputs = None
 
     # -- committed context ---------------------------------------------------------------
-    def fill_synthetic_context(self) -> None:
+    def fill_synthetic_context(self, slim_only: bool = False) -> None:
         wl = self.wl
         for cache_id, (kc, vc, nl) in enumerate(((self.k_full, self.v_full, wl.shape.n_layers),
                                                  (self.k_slim, self.v_slim, len(self.routed)))):
+            if slim_only and cache_id == 0:
+                continue
             for o in range(nl):
                 kc[o, :, :, :wl.ctx] = to_device(W.context_kv(wl, cache_id, o, 0), self.device)
                 vc[o, :, :, :wl.ctx] = to_device(W.context_kv(wl, cache_id, o, 1), self.device)

@@ -655,6 +655,111 @@ def test_argument_and_capacity_errors():
 
 
 # ---------------------------------------------------------------------------------------------
+# more than one slim verifier (n tiers)
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("name,mode,n_judges", [("mini_7b", "greedy", 3), ("mini_8b_tree", "sampling", 3),
+                                               ("mini_8b_tree_greedy", "greedy", 4), ("mini_32b", "sampling", 4)])
+def test_accept_with_n_judges_on_oracle_logits(name, mode, n_judges):
+    """viasd_tier_accept_n on oracle-supplied logits of three and four verifiers (four and five tiers): tiers bit-exact,
+    every decision with a margin above the fp32 noise as the oracle's."""
+    wl = replace(W.get(name), mode=mode)
+    vb = _vb()
+    eng = _tier_only_engine(wl)
+    B, N, M, V = wl.batch, wl.n_nodes, wl.rows, wl.shape.vocab
+    d_cal = tiers.tier_rule(*[W.step_inputs(wl, 0).drafter_logits, W.step_inputs(wl, 0).draft_tok, W.step_inputs(wl, 0).prow], 0.0, 0.0)[1]
+    taus = [float(np.quantile(d_cal, 1.0 - (k + 1) / (n_judges + 1))) for k in range(n_judges)]     # descending, even tiers
+    assert all(taus[k] > taus[k + 1] for k in range(n_judges - 1))
+    seen, pinned, total, full = set(), 0, 0, 0
+    for it in range(5):
+        si = W.step_inputs(wl, it)
+        jl = [synth.normal_f32(900 + k, 10 + it, (B, M, V), 1.5) for k in range(n_judges)]
+        for b in range(B):
+            for n in range(N):
+                if (n + b + it) % 4 != 3:
+                    for j in jl:
+                        j[b, wl.parent[n] + 1, si.draft_tok[b, n]] += 6.0 if mode == "greedy" else 3.0
+        tier, conf = tiers.tier_rule_n(si.drafter_logits, si.draft_tok, si.prow, taus)
+        P = tiers.Params(mode=mode, seed=wl.seed, step=it)
+        want = tiers.resolve_n(si.draft_tok, wl.parent, si.prow, tier, si.drafter_logits, jl, P)
+        eng.set_inputs(si)
+        res = vb.alloc_result(B, N)
+        vb.tier_accept_n(eng.model, eng.draft, eng.params(step=it, mode=1 if mode == "sampling" else 0), taus,
+                         [torch.from_numpy(j).cuda() for j in jl], 3, res)
+        torch.cuda.synchronize()
+        assert np.array_equal(res.tier.cpu().numpy(), tier) and np.array_equal(res.conf.cpu().numpy(), conf)
+        seen.update(int(t) for t in tier.ravel())
+        p_, t_, f_ = PU.compare_resolution(want, res.n_acc.cpu().numpy(), res.path.cpu().numpy(), res.out_tok.cpu().numpy(),
+                                           res.n_emit.cpu().numpy(), res.corr_src.cpu().numpy(), eps_row=2.5e-5)
+        for b, sq in enumerate(want):
+            if all(d.margin > 1e-4 for d in sq.decisions):
+                assert np.array_equal(res.judge[b].cpu().numpy(), sq.judge), (b, res.judge[b], sq.judge)
+        pinned += p_; total += t_; full += f_
+    assert vb.get_stats(eng.model).device_status == 0
+    assert seen == set(range(n_judges + 1)), seen
+    PU.assert_pinned(f"{name} {n_judges} judges", pinned, total, full, 5 * B, 0.9, int(0.9 * 5 * B))
+
+
+def test_four_tier_decoding_loop_with_two_slim_verifiers():
+    """Two slim verifiers nested in the full one (layers {0} within {0, 2} within all four): a handle per slim verifier
+    over the same weights and the same full cache, each pass through viasd_slim_forward / viasd_full_forward, the
+    four-tier rule through viasd_tier_accept_n, commits through viasd_kv_commit_slim and viasd_kv_commit; against the
+    oracle's forwards of the three sub-networks and its n-tier walk, over a loop of steps."""
+    wl2 = W.get("mini_7b")                                   # routes layers {0, 2}
+    wl1 = replace(wl2, n_routed=1)                           # routes layer {0}
+    assert wl1.routed == [0] and wl2.routed == [0, 2]
+    vb = _vb()
+    n_steps, M = 6, wl2.rows
+    e2 = _engine(wl2, extra_ctx=n_steps * M)
+    e1 = _engine(wl1, extra_ctx=n_steps * M, weights_from=e2, state_from=e2)
+    model = W.Model(wl2, keep=True)
+    st = PU.oracle_state(wl2, np.float64, extra=n_steps * M)
+    cap = wl2.ctx + M + n_steps * M
+    u1_cache = decoder.KVCache(1, wl2.batch, wl2.shape.n_kv_heads, wl2.shape.head_dim, cap, np.float64, wl2.ctx,
+                               lambda o, w: W.context_kv(wl1, 1, o, w))
+    inputs = [W.step_inputs(wl2, i) for i in range(n_steps)]
+    d_all = np.concatenate([tiers.tier_rule(si.drafter_logits, si.draft_tok, si.prow, 0.0, 0.0)[1].ravel() for si in inputs])
+    taus = [float(np.quantile(d_all, q)) for q in (0.75, 0.5, 0.25)]
+    st.pending[:] = inputs[0].pending
+    e2.set_inputs(inputs[0])
+    bufs = [e2.logits_buffer() for _ in range(3)]
+    res = vb.alloc_result(wl2.batch, wl2.n_nodes)
+    seen = set()
+    for i, si in enumerate(inputs):
+        rows = step.block_rows(st.pending, si.draft_tok)
+        want_l = [decoder.forward(model, wl2.shape, [0], u1_cache, st.lens, rows, wl2.parent),
+                  decoder.forward(model, wl2.shape, [0, 2], st.slim, st.lens, rows, wl2.parent),
+                  decoder.forward(model, wl2.shape, range(4), st.full, st.lens, rows, wl2.parent)]
+        tier, _ = tiers.tier_rule_n(si.drafter_logits, si.draft_tok, si.prow, taus)
+        want = tiers.resolve_n(si.draft_tok, wl2.parent, si.prow, tier, si.drafter_logits, want_l, PU.oracle_params(wl2, i))
+        decoder.commit([st.full, st.slim, u1_cache], st.lens, st.pending, st.tokens, [s_.n_acc for s_ in want],
+                       [s_.path for s_ in want], [s_.out_tok for s_ in want])
+        e2.set_inputs(si, set_pending=False)
+        e1.draft = e2.draft
+        vb.slim_forward(e1.model, e1.cache, e2.draft, bufs[0])
+        vb.slim_forward(e2.model, e2.cache, e2.draft, bufs[1])
+        vb.full_forward(e2.model, e2.cache, e2.draft, bufs[2])
+        vb.tier_accept_n(e2.model, e2.draft, e2.params(step=i), taus, bufs, 3, res)
+        vb.kv_commit_slim(e1.model, e1.cache, e2.draft, res)
+        vb.kv_commit(e2.model, e2.cache, e2.draft, res)
+        torch.cuda.synchronize()
+        assert vb.get_stats(e2.model).device_status == 0 and vb.get_stats(e1.model).device_status == 0
+        assert np.array_equal(res.tier.cpu().numpy(), tier)
+        seen.update(int(t) for t in tier.ravel())
+        errs = [PU.assert_logits_close(bufs[k].cpu().numpy(), want_l[k], "bf16", f"verifier {k + 1} step {i}")[0] for k in range(3)]
+        _, _, f_ = PU.compare_resolution(want, res.n_acc.cpu().numpy(), res.path.cpu().numpy(), res.out_tok.cpu().numpy(),
+                                         res.n_emit.cpu().numpy(), res.corr_src.cpu().numpy(), eps_row=max(errs))
+        if f_ != wl2.batch:
+            break                                            # an unpinned decision: the two loops may part ways from here
+        assert e2.len.cpu().tolist() == [int(x) for x in st.lens] and e2.pending.cpu().tolist() == [int(x) for x in st.pending]
+    assert i >= 2 and seen == {0, 1, 2, 3}
+    # the weakest verifier's own cache followed the commits: its committed rows are the oracle's
+    n = int(st.lens[0])
+    got = e1.k_slim[0, 0, :, wl2.ctx:n].float().cpu().numpy()
+    ref = u1_cache.k[0][0, :, :n - wl2.ctx]
+    assert np.abs(got - ref).max() <= 2e-2 * max(1.0, np.abs(ref).max())
+
+
+# ---------------------------------------------------------------------------------------------
 # a draft tree per sequence (dynamic drafts)
 # ---------------------------------------------------------------------------------------------
 @pytest.mark.parametrize("name", ["mini_8b_tree_greedy", "mini_8b_tree"])

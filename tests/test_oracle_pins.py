@@ -710,3 +710,78 @@ def test_algorithm_2_gate_reads_the_slim_verifier_at_the_parent_row():
         seen_ends.add(src)
     assert seen_regions == {0, 1, 2} and seen_ends == {0, 1, 2}
     assert discriminating > 20          # the other candidate rows would have placed many tokens elsewhere
+
+
+# --------------------------------------------------------------------------
+# more than one slim verifier (the n-tier remark of Sec. 3.2; Table 1)
+# --------------------------------------------------------------------------
+def test_n_tier_rule_cuts_the_confidence_axis_and_contains_the_three_tier_rule():
+    rng = np.random.default_rng(9)
+    d = rng.uniform(-8.0, 0.0, size=400).astype(np.float32)
+    taus = [-1.0, -2.5, -4.0, -6.5]                       # descending: five tiers
+    t = np.array([tiers.tier_of_n(x, taus) for x in d])
+    for k in range(5):
+        hi = 0.0 if k == 0 else taus[k - 1]
+        lo = -np.inf if k == 4 else taus[k]
+        inside = (d >= np.float32(lo)) & ((d < np.float32(hi)) if k else np.ones_like(d, dtype=bool))
+        assert np.array_equal(t == k, inside), k
+    assert set(t) == {0, 1, 2, 3, 4}
+    # two thresholds: exactly the three-tier rule of Eq. B.1-B.3
+    assert [tiers.tier_of_n(x, [-2.0, -5.0]) for x in d] == [tiers.tier_of(x, -5.0, -2.0) for x in d]
+    # lowering a threshold can only move tokens to a weaker tier
+    t2 = np.array([tiers.tier_of_n(x, [-1.0, -3.0, -4.0, -6.5]) for x in d])
+    assert (t2 <= t).all() and (t2 < t).any()
+
+
+def test_n_tier_sampling_draws_from_the_judge_of_the_token_s_tier():
+    """Four verifiers (five tiers): a tier-k token ends as a draw from verifier k (lossless rule, Eq. A.2-A.3 with
+    u_k as the judge), rejected with probability D_TV(p, u_k); a full acceptance with the bonus flag draws from q."""
+    rng = np.random.default_rng(4)
+    V, n_trials = 6, 16000
+    p = _rand_dist(rng, V)
+    judges = [_rand_dist(rng, V) for _ in range(4)]
+    dl = _fake_logits(p)[None, :]
+    jl = [np.stack([_fake_logits(j)] * 2) for j in judges]
+    draws = rng.choice(V, size=n_trials, p=p)
+    for t in (1, 2, 3, 4):
+        cnt, nrej = np.zeros(V), 0
+        for i in range(n_trials):
+            P = tiers.Params(mode="sampling", seed=99, step=i)
+            r = tiers.resolve_sequence_n(0, [int(draws[i])], (-1,), (0,), (t,), dl, jl, P)
+            cnt[r.out_tok[0]] += 1
+            nrej += r.n_acc == 0
+            assert r.corr_src == (0 if r.n_acc else t)
+        assert np.abs(cnt / n_trials - judges[t - 1]).max() < 0.015, (t, cnt / n_trials, judges[t - 1])
+        assert abs(nrej / n_trials - 0.5 * np.abs(p - judges[t - 1]).sum()) < 0.015
+    r = tiers.resolve_sequence_n(0, [2], (-1,), (0,), (0,), dl, jl, tiers.Params(mode="sampling", emit_bonus=True, seed=5))
+    assert r.n_acc == 1 and r.corr_src == 4 and len(r.out_tok) == 2
+
+
+def test_n_tier_greedy_cases():
+    V = 6
+    def row(best):
+        r = np.zeros(V); r[best] = 2.0
+        return r
+    par, prow, dl = W.chain(3), (0, 1, 2), np.zeros((3, V))
+    u1 = np.stack([row(1), row(5), row(5), row(5)])      # weakest verifier
+    u2 = np.stack([row(1), row(2), row(4), row(5)])
+    q = np.stack([row(1), row(2), row(3), row(0)])
+    J = [u1, u2, q]
+    # every node in the tier of a verifier that agrees: all accepted, nothing added; the bonus comes from q
+    r = tiers.resolve_sequence_n(0, [1, 2, 3], par, prow, (1, 2, 3), dl, J, tiers.Params())
+    assert (r.n_acc, r.out_tok, r.corr_src) == (3, [1, 2, 3], 0) and list(r.judge) == [1 | 16, 1 | 32, 1 | 48]
+    r = tiers.resolve_sequence_n(0, [1, 2, 3], par, prow, (1, 2, 3), dl, J, tiers.Params(emit_bonus=True))
+    assert r.out_tok == [1, 2, 3, 0] and r.corr_src == 3
+    # the second node left to the weakest verifier, which wants token 5: it rewrites, the rest is dropped
+    r = tiers.resolve_sequence_n(0, [1, 2, 3], par, prow, (1, 1, 3), dl, J, tiers.Params())
+    assert (r.n_acc, r.out_tok, r.corr_src) == (1, [1, 5], 1) and list(r.judge) == [1 | 16, 2 | 16, 0]
+    # the third node left to the middle verifier (wants 4): replacement from it, not from q (wants 3)
+    r = tiers.resolve_sequence_n(0, [1, 2, 3], par, prow, (3, 3, 2), dl, J, tiers.Params())
+    assert (r.n_acc, r.out_tok, r.corr_src) == (2, [1, 2, 4], 2)
+    # Algorithm 2's literal break applies to every slim verifier's acceptance, not to q's
+    r = tiers.resolve_sequence_n(0, [1, 2, 3], par, prow, (3, 2, 3), dl, J, tiers.Params(strict_break=True))
+    assert (r.n_acc, r.out_tok, r.corr_src) == (1, [1, 2], 2)
+    # two verifiers: the three-tier walk
+    a = tiers.resolve_sequence_n(0, [1, 2, 0], par, prow, (1, 2, 2), dl, [u2, q], tiers.Params())
+    b = tiers.resolve_sequence(0, [1, 2, 0], par, prow, (1, 2, 2), dl, u2, q, tiers.Params())
+    assert (a.n_acc, a.out_tok, a.corr_src, list(a.judge)) == (b.n_acc, b.out_tok, b.corr_src, list(b.judge)) == (2, [1, 2, 3], 2, [17, 33, 34])
