@@ -595,7 +595,7 @@ def run_ours(args, wl) -> None:
                           "ms_at_70pct_of_8tbs": ff["algorithmic_bytes"] / (0.7 * HBM_NOMINAL_GBS * 1e9) * 1e3,
                           "met": bool(ff.get("frac_of_8tbs", 0.0) >= 0.7)}
         assert b.status_ok()
-        if not args.no_sweep:
+        if not args.no_sweep and wl.name == DEFAULT_WORKLOAD:
             line["sweep"] = run_sweep(b, peak, tf_peak, 20)
         if not args.no_cpu_baseline:
             del b, eng
@@ -618,7 +618,8 @@ def main() -> None:
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-sweep", action="store_true", help="time the named workload only")
+    ap.add_argument("--no-sweep", action="store_true",
+                    help="time the named workload only (the sweep over the other configurations runs with the default workload)")
     ap.add_argument("--gate", default="drafter", choices=["drafter", "slim"],
                     help="whose confidence sets the tiers: the drafter's (default, what the benchmark configurations "
                          "say) or the slim verifier's with a tier-1 acceptance ending the block (Algorithm 2 as printed)")

@@ -92,6 +92,8 @@ def call_bytes(wl: Workload) -> dict:
 NCU_GEMM_TRAFFIC_MB = {
     # 7B layer shapes (captured with 18 token rows)
     (12288, 4096): 105.2, (4096, 4096): 34.1, (22016, 4096): 185.3, (4096, 11008): 96.6, (32000, 4096): 271.6,
+    # 8B layer shapes (captured with 27 token rows; the head with 54); (4096, 4096) is shared with the 7B shapes
+    (6144, 4096): 51.5, (28672, 4096): 243.0, (4096, 14336): 124.7, (128256, 4096): 1085.1,
 }
 
 
