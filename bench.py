@@ -359,6 +359,33 @@ def per_call(b: Bench, n: int, peak: float, tf_peak: float) -> dict:
     return out
 
 
+def graph_replay(b: Bench, n: int) -> dict:
+    """The same verify step captured once into a CUDA graph (the library's launches are capturable: caller's stream
+    only, no synchronisation, no allocation) and replayed: what the host-side launch cost of the ~170 kernels is worth."""
+    torch = b.torch
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            b.verify_step(0)
+        torch.cuda.current_stream().wait_stream(side)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            b.verify_step(0)
+        for _ in range(3):
+            g.replay()
+        torch.cuda.synchronize()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for _ in range(n):
+            g.replay()
+        ev1.record()
+        torch.cuda.synchronize()
+        return {"ms_per_step": ev0.elapsed_time(ev1) / n, "steps": n, "device_status_ok": b.status_ok()}
+    except Exception as e:                                       # a bench key, not a requirement of the path
+        return {"error": repr(e)[:200]}
+
+
 def run_routed_policy(weights_from: Bench, n_steps: int = 48, replay: int = 18) -> dict:
     """Decoding loops of n_steps verify steps on the 7B-shaped workload with thresholds at the 5th / 50th percentile
     of drafter confidence (most drafted tokens in tiers 0 and 1), once with both passes in every step (policy 0) and
@@ -587,6 +614,7 @@ def run_ours(args, wl) -> None:
     if world == 1:
         n_each = max(args.steps, 20)
         line["per_call"] = per_call(b, n_each, peak, tf_peak)
+        line["graph_replay"] = graph_replay(b, n_each)
         ff = line["per_call"]["full_forward"]
         line["target"] = {"what": "full-tier pass (viasd_full_forward) of the 8B-shaped model at batch 1: >= 70 % of "
                                   "the HBM roofline at 8 TB/s",

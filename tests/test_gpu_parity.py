@@ -521,6 +521,44 @@ def test_repeated_verify_steps_are_bit_identical(name, env, monkeypatch):
     assert vb.get_stats(eng.model).device_status == 0
 
 
+@pytest.mark.parametrize("name", ["mini_7b", "mini_8b_tree_greedy", "mini_13b"])
+def test_verify_step_replayed_from_a_cuda_graph_gives_the_same_bits(name):
+    """Every launch of a step goes to the caller's stream and nothing in it synchronises or allocates, so after one
+    ordinary call (which builds the tensor maps and sets the kernel attributes) a step can be captured into a CUDA graph
+    - programmatic dependent launches included - and replayed: same logits, same tokens, bit for bit."""
+    wl = W.get(name)
+    vb = _vb()
+    eng, st, si, model = _prepare(wl)
+    sl, fl = eng.logits_buffer(), eng.logits_buffer()
+    res = vb.alloc_result(wl.batch, wl.n_nodes)
+    len0, pend0 = eng.len.clone(), eng.pending.clone()
+    params = eng.params()
+
+    def one_step():
+        eng.len.copy_(len0)
+        eng.pending.copy_(pend0)
+        vb.verify_step(eng.model, eng.cache, eng.draft, params, sl, fl, res)
+
+    one_step()
+    torch.cuda.synchronize()
+    ref = [t.clone() for t in (sl, fl, res.tier, res.n_acc, res.path, res.out_tok, res.n_emit, eng.len, eng.pending, eng.k_full)]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        one_step()
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        one_step()
+    for _ in range(3):
+        sl.zero_(); fl.zero_(); res.out_tok.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        for a, b in zip(ref, (sl, fl, res.tier, res.n_acc, res.path, res.out_tok, res.n_emit, eng.len, eng.pending, eng.k_full)):
+            assert torch.equal(a, b)
+    assert vb.get_stats(eng.model).device_status == 0
+
+
 @pytest.mark.parametrize("name", ["mini_8b_tree", "mini_7b", "mini_13b"])
 def test_step_pieces_equal_fused_call(name):
     wl = W.get(name)
