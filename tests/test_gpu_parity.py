@@ -684,6 +684,36 @@ def test_argument_and_capacity_errors():
                        vb.alloc_result(wl.batch, wl.n_nodes))
     cfg = vb.make_config(2, 256, 4, 4, 48, 512, 1000, "bf16", 1, 64, 8)   # head_dim 48 unsupported
     assert vb.workspace_bytes(cfg, 1) == 0
+    # options: unknown option, value out of range
+    for opt, val in (("attention_kernel", 7), ("accept_team", 3), ("dual_max_rows", 500), ("gemm_ring_kb", 8)):
+        with pytest.raises(vb.ViasdError) as e:
+            vb.set_option(eng.model, opt, val)
+        assert e.value.code == vb.VIASD_EINVAL
+    assert vb.lib().viasd_set_option(eng.model.handle, 99, 0) == vb.VIASD_EINVAL
+    vb.set_option(eng.model, "attention_kernel", "tk")
+    vb.set_option(eng.model, "attention_kernel", "auto")
+    # the n-tier call: no judges, too many, thresholds that do not descend
+    res = vb.alloc_result(wl.batch, wl.n_nodes)
+    sl = eng.logits_buffer()
+    for taus, logits in (([], []), ([0.0] * 5, [sl] * 5), ([-3.0, -1.0], [sl, sl])):
+        with pytest.raises((vb.ViasdError, AssertionError)) as e:
+            vb.tier_accept_n(eng.model, eng.draft, eng.params(), taus, logits, 3, res)
+        assert isinstance(e.value, AssertionError) or e.value.code == vb.VIASD_EINVAL
+    # routed execution needs the token list and the full verifier's own length, and room for replayed rows
+    with pytest.raises(vb.ViasdError) as e:                  # max_query == M: nothing can be replayed
+        vb.verify_step(eng.model, eng.cache, eng.draft, eng.params(policy=1), sl, fl, res)
+    assert e.value.code == vb.VIASD_ECAPACITY
+    roomy = _engine(wl, max_query=wl.rows + 4)
+    roomy.set_inputs(si)
+    no_len_full = vb.make_cache(roomy.k_full, roomy.v_full, roomy.k_slim, roomy.v_slim, roomy.len, roomy.pending, roomy.tokens)
+    with pytest.raises(vb.ViasdError) as e:
+        vb.verify_step(roomy.model, no_len_full, roomy.draft, roomy.params(policy=1), roomy.logits_buffer(), roomy.logits_buffer(), res)
+    assert e.value.code == vb.VIASD_EINVAL
+    with pytest.raises(vb.ViasdError) as e:
+        vb.verify_step(roomy.model, roomy.cache, roomy.draft, roomy.params(policy=2), roomy.logits_buffer(), roomy.logits_buffer(), res)
+    assert e.value.code == vb.VIASD_EINVAL
+    torch.cuda.synchronize()
+    assert vb.get_stats(eng.model).device_status == 0
     # a sequence already at capacity: the pass clamps, stays in bounds and records the condition
     eng.len.fill_(eng.max_ctx - 2)
     vb.full_forward(eng.model, eng.cache, eng.draft, fl)
@@ -905,13 +935,15 @@ def test_expired_wait_is_reported_and_the_context_stays_usable():
 # ---------------------------------------------------------------------------------------------
 # routed execution policy: the full verifier runs only when the walk needs it
 # ---------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("name,replay", [("mini_7b", 18), ("mini_8b_tree_greedy", 12), ("mini_13b", 14)])
-def test_routed_policy_emits_what_running_both_passes_emits(name, replay):
+@pytest.mark.parametrize("name,replay,alg2", [("mini_7b", 18, False), ("mini_8b_tree_greedy", 12, False), ("mini_13b", 14, False),
+                                              ("mini_13b", 14, True)])
+def test_routed_policy_emits_what_running_both_passes_emits(name, replay, alg2):
     """A decoding loop under policy 1 (q' in every step, q only when a tier-2 node is reached before the first break,
     its cache caught up by replaying the last committed tokens) against the same loop under policy 0 and against the
     oracle, with thresholds that leave most blocks to tiers 0 and 1: same tiers, same accepted paths, same emitted
     tokens in every step; q's pass skipped in some steps and run in others; q''s cache identical, q's cache equal as
-    far as it is complete and complete again after a pass of q."""
+    far as it is complete and complete again after a pass of q.  alg2: the same with the slim verifier's own confidence
+    as the gate and a tier-1 acceptance ending the block (Algorithm 2 as printed)."""
     wl = W.get(name)
     vb = _vb()
     n_steps, M = 12, wl.rows
@@ -926,20 +958,26 @@ def test_routed_policy_emits_what_running_both_passes_emits(name, replay):
     for e in engs:
         e.set_inputs(inputs[0])
     bufs = [(e.logits_buffer(), e.logits_buffer(), vb.alloc_result(wl.batch, wl.n_nodes)) for e in engs]
-    ran, max_err = [], 0.0
+    ran, max_err, oracle_steps = [], 0.0, 0
+    oracle_on = True              # until a decision the margin rule leaves open lets the oracle's loop take another course
     for i, si in enumerate(inputs):
+        okw = dict(strict_break=True) if alg2 else {}
         want = step.verify_step(model, wl.shape, wl.routed, st, si.draft_tok, wl.parent, si.prow, si.drafter_logits,
-                                float(lo), float(hi), PU.oracle_params(wl, i))
+                                float(lo), float(hi), PU.oracle_params(wl, i, **okw),
+                                conf_source=1 if alg2 else 0) if oracle_on else None
+        gkw = dict(conf_source=1, strict_break=1) if alg2 else {}
         for pol, (e, (sl, fl, res)) in enumerate(zip(engs, bufs)):
             e.set_inputs(si, set_pending=False)
-            vb.verify_step(e.model, e.cache, e.draft, e.params(step=i, log_tau_lo=float(lo), log_tau_hi=float(hi), policy=pol),
+            vb.verify_step(e.model, e.cache, e.draft, e.params(step=i, log_tau_lo=float(lo), log_tau_hi=float(hi), policy=pol, **gkw),
                            sl, fl, res)
         torch.cuda.synchronize()
         stats = vb.get_stats(engs[1].model)
         assert stats.device_status == 0 and vb.get_stats(engs[0].model).device_status == 0
         ran.append(stats.full_ran)
         (sl0, fl0, r0), (sl1, fl1, r1) = bufs
-        assert np.array_equal(r0.tier.cpu().numpy(), want.tier) and torch.equal(r0.tier, r1.tier)
+        assert torch.equal(r0.tier, r1.tier)
+        if not alg2:                                          # the drafter's confidences are inputs: tiers are exact
+            assert np.array_equal(r0.tier.cpu().numpy(), want.tier)
         assert torch.equal(sl0, sl1), "the slim verifier's pass does not depend on the policy"
         for a, b in ((r0.n_acc, r1.n_acc), (r0.n_emit, r1.n_emit), (r0.corr_src, r1.corr_src)):
             assert torch.equal(a, b), (i, a, b)
@@ -947,18 +985,26 @@ def test_routed_policy_emits_what_running_both_passes_emits(name, replay):
             ne = int(r0.n_emit[b])
             assert r0.out_tok[b, :ne].tolist() == r1.out_tok[b, :ne].tolist(), (i, b)
             assert r0.path[b, :int(r0.n_acc[b])].tolist() == r1.path[b, :int(r1.n_acc[b])].tolist()
-        e1, _ = PU.assert_logits_close(sl1.cpu().numpy(), want.slim_logits, wl.shape.dtype, "slim")
-        if stats.full_ran:
-            e2, _ = PU.assert_logits_close(fl1.cpu().numpy(), want.full_logits, wl.shape.dtype, "full (replay pass)")
-            max_err = max(max_err, e2)
-        # the oracle's emitted tokens, wherever its decisions are pinned
-        PU.compare_resolution(want.seqs, r1.n_acc.cpu().numpy(), r1.path.cpu().numpy(), r1.out_tok.cpu().numpy(),
-                              r1.n_emit.cpu().numpy(), r1.corr_src.cpu().numpy(), eps_row=max(e1, max_err, 1e-3))
+        if oracle_on:
+            oracle_steps += 1
+            e1, _ = PU.assert_logits_close(sl1.cpu().numpy(), want.slim_logits, wl.shape.dtype, "slim")
+            if stats.full_ran:
+                e2, _ = PU.assert_logits_close(fl1.cpu().numpy(), want.full_logits, wl.shape.dtype, "full (replay pass)")
+                max_err = max(max_err, e2)
+            # the oracle's emitted tokens, wherever its decisions are pinned; with the slim verifier's confidence as the
+            # gate a tier next to a threshold may fall on the other side, and that sequence is then not compared
+            same = [b for b in range(wl.batch) if np.array_equal(r1.tier[b].cpu().numpy(), want.tier[b])]
+            _, _, whole = PU.compare_resolution(want.seqs, r1.n_acc.cpu().numpy(), r1.path.cpu().numpy(),
+                                                r1.out_tok.cpu().numpy(), r1.n_emit.cpu().numpy(), r1.corr_src.cpu().numpy(),
+                                                eps_row=max(e1, max_err, 1e-3), only=same)
+            if alg2 and whole != wl.batch:
+                oracle_on = False                             # from here on the two policies are compared with each other only
         assert torch.equal(engs[0].len, engs[1].len) and torch.equal(engs[0].pending, engs[1].pending)
         assert bool((engs[1].len_full <= engs[1].len).all())
         if stats.full_ran:
             assert torch.equal(engs[1].len_full, engs[1].len)
     assert 0 < sum(ran) < n_steps, f"q ran in steps {ran}: the loop must cover both a skipped and an executed pass"
+    assert oracle_steps >= (3 if alg2 else n_steps), oracle_steps
     assert vb.get_stats(engs[1].model).full_skipped == n_steps - sum(ran)
     assert vb.get_stats(engs[0].model).full_skipped == 0
     # caches: q' identical; q equal up to where policy 1 has it complete (values recomputed by a replay pass may differ
@@ -969,7 +1015,7 @@ def test_routed_policy_emits_what_running_both_passes_emits(name, replay):
         for c0, c1 in ((engs[0].k_full, engs[1].k_full), (engs[0].v_full, engs[1].v_full)):
             a, bb = c0[:, b, :, :n].float(), c1[:, b, :, :n].float()
             assert float((a - bb).abs().max()) <= 2.0 ** -7 * max(1.0, float(a.abs().max()))
-    print(f"{name}: full verifier ran in {sum(ran)} of {n_steps} steps")
+    print(f"{name}: full verifier ran in {sum(ran)} of {n_steps} steps; oracle compared in {oracle_steps}")
 
 
 # ---------------------------------------------------------------------------------------------
