@@ -55,9 +55,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int *st
     }
     return true;
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y) {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                 ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+// K/V tiles are read once per layer: their lines are marked to leave L2 first (what the kernels around this one hand
+// over to each other, and their instructions, stay)
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y, uint64_t pol) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "l"(pol) : "memory");
 }
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -268,6 +275,7 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
 
     // producer cursor (thread 0 only): next tile to request, in the CTA's flattened (item, tile) order
     int p_item = i0, p_tile = 0, p_count = 0;
+    const uint64_t kvpol = l2_evict_first_policy();
     Item pit = i0 < i1 ? decode_item(a, i0) : Item{};
     auto issue_next = [&](bool context_only) -> bool {      // false: nothing (more) to request under this condition
         while (p_item < i1 && p_tile >= pit.n_tiles) { ++p_item; p_tile = 0; if (p_item < i1) pit = decode_item(a, p_item); }
@@ -279,10 +287,10 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
         const CUtensorMap *mk = pit.stream ? &map_k2 : &map_k, *mv = pit.stream ? &map_v2 : &map_v;
         const int y = pit.row_base + k0;
         mbar_expect_tx(bar, STAGE_BYTES);
-        tma_load_2d(dst, mk, bar, 0, y);
-        tma_load_2d(dst + HALF_BYTES, mk, bar, 64, y);
-        tma_load_2d(dst + 2 * HALF_BYTES, mv, bar, 0, y);
-        tma_load_2d(dst + 3 * HALF_BYTES, mv, bar, 64, y);
+        tma_load_2d(dst, mk, bar, 0, y, kvpol);
+        tma_load_2d(dst + HALF_BYTES, mk, bar, 64, y, kvpol);
+        tma_load_2d(dst + 2 * HALF_BYTES, mv, bar, 0, y, kvpol);
+        tma_load_2d(dst + 3 * HALF_BYTES, mv, bar, 64, y, kvpol);
         ++p_tile; ++p_count;
         return true;
     };

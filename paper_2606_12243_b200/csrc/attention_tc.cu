@@ -200,6 +200,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     if (warp == 0) {
         // ---------------- TMA producer: the CTA's (item, tile) list, flattened ----------------
         if (lane == 0) {
+            const uint64_t kvpol = l2_evict_first_policy();    // the cache passes through once per layer
             int p_item = i0, p_tile = 0, p_count = 0;
             bool ok = true;
             Item pit = i0 < i1 ? decode_item(a, i0) : Item{};
@@ -214,10 +215,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 const CUtensorMap *mk = pit.stream ? &map_k2 : &map_k, *mv = pit.stream ? &map_v2 : &map_v;
                 const int y = pit.row_base + k0;
                 mbar_expect_tx(bar, STAGE_BYTES);
-                tma_load_2d(dst, mk, bar, 0, y);
-                tma_load_2d(dst + HALF_BYTES, mk, bar, 64, y);
-                tma_load_2d(dst + 2 * HALF_BYTES, mv, bar, 0, y);
-                tma_load_2d(dst + 3 * HALF_BYTES, mv, bar, 64, y);
+                tma_load_2d_hint(dst, mk, bar, 0, y, kvpol);
+                tma_load_2d_hint(dst + HALF_BYTES, mk, bar, 64, y, kvpol);
+                tma_load_2d_hint(dst + 2 * HALF_BYTES, mv, bar, 0, y, kvpol);
+                tma_load_2d_hint(dst + 3 * HALF_BYTES, mv, bar, 64, y, kvpol);
                 ++p_tile; ++p_count;
                 return true;
             };

@@ -250,6 +250,7 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     if (warp == 0) {
         // ---------------- TMA producer: the CTA's (item, tile) list, flattened ----------------
         if (lane == 0) {
+            const uint64_t kvpol = l2_evict_first_policy();    // the cache passes through once per layer
             if constexpr (!SPLIT) {
                 // few query rows: a tile's K and V share a ring slot and are requested together
                 int p_tile = 0, p_count = 0;
@@ -269,10 +270,10 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     const CUtensorMap *mk = pit.stream ? &map_k2 : &map_k, *mv = pit.stream ? &map_v2 : &map_v;
                     const int y = pit.row_base + k0;
                     mbar_expect_tx(bar, 2 * SLOT_BYTES);
-                    tma_load_2d(dst, mk, bar, 0, y);
-                    tma_load_2d(dst + HALF_BYTES, mk, bar, 64, y);
-                    tma_load_2d(dst + 2 * HALF_BYTES, mv, bar, 0, y);
-                    tma_load_2d(dst + 3 * HALF_BYTES, mv, bar, 64, y);
+                    tma_load_2d_hint(dst, mk, bar, 0, y, kvpol);
+                    tma_load_2d_hint(dst + HALF_BYTES, mk, bar, 64, y, kvpol);
+                    tma_load_2d_hint(dst + 2 * HALF_BYTES, mv, bar, 0, y, kvpol);
+                    tma_load_2d_hint(dst + 3 * HALF_BYTES, mv, bar, 64, y, kvpol);
                     ++p_tile; ++p_count;
                     return true;
                 };
@@ -299,8 +300,8 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 const CUtensorMap *mp = is_v ? (c.it.stream ? &map_v2 : &map_v) : (c.it.stream ? &map_k2 : &map_k);
                 const int y = c.it.row_base + k0;
                 mbar_expect_tx(bar, SLOT_BYTES);
-                tma_load_2d(dst, mp, bar, 0, y);
-                tma_load_2d(dst + HALF_BYTES, mp, bar, 64, y);
+                tma_load_2d_hint(dst, mp, bar, 0, y, kvpol);
+                tma_load_2d_hint(dst + HALF_BYTES, mp, bar, 64, y, kvpol);
                 ++c.tile; ++c.count;
                 return 1;
             };

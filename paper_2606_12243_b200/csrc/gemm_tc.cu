@@ -93,10 +93,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                 wrow = (tile - t0) * TILE_F;
                 sidx = s;
             };
+            const uint64_t wpol = l2_evict_first_policy();     // weights pass through once
             auto load_w = [&](int st, const CUtensorMap *mw, int wrow, int kt) {
                 const uint32_t base = smem_base + st * stage_bytes;
-                tma_load_2d(base, mw, full_bar(st), kt * TILE_K, wrow);
-                if (DUAL) tma_load_2d(base + a_bytes, &map_w1, full_bar(st), kt * TILE_K, wrow);
+                tma_load_2d_hint(base, mw, full_bar(st), kt * TILE_K, wrow, wpol);
+                if (DUAL) tma_load_2d_hint(base + a_bytes, &map_w1, full_bar(st), kt * TILE_K, wrow, wpol);
             };
             auto load_x = [&](int st, int kt) {
                 const uint32_t base = smem_base + st * stage_bytes + NACC * a_bytes;
