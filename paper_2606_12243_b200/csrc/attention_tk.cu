@@ -396,32 +396,25 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             ++wg_phase;
             return done;
         };
-        // The loop starts with a dry item: one tile and one result on whatever TMEM holds, no waits on the other
-        // roles, nothing stored.  A launch runs this code only a few times per CTA, and the first time through comes
-        // from a cold instruction cache (several microseconds); the dry item takes that hit before the kernel's
-        // predecessor has finished.
+        // (A dry first item, run on whatever TMEM holds before the dependency wait to warm the instruction cache, paid
+        // while the streamed weights pushed the kernels' code out of L2 between launches; with the weights marked
+        // evict-first the code stays in L2 and the dry item only delayed the first real one: removed.)
         ItemSrc src;
         src_init(a, src);
-        for (int n_item = -1; ok; ++n_item) {
-            const bool dry = n_item < 0;
+        for (int n_item = 0; ok; ++n_item) {
             Item it;
-            if (dry) {
-                it.be = it.b = it.g = it.stream = it.split = it.row_base = it.k_begin = 0;
-                it.n_ctx = it.k_end = TKEYS; it.n_tiles = 1; it.n_split = 1;
-            } else if (!next_item(a, per, src, it)) {
-                break;
-            }
+            if (!next_item(a, per, src, it)) break;
             if (n_item == 0) {
                 PDL_WAIT();
             }
-            if (!dry && it.b != anc_b) {
+            if (it.b != anc_b) {
                 // the ancestor sets of this sequence's draft tree (every sequence may have its own)
                 if (n_item > 0 && !(ok = wg_sync())) break;           // nobody reads the previous sequence's sets any more
                 if (et < a.M) anc_sh[et] = a.tree[it.b].anc[et];
                 if (!(ok = wg_sync())) break;                         // anc_sh is visible
                 anc_b = it.b;
             }
-            if (dry || it.be != q_be || it.g != q_g) {
+            if (it.be != q_be || it.g != q_g) {
                 // stage the query rows of this (sequence, kv head): rows 0..NR-1 the hi parts, NR..2NR-1 the lo parts,
                 // pre-scaled, in the K-major 128-byte-swizzled layout the MMA reads; loads first
                 for (int idx0 = et; idx0 < NR * (HD / 2); idx0 += 4 * ST) {
@@ -449,8 +442,8 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> the MMA's reads
                 __syncwarp();
-                if (lane == 0 && !dry) mbar_arrive(qfull_bar);
-                if (!dry) { q_be = it.be; q_g = it.g; }
+                if (lane == 0) mbar_arrive(qfull_bar);
+                q_be = it.be; q_g = it.g;
             }
             // Lane r of every warp keeps row r's running maximum (the four warps compute the same values); the other
             // lanes read it, as the exponent's reference, from the warp's copy in shared memory.
@@ -462,7 +455,7 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 
             for (int t = 0; t < it.n_tiles; ++t) {
                 const int sb = s_cnt & 1;
-                if (!dry && !(ok = mbar_wait(sfull_bar(sb), (s_cnt >> 1) & 1, &abort_sh, a.status))) break;
+                if (!(ok = mbar_wait(sfull_bar(sb), (s_cnt >> 1) & 1, &abort_sh, a.status))) break;
                 tc_fence_after();
                 float s[RG];
                 load_rows<NR, RG>(tlane + TM_S + sb * 64, row0, s);
@@ -509,7 +502,7 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     // together; O^T is rescaled once the previous tile's MMAs have written it.
 #pragma unroll
                     for (int r = 0; r < RG; ++r) l_run[r] *= corr_sh[sw][r];
-                    if (!dry) {
+                    {
                         if (!(ok = mbar_wait(pvdone_bar(sb ^ 1), ((s_cnt - 1) >> 1) & 1, &abort_sh, a.status))) break;
                         tc_fence_after();
 #pragma unroll
@@ -540,14 +533,14 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> the MMA's reads
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0 && !dry) mbar_arrive(pfull_bar(sb));     // S^T is read, P^T (and the rescaled O^T) are in place
-                if (!dry) ++s_cnt;
+                if (lane == 0) mbar_arrive(pfull_bar(sb));     // S^T is read, P^T (and the rescaled O^T) are in place
+                ++s_cnt;
             }
             if (!ok) break;
             // ---- the item's result ----
             if (quarter == 0 && lane < RG) mraw_sh[row0 + lane] = m_lane;
             // the last MMA into O^T of the item (and with it all earlier ones) is complete
-            if (!dry && it.n_tiles > 0 && !(ok = mbar_wait(pvdone_bar((s_cnt - 1) & 1), ((s_cnt - 1) >> 1) & 1, &abort_sh, a.status))) break;
+            if (it.n_tiles > 0 && !(ok = mbar_wait(pvdone_bar((s_cnt - 1) & 1), ((s_cnt - 1) >> 1) & 1, &abort_sh, a.status))) break;
             tc_fence_after();
             float o[RG];
             if (it.n_tiles > 0) {
@@ -565,7 +558,7 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 #pragma unroll
             for (int r = 0; r < RG; ++r) { osm[(row0 + r) * HD + kl] = o[r]; lsm[(row0 + r) * HD + kl] = l_run[r]; }
             if (!(ok = wg_sync())) break;
-            const int rows_out = dry ? 1 : QR;                          // the dry item runs the loop's code once, without the stores
+            const int rows_out = QR;
 #pragma unroll 1
             for (int r = sw; r < rows_out; r += SW) {
                 const float *lr = lsm + r * HD + lane;
@@ -578,25 +571,25 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     const __nv_bfloat162 l01 = __floats2bfloat162_rn(x0 - __low2float(h01), x1 - __high2float(h01));
                     const __nv_bfloat162 l23 = __floats2bfloat162_rn(x2 - __low2float(h23), x3 - __high2float(h23));
                     __nv_bfloat16 *dst = a.out + ((size_t)(it.be * a.M + node) * a.H + h) * HD + lane * 4;
-                    if (!dry) {
+                    {
                         *reinterpret_cast<uint2 *>(dst) = make_uint2(*reinterpret_cast<const uint32_t *>(&h01), *reinterpret_cast<const uint32_t *>(&h23));
                         if (a.out_plane)
                             *reinterpret_cast<uint2 *>(dst + a.out_plane) =
                                 make_uint2(*reinterpret_cast<const uint32_t *>(&l01), *reinterpret_cast<const uint32_t *>(&l23));
                     }
-                } else if (!dry) {
+                } else {
                     float *pdst = a.part + ((((size_t)it.be * a.H + h) * a.M + node) * a.part_slots + it.split) * ROWF;
                     *reinterpret_cast<float2 *>(pdst + lane * 4) = make_float2(v.x, v.y);       // rows are 8-byte aligned (HD + 2 floats)
                     *reinterpret_cast<float2 *>(pdst + lane * 4 + 2) = make_float2(v.z, v.w);
                     if (lane == 0) { pdst[HD] = mraw_sh[r] * 0.6931471805599453f; pdst[HD + 1] = l; }   // natural-log units
                 }
             }
-            if (!dry && it.n_tiles > 0) {
+            if (it.n_tiles > 0) {
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(ofree_bar);                 // the next item may overwrite O^T
             }
-            if (!dry && !single && a.fuse_merge) {
+            if (!single && a.fuse_merge) {
                 // last key range of this (sequence, kv head) to finish merges all of them, in range order
                 // (one acquire-release atomic after the barrier instead of a fence per thread on both sides)
                 if (!(ok = wg_sync())) break;
