@@ -569,8 +569,12 @@ int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {
     const CUtensorMap &w0 = *L.map_w[0], &w1 = *L.map_w[L.n_seg > 1 ? 1 : 0], &w2 = *L.map_w[L.n_seg > 2 ? 2 : 0];
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
-    // a second epilogue group above token tiles of 48 unless the caller says otherwise
-    const int groups = L.epi_groups == 1 || L.epi_groups == 2 ? L.epi_groups : (p.nt > 48 ? 2 : 1);
+    // a second epilogue group above token tiles of 48 unless the caller says otherwise; the gate/up launch already from
+    // 17 rows on: its split tiles have two or three contributors, so a finisher has two chunks of 8 rows of two
+    // accumulators to finish, and the groups take one each (8B, 27 rows: finishing 7.5 -> 5.7 us; with 9 rows, or for
+    // the other epilogues, whose finishers have one chunk each, the second group only costs)
+    const int groups = L.epi_groups == 1 || L.epi_groups == 2 ? L.epi_groups
+                       : (p.nt > 48 || (L.epi == EPI_SWIGLU && L.rows > 16) ? 2 : 1);
     pdl_config(cfg, attr, dim3(grid), dim3(64 + 128 * groups), smem, st);
     static bool attr_done[64][8];            // the attribute belongs to a (kernel, device) pair
     int dev = 0;
