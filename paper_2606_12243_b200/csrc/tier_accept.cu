@@ -90,7 +90,7 @@ __device__ float block_max(float x, float *sh) {
 struct TierCuts { int n; float log_tau[MAXJ]; };
 // grid (gate rows per sequence, B).  conf_source 0: gate row of node n = prow[n], rows = drafter logits
 // [B, R, V]; conf_source 1: gate row = parent[n] + 1, rows = slim logits [B, M, V].
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(1024)
 tier_kernel(unsigned char *__restrict__ tier, float *__restrict__ conf, DeviceStats *stats,
             const float *__restrict__ gate_logits, const int *__restrict__ draft_tok, const int *__restrict__ prow,
             const int *__restrict__ parent, int per_seq, int conf_source, int rows_per_seq, int N, int V, TierCuts cuts) {
@@ -137,7 +137,7 @@ constexpr int RS_STRIDE = VIASD_MAX_ROWS_PER_SEQ;
 struct RowStats { float *mx; int *arg; float *z; };       // each [B, KINDS, RS_STRIDE]
 struct RowPtrs { const float *p[KINDS]; };                // drafter logits, then each judge's
 
-__global__ void __launch_bounds__(512)
+__global__ void __launch_bounds__(1024)
 row_stats_kernel(RowStats rs, RowPtrs src, int R, int M, int V, float inv_temp, int want_z) {
     __shared__ float sh[32];
     __shared__ MaxIdx shm[32];
@@ -473,10 +473,34 @@ int launch_tier(const viasd_model *m, const viasd_draft *d, const viasd_params *
     TierCuts cuts;
     cuts.n = js.n;
     for (int k = 0; k < MAXJ; ++k) cuts.log_tau[k] = k < js.n ? js.log_tau[k] : 0.f;
-    tier_kernel<<<dim3(rows, d->batch), 256, 0, st>>>(r->tier, r->conf, m->ws.stats, gate, d->draft_tok, d->prow,
+    // (a CTA per gate row: with few rows the launch is bound by the loads each CTA has in flight, hence 1024 threads)
+    tier_kernel<<<dim3(rows, d->batch), 1024, 0, st>>>(r->tier, r->conf, m->ws.stats, gate, d->draft_tok, d->prow,
         d->parent, d->per_sequence, p->conf_source, rows, d->n_nodes, m->cfg.vocab, cuts);
     LAUNCH_CHECK();
     return VIASD_OK;
+}
+
+// A cluster of 16 CTAs (beyond the portable 8) where the device takes it: asked once per device.
+static bool accept_team16_ok() {
+    static int state[64];                    // 0 unknown, 1 yes, -1 no
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    if (state[dev] == 0) {
+        state[dev] = -1;
+        if (cudaFuncSetAttribute(accept_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+            cudaLaunchConfig_t cfg;
+            memset(&cfg, 0, sizeof(cfg));
+            cfg.gridDim = dim3(16); cfg.blockDim = dim3(ACC_THREADS);
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = 16; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr; cfg.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, accept_kernel, &cfg) == cudaSuccess && n >= 1) state[dev] = 1;
+        }
+        (void)cudaGetLastError();
+    }
+    return state[dev] == 1;
 }
 
 int launch_accept(const viasd_model *m, const viasd_draft *d, const viasd_params *p, const JudgeSet &js, viasd_result *r,
@@ -497,7 +521,7 @@ int launch_accept(const viasd_model *m, const viasd_draft *d, const viasd_params
         RowPtrs src;
         src.p[0] = p->mode == 1 ? d->drafter_logits : nullptr;
         for (int k = 1; k < KINDS; ++k) src.p[k] = k <= js.n ? js.logits[k - 1] : nullptr;
-        row_stats_kernel<<<dim3(rows, d->batch, js.n + 1), 512, 0, st>>>(a.rs, src, d->n_prows, M, m->cfg.vocab,
+        row_stats_kernel<<<dim3(rows, d->batch, js.n + 1), 1024, 0, st>>>(a.rs, src, d->n_prows, M, m->cfg.vocab,
                                                                          1.0f / p->temperature, p->mode == 1);
         LAUNCH_CHECK();
     }
@@ -525,6 +549,7 @@ int launch_accept(const viasd_model *m, const viasd_draft *d, const viasd_params
     a.len_full = probe ? probe->len_full : nullptr;
     // sampling over a large vocabulary: a cluster of CTAs per sequence shares every sweep of the vocabulary
     int team = (p->mode == 1 && m->cfg.vocab >= 16384) ? ACC_TEAM : 1;
+    if (team == ACC_TEAM && m->cfg.vocab >= 65536 && accept_team16_ok()) team = 16;     // every sweep of the vocabulary is shared
     { const int t = m->opt.accept_team; if (t == 1 || t == 2 || t == 4 || t == 8) team = t; }
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
