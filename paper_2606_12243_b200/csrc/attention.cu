@@ -219,7 +219,9 @@ static int mma_attention(viasd_model *m, const void *kc, const void *vc, bool sl
     const int subs = hpi ? grp / hpi : 1, QRi = hpi * M;       // keys-on-lanes: items per kv head, query rows per item
     // (with more than 32 query rows per kv head the mma.sync kernel has one key group per query tile and is bound by
     // its MMA issue: there the keys-on-lanes kernel wins from two tiles per SM on)
-    int use = kind == 3 ? (hpi && tiles_total * subs >= (subs > 1 ? 2LL : 8LL) * m->sm_count ? 2 : 0) : kind;
+    // (and with 17 - 32 query rows per kv head, two query tiles for the mma.sync kernel, from one tile per SM on: 32B
+    // shape at batch 1, 264 tiles, attention 1.78 -> 1.61 ms per step)
+    int use = kind == 3 ? (hpi && tiles_total * subs >= (subs > 1 ? 2LL : QRi > 16 ? 1LL : 8LL) * m->sm_count ? 2 : 0) : kind;
     if (use == 2 && !hpi) use = 0;
     const int reps = use == 1 ? attention_tc_replicas(QR) : 1;
     const int nsplit = mma_nsplit(m, batch, M, streams, use != 0, reps, use == 2 ? subs : 1, use == 2 ? QRi : 0);

@@ -601,37 +601,60 @@ attention_tk_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 }
                 if (!(ok = wg_sync())) break;
                 if (last_sh) {
-                    for (int r = sw; r < QR; r += SW) {
-                        const int hh = it.g * grp + r / a.M, i = r % a.M;
-                        const float *psrc = a.part + (((size_t)it.be * a.H + hh) * a.M + i) * (size_t)a.part_slots * ROWF;
-                        // lane s holds range s's (max, sum); the weights go round by shuffle (at most 32 ranges when fused)
-                        float ms = -INFINITY, ls = 0.f;
-                        if (lane < it.n_split) { ms = __ldcg(psrc + (size_t)lane * ROWF + HD); ls = __ldcg(psrc + (size_t)lane * ROWF + HD + 1); }
-                        float num[HD / 32];
+                    // Four rows per warp at a time, every load of a round (the ranges' maxima and sums, four ranges'
+                    // vectors) issued before the first use: a row at a time is a trip to L2 per row, one after the other.
+                    constexpr int MB = 4;
+#pragma unroll 1
+                    for (int rb = sw; rb < QR; rb += MB * SW) {
+                        const float *psrc[MB];
+                        size_t odst[MB];
+                        float ms[MB], ls[MB], w[MB], den[MB], num[MB][HD / 32];
 #pragma unroll
-                        for (int e = 0; e < HD / 32; ++e) num[e] = 0.f;
-                        const float mmax = warp_max(ms);
-                        const float w = (ms == -INFINITY) ? 0.f : expf(ms - mmax);
-                        const float den = warp_sum(ls * w);
-                        for (int s0 = 0; s0 < it.n_split; s0 += 4) {
-                            float v[4][HD / 32];
+                        for (int j = 0; j < MB; ++j) {
+                            const int r = min(rb + j * SW, QR - 1);               // rows past the end repeat the last one, unstored
+                            const int hh = it.g * grp + r / a.M, i = r % a.M;
+                            psrc[j] = a.part + (((size_t)it.be * a.H + hh) * a.M + i) * (size_t)a.part_slots * ROWF;
+                            odst[j] = ((size_t)(it.be * a.M + i) * a.H + hh) * HD;
+                            // lane s holds range s's (max, sum); the weights go round by shuffle (at most 32 ranges when fused)
+                            ms[j] = -INFINITY; ls[j] = 0.f;
+                            if (lane < it.n_split) { ms[j] = __ldcg(psrc[j] + (size_t)lane * ROWF + HD); ls[j] = __ldcg(psrc[j] + (size_t)lane * ROWF + HD + 1); }
 #pragma unroll
-                            for (int q = 0; q < 4; ++q)
-#pragma unroll
-                                for (int e = 0; e < HD / 32; ++e)
-                                    v[q][e] = s0 + q < it.n_split ? __ldcg(psrc + (size_t)(s0 + q) * ROWF + lane + 32 * e) : 0.f;
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                const float wq = __shfl_sync(0xffffffffu, w, (s0 + q) & 31);
-#pragma unroll
-                                for (int e = 0; e < HD / 32; ++e) num[e] = fmaf(v[q][e], s0 + q < it.n_split ? wq : 0.f, num[e]);
-                            }
+                            for (int e = 0; e < HD / 32; ++e) num[j][e] = 0.f;
                         }
-                        const float invd = 1.f / den;
+                        for (int s0 = 0; s0 < it.n_split; s0 += 4) {
+                            float v[MB][4][HD / 32];
 #pragma unroll
-                        for (int e = 0; e < HD / 32; ++e)
-                            store_act<__nv_bfloat16>(a.out, a.out_plane, ((size_t)(it.be * a.M + i) * a.H + hh) * HD + lane + 32 * e,
-                                                     num[e] * invd);
+                            for (int j = 0; j < MB; ++j)
+#pragma unroll
+                                for (int q = 0; q < 4; ++q)
+#pragma unroll
+                                    for (int e = 0; e < HD / 32; ++e)
+                                        v[j][q][e] = s0 + q < it.n_split ? __ldcg(psrc[j] + (size_t)(s0 + q) * ROWF + lane + 32 * e) : 0.f;
+                            if (s0 == 0) {
+#pragma unroll
+                                for (int j = 0; j < MB; ++j) {
+                                    const float mmax = warp_max(ms[j]);
+                                    w[j] = (ms[j] == -INFINITY) ? 0.f : expf(ms[j] - mmax);
+                                    den[j] = warp_sum(ls[j] * w[j]);
+                                }
+                            }
+#pragma unroll
+                            for (int j = 0; j < MB; ++j)
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    const float wq = __shfl_sync(0xffffffffu, w[j], (s0 + q) & 31);
+#pragma unroll
+                                    for (int e = 0; e < HD / 32; ++e) num[j][e] = fmaf(v[j][q][e], s0 + q < it.n_split ? wq : 0.f, num[j][e]);
+                                }
+                        }
+#pragma unroll
+                        for (int j = 0; j < MB; ++j) {
+                            if (rb + j * SW >= QR) continue;
+                            const float invd = 1.f / den[j];
+#pragma unroll
+                            for (int e = 0; e < HD / 32; ++e)
+                                store_act<__nv_bfloat16>(a.out, a.out_plane, odst[j] + lane + 32 * e, num[j][e] * invd);
+                        }
                     }
                 }
                 if (!(ok = wg_sync())) break;                          // last_sh and the staged rows are reused by the next item
