@@ -213,7 +213,9 @@ enum {
     VIASD_OPT_ATTENTION_SPLITS,        /* key ranges per (sequence, kv head), 1..16; 0 = cost model (default) */
     VIASD_OPT_ATTENTION_LO,            /* mma.sync kernel: hi/lo split of queries and probabilities 2 (default),
                                           queries only 1, neither 0 (fails the logit tolerance at full size) */
-    VIASD_OPT_ACCEPT_TEAM,             /* CTAs per sequence in the accept walk: 1, 2, 4, 8; 0 = by mode and vocabulary */
+    VIASD_OPT_ACCEPT_TEAM,             /* CTAs per sequence in the accept walk: 1, 2, 4, 8; 0 = by mode and vocabulary (1 for
+                                          greedy; sampling: 8 from 16384 tokens on, 16 from 65536 on where the device
+                                          takes clusters of 16) */
     VIASD_OPT_DUAL_MAX_ROWS,           /* most token rows (both verifiers together) that viasd_verify_step runs as one
                                           sweep over the layers, 0..128 (default 128); above it the passes run in turn */
     VIASD_OPT_TK_GRID,                 /* keys-on-lanes attention with tiles dealt evenly: CTAs to use; 0 = one per SM */
