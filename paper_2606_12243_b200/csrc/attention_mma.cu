@@ -473,37 +473,60 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             }
             __syncthreads();
             if (last_sh) {
-                for (int row = warp; row < QR; row += WARPS) {
-                    const int h = it.g * grp + row / a.M, i = row % a.M;
-                    const float *src = a.part + (((size_t)it.be * a.H + h) * a.M + i) * (size_t)a.nsplit * ROWF;
-                    // lane s holds range s's (max, sum); the weights go round by shuffle (nsplit <= 32 when fused)
-                    float ms = -INFINITY, ls = 0.f;
-                    if (lane < a.nsplit) { ms = __ldcg(src + (size_t)lane * ROWF + HD); ls = __ldcg(src + (size_t)lane * ROWF + HD + 1); }
-                    float num[HD / 32];
+                // two rows per warp at a time, all loads of a round in flight before the first use (a row at a time is a
+                // trip to L2 per row, one after the other; the kernel has no registers to spare for more)
+                constexpr int MB = 2;
+#pragma unroll 1
+                for (int rb = warp; rb < QR; rb += MB * WARPS) {
+                    const float *src[MB];
+                    size_t odst[MB];
+                    float ms[MB], ls[MB], w[MB], den[MB], num[MB][HD / 32];
 #pragma unroll
-                    for (int e = 0; e < HD / 32; ++e) num[e] = 0.f;
-                    const float mmax = warp_max(ms);
-                    const float w = (ms == -INFINITY) ? 0.f : expf(ms - mmax);
-                    const float den = warp_sum(ls * w);
-                    for (int s0 = 0; s0 < a.nsplit; s0 += 4) {
-                        float v[4][HD / 32];
+                    for (int j = 0; j < MB; ++j) {
+                        const int row = min(rb + j * WARPS, QR - 1);            // rows past the end repeat the last one, unstored
+                        const int h = it.g * grp + row / a.M, i = row % a.M;
+                        src[j] = a.part + (((size_t)it.be * a.H + h) * a.M + i) * (size_t)a.nsplit * ROWF;
+                        odst[j] = ((size_t)(it.be * a.M + i) * a.H + h) * HD;
+                        // lane s holds range s's (max, sum); the weights go round by shuffle (nsplit <= 32 when fused)
+                        ms[j] = -INFINITY; ls[j] = 0.f;
+                        if (lane < a.nsplit) { ms[j] = __ldcg(src[j] + (size_t)lane * ROWF + HD); ls[j] = __ldcg(src[j] + (size_t)lane * ROWF + HD + 1); }
 #pragma unroll
-                        for (int q = 0; q < 4; ++q)
-#pragma unroll
-                            for (int e = 0; e < HD / 32; ++e)
-                                v[q][e] = s0 + q < a.nsplit ? __ldcg(src + (size_t)(s0 + q) * ROWF + lane + 32 * e) : 0.f;
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const float wq = __shfl_sync(0xffffffffu, w, (s0 + q) & 31);
-#pragma unroll
-                            for (int e = 0; e < HD / 32; ++e) num[e] = fmaf(v[q][e], s0 + q < a.nsplit ? wq : 0.f, num[e]);
-                        }
+                        for (int e = 0; e < HD / 32; ++e) num[j][e] = 0.f;
                     }
-                    const float inv = 1.f / den;
+                    for (int s0 = 0; s0 < a.nsplit; s0 += 4) {
+                        float v[MB][4][HD / 32];
 #pragma unroll
-                    for (int e = 0; e < HD / 32; ++e)
-                        store_act<__nv_bfloat16>(a.out, a.out_plane, ((size_t)(it.be * a.M + i) * a.H + h) * HD + lane + 32 * e,
-                                                 num[e] * inv);
+                        for (int j = 0; j < MB; ++j)
+#pragma unroll
+                            for (int q = 0; q < 4; ++q)
+#pragma unroll
+                                for (int e = 0; e < HD / 32; ++e)
+                                    v[j][q][e] = s0 + q < a.nsplit ? __ldcg(src[j] + (size_t)(s0 + q) * ROWF + lane + 32 * e) : 0.f;
+                        if (s0 == 0) {
+#pragma unroll
+                            for (int j = 0; j < MB; ++j) {
+                                const float mmax = warp_max(ms[j]);
+                                w[j] = (ms[j] == -INFINITY) ? 0.f : expf(ms[j] - mmax);
+                                den[j] = warp_sum(ls[j] * w[j]);
+                            }
+                        }
+#pragma unroll
+                        for (int j = 0; j < MB; ++j)
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const float wq = __shfl_sync(0xffffffffu, w[j], (s0 + q) & 31);
+#pragma unroll
+                                for (int e = 0; e < HD / 32; ++e) num[j][e] = fmaf(v[j][q][e], s0 + q < a.nsplit ? wq : 0.f, num[j][e]);
+                            }
+                    }
+#pragma unroll
+                    for (int j = 0; j < MB; ++j) {
+                        if (rb + j * WARPS >= QR) continue;
+                        const float inv = 1.f / den[j];
+#pragma unroll
+                        for (int e = 0; e < HD / 32; ++e)
+                            store_act<__nv_bfloat16>(a.out, a.out_plane, odst[j] + lane + 32 * e, num[j][e] * inv);
+                    }
                 }
             }
             __syncthreads();
