@@ -38,7 +38,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
     __shared__ int abort_sh;
     __shared__ float inv_sh[128];                       // per-row 1/rms of the input (fused RMSNorm)
     __shared__ float xch[GROUPS * CH * TILE_F];         // rotary partner exchange, one buffer per epilogue group
-    __shared__ int4 rowmeta[128];                       // per token row: rotary position, cache slot, sequence
+    __shared__ int4 rowmeta[128];                       // per token row: rotary position, cache slot, offset in its cache
 
     constexpr bool DUAL = EPI == EPI_SWIGLU;
     RUN_FLAG_EXIT(p.run_flag);
@@ -429,7 +429,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                         const int n_ctx = p.len_eff[b];
                         // replay pass: rows that fall on slots the cache already holds are recomputed but not stored
                         const int slot = (p.kv_keep && n_ctx + i < p.kv_keep[b]) ? -1 : n_ctx + i;
-                        rowmeta[et] = make_int4(n_ctx + p.depth[(size_t)b * p.tree_stride + i], slot, b, stream);
+                        // the row's place in its cache, without the head (element offset, 64 bits in .z / .w, the stream in
+                        // bit 30 of .w): worked out once here, not per row and tile in the epilogue
+                        const int lo = stream ? p.layer_ord2 : p.layer_ord;
+                        const unsigned long long off = slot < 0 ? 0ull
+                            : (((unsigned long long)lo * p.max_batch + b) * p.rope_Hkv * p.max_ctx + slot) * TILE_F;
+                        rowmeta[et] = make_int4(n_ctx + p.depth[(size_t)b * p.tree_stride + i], slot, (int)(unsigned)(off & 0xffffffffull),
+                                                (int)((unsigned)(off >> 32) | ((unsigned)stream << 30)));
                     }
                 }
                 asm volatile("bar.sync 1, %0;" ::"n"(epi_threads) : "memory");

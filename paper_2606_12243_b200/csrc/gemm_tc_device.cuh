@@ -156,14 +156,14 @@ __device__ __forceinline__ void finish_chunk(const TcParams &p, int tile, int f,
 #pragma unroll
             for (int j = 0; j < CH; ++j) if (j < nrow) dst[(size_t)j * p.rope_H * TILE_F] = g[j];
         } else {
+            __nv_bfloat16 *c0 = s == 1 ? p.kc : p.vc, *c1 = s == 1 ? p.kc2 : p.vc2;
+            const size_t head_off = (size_t)head * p.max_ctx * TILE_F + f;
 #pragma unroll
             for (int j = 0; j < CH; ++j) {
-                const int4 rm = rowmeta[min(r0 + j, 127)];
+                const int4 rm = rowmeta[min(r0 + j, 127)];          // .z / .w: the row's offset in its cache (set with the table)
                 if (j < nrow && rm.y >= 0) {
-                    __nv_bfloat16 *cache = rm.w ? (s == 1 ? p.kc2 : p.vc2) : (s == 1 ? p.kc : p.vc);
-                    const int lo = rm.w ? p.layer_ord2 : p.layer_ord;
-                    cache[((((size_t)lo * p.max_batch + rm.z) * p.rope_Hkv + head) * p.max_ctx + rm.y) * TILE_F + f] =
-                        __float2bfloat16_rn(g[j]);
+                    const size_t off = ((size_t)((unsigned)rm.w & 0x3fffffffu) << 32) | (unsigned)rm.z;
+                    (((unsigned)rm.w >> 30) & 1u ? c1 : c0)[off + head_off] = __float2bfloat16_rn(g[j]);
                 }
             }
         }
