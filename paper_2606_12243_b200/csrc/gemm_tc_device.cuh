@@ -134,12 +134,20 @@ __device__ __forceinline__ void finish_chunk(const TcParams &p, int tile, int f,
         const int head = tile - t0, pidx = f & 63;
         if (s < 2) {
             float c[CH], sn[CH];
+            if (aux) {                                           // the rows' tables are staged in shared memory
 #pragma unroll
-            for (int j = 0; j < CH; ++j) {
-                const int pos = rowmeta[min(r0 + j, 127)].x;
-                const float *ar = aux + min(r0 + j, p.rows - 1) * TILE_F + pidx;
-                c[j] = aux ? ar[0] : p.cosv[(size_t)pos * 64 + pidx];
-                sn[j] = aux ? ar[64] : p.sinv[(size_t)pos * 64 + pidx];
+                for (int j = 0; j < CH; ++j) {
+                    const float *ar = aux + min(r0 + j, p.rows - 1) * TILE_F + pidx;
+                    c[j] = ar[0];
+                    sn[j] = ar[64];
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < CH; ++j) {
+                    const int pos = rowmeta[min(r0 + j, 127)].x;
+                    c[j] = p.cosv[(size_t)pos * 64 + pidx];
+                    sn[j] = p.sinv[(size_t)pos * 64 + pidx];
+                }
             }
 #pragma unroll
             for (int j = 0; j < CH; ++j) {
