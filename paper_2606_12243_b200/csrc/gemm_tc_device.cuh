@@ -105,9 +105,13 @@ __device__ __forceinline__ void finish_chunk(const TcParams &p, int tile, int f,
         __nv_bfloat16 *ap = p.next_act + (size_t)(p.row0 + r0) * p.ld_out + n;
         if (touch) { want(hp); want(ap); want(ap + p.next_plane); want(p.ssq_out + ((size_t)tile * 4 + (f >> 5)) * p.ssq_stride + p.row0 + r0); }
         float v[CH];
+        if (aux) {                                               // the residual rows are staged in shared memory
 #pragma unroll
-        for (int j = 0; j < CH; ++j)
-            v[j] = (valid && j < nrow) ? (aux ? aux[(r0 + j) * TILE_F + f] : __ldcg(hp + (size_t)j * p.ld_out)) + g[j] : 0.f;
+            for (int j = 0; j < CH; ++j) v[j] = (valid && j < nrow) ? aux[(r0 + j) * TILE_F + f] + g[j] : 0.f;
+        } else {
+#pragma unroll
+            for (int j = 0; j < CH; ++j) v[j] = (valid && j < nrow) ? __ldcg(hp + (size_t)j * p.ld_out) + g[j] : 0.f;
+        }
 #pragma unroll
         for (int j = 0; j < CH; ++j) {
             if (valid && j < nrow) {
