@@ -220,18 +220,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                     float *slot = p.scratch + ((size_t)blockIdx.x * 2 + (seg_i == 0 ? 0 : 1)) * slot_floats;
                     for (int c = group * CH; c < p.rows; c += n_groups * CH) {   // padding rows beyond p.rows are never read
                         float g[CH], uu[CH];
-                        tc_ld8(t0 + c, g);
-                        if (DUAL) tc_ld8(t0 + NB + c, uu);
                         if (p.has_lo) {                          // add the product with the lo plane
                             float lo[CH];
-                            tc_ld8(t0 + NT + c, lo);
+                            tc_ld8x2(t0 + c, t0 + NT + c, g, lo);
 #pragma unroll
                             for (int j = 0; j < CH; ++j) g[j] += lo[j];
                             if (DUAL) {
-                                tc_ld8(t0 + NB + NT + c, lo);
+                                tc_ld8x2(t0 + NB + c, t0 + NB + NT + c, uu, lo);
 #pragma unroll
                                 for (int j = 0; j < CH; ++j) uu[j] += lo[j];
                             }
+                        } else {
+                            tc_ld8(t0 + c, g);
+                            if (DUAL) tc_ld8(t0 + NB + c, uu);
                         }
 #pragma unroll
                         for (int j = 0; j < CH; ++j) {
