@@ -148,11 +148,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                     const uint32_t base = smem_base + st * stage_bytes;
                     // the hi tile is followed by the lo tile: together one K-major operand of NB rows
                     const uint32_t bh = base + NACC * a_bytes;
+                    // one descriptor per operand and stage; a k-step of 16 columns is 32 bytes further on, 2 in the
+                    // descriptor's address field (the MMA-issuing thread is a single instruction stream that has about
+                    // the arrival time of a stage to get through all this: every instruction here counts)
+                    const uint64_t da = smem_desc(base), db = smem_desc(bh), da2 = DUAL ? smem_desc(base + a_bytes) : 0ull;
 #pragma unroll
                     for (int k = 0; k < TILE_K / 16; ++k) {
                         const uint32_t acc = (kt > sg.ka || k > 0) ? 1u : 0u;
-                        tc_mma(d0, smem_desc(base + k * 32), smem_desc(bh + k * 32), idesc, acc);
-                        if (DUAL) tc_mma(d0 + NB, smem_desc(base + a_bytes + k * 32), smem_desc(bh + k * 32), idesc, acc);
+                        tc_mma(d0, da + 2 * k, db + 2 * k, idesc, acc);
+                        if (DUAL) tc_mma(d0 + NB, da2 + 2 * k, db + 2 * k, idesc, acc);
                     }
                     tc_commit(empty_bar(st));              // the stage is free once these MMAs have read it
                 }
