@@ -47,8 +47,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int NT = p.nt, S = p.stages;
     constexpr int NACC = DUAL ? 2 : 1;
+    // A stage holds KB boxes of 64 k-columns of every operand: two for the single-matrix launches (32 KB of weights per
+    // stage, as the gate/up launch has with its two matrices).  With 16 KB per stage the bookkeeping of a stage - a
+    // barrier wait, a fence and a commit in the MMA thread, a wait and the copies' issue in the TMA thread - took
+    // longer than the stage's weights take to arrive: those launches streamed at 5.9 TB/s, not 6.5.
+    constexpr int KB = (DUAL || GROUPS > 1) ? 1 : 2;     // (wide token tiles: two boxes per stage would leave two stages)
     const uint32_t a_bytes = TILE_F * TILE_K * 2, b_bytes = (uint32_t)NT * TILE_K * 2;
-    const uint32_t stage_bytes = NACC * a_bytes + 2 * b_bytes;
+    const uint32_t box_bytes = NACC * a_bytes + 2 * b_bytes;          // one k-box of every operand
+    const uint32_t stage_bytes = KB * box_bytes;
     auto full_bar = [&](int s) { return smem_u32(&bars[s]); };
     auto empty_bar = [&](int s) { return smem_u32(&bars[MAX_STAGES + s]); };
     auto tfull_bar = [&](int b) { return smem_u32(&bars[2 * MAX_STAGES + b]); };
@@ -82,10 +88,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            const int n_it = u_end - u_begin;
+            const int n_it = (u_end - u_begin) / KB;          // stages: ranges and tiles are whole numbers of KB boxes
             // unit -> weight matrix, its first row, k-block
             auto unit = [&](int it, const CUtensorMap *&mw, int &wrow, int &kt, int &sidx) {
-                const int u = u_begin + it, tile = u / p.k_tiles;
+                const int u = u_begin + it * KB, tile = u / p.k_tiles;
                 kt = u - tile * p.k_tiles;
                 int s = 0, t0 = 0;
                 if (!DUAL) while (s < 2 && tile >= p.seg_tile_end[s]) { t0 = p.seg_tile_end[s]; ++s; }
@@ -96,13 +102,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
             const uint64_t wpol = l2_evict_first_policy();     // weights pass through once
             auto load_w = [&](int st, const CUtensorMap *mw, int wrow, int kt) {
                 const uint32_t base = smem_base + st * stage_bytes;
-                tma_load_2d_hint(base, mw, full_bar(st), kt * TILE_K, wrow, wpol);
+#pragma unroll
+                for (int kb = 0; kb < KB; ++kb)
+                    tma_load_2d_hint(base + kb * box_bytes, mw, full_bar(st), (kt + kb) * TILE_K, wrow, wpol);
                 if (DUAL) tma_load_2d_hint(base + a_bytes, &map_w1, full_bar(st), kt * TILE_K, wrow, wpol);
             };
             auto load_x = [&](int st, int kt) {
                 const uint32_t base = smem_base + st * stage_bytes + NACC * a_bytes;
-                tma_load_2d(base, &map_x, full_bar(st), kt * TILE_K, p.row0);
-                tma_load_2d(base + b_bytes, &map_x, full_bar(st), kt * TILE_K, p.row0 + p.lo_row_offset);
+#pragma unroll
+                for (int kb = 0; kb < KB; ++kb) {
+                    tma_load_2d(base + kb * box_bytes, &map_x, full_bar(st), (kt + kb) * TILE_K, p.row0);
+                    tma_load_2d(base + kb * box_bytes + b_bytes, &map_x, full_bar(st), (kt + kb) * TILE_K, p.row0 + p.lo_row_offset);
+                }
             };
             const CUtensorMap *mw; int wrow, kt, sidx;
             // Weights do not depend on the kernel before this one: fill the ring with them first, and only then
@@ -111,20 +122,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
             for (int it = 0; it < pre; ++it) {
                 unit(it, mw, wrow, kt, sidx);
                 asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(full_bar(it)),
-                             "r"(DUAL ? 2 * p.a_tx[0] : p.a_tx[sidx]) : "memory");
+                             "r"(DUAL ? 2 * p.a_tx[0] : KB * p.a_tx[sidx]) : "memory");
                 load_w(it, mw, wrow, kt);
             }
             asm volatile("griddepcontrol.wait;" ::: "memory");
             for (int it = 0; it < pre; ++it) {
                 unit(it, mw, wrow, kt, sidx);
-                mbar_expect_tx(full_bar(it), 2 * p.b_tx);
+                mbar_expect_tx(full_bar(it), KB * 2 * p.b_tx);
                 load_x(it, kt);
             }
             for (int it = pre; it < n_it; ++it) {
                 const int st = it % S;
                 if (!mbar_wait(empty_bar(st), ((it / S) & 1) ^ 1, &abort_sh, p.status)) break;
                 unit(it, mw, wrow, kt, sidx);
-                mbar_expect_tx(full_bar(st), (DUAL ? 2 * p.a_tx[0] : p.a_tx[sidx]) + 2 * p.b_tx);
+                mbar_expect_tx(full_bar(st), (DUAL ? 2 * p.a_tx[0] : KB * p.a_tx[sidx]) + KB * 2 * p.b_tx);
                 load_w(st, mw, wrow, kt);
                 load_x(st, kt);
             }
@@ -141,7 +152,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                 if (!(ok = mbar_wait(tempty_bar(buf), ((acc_it / p.acc_bufs) & 1) ^ 1, &abort_sh, p.status))) break;
                 tc_fence_after();
                 const uint32_t d0 = tmem_base + buf * acc_cols;
-                for (int kt = sg.ka; kt < sg.kb; ++kt, ++it) {
+                for (int kt = sg.ka; kt < sg.kb; kt += KB, ++it) {
                     const int st = it % S;
                     if (!(ok = mbar_wait(full_bar(st), (it / S) & 1, &abort_sh, p.status))) break;
                     tc_fence_after();
@@ -151,12 +162,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
                     // one descriptor per operand and stage; a k-step of 16 columns is 32 bytes further on, 2 in the
                     // descriptor's address field (the MMA-issuing thread is a single instruction stream that has about
                     // the arrival time of a stage to get through all this: every instruction here counts)
-                    const uint64_t da = smem_desc(base), db = smem_desc(bh), da2 = DUAL ? smem_desc(base + a_bytes) : 0ull;
+                    const uint64_t da2 = DUAL ? smem_desc(base + a_bytes) : 0ull;
 #pragma unroll
-                    for (int k = 0; k < TILE_K / 16; ++k) {
-                        const uint32_t acc = (kt > sg.ka || k > 0) ? 1u : 0u;
-                        tc_mma(d0, da + 2 * k, db + 2 * k, idesc, acc);
-                        if (DUAL) tc_mma(d0 + NB, da2 + 2 * k, db + 2 * k, idesc, acc);
+                    for (int kb = 0; kb < KB; ++kb) {
+                        const uint64_t da = smem_desc(base + kb * box_bytes), db = smem_desc(bh + kb * box_bytes);
+#pragma unroll
+                        for (int k = 0; k < TILE_K / 16; ++k) {
+                            const uint32_t acc = (kt > sg.ka || kb > 0 || k > 0) ? 1u : 0u;
+                            tc_mma(d0, da + 2 * k, db + 2 * k, idesc, acc);
+                            if (DUAL) tc_mma(d0 + NB, da2 + 2 * k, db + 2 * k, idesc, acc);
+                        }
                     }
                     tc_commit(empty_bar(st));              // the stage is free once these MMAs have read it
                 }
@@ -511,6 +526,16 @@ size_t tc_scratch_floats(int sm_count, int nt, bool dual) { return (size_t)sm_co
 
 int tc_tiles(int n) { return (n + TILE_F - 1) / TILE_F; }
 
+// Groups of four epilogue warps: a second one above token tiles of 48 unless the caller says otherwise; the gate/up
+// launch already from 17 rows on: its split tiles have two or three contributors, so a finisher has two chunks of 8 rows
+// of two accumulators to finish, and the groups take one each (8B, 27 rows: finishing 7.5 -> 5.7 us; with 9 rows, or for
+// the other epilogues, whose finishers have one chunk each, the second group only costs)
+static int tc_groups(const TcLaunch &L) {
+    return L.epi_groups == 1 || L.epi_groups == 2 ? L.epi_groups : (L.nt > 48 || (L.epi == EPI_SWIGLU && L.rows > 16) ? 2 : 1);
+}
+// k-boxes of 64 columns per ring stage and scheduling unit (as the kernel instance has it)
+static int tc_boxes(const TcLaunch &L) { return L.epi == EPI_SWIGLU || tc_groups(L) > 1 ? 1 : 2; }
+
 // TcLaunch (host description) -> TcParams (kernel argument block), schedule fields left to the caller
 void tc_fill_params(const TcLaunch &L, TcParams &p) {
     memset(&p, 0, sizeof(p));
@@ -518,7 +543,9 @@ void tc_fill_params(const TcLaunch &L, TcParams &p) {
     p.nt = L.nt;
     p.rows = L.rows;
     p.row0 = L.row0;
-    p.k_tiles = (L.k + TILE_K - 1) / TILE_K;
+    // k-boxes of 64 columns; an even number per tile for the single-matrix launches, whose narrow-tile instance takes
+    // two boxes per stage (the columns past k read as zeros), so that both instances cut k at the same places
+    p.k_tiles = dual ? (L.k + TILE_K - 1) / TILE_K : 2 * ((L.k + 2 * TILE_K - 1) / (2 * TILE_K));
     int tiles = 0;
     for (int s = 0; s < 3; ++s) {
         p.seg_n[s] = s < L.n_seg ? L.seg_n[s] : 0;
@@ -560,9 +587,10 @@ int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {
     int ctas_per_sm = 1;
     int grid = L.sm_count * ctas_per_sm < units ? L.sm_count * ctas_per_sm : units;
     p.units_per_cta = (units + grid - 1) / grid;
+    if (!dual) p.units_per_cta += p.units_per_cta & 1;        // whole stages of two boxes
     grid = (units + p.units_per_cta - 1) / p.units_per_cta;
     const int nacc = dual ? 2 : 1;
-    const size_t stage = (size_t)nacc * TILE_F * TILE_K * 2 + 2 * (size_t)L.nt * TILE_K * 2;
+    const size_t stage = tc_boxes(L) * ((size_t)nacc * TILE_F * TILE_K * 2 + 2 * (size_t)L.nt * TILE_K * 2);
     // The depth of the ring bounds the streaming rate (bytes in flight per SM): 200 KB, one CTA per SM, measured
     // faster than 100 KB with the next kernel's CTA resident beside this one.
     const int ring_kb = L.ring_kb > 0 ? L.ring_kb : 200;
@@ -580,12 +608,7 @@ int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {
     const CUtensorMap &w0 = *L.map_w[0], &w1 = *L.map_w[L.n_seg > 1 ? 1 : 0], &w2 = *L.map_w[L.n_seg > 2 ? 2 : 0];
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
-    // a second epilogue group above token tiles of 48 unless the caller says otherwise; the gate/up launch already from
-    // 17 rows on: its split tiles have two or three contributors, so a finisher has two chunks of 8 rows of two
-    // accumulators to finish, and the groups take one each (8B, 27 rows: finishing 7.5 -> 5.7 us; with 9 rows, or for
-    // the other epilogues, whose finishers have one chunk each, the second group only costs)
-    const int groups = L.epi_groups == 1 || L.epi_groups == 2 ? L.epi_groups
-                       : (p.nt > 48 || (L.epi == EPI_SWIGLU && L.rows > 16) ? 2 : 1);
+    const int groups = tc_groups(L);
     pdl_config(cfg, attr, dim3(grid), dim3(64 + 128 * groups), smem, st);
     static bool attr_done[64][8];            // the attribute belongs to a (kernel, device) pair
     int dev = 0;
