@@ -28,7 +28,7 @@
 
 namespace {
 
-template <int EPI, int GROUPS>
+template <int EPI, int GROUPS, int KBT>
 __global__ void __launch_bounds__(64 + 128 * GROUPS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
                const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_x, const TcParams p) {
@@ -51,7 +51,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant
     // stage, as the gate/up launch has with its two matrices).  With 16 KB per stage the bookkeeping of a stage - a
     // barrier wait, a fence and a commit in the MMA thread, a wait and the copies' issue in the TMA thread - took
     // longer than the stage's weights take to arrive: those launches streamed at 5.9 TB/s, not 6.5.
-    constexpr int KB = (DUAL || GROUPS > 1) ? 1 : 2;     // (wide token tiles: two boxes per stage would leave two stages)
+    constexpr int KB = DUAL ? 1 : KBT;                    // (the launch picks one box at wide token tiles: two would leave two stages)
     const uint32_t a_bytes = TILE_F * TILE_K * 2, b_bytes = (uint32_t)NT * TILE_K * 2;
     const uint32_t box_bytes = NACC * a_bytes + 2 * b_bytes;          // one k-box of every operand
     const uint32_t stage_bytes = KB * box_bytes;
@@ -534,7 +534,7 @@ static int tc_groups(const TcLaunch &L) {
     return L.epi_groups == 1 || L.epi_groups == 2 ? L.epi_groups : (L.nt > 48 || (L.epi == EPI_SWIGLU && L.rows > 16) ? 2 : 1);
 }
 // k-boxes of 64 columns per ring stage and scheduling unit (as the kernel instance has it)
-static int tc_boxes(const TcLaunch &L) { return L.epi == EPI_SWIGLU || tc_groups(L) > 1 ? 1 : 2; }
+static int tc_boxes(const TcLaunch &L) { return L.epi == EPI_SWIGLU || L.nt > 64 ? 1 : 2; }
 
 // TcLaunch (host description) -> TcParams (kernel argument block), schedule fields left to the caller
 void tc_fill_params(const TcLaunch &L, TcParams &p) {
@@ -610,19 +610,21 @@ int launch_gemm_tc(const TcLaunch &L, cudaStream_t st) {
     cudaLaunchAttribute attr[1];
     const int groups = tc_groups(L);
     pdl_config(cfg, attr, dim3(grid), dim3(64 + 128 * groups), smem, st);
-    static bool attr_done[64][8];            // the attribute belongs to a (kernel, device) pair
+    static bool attr_done[64][16];           // the attribute belongs to a (kernel, device) pair
+    const int boxes = tc_boxes(L);
     int dev = 0;
     CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return VIASD_EUNSUPPORTED;
-#define TC_LAUNCH_G(IDX, KIND, G)                                                                                     \
+#define TC_LAUNCH_G(IDX, KIND, G, KBX)                                                                                     \
     do {                                                                                                              \
         if (!attr_done[dev][IDX]) {                                                                                   \
-            CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<KIND, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, 208 * 1024)); \
+            CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<KIND, G, KBX>, cudaFuncAttributeMaxDynamicSharedMemorySize, 208 * 1024)); \
             attr_done[dev][IDX] = true;                                                                               \
         }                                                                                                             \
-        CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<KIND, G>, w0, w1, w2, *L.map_x, p));                         \
+        CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<KIND, G, KBX>, w0, w1, w2, *L.map_x, p));                    \
     } while (0)
-#define TC_LAUNCH(IDX, KIND) do { if (groups == 2) TC_LAUNCH_G(IDX + 4, KIND, 2); else TC_LAUNCH_G(IDX, KIND, 1); } while (0)
+#define TC_LAUNCH(IDX, KIND) do { if (boxes == 2) { if (groups == 2) TC_LAUNCH_G(IDX + 12, KIND, 2, 2); else TC_LAUNCH_G(IDX + 8, KIND, 1, 2); } \
+                                   else { if (groups == 2) TC_LAUNCH_G(IDX + 4, KIND, 2, 1); else TC_LAUNCH_G(IDX, KIND, 1, 1); } } while (0)
     switch (L.epi) {
     case EPI_SWIGLU: TC_LAUNCH(0, EPI_SWIGLU); break;
     case EPI_ADD_NORM: TC_LAUNCH(1, EPI_ADD_NORM); break;
