@@ -533,8 +533,9 @@ int tc_tiles(int n) { return (n + TILE_F - 1) / TILE_F; }
 static int tc_groups(const TcLaunch &L) {
     return L.epi_groups == 1 || L.epi_groups == 2 ? L.epi_groups : (L.nt > 48 || (L.epi == EPI_SWIGLU && L.rows > 16) ? 2 : 1);
 }
-// k-boxes of 64 columns per ring stage and scheduling unit (as the kernel instance has it)
-static int tc_boxes(const TcLaunch &L) { return L.epi == EPI_SWIGLU || L.nt > 64 ? 1 : 2; }
+// k-boxes of 64 columns per ring stage (the kernel's KBT): two for the single-matrix launches up to token tiles of 96
+// (32B batch 16, 96 rows: step 27.9 -> 27.1 ms with two stages of 80 KB; at 112 rows, two stages of 88 KB, no gain)
+static int tc_boxes(const TcLaunch &L) { return L.epi == EPI_SWIGLU || L.nt > 96 ? 1 : 2; }
 
 // TcLaunch (host description) -> TcParams (kernel argument block), schedule fields left to the caller
 void tc_fill_params(const TcLaunch &L, TcParams &p) {
